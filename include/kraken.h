@@ -1,0 +1,226 @@
+/*
+ * kraken.h - C ABI of the single-GPU Kraken prefill / decode library (sm_100a).
+ *
+ * A Kraken model (Prabhakar et al., "Kraken: Inherently Parallel Transformers For
+ * Efficient Multi-Device Inference") has L layers of N independent sub-layers
+ * ("branches").  Algorithm 1 defines one sub-layer:
+ *     res = x;  y = AllReduce(x);  x = LN(x);  x = res + MHA(x);
+ *     res = x;  x = LN(x + y);     out = res + FFN(x)
+ * with the AllReduce an element-wise sum over the N sub-layer inputs (identity in the
+ * first layer), one shared token+position embedding, and a final linear map W_concat
+ * over the concatenated N outputs before the tied unembedding (Sec. 3.1).  This library
+ * runs all N branches on ONE device: the branches are the group dimension of grouped
+ * GEMMs and the AllReduce is a sum inside the down-projection's epilogue.
+ *
+ * Conventions for every call
+ *   - "device" pointers are CUDA device memory of the current device; "host" pointers
+ *     are ordinary (preferably pinned) host memory.  The library never allocates device
+ *     memory: weights, KV cache, scratch, tokens and logits are caller-owned.
+ *   - bf16 tensors are raw 16-bit patterns, row-major, innermost dimension contiguous.
+ *   - Calls only enqueue work on the given stream (a cudaStream_t passed as void*; NULL
+ *     is the legacy default stream) unless stated otherwise.
+ *   - Every call returns 0 or a negative kraken_status.  Nothing aborts, throws across
+ *     the boundary or traps on the device.
+ */
+#ifndef KRAKEN_H_
+#define KRAKEN_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum kraken_status {
+    KRAKEN_OK = 0,
+    KRAKEN_EINVAL = -1,       /* null / non-positive / inconsistent argument                  */
+    KRAKEN_EUNSUPPORTED = -2, /* shape outside what the kernels support (see kraken_create)   */
+    KRAKEN_ECAPACITY = -3,    /* batch, sequence or buffer larger than the handle was sized for */
+    KRAKEN_ESTATE = -4,       /* call order violated (decode before prefill, batch changed)   */
+    KRAKEN_ECUDA = -5         /* a CUDA runtime / driver call failed                          */
+} kraken_status;
+
+/* Model hyper-parameters and capacity (the analogue of an inference engine's build-time maxima). */
+typedef struct kraken_config {
+    int32_t n_branch;  /* N: sub-layers per layer, the paper's degree of parallelism (Sec. 3.1) */
+    int32_t n_layer;   /* L                                                                   */
+    int32_t d_model;   /* d: width of ONE sub-layer                                           */
+    int32_t n_head;    /* attention heads per sub-layer (Table 3 caption); head_dim = d / n_head */
+    int32_t d_ff;      /* FFN hidden width (4d standard, 2d for parameter parity; Sec. 3.2)   */
+    int32_t vocab;     /* V                                                                   */
+    int32_t max_pos;   /* rows of the position table = KV capacity per sequence               */
+    int32_t max_batch; /* sequences per call                                                  */
+    float ln_eps;      /* LayerNorm epsilon (1e-5)                                            */
+    int32_t gelu_tanh; /* 0: GELU by erf (default), 1: tanh approximation                     */
+    int32_t final_ln;  /* 1: LayerNorm between W_concat and the unembedding (default), 0: none */
+    int32_t reserved[5];
+} kraken_config;
+
+/* Device pointers to bf16 weights, row-major [out_features, in_features]; BORROWED until
+ * kraken_destroy.  Any bias or LayerNorm-beta pointer may be NULL (= zeros).
+ * w_qkv rows 0..d-1 produce Q, d..2d-1 K, 2d..3d-1 V; head h owns rows h*hd..(h+1)*hd-1 of each.
+ * w_concat input index n*d + j is feature j of branch n (branch-major concatenation). */
+typedef struct kraken_weights {
+    const void *wte;                /* [V, d] token embedding, also the unembedding (tied) */
+    const void *wpe;                /* [max_pos, d] learned positions                     */
+    const void *ln1_g, *ln1_b;      /* [L][N][d]                                          */
+    const void *w_qkv, *b_qkv;      /* [L][N][3d][d], [L][N][3d]                          */
+    const void *w_proj, *b_proj;    /* [L][N][d][d],  [L][N][d]                           */
+    const void *ln2_g, *ln2_b;      /* [L][N][d]                                          */
+    const void *w_up, *b_up;        /* [L][N][F][d],  [L][N][F]                           */
+    const void *w_down, *b_down;    /* [L][N][d][F],  [L][N][d]                           */
+    const void *w_concat, *b_concat;/* [d][N*d], [d]                                      */
+    const void *lnf_g, *lnf_b;      /* [d]; ignored when final_ln == 0                    */
+} kraken_weights;
+
+typedef struct kraken_handle kraken_handle;
+
+/* Bytes of KV cache and scratch a handle of this configuration needs.  Pure host
+ * arithmetic, usable without a GPU.  KV layout: [L][N][2 (K,V)][max_batch][n_head][max_pos][head_dim] bf16.
+ * Errors: EINVAL (null, non-positive field, d % n_head != 0), EUNSUPPORTED (see kraken_create). */
+int kraken_query_sizes(const kraken_config *cfg, size_t *kv_bytes, size_t *scratch_bytes);
+
+/* Build a handle: validates the configuration, records the borrowed weight pointers and
+ * the caller's KV and scratch buffers (device, 256-byte aligned, at least the queried
+ * sizes), encodes the TMA descriptors of the weights.  Host work only.
+ * Supported shapes: head_dim in {64, 128}; d_model and d_ff multiples of 64.
+ * Errors: EINVAL, EUNSUPPORTED, ECAPACITY (undersized buffers), ECUDA. */
+int kraken_create(const kraken_config *cfg, const kraken_weights *weights, void *d_kv, size_t kv_bytes,
+                  void *d_scratch, size_t scratch_bytes, kraken_handle **out);
+
+/* Prefill (Sec. 2.1: the step that produces the first token and the KV cache).
+ * d_tokens: device int32 [batch, seqlen] row-major, all sequences the same length;
+ * d_logits: device fp32 [batch, V], logits of the LAST position of each sequence.
+ * Fills the KV cache rows 0..seqlen-1 of sequences 0..batch-1 and sets the handle's
+ * length to seqlen.  Token ids outside [0, V) are read as 0 and raise status bit 0.
+ * Errors: EINVAL, ECAPACITY (batch > max_batch, seqlen > max_pos), ECUDA. */
+int kraken_prefill(kraken_handle *h, const int32_t *d_tokens, int32_t batch, int32_t seqlen,
+                   float *d_logits, void *stream);
+
+/* Same with HOST buffers: copies the tokens to the device, runs the prefill, copies the
+ * logits back and synchronises the stream before returning.  h_tokens [batch, seqlen],
+ * h_logits [batch, V]. */
+int kraken_prefill_host(kraken_handle *h, const int32_t *h_tokens, int32_t batch, int32_t seqlen,
+                        float *h_logits, void *stream);
+
+/* Prefill that returns the logits of EVERY position: d_logits device fp32 [batch, seqlen, V].
+ * Same cache side effects as kraken_prefill.  Meant for tests and evaluation. */
+int kraken_prefill_all_logits(kraken_handle *h, const int32_t *d_tokens, int32_t batch, int32_t seqlen,
+                              float *d_logits, void *stream);
+
+/* Logits of chosen token rows of the most recent prefill (its last-layer outputs stay in
+ * scratch until the next call that runs the model).  h_rows: HOST int32 [n_rows], row = b*seqlen + t;
+ * d_logits: device fp32 [n_rows, V].  Errors: EINVAL, ESTATE (no prefill yet), ECAPACITY (n_rows
+ * larger than max_batch * max_pos). */
+int kraken_logits_rows(kraken_handle *h, const int32_t *h_rows, int32_t n_rows, float *d_logits, void *stream);
+
+/* One decode step (Sec. 2.1): one new token per sequence at position cur_len, attending to
+ * cache rows 0..cur_len (the new one included); appends K,V; cur_len += 1.
+ * d_tokens device int32 [batch]; d_logits device fp32 [batch, V].
+ * Errors: ESTATE (no prefill, or batch differs from the prefill's), ECAPACITY (cur_len == max_pos). */
+int kraken_decode_step(kraken_handle *h, const int32_t *d_tokens, int32_t batch, float *d_logits, void *stream);
+
+/* Where the cache of (layer, branch, which: 0 = K, 1 = V) lives: base device pointer and
+ * strides in ELEMENTS for (batch, head, position, dim). */
+int kraken_kv_view(kraken_handle *h, int32_t layer, int32_t branch, int32_t which, const void **ptr,
+                   int64_t strides[4]);
+
+/* Synchronises the stream of the last call and reports the device status word:
+ * bit 0 = a token id was out of range, bit 1 = a bounded wait inside a kernel gave up. */
+int kraken_device_status(kraken_handle *h, uint32_t *flags);
+
+/* Current sequence length held in the cache (0 before any prefill). */
+int kraken_cur_len(kraken_handle *h, int32_t *cur_len);
+
+/* Launch accounting and per-kernel timing.  Every call that runs the model counts its kernel
+ * launches per category; with profiling enabled each launch is also bracketed by CUDA events on
+ * the call's stream.  kraken_profile_read synchronises that stream, returns the accumulated
+ * device milliseconds (0 when profiling was off) and launch counts since the last read, and
+ * resets them.  ms, launches: HOST arrays of KRAKEN_PROF_COUNT entries. */
+typedef enum kraken_prof_category {
+    KRAKEN_PROF_EMBED = 0,
+    KRAKEN_PROF_LAYERNORM = 1,
+    KRAKEN_PROF_GEMM_QKV = 2,
+    KRAKEN_PROF_ATTENTION = 3,
+    KRAKEN_PROF_GEMM_PROJ = 4,
+    KRAKEN_PROF_GEMM_UP = 5,
+    KRAKEN_PROF_GEMM_DOWN = 6,
+    KRAKEN_PROF_TAIL = 7,      /* row gather, W_concat, final LayerNorm, unembedding */
+    KRAKEN_PROF_COUNT = 8
+} kraken_prof_category;
+int kraken_profile_enable(kraken_handle *h, int32_t on);
+int kraken_profile_read(kraken_handle *h, double *ms, int64_t *launches);
+
+/* Forget the cached sequences (cur_len = 0, status word cleared). */
+int kraken_reset(kraken_handle *h);
+void kraken_destroy(kraken_handle *h);
+const char *kraken_strerror(int status);
+
+/* ------------------------------------------------------------------------------------------
+ * Single steps of the path, exposed so that each kernel can be checked on its own.  All
+ * pointers are device pointers.  G is the number of groups (branches); a group stride of 0
+ * shares one tensor between all groups.
+ * ------------------------------------------------------------------------------------------ */
+
+/* Shared embedding (Sec. 3.1): out[t, :] = wte[id[t], :] + wpe[pos0 + t % seqlen, :], fp32 [T, d].
+ * d_status: device uint32, bit 0 is set when an id is outside [0, vocab) (that id reads row 0). */
+int kraken_op_embed(const int32_t *d_ids, int32_t n_tokens, int32_t seqlen, int32_t pos0, const void *wte,
+                    const void *wpe, int32_t d_model, int32_t vocab, float *d_out, uint32_t *d_status,
+                    void *stream);
+
+/* LayerNorm of Algorithm 1, both placements: out_g = LN(a_g + y; gamma_g, beta_g) -> bf16 [G][rows, d].
+ * a: fp32 [G][rows, d] with group stride a_gstride elements (0 = shared); y: fp32 [rows, d] or NULL;
+ * gamma/beta bf16 [G][d] (beta may be NULL). */
+int kraken_op_layernorm(const float *d_a, int64_t a_gstride, const float *d_y, const void *gamma,
+                        const void *beta, int32_t groups, int32_t rows, int32_t d_model, float eps,
+                        void *d_out_bf16, void *stream);
+
+/* Epilogues of the grouped GEMM  C_g = A_g . W_g^T (+ bias_g) ; A bf16 [G][M, K], W bf16 [G][Nout, K]. */
+typedef enum kraken_epilogue {
+    KRAKEN_EPI_F32 = 0,       /* out_f32[g] = acc + bias                                              */
+    KRAKEN_EPI_BF16 = 1,      /* out_bf16[g] = bf16(acc + bias)                                       */
+    KRAKEN_EPI_GELU_BF16 = 2, /* out_bf16[g] = bf16(GELU(acc + bias))             (FFN up-projection)  */
+    KRAKEN_EPI_RESID_F32 = 3, /* out_f32[g] = resid[g] + acc + bias               (x = res + MHA(x))   */
+    KRAKEN_EPI_RESID_SUM = 4, /* out_f32[g] = resid[g] + acc + bias; sum = SUM_g out_f32[g]
+                                 (out = res + FFN(x), then the AllReduce of Algorithm 1)              */
+    KRAKEN_EPI_QKV = 5        /* cols [0,d): out_bf16[g] (queries); [d,2d), [2d,3d): K, V rows written
+                                 into the cache at [b][head][pos0 + t][dim], b = row / seqlen         */
+} kraken_epilogue;
+
+typedef struct kraken_gemm_args {
+    const void *a;       int64_t a_gstride;    int32_t lda;   /* bf16 [G][M, K], row stride lda elements     */
+    const void *w;       int64_t w_gstride;    int32_t ldw;   /* bf16 [G][Nout, K]                            */
+    const void *bias;    int64_t bias_gstride;                /* bf16 [G][Nout] or NULL                       */
+    int32_t groups, m, n_out, k;
+    int32_t epilogue;                                         /* kraken_epilogue                              */
+    float *out_f32;      int64_t out_f32_gstride;  int32_t ld_out_f32;
+    void *out_bf16;      int64_t out_bf16_gstride; int32_t ld_out_bf16;
+    const float *resid;  int64_t resid_gstride;    int32_t ld_resid; /* may alias out_f32 element for element  */
+    float *sum;          int32_t ld_sum;                      /* fp32 [M, Nout], RESID_SUM only               */
+    void *k_cache, *v_cache; int64_t cache_gstride;           /* QKV only: bases of this layer's K and V      */
+    int32_t seqlen, pos0, n_head, head_dim, max_pos;          /* QKV only                                     */
+    int32_t gelu_tanh;
+    int32_t n_tile;                                           /* N tile: 0 = automatic, else 64, 128 or 256    */
+    int32_t reserved[2];
+} kraken_gemm_args;
+
+/* Grouped bf16 GEMM on the tensor cores (tcgen05 + TMEM accumulators, TMA operand loads).
+ * Requirements: a, w 16-byte aligned; lda, ldw multiples of 8; k >= 8.  d_status as above (bit 1).
+ * Errors: EINVAL, EUNSUPPORTED, ECUDA. */
+int kraken_op_grouped_gemm(const kraken_gemm_args *args, uint32_t *d_status, void *stream);
+
+/* Causal multi-head attention over a prefix held in the cache layout (Sec. 2.1):
+ * for sequence b, head h, query row t (position pos0 + t): softmax over keys 0..pos0+t of
+ * q.k / sqrt(head_dim), times V.  q, out: bf16 [G][batch*seqlen, n_head*head_dim];
+ * k_cache, v_cache: bf16 [G][.][batch_stride][n_head][max_pos][head_dim] as described by
+ * cache_gstride / cache_bstride (elements). */
+int kraken_op_attention(const void *q, int64_t q_gstride, const void *k_cache, const void *v_cache,
+                        int64_t cache_gstride, int64_t cache_bstride, int32_t groups, int32_t batch,
+                        int32_t seqlen, int32_t pos0, int32_t n_head, int32_t head_dim, int32_t max_pos,
+                        void *out, int64_t out_gstride, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* KRAKEN_H_ */

@@ -1,0 +1,292 @@
+"""Python binding of libkraken.so: argument marshalling only.
+
+Every step of the Kraken prefill / decode path runs inside the CUDA library; this module
+turns torch tensors (used purely as device-memory owners) into the pointers and sizes of the
+C ABI declared in include/kraken.h.  There is no fallback: without the built library every
+call raises.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Dict, Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libkraken.so")
+
+OK, EINVAL, EUNSUPPORTED, ECAPACITY, ESTATE, ECUDA = 0, -1, -2, -3, -4, -5
+EPI_F32, EPI_BF16, EPI_GELU_BF16, EPI_RESID_F32, EPI_RESID_SUM, EPI_QKV = range(6)
+
+WEIGHT_FIELDS = (
+    "wte", "wpe", "ln1_g", "ln1_b", "w_qkv", "b_qkv", "w_proj", "b_proj",
+    "ln2_g", "ln2_b", "w_up", "b_up", "w_down", "b_down",
+    "w_concat", "b_concat", "lnf_g", "lnf_b",
+)
+
+PROF_CATEGORIES = ("embed", "layernorm", "gemm_qkv", "attention", "gemm_proj", "gemm_up", "gemm_down", "tail")
+PROF_COUNT = len(PROF_CATEGORIES)
+
+EXPORTS = (
+    "kraken_query_sizes", "kraken_create", "kraken_prefill", "kraken_prefill_host",
+    "kraken_prefill_all_logits", "kraken_logits_rows", "kraken_decode_step", "kraken_kv_view",
+    "kraken_device_status", "kraken_cur_len", "kraken_profile_enable", "kraken_profile_read", "kraken_reset", "kraken_destroy", "kraken_strerror",
+    "kraken_op_embed", "kraken_op_layernorm", "kraken_op_grouped_gemm", "kraken_op_attention",
+)
+
+
+class KrakenConfig(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in
+                ("n_branch", "n_layer", "d_model", "n_head", "d_ff", "vocab", "max_pos", "max_batch")] + [
+        ("ln_eps", C.c_float), ("gelu_tanh", C.c_int32), ("final_ln", C.c_int32), ("reserved", C.c_int32 * 5)]
+
+
+class KrakenWeights(C.Structure):
+    _fields_ = [(n, C.c_void_p) for n in WEIGHT_FIELDS]
+
+
+class GemmArgs(C.Structure):
+    _fields_ = [
+        ("a", C.c_void_p), ("a_gstride", C.c_int64), ("lda", C.c_int32),
+        ("w", C.c_void_p), ("w_gstride", C.c_int64), ("ldw", C.c_int32),
+        ("bias", C.c_void_p), ("bias_gstride", C.c_int64),
+        ("groups", C.c_int32), ("m", C.c_int32), ("n_out", C.c_int32), ("k", C.c_int32),
+        ("epilogue", C.c_int32),
+        ("out_f32", C.c_void_p), ("out_f32_gstride", C.c_int64), ("ld_out_f32", C.c_int32),
+        ("out_bf16", C.c_void_p), ("out_bf16_gstride", C.c_int64), ("ld_out_bf16", C.c_int32),
+        ("resid", C.c_void_p), ("resid_gstride", C.c_int64), ("ld_resid", C.c_int32),
+        ("sum", C.c_void_p), ("ld_sum", C.c_int32),
+        ("k_cache", C.c_void_p), ("v_cache", C.c_void_p), ("cache_gstride", C.c_int64),
+        ("seqlen", C.c_int32), ("pos0", C.c_int32), ("n_head", C.c_int32), ("head_dim", C.c_int32),
+        ("max_pos", C.c_int32), ("gelu_tanh", C.c_int32), ("n_tile", C.c_int32), ("reserved", C.c_int32 * 2),
+    ]
+
+
+class KrakenError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        self.status = status
+        super().__init__(f"{what}: {strerror(status)} ({status})")
+
+
+_lib = None
+
+
+def lib() -> C.CDLL:
+    """Loads libkraken.so; raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2408_07802_b200.build` "
+                "(there is no CPU or PyTorch fallback)")
+        L = C.CDLL(LIB_PATH)
+        vp, i32, i64 = C.c_void_p, C.c_int32, C.c_int64
+        L.kraken_query_sizes.argtypes = [C.POINTER(KrakenConfig), C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]
+        L.kraken_create.argtypes = [C.POINTER(KrakenConfig), C.POINTER(KrakenWeights), vp, C.c_size_t, vp,
+                                    C.c_size_t, C.POINTER(vp)]
+        L.kraken_prefill.argtypes = [vp, vp, i32, i32, vp, vp]
+        L.kraken_prefill_host.argtypes = [vp, vp, i32, i32, vp, vp]
+        L.kraken_prefill_all_logits.argtypes = [vp, vp, i32, i32, vp, vp]
+        L.kraken_logits_rows.argtypes = [vp, vp, i32, vp, vp]
+        L.kraken_decode_step.argtypes = [vp, vp, i32, vp, vp]
+        L.kraken_kv_view.argtypes = [vp, i32, i32, i32, C.POINTER(vp), C.POINTER(i64 * 4)]
+        L.kraken_device_status.argtypes = [vp, C.POINTER(C.c_uint32)]
+        L.kraken_cur_len.argtypes = [vp, C.POINTER(i32)]
+        L.kraken_profile_enable.argtypes = [vp, i32]
+        L.kraken_profile_read.argtypes = [vp, C.POINTER(C.c_double * PROF_COUNT), C.POINTER(i64 * PROF_COUNT)]
+        L.kraken_reset.argtypes = [vp]
+        L.kraken_destroy.argtypes = [vp]
+        L.kraken_destroy.restype = None
+        L.kraken_strerror.argtypes = [C.c_int]
+        L.kraken_strerror.restype = C.c_char_p
+        L.kraken_op_embed.argtypes = [vp, i32, i32, i32, vp, vp, i32, i32, vp, vp, vp]
+        L.kraken_op_layernorm.argtypes = [vp, i64, vp, vp, vp, i32, i32, i32, C.c_float, vp, vp]
+        L.kraken_op_grouped_gemm.argtypes = [C.POINTER(GemmArgs), vp, vp]
+        L.kraken_op_attention.argtypes = [vp, i64, vp, vp, i64, i64, i32, i32, i32, i32, i32, i32, i32, vp, i64, vp]
+        _lib = L
+    return _lib
+
+
+def strerror(status: int) -> str:
+    return lib().kraken_strerror(int(status)).decode()
+
+
+def _check(status: int, what: str):
+    if status != OK:
+        raise KrakenError(status, what)
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else t.data_ptr()
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def make_config(shape, max_batch: Optional[int] = None, max_pos: Optional[int] = None, **over) -> KrakenConfig:
+    """kraken_config from any object with the hyper-parameter attributes (e.g. kraken_inputs.KrakenShape)."""
+    cfg = KrakenConfig(
+        n_branch=shape.n_branch, n_layer=shape.n_layer, d_model=shape.d_model, n_head=shape.n_head,
+        d_ff=shape.d_ff, vocab=shape.vocab, max_pos=max_pos or shape.max_pos,
+        max_batch=max_batch or shape.batch, ln_eps=shape.ln_eps, gelu_tanh=shape.gelu_tanh,
+        final_ln=shape.final_ln)
+    for k, v in over.items():
+        setattr(cfg, k, v)
+    return cfg
+
+
+def query_sizes(cfg: KrakenConfig):
+    kv, sc = C.c_size_t(0), C.c_size_t(0)
+    _check(lib().kraken_query_sizes(C.byref(cfg), C.byref(kv), C.byref(sc)), "kraken_query_sizes")
+    return kv.value, sc.value
+
+
+class KrakenModel:
+    """Owns the device buffers (through torch) and a kraken_handle."""
+
+    def __init__(self, cfg: KrakenConfig, weights: Dict[str, Optional[torch.Tensor]], device="cuda:0"):
+        self.cfg = cfg
+        self.device = torch.device(device)
+        for k in WEIGHT_FIELDS:
+            t = weights.get(k)
+            if t is not None:
+                assert t.dtype == torch.bfloat16 and t.is_contiguous() and t.device == self.device, k
+        self.weights = dict(weights)
+        kv_bytes, scratch_bytes = query_sizes(cfg)
+        self.kv = torch.empty(kv_bytes, dtype=torch.uint8, device=self.device)
+        self.scratch = torch.empty(scratch_bytes, dtype=torch.uint8, device=self.device)
+        w = KrakenWeights(**{k: _ptr(weights.get(k)) for k in WEIGHT_FIELDS})
+        h = C.c_void_p()
+        with torch.cuda.device(self.device):
+            _check(lib().kraken_create(C.byref(cfg), C.byref(w), self.kv.data_ptr(), kv_bytes,
+                                       self.scratch.data_ptr(), scratch_bytes, C.byref(h)), "kraken_create")
+        self._h = h
+
+    def close(self):
+        if getattr(self, "_h", None):
+            lib().kraken_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        self.close()
+
+    # -------- the three calls of the path
+    def prefill(self, tokens: torch.Tensor, logits: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """tokens: device int32 [batch, seqlen] -> fp32 [batch, V] logits of the last position."""
+        b, l = tokens.shape
+        assert tokens.dtype == torch.int32 and tokens.is_contiguous() and tokens.device == self.device
+        if logits is None:
+            logits = torch.empty(b, self.cfg.vocab, dtype=torch.float32, device=self.device)
+        _check(lib().kraken_prefill(self._h, tokens.data_ptr(), b, l, logits.data_ptr(), _stream()), "kraken_prefill")
+        return logits
+
+    def prefill_host(self, tokens: torch.Tensor, logits: torch.Tensor) -> torch.Tensor:
+        """tokens / logits: HOST tensors (pinned for full-rate copies); blocks until the logits are there."""
+        b, l = tokens.shape
+        assert tokens.dtype == torch.int32 and tokens.device.type == "cpu" and logits.device.type == "cpu"
+        _check(lib().kraken_prefill_host(self._h, tokens.data_ptr(), b, l, logits.data_ptr(), _stream()),
+               "kraken_prefill_host")
+        return logits
+
+    def prefill_all_logits(self, tokens: torch.Tensor) -> torch.Tensor:
+        b, l = tokens.shape
+        assert tokens.dtype == torch.int32 and tokens.is_contiguous() and tokens.device == self.device
+        logits = torch.empty(b, l, self.cfg.vocab, dtype=torch.float32, device=self.device)
+        _check(lib().kraken_prefill_all_logits(self._h, tokens.data_ptr(), b, l, logits.data_ptr(), _stream()),
+               "kraken_prefill_all_logits")
+        return logits
+
+    def logits_rows(self, rows) -> torch.Tensor:
+        rows_t = torch.as_tensor(rows, dtype=torch.int32).contiguous()
+        out = torch.empty(rows_t.numel(), self.cfg.vocab, dtype=torch.float32, device=self.device)
+        _check(lib().kraken_logits_rows(self._h, rows_t.data_ptr(), rows_t.numel(), out.data_ptr(), _stream()),
+               "kraken_logits_rows")
+        torch.cuda.current_stream().synchronize()  # rows_t (host) must outlive the copy
+        return out
+
+    def decode_step(self, tokens: torch.Tensor, logits: Optional[torch.Tensor] = None) -> torch.Tensor:
+        assert tokens.dtype == torch.int32 and tokens.is_contiguous() and tokens.device == self.device
+        b = tokens.numel()
+        if logits is None:
+            logits = torch.empty(b, self.cfg.vocab, dtype=torch.float32, device=self.device)
+        _check(lib().kraken_decode_step(self._h, tokens.data_ptr(), b, logits.data_ptr(), _stream()),
+               "kraken_decode_step")
+        return logits
+
+    # -------- inspection
+    def kv_view(self, layer: int, branch: int, which: int) -> torch.Tensor:
+        """bf16 view [max_batch, n_head, max_pos, head_dim] of the K (0) or V (1) cache of (layer, branch)."""
+        p = C.c_void_p()
+        st = (C.c_int64 * 4)()
+        _check(lib().kraken_kv_view(self._h, layer, branch, which, C.byref(p), C.byref(st)), "kraken_kv_view")
+        c = self.cfg
+        hd = c.d_model // c.n_head
+        off = (p.value - self.kv.data_ptr()) // 2
+        flat = self.kv.view(torch.bfloat16)
+        return flat.as_strided((c.max_batch, c.n_head, c.max_pos, hd), tuple(st), off)
+
+    def device_status(self) -> int:
+        f = C.c_uint32(0)
+        _check(lib().kraken_device_status(self._h, C.byref(f)), "kraken_device_status")
+        return f.value
+
+    @property
+    def cur_len(self) -> int:
+        v = C.c_int32(0)
+        _check(lib().kraken_cur_len(self._h, C.byref(v)), "kraken_cur_len")
+        return v.value
+
+    def profile_enable(self, on: bool):
+        _check(lib().kraken_profile_enable(self._h, int(on)), "kraken_profile_enable")
+
+    def profile_read(self):
+        """({category: device ms}, {category: launches}) since the last read; synchronises."""
+        ms = (C.c_double * PROF_COUNT)()
+        n = (C.c_int64 * PROF_COUNT)()
+        _check(lib().kraken_profile_read(self._h, C.byref(ms), C.byref(n)), "kraken_profile_read")
+        return dict(zip(PROF_CATEGORIES, list(ms))), dict(zip(PROF_CATEGORIES, list(n)))
+
+    def reset(self):
+        _check(lib().kraken_reset(self._h), "kraken_reset")
+
+
+# ------------------------------------------------------------------ single steps
+
+def op_embed(ids: torch.Tensor, seqlen: int, pos0: int, wte: torch.Tensor, wpe: torch.Tensor,
+             status: Optional[torch.Tensor] = None) -> torch.Tensor:
+    n = ids.numel()
+    d = wte.shape[1]
+    out = torch.empty(n, d, dtype=torch.float32, device=ids.device)
+    _check(lib().kraken_op_embed(ids.data_ptr(), n, seqlen, pos0, wte.data_ptr(), wpe.data_ptr(), d, wte.shape[0],
+                                 out.data_ptr(), _ptr(status), _stream()), "kraken_op_embed")
+    return out
+
+
+def op_layernorm(a: torch.Tensor, y: Optional[torch.Tensor], gamma: torch.Tensor, beta: Optional[torch.Tensor],
+                 eps: float = 1e-5, shared_a: bool = False) -> torch.Tensor:
+    """a fp32 [G, rows, d] (or [rows, d] with shared_a, used by every group); gamma [G, d]."""
+    G, d = gamma.shape
+    rows = a.shape[-2]
+    out = torch.empty(G, rows, d, dtype=torch.bfloat16, device=a.device)
+    _check(lib().kraken_op_layernorm(a.data_ptr(), 0 if shared_a else rows * d, _ptr(y), gamma.data_ptr(),
+                                     _ptr(beta), G, rows, d, eps, out.data_ptr(), _stream()), "kraken_op_layernorm")
+    return out
+
+
+def op_grouped_gemm(args: GemmArgs, status: Optional[torch.Tensor] = None):
+    _check(lib().kraken_op_grouped_gemm(C.byref(args), _ptr(status), _stream()), "kraken_op_grouped_gemm")
+
+
+def op_attention(q: torch.Tensor, k_cache: torch.Tensor, v_cache: torch.Tensor, batch: int, seqlen: int, pos0: int,
+                 n_head: int) -> torch.Tensor:
+    """q bf16 [G, batch*seqlen, d]; k_cache / v_cache bf16 [G, batch, n_head, max_pos, head_dim]."""
+    G, _, d = q.shape
+    _, _, H, P, hd = k_cache.shape
+    assert H == n_head and H * hd == d
+    out = torch.empty_like(q)
+    _check(lib().kraken_op_attention(q.data_ptr(), q.stride(0), k_cache.data_ptr(), v_cache.data_ptr(),
+                                     k_cache.stride(0), k_cache.stride(1), G, batch, seqlen, pos0, H, hd, P,
+                                     out.data_ptr(), out.stride(0), _stream()), "kraken_op_attention")
+    return out

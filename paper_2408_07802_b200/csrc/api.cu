@@ -1,0 +1,596 @@
+// The C ABI: configuration checks, handle, and the kernel sequence of prefill / decode.
+//
+// kraken_prefill enqueues, on the caller's stream, with no host synchronisation:
+//   embed -> for every layer { LN1[N] -> GEMM qkv[N] (K,V scattered into the cache) -> attention[N,B,H]
+//            -> GEMM proj[N] (+bias +residual) -> LN2[N] on (a_n + y) -> GEMM up[N] (+bias, GELU)
+//            -> GEMM down[N] (+bias +residual, cross-branch sum -> y of the next layer) }
+//   -> gather of the wanted rows -> GEMM W_concat -> final LN -> GEMM unembedding -> fp32 logits.
+#include <string.h>
+
+#include <new>
+#include <vector>
+
+#include "internal.h"
+#include "ptx.cuh"
+
+using namespace kr;
+
+namespace {
+
+constexpr size_t ALIGN = 256;
+size_t align_up(size_t v) { return (v + ALIGN - 1) / ALIGN * ALIGN; }
+
+struct Layout {
+    size_t status, tokens, rows, logits, x0, x, a, s, u, q, o, g, total;
+};
+
+int check_config(const kraken_config *c) {
+    if (!c) return KRAKEN_EINVAL;
+    if (c->n_branch < 1 || c->n_layer < 1 || c->d_model < 1 || c->n_head < 1 || c->d_ff < 1 || c->vocab < 1 ||
+        c->max_pos < 1 || c->max_batch < 1 || !(c->ln_eps > 0.f))
+        return KRAKEN_EINVAL;
+    if (c->d_model % c->n_head != 0) return KRAKEN_EINVAL;
+    const int hd = c->d_model / c->n_head;
+    if (hd != 64 && hd != 128) return KRAKEN_EUNSUPPORTED;
+    if (c->d_model % 64 != 0 || c->d_ff % 64 != 0) return KRAKEN_EUNSUPPORTED;
+    return KRAKEN_OK;
+}
+
+size_t kv_bytes_of(const kraken_config *c) {
+    return (size_t)c->n_layer * c->n_branch * 2 * c->max_batch * c->max_pos * (size_t)c->d_model * 2;
+}
+
+Layout layout_of(const kraken_config *c) {
+    const size_t T = (size_t)c->max_batch * c->max_pos, d = c->d_model, N = c->n_branch, F = c->d_ff;
+    Layout l;
+    size_t off = 0;
+    auto take = [&](size_t bytes) {
+        size_t o = off;
+        off += align_up(bytes);
+        return o;
+    };
+    l.status = take(256);
+    l.tokens = take(T * 4);
+    l.rows = take(T * 4);
+    l.logits = take((size_t)c->max_batch * c->vocab * 4);
+    l.x0 = take(T * d * 4);
+    l.x = take(N * T * d * 4);
+    l.a = take(N * T * d * 4);
+    l.s = take(T * d * 4);
+    l.u = take(N * T * d * 2);
+    l.q = take(N * T * d * 2);
+    l.o = take(N * T * d * 2);
+    l.g = take(N * T * F * 2);
+    l.total = off;
+    return l;
+}
+
+enum GemmKind { G_QKV = 0, G_PROJ, G_UP, G_DOWN, G_CONCAT, G_HEAD, G_COUNT };
+
+}  // namespace
+
+struct kraken_handle {
+    kraken_config cfg;
+    kraken_weights w;
+    uint8_t *kv;
+    uint8_t *scratch;
+    Layout lay;
+    int cur_len, batch, last_seqlen, last_rows;  // last_rows: token rows of the last model run
+    cudaStream_t last_stream;
+    bool naive;
+    // weight tensor maps, one per GEMM kind, re-encoded when the N tile changes
+    CUtensorMap tmB[G_COUNT];
+    int tmB_bn[G_COUNT];
+    // activation tensor maps, re-encoded when the token count changes
+    CUtensorMap tmA[G_COUNT];
+    int tmA_rows[G_COUNT];
+    // launch accounting and optional per-kernel timing
+    long long launches[KRAKEN_PROF_COUNT];
+    bool prof_on;
+    std::vector<cudaEvent_t> ev_pool;
+    size_t ev_used;
+    struct Span { int cat; size_t e0, e1; };
+    std::vector<Span> spans;
+};
+
+namespace {
+
+template <typename T>
+T *at(kraken_handle *h, size_t off) {
+    return reinterpret_cast<T *>(h->scratch + off);
+}
+
+cudaEvent_t prof_event(kraken_handle *h) {
+    if (h->ev_used == h->ev_pool.size()) {
+        cudaEvent_t e;
+        if (cudaEventCreate(&e) != cudaSuccess) return nullptr;
+        h->ev_pool.push_back(e);
+    }
+    return h->ev_pool[h->ev_used++];
+}
+
+// Counts a kernel launch of category `cat`; with profiling on, brackets it with events.
+struct LaunchScope {
+    kraken_handle *h;
+    cudaStream_t st;
+    bool timed;
+    LaunchScope(kraken_handle *h_, int cat, cudaStream_t st_) : h(h_), st(st_), timed(false) {
+        h->launches[cat]++;
+        if (h->prof_on) {
+            cudaEvent_t e0 = prof_event(h), e1 = prof_event(h);
+            if (e0 && e1) {
+                cudaEventRecord(e0, st);
+                h->spans.push_back({cat, h->ev_used - 2, h->ev_used - 1});
+                timed = true;
+            }
+        }
+    }
+    ~LaunchScope() {
+        if (timed) cudaEventRecord(h->ev_pool[h->spans.back().e1], st);
+    }
+};
+
+struct RunCtx {
+    kraken_handle *h;
+    cudaStream_t st;
+    int batch, seqlen, pos0, T;
+};
+
+// One grouped GEMM of the model: weights of `kind` at `layer`.
+int model_gemm(const RunCtx &rc, GemmKind kind, int layer, int m_rows, const uint16_t *a, long long a_gstride,
+               EpiParams epi) {
+    kraken_handle *h = rc.h;
+    const kraken_config &c = h->cfg;
+    const int d = c.d_model, F = c.d_ff, N = c.n_branch;
+    GemmOperands op;
+    GemmShape s;
+    int total_groups;  // groups held by the weight tensor across all layers
+    const uint16_t *wbase;
+    const uint16_t *bias = nullptr;
+    switch (kind) {
+        case G_QKV: s = {N, m_rows, 3 * d, d}; wbase = (const uint16_t *)h->w.w_qkv; bias = (const uint16_t *)h->w.b_qkv; break;
+        case G_PROJ: s = {N, m_rows, d, d}; wbase = (const uint16_t *)h->w.w_proj; bias = (const uint16_t *)h->w.b_proj; break;
+        case G_UP: s = {N, m_rows, F, d}; wbase = (const uint16_t *)h->w.w_up; bias = (const uint16_t *)h->w.b_up; break;
+        case G_DOWN: s = {N, m_rows, d, F}; wbase = (const uint16_t *)h->w.w_down; bias = (const uint16_t *)h->w.b_down; break;
+        case G_CONCAT: s = {1, m_rows, d, N * d}; wbase = (const uint16_t *)h->w.w_concat; bias = (const uint16_t *)h->w.b_concat; break;
+        default: s = {1, m_rows, c.vocab, d}; wbase = (const uint16_t *)h->w.wte; break;
+    }
+    const bool layered = kind <= G_DOWN;
+    total_groups = layered ? c.n_layer * N : 1;
+    const long long w_gstride = (long long)s.n_out * s.k;
+    op.a = a;
+    op.a_gstride = a_gstride;
+    op.lda = s.k;
+    op.ldw = s.k;
+    op.w_gstride = w_gstride;
+    op.w = wbase + (layered ? (long long)layer * N * w_gstride : 0);
+    if (bias) {
+        epi.bias = bias + (layered ? (long long)layer * N * s.n_out : 0);
+        epi.bias_gstride = s.n_out;
+    } else {
+        epi.bias = nullptr;
+        epi.bias_gstride = 0;
+    }
+    static const int cat_of[G_COUNT] = {KRAKEN_PROF_GEMM_QKV, KRAKEN_PROF_GEMM_PROJ, KRAKEN_PROF_GEMM_UP,
+                                        KRAKEN_PROF_GEMM_DOWN, KRAKEN_PROF_TAIL, KRAKEN_PROF_TAIL};
+    LaunchScope scope(h, cat_of[kind], rc.st);
+    if (h->naive) return launch_gemm_naive(op, s, epi, rc.st);
+
+    const int bn = gemm_pick_bn(s);
+    if (h->tmB_bn[kind] != bn) {
+        GemmOperands all = op;
+        all.w = wbase;
+        GemmShape sa = s;
+        sa.groups = total_groups;
+        int r = gemm_encode_b(&h->tmB[kind], all, sa, bn);
+        if (r) return r;
+        h->tmB_bn[kind] = bn;
+    }
+    // A maps: the up-projection reads the same buffer as qkv but after LN2, same shape -> same map works.
+    if (h->tmA_rows[kind] != m_rows) {
+        int r = gemm_encode_a(&h->tmA[kind], op, s);
+        if (r) return r;
+        h->tmA_rows[kind] = m_rows;
+    }
+    return launch_gemm_tc(op, s, epi, &h->tmA[kind], &h->tmB[kind], layered ? layer * N : 0, bn,
+                          at<uint32_t>(h, h->lay.status), rc.st);
+}
+
+EpiParams epi_zero() {
+    EpiParams e;
+    memset(&e, 0, sizeof(e));
+    return e;
+}
+
+#define KR_TRY(x)            \
+    do {                     \
+        int _rc = (x);       \
+        if (_rc) return _rc; \
+    } while (0)
+
+// Runs the L layers on `T = batch * seqlen` new tokens at positions pos0 .. pos0 + seqlen - 1.
+int run_layers(const RunCtx &rc, const int32_t *d_tokens) {
+    kraken_handle *h = rc.h;
+    const kraken_config &c = h->cfg;
+    const int d = c.d_model, F = c.d_ff, N = c.n_branch, L = c.n_layer, H = c.n_head, hd = d / H, T = rc.T;
+    const long long td = (long long)T * d;
+    float *x0 = at<float>(h, h->lay.x0), *x = at<float>(h, h->lay.x), *a = at<float>(h, h->lay.a),
+          *S = at<float>(h, h->lay.s);
+    uint16_t *u = at<uint16_t>(h, h->lay.u), *q = at<uint16_t>(h, h->lay.q), *o = at<uint16_t>(h, h->lay.o),
+             *gb = at<uint16_t>(h, h->lay.g);
+    uint32_t *status = at<uint32_t>(h, h->lay.status);
+    const long long cache_b = (long long)H * c.max_pos * hd;      // one sequence of one of K / V
+    const long long cache_kv = (long long)c.max_batch * cache_b;  // all of K (or V) of one (layer, branch)
+    uint16_t *kv = reinterpret_cast<uint16_t *>(h->kv);
+
+    {
+        LaunchScope scope(h, KRAKEN_PROF_EMBED, rc.st);
+        KR_TRY(launch_embed(d_tokens, T, rc.seqlen, rc.pos0, (const uint16_t *)h->w.wte, (const uint16_t *)h->w.wpe, d,
+                            c.vocab, x0, status, rc.st));
+    }
+    for (int l = 0; l < L; ++l) {
+        const float *xin = l == 0 ? x0 : x;
+        const long long xin_gs = l == 0 ? 0 : td;
+        const long long ln_off = (long long)l * N * d;
+        // x = LN(x)
+        {
+            LaunchScope scope(h, KRAKEN_PROF_LAYERNORM, rc.st);
+            KR_TRY(launch_layernorm(xin, xin_gs, nullptr, (const uint16_t *)h->w.ln1_g + ln_off,
+                                    h->w.ln1_b ? (const uint16_t *)h->w.ln1_b + ln_off : nullptr, N, T, d, c.ln_eps,
+                                    u, rc.st));
+        }
+        // q | k | v ; K and V go straight into the cache
+        uint16_t *kc = kv + (long long)l * N * 2 * cache_kv;
+        EpiParams e = epi_zero();
+        e.kind = KRAKEN_EPI_QKV;
+        e.out_bf16 = q; e.out_bf16_gstride = td; e.ld_out_bf16 = d;
+        e.k_cache = kc; e.v_cache = kc + cache_kv; e.cache_gstride = 2 * cache_kv;
+        e.seqlen = rc.seqlen; e.pos0 = rc.pos0; e.n_head = H; e.head_dim = hd; e.max_pos = c.max_pos; e.d_model = d;
+        KR_TRY(model_gemm(rc, G_QKV, l, T, u, td, e));
+        // attention over the cached prefix
+        AttnParams ap;
+        ap.q = q; ap.q_gstride = td;
+        ap.k_cache = kc; ap.v_cache = kc + cache_kv; ap.cache_gstride = 2 * cache_kv; ap.cache_bstride = cache_b;
+        ap.groups = N; ap.batch = rc.batch; ap.seqlen = rc.seqlen; ap.pos0 = rc.pos0; ap.n_head = H; ap.head_dim = hd;
+        ap.max_pos = c.max_pos; ap.out = o; ap.out_gstride = td;
+        {
+            LaunchScope scope(h, KRAKEN_PROF_ATTENTION, rc.st);
+            KR_TRY(h->naive ? launch_attention_naive(ap, rc.st) : launch_attention_prefill(ap, rc.st));
+        }
+        // x = res + MHA(x)
+        e = epi_zero();
+        e.kind = KRAKEN_EPI_RESID_F32;
+        e.out_f32 = a; e.out_f32_gstride = td; e.ld_out_f32 = d;
+        e.resid = xin; e.resid_gstride = xin_gs; e.ld_resid = d;
+        KR_TRY(model_gemm(rc, G_PROJ, l, T, o, td, e));
+        // x = LN(x + y): y is the shared embedding in the first layer, the cross-branch sum afterwards
+        {
+            LaunchScope scope(h, KRAKEN_PROF_LAYERNORM, rc.st);
+            KR_TRY(launch_layernorm(a, td, l == 0 ? x0 : S, (const uint16_t *)h->w.ln2_g + ln_off,
+                                    h->w.ln2_b ? (const uint16_t *)h->w.ln2_b + ln_off : nullptr, N, T, d, c.ln_eps,
+                                    u, rc.st));
+        }
+        // FFN up + GELU
+        e = epi_zero();
+        e.kind = KRAKEN_EPI_GELU_BF16;
+        e.out_bf16 = gb; e.out_bf16_gstride = (long long)T * F; e.ld_out_bf16 = F; e.gelu_tanh = c.gelu_tanh;
+        KR_TRY(model_gemm(rc, G_UP, l, T, u, td, e));
+        // out = res + FFN ; the sum over branches (the AllReduce feeding the next layer) in the epilogue
+        e = epi_zero();
+        e.kind = l + 1 < L ? KRAKEN_EPI_RESID_SUM : KRAKEN_EPI_RESID_F32;
+        e.out_f32 = x; e.out_f32_gstride = td; e.ld_out_f32 = d;
+        e.resid = a; e.resid_gstride = td; e.ld_resid = d;
+        e.sum = S; e.ld_sum = d;
+        KR_TRY(model_gemm(rc, G_DOWN, l, T, gb, (long long)T * F, e));
+    }
+    h->last_rows = T;
+    return KRAKEN_OK;
+}
+
+__global__ void make_rows_kernel(int32_t *rows, int n, int mul, int add) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) rows[i] = i * mul + add;
+}
+
+// W_concat, final LayerNorm and the tied unembedding for n_rows token rows (device index list).
+int run_tail(const RunCtx &rc, const int32_t *d_rows, int n_rows, float *d_logits) {
+    kraken_handle *h = rc.h;
+    const kraken_config &c = h->cfg;
+    const int d = c.d_model, N = c.n_branch;
+    const long long td = (long long)h->last_rows * d;
+    float *x = at<float>(h, h->lay.x), *z = at<float>(h, h->lay.s);
+    uint16_t *cat = at<uint16_t>(h, h->lay.u), *zf = at<uint16_t>(h, h->lay.q);
+    {
+        LaunchScope scope(h, KRAKEN_PROF_TAIL, rc.st);
+        KR_TRY(launch_gather_concat(x, td, N, d, d_rows, n_rows, cat, rc.st));
+    }
+    EpiParams e = epi_zero();
+    e.kind = KRAKEN_EPI_F32;
+    e.out_f32 = z; e.ld_out_f32 = d;
+    KR_TRY(model_gemm(rc, G_CONCAT, 0, n_rows, cat, 0, e));
+    {
+        LaunchScope scope(h, KRAKEN_PROF_TAIL, rc.st);
+        if (c.final_ln) {
+            KR_TRY(launch_layernorm(z, 0, nullptr, (const uint16_t *)h->w.lnf_g, (const uint16_t *)h->w.lnf_b, 1,
+                                    n_rows, d, c.ln_eps, zf, rc.st));
+        } else {
+            KR_TRY(launch_f32_to_bf16(z, zf, (long long)n_rows * d, rc.st));
+        }
+    }
+    e = epi_zero();
+    e.kind = KRAKEN_EPI_F32;
+    e.out_f32 = d_logits; e.ld_out_f32 = c.vocab;
+    KR_TRY(model_gemm(rc, G_HEAD, 0, n_rows, zf, 0, e));
+    return KRAKEN_OK;
+}
+
+int prefill_common(kraken_handle *h, const int32_t *d_tokens, int batch, int seqlen, float *d_logits, void *stream,
+                   bool all_logits) {
+    if (!h || !d_tokens || !d_logits || batch < 1 || seqlen < 1) return KRAKEN_EINVAL;
+    if (batch > h->cfg.max_batch || seqlen > h->cfg.max_pos) return KRAKEN_ECAPACITY;
+    RunCtx rc{h, static_cast<cudaStream_t>(stream), batch, seqlen, 0, batch * seqlen};
+    h->last_stream = rc.st;
+    KR_TRY(run_layers(rc, d_tokens));
+    h->cur_len = seqlen;
+    h->batch = batch;
+    h->last_seqlen = seqlen;
+    int32_t *rows = at<int32_t>(h, h->lay.rows);
+    const int n_rows = all_logits ? batch * seqlen : batch;
+    h->launches[KRAKEN_PROF_TAIL]++;
+    make_rows_kernel<<<(n_rows + 255) / 256, 256, 0, rc.st>>>(rows, n_rows, all_logits ? 1 : seqlen,
+                                                              all_logits ? 0 : seqlen - 1);
+    if (cudaGetLastError() != cudaSuccess) return KRAKEN_ECUDA;
+    return run_tail(rc, rows, n_rows, d_logits);
+}
+
+}  // namespace
+
+extern "C" {
+
+int kraken_query_sizes(const kraken_config *cfg, size_t *kv_bytes, size_t *scratch_bytes) {
+    int rc = check_config(cfg);
+    if (rc) return rc;
+    if (!kv_bytes || !scratch_bytes) return KRAKEN_EINVAL;
+    *kv_bytes = kv_bytes_of(cfg);
+    *scratch_bytes = layout_of(cfg).total;
+    return KRAKEN_OK;
+}
+
+int kraken_create(const kraken_config *cfg, const kraken_weights *w, void *d_kv, size_t kv_bytes, void *d_scratch,
+                  size_t scratch_bytes, kraken_handle **out) {
+    int rc = check_config(cfg);
+    if (rc) return rc;
+    if (!w || !d_kv || !d_scratch || !out) return KRAKEN_EINVAL;
+    if (!w->wte || !w->wpe || !w->ln1_g || !w->w_qkv || !w->w_proj || !w->ln2_g || !w->w_up || !w->w_down ||
+        !w->w_concat || (cfg->final_ln && !w->lnf_g))
+        return KRAKEN_EINVAL;
+    if ((reinterpret_cast<uintptr_t>(d_kv) & (ALIGN - 1)) || (reinterpret_cast<uintptr_t>(d_scratch) & (ALIGN - 1)))
+        return KRAKEN_EINVAL;
+    Layout lay = layout_of(cfg);
+    if (kv_bytes < kv_bytes_of(cfg) || scratch_bytes < lay.total) return KRAKEN_ECAPACITY;
+    kraken_handle *h = new (std::nothrow) kraken_handle();
+    if (!h) return KRAKEN_EINVAL;
+    h->cfg = *cfg;
+    h->w = *w;
+    h->kv = static_cast<uint8_t *>(d_kv);
+    h->scratch = static_cast<uint8_t *>(d_scratch);
+    h->lay = lay;
+    h->cur_len = 0;
+    h->batch = 0;
+    h->last_seqlen = 0;
+    h->last_rows = 0;
+    h->last_stream = nullptr;
+    h->naive = env_flag("KRAKEN_NAIVE");
+    h->prof_on = false;
+    h->ev_used = 0;
+    for (int i = 0; i < KRAKEN_PROF_COUNT; ++i) h->launches[i] = 0;
+    for (int i = 0; i < G_COUNT; ++i) {
+        h->tmB_bn[i] = 0;
+        h->tmA_rows[i] = 0;
+    }
+    if (cudaMemset(h->scratch + lay.status, 0, 256) != cudaSuccess) {
+        delete h;
+        return KRAKEN_ECUDA;
+    }
+    *out = h;
+    return KRAKEN_OK;
+}
+
+int kraken_prefill(kraken_handle *h, const int32_t *d_tokens, int32_t batch, int32_t seqlen, float *d_logits,
+                   void *stream) {
+    return prefill_common(h, d_tokens, batch, seqlen, d_logits, stream, false);
+}
+
+int kraken_prefill_all_logits(kraken_handle *h, const int32_t *d_tokens, int32_t batch, int32_t seqlen,
+                              float *d_logits, void *stream) {
+    return prefill_common(h, d_tokens, batch, seqlen, d_logits, stream, true);
+}
+
+int kraken_prefill_host(kraken_handle *h, const int32_t *h_tokens, int32_t batch, int32_t seqlen, float *h_logits,
+                        void *stream) {
+    if (!h || !h_tokens || !h_logits || batch < 1 || seqlen < 1) return KRAKEN_EINVAL;
+    if (batch > h->cfg.max_batch || seqlen > h->cfg.max_pos) return KRAKEN_ECAPACITY;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int32_t *d_tok = at<int32_t>(h, h->lay.tokens);
+    float *d_log = at<float>(h, h->lay.logits);
+    if (cudaMemcpyAsync(d_tok, h_tokens, (size_t)batch * seqlen * 4, cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return KRAKEN_ECUDA;
+    KR_TRY(prefill_common(h, d_tok, batch, seqlen, d_log, stream, false));
+    if (cudaMemcpyAsync(h_logits, d_log, (size_t)batch * h->cfg.vocab * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return KRAKEN_ECUDA;
+    return cudaStreamSynchronize(st) == cudaSuccess ? KRAKEN_OK : KRAKEN_ECUDA;
+}
+
+int kraken_logits_rows(kraken_handle *h, const int32_t *h_rows, int32_t n_rows, float *d_logits, void *stream) {
+    if (!h || !h_rows || !d_logits || n_rows < 1) return KRAKEN_EINVAL;
+    if (h->last_rows < 1) return KRAKEN_ESTATE;
+    if ((long long)n_rows > (long long)h->cfg.max_batch * h->cfg.max_pos) return KRAKEN_ECAPACITY;
+    for (int i = 0; i < n_rows; ++i)
+        if (h_rows[i] < 0 || h_rows[i] >= h->last_rows) return KRAKEN_EINVAL;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int32_t *rows = at<int32_t>(h, h->lay.rows);
+    if (cudaMemcpyAsync(rows, h_rows, (size_t)n_rows * 4, cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return KRAKEN_ECUDA;
+    RunCtx rc{h, st, h->batch, h->last_seqlen, 0, h->last_rows};
+    h->last_stream = st;
+    return run_tail(rc, rows, n_rows, d_logits);
+}
+
+int kraken_decode_step(kraken_handle *h, const int32_t *d_tokens, int32_t batch, float *d_logits, void *stream) {
+    if (!h || !d_tokens || !d_logits || batch < 1) return KRAKEN_EINVAL;
+    if (h->cur_len < 1 || batch != h->batch) return KRAKEN_ESTATE;
+    if (h->cur_len + 1 > h->cfg.max_pos) return KRAKEN_ECAPACITY;
+    RunCtx rc{h, static_cast<cudaStream_t>(stream), batch, 1, h->cur_len, batch};
+    h->last_stream = rc.st;
+    KR_TRY(run_layers(rc, d_tokens));
+    h->last_seqlen = 1;
+    int32_t *rows = at<int32_t>(h, h->lay.rows);
+    h->launches[KRAKEN_PROF_TAIL]++;
+    make_rows_kernel<<<(batch + 255) / 256, 256, 0, rc.st>>>(rows, batch, 1, 0);
+    if (cudaGetLastError() != cudaSuccess) return KRAKEN_ECUDA;
+    KR_TRY(run_tail(rc, rows, batch, d_logits));
+    h->cur_len += 1;
+    return KRAKEN_OK;
+}
+
+int kraken_kv_view(kraken_handle *h, int32_t layer, int32_t branch, int32_t which, const void **ptr,
+                   int64_t strides[4]) {
+    if (!h || !ptr || !strides) return KRAKEN_EINVAL;
+    const kraken_config &c = h->cfg;
+    if (layer < 0 || layer >= c.n_layer || branch < 0 || branch >= c.n_branch || which < 0 || which > 1)
+        return KRAKEN_EINVAL;
+    const int hd = c.d_model / c.n_head;
+    const long long cache_b = (long long)c.n_head * c.max_pos * hd, cache_kv = (long long)c.max_batch * cache_b;
+    *ptr = reinterpret_cast<uint16_t *>(h->kv) + (((long long)layer * c.n_branch + branch) * 2 + which) * cache_kv;
+    strides[0] = cache_b;
+    strides[1] = (long long)c.max_pos * hd;
+    strides[2] = hd;
+    strides[3] = 1;
+    return KRAKEN_OK;
+}
+
+int kraken_device_status(kraken_handle *h, uint32_t *flags) {
+    if (!h || !flags) return KRAKEN_EINVAL;
+    if (cudaStreamSynchronize(h->last_stream) != cudaSuccess) return KRAKEN_ECUDA;
+    if (cudaMemcpy(flags, h->scratch + h->lay.status, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return KRAKEN_ECUDA;
+    return KRAKEN_OK;
+}
+
+int kraken_cur_len(kraken_handle *h, int32_t *cur_len) {
+    if (!h || !cur_len) return KRAKEN_EINVAL;
+    *cur_len = h->cur_len;
+    return KRAKEN_OK;
+}
+
+int kraken_reset(kraken_handle *h) {
+    if (!h) return KRAKEN_EINVAL;
+    if (cudaStreamSynchronize(h->last_stream) != cudaSuccess) return KRAKEN_ECUDA;
+    if (cudaMemset(h->scratch + h->lay.status, 0, 256) != cudaSuccess) return KRAKEN_ECUDA;
+    h->cur_len = 0;
+    h->batch = 0;
+    h->last_rows = 0;
+    h->last_seqlen = 0;
+    return KRAKEN_OK;
+}
+
+void kraken_destroy(kraken_handle *h) {
+    if (!h) return;
+    for (cudaEvent_t e : h->ev_pool) cudaEventDestroy(e);
+    delete h;
+}
+
+int kraken_profile_enable(kraken_handle *h, int32_t on) {
+    if (!h) return KRAKEN_EINVAL;
+    h->prof_on = on != 0;
+    return KRAKEN_OK;
+}
+
+int kraken_profile_read(kraken_handle *h, double *ms, int64_t *launches) {
+    if (!h || !ms || !launches) return KRAKEN_EINVAL;
+    if (cudaStreamSynchronize(h->last_stream) != cudaSuccess) return KRAKEN_ECUDA;
+    for (int i = 0; i < KRAKEN_PROF_COUNT; ++i) {
+        ms[i] = 0.0;
+        launches[i] = h->launches[i];
+        h->launches[i] = 0;
+    }
+    for (const auto &sp : h->spans) {
+        float t = 0.f;
+        if (cudaEventElapsedTime(&t, h->ev_pool[sp.e0], h->ev_pool[sp.e1]) != cudaSuccess) return KRAKEN_ECUDA;
+        ms[sp.cat] += t;
+    }
+    h->spans.clear();
+    h->ev_used = 0;
+    return KRAKEN_OK;
+}
+
+const char *kraken_strerror(int status) {
+    switch (status) {
+        case KRAKEN_OK: return "ok";
+        case KRAKEN_EINVAL: return "invalid argument";
+        case KRAKEN_EUNSUPPORTED: return "unsupported shape (head_dim must be 64 or 128; d_model and d_ff multiples of 64)";
+        case KRAKEN_ECAPACITY: return "capacity exceeded (batch, sequence length or buffer size)";
+        case KRAKEN_ESTATE: return "call order violated (prefill first; decode batch must equal the prefill batch)";
+        case KRAKEN_ECUDA: return "a CUDA call failed";
+        default: return "unknown status";
+    }
+}
+
+// ------------------------------------------------------------------ single steps
+
+int kraken_op_embed(const int32_t *d_ids, int32_t n_tokens, int32_t seqlen, int32_t pos0, const void *wte,
+                    const void *wpe, int32_t d_model, int32_t vocab, float *d_out, uint32_t *d_status, void *stream) {
+    return launch_embed(d_ids, n_tokens, seqlen, pos0, (const uint16_t *)wte, (const uint16_t *)wpe, d_model, vocab,
+                        d_out, d_status, static_cast<cudaStream_t>(stream));
+}
+
+int kraken_op_layernorm(const float *d_a, int64_t a_gstride, const float *d_y, const void *gamma, const void *beta,
+                        int32_t groups, int32_t rows, int32_t d_model, float eps, void *d_out_bf16, void *stream) {
+    return launch_layernorm(d_a, a_gstride, d_y, (const uint16_t *)gamma, (const uint16_t *)beta, groups, rows,
+                            d_model, eps, (uint16_t *)d_out_bf16, static_cast<cudaStream_t>(stream));
+}
+
+int kraken_op_grouped_gemm(const kraken_gemm_args *g, uint32_t *d_status, void *stream) {
+    if (!g || !g->a || !g->w) return KRAKEN_EINVAL;
+    if (g->epilogue < KRAKEN_EPI_F32 || g->epilogue > KRAKEN_EPI_QKV) return KRAKEN_EINVAL;
+    const int k = g->epilogue;
+    const bool need_f32 = k == KRAKEN_EPI_F32 || k == KRAKEN_EPI_RESID_F32 || k == KRAKEN_EPI_RESID_SUM;
+    const bool need_bf16 = k == KRAKEN_EPI_BF16 || k == KRAKEN_EPI_GELU_BF16 || k == KRAKEN_EPI_QKV;
+    if ((need_f32 && !g->out_f32) || (need_bf16 && !g->out_bf16)) return KRAKEN_EINVAL;
+    if ((k == KRAKEN_EPI_RESID_F32 || k == KRAKEN_EPI_RESID_SUM) && !g->resid) return KRAKEN_EINVAL;
+    if (k == KRAKEN_EPI_RESID_SUM && !g->sum) return KRAKEN_EINVAL;
+    if (k == KRAKEN_EPI_QKV) {
+        if (!g->k_cache || !g->v_cache || g->seqlen < 1 || g->n_head < 1 || g->pos0 < 0) return KRAKEN_EINVAL;
+        if (g->head_dim % 32 != 0 || g->n_out != 3 * g->n_head * g->head_dim) return KRAKEN_EUNSUPPORTED;
+    }
+    GemmOperands op{g->a, g->a_gstride, g->lda, g->w, g->w_gstride, g->ldw};
+    GemmShape s{g->groups, g->m, g->n_out, g->k};
+    EpiParams e = epi_zero();
+    e.kind = k;
+    e.bias = (const uint16_t *)g->bias; e.bias_gstride = g->bias_gstride;
+    e.out_f32 = g->out_f32; e.out_f32_gstride = g->out_f32_gstride; e.ld_out_f32 = g->ld_out_f32;
+    e.out_bf16 = (uint16_t *)g->out_bf16; e.out_bf16_gstride = g->out_bf16_gstride; e.ld_out_bf16 = g->ld_out_bf16;
+    e.resid = g->resid; e.resid_gstride = g->resid_gstride; e.ld_resid = g->ld_resid;
+    e.sum = g->sum; e.ld_sum = g->ld_sum;
+    e.k_cache = (uint16_t *)g->k_cache; e.v_cache = (uint16_t *)g->v_cache; e.cache_gstride = g->cache_gstride;
+    e.seqlen = g->seqlen; e.pos0 = g->pos0; e.n_head = g->n_head; e.head_dim = g->head_dim; e.max_pos = g->max_pos;
+    e.d_model = g->n_head * g->head_dim;
+    e.gelu_tanh = g->gelu_tanh;
+    if (env_flag("KRAKEN_NAIVE")) return launch_gemm_naive(op, s, e, static_cast<cudaStream_t>(stream));
+    return launch_gemm_tc(op, s, e, nullptr, nullptr, 0, g->n_tile, d_status, static_cast<cudaStream_t>(stream));
+}
+
+int kraken_op_attention(const void *q, int64_t q_gstride, const void *k_cache, const void *v_cache,
+                        int64_t cache_gstride, int64_t cache_bstride, int32_t groups, int32_t batch, int32_t seqlen,
+                        int32_t pos0, int32_t n_head, int32_t head_dim, int32_t max_pos, void *out,
+                        int64_t out_gstride, void *stream) {
+    AttnParams p;
+    p.q = (const uint16_t *)q; p.q_gstride = q_gstride;
+    p.k_cache = (const uint16_t *)k_cache; p.v_cache = (const uint16_t *)v_cache;
+    p.cache_gstride = cache_gstride; p.cache_bstride = cache_bstride;
+    p.groups = groups; p.batch = batch; p.seqlen = seqlen; p.pos0 = pos0; p.n_head = n_head; p.head_dim = head_dim;
+    p.max_pos = max_pos; p.out = (uint16_t *)out; p.out_gstride = out_gstride;
+    if (env_flag("KRAKEN_NAIVE")) return launch_attention_naive(p, static_cast<cudaStream_t>(stream));
+    return launch_attention_prefill(p, static_cast<cudaStream_t>(stream));
+}
+
+}  // extern "C"

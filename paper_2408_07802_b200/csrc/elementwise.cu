@@ -1,0 +1,194 @@
+// HBM-bound steps of the path: shared embedding, the two LayerNorms of Algorithm 1 (the second
+// one fused with the addition of the cross-branch sum y), and the W_concat input gather.
+// One warp per row, 16-byte loads and stores, statistics in fp32.
+#include "internal.h"
+#include "ptx.cuh"
+
+namespace kr {
+
+namespace {
+
+constexpr int ROW_WARPS = 8;  // warps (rows) per CTA
+
+__global__ void __launch_bounds__(ROW_WARPS * 32)
+embed_kernel(const int32_t *__restrict__ ids, int n_tokens, int seqlen, int pos0, const uint16_t *__restrict__ wte,
+             const uint16_t *__restrict__ wpe, int d, int vocab, float *__restrict__ out, uint32_t *status) {
+    const int t = blockIdx.x * ROW_WARPS + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (t >= n_tokens) return;
+    int id = ids[t];
+    if (id < 0 || id >= vocab) {
+        if (lane == 0 && status) atomicOr(status, STATUS_BAD_TOKEN);
+        id = 0;
+    }
+    const int pos = pos0 + t % seqlen;
+    const uint4 *te = reinterpret_cast<const uint4 *>(wte + (size_t)id * d);
+    const uint4 *pe = reinterpret_cast<const uint4 *>(wpe + (size_t)pos * d);
+    float4 *o = reinterpret_cast<float4 *>(out + (size_t)t * d);
+    for (int v = lane; v < d / 8; v += 32) {
+        const uint4 a = __ldg(te + v), b = __ldg(pe + v);
+        o[2 * v] = make_float4(bf16_lo(a.x) + bf16_lo(b.x), bf16_hi(a.x) + bf16_hi(b.x),
+                               bf16_lo(a.y) + bf16_lo(b.y), bf16_hi(a.y) + bf16_hi(b.y));
+        o[2 * v + 1] = make_float4(bf16_lo(a.z) + bf16_lo(b.z), bf16_hi(a.z) + bf16_hi(b.z),
+                                   bf16_lo(a.w) + bf16_lo(b.w), bf16_hi(a.w) + bf16_hi(b.w));
+    }
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+    return v;
+}
+
+constexpr int LN_CACHE = 16;  // float4 per lane kept in registers: rows up to 2048 wide in one pass
+
+// out[g][r, :] = bf16( gamma_g * (v - mean) * rstd + beta_g ),  v = a[g][r, :] (+ y[r, :])
+__global__ void __launch_bounds__(ROW_WARPS * 32)
+layernorm_kernel(const float *__restrict__ a, long long a_gstride, const float *__restrict__ y,
+                 const uint16_t *__restrict__ gamma, const uint16_t *__restrict__ beta, int groups, int rows, int d,
+                 float eps, uint16_t *__restrict__ out) {
+    const long long wr = (long long)blockIdx.x * ROW_WARPS + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (wr >= (long long)groups * rows) return;
+    const int g = static_cast<int>(wr / rows), r = static_cast<int>(wr % rows);
+    const float4 *pa = reinterpret_cast<const float4 *>(a + g * a_gstride + (size_t)r * d);
+    const float4 *py = y ? reinterpret_cast<const float4 *>(y + (size_t)r * d) : nullptr;
+    const int nvec = d / 4;
+
+    float4 cache[LN_CACHE];
+    float sum = 0.f;
+#pragma unroll
+    for (int i = 0; i < LN_CACHE; ++i) {
+        const int v = lane + 32 * i;
+        if (v < nvec) {
+            float4 t = pa[v];
+            if (py) {
+                const float4 u = py[v];
+                t.x += u.x; t.y += u.y; t.z += u.z; t.w += u.w;
+            }
+            cache[i] = t;
+            sum += (t.x + t.y) + (t.z + t.w);
+        }
+    }
+    for (int v = lane + 32 * LN_CACHE; v < nvec; v += 32) {
+        float4 t = pa[v];
+        if (py) {
+            const float4 u = py[v];
+            t.x += u.x; t.y += u.y; t.z += u.z; t.w += u.w;
+        }
+        sum += (t.x + t.y) + (t.z + t.w);
+    }
+    const float mean = warp_sum(sum) / d;
+    float sq = 0.f;
+#pragma unroll
+    for (int i = 0; i < LN_CACHE; ++i) {
+        const int v = lane + 32 * i;
+        if (v < nvec) {
+            const float4 t = cache[i];
+            const float dx = t.x - mean, dy = t.y - mean, dz = t.z - mean, dw = t.w - mean;
+            sq += (dx * dx + dy * dy) + (dz * dz + dw * dw);
+        }
+    }
+    for (int v = lane + 32 * LN_CACHE; v < nvec; v += 32) {
+        float4 t = pa[v];
+        if (py) {
+            const float4 u = py[v];
+            t.x += u.x; t.y += u.y; t.z += u.z; t.w += u.w;
+        }
+        const float dx = t.x - mean, dy = t.y - mean, dz = t.z - mean, dw = t.w - mean;
+        sq += (dx * dx + dy * dy) + (dz * dz + dw * dw);
+    }
+    const float rstd = rsqrtf(warp_sum(sq) / d + eps);
+
+    const uint2 *pg = reinterpret_cast<const uint2 *>(gamma + (size_t)g * d);
+    const uint2 *pb = beta ? reinterpret_cast<const uint2 *>(beta + (size_t)g * d) : nullptr;
+    uint2 *po = reinterpret_cast<uint2 *>(out + ((size_t)g * rows + r) * d);
+    auto emit = [&](int v, const float4 &t) {
+        const uint2 gm = __ldg(pg + v);
+        uint2 bt = make_uint2(0u, 0u);
+        if (pb) bt = __ldg(pb + v);
+        const float o0 = (t.x - mean) * rstd * bf16_lo(gm.x) + bf16_lo(bt.x);
+        const float o1 = (t.y - mean) * rstd * bf16_hi(gm.x) + bf16_hi(bt.x);
+        const float o2 = (t.z - mean) * rstd * bf16_lo(gm.y) + bf16_lo(bt.y);
+        const float o3 = (t.w - mean) * rstd * bf16_hi(gm.y) + bf16_hi(bt.y);
+        po[v] = make_uint2(pack_bf16x2(o0, o1), pack_bf16x2(o2, o3));
+    };
+#pragma unroll
+    for (int i = 0; i < LN_CACHE; ++i) {
+        const int v = lane + 32 * i;
+        if (v < nvec) emit(v, cache[i]);
+    }
+    for (int v = lane + 32 * LN_CACHE; v < nvec; v += 32) {
+        float4 t = pa[v];
+        if (py) {
+            const float4 u = py[v];
+            t.x += u.x; t.y += u.y; t.z += u.z; t.w += u.w;
+        }
+        emit(v, t);
+    }
+}
+
+__global__ void __launch_bounds__(ROW_WARPS * 32)
+gather_concat_kernel(const float *__restrict__ x, long long x_gstride, int groups, int d,
+                     const int32_t *__restrict__ rows, int n_rows, uint16_t *__restrict__ out) {
+    const long long w = (long long)blockIdx.x * ROW_WARPS + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (w >= (long long)n_rows * groups) return;
+    const int r = static_cast<int>(w / groups), g = static_cast<int>(w % groups);
+    const int src_row = rows ? rows[r] : r;
+    const float4 *src = reinterpret_cast<const float4 *>(x + g * x_gstride + (size_t)src_row * d);
+    uint2 *dst = reinterpret_cast<uint2 *>(out + ((size_t)r * groups + g) * d);
+    for (int v = lane; v < d / 4; v += 32) {
+        const float4 t = src[v];
+        dst[v] = make_uint2(pack_bf16x2(t.x, t.y), pack_bf16x2(t.z, t.w));
+    }
+}
+
+__global__ void f32_to_bf16_kernel(const float *__restrict__ in, uint16_t *__restrict__ out, long long n) {
+    long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (; i < n; i += stride) out[i] = __bfloat16_as_ushort(__float2bfloat16_rn(in[i]));
+}
+
+int done() { return cudaGetLastError() == cudaSuccess ? KRAKEN_OK : KRAKEN_ECUDA; }
+
+}  // namespace
+
+int launch_embed(const int32_t *ids, int n_tokens, int seqlen, int pos0, const uint16_t *wte, const uint16_t *wpe,
+                 int d, int vocab, float *out, uint32_t *status, cudaStream_t stream) {
+    if (!ids || !wte || !wpe || !out || n_tokens < 1 || seqlen < 1 || pos0 < 0 || d < 8 || (d & 7) || vocab < 1)
+        return KRAKEN_EINVAL;
+    embed_kernel<<<(n_tokens + ROW_WARPS - 1) / ROW_WARPS, ROW_WARPS * 32, 0, stream>>>(ids, n_tokens, seqlen, pos0,
+                                                                                         wte, wpe, d, vocab, out,
+                                                                                         status);
+    return done();
+}
+
+int launch_layernorm(const float *a, long long a_gstride, const float *y, const uint16_t *gamma,
+                     const uint16_t *beta, int groups, int rows, int d, float eps, uint16_t *out,
+                     cudaStream_t stream) {
+    if (!a || !gamma || !out || groups < 1 || rows < 1 || d < 4 || (d & 3)) return KRAKEN_EINVAL;
+    const long long warps = (long long)groups * rows;
+    layernorm_kernel<<<static_cast<unsigned>((warps + ROW_WARPS - 1) / ROW_WARPS), ROW_WARPS * 32, 0, stream>>>(
+        a, a_gstride, y, gamma, beta, groups, rows, d, eps, out);
+    return done();
+}
+
+int launch_gather_concat(const float *x, long long x_gstride, int groups, int d, const int32_t *rows, int n_rows,
+                         uint16_t *out, cudaStream_t stream) {
+    if (!x || !out || groups < 1 || n_rows < 1 || (d & 3)) return KRAKEN_EINVAL;
+    const long long warps = (long long)groups * n_rows;
+    gather_concat_kernel<<<static_cast<unsigned>((warps + ROW_WARPS - 1) / ROW_WARPS), ROW_WARPS * 32, 0, stream>>>(
+        x, x_gstride, groups, d, rows, n_rows, out);
+    return done();
+}
+
+int launch_f32_to_bf16(const float *in, uint16_t *out, long long n, cudaStream_t stream) {
+    if (n < 1) return KRAKEN_EINVAL;
+    long long blocks = (n + 255) / 256;
+    if (blocks > 148 * 16) blocks = 148 * 16;
+    f32_to_bf16_kernel<<<static_cast<unsigned>(blocks), 256, 0, stream>>>(in, out, n);
+    return done();
+}
+
+}  // namespace kr

@@ -1,0 +1,138 @@
+// Fused GEMM epilogues (bias, GELU, residual add, cross-branch sum, K/V scatter into the cache).
+#pragma once
+#include "internal.h"
+#include "ptx.cuh"
+
+namespace kr {
+
+__device__ __forceinline__ float gelu_f(float x, int tanh_form) {
+    if (tanh_form) {
+        const float c = 0.7978845608028654f;
+        return 0.5f * x * (1.0f + tanhf(c * (x + 0.044715f * x * x * x)));
+    }
+    return 0.5f * x * (1.0f + erff(x * 0.7071067811865476f));
+}
+
+__device__ __forceinline__ void store_bf16_chunk(uint16_t *dst, const float (&v)[32], int ncols) {
+    if (ncols == 32 && (reinterpret_cast<uintptr_t>(dst) & 15u) == 0) {
+        uint4 *d4 = reinterpret_cast<uint4 *>(dst);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            uint4 u;
+            u.x = pack_bf16x2(v[8 * i + 0], v[8 * i + 1]);
+            u.y = pack_bf16x2(v[8 * i + 2], v[8 * i + 3]);
+            u.z = pack_bf16x2(v[8 * i + 4], v[8 * i + 5]);
+            u.w = pack_bf16x2(v[8 * i + 6], v[8 * i + 7]);
+            d4[i] = u;
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < 32; ++i)
+            if (i < ncols) dst[i] = __bfloat16_as_ushort(__float2bfloat16_rn(v[i]));
+    }
+}
+
+__device__ __forceinline__ void store_f32_chunk(float *dst, const float (&v)[32], int ncols) {
+    if (ncols == 32 && (reinterpret_cast<uintptr_t>(dst) & 15u) == 0) {
+        float4 *d4 = reinterpret_cast<float4 *>(dst);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) d4[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+    } else {
+#pragma unroll
+        for (int i = 0; i < 32; ++i)
+            if (i < ncols) dst[i] = v[i];
+    }
+}
+
+__device__ __forceinline__ void add_f32_chunk(const float *src, float (&v)[32], int ncols) {
+    if (ncols == 32 && (reinterpret_cast<uintptr_t>(src) & 15u) == 0) {
+        const float4 *s4 = reinterpret_cast<const float4 *>(src);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            float4 t = s4[i];
+            v[4 * i] += t.x;
+            v[4 * i + 1] += t.y;
+            v[4 * i + 2] += t.z;
+            v[4 * i + 3] += t.w;
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < 32; ++i)
+            if (i < ncols) v[i] += src[i];
+    }
+}
+
+__device__ __forceinline__ void add_bias_chunk(const uint16_t *bias, float (&v)[32], int ncols) {
+    if (ncols == 32 && (reinterpret_cast<uintptr_t>(bias) & 15u) == 0) {
+        const uint4 *b4 = reinterpret_cast<const uint4 *>(bias);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            uint4 u = __ldg(b4 + i);
+            v[8 * i + 0] += bf16_lo(u.x);
+            v[8 * i + 1] += bf16_hi(u.x);
+            v[8 * i + 2] += bf16_lo(u.y);
+            v[8 * i + 3] += bf16_hi(u.y);
+            v[8 * i + 4] += bf16_lo(u.z);
+            v[8 * i + 5] += bf16_hi(u.z);
+            v[8 * i + 6] += bf16_lo(u.w);
+            v[8 * i + 7] += bf16_hi(u.w);
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < 32; ++i)
+            if (i < ncols) v[i] += __uint_as_float(static_cast<uint32_t>(bias[i]) << 16);
+    }
+}
+
+// One thread finishes 32 consecutive columns (col0 .. col0+31, the first ncols of them valid)
+// of output row `row` of group g.  For KRAKEN_EPI_RESID_SUM the same thread must see the
+// groups of one (row, column) in ascending order (the running sum is read back by its writer).
+__device__ __forceinline__ void epilogue_chunk(const EpiParams &p, int g, int row, int col0, int ncols,
+                                               float (&v)[32]) {
+    if (p.bias) add_bias_chunk(p.bias + g * p.bias_gstride + col0, v, ncols);
+    switch (p.kind) {
+        case KRAKEN_EPI_F32:
+            store_f32_chunk(p.out_f32 + g * p.out_f32_gstride + (long long)row * p.ld_out_f32 + col0, v, ncols);
+            break;
+        case KRAKEN_EPI_BF16:
+            store_bf16_chunk(p.out_bf16 + g * p.out_bf16_gstride + (long long)row * p.ld_out_bf16 + col0, v, ncols);
+            break;
+        case KRAKEN_EPI_GELU_BF16:
+#pragma unroll
+            for (int i = 0; i < 32; ++i) v[i] = gelu_f(v[i], p.gelu_tanh);
+            store_bf16_chunk(p.out_bf16 + g * p.out_bf16_gstride + (long long)row * p.ld_out_bf16 + col0, v, ncols);
+            break;
+        case KRAKEN_EPI_RESID_F32:
+            add_f32_chunk(p.resid + g * p.resid_gstride + (long long)row * p.ld_resid + col0, v, ncols);
+            store_f32_chunk(p.out_f32 + g * p.out_f32_gstride + (long long)row * p.ld_out_f32 + col0, v, ncols);
+            break;
+        case KRAKEN_EPI_RESID_SUM: {
+            add_f32_chunk(p.resid + g * p.resid_gstride + (long long)row * p.ld_resid + col0, v, ncols);
+            store_f32_chunk(p.out_f32 + g * p.out_f32_gstride + (long long)row * p.ld_out_f32 + col0, v, ncols);
+            float *s = p.sum + (long long)row * p.ld_sum + col0;
+            if (g > 0) add_f32_chunk(s, v, ncols);
+            store_f32_chunk(s, v, ncols);
+            break;
+        }
+        case KRAKEN_EPI_QKV: {
+            const int d = p.d_model;
+            if (col0 < d) {
+                store_bf16_chunk(p.out_bf16 + g * p.out_bf16_gstride + (long long)row * p.ld_out_bf16 + col0, v,
+                                 ncols);
+            } else {
+                const int which = col0 >= 2 * d;
+                const int c = col0 - (1 + which) * d;
+                const int head = c / p.head_dim, e0 = c % p.head_dim;
+                const int b = row / p.seqlen, pos = p.pos0 + row % p.seqlen;
+                uint16_t *base = (which ? p.v_cache : p.k_cache) + g * p.cache_gstride;
+                store_bf16_chunk(base + (((long long)b * p.n_head + head) * p.max_pos + pos) * p.head_dim + e0, v,
+                                 ncols);
+            }
+            break;
+        }
+        default:
+            break;
+    }
+}
+
+}  // namespace kr

@@ -1,0 +1,301 @@
+// Grouped bf16 GEMM  C_g[M, Nout] = A_g[M, K] . W_g[Nout, K]^T  on the sm_100a tensor cores.
+//
+// One persistent CTA per SM, six warps:
+//   warp 0    TMA producer: 128 x 64 tile of A and BN x 64 tile of W per stage, 128-byte swizzle;
+//   warp 1    allocates TMEM and issues tcgen05.mma (128 x BN x 16 per instruction, fp32
+//             accumulators in TMEM, two accumulator buffers so that draining tile i overlaps
+//             the MMAs of tile i+1);
+//   warps 2-5 epilogue: tcgen05.ld of their 32-lane quarter, fused epilogue, global stores.
+// The group (branch) index is the outermost TMA coordinate.  Rows past M, columns past Nout
+// and the K tail are zero-filled by TMA and masked in the epilogue.
+//
+// The down-projection's cross-branch sum (the AllReduce of Algorithm 1) needs the N groups
+// of one output tile on the same CTA in ascending order: `group_serial` scheduling.
+#include <stdio.h>
+#include <stdlib.h>
+
+#include "epilogue.cuh"
+#include "internal.h"
+#include "ptx.cuh"
+
+namespace kr {
+
+namespace {
+
+constexpr int BM = 128;
+constexpr int BK = 64;
+constexpr int UMMA_K = 16;
+constexpr int NUM_THREADS = 192;
+constexpr int SMEM_BUDGET = 200 * 1024;
+
+template <int BN>
+struct TileCfg {
+    static constexpr int A_BYTES = BM * BK * 2;
+    static constexpr int B_BYTES = BN * BK * 2;
+    static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+    static constexpr int STAGES = SMEM_BUDGET / STAGE_BYTES > 8 ? 8 : SMEM_BUDGET / STAGE_BYTES;
+    static constexpr int TMEM_COLS = 2 * BN;  // two accumulators; 128, 256 or 512 columns
+    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+};
+
+struct KernelArgs {
+    GemmShape shape;
+    EpiParams epi;
+    int tiles_m, tiles_n;
+    int a_gmul, b_gmul;  // 0 when the operand is shared by all groups
+    int a_g0, b_g0;      // first group's index along the outermost TMA dimension
+    int group_serial;
+    uint32_t *status;
+};
+
+__device__ __forceinline__ bool next_item(const KernelArgs &ka, int it, int &m_blk, int &n_blk, int &g) {
+    const int G = ka.shape.groups;
+    const int num_tiles = ka.tiles_m * ka.tiles_n;
+    int tile;
+    if (ka.group_serial) {
+        tile = blockIdx.x + (it / G) * gridDim.x;
+        g = it % G;
+    } else {
+        const long long idx = blockIdx.x + (long long)it * gridDim.x;
+        tile = static_cast<int>(idx / G);
+        g = static_cast<int>(idx % G);
+    }
+    if (tile >= num_tiles) return false;
+    m_blk = tile % ka.tiles_m;  // m fastest: one wave shares few W tiles, A stays in L2
+    n_blk = tile / ka.tiles_m;
+    return true;
+}
+
+template <int BN>
+__global__ void __launch_bounds__(NUM_THREADS, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+               const KernelArgs ka) {
+    using Cfg = TileCfg<BN>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t *tiles = smem;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + Cfg::STAGES * Cfg::STAGE_BYTES);
+    uint64_t *full_bar = bars;                      // [STAGES]
+    uint64_t *empty_bar = bars + Cfg::STAGES;       // [STAGES]
+    uint64_t *acc_full = bars + 2 * Cfg::STAGES;    // [2]
+    uint64_t *acc_empty = bars + 2 * Cfg::STAGES + 2;  // [2]
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * Cfg::STAGES + 4);
+    volatile uint32_t *abort_flag = tmem_slot + 1;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int k_blocks = (ka.shape.k + BK - 1) / BK;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < Cfg::STAGES; ++s) {
+            mbar_init(full_bar + s, 1);
+            mbar_init(empty_bar + s, 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(acc_full + a, 1);
+            mbar_init(acc_empty + a, 4);
+        }
+        *abort_flag = 0;
+        fence_barrier_init();
+        prefetch_tensormap(&tmA);
+        prefetch_tensormap(&tmB);
+    }
+    if (warp == 1) {
+        tmem_alloc(tmem_slot, Cfg::TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            int m_blk, n_blk, g;
+            for (int it = 0; ok && next_item(ka, it, m_blk, n_blk, g); ++it) {
+                for (int kb = 0; kb < k_blocks; ++kb) {
+                    if (!(ok = mbar_wait(empty_bar + stage, phase ^ 1u, abort_flag))) break;
+                    uint8_t *sa = tiles + stage * Cfg::STAGE_BYTES;
+                    uint8_t *sb = sa + Cfg::A_BYTES;
+                    mbar_expect_tx(full_bar + stage, Cfg::STAGE_BYTES);
+                    tma_load_3d(sa, &tmA, full_bar + stage, kb * BK, m_blk * BM, ka.a_g0 + g * ka.a_gmul);
+                    tma_load_3d(sb, &tmB, full_bar + stage, kb * BK, n_blk * BN, ka.b_g0 + g * ka.b_gmul);
+                    if (++stage == Cfg::STAGES) {
+                        stage = 0;
+                        phase ^= 1u;
+                    }
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t idesc = umma_idesc_bf16(BM, BN);
+            int stage = 0;
+            uint32_t phase = 0;
+            int acc = 0;
+            uint32_t acc_phase = 0;
+            bool ok = true;
+            int m_blk, n_blk, g;
+            for (int it = 0; ok && next_item(ka, it, m_blk, n_blk, g); ++it) {
+                if (!(ok = mbar_wait(acc_empty + acc, acc_phase ^ 1u, abort_flag))) break;
+                tc_fence_after_sync();
+                const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * BN);
+                for (int kb = 0; kb < k_blocks; ++kb) {
+                    if (!(ok = mbar_wait(full_bar + stage, phase, abort_flag))) break;
+                    tc_fence_after_sync();
+                    const uint32_t sa = smem_u32(tiles + stage * Cfg::STAGE_BYTES);
+                    const uint32_t sb = sa + Cfg::A_BYTES;
+#pragma unroll
+                    for (int k = 0; k < BK / UMMA_K; ++k) {
+                        umma_bf16_ss(d_tmem, umma_desc_sw128_kmajor(sa + k * UMMA_K * 2),
+                                     umma_desc_sw128_kmajor(sb + k * UMMA_K * 2), idesc, (kb | k) != 0 ? 1u : 0u);
+                    }
+                    umma_commit(empty_bar + stage);  // frees the stage once these MMAs have read it
+                    if (++stage == Cfg::STAGES) {
+                        stage = 0;
+                        phase ^= 1u;
+                    }
+                }
+                if (!ok) break;
+                umma_commit(acc_full + acc);  // accumulator complete
+                if (++acc == 2) {
+                    acc = 0;
+                    acc_phase ^= 1u;
+                }
+            }
+        }
+        __syncwarp();
+    } else {
+        const int quarter = warp & 3;  // TMEM lanes this warp may read
+        int acc = 0;
+        uint32_t acc_phase = 0;
+        bool ok = true;
+        int m_blk, n_blk, g;
+        for (int it = 0; ok && next_item(ka, it, m_blk, n_blk, g); ++it) {
+            ok = mbar_wait(acc_full + acc, acc_phase, abort_flag);
+            ok = __all_sync(0xFFFFFFFFu, ok);
+            if (!ok) break;
+            tc_fence_after_sync();
+            const int row = m_blk * BM + quarter * 32 + lane;
+            const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
+                                   static_cast<uint32_t>(acc * BN);
+#pragma unroll 1
+            for (int c = 0; c < BN / 32; ++c) {
+                const int col0 = n_blk * BN + c * 32;
+                if (col0 >= ka.shape.n_out) break;  // uniform across the warp
+                uint32_t r[32];
+                tmem_ld_32x32(t_row + static_cast<uint32_t>(c * 32), r);
+                tmem_ld_wait();
+                if (row < ka.shape.m) {
+                    float v[32];
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+                    const int ncols = min(32, ka.shape.n_out - col0);
+                    epilogue_chunk(ka.epi, g, row, col0, ncols, v);
+                }
+            }
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(acc_empty + acc);
+            if (++acc == 2) {
+                acc = 0;
+                acc_phase ^= 1u;
+            }
+        }
+    }
+
+    // teardown (also reached when a bounded wait gave up)
+    if (*abort_flag) {
+        // give copies and MMAs still in flight time to land before shared memory and TMEM go away
+        for (int i = 0; i < 64; ++i) __nanosleep(10000);
+        if (threadIdx.x == 0 && ka.status) atomicOr(ka.status, STATUS_WAIT_LIMIT);
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) tmem_dealloc(tmem_base, Cfg::TMEM_COLS);
+}
+
+template <int BN>
+int launch_bn(const CUtensorMap &tmA, const CUtensorMap &tmB, const KernelArgs &ka, int grid, cudaStream_t stream) {
+    using Cfg = TileCfg<BN>;
+    static bool configured = false;
+    if (!configured) {
+        if (cudaFuncSetAttribute(gemm_tc_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES) !=
+            cudaSuccess)
+            return KRAKEN_ECUDA;
+        configured = true;
+    }
+    gemm_tc_kernel<BN><<<grid, NUM_THREADS, Cfg::SMEM_BYTES, stream>>>(tmA, tmB, ka);
+    return cudaGetLastError() == cudaSuccess ? KRAKEN_OK : KRAKEN_ECUDA;
+}
+
+}  // namespace
+
+int gemm_pick_bn(const GemmShape &s) {
+    const int sms = sm_count() > 0 ? sm_count() : 148;
+    const long long tiles_m = (s.m + BM - 1) / BM;
+    // Largest N tile that still gives every SM about one work item.
+    for (int bn : {256, 128}) {
+        const long long items = tiles_m * ((s.n_out + bn - 1) / bn) * s.groups;
+        if (items >= sms) return bn;
+    }
+    return 64;
+}
+
+int gemm_encode_a(CUtensorMap *map, const GemmOperands &op, const GemmShape &s) {
+    const bool shared = op.a_gstride == 0 || s.groups == 1;
+    return encode_tma_3d_bf16(map, op.a, s.k, s.m, shared ? 1 : s.groups, op.lda,
+                              shared ? (uint64_t)op.lda * s.m : (uint64_t)op.a_gstride, BK, BM);
+}
+
+int gemm_encode_b(CUtensorMap *map, const GemmOperands &op, const GemmShape &s, int bn) {
+    const bool shared = op.w_gstride == 0 || s.groups == 1;
+    return encode_tma_3d_bf16(map, op.w, s.k, s.n_out, shared ? 1 : s.groups, op.ldw,
+                              shared ? (uint64_t)op.ldw * s.n_out : (uint64_t)op.w_gstride, BK, bn);
+}
+
+int launch_gemm_tc(const GemmOperands &op, const GemmShape &s, const EpiParams &epi, const CUtensorMap *tmA,
+                   const CUtensorMap *tmB, int b_g0, int bn_hint, uint32_t *d_status, cudaStream_t stream) {
+    if (s.groups < 1 || s.m < 1 || s.n_out < 1 || s.k < 8) return KRAKEN_EINVAL;
+    if ((op.lda & 7) || (op.ldw & 7) || (reinterpret_cast<uintptr_t>(op.a) & 15) ||
+        (reinterpret_cast<uintptr_t>(op.w) & 15) || (op.a_gstride & 7) || (op.w_gstride & 7))
+        return KRAKEN_EUNSUPPORTED;
+    const int bn = bn_hint ? bn_hint : gemm_pick_bn(s);
+    CUtensorMap la, lb;
+    if (!tmA) {
+        int rc = gemm_encode_a(&la, op, s);
+        if (rc) return rc;
+        tmA = &la;
+    }
+    if (!tmB) {
+        int rc = gemm_encode_b(&lb, op, s, bn);
+        if (rc) return rc;
+        tmB = &lb;
+    }
+    KernelArgs ka;
+    ka.shape = s;
+    ka.epi = epi;
+    ka.tiles_m = (s.m + BM - 1) / BM;
+    ka.tiles_n = (s.n_out + bn - 1) / bn;
+    ka.a_gmul = (op.a_gstride == 0 || s.groups == 1) ? 0 : 1;
+    ka.b_gmul = (op.w_gstride == 0 || s.groups == 1) ? 0 : 1;
+    ka.a_g0 = 0;
+    ka.b_g0 = b_g0;
+    ka.group_serial = epi.kind == KRAKEN_EPI_RESID_SUM ? 1 : 0;
+    ka.status = d_status;
+    const long long tiles = (long long)ka.tiles_m * ka.tiles_n;
+    const long long units = ka.group_serial ? tiles : tiles * s.groups;
+    const int sms = sm_count() > 0 ? sm_count() : 148;
+    const int grid = static_cast<int>(units < sms ? units : sms);
+    switch (bn) {
+        case 256: return launch_bn<256>(*tmA, *tmB, ka, grid, stream);
+        case 128: return launch_bn<128>(*tmA, *tmB, ka, grid, stream);
+        case 64: return launch_bn<64>(*tmA, *tmB, ka, grid, stream);
+        default: return KRAKEN_EINVAL;
+    }
+}
+
+}  // namespace kr

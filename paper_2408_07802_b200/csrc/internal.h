@@ -1,0 +1,91 @@
+// Declarations shared by the translation units of the library (host side).
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/kraken.h"
+
+namespace kr {
+
+// Epilogue description handed to the GEMM kernels (device pointers, strides in elements).
+struct EpiParams {
+    int kind;  // kraken_epilogue
+    const uint16_t *bias;
+    long long bias_gstride;
+    float *out_f32;
+    long long out_f32_gstride;
+    int ld_out_f32;
+    uint16_t *out_bf16;
+    long long out_bf16_gstride;
+    int ld_out_bf16;
+    const float *resid;
+    long long resid_gstride;
+    int ld_resid;
+    float *sum;
+    int ld_sum;
+    uint16_t *k_cache, *v_cache;
+    long long cache_gstride;
+    int seqlen, pos0, n_head, head_dim, max_pos, d_model;
+    int gelu_tanh;
+};
+
+struct GemmShape {
+    int groups, m, n_out, k;
+};
+
+// Host-resolved driver entry point for tensor-map encoding; returns KRAKEN_ECUDA if unavailable.
+int encode_tma_3d_bf16(CUtensorMap *map, const void *base, uint64_t dim0, uint64_t dim1, uint64_t dim2,
+                       uint64_t stride1_elems, uint64_t stride2_elems, uint32_t box0, uint32_t box1);
+int encode_tma_4d_bf16(CUtensorMap *map, const void *base, const uint64_t dims[4], const uint64_t strides_elems[3],
+                       const uint32_t box[4]);
+
+int sm_count();
+
+// Tensor-core grouped GEMM.  tmA / tmB may be NULL: they are then encoded from the operands.
+// b_g0: index of the first group along the outermost dimension of a caller-made tmB (a map
+// that spans the weights of every layer).
+struct GemmOperands {
+    const void *a;
+    long long a_gstride;
+    int lda;
+    const void *w;
+    long long w_gstride;
+    int ldw;
+};
+int launch_gemm_tc(const GemmOperands &op, const GemmShape &shape, const EpiParams &epi, const CUtensorMap *tmA,
+                   const CUtensorMap *tmB, int b_g0, int bn_hint, uint32_t *d_status, cudaStream_t stream);
+// Picks the N tile for a shape (64, 128 or 256).
+int gemm_pick_bn(const GemmShape &shape);
+int gemm_encode_a(CUtensorMap *map, const GemmOperands &op, const GemmShape &shape);
+int gemm_encode_b(CUtensorMap *map, const GemmOperands &op, const GemmShape &shape, int bn);
+
+// One thread per output element; for bring-up comparisons only (KRAKEN_NAIVE=1).
+int launch_gemm_naive(const GemmOperands &op, const GemmShape &shape, const EpiParams &epi, cudaStream_t stream);
+
+int launch_embed(const int32_t *ids, int n_tokens, int seqlen, int pos0, const uint16_t *wte, const uint16_t *wpe,
+                 int d, int vocab, float *out, uint32_t *status, cudaStream_t stream);
+int launch_layernorm(const float *a, long long a_gstride, const float *y, const uint16_t *gamma,
+                     const uint16_t *beta, int groups, int rows, int d, float eps, uint16_t *out,
+                     cudaStream_t stream);
+// rows of N fp32 branch outputs -> bf16 branch-major concatenation [n_rows, N*d]; rows picked by index list
+// (device int32, NULL = identity).
+int launch_gather_concat(const float *x, long long x_gstride, int groups, int d, const int32_t *rows, int n_rows,
+                         uint16_t *out, cudaStream_t stream);
+int launch_f32_to_bf16(const float *in, uint16_t *out, long long n, cudaStream_t stream);
+
+struct AttnParams {
+    const uint16_t *q;
+    long long q_gstride;
+    const uint16_t *k_cache, *v_cache;
+    long long cache_gstride, cache_bstride;
+    int groups, batch, seqlen, pos0, n_head, head_dim, max_pos;
+    uint16_t *out;
+    long long out_gstride;
+};
+int launch_attention_prefill(const AttnParams &p, cudaStream_t stream);
+int launch_attention_naive(const AttnParams &p, cudaStream_t stream);
+
+bool env_flag(const char *name);
+
+}  // namespace kr

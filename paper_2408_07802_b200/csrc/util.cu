@@ -1,0 +1,81 @@
+// Host utilities: tensor-map encoding through the driver entry point, device queries, env flags.
+#include <stdlib.h>
+#include <string.h>
+
+#include <mutex>
+
+#include "internal.h"
+
+namespace kr {
+
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static std::once_flag once;
+    std::call_once(once, [] {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+    });
+    return fn;
+}
+
+int encode(CUtensorMap *map, const void *base, int rank, const uint64_t *dims, const uint64_t *strides_elems,
+           const uint32_t *box) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return KRAKEN_ECUDA;
+    cuuint64_t gdim[5], gstride[4];
+    cuuint32_t bdim[5], estride[5];
+    for (int i = 0; i < rank; ++i) {
+        gdim[i] = dims[i];
+        bdim[i] = box[i];
+        estride[i] = 1;
+    }
+    for (int i = 0; i + 1 < rank; ++i) gstride[i] = strides_elems[i] * 2;  // bytes
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, rank, const_cast<void *>(base), gdim, gstride, bdim,
+                    estride, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                    CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? KRAKEN_OK : KRAKEN_ECUDA;
+}
+
+}  // namespace
+
+int encode_tma_3d_bf16(CUtensorMap *map, const void *base, uint64_t dim0, uint64_t dim1, uint64_t dim2,
+                       uint64_t stride1_elems, uint64_t stride2_elems, uint32_t box0, uint32_t box1) {
+    const uint64_t dims[3] = {dim0, dim1, dim2};
+    const uint64_t strides[2] = {stride1_elems, stride2_elems};
+    const uint32_t box[3] = {box0, box1, 1};
+    return encode(map, base, 3, dims, strides, box);
+}
+
+int encode_tma_4d_bf16(CUtensorMap *map, const void *base, const uint64_t dims[4], const uint64_t strides_elems[3],
+                       const uint32_t box[4]) {
+    return encode(map, base, 4, dims, strides_elems, box);
+}
+
+int sm_count() {
+    static int n = -1;
+    if (n < 0) {
+        int dev = 0, v = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess &&
+            cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess)
+            n = v;
+        else
+            return 0;
+    }
+    return n;
+}
+
+bool env_flag(const char *name) {
+    const char *v = getenv(name);
+    return v && *v && strcmp(v, "0") != 0;
+}
+
+}  // namespace kr

@@ -1,0 +1,269 @@
+"""Whole-path parity: the CUDA library through its C ABI against the CPU oracle, same seeded inputs.
+
+Bounds (stated by the benchmark definition): relative L2 <= 1e-2 and max |error| <= 5e-2 on the
+logits against the fp32 oracle; arg-max agreement >= 99.9 % of positions against the oracle that
+rounds activations to bf16 at the same points (a disagreement counts as a tie, not an error, when
+the oracle's own margin between the two tokens is below twice the measured max error); token and
+KV-cache indexing exact.
+"""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import kraken_inputs as ki
+import oracle
+import paper_2408_07802_b200 as kr
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+REL_L2_MAX = 1e-2
+MAX_ABS_MAX = 5e-2
+ARGMAX_MIN = 0.999
+
+
+def host_bits(w):
+    return {k: (None if v is None else ki.bf16_tensor_to_bits(v)) for k, v in w.items()}
+
+
+def build(shape, seed=0, bias=True, max_batch=None, **over):
+    w = ki.make_weights(shape, seed=seed, device=DEV, bias=bias)
+    cfg = kr.make_config(shape, max_batch=max_batch, **over)
+    return kr.KrakenModel(cfg, w, DEV), w
+
+
+def logits_metrics(got, ref):
+    got, ref = got.astype(np.float64), ref.astype(np.float64)
+    rel = np.linalg.norm(got - ref) / np.linalg.norm(ref)
+    return rel, np.abs(got - ref).max()
+
+
+def argmax_agreement(got, ref):
+    """(raw rate, tie-adjusted rate) over rows of [rows, V]."""
+    ga, ra = got.argmax(1), ref.argmax(1)
+    same = ga == ra
+    err = np.abs(got - ref).max()
+    rows = np.arange(len(ga))
+    margin = ref[rows, ra] - ref[rows, ga]
+    tie = (~same) & (margin <= 2 * err)
+    return same.mean(), (same | tie).mean()
+
+
+def check_parity(got, ref32, refbf, what):
+    assert not np.isnan(got).any(), what
+    rel, mx = logits_metrics(got, ref32)
+    raw, adj = argmax_agreement(got, refbf)
+    print(f"[parity] {what}: relL2={rel:.3e} maxabs={mx:.3e} argmax raw={raw:.4f} tie-adjusted={adj:.4f}")
+    assert rel <= REL_L2_MAX, (what, rel)
+    assert mx <= MAX_ABS_MAX, (what, mx)
+    assert adj >= ARGMAX_MIN, (what, raw, adj)
+    return rel, mx, raw, adj
+
+
+def oracle_all_logits(shape, wb, ids_row, bf16_store, logits_from=0):
+    orc = oracle.Oracle(shape, wb, bf16_store=bf16_store)
+    lg, _ = orc.prefill(ids_row, logits_from=logits_from)
+    return lg, orc
+
+
+# ------------------------------------------------------------------ C0: everything, element by element
+
+def test_c0_prefill_parity_all_positions_and_cache():
+    s = ki.CONFIGS["C0"]
+    m, w = build(s)
+    wb = host_bits(w)
+    tok = ki.uniform_tokens(1, s.vocab, s.batch, s.seqlen, DEV)
+    got_all = m.prefill_all_logits(tok).cpu().numpy()[0]
+    ref32, _ = oracle_all_logits(s, wb, tok[0].cpu().numpy(), False)
+    refbf, orc = oracle_all_logits(s, wb, tok[0].cpu().numpy(), True)
+    check_parity(got_all, ref32, refbf, "C0 all positions")
+    # the call the benchmark times returns the last position of that same computation
+    last = m.prefill(tok).cpu().numpy()
+    assert np.allclose(last[0], got_all[-1], atol=1e-5)
+    assert m.device_status() == 0 and m.cur_len == s.seqlen
+    # KV cache: the bf16 k, v rows, in [batch, head, position, dim] order
+    worst = 0
+    for layer in range(s.n_layer):
+        for n in range(s.n_branch):
+            for which in (0, 1):
+                g = m.kv_view(layer, n, which)[0, :, :s.seqlen].float().cpu().numpy()
+                r = orc.cache(layer, n, which)
+                ulp = np.abs(g - r) / (np.abs(r) * 2.0 ** -7 + 1e-6)
+                worst = max(worst, ulp.max())
+                assert (ulp <= 2.0).all(), (layer, n, which, ulp.max())
+                assert (g == r).mean() > 0.9
+    print(f"[parity] C0 cache worst bf16-ulp distance {worst:.2f}")
+
+
+def test_c0_without_biases_and_without_final_ln():
+    s = ki.CONFIGS["C0"]
+    for bias, final_ln in ((False, 1), (True, 0)):
+        m, w = build(s, bias=bias, final_ln=final_ln)
+        wb = host_bits(w)
+        tok = ki.uniform_tokens(1, s.vocab, 1, 96, DEV)
+        got = m.prefill_all_logits(tok).cpu().numpy()[0]
+        orc = oracle.Oracle(s, wb, final_ln=bool(final_ln))
+        ref, _ = orc.prefill(tok[0].cpu().numpy())
+        rel, mx = logits_metrics(got, ref)
+        print(f"[parity] C0 bias={bias} final_ln={final_ln}: relL2={rel:.3e} maxabs={mx:.3e}")
+        assert rel <= REL_L2_MAX and mx <= MAX_ABS_MAX
+
+
+def test_ragged_lengths_and_batches():
+    """Sequence lengths that are not tile multiples, batch > 1: each sequence equals its own oracle run."""
+    s = ki.CONFIGS["C0"]
+    m, w = build(s, max_batch=3)
+    wb = host_bits(w)
+    for seqlen in (1, 7, 65, 127):
+        tok = ki.uniform_tokens(seqlen, s.vocab, 3, seqlen, DEV)
+        got = m.prefill_all_logits(tok).cpu().numpy()
+        for b in range(3):
+            ref, _ = oracle_all_logits(s, wb, tok[b].cpu().numpy(), False)
+            rel, mx = logits_metrics(got[b], ref)
+            assert rel <= REL_L2_MAX and mx <= MAX_ABS_MAX, (seqlen, b, rel, mx)
+
+
+def test_naive_kernels_agree_with_tensor_core_path():
+    s = ki.CONFIGS["C0"]
+    tok = ki.uniform_tokens(1, s.vocab, 1, 100, DEV)
+    m, _ = build(s)
+    fast = m.prefill_all_logits(tok).cpu().numpy()
+    os.environ["KRAKEN_NAIVE"] = "1"
+    try:
+        m2, _ = build(s)
+        slow = m2.prefill_all_logits(tok).cpu().numpy()
+    finally:
+        del os.environ["KRAKEN_NAIVE"]
+    rel, mx = logits_metrics(fast[0], slow[0])
+    assert rel < 5e-3 and mx < 3e-2, (rel, mx)
+
+
+def test_prefill_host_matches_device_call():
+    s = ki.CONFIGS["C0"]
+    m, _ = build(s)
+    tok = ki.uniform_tokens(1, s.vocab, 1, s.seqlen, DEV)
+    dev = m.prefill(tok).cpu()
+    h_tok = tok.cpu().pin_memory()
+    h_log = torch.empty(1, s.vocab, dtype=torch.float32).pin_memory()
+    m.prefill_host(h_tok, h_log)
+    assert torch.equal(h_log, dev)
+
+
+def test_run_to_run_determinism():
+    s = ki.CONFIGS["C0"]
+    m, _ = build(s)
+    tok = ki.uniform_tokens(1, s.vocab, 1, s.seqlen, DEV)
+    a = m.prefill_all_logits(tok).clone()
+    b = m.prefill_all_logits(tok)
+    assert torch.equal(a, b)
+
+
+def test_status_flags_and_error_codes():
+    s = ki.CONFIGS["C0"]
+    m, _ = build(s)
+    tok = ki.uniform_tokens(1, s.vocab, 1, 16, DEV)
+    with pytest.raises(kr.KrakenError) as e:
+        m.decode_step(tok[:, 0].contiguous())
+    assert e.value.status == kr.ESTATE
+    with pytest.raises(kr.KrakenError) as e:
+        m.prefill(ki.uniform_tokens(1, s.vocab, 2, 16, DEV))
+    assert e.value.status == kr.ECAPACITY
+    with pytest.raises(kr.KrakenError) as e:
+        m.prefill(ki.uniform_tokens(1, s.vocab, 1, s.max_pos + 1, DEV))
+    assert e.value.status == kr.ECAPACITY
+    bad = tok.clone()
+    bad[0, 3] = s.vocab + 5
+    m.prefill(bad)
+    assert m.device_status() & 1
+    m.reset()
+    assert m.device_status() == 0 and m.cur_len == 0
+    m.prefill(ki.uniform_tokens(1, s.vocab, 1, s.max_pos, DEV))
+    with pytest.raises(kr.KrakenError) as e:
+        m.decode_step(tok[:, 0].contiguous())
+    assert e.value.status == kr.ECAPACITY
+
+
+# ------------------------------------------------------------------ decode
+
+def test_decode_teacher_forced_matches_oracle():
+    s = ki.CONFIGS["C0"]
+    B, l0, steps = 2, 40, 8
+    m, w = build(s, max_batch=B)
+    wb = host_bits(w)
+    tok = ki.uniform_tokens(3, s.vocab, B, l0 + steps, DEV)
+    m.prefill(tok[:, :l0].contiguous())
+    orcs = [oracle.Oracle(s, wb, bf16_store=False) for _ in range(B)]
+    for b in range(B):
+        orcs[b].prefill(tok[b, :l0].cpu().numpy())
+    for t in range(l0, l0 + steps):
+        got = m.decode_step(tok[:, t].contiguous()).cpu().numpy()
+        for b in range(B):
+            ref = orcs[b].decode_step(int(tok[b, t]))
+            rel, mx = logits_metrics(got[b], ref)
+            assert rel <= REL_L2_MAX and mx <= MAX_ABS_MAX, (t, b, rel, mx)
+    assert m.cur_len == l0 + steps
+    # prefill + decode equals one longer prefill at the last position
+    m2, _ = build(s, max_batch=B)
+    longer = m2.prefill(tok).cpu().numpy()
+    rel, mx = logits_metrics(got, longer)
+    assert rel < 5e-3 and mx < 3e-2, (rel, mx)
+    # and the appended cache rows equal the longer prefill's rows
+    for which in (0, 1):
+        a = m.kv_view(s.n_layer - 1, 1, which)[:B, :, :l0 + steps].float()
+        b_ = m2.kv_view(s.n_layer - 1, 1, which)[:B, :, :l0 + steps].float()
+        assert (a - b_).abs().max() <= 2.0 ** -6 * b_.abs().max()
+
+
+# ------------------------------------------------------------------ C1 .. C3 at full size
+
+def test_c1_full_parity():
+    s = ki.CONFIGS["C1"]
+    m, w = build(s)
+    wb = host_bits(w)
+    tok = ki.uniform_tokens(1, s.vocab, s.batch, s.seqlen, DEV)
+    got = m.prefill_all_logits(tok).cpu().numpy()[0]
+    ref32, _ = oracle_all_logits(s, wb, tok[0].cpu().numpy(), False)
+    refbf, _ = oracle_all_logits(s, wb, tok[0].cpu().numpy(), True)
+    check_parity(got, ref32, refbf, "C1 all positions")
+    last = m.prefill(tok).cpu().numpy()
+    assert np.allclose(last[0], got[-1], atol=1e-5)
+
+
+def prefix_parity(name, prefix, seqs):
+    """Full-size run in the launch configuration the benchmark times; by causality the logits and
+    cache rows of the first `prefix` positions equal an oracle run on that prefix alone."""
+    s = ki.CONFIGS[name]
+    m, w = build(s)
+    wb = host_bits(w)
+    tok = ki.uniform_tokens(1, s.vocab, s.batch, s.seqlen, DEV)
+    last = m.prefill(tok)
+    assert torch.isfinite(last).all()
+    assert m.device_status() == 0
+    for b in seqs:
+        rows = [b * s.seqlen + t for t in range(prefix)]
+        got = m.logits_rows(rows).cpu().numpy()
+        ids = tok[b, :prefix].cpu().numpy()
+        ref32, _ = oracle_all_logits(s, wb, ids, False)
+        refbf, orc = oracle_all_logits(s, wb, ids, True)
+        check_parity(got, ref32, refbf, f"{name} seq {b} first {prefix} positions of the full-size run")
+        for layer in (0, s.n_layer // 2, s.n_layer - 1):
+            for n in (0, s.n_branch - 1):
+                for which in (0, 1):
+                    g = m.kv_view(layer, n, which)[b, :, :prefix].float().cpu().numpy()
+                    r = orc.cache(layer, n, which)
+                    ulp = np.abs(g - r) / (np.abs(r) * 2.0 ** -7 + 1e-5)
+                    assert np.quantile(ulp, 0.999) <= 2.0, (layer, n, which, ulp.max())
+    # last-position logits of the timed call equal the row-wise evaluation of the same run
+    again = m.logits_rows([b * s.seqlen + s.seqlen - 1 for b in range(s.batch)])
+    assert torch.allclose(again, last, atol=1e-4)
+    m.close()
+
+
+def test_c2_full_size_prefix_parity():
+    prefix_parity("C2", 128, [0])
+
+
+def test_c3_full_size_prefix_parity():
+    prefix_parity("C3", 32, [0, 3])

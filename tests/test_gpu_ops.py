@@ -1,0 +1,246 @@
+"""Each CUDA kernel of the path, called through the C ABI, against the oracle's matching step."""
+import ctypes as C
+
+import numpy as np
+import pytest
+import torch
+
+import kraken_inputs as ki
+import oracle
+import paper_2408_07802_b200 as kr
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+def bits(t):
+    return ki.bf16_tensor_to_bits(t)
+
+
+def bf16_ulp_close(got: np.ndarray, ref: np.ndarray, ulps=1.0, atol=1e-6):
+    """got (bf16 values as fp32) within `ulps` bf16 steps of ref (fp32)."""
+    tol = ulps * np.abs(ref) * 2.0 ** -7 + atol
+    bad = np.abs(got - ref) > tol
+    return not bad.any(), float(np.max(np.abs(got - ref) - tol))
+
+
+# ------------------------------------------------------------------ embedding
+
+def test_embed_and_bad_token_flag():
+    V, P, d = 300, 50, 128
+    wte = ki.normal_bf16(1, 0, (V, d), 0.5, DEV)
+    wpe = ki.normal_bf16(1, 1, (P, d), 0.5, DEV)
+    ids = ki.uniform_tokens(2, V, 3, 17, DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    out = kr.op_embed(ids.reshape(-1), 17, 5, wte, wpe, status).cpu().numpy()
+    pos = np.tile(np.arange(5, 22), 3)
+    ref = wte.float().cpu().numpy()[ids.cpu().numpy().reshape(-1)] + wpe.float().cpu().numpy()[pos]
+    assert np.array_equal(out, ref)
+    assert int(status.item()) == 0
+    bad = ids.clone().reshape(-1)
+    bad[4] = V
+    bad[9] = -1
+    out2 = kr.op_embed(bad, 17, 5, wte, wpe, status).cpu().numpy()
+    assert int(status.item()) & 1
+    assert np.array_equal(out2[4], wte.float().cpu().numpy()[0] + wpe.float().cpu().numpy()[pos[4]])
+    assert np.array_equal(out2[5], ref[5])
+
+
+# ------------------------------------------------------------------ LayerNorm
+
+@pytest.mark.parametrize("d", [128, 768, 2048, 4096])
+@pytest.mark.parametrize("with_y", [False, True])
+def test_layernorm(d, with_y):
+    G, rows = 3, 37
+    a = (ki.normal_bf16(3, 0, (G, rows, d), 1.0, DEV).float() * 1.7 + 0.3).contiguous()
+    y = ki.normal_bf16(3, 1, (rows, d), 2.0, DEV).float().contiguous() if with_y else None
+    gamma = (1 + ki.normal_bf16(3, 2, (G, d), 0.3, DEV).float()).to(torch.bfloat16)
+    beta = ki.normal_bf16(3, 3, (G, d), 0.3, DEV)
+    out = kr.op_layernorm(a, y, gamma, beta).float().cpu().numpy()
+    for g in range(G):
+        ref = oracle.layernorm(a[g].cpu().numpy(), None if y is None else y.cpu().numpy(), bits(gamma[g]),
+                               bits(beta[g]))
+        ok, worst = bf16_ulp_close(out[g], ref, ulps=1.0, atol=1e-5)
+        assert ok, (g, worst)
+    # one input shared by every group, no beta
+    out2 = kr.op_layernorm(a[0].contiguous(), y, gamma, None, shared_a=True).float().cpu().numpy()
+    ref = oracle.layernorm(a[0].cpu().numpy(), None if y is None else y.cpu().numpy(), bits(gamma[2]), None)
+    ok, worst = bf16_ulp_close(out2[2], ref, ulps=1.0, atol=1e-5)
+    assert ok, worst
+
+
+# ------------------------------------------------------------------ grouped GEMM
+
+def gemm_case(G, M, Nout, K, epi, n_tile, seed=0, integer=False, shared_resid=False):
+    if integer:
+        a = (ki.hash32(seed, 60, 0, G * M * K, DEV) % 5 - 2).to(torch.bfloat16).reshape(G, M, K)
+        w = (ki.hash32(seed, 61, 0, G * Nout * K, DEV) % 5 - 2).to(torch.bfloat16).reshape(G, Nout, K)
+        bias = (ki.hash32(seed, 62, 0, G * Nout, DEV) % 7 - 3).to(torch.bfloat16).reshape(G, Nout)
+    else:
+        a = ki.normal_bf16(seed, 60, (G, M, K), 1.0, DEV)
+        w = ki.normal_bf16(seed, 61, (G, Nout, K), 1.0 / np.sqrt(K), DEV)
+        bias = ki.normal_bf16(seed, 62, (G, Nout), 0.5, DEV)
+    args = kr.GemmArgs()
+    args.a, args.a_gstride, args.lda = a.data_ptr(), M * K, K
+    args.w, args.w_gstride, args.ldw = w.data_ptr(), Nout * K, K
+    args.bias, args.bias_gstride = bias.data_ptr(), Nout
+    args.groups, args.m, args.n_out, args.k = G, M, Nout, K
+    args.epilogue, args.n_tile = epi, n_tile
+    keep = [a, w, bias]
+    out_f32 = out_bf16 = resid = ssum = None
+    if epi in (kr.EPI_F32, kr.EPI_RESID_F32, kr.EPI_RESID_SUM):
+        out_f32 = torch.full((G, M, Nout), float("nan"), dtype=torch.float32, device=DEV)
+        args.out_f32, args.out_f32_gstride, args.ld_out_f32 = out_f32.data_ptr(), M * Nout, Nout
+    if epi in (kr.EPI_BF16, kr.EPI_GELU_BF16):
+        out_bf16 = torch.full((G, M, Nout), float("nan"), dtype=torch.bfloat16, device=DEV)
+        args.out_bf16, args.out_bf16_gstride, args.ld_out_bf16 = out_bf16.data_ptr(), M * Nout, Nout
+    if epi in (kr.EPI_RESID_F32, kr.EPI_RESID_SUM):
+        if integer:
+            resid = (ki.hash32(seed, 63, 0, G * M * Nout, DEV) % 9 - 4).float().reshape(G, M, Nout)
+        else:
+            resid = ki.normal_bf16(seed, 63, (G, M, Nout), 1.0, DEV).float() * 1.37
+        if shared_resid:
+            resid = resid[:1].contiguous()
+        args.resid, args.resid_gstride, args.ld_resid = resid.data_ptr(), 0 if shared_resid else M * Nout, Nout
+    if epi == kr.EPI_RESID_SUM:
+        ssum = torch.full((M, Nout), float("nan"), dtype=torch.float32, device=DEV)
+        args.sum, args.ld_sum = ssum.data_ptr(), Nout
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    kr.op_grouped_gemm(args, status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+
+    # oracle
+    ref = np.stack([oracle.linear(a[g].float().cpu().numpy(), bits(w[g]), bits(bias[g])) for g in range(G)])
+    if resid is not None:
+        r = resid.cpu().numpy()
+        ref = ref + (r if not shared_resid else np.broadcast_to(r, ref.shape))
+    if epi == kr.EPI_GELU_BF16:
+        ref = np.vectorize(lambda t: oracle.gelu(float(t)))(ref).astype(np.float32)
+    return dict(out_f32=None if out_f32 is None else out_f32.cpu().numpy(),
+                out_bf16=None if out_bf16 is None else out_bf16.float().cpu().numpy(),
+                sum=None if ssum is None else ssum.cpu().numpy(), ref=ref, keep=keep)
+
+
+@pytest.mark.parametrize("n_tile", [64, 128, 256])
+def test_gemm_integer_exact_ragged(n_tile):
+    """Small integers make every product and partial sum exact: any mis-placed element shows."""
+    r = gemm_case(2, 300, 200, 136, kr.EPI_F32, n_tile, integer=True)
+    assert np.array_equal(r["out_f32"], r["ref"])
+
+
+@pytest.mark.parametrize("n_tile", [0, 64, 128, 256])
+def test_gemm_f32_many_tiles(n_tile):
+    r = gemm_case(2, 2048, 2304, 768, kr.EPI_F32, n_tile, seed=1)
+    err = np.abs(r["out_f32"] - r["ref"])
+    assert err.max() < 2e-4, err.max()
+
+
+@pytest.mark.parametrize("epi", [kr.EPI_BF16, kr.EPI_GELU_BF16])
+def test_gemm_bf16_epilogues(epi):
+    r = gemm_case(3, 200, 320, 256, epi, 0, seed=2)
+    ok, worst = bf16_ulp_close(r["out_bf16"], r["ref"], ulps=1.0, atol=2e-4)
+    assert ok, worst
+
+
+@pytest.mark.parametrize("shared", [False, True])
+def test_gemm_residual(shared):
+    r = gemm_case(3, 260, 192, 320, kr.EPI_RESID_F32, 0, seed=3, shared_resid=shared)
+    assert np.abs(r["out_f32"] - r["ref"]).max() < 2e-4
+
+
+@pytest.mark.parametrize("n_tile", [64, 128])
+def test_gemm_cross_branch_sum(n_tile):
+    """The AllReduce of Algorithm 1 inside the epilogue: sum equals the explicit sum of the branch outputs."""
+    r = gemm_case(4, 700, 384, 512, kr.EPI_RESID_SUM, n_tile, seed=4)
+    assert np.abs(r["out_f32"] - r["ref"]).max() < 3e-4
+    explicit = r["ref"].astype(np.float64).sum(0)
+    assert np.abs(r["sum"] - explicit).max() < 1e-3
+    # integer case: bit exact, and equal to the sum of the kernel's own branch outputs in order
+    r = gemm_case(4, 300, 256, 128, kr.EPI_RESID_SUM, n_tile, seed=5, integer=True)
+    assert np.array_equal(r["out_f32"], r["ref"])
+    assert np.array_equal(r["sum"], r["ref"].sum(0))
+
+
+@pytest.mark.parametrize("hd,H", [(64, 2), (128, 1)])
+def test_gemm_qkv_scatter_is_index_exact(hd, H):
+    """One-hot activations times integer-coded weights: every cache element names its source."""
+    d = H * hd
+    G, batch, seqlen, pos0, P, K = 2, 3, 50, 7, 64, 64
+    M = batch * seqlen
+    t = torch.arange(M, device=DEV)
+    a = torch.zeros(G, M, K, dtype=torch.bfloat16, device=DEV)
+    a[:, t, t % K] = 1.0
+    o = torch.arange(3 * d, device=DEV)[:, None]
+    k = torch.arange(K, device=DEV)[None, :]
+    w = torch.stack([((o * 7 + k * 13 + g * 29) % 251 - 125) for g in range(G)]).to(torch.bfloat16).contiguous()
+    qbuf = torch.zeros(G, M, d, dtype=torch.bfloat16, device=DEV)
+    cache = torch.full((G, 2, batch, H, P, hd), -7.0, dtype=torch.bfloat16, device=DEV)
+    args = kr.GemmArgs()
+    args.a, args.a_gstride, args.lda = a.data_ptr(), M * K, K
+    args.w, args.w_gstride, args.ldw = w.data_ptr(), 3 * d * K, K
+    args.groups, args.m, args.n_out, args.k = G, M, 3 * d, K
+    args.epilogue = kr.EPI_QKV
+    args.out_bf16, args.out_bf16_gstride, args.ld_out_bf16 = qbuf.data_ptr(), M * d, d
+    args.k_cache, args.v_cache = cache[0, 0].data_ptr(), cache[0, 1].data_ptr()
+    args.cache_gstride = cache.stride(0)
+    args.seqlen, args.pos0, args.n_head, args.head_dim, args.max_pos = seqlen, pos0, H, hd, P
+    kr.op_grouped_gemm(args)
+    torch.cuda.synchronize()
+    wf = w.float().cpu().numpy()
+    got_q, got_c = qbuf.float().cpu().numpy(), cache.float().cpu().numpy()
+    tk = np.arange(M) % K
+    for g in range(G):
+        assert np.array_equal(got_q[g], wf[g][:d, tk].T)
+        for which in (0, 1):
+            for b in range(batch):
+                for h in range(H):
+                    rows = wf[g][d * (1 + which) + h * hd: d * (1 + which) + (h + 1) * hd]  # [hd, K]
+                    want = rows[:, tk[b * seqlen:(b + 1) * seqlen]].T                          # [seqlen, hd]
+                    assert np.array_equal(got_c[g, which, b, h, pos0:pos0 + seqlen], want)
+                    # rows outside the written range are untouched
+                    assert np.all(got_c[g, which, b, h, :pos0] == -7.0)
+                    assert np.all(got_c[g, which, b, h, pos0 + seqlen:] == -7.0)
+
+
+def test_gemm_rejects_unaligned():
+    a = torch.zeros(1, 8, 68, dtype=torch.bfloat16, device=DEV)
+    args = kr.GemmArgs()
+    args.a, args.lda, args.w, args.ldw = a.data_ptr(), 68, a.data_ptr(), 68
+    args.groups, args.m, args.n_out, args.k = 1, 8, 8, 68
+    args.epilogue = kr.EPI_F32
+    out = torch.zeros(8, 8, device=DEV)
+    args.out_f32, args.ld_out_f32 = out.data_ptr(), 8
+    with pytest.raises(kr.KrakenError) as e:
+        kr.op_grouped_gemm(args)
+    assert e.value.status == kr.EUNSUPPORTED
+
+
+# ------------------------------------------------------------------ attention
+
+@pytest.mark.parametrize("hd", [64, 128])
+@pytest.mark.parametrize("seqlen,pos0", [(200, 0), (100, 37), (1, 90), (64, 0)])
+def test_attention_matches_oracle(hd, seqlen, pos0):
+    G, B, H, P = 2, 2, 2, 256
+    d = H * hd
+    q = ki.normal_bf16(7, 0, (G, B * seqlen, d), 1.0, DEV)
+    kc = ki.normal_bf16(7, 1, (G, B, H, P, hd), 1.0, DEV)
+    vc = ki.normal_bf16(7, 2, (G, B, H, P, hd), 1.0, DEV)
+    # rows past the sequence hold garbage that must not leak (NaN would poison a masked product)
+    kc[:, :, :, pos0 + seqlen:] = float("nan")
+    vc[:, :, :, pos0 + seqlen:] = float("nan")
+    out = kr.op_attention(q, kc, vc, B, seqlen, pos0, H).float().cpu().numpy()
+    assert not np.isnan(out).any()
+    qn, kn, vn = q.float().cpu().numpy(), kc.float().cpu().numpy(), vc.float().cpu().numpy()
+    worst, num, den = 0.0, 0.0, 0.0
+    for g in range(G):
+        for b in range(B):
+            for h in range(H):
+                ref = oracle.attention_head(qn[g, b * seqlen:(b + 1) * seqlen, h * hd:(h + 1) * hd],
+                                            kn[g, b, h, :pos0 + seqlen], vn[g, b, h, :pos0 + seqlen], q_pos0=pos0)
+                got = out[g, b * seqlen:(b + 1) * seqlen, h * hd:(h + 1) * hd]
+                worst = max(worst, np.abs(got - ref).max())
+                num += ((got - ref) ** 2).sum()
+                den += (ref ** 2).sum()
+    assert worst < 3e-2, worst
+    assert np.sqrt(num / den) < 6e-3, np.sqrt(num / den)
