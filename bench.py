@@ -1,0 +1,330 @@
+#!/usr/bin/env python
+"""Benchmark of the single-GPU Kraken prefill path (and of the CPU oracle as the reference arm).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload C3] [--impl ours|reference]
+
+One step = one whole prefill (embedding, L layers of N branches, W_concat, final LayerNorm,
+unembedding of the last positions) over one batch of seeded synthetic tokens.  Rank 0 prints ONE
+JSON line.  With N > 1 (torchrun) every rank runs an independent replica on its own GPU
+("replicas only": the path has no inter-GPU step), timed between barriers, max over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+PAPER_CONTEXT = ("paper: 35.6% geomean TTFT speedup of Kraken over standard Transformers, TensorRT-LLM fp16 on "
+                 "8xA100-40GB NVSwitch (another machine and other shapes: context, not a target)")
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            d = json.load(open(p))
+            return {k: float(d[k]) for k in FALLBACK_PEAKS}, "measured"
+        except Exception:
+            pass
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples of one GPU while a region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.proc = index, None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if not self.proc:
+            return out
+        self.proc.terminate()
+        try:
+            text, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            text = ""
+        sm, mx, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for line in text.splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+def host_weight_bits(w):
+    import kraken_inputs as ki
+    return {k: (None if v is None else ki.bf16_tensor_to_bits(v)) for k, v in w.items()}
+
+
+def oracle_tokens_per_s(shape, wb, ids, n_tokens):
+    """Oracle prefill of the first n_tokens of one sequence (last-position logits only)."""
+    import oracle
+    orc = oracle.Oracle(shape, wb)
+    t0 = time.perf_counter()
+    orc.prefill(ids[:n_tokens], logits_from=n_tokens - 1)
+    dt = time.perf_counter() - t0
+    orc.close()
+    return n_tokens / dt, dt
+
+
+def run_reference(args, shape):
+    """Reference arm: the CPU oracle, as it stands, on a bounded sample of the same workload."""
+    import torch
+    import kraken_inputs as ki
+    import oracle
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    dev = "cuda:0" if torch.cuda.is_available() else "cpu"
+    w = ki.make_weights(shape, seed=0, device=dev)
+    wb = host_weight_bits(w)
+    del w
+    ids = ki.uniform_tokens(1, shape.vocab, shape.batch, shape.seqlen)[0].numpy()
+    n = max(1, min(shape.seqlen, args.ref_tokens))
+    for _ in range(args.warmup):
+        oracle_tokens_per_s(shape, wb, ids, n)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_tokens_per_s(shape, wb, ids, n)
+    dt = (time.perf_counter() - t0) / args.steps
+    value = n / dt
+    sample = f"oracle prefill of the first {n} tokens of sequence 0 of {shape.name} per step"
+    line = {
+        "impl": "reference", "metric": "prefill_tokens_per_s", "value": value, "unit": "tokens/s",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32 values, f64 accumulation",
+        "data": "synthetic", "config": workload_config(shape, args),
+        "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": oracle.num_threads(), "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def workload_config(shape, args):
+    return {"workload": f"{shape.name} prefill", "n_branch": shape.n_branch, "n_layer": shape.n_layer,
+            "d_model": shape.d_model, "n_head": shape.n_head, "d_ff": shape.d_ff, "vocab": shape.vocab,
+            "batch": shape.batch, "seqlen": shape.seqlen, "tokens_per_step": shape.batch * shape.seqlen,
+            "parallelism": f"replicas x{args.gpus}" if args.gpus > 1 else "single GPU",
+            "l2": "inputs larger than L2 (weights read every step exceed 126 MB)"
+                  if weight_bytes(shape) > 126e6 else "L2 flushed between steps",
+            "context": PAPER_CONTEXT}
+
+
+def weight_bytes(s):
+    return 2 * (s.n_layer * s.n_branch * (4 * s.d_model ** 2 + 2 * s.d_model * s.d_ff) + s.vocab * s.d_model)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="C3")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--ref-tokens", type=int, default=8, help="tokens per step of the reference arm")
+    ap.add_argument("--cpu-baseline-seconds", type=float, default=15.0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+
+    import kraken_inputs as ki
+    shape = ki.CONFIGS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, shape)
+        return
+
+    import torch
+    import paper_2408_07802_b200 as kr
+    from paper_2408_07802_b200 import build as kbuild
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = f"cuda:{local_rank}"
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+    if rank == 0:
+        kbuild.build()
+    if dist:
+        dist.barrier()
+    kr.lib()
+
+    w = ki.make_weights(shape, seed=0, device=dev)
+    model = kr.KrakenModel(kr.make_config(shape), w, dev)
+    tok = ki.uniform_tokens(1 + rank, shape.vocab, shape.batch, shape.seqlen, dev)
+    logits = torch.empty(shape.batch, shape.vocab, dtype=torch.float32, device=dev)
+    flush = None
+    if weight_bytes(shape) <= 126e6:
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+
+    def step():
+        if flush is not None:
+            flush.zero_()
+        model.prefill(tok, logits)
+
+    def barrier():
+        if dist:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    model.profile_read()  # reset the launch counters
+
+    # ---- timed region: K steps, device time by events on the launching stream
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    time.sleep(0.25)
+    e0 = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    e1 = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+    barrier()
+    for i in range(args.steps):
+        if flush is not None:
+            flush.zero_()
+        e0[i].record()
+        model.prefill(tok, logits)
+        e1[i].record()
+    barrier()
+    clocks = sampler.stop()
+    per_step = [a.elapsed_time(b) for a, b in zip(e0, e1)]
+    total_ms = sum(per_step)
+    _, launches = model.profile_read()
+    gpu_launches = int(sum(launches.values()))
+    if dist:
+        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    tokens = shape.batch * shape.seqlen
+    value = world * tokens / (ms_per_step * 1e-3)
+
+    # ---- the same K steps again with every launch bracketed by events: per-kernel device time
+    model.profile_enable(True)
+    for _ in range(args.steps):
+        step()
+    prof_ms, prof_n = model.profile_read()
+    model.profile_enable(False)
+
+    # ---- end to end through the host-buffer call: pinned tokens in, logits out, every step
+    h_tok = tok.cpu().pin_memory()
+    h_log = torch.empty(shape.batch, shape.vocab, dtype=torch.float32).pin_memory()
+    for _ in range(2):
+        model.prefill_host(h_tok, h_log)
+    barrier()
+    t0 = time.perf_counter()
+    s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    s0.record()
+    for _ in range(args.steps):
+        if flush is not None:
+            flush.zero_()
+        model.prefill_host(h_tok, h_log)
+    s1.record()
+    barrier()
+    e2e_ms = s0.elapsed_time(s1) / args.steps
+    if dist:
+        t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+    e2e_value = world * tokens / (e2e_ms * 1e-3)
+    status = model.device_status()
+
+    if rank != 0:
+        if dist:
+            dist.destroy_process_group()
+        return
+
+    peaks, peak_kind = load_peaks()
+    fl = ki.algorithmic_flops(shape)
+    gemm_ms = sum(prof_ms[k] for k in ("gemm_qkv", "gemm_proj", "gemm_up", "gemm_down")) / args.steps
+    gemm_launches = sum(prof_n[k] for k in ("gemm_qkv", "gemm_proj", "gemm_up", "gemm_down")) // args.steps
+    achieved = fl["gemm"] / (gemm_ms * 1e-3) / 1e12 if gemm_ms > 0 else 0.0
+    peak = peaks["bf16_tflops_sustained"]
+    T, N, L, d, F = tokens, shape.n_branch, shape.n_layer, shape.d_model, shape.d_ff
+    kind_flops = {"gemm_qkv": 2.0 * T * N * L * 3 * d * d, "gemm_proj": 2.0 * T * N * L * d * d,
+                  "gemm_up": 2.0 * T * N * L * d * F, "gemm_down": 2.0 * T * N * L * d * F,
+                  "attention": fl["attn"]}
+    kernels = {}
+    for k, ms in prof_ms.items():
+        ent = {"ms_per_step": ms / args.steps, "launches_per_step": prof_n[k] // args.steps}
+        if k in kind_flops and ms > 0:
+            ent["tflops"] = kind_flops[k] / (ms / args.steps * 1e-3) / 1e12
+        kernels[k] = ent
+    line = {
+        "metric": "prefill_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": world,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_per_step, "ttft_ms": ms_per_step,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic", "config": workload_config(shape, args),
+        "model_tflops": fl["total"] / (ms_per_step * 1e-3) / 1e12,
+        "frac_of_nominal_2250": fl["total"] / (ms_per_step * 1e-3) / 2.25e15,
+        "frac_of_measured_sustained": fl["total"] / (ms_per_step * 1e-3) / 1e12 / peak,
+        "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": "tokens/s", "ms_per_step": e2e_ms,
+                "h2d_bytes_per_step": tokens * 4, "d2h_bytes_per_step": shape.batch * shape.vocab * 4},
+        "gpu_launches": gpu_launches,
+        "roofline": {"bound": "tensor", "kernel": "gemm_tc_kernel (grouped tcgen05 GEMM: qkv, proj, up, down)",
+                     "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
+                     "peak_source": f"bf16_tflops_sustained of {peak_kind}",
+                     "launches_per_step": int(gemm_launches), "avg_launch_ms": gemm_ms / max(1, gemm_launches),
+                     "flops_per_step": fl["gemm"], "timed_in": "separate pass of the same K steps with events "
+                     "around every launch", "traffic": None},
+        "kernels": kernels,
+        "device_status": status,
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        import oracle
+        wb = host_weight_bits(w)
+        ids = tok[0].cpu().numpy()
+        probe_n = min(shape.seqlen, 4)
+        rate, _ = oracle_tokens_per_s(shape, wb, ids, probe_n)
+        n = int(max(probe_n, min(shape.seqlen, rate * args.cpu_baseline_seconds)))
+        rate, dt = oracle_tokens_per_s(shape, wb, ids, n)
+        line["cpu_baseline"] = {"value": rate, "unit": "tokens/s", "cores": oracle.num_threads(), "kind": "oracle",
+                                "sample": f"oracle prefill of the first {n} tokens of sequence 0 ({dt:.1f} s)"}
+    print(json.dumps(line))
+    if dist:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
