@@ -152,17 +152,17 @@ __global__ void __launch_bounds__(128) attn_prefill_kernel(const AttnParams p) {
             mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xFFFFFFFFu, mx[r], 1));
             mx[r] = fmaxf(mx[r], __shfl_xor_sync(0xFFFFFFFFu, mx[r], 2));
             const float m_new = fmaxf(m_i[r], mx[r]);  // finite: key 0 is visible to every row
-            corr[r] = exp2f((m_i[r] - m_new) * sl2);
+            corr[r] = ex2_approx((m_i[r] - m_new) * sl2);
             m_i[r] = m_new;
             mscaled[r] = m_new * sl2;
         }
         float rs[2] = {0.f, 0.f};
 #pragma unroll
         for (int nt = 0; nt < ABN / 8; ++nt) {
-            s[nt][0] = exp2f(s[nt][0] * sl2 - mscaled[0]);
-            s[nt][1] = exp2f(s[nt][1] * sl2 - mscaled[0]);
-            s[nt][2] = exp2f(s[nt][2] * sl2 - mscaled[1]);
-            s[nt][3] = exp2f(s[nt][3] * sl2 - mscaled[1]);
+            s[nt][0] = ex2_approx(s[nt][0] * sl2 - mscaled[0]);
+            s[nt][1] = ex2_approx(s[nt][1] * sl2 - mscaled[0]);
+            s[nt][2] = ex2_approx(s[nt][2] * sl2 - mscaled[1]);
+            s[nt][3] = ex2_approx(s[nt][3] * sl2 - mscaled[1]);
             rs[0] += s[nt][0] + s[nt][1];
             rs[1] += s[nt][2] + s[nt][3];
         }

@@ -50,7 +50,8 @@ layernorm_kernel(const float *__restrict__ a, long long a_gstride, const float *
     const long long wr = (long long)blockIdx.x * ROW_WARPS + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (wr >= (long long)groups * rows) return;
-    const int g = static_cast<int>(wr / rows), r = static_cast<int>(wr % rows);
+    // neighbouring warps take the groups of one row, so the shared y row is fetched from DRAM once
+    const int r = static_cast<int>(wr / groups), g = static_cast<int>(wr % groups);
     const float4 *pa = reinterpret_cast<const float4 *>(a + g * a_gstride + (size_t)r * d);
     const float4 *py = y ? reinterpret_cast<const float4 *>(y + (size_t)r * d) : nullptr;
     const int nvec = d / 4;

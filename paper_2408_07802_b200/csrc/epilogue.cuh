@@ -5,12 +5,26 @@
 
 namespace kr {
 
+// erf by the rational-times-Gaussian form 1 - (a1 t + ... + a5 t^5) exp(-z^2), t = 1 / (1 + p z)
+// (Abramowitz & Stegun 7.1.26, |error| <= 1.5e-7): branch-free, two special-function-unit ops.
+__device__ __forceinline__ float erf_as(float z) {
+    const float az = fabsf(z);
+    const float t = rcp_approx(fmaf(0.3275911f, az, 1.0f));
+    float poly = fmaf(1.061405429f, t, -1.453152027f);
+    poly = fmaf(poly, t, 1.421413741f);
+    poly = fmaf(poly, t, -0.284496736f);
+    poly = fmaf(poly, t, 0.254829592f);
+    poly *= t;
+    const float e = ex2_approx(-1.4426950408889634f * az * az);
+    return copysignf(fmaf(-poly, e, 1.0f), z);
+}
+
 __device__ __forceinline__ float gelu_f(float x, int tanh_form) {
     if (tanh_form) {
         const float c = 0.7978845608028654f;
         return 0.5f * x * (1.0f + tanhf(c * (x + 0.044715f * x * x * x)));
     }
-    return 0.5f * x * (1.0f + erff(x * 0.7071067811865476f));
+    return 0.5f * x * (1.0f + erf_as(x * 0.7071067811865476f));
 }
 
 __device__ __forceinline__ void store_bf16_chunk(uint16_t *dst, const float (&v)[32], int ncols) {

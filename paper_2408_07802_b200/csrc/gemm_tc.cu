@@ -5,12 +5,16 @@
 //   warp 1    allocates TMEM and issues tcgen05.mma (128 x BN x 16 per instruction, fp32
 //             accumulators in TMEM, two accumulator buffers so that draining tile i overlaps
 //             the MMAs of tile i+1);
-//   warps 2-5 epilogue: tcgen05.ld of their 32-lane quarter, fused epilogue, global stores.
+//   warps 2-9 epilogue: tcgen05.ld of their 32-lane quarter (two warps per quarter, each one half
+//             of the tile's columns), fused epilogue, global stores.
 // The group (branch) index is the outermost TMA coordinate.  Rows past M, columns past Nout
 // and the K tail are zero-filled by TMA and masked in the epilogue.
 //
-// The down-projection's cross-branch sum (the AllReduce of Algorithm 1) needs the N groups
-// of one output tile on the same CTA in ascending order: `group_serial` scheduling.
+// Tile order: the group is the slowest index, so the operands of one group (tens of MB) stay
+// in L2 while its tiles are walked.  The down-projection's cross-branch sum (the AllReduce of
+// Algorithm 1) instead needs the N groups of one output tile on the same CTA in ascending order
+// (`group_serial`); there the dimension with fewer tiles runs fastest so that one wave of CTAs
+// spans it completely and shares those operand tiles through L2.
 #include <stdio.h>
 #include <stdlib.h>
 
@@ -25,7 +29,8 @@ namespace {
 constexpr int BM = 128;
 constexpr int BK = 64;
 constexpr int UMMA_K = 16;
-constexpr int NUM_THREADS = 192;
+constexpr int EPI_WARPS = 8;
+constexpr int NUM_THREADS = 64 + 32 * EPI_WARPS;
 constexpr int SMEM_BUDGET = 200 * 1024;
 
 template <int BN>
@@ -45,6 +50,7 @@ struct KernelArgs {
     int a_gmul, b_gmul;  // 0 when the operand is shared by all groups
     int a_g0, b_g0;      // first group's index along the outermost TMA dimension
     int group_serial;
+    int n_fastest;  // tile order inside a group: 1 = n-tiles fastest, 0 = m-tiles fastest
     uint32_t *status;
 };
 
@@ -57,12 +63,18 @@ __device__ __forceinline__ bool next_item(const KernelArgs &ka, int it, int &m_b
         g = it % G;
     } else {
         const long long idx = blockIdx.x + (long long)it * gridDim.x;
-        tile = static_cast<int>(idx / G);
-        g = static_cast<int>(idx % G);
+        g = static_cast<int>(idx / num_tiles);
+        if (g >= G) return false;
+        tile = static_cast<int>(idx % num_tiles);
     }
     if (tile >= num_tiles) return false;
-    m_blk = tile % ka.tiles_m;  // m fastest: one wave shares few W tiles, A stays in L2
-    n_blk = tile / ka.tiles_m;
+    if (ka.n_fastest) {
+        n_blk = tile % ka.tiles_n;
+        m_blk = tile / ka.tiles_n;
+    } else {
+        m_blk = tile % ka.tiles_m;
+        n_blk = tile / ka.tiles_m;
+    }
     return true;
 }
 
@@ -92,7 +104,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(acc_full + a, 1);
-            mbar_init(acc_empty + a, 4);
+            mbar_init(acc_empty + a, EPI_WARPS);
         }
         *abort_flag = 0;
         fence_barrier_init();
@@ -169,7 +181,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         }
         __syncwarp();
     } else {
-        const int quarter = warp & 3;  // TMEM lanes this warp may read
+        const int quarter = warp & 3;          // TMEM lanes this warp may read
+        const int half = (warp - 2) >> 2;      // which half of the tile's columns it drains
+        constexpr int CHUNKS = BN / 32 / 2;    // 32-column chunks per warp
         int acc = 0;
         uint32_t acc_phase = 0;
         bool ok = true;
@@ -183,7 +197,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
                                    static_cast<uint32_t>(acc * BN);
 #pragma unroll 1
-            for (int c = 0; c < BN / 32; ++c) {
+            for (int cc = 0; cc < CHUNKS; ++cc) {
+                const int c = half * CHUNKS + cc;
                 const int col0 = n_blk * BN + c * 32;
                 if (col0 >= ka.shape.n_out) break;  // uniform across the warp
                 uint32_t r[32];
@@ -285,6 +300,7 @@ int launch_gemm_tc(const GemmOperands &op, const GemmShape &s, const EpiParams &
     ka.a_g0 = 0;
     ka.b_g0 = b_g0;
     ka.group_serial = epi.kind == KRAKEN_EPI_RESID_SUM ? 1 : 0;
+    ka.n_fastest = (ka.group_serial && ka.tiles_n <= ka.tiles_m) ? 1 : 0;
     ka.status = d_status;
     const long long tiles = (long long)ka.tiles_m * ka.tiles_n;
     const long long units = ka.group_serial ? tiles : tiles * s.groups;
