@@ -172,17 +172,15 @@ def main():
     import paper_2408_07802_b200 as kr
     from paper_2408_07802_b200 import build as kbuild
 
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
+    from paper_2408_07802_b200 import replicas
+    rank, local_rank, world = replicas.rank_env()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
     torch.cuda.set_device(local_rank)
     dev = f"cuda:{local_rank}"
     dist = None
     if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device(dev))
+        dist = replicas.init_process_group("nccl", torch.device(dev))
     if rank == 0:
         kbuild.build()
     if dist:
@@ -191,7 +189,7 @@ def main():
 
     w = ki.make_weights(shape, seed=0, device=dev)
     model = kr.KrakenModel(kr.make_config(shape), w, dev)
-    tok = ki.uniform_tokens(1 + rank, shape.vocab, shape.batch, shape.seqlen, dev)
+    tok = ki.uniform_tokens(replicas.token_seed(rank), shape.vocab, shape.batch, shape.seqlen, dev)
     logits = torch.empty(shape.batch, shape.vocab, dtype=torch.float32, device=dev)
     flush = None
     if weight_bytes(shape) <= 126e6:
@@ -203,8 +201,7 @@ def main():
         model.prefill(tok, logits)
 
     def barrier():
-        if dist:
-            dist.barrier()
+        replicas.barrier()
         torch.cuda.synchronize()
 
     for _ in range(args.warmup):
@@ -231,13 +228,10 @@ def main():
     total_ms = sum(per_step)
     _, launches = model.profile_read()
     gpu_launches = int(sum(launches.values()))
-    if dist:
-        t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = replicas.max_over_ranks(total_ms, dev)
     ms_per_step = total_ms / args.steps
     tokens = shape.batch * shape.seqlen
-    value = world * tokens / (ms_per_step * 1e-3)
+    value = replicas.whole_job_throughput(tokens, ms_per_step, world)
 
     # ---- the same K steps again with every launch bracketed by events: per-kernel device time
     model.profile_enable(True)
@@ -252,7 +246,6 @@ def main():
     for _ in range(2):
         model.prefill_host(h_tok, h_log)
     barrier()
-    t0 = time.perf_counter()
     s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     s0.record()
     for _ in range(args.steps):
@@ -262,11 +255,8 @@ def main():
     s1.record()
     barrier()
     e2e_ms = s0.elapsed_time(s1) / args.steps
-    if dist:
-        t = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
-    e2e_value = world * tokens / (e2e_ms * 1e-3)
+    e2e_ms = replicas.max_over_ranks(e2e_ms, dev)
+    e2e_value = replicas.whole_job_throughput(tokens, e2e_ms, world)
     status = model.device_status()
 
     if rank != 0:
