@@ -136,7 +136,8 @@ def run_reference(args, shape):
 
 
 def workload_config(shape, args):
-    return {"workload": f"{shape.name} prefill", "n_branch": shape.n_branch, "n_layer": shape.n_layer,
+    what = "decode after prefill" if shape.decode_steps else "prefill"
+    return {"workload": f"{shape.name} {what}", "n_branch": shape.n_branch, "n_layer": shape.n_layer,
             "d_model": shape.d_model, "n_head": shape.n_head, "d_ff": shape.d_ff, "vocab": shape.vocab,
             "batch": shape.batch, "seqlen": shape.seqlen, "tokens_per_step": shape.batch * shape.seqlen,
             "parallelism": f"replicas x{args.gpus}" if args.gpus > 1 else "single GPU",
@@ -147,6 +148,137 @@ def workload_config(shape, args):
 
 def weight_bytes(s):
     return 2 * (s.n_layer * s.n_branch * (4 * s.d_model ** 2 + 2 * s.d_model * s.d_ff) + s.vocab * s.d_model)
+
+
+def decode_bytes(shape, t):
+    """Bytes one decode step must move at cache length t: every weight once, K and V rows 0..t."""
+    s = shape
+    w = 2 * (s.n_layer * s.n_branch * (4 * s.d_model ** 2 + 2 * s.d_model * s.d_ff) + s.vocab * s.d_model
+             + s.n_branch * s.d_model ** 2)
+    kv = 2 * s.n_layer * s.n_branch * s.batch * (t + 1) * s.d_model * 2
+    return w, kv
+
+
+def run_decode(args, shape, kr, ki, replicas, torch):
+    """C4: prefill `seqlen` tokens per sequence, then time greedy decode steps (one step = one
+    kraken_decode_step over the whole batch; the arg-max feeding the next step is the caller's)."""
+    rank, local_rank, world = replicas.rank_env()
+    dev = f"cuda:{local_rank}"
+    steps = min(args.steps, shape.decode_steps)
+    w = ki.make_weights(shape, seed=0, device=dev)
+    model = kr.KrakenModel(kr.make_config(shape), w, dev)
+    tok = ki.uniform_tokens(replicas.token_seed(rank), shape.vocab, shape.batch, shape.seqlen, dev)
+    logits = torch.empty(shape.batch, shape.vocab, dtype=torch.float32, device=dev)
+
+    def barrier():
+        replicas.barrier()
+        torch.cuda.synchronize()
+
+    def start():
+        model.prefill(tok, logits)
+        return logits.argmax(1).to(torch.int32)
+
+    nxt = start()
+    for _ in range(max(args.warmup, 3)):
+        model.decode_step(nxt, logits)
+        nxt = logits.argmax(1).to(torch.int32)
+    nxt = start()
+    barrier()
+    model.profile_read()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    time.sleep(0.25)
+    e0 = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+    e1 = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+    barrier()
+    for i in range(steps):
+        e0[i].record()
+        model.decode_step(nxt, logits)
+        e1[i].record()
+        nxt = logits.argmax(1).to(torch.int32)
+    barrier()
+    clocks = sampler.stop()
+    per_step = [a.elapsed_time(b) for a, b in zip(e0, e1)]
+    _, launches = model.profile_read()
+    ms_per_step = replicas.max_over_ranks(sum(per_step), dev) / steps
+    value = replicas.whole_job_throughput(shape.batch, ms_per_step, world)
+
+    # per-kernel device time: the same steps again from the same start, events around every launch
+    nxt = start()
+    model.profile_read()
+    model.profile_enable(True)
+    for _ in range(steps):
+        model.decode_step(nxt, logits)
+        nxt = logits.argmax(1).to(torch.int32)
+    prof_ms, prof_n = model.profile_read()
+    model.profile_enable(False)
+
+    # end to end: host token ids in, host logits out, every step
+    nxt = start()
+    h_tok = nxt.cpu().pin_memory()
+    h_log = torch.empty(shape.batch, shape.vocab, dtype=torch.float32).pin_memory()
+    barrier()
+    s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    s0.record()
+    for _ in range(steps):
+        model.decode_step_host(h_tok, h_log)
+        h_tok.copy_(h_log.argmax(1).to(torch.int32))
+    s1.record()
+    barrier()
+    e2e_ms = replicas.max_over_ranks(s0.elapsed_time(s1), dev) / steps
+    status = model.device_status()
+    if rank != 0:
+        return
+
+    peaks, peak_kind = load_peaks()
+    t_mid = shape.seqlen + steps // 2
+    wb_, kvb = decode_bytes(shape, t_mid)
+    total_bytes = wb_ + kvb
+    attn_ms = prof_ms["attention"] / steps
+    attn_launch = prof_n["attention"] / steps
+    kv_per_layer = kvb / shape.n_layer
+    attn_gbs = kvb / (attn_ms * 1e-3) / 1e9 if attn_ms > 0 else 0.0
+    kernels = {k: {"ms_per_step": v / steps, "launches_per_step": prof_n[k] / steps} for k, v in prof_ms.items()}
+    gemm_ms = sum(prof_ms[k] for k in ("gemm_qkv", "gemm_proj", "gemm_up", "gemm_down", "tail")) / steps
+    line = {
+        "metric": "decode_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": world, "steps": steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": workload_config(shape, args),
+        "hbm_gbs": total_bytes / (ms_per_step * 1e-3) / 1e9,
+        "frac_of_measured_hbm": total_bytes / (ms_per_step * 1e-3) / 1e9 / peaks["hbm_gbs"],
+        "bytes_per_step": {"weights": wb_, "kv_cache": kvb, "at_cache_length": t_mid},
+        "clocks": clocks,
+        "e2e": {"value": replicas.whole_job_throughput(shape.batch, e2e_ms, world), "unit": "tokens/s",
+                "ms_per_step": e2e_ms, "h2d_bytes_per_step": shape.batch * 4,
+                "d2h_bytes_per_step": shape.batch * shape.vocab * 4},
+        "gpu_launches": int(sum(launches.values())),
+        "roofline": {"bound": "hbm", "kernel": "attn_decode_kernel (split-KV cache streaming)",
+                     "achieved": attn_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                     "frac": attn_gbs / peaks["hbm_gbs"], "peak_source": f"hbm_gbs of {peak_kind}",
+                     "bytes_per_launch": kv_per_layer, "launches_per_step": attn_launch,
+                     "avg_launch_ms": attn_ms / shape.n_layer,
+                     "timed_in": "separate pass of the same steps with events around every launch",
+                     "traffic": None},
+        "weight_streaming": {"ms_per_step": gemm_ms, "gbs": wb_ / (gemm_ms * 1e-3) / 1e9 if gemm_ms > 0 else 0.0},
+        "kernels": kernels, "device_status": status,
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        import oracle
+        hb = host_weight_bits(w)
+        ctx, n_dec = 256, 8
+        orc = oracle.Oracle(shape, hb)
+        ids = tok[0].cpu().numpy()
+        orc.prefill(ids[:ctx], logits_from=ctx - 1)
+        t0 = time.perf_counter()
+        nid = int(ids[ctx])
+        for _ in range(n_dec):
+            nid = int(orc.decode_step(nid).argmax())
+        dt = time.perf_counter() - t0
+        line["cpu_baseline"] = {"value": n_dec / dt, "unit": "tokens/s", "cores": oracle.num_threads(),
+                                "kind": "oracle", "sample": f"{n_dec} oracle decode steps of ONE sequence after a "
+                                f"{ctx}-token prefill ({dt:.1f} s); the GPU figure is {shape.batch} sequences at "
+                                f"context {shape.seqlen}"}
+    print(json.dumps(line))
 
 
 def main():
@@ -186,6 +318,13 @@ def main():
     if dist:
         dist.barrier()
     kr.lib()
+    if shape.decode_steps:
+        if args.steps == 10:
+            args.steps = shape.decode_steps
+        run_decode(args, shape, kr, ki, replicas, torch)
+        if dist:
+            dist.destroy_process_group()
+        return
 
     w = ki.make_weights(shape, seed=0, device=dev)
     model = kr.KrakenModel(kr.make_config(shape), w, dev)

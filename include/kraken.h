@@ -121,6 +121,9 @@ int kraken_logits_rows(kraken_handle *h, const int32_t *h_rows, int32_t n_rows, 
  * Errors: ESTATE (no prefill, or batch differs from the prefill's), ECAPACITY (cur_len == max_pos). */
 int kraken_decode_step(kraken_handle *h, const int32_t *d_tokens, int32_t batch, float *d_logits, void *stream);
 
+/* Same with HOST buffers (h_tokens [batch], h_logits [batch, V]); synchronises the stream. */
+int kraken_decode_step_host(kraken_handle *h, const int32_t *h_tokens, int32_t batch, float *h_logits, void *stream);
+
 /* Where the cache of (layer, branch, which: 0 = K, 1 = V) lives: base device pointer and
  * strides in ELEMENTS for (batch, head, position, dim). */
 int kraken_kv_view(kraken_handle *h, int32_t layer, int32_t branch, int32_t which, const void **ptr,
@@ -219,6 +222,23 @@ int kraken_op_attention(const void *q, int64_t q_gstride, const void *k_cache, c
                         int64_t cache_gstride, int64_t cache_bstride, int32_t groups, int32_t batch,
                         int32_t seqlen, int32_t pos0, int32_t n_head, int32_t head_dim, int32_t max_pos,
                         void *out, int64_t out_gstride, void *stream);
+
+/* Decode-step attention (Sec. 2.1: the decode step reads the whole KV cache): one query row per
+ * (group, sequence, head) at position n_keys - 1 against cache rows 0..n_keys-1.  The keys are split
+ * over `splits` CTAs per (group, sequence, head); each split leaves an unnormalised partial in
+ * d_partials (device scratch, fp32 [groups*batch*n_head][splits][head_dim + 2]) and a second kernel
+ * merges them.  splits = 0 lets the library choose; splits = 1 needs no scratch (d_partials may be NULL).
+ * q, out: bf16 [G][batch, n_head*head_dim].  Errors: EINVAL, EUNSUPPORTED (head_dim), ECAPACITY
+ * (partial_bytes too small). */
+int kraken_op_decode_attention(const void *q, int64_t q_gstride, const void *k_cache, const void *v_cache,
+                               int64_t cache_gstride, int64_t cache_bstride, int32_t groups, int32_t batch,
+                               int32_t n_keys, int32_t n_head, int32_t head_dim, int32_t max_pos, int32_t splits,
+                               void *d_partials, size_t partial_bytes, void *out, int64_t out_gstride, void *stream);
+
+/* Split count the library would choose (when *splits == 0 on entry; otherwise *splits is validated and kept)
+ * and the scratch bytes kraken_op_decode_attention needs for it.  Pure host arithmetic. */
+int kraken_decode_attention_sizes(int32_t groups, int32_t batch, int32_t n_keys, int32_t n_head, int32_t head_dim,
+                                  int32_t *splits, size_t *partial_bytes);
 
 #ifdef __cplusplus
 }

@@ -30,9 +30,10 @@ PROF_COUNT = len(PROF_CATEGORIES)
 
 EXPORTS = (
     "kraken_query_sizes", "kraken_create", "kraken_prefill", "kraken_prefill_host",
-    "kraken_prefill_all_logits", "kraken_logits_rows", "kraken_decode_step", "kraken_kv_view",
+    "kraken_prefill_all_logits", "kraken_logits_rows", "kraken_decode_step", "kraken_decode_step_host", "kraken_kv_view",
     "kraken_device_status", "kraken_cur_len", "kraken_profile_enable", "kraken_profile_read", "kraken_reset", "kraken_destroy", "kraken_strerror",
     "kraken_op_embed", "kraken_op_layernorm", "kraken_op_grouped_gemm", "kraken_op_attention",
+    "kraken_op_decode_attention", "kraken_decode_attention_sizes",
 )
 
 
@@ -90,6 +91,7 @@ def lib() -> C.CDLL:
         L.kraken_prefill_all_logits.argtypes = [vp, vp, i32, i32, vp, vp]
         L.kraken_logits_rows.argtypes = [vp, vp, i32, vp, vp]
         L.kraken_decode_step.argtypes = [vp, vp, i32, vp, vp]
+        L.kraken_decode_step_host.argtypes = [vp, vp, i32, vp, vp]
         L.kraken_kv_view.argtypes = [vp, i32, i32, i32, C.POINTER(vp), C.POINTER(i64 * 4)]
         L.kraken_device_status.argtypes = [vp, C.POINTER(C.c_uint32)]
         L.kraken_cur_len.argtypes = [vp, C.POINTER(i32)]
@@ -104,6 +106,9 @@ def lib() -> C.CDLL:
         L.kraken_op_layernorm.argtypes = [vp, i64, vp, vp, vp, i32, i32, i32, C.c_float, vp, vp]
         L.kraken_op_grouped_gemm.argtypes = [C.POINTER(GemmArgs), vp, vp]
         L.kraken_op_attention.argtypes = [vp, i64, vp, vp, i64, i64, i32, i32, i32, i32, i32, i32, i32, vp, i64, vp]
+        L.kraken_op_decode_attention.argtypes = [vp, i64, vp, vp, i64, i64, i32, i32, i32, i32, i32, i32, i32, vp,
+                                                 C.c_size_t, vp, i64, vp]
+        L.kraken_decode_attention_sizes.argtypes = [i32, i32, i32, i32, i32, C.POINTER(i32), C.POINTER(C.c_size_t)]
         _lib = L
     return _lib
 
@@ -215,6 +220,13 @@ class KrakenModel:
                "kraken_decode_step")
         return logits
 
+    def decode_step_host(self, tokens: torch.Tensor, logits: torch.Tensor) -> torch.Tensor:
+        """tokens [batch] / logits [batch, V]: HOST tensors; blocks until the logits are there."""
+        assert tokens.dtype == torch.int32 and tokens.device.type == "cpu" and logits.device.type == "cpu"
+        _check(lib().kraken_decode_step_host(self._h, tokens.data_ptr(), tokens.numel(), logits.data_ptr(),
+                                             _stream()), "kraken_decode_step_host")
+        return logits
+
     # -------- inspection
     def kv_view(self, layer: int, branch: int, which: int) -> torch.Tensor:
         """bf16 view [max_batch, n_head, max_pos, head_dim] of the K (0) or V (1) cache of (layer, branch)."""
@@ -289,4 +301,28 @@ def op_attention(q: torch.Tensor, k_cache: torch.Tensor, v_cache: torch.Tensor, 
     _check(lib().kraken_op_attention(q.data_ptr(), q.stride(0), k_cache.data_ptr(), v_cache.data_ptr(),
                                      k_cache.stride(0), k_cache.stride(1), G, batch, seqlen, pos0, H, hd, P,
                                      out.data_ptr(), out.stride(0), _stream()), "kraken_op_attention")
+    return out
+
+
+def decode_attention_sizes(groups: int, batch: int, n_keys: int, n_head: int, head_dim: int, splits: int = 0):
+    """(splits, scratch bytes) for op_decode_attention."""
+    sp, nb = C.c_int32(splits), C.c_size_t(0)
+    _check(lib().kraken_decode_attention_sizes(groups, batch, n_keys, n_head, head_dim, C.byref(sp), C.byref(nb)),
+           "kraken_decode_attention_sizes")
+    return sp.value, nb.value
+
+
+def op_decode_attention(q: torch.Tensor, k_cache: torch.Tensor, v_cache: torch.Tensor, n_keys: int,
+                        splits: int = 0, partials: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """q bf16 [G, batch, d]; caches bf16 [G, batch, n_head, max_pos, head_dim]; attends to rows 0..n_keys-1."""
+    G, B, d = q.shape
+    _, _, H, P, hd = k_cache.shape
+    splits, nbytes = decode_attention_sizes(G, B, n_keys, H, hd, splits)
+    if partials is None and nbytes:
+        partials = torch.empty(nbytes, dtype=torch.uint8, device=q.device)
+    out = torch.empty_like(q)
+    _check(lib().kraken_op_decode_attention(q.data_ptr(), q.stride(0), k_cache.data_ptr(), v_cache.data_ptr(),
+                                            k_cache.stride(0), k_cache.stride(1), G, B, n_keys, H, hd, P, splits,
+                                            _ptr(partials), 0 if partials is None else partials.numel(),
+                                            out.data_ptr(), out.stride(0), _stream()), "kraken_op_decode_attention")
     return out

@@ -87,6 +87,16 @@ def run_case(kind: str, workload: str, reps: int, warmup: int, n_tile: int = 0, 
         fn = lambda: kr.op_attention(q, kc, vc, batch, seqlen, 0, H)
         flops = float(N * batch * H) * 4 * hd * (seqlen * (seqlen + 1) / 2)
         byts = 4 * N * T * d * 2
+    elif kind == "decode_attention":
+        ctx = seqlen
+        q = ki.normal_bf16(12, 0, (N, batch, d), 1.0, DEV)
+        kc = ki.normal_bf16(12, 1, (N, batch, H, ctx, hd), 1.0, DEV)
+        vc = ki.normal_bf16(12, 2, (N, batch, H, ctx, hd), 1.0, DEV)
+        sp, nb = kr.decode_attention_sizes(N, batch, ctx, H, hd, n_tile)
+        part = torch.empty(max(nb, 16), dtype=torch.uint8, device=DEV)
+        fn = lambda: kr.op_decode_attention(q, kc, vc, ctx, sp, part)
+        flops = 4.0 * N * batch * ctx * d
+        byts = 2 * N * batch * ctx * d * 2 + 2 * N * batch * d * 2
     elif kind == "layernorm":
         a = ki.normal_bf16(13, 0, (N, T, d), 1.0, DEV).float()
         y = ki.normal_bf16(13, 1, (T, d), 1.0, DEV).float()
@@ -118,11 +128,11 @@ def run_case(kind: str, workload: str, reps: int, warmup: int, n_tile: int = 0, 
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("case", help="gemm_qkv | gemm_proj | gemm_up | gemm_down | attention | layernorm | all")
+    ap.add_argument("case", help="gemm_qkv | gemm_proj | gemm_up | gemm_down | attention | layernorm | decode_attention | all")
     ap.add_argument("--workload", default="C3")
     ap.add_argument("--reps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=2)
-    ap.add_argument("--n-tile", type=int, default=0)
+    ap.add_argument("--n-tile", type=int, default=0, help="GEMM N tile, or split count for decode_attention")
     ap.add_argument("--batch", type=int, default=None)
     ap.add_argument("--seqlen", type=int, default=None)
     a = ap.parse_args()

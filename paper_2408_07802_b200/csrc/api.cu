@@ -21,7 +21,7 @@ constexpr size_t ALIGN = 256;
 size_t align_up(size_t v) { return (v + ALIGN - 1) / ALIGN * ALIGN; }
 
 struct Layout {
-    size_t status, tokens, rows, logits, x0, x, a, s, u, q, o, g, total;
+    size_t status, tokens, rows, logits, x0, x, a, s, u, q, o, g, dec_part, total;
 };
 
 int check_config(const kraken_config *c) {
@@ -61,6 +61,8 @@ Layout layout_of(const kraken_config *c) {
     l.q = take(N * T * d * 2);
     l.o = take(N * T * d * 2);
     l.g = take(N * T * F * 2);
+    l.dec_part = take(decode_attention_partial_bytes(c->n_branch, c->max_batch, c->n_head, c->d_model / c->n_head,
+                                                     DECODE_MAX_SPLITS));
     l.total = off;
     return l;
 }
@@ -255,7 +257,24 @@ int run_layers(const RunCtx &rc, const int32_t *d_tokens) {
         ap.max_pos = c.max_pos; ap.out = o; ap.out_gstride = td;
         {
             LaunchScope scope(h, KRAKEN_PROF_ATTENTION, rc.st);
-            KR_TRY(h->naive ? launch_attention_naive(ap, rc.st) : launch_attention_prefill(ap, rc.st));
+            if (h->naive) {
+                KR_TRY(launch_attention_naive(ap, rc.st));
+            } else if (rc.seqlen == 1) {
+                // decode step: stream the cache with the split-KV kernel
+                DecodeAttnParams dp;
+                dp.q = q; dp.q_gstride = td;
+                dp.k_cache = ap.k_cache; dp.v_cache = ap.v_cache;
+                dp.cache_gstride = ap.cache_gstride; dp.cache_bstride = ap.cache_bstride;
+                dp.groups = N; dp.batch = rc.batch; dp.n_keys = rc.pos0 + 1; dp.n_head = H; dp.head_dim = hd;
+                dp.max_pos = c.max_pos;
+                dp.splits = decode_attention_splits(N, rc.batch, H, dp.n_keys);
+                dp.partials = at<float>(h, h->lay.dec_part);
+                dp.out = o; dp.out_gstride = td;
+                h->launches[KRAKEN_PROF_ATTENTION] += dp.splits > 1 ? 1 : 0;
+                KR_TRY(launch_attention_decode(dp, rc.st));
+            } else {
+                KR_TRY(launch_attention_prefill(ap, rc.st));
+            }
         }
         // x = res + MHA(x)
         e = epi_zero();
@@ -453,6 +472,20 @@ int kraken_decode_step(kraken_handle *h, const int32_t *d_tokens, int32_t batch,
     return KRAKEN_OK;
 }
 
+int kraken_decode_step_host(kraken_handle *h, const int32_t *h_tokens, int32_t batch, float *h_logits, void *stream) {
+    if (!h || !h_tokens || !h_logits || batch < 1) return KRAKEN_EINVAL;
+    if (batch > h->cfg.max_batch) return KRAKEN_ECAPACITY;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    int32_t *d_tok = at<int32_t>(h, h->lay.tokens);
+    float *d_log = at<float>(h, h->lay.logits);
+    if (cudaMemcpyAsync(d_tok, h_tokens, (size_t)batch * 4, cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return KRAKEN_ECUDA;
+    KR_TRY(kraken_decode_step(h, d_tok, batch, d_log, stream));
+    if (cudaMemcpyAsync(h_logits, d_log, (size_t)batch * h->cfg.vocab * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return KRAKEN_ECUDA;
+    return cudaStreamSynchronize(st) == cudaSuccess ? KRAKEN_OK : KRAKEN_ECUDA;
+}
+
 int kraken_kv_view(kraken_handle *h, int32_t layer, int32_t branch, int32_t which, const void **ptr,
                    int64_t strides[4]) {
     if (!h || !ptr || !strides) return KRAKEN_EINVAL;
@@ -591,6 +624,36 @@ int kraken_op_attention(const void *q, int64_t q_gstride, const void *k_cache, c
     p.max_pos = max_pos; p.out = (uint16_t *)out; p.out_gstride = out_gstride;
     if (env_flag("KRAKEN_NAIVE")) return launch_attention_naive(p, static_cast<cudaStream_t>(stream));
     return launch_attention_prefill(p, static_cast<cudaStream_t>(stream));
+}
+
+int kraken_op_decode_attention(const void *q, int64_t q_gstride, const void *k_cache, const void *v_cache,
+                               int64_t cache_gstride, int64_t cache_bstride, int32_t groups, int32_t batch,
+                               int32_t n_keys, int32_t n_head, int32_t head_dim, int32_t max_pos, int32_t splits,
+                               void *d_partials, size_t partial_bytes, void *out, int64_t out_gstride, void *stream) {
+    if (groups < 1 || batch < 1 || n_head < 1 || n_keys < 1) return KRAKEN_EINVAL;
+    if (head_dim != 64 && head_dim != 128) return KRAKEN_EUNSUPPORTED;
+    if (splits == 0) splits = decode_attention_splits(groups, batch, n_head, n_keys);
+    if (splits < 1 || splits > DECODE_MAX_SPLITS) return KRAKEN_EINVAL;
+    if (splits > 1 && (!d_partials || partial_bytes < decode_attention_partial_bytes(groups, batch, n_head, head_dim, splits)))
+        return KRAKEN_ECAPACITY;
+    DecodeAttnParams p;
+    p.q = (const uint16_t *)q; p.q_gstride = q_gstride;
+    p.k_cache = (const uint16_t *)k_cache; p.v_cache = (const uint16_t *)v_cache;
+    p.cache_gstride = cache_gstride; p.cache_bstride = cache_bstride;
+    p.groups = groups; p.batch = batch; p.n_keys = n_keys; p.n_head = n_head; p.head_dim = head_dim;
+    p.max_pos = max_pos; p.splits = splits; p.partials = (float *)d_partials;
+    p.out = (uint16_t *)out; p.out_gstride = out_gstride;
+    return launch_attention_decode(p, static_cast<cudaStream_t>(stream));
+}
+
+int kraken_decode_attention_sizes(int32_t groups, int32_t batch, int32_t n_keys, int32_t n_head, int32_t head_dim,
+                                  int32_t *splits, size_t *partial_bytes) {
+    if (groups < 1 || batch < 1 || n_head < 1 || n_keys < 1 || !splits || !partial_bytes) return KRAKEN_EINVAL;
+    if (head_dim != 64 && head_dim != 128) return KRAKEN_EUNSUPPORTED;
+    if (*splits == 0) *splits = decode_attention_splits(groups, batch, n_head, n_keys);
+    if (*splits < 1 || *splits > DECODE_MAX_SPLITS) return KRAKEN_EINVAL;
+    *partial_bytes = *splits > 1 ? decode_attention_partial_bytes(groups, batch, n_head, head_dim, *splits) : 0;
+    return KRAKEN_OK;
 }
 
 }  // extern "C"

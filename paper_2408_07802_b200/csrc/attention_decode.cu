@@ -1,0 +1,217 @@
+// Decode-step attention: one query row per (branch, sequence, head) against all cached keys.
+// Pure HBM streaming of the K/V cache (the dominant bytes of a decode step), so the design is
+// about bytes in flight: the keys of one (branch, sequence, head) are split over several CTAs
+// (split-KV), every warp issues UNROLL independent 16-byte loads of K and of V per lane before
+// it consumes them, rows are read whole and coalesced (8 or 16 lanes per 128/256-byte row),
+// scores and the online softmax stay in fp32 registers.  Each split writes an unnormalised
+// partial (max, sum, output) to scratch; a second small kernel merges the splits.
+#include <math.h>
+
+#include "internal.h"
+#include "ptx.cuh"
+
+namespace kr {
+
+namespace {
+
+constexpr int DEC_WARPS = 4;
+constexpr int UNROLL = 4;
+
+template <int HD>
+__global__ void __launch_bounds__(DEC_WARPS * 32)
+attn_decode_kernel(const DecodeAttnParams p) {
+    constexpr int LPR = HD / 8;       // lanes per cache row (16 bytes each)
+    constexpr int RPW = 32 / LPR;     // rows per warp-wide load
+    const int split = blockIdx.x, h = blockIdx.y;
+    const int b = blockIdx.z % p.batch, g = blockIdx.z / p.batch;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int sub = lane % LPR, rg = lane / LPR;
+    const int d = p.n_head * HD;
+
+    // keys of this split
+    const int per = (p.n_keys + p.splits - 1) / p.splits;
+    const int k_begin = split * per;
+    const int k_end = min(p.n_keys, k_begin + per);
+
+    const uint16_t *gq = p.q + g * p.q_gstride + (long long)b * d + h * HD + sub * 8;
+    const uint16_t *gk = p.k_cache + g * p.cache_gstride + b * p.cache_bstride + (long long)h * p.max_pos * HD;
+    const uint16_t *gv = p.v_cache + g * p.cache_gstride + b * p.cache_bstride + (long long)h * p.max_pos * HD;
+
+    // this lane's 8 query elements, pre-scaled by log2(e) / sqrt(hd)
+    const float sl2 = rsqrtf(static_cast<float>(HD)) * 1.4426950408889634f;
+    float qf[8];
+    {
+        const uint4 u = *reinterpret_cast<const uint4 *>(gq);
+        qf[0] = bf16_lo(u.x) * sl2; qf[1] = bf16_hi(u.x) * sl2; qf[2] = bf16_lo(u.y) * sl2; qf[3] = bf16_hi(u.y) * sl2;
+        qf[4] = bf16_lo(u.z) * sl2; qf[5] = bf16_hi(u.z) * sl2; qf[6] = bf16_lo(u.w) * sl2; qf[7] = bf16_hi(u.w) * sl2;
+    }
+    float m = -INFINITY, l = 0.f, o[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) o[i] = 0.f;
+
+    // warp w takes row groups w, w + DEC_WARPS, ...; UNROLL groups per iteration
+    for (int r0 = k_begin + warp * RPW * UNROLL; r0 < k_end; r0 += DEC_WARPS * RPW * UNROLL) {
+        uint4 kk[UNROLL], vv[UNROLL];
+        bool valid[UNROLL];
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) {
+            const int key = r0 + u * RPW + rg;
+            valid[u] = key < k_end;
+            const long long off = (long long)(valid[u] ? key : k_begin) * HD + sub * 8;
+            kk[u] = *reinterpret_cast<const uint4 *>(gk + off);
+            vv[u] = *reinterpret_cast<const uint4 *>(gv + off);
+        }
+        float s[UNROLL];
+        float mx = m;
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) {
+            float acc = qf[0] * bf16_lo(kk[u].x);
+            acc = fmaf(qf[1], bf16_hi(kk[u].x), acc);
+            acc = fmaf(qf[2], bf16_lo(kk[u].y), acc);
+            acc = fmaf(qf[3], bf16_hi(kk[u].y), acc);
+            acc = fmaf(qf[4], bf16_lo(kk[u].z), acc);
+            acc = fmaf(qf[5], bf16_hi(kk[u].z), acc);
+            acc = fmaf(qf[6], bf16_lo(kk[u].w), acc);
+            acc = fmaf(qf[7], bf16_hi(kk[u].w), acc);
+#pragma unroll
+            for (int off = 1; off < LPR; off <<= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, off);
+            s[u] = valid[u] ? acc : -INFINITY;
+            mx = fmaxf(mx, s[u]);
+        }
+        if (mx > -INFINITY) {  // false only while every key seen by this lane group was out of range
+            const float corr = ex2_approx(m - mx);
+            l *= corr;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) o[i] *= corr;
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u) {
+                const float pu = ex2_approx(s[u] - mx);
+                l += pu;
+                o[0] = fmaf(pu, bf16_lo(vv[u].x), o[0]);
+                o[1] = fmaf(pu, bf16_hi(vv[u].x), o[1]);
+                o[2] = fmaf(pu, bf16_lo(vv[u].y), o[2]);
+                o[3] = fmaf(pu, bf16_hi(vv[u].y), o[3]);
+                o[4] = fmaf(pu, bf16_lo(vv[u].z), o[4]);
+                o[5] = fmaf(pu, bf16_hi(vv[u].z), o[5]);
+                o[6] = fmaf(pu, bf16_lo(vv[u].w), o[6]);
+                o[7] = fmaf(pu, bf16_hi(vv[u].w), o[7]);
+            }
+            m = mx;
+        }
+    }
+
+    // merge the row groups of the warp (lanes with equal `sub`), then the warps through shared memory
+#pragma unroll
+    for (int off = LPR; off < 32; off <<= 1) {
+        const float m2 = __shfl_xor_sync(0xFFFFFFFFu, m, off);
+        const float l2 = __shfl_xor_sync(0xFFFFFFFFu, l, off);
+        const float mn = fmaxf(m, m2);
+        const float c1 = mn > -INFINITY ? ex2_approx(m - mn) : 0.f;
+        const float c2 = mn > -INFINITY ? ex2_approx(m2 - mn) : 0.f;
+        l = l * c1 + l2 * c2;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const float o2 = __shfl_xor_sync(0xFFFFFFFFu, o[i], off);
+            o[i] = o[i] * c1 + o2 * c2;
+        }
+        m = mn;
+    }
+    __shared__ float sm_m[DEC_WARPS], sm_l[DEC_WARPS], sm_o[DEC_WARPS][HD];
+    if (rg == 0) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) sm_o[warp][sub * 8 + i] = o[i];
+        if (sub == 0) {
+            sm_m[warp] = m;
+            sm_l[warp] = l;
+        }
+    }
+    __syncthreads();
+    if (threadIdx.x < HD) {
+        const int e = threadIdx.x;
+        float mn = -INFINITY;
+#pragma unroll
+        for (int w = 0; w < DEC_WARPS; ++w) mn = fmaxf(mn, sm_m[w]);
+        float lt = 0.f, ot = 0.f;
+#pragma unroll
+        for (int w = 0; w < DEC_WARPS; ++w) {
+            const float c = sm_m[w] > -INFINITY ? ex2_approx(sm_m[w] - mn) : 0.f;
+            lt += sm_l[w] * c;
+            ot += sm_o[w][e] * c;
+        }
+        const long long stream = ((long long)blockIdx.z * p.n_head + h);
+        if (p.splits == 1) {
+            p.out[g * p.out_gstride + (long long)b * d + h * HD + e] =
+                __bfloat16_as_ushort(__float2bfloat16_rn(ot / lt));
+        } else {
+            float *part = p.partials + (stream * p.splits + split) * (HD + 2);
+            part[2 + e] = ot;
+            if (e == 0) {
+                part[0] = mn;
+                part[1] = lt;
+            }
+        }
+    }
+}
+
+// out = sum_s o_s 2^(m_s - m) / sum_s l_s 2^(m_s - m)
+template <int HD>
+__global__ void __launch_bounds__(HD) attn_decode_merge_kernel(const DecodeAttnParams p) {
+    const int h = blockIdx.x;
+    const int b = blockIdx.y % p.batch, g = blockIdx.y / p.batch;
+    const int e = threadIdx.x;
+    const long long stream = ((long long)blockIdx.y * p.n_head + h);
+    const float *part = p.partials + stream * p.splits * (HD + 2);
+    float mn = -INFINITY;
+    for (int s = 0; s < p.splits; ++s) mn = fmaxf(mn, part[s * (HD + 2)]);
+    float lt = 0.f, ot = 0.f;
+    for (int s = 0; s < p.splits; ++s) {
+        const float ms = part[s * (HD + 2)];
+        const float c = ms > -INFINITY ? ex2_approx(ms - mn) : 0.f;
+        lt += part[s * (HD + 2) + 1] * c;
+        ot += part[s * (HD + 2) + 2 + e] * c;
+    }
+    const int d = p.n_head * HD;
+    p.out[g * p.out_gstride + (long long)b * d + h * HD + e] = __bfloat16_as_ushort(__float2bfloat16_rn(ot / lt));
+}
+
+template <int HD>
+int launch(const DecodeAttnParams &p, cudaStream_t stream) {
+    dim3 grid(p.splits, p.n_head, p.batch * p.groups);
+    attn_decode_kernel<HD><<<grid, DEC_WARPS * 32, 0, stream>>>(p);
+    if (cudaGetLastError() != cudaSuccess) return KRAKEN_ECUDA;
+    if (p.splits > 1) {
+        dim3 g2(p.n_head, p.batch * p.groups);
+        attn_decode_merge_kernel<HD><<<g2, HD, 0, stream>>>(p);
+        if (cudaGetLastError() != cudaSuccess) return KRAKEN_ECUDA;
+    }
+    return KRAKEN_OK;
+}
+
+}  // namespace
+
+int decode_attention_splits(int groups, int batch, int n_head, int n_keys) {
+    const long long streams = (long long)groups * batch * n_head;
+    const int sms = sm_count() > 0 ? sm_count() : 148;
+    const long long want = 6LL * sms;  // CTAs to aim for
+    long long s = (want + streams - 1) / streams;
+    const long long by_len = (n_keys + 127) / 128;  // at least 128 keys per split
+    if (s > by_len) s = by_len;
+    if (s > DECODE_MAX_SPLITS) s = DECODE_MAX_SPLITS;
+    if (s < 1) s = 1;
+    return static_cast<int>(s);
+}
+
+size_t decode_attention_partial_bytes(int groups, int batch, int n_head, int head_dim, int splits) {
+    return (size_t)groups * batch * n_head * splits * (head_dim + 2) * sizeof(float);
+}
+
+int launch_attention_decode(const DecodeAttnParams &p, cudaStream_t stream) {
+    if (!p.q || !p.k_cache || !p.v_cache || !p.out || p.groups < 1 || p.batch < 1 || p.n_head < 1 || p.n_keys < 1 ||
+        p.n_keys > p.max_pos || p.splits < 1 || p.splits > DECODE_MAX_SPLITS || (p.splits > 1 && !p.partials))
+        return KRAKEN_EINVAL;
+    if (p.head_dim == 64) return launch<64>(p, stream);
+    if (p.head_dim == 128) return launch<128>(p, stream);
+    return KRAKEN_EUNSUPPORTED;
+}
+
+}  // namespace kr

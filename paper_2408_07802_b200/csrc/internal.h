@@ -86,6 +86,23 @@ struct AttnParams {
 int launch_attention_prefill(const AttnParams &p, cudaStream_t stream);
 int launch_attention_naive(const AttnParams &p, cudaStream_t stream);
 
+// Decode-step attention (one query row per sequence and head) with split-KV partials in scratch.
+constexpr int DECODE_MAX_SPLITS = 32;
+struct DecodeAttnParams {
+    const uint16_t *q;  // [G][batch, d]
+    long long q_gstride;
+    const uint16_t *k_cache, *v_cache;
+    long long cache_gstride, cache_bstride;
+    int groups, batch, n_keys, n_head, head_dim, max_pos;
+    int splits;
+    float *partials;  // [G*batch*n_head][splits][head_dim + 2] fp32 (max, sum, output); unused when splits == 1
+    uint16_t *out;    // [G][batch, d]
+    long long out_gstride;
+};
+int decode_attention_splits(int groups, int batch, int n_head, int n_keys);
+size_t decode_attention_partial_bytes(int groups, int batch, int n_head, int head_dim, int splits);
+int launch_attention_decode(const DecodeAttnParams &p, cudaStream_t stream);
+
 bool env_flag(const char *name);
 
 }  // namespace kr

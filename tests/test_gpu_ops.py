@@ -244,3 +244,38 @@ def test_attention_matches_oracle(hd, seqlen, pos0):
                 den += (ref ** 2).sum()
     assert worst < 3e-2, worst
     assert np.sqrt(num / den) < 6e-3, np.sqrt(num / den)
+
+
+@pytest.mark.parametrize("hd", [64, 128])
+@pytest.mark.parametrize("n_keys,splits", [(1, 1), (2, 0), (131, 3), (700, 0), (2049, 32), (300, 1)])
+def test_decode_attention_matches_oracle(hd, n_keys, splits):
+    G, B, H, P = 2, 3, 2, 2112
+    d = H * hd
+    q = ki.normal_bf16(8, 0, (G, B, d), 1.0, DEV)
+    kc = ki.normal_bf16(8, 1, (G, B, H, P, hd), 1.0, DEV)
+    vc = ki.normal_bf16(8, 2, (G, B, H, P, hd), 1.0, DEV)
+    kc[:, :, :, n_keys:] = float("nan")   # rows past the sequence must never be read into the result
+    vc[:, :, :, n_keys:] = float("nan")
+    out = kr.op_decode_attention(q, kc, vc, n_keys, splits).float().cpu().numpy()
+    assert not np.isnan(out).any()
+    qn, kn, vn = q.float().cpu().numpy(), kc.float().cpu().numpy(), vc.float().cpu().numpy()
+    worst = 0.0
+    for g in range(G):
+        for b in range(B):
+            for h in range(H):
+                ref = oracle.attention_head(qn[g, b:b + 1, h * hd:(h + 1) * hd], kn[g, b, h, :n_keys],
+                                            vn[g, b, h, :n_keys], q_pos0=n_keys - 1)
+                worst = max(worst, np.abs(out[g, b, h * hd:(h + 1) * hd] - ref[0]).max())
+    assert worst < 2e-2, worst
+
+
+def test_decode_attention_scratch_checks():
+    sp, nb = kr.decode_attention_sizes(4, 16, 2048, 16, 64)
+    assert 1 <= sp <= 32 and nb == (0 if sp == 1 else 4 * 16 * 16 * sp * 66 * 4)
+    assert kr.decode_attention_sizes(1, 1, 50, 2, 64, 1) == (1, 0)
+    q = torch.zeros(1, 1, 128, dtype=torch.bfloat16, device=DEV)
+    kc = torch.zeros(1, 1, 2, 64, 64, dtype=torch.bfloat16, device=DEV)
+    small = torch.empty(16, dtype=torch.uint8, device=DEV)
+    with pytest.raises(kr.KrakenError) as e:
+        kr.op_decode_attention(q, kc, kc, 40, splits=4, partials=small)
+    assert e.value.status == kr.ECAPACITY
