@@ -177,6 +177,7 @@ int model_gemm(const RunCtx &rc, GemmKind kind, int layer, int m_rows, const uin
                                         KRAKEN_PROF_GEMM_DOWN, KRAKEN_PROF_TAIL, KRAKEN_PROF_TAIL};
     LaunchScope scope(h, cat_of[kind], rc.st);
     if (h->naive) return launch_gemm_naive(op, s, epi, rc.st);
+    if (m_rows <= SKINNY_MAX_ROWS && epi.kind != KRAKEN_EPI_RESID_SUM) return launch_gemm_skinny(op, s, epi, rc.st);
 
     const int bn = gemm_pick_bn(s);
     if (h->tmB_bn[kind] != bn) {
@@ -216,6 +217,7 @@ int run_layers(const RunCtx &rc, const int32_t *d_tokens) {
     const kraken_config &c = h->cfg;
     const int d = c.d_model, F = c.d_ff, N = c.n_branch, L = c.n_layer, H = c.n_head, hd = d / H, T = rc.T;
     const long long td = (long long)T * d;
+    const bool small_rows = T <= SKINNY_MAX_ROWS && !h->naive;
     float *x0 = at<float>(h, h->lay.x0), *x = at<float>(h, h->lay.x), *a = at<float>(h, h->lay.a),
           *S = at<float>(h, h->lay.s);
     uint16_t *u = at<uint16_t>(h, h->lay.u), *q = at<uint16_t>(h, h->lay.q), *o = at<uint16_t>(h, h->lay.o),
@@ -285,9 +287,13 @@ int run_layers(const RunCtx &rc, const int32_t *d_tokens) {
         // x = LN(x + y): y is the shared embedding in the first layer, the cross-branch sum afterwards
         {
             LaunchScope scope(h, KRAKEN_PROF_LAYERNORM, rc.st);
-            KR_TRY(launch_layernorm(a, td, l == 0 ? x0 : S, (const uint16_t *)h->w.ln2_g + ln_off,
+            // with few rows the cross-branch sum is formed here from the N branch inputs (same order as
+            // the down-projection epilogue forms it for long prompts)
+            const bool sum_here = small_rows && l > 0;
+            KR_TRY(launch_layernorm(a, td, sum_here ? nullptr : (l == 0 ? x0 : S),
+                                    (const uint16_t *)h->w.ln2_g + ln_off,
                                     h->w.ln2_b ? (const uint16_t *)h->w.ln2_b + ln_off : nullptr, N, T, d, c.ln_eps,
-                                    u, rc.st));
+                                    u, rc.st, sum_here ? x : nullptr, td, N));
         }
         // FFN up + GELU
         e = epi_zero();
@@ -296,7 +302,7 @@ int run_layers(const RunCtx &rc, const int32_t *d_tokens) {
         KR_TRY(model_gemm(rc, G_UP, l, T, u, td, e));
         // out = res + FFN ; the sum over branches (the AllReduce feeding the next layer) in the epilogue
         e = epi_zero();
-        e.kind = l + 1 < L ? KRAKEN_EPI_RESID_SUM : KRAKEN_EPI_RESID_F32;
+        e.kind = (l + 1 < L && !small_rows) ? KRAKEN_EPI_RESID_SUM : KRAKEN_EPI_RESID_F32;
         e.out_f32 = x; e.out_f32_gstride = td; e.ld_out_f32 = d;
         e.resid = a; e.resid_gstride = td; e.ld_resid = d;
         e.sum = S; e.ld_sum = d;
@@ -609,6 +615,7 @@ int kraken_op_grouped_gemm(const kraken_gemm_args *g, uint32_t *d_status, void *
     e.d_model = g->n_head * g->head_dim;
     e.gelu_tanh = g->gelu_tanh;
     if (env_flag("KRAKEN_NAIVE")) return launch_gemm_naive(op, s, e, static_cast<cudaStream_t>(stream));
+    if (g->n_tile == 8) return launch_gemm_skinny(op, s, e, static_cast<cudaStream_t>(stream));
     return launch_gemm_tc(op, s, e, nullptr, nullptr, 0, g->n_tile, d_status, static_cast<cudaStream_t>(stream));
 }
 

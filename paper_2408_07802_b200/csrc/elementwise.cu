@@ -42,9 +42,12 @@ __device__ __forceinline__ float warp_sum(float v) {
 
 constexpr int LN_CACHE = 16;  // float4 per lane kept in registers: rows up to 2048 wide in one pass
 
-// out[g][r, :] = bf16( gamma_g * (v - mean) * rstd + beta_g ),  v = a[g][r, :] (+ y[r, :])
+// out[g][r, :] = bf16( gamma_g * (v - mean) * rstd + beta_g ),  v = a[g][r, :] + y[r, :]
+// where y is absent, a given [rows, d] tensor, or the sum over `ysum_groups` tensors taken in
+// ascending order (the cross-branch sum computed on the fly when the row count is small).
 __global__ void __launch_bounds__(ROW_WARPS * 32)
 layernorm_kernel(const float *__restrict__ a, long long a_gstride, const float *__restrict__ y,
+                 const float *__restrict__ ysum, long long ysum_gstride, int ysum_groups,
                  const uint16_t *__restrict__ gamma, const uint16_t *__restrict__ beta, int groups, int rows, int d,
                  float eps, uint16_t *__restrict__ out) {
     const long long wr = (long long)blockIdx.x * ROW_WARPS + (threadIdx.x >> 5);
@@ -54,7 +57,24 @@ layernorm_kernel(const float *__restrict__ a, long long a_gstride, const float *
     const int r = static_cast<int>(wr / groups), g = static_cast<int>(wr % groups);
     const float4 *pa = reinterpret_cast<const float4 *>(a + g * a_gstride + (size_t)r * d);
     const float4 *py = y ? reinterpret_cast<const float4 *>(y + (size_t)r * d) : nullptr;
+    const float4 *ps = ysum ? reinterpret_cast<const float4 *>(ysum + (size_t)r * d) : nullptr;
     const int nvec = d / 4;
+
+    auto load = [&](int v) {
+        float4 t = pa[v];
+        if (py) {
+            const float4 u = py[v];
+            t.x += u.x; t.y += u.y; t.z += u.z; t.w += u.w;
+        } else if (ps) {
+            float4 acc = ps[v];
+            for (int m = 1; m < ysum_groups; ++m) {
+                const float4 u = ps[(size_t)m * (ysum_gstride / 4) + v];
+                acc.x += u.x; acc.y += u.y; acc.z += u.z; acc.w += u.w;
+            }
+            t.x += acc.x; t.y += acc.y; t.z += acc.z; t.w += acc.w;
+        }
+        return t;
+    };
 
     float4 cache[LN_CACHE];
     float sum = 0.f;
@@ -62,21 +82,13 @@ layernorm_kernel(const float *__restrict__ a, long long a_gstride, const float *
     for (int i = 0; i < LN_CACHE; ++i) {
         const int v = lane + 32 * i;
         if (v < nvec) {
-            float4 t = pa[v];
-            if (py) {
-                const float4 u = py[v];
-                t.x += u.x; t.y += u.y; t.z += u.z; t.w += u.w;
-            }
+            const float4 t = load(v);
             cache[i] = t;
             sum += (t.x + t.y) + (t.z + t.w);
         }
     }
     for (int v = lane + 32 * LN_CACHE; v < nvec; v += 32) {
-        float4 t = pa[v];
-        if (py) {
-            const float4 u = py[v];
-            t.x += u.x; t.y += u.y; t.z += u.z; t.w += u.w;
-        }
+        const float4 t = load(v);
         sum += (t.x + t.y) + (t.z + t.w);
     }
     const float mean = warp_sum(sum) / d;
@@ -91,11 +103,7 @@ layernorm_kernel(const float *__restrict__ a, long long a_gstride, const float *
         }
     }
     for (int v = lane + 32 * LN_CACHE; v < nvec; v += 32) {
-        float4 t = pa[v];
-        if (py) {
-            const float4 u = py[v];
-            t.x += u.x; t.y += u.y; t.z += u.z; t.w += u.w;
-        }
+        const float4 t = load(v);
         const float dx = t.x - mean, dy = t.y - mean, dz = t.z - mean, dw = t.w - mean;
         sq += (dx * dx + dy * dy) + (dz * dz + dw * dw);
     }
@@ -119,14 +127,7 @@ layernorm_kernel(const float *__restrict__ a, long long a_gstride, const float *
         const int v = lane + 32 * i;
         if (v < nvec) emit(v, cache[i]);
     }
-    for (int v = lane + 32 * LN_CACHE; v < nvec; v += 32) {
-        float4 t = pa[v];
-        if (py) {
-            const float4 u = py[v];
-            t.x += u.x; t.y += u.y; t.z += u.z; t.w += u.w;
-        }
-        emit(v, t);
-    }
+    for (int v = lane + 32 * LN_CACHE; v < nvec; v += 32) emit(v, load(v));
 }
 
 __global__ void __launch_bounds__(ROW_WARPS * 32)
@@ -167,11 +168,12 @@ int launch_embed(const int32_t *ids, int n_tokens, int seqlen, int pos0, const u
 
 int launch_layernorm(const float *a, long long a_gstride, const float *y, const uint16_t *gamma,
                      const uint16_t *beta, int groups, int rows, int d, float eps, uint16_t *out,
-                     cudaStream_t stream) {
+                     cudaStream_t stream, const float *ysum, long long ysum_gstride, int ysum_groups) {
     if (!a || !gamma || !out || groups < 1 || rows < 1 || d < 4 || (d & 3)) return KRAKEN_EINVAL;
+    if (ysum && (y || ysum_groups < 1 || (ysum_gstride & 3))) return KRAKEN_EINVAL;
     const long long warps = (long long)groups * rows;
     layernorm_kernel<<<static_cast<unsigned>((warps + ROW_WARPS - 1) / ROW_WARPS), ROW_WARPS * 32, 0, stream>>>(
-        a, a_gstride, y, gamma, beta, groups, rows, d, eps, out);
+        a, a_gstride, y, ysum, ysum_gstride, ysum_groups, gamma, beta, groups, rows, d, eps, out);
     return done();
 }
 

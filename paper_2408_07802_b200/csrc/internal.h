@@ -60,14 +60,21 @@ int gemm_pick_bn(const GemmShape &shape);
 int gemm_encode_a(CUtensorMap *map, const GemmOperands &op, const GemmShape &shape);
 int gemm_encode_b(CUtensorMap *map, const GemmOperands &op, const GemmShape &shape, int bn);
 
+// Weight-streaming GEMM for M <= 32 rows (decode, last-position tail); every epilogue except RESID_SUM.
+int launch_gemm_skinny(const GemmOperands &op, const GemmShape &shape, const EpiParams &epi, cudaStream_t stream);
+constexpr int SKINNY_MAX_ROWS = 32;
+
 // One thread per output element; for bring-up comparisons only (KRAKEN_NAIVE=1).
 int launch_gemm_naive(const GemmOperands &op, const GemmShape &shape, const EpiParams &epi, cudaStream_t stream);
 
 int launch_embed(const int32_t *ids, int n_tokens, int seqlen, int pos0, const uint16_t *wte, const uint16_t *wpe,
                  int d, int vocab, float *out, uint32_t *status, cudaStream_t stream);
+// y: [rows, d] added before normalisation (or NULL); alternatively ysum: `ysum_groups` tensors
+// [rows, d], ysum_gstride apart, whose sum is added.
 int launch_layernorm(const float *a, long long a_gstride, const float *y, const uint16_t *gamma,
                      const uint16_t *beta, int groups, int rows, int d, float eps, uint16_t *out,
-                     cudaStream_t stream);
+                     cudaStream_t stream, const float *ysum = nullptr, long long ysum_gstride = 0,
+                     int ysum_groups = 0);
 // rows of N fp32 branch outputs -> bf16 branch-major concatenation [n_rows, N*d]; rows picked by index list
 // (device int32, NULL = identity).
 int launch_gather_concat(const float *x, long long x_gstride, int groups, int d, const int32_t *rows, int n_rows,

@@ -279,3 +279,35 @@ def test_decode_attention_scratch_checks():
     with pytest.raises(kr.KrakenError) as e:
         kr.op_decode_attention(q, kc, kc, 40, splits=4, partials=small)
     assert e.value.status == kr.ECAPACITY
+
+
+@pytest.mark.parametrize("M", [1, 16, 17, 32])
+def test_skinny_gemm_integer_exact(M):
+    """The weight-streaming kernel used for decode and the tail (n_tile = 8), ragged N and K."""
+    r = gemm_case(3, M, 203 * 8 + 8, 136, kr.EPI_F32, 8, integer=True, seed=6)
+    assert np.array_equal(r["out_f32"], r["ref"])
+
+
+@pytest.mark.parametrize("epi", [kr.EPI_F32, kr.EPI_BF16, kr.EPI_GELU_BF16, kr.EPI_RESID_F32])
+def test_skinny_gemm_epilogues(epi):
+    r = gemm_case(4, 16, 1024, 4096, epi, 8, seed=7)
+    if r["out_f32"] is not None:
+        assert np.abs(r["out_f32"] - r["ref"]).max() < 5e-4
+    else:
+        ok, worst = bf16_ulp_close(r["out_bf16"], r["ref"], ulps=1.0, atol=2e-4)
+        assert ok, worst
+
+
+def test_skinny_gemm_unaligned_output_rows():
+    """fp32 output with an odd row stride (the logits of a 50257-word vocabulary)."""
+    G, M, Nout, K = 1, 5, 1001, 256
+    a = ki.normal_bf16(9, 0, (G, M, K), 1.0, DEV)
+    w = ki.normal_bf16(9, 1, (G, Nout, K), 0.06, DEV)
+    out = torch.full((M, Nout), float("nan"), dtype=torch.float32, device=DEV)
+    args = kr.GemmArgs()
+    args.a, args.lda, args.w, args.ldw = a.data_ptr(), K, w.data_ptr(), K
+    args.groups, args.m, args.n_out, args.k, args.epilogue, args.n_tile = G, M, Nout, K, kr.EPI_F32, 8
+    args.out_f32, args.ld_out_f32 = out.data_ptr(), Nout
+    kr.op_grouped_gemm(args)
+    ref = oracle.linear(a[0].float().cpu().numpy(), bits(w[0]))
+    assert np.abs(out.cpu().numpy() - ref).max() < 2e-4
