@@ -241,6 +241,29 @@ int kraken_op_decode_attention(const void *q, int64_t q_gstride, const void *k_c
 int kraken_decode_attention_sizes(int32_t groups, int32_t batch, int32_t n_keys, int32_t n_head, int32_t head_dim,
                                   int32_t *splits, size_t *partial_bytes);
 
+/* (The paper has no counterpart to this call; it exists for hosts that cannot allocate.)
+ * kraken_op_decode_attention without a scratch argument.  Meant for callers that have no way to
+ * give the library device memory of their own: servers whose memory pool already owns the whole
+ * device so that a fresh cudaMalloc fails, plugin-style integrations that are handed only input and
+ * output pointers, and loops that cannot afford the device-wide synchronisation an allocation
+ * implies.  The split-KV partials go to a fixed 8 MiB array inside the library image (held by every
+ * GPU that loads the library, until the process exits); the call itself allocates nothing, on the
+ * host side of CUDA or on the device.
+ *   - Same arguments, layouts and results as kraken_op_decode_attention (q, out: device bf16
+ *     [G][batch, n_head*head_dim]; caches as there; splits = 0 lets the library choose).
+ *   - ECAPACITY when groups * batch * n_head * splits * (head_dim + 2) * 4 bytes exceeds
+ *     kraken_decode_attention_static_capacity(); pass a smaller `splits` (1 needs no partials).
+ *   - The first call on each device looks up the array's device address (once per device, with that
+ *     device current); make that first call before starting any stream capture.
+ *   - All calls share the one array and it keeps whatever the previous call left.  Nothing in it has
+ *     to start at zero: each call overwrites every partial it later reads.  Two calls whose kernels
+ *     may overlap on the GPU (different streams) race on it; serialise them. */
+int kraken_op_decode_attention_static(const void *q, int64_t q_gstride, const void *k_cache, const void *v_cache,
+                                      int64_t cache_gstride, int64_t cache_bstride, int32_t groups, int32_t batch,
+                                      int32_t n_keys, int32_t n_head, int32_t head_dim, int32_t max_pos,
+                                      int32_t splits, void *out, int64_t out_gstride, void *stream);
+size_t kraken_decode_attention_static_capacity(void);
+
 #ifdef __cplusplus
 }
 #endif

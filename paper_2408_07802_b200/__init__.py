@@ -34,6 +34,7 @@ EXPORTS = (
     "kraken_device_status", "kraken_cur_len", "kraken_profile_enable", "kraken_profile_read", "kraken_reset", "kraken_destroy", "kraken_strerror",
     "kraken_op_embed", "kraken_op_layernorm", "kraken_op_grouped_gemm", "kraken_op_attention",
     "kraken_op_decode_attention", "kraken_decode_attention_sizes",
+    "kraken_op_decode_attention_static", "kraken_decode_attention_static_capacity",
 )
 
 
@@ -109,6 +110,10 @@ def lib() -> C.CDLL:
         L.kraken_op_decode_attention.argtypes = [vp, i64, vp, vp, i64, i64, i32, i32, i32, i32, i32, i32, i32, vp,
                                                  C.c_size_t, vp, i64, vp]
         L.kraken_decode_attention_sizes.argtypes = [i32, i32, i32, i32, i32, C.POINTER(i32), C.POINTER(C.c_size_t)]
+        L.kraken_op_decode_attention_static.argtypes = [vp, i64, vp, vp, i64, i64, i32, i32, i32, i32, i32, i32, i32,
+                                                        vp, i64, vp]
+        L.kraken_decode_attention_static_capacity.argtypes = []
+        L.kraken_decode_attention_static_capacity.restype = C.c_size_t
         _lib = L
     return _lib
 
@@ -326,3 +331,22 @@ def op_decode_attention(q: torch.Tensor, k_cache: torch.Tensor, v_cache: torch.T
                                             _ptr(partials), 0 if partials is None else partials.numel(),
                                             out.data_ptr(), out.stride(0), _stream()), "kraken_op_decode_attention")
     return out
+
+
+def op_decode_attention_static(q: torch.Tensor, k_cache: torch.Tensor, v_cache: torch.Tensor, n_keys: int,
+                               splits: int = 0) -> torch.Tensor:
+    """op_decode_attention for callers that cannot provide scratch: the partials live in a fixed
+    array inside the library (see kraken_op_decode_attention_static).  The output tensor is still the
+    caller's; this wrapper creates it with torch only for convenience."""
+    G, B, d = q.shape
+    _, _, H, P, hd = k_cache.shape
+    out = torch.empty_like(q)
+    _check(lib().kraken_op_decode_attention_static(q.data_ptr(), q.stride(0), k_cache.data_ptr(), v_cache.data_ptr(),
+                                                   k_cache.stride(0), k_cache.stride(1), G, B, n_keys, H, hd, P,
+                                                   splits, out.data_ptr(), out.stride(0), _stream()),
+           "kraken_op_decode_attention_static")
+    return out
+
+
+def decode_attention_static_capacity() -> int:
+    return int(lib().kraken_decode_attention_static_capacity())
