@@ -274,6 +274,8 @@ int run_layers(const RunCtx &rc, const int32_t *d_tokens) {
                 dp.out = o; dp.out_gstride = td;
                 h->launches[KRAKEN_PROF_ATTENTION] += dp.splits > 1 ? 1 : 0;
                 KR_TRY(launch_attention_decode(dp, rc.st));
+            } else if (attention_tc_supported(ap) && !env_flag("KRAKEN_ATTN_WARP_MMA")) {
+                KR_TRY(launch_attention_tc(ap, nullptr, nullptr, nullptr, status, rc.st));
             } else {
                 KR_TRY(launch_attention_prefill(ap, rc.st));
             }
@@ -630,6 +632,8 @@ int kraken_op_attention(const void *q, int64_t q_gstride, const void *k_cache, c
     p.groups = groups; p.batch = batch; p.seqlen = seqlen; p.pos0 = pos0; p.n_head = n_head; p.head_dim = head_dim;
     p.max_pos = max_pos; p.out = (uint16_t *)out; p.out_gstride = out_gstride;
     if (env_flag("KRAKEN_NAIVE")) return launch_attention_naive(p, static_cast<cudaStream_t>(stream));
+    if (attention_tc_supported(p) && !env_flag("KRAKEN_ATTN_WARP_MMA"))
+        return launch_attention_tc(p, nullptr, nullptr, nullptr, nullptr, static_cast<cudaStream_t>(stream));
     return launch_attention_prefill(p, static_cast<cudaStream_t>(stream));
 }
 

@@ -92,6 +92,11 @@ struct AttnParams {
 };
 int launch_attention_prefill(const AttnParams &p, cudaStream_t stream);
 int launch_attention_naive(const AttnParams &p, cudaStream_t stream);
+// tcgen05 / TMEM attention for tiles of 128 queries x 128 keys; tensor maps may be NULL (encoded per call).
+bool attention_tc_supported(const AttnParams &p);
+int attention_tc_encode(const AttnParams &p, CUtensorMap *tmQ, CUtensorMap *tmK, CUtensorMap *tmV);
+int launch_attention_tc(const AttnParams &p, const CUtensorMap *tmQ, const CUtensorMap *tmK, const CUtensorMap *tmV,
+                        uint32_t *d_status, cudaStream_t stream);
 
 // Decode-step attention (one query row per sequence and head) with split-KV partials in scratch.
 constexpr int DECODE_MAX_SPLITS = 32;

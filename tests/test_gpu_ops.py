@@ -218,10 +218,13 @@ def test_gemm_rejects_unaligned():
 
 # ------------------------------------------------------------------ attention
 
+@pytest.mark.parametrize("kernel", ["tcgen05", "warp_mma"])
 @pytest.mark.parametrize("hd", [64, 128])
-@pytest.mark.parametrize("seqlen,pos0", [(200, 0), (100, 37), (1, 90), (64, 0)])
-def test_attention_matches_oracle(hd, seqlen, pos0):
-    G, B, H, P = 2, 2, 2, 256
+@pytest.mark.parametrize("seqlen,pos0", [(200, 0), (100, 37), (1, 90), (64, 0), (300, 0), (129, 127)])
+def test_attention_matches_oracle(hd, seqlen, pos0, kernel, monkeypatch):
+    if kernel == "warp_mma":
+        monkeypatch.setenv("KRAKEN_ATTN_WARP_MMA", "1")   # the m16n8k16 kernel kept for odd cache strides
+    G, B, H, P = 2, 2, 2, 512
     d = H * hd
     q = ki.normal_bf16(7, 0, (G, B * seqlen, d), 1.0, DEV)
     kc = ki.normal_bf16(7, 1, (G, B, H, P, hd), 1.0, DEV)
