@@ -1,17 +1,24 @@
-// Causal prefill attention on the sm_100a tensor cores (tcgen05 + TMEM), one CTA per tile of 128
-// query rows of one (branch, sequence, head), streaming K/V tiles of 128 keys by TMA.
+// Causal prefill attention on the sm_100a tensor cores (tcgen05 + TMEM).
 //
-//   warp 0      TMA producer: Q once, then K and V tiles into two-stage rings (128-byte swizzle);
-//   warp 1      MMA issuer:   S_j = Q K_j^T  (both operands K-major in shared memory) into one of two
-//                             S buffers in TMEM, then O_j = P_j V_j with P_j read from TMEM (it
-//                             overwrites S_j in place as packed bf16) and V_j MN-major in shared memory;
-//   warps 2-5   softmax:      one thread per query row (TMEM lane = row, so row max and row sum need
-//                             no shuffles): tcgen05.ld of S_j, causal mask, exp2 with the scale folded
-//                             in, tcgen05.st of P_j, then the running output kept in registers
-//                             acc = acc * corr + O_j  with O_j fetched from TMEM.
-// S_{j+1} = Q K_{j+1}^T is issued before P_j V_j, so the tensor pipe works on the next scores while
-// the softmax warps are busy with the current ones.  TMEM: 2 x 128 columns of S/P, 2 x HD of O_j.
-// Every mbarrier wait is time-bounded and falls through to a common teardown.
+// One CTA owns TWO tiles of 128 query rows of one (branch, sequence, head) and streams K/V tiles of
+// 128 keys by TMA; the two query tiles share every K/V tile and take turns on the tensor pipe, so
+// that while one tile's scores are in the softmax the other tile's matrix products run.
+//
+//   warp 0      TMA producer: both Q tiles once, then K and V tiles into two-stage rings
+//               (128-byte swizzle; rows past the keys written so far are out of bounds = zeros);
+//   warp 1      MMA issuer, per K/V tile j and query tile w:
+//                   S_w = Q_w K_j^T          both operands K-major in shared memory -> TMEM
+//                   O_w (+)= P_w V_j         P_w read from TMEM (it overwrites S_w in place as packed
+//                                            bf16), V_j MN-major in shared memory, O_w accumulates in TMEM
+//               issued in the order PV_0(j), QK_0(j+1), PV_1(j), QK_1(j+1);
+//   warps 2-5   softmax of query tile 0, warps 6-9 of query tile 1: one thread per query row (TMEM
+//               lane = row: row max and row sum need no shuffles).  The whole score row is pulled into
+//               registers with tcgen05.ld, masked on diagonal tiles, exponentiated with the scale folded
+//               into one packed FMA, stored back as P with tcgen05.st.
+// The running maximum is only raised when a row's new maximum exceeds the one in use by more than
+// 2^8 in the exponent; then (rarely) the warp rescales its rows of O in TMEM before releasing P.
+// Using a stale maximum is exact: numerator and denominator carry the same factor.
+// TMEM: S/P of tile w at column 128 w, O of tile w at 256 + 128 w.  All waits are time-bounded.
 #include <math.h>
 
 #include "internal.h"
@@ -21,9 +28,10 @@ namespace kr {
 
 namespace {
 
-constexpr int TQ = 128;   // query rows per CTA
+constexpr int TQ = 128;   // query rows per tile (two tiles per CTA)
 constexpr int TK = 128;   // keys per tile
-constexpr int ATC_THREADS = 192;
+constexpr int ATC_THREADS = 320;
+constexpr float RESCALE_LOG2 = 8.0f;
 
 struct AttnTcArgs {
     int groups, batch, seqlen, pos0, n_head;
@@ -31,18 +39,6 @@ struct AttnTcArgs {
     long long out_gstride;
     uint32_t *status;
 };
-
-__device__ __forceinline__ void tmem_ld_32x32_nowait(uint32_t taddr, uint32_t (&r)[32]) { tmem_ld_32x32(taddr, r); }
-
-// 32 lanes x 16 columns store
-__device__ __forceinline__ void tmem_st_32x16(uint32_t taddr, const uint32_t (&r)[16]) {
-    asm volatile(
-        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
-        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};" ::"r"(taddr),
-        "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
-        "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
-        : "memory");
-}
 
 // MN-major operand (V: rows = keys, 64 head-dim columns = 128 bytes per row, 128-byte swizzle):
 // groups of 8 keys are 1024 bytes apart (stride byte offset); the next 64 columns of the head
@@ -57,16 +53,36 @@ __device__ __forceinline__ uint64_t umma_desc_sw128_mnmajor(uint32_t smem_addr, 
     return d;
 }
 
+__device__ __forceinline__ float max3f(float a, float b, float c) {
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+
+// (x0, x1) * a + b on the packed fp32 pipe
+__device__ __forceinline__ void fma2(float &x0, float &x1, float a, float b) {
+    asm("{\n"
+        ".reg .b64 rx, ra, rb;\n"
+        "mov.b64 rx, {%0, %1};\n"
+        "mov.b64 ra, {%2, %2};\n"
+        "mov.b64 rb, {%3, %3};\n"
+        "fma.rn.f32x2 rx, rx, ra, rb;\n"
+        "mov.b64 {%0, %1}, rx;\n"
+        "}\n"
+        : "+f"(x0), "+f"(x1)
+        : "f"(a), "f"(b));
+}
+
 template <int HD>
 struct AtcCfg {
     static constexpr int HALVES = HD / 64;                 // 64-column (128-byte) pieces of the head dim
     static constexpr int TILE_BYTES = TK * 128;            // one 128 x 64 bf16 piece
-    static constexpr int Q_BYTES = HALVES * TILE_BYTES;
+    static constexpr int Q_BYTES = HALVES * TILE_BYTES;    // one Q tile
     static constexpr int KV_BYTES = HALVES * TILE_BYTES;   // one K (or V) tile
     static constexpr int STAGES = 2;
-    static constexpr int SMEM_BYTES = Q_BYTES + 2 * STAGES * KV_BYTES + 1024 + 256;
-    static constexpr int S_COL0 = 0;                       // S buffers at columns 0 and 128
-    static constexpr int O_COL0 = 256;                     // O buffers at 256 and 256 + HD
+    static constexpr int SMEM_BYTES = 2 * Q_BYTES + 2 * STAGES * KV_BYTES + 1024 + 256;
+    static constexpr int S_COL0 = 0;                       // S / P of query tile w at 128 w
+    static constexpr int O_COL0 = 256;                     // O of query tile w at 256 + 128 w
     static constexpr int TMEM_COLS = 512;
 };
 
@@ -77,8 +93,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     using Cfg = AtcCfg<HD>;
     extern __shared__ uint8_t smem_raw_atc[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw_atc) + 1023) & ~uintptr_t(1023));
-    uint8_t *sQ = smem;
-    uint8_t *sK = sQ + Cfg::Q_BYTES;                       // [STAGES][KV_BYTES]
+    uint8_t *sQ = smem;                                    // [2][Q_BYTES]
+    uint8_t *sK = sQ + 2 * Cfg::Q_BYTES;                   // [STAGES][KV_BYTES]
     uint8_t *sV = sK + Cfg::STAGES * Cfg::KV_BYTES;        // [STAGES][KV_BYTES]
     uint64_t *bars = reinterpret_cast<uint64_t *>(sV + Cfg::STAGES * Cfg::KV_BYTES);
     uint64_t *q_full = bars;            // 1
@@ -86,21 +102,24 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     uint64_t *k_empty = bars + 3;       // [2]
     uint64_t *v_full = bars + 5;        // [2]
     uint64_t *v_empty = bars + 7;       // [2]
-    uint64_t *s_full = bars + 9;        // [2]  scores ready            (MMA -> softmax)
-    uint64_t *p_ready = bars + 11;      // [2]  probabilities in TMEM   (softmax -> MMA)
-    uint64_t *o_full = bars + 13;       // [2]  P V product ready       (MMA -> softmax)
-    uint64_t *o_empty = bars + 15;      // [2]  product consumed        (softmax -> MMA)
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 17);
+    uint64_t *s_full = bars + 9;        // [2]  scores of query tile w ready      (MMA -> softmax w)
+    uint64_t *p_ready = bars + 11;      // [2]  probabilities of tile w in TMEM   (softmax w -> MMA)
+    uint64_t *pv_done = bars + 13;      // [2]  O_w holds every product issued so far (MMA -> softmax w)
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 15);
     volatile uint32_t *abort_flag = tmem_slot + 1;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int mt = gridDim.x - 1 - blockIdx.x;             // longest rows first
+    const int pair = gridDim.x - 1 - blockIdx.x;           // longest rows first
     const int h = blockIdx.y;
     const int b = blockIdx.z % a.batch, g = blockIdx.z / a.batch;
-    const int q0 = mt * TQ;
-    const int rows_valid = min(TQ, a.seqlen - q0);
-    const int n_keys = a.pos0 + q0 + rows_valid;           // keys visible to the last valid row
-    const int n_tiles = (n_keys + TK - 1) / TK;
+    const int q0 = pair * 2 * TQ;
+    int n_tiles[2];
+#pragma unroll
+    for (int w = 0; w < 2; ++w) {
+        const int rows = min(TQ, a.seqlen - (q0 + w * TQ));
+        n_tiles[w] = rows > 0 ? (a.pos0 + q0 + w * TQ + rows + TK - 1) / TK : 0;
+    }
+    const int n_max = max(n_tiles[0], n_tiles[1]);
 
     if (threadIdx.x == 0) {
         mbar_init(q_full, 1);
@@ -111,8 +130,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             mbar_init(v_empty + s, 1);
             mbar_init(s_full + s, 1);
             mbar_init(p_ready + s, 4);
-            mbar_init(o_full + s, 1);
-            mbar_init(o_empty + s, 4);
+            mbar_init(pv_done + s, 1);
         }
         *abort_flag = 0;
         fence_barrier_init();
@@ -131,13 +149,15 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
 
     if (warp == 0) {
         if (lane == 0) {
-            // Q: rows of this sequence's tile, columns of this head
-            mbar_expect_tx(q_full, Cfg::Q_BYTES);
+            const int q_tiles = n_tiles[1] > 0 ? 2 : 1;
+            mbar_expect_tx(q_full, q_tiles * Cfg::Q_BYTES);
+            for (int w = 0; w < q_tiles; ++w)
 #pragma unroll
-            for (int hf = 0; hf < Cfg::HALVES; ++hf)
-                tma_load_3d(sQ + hf * Cfg::TILE_BYTES, &tmQ, q_full, h * HD + hf * 64, b * a.seqlen + q0, g);
+                for (int hf = 0; hf < Cfg::HALVES; ++hf)
+                    tma_load_3d(sQ + w * Cfg::Q_BYTES + hf * Cfg::TILE_BYTES, &tmQ, q_full, h * HD + hf * 64,
+                                b * a.seqlen + q0 + w * TQ, g);
             bool ok = true;
-            for (int j = 0; ok && j < n_tiles; ++j) {
+            for (int j = 0; ok && j < n_max; ++j) {
                 const int st = j & 1;
                 const uint32_t ph = (j >> 1) & 1;
                 if (!(ok = mbar_wait(k_empty + st, ph ^ 1u, abort_flag))) break;
@@ -159,150 +179,165 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         if (lane == 0) {
             constexpr uint32_t idesc_qk = umma_idesc_bf16(TQ, TK);
             constexpr uint32_t idesc_pv = umma_idesc_bf16(TQ, HD) | (1u << 16);  // B (V) is MN-major
-            bool ok = mbar_wait(q_full, 0, abort_flag);
-            const uint32_t q_addr = smem_u32(sQ);
-            auto issue_qk = [&](int j) -> bool {
-                const int st = j & 1;
-                if (!mbar_wait(k_full + st, (j >> 1) & 1, abort_flag)) return false;
-                tc_fence_after_sync();
-                const uint32_t k_addr = smem_u32(sK + st * Cfg::KV_BYTES);
-                const uint32_t d_tmem = tmem_base + Cfg::S_COL0 + st * TK;
+            auto issue_qk = [&](int w, int j) {
+                const uint32_t q_addr = smem_u32(sQ + w * Cfg::Q_BYTES);
+                const uint32_t k_addr = smem_u32(sK + (j & 1) * Cfg::KV_BYTES);
+                const uint32_t d_tmem = tmem_base + Cfg::S_COL0 + w * TK;
 #pragma unroll
                 for (int ks = 0; ks < HD / 16; ++ks) {
                     const uint32_t off = (ks >> 2) * Cfg::TILE_BYTES + (ks & 3) * 32;
                     umma_bf16_ss(d_tmem, umma_desc_sw128_kmajor(q_addr + off), umma_desc_sw128_kmajor(k_addr + off),
                                  idesc_qk, ks != 0 ? 1u : 0u);
                 }
-                umma_commit(k_empty + st);
-                umma_commit(s_full + st);
-                return true;
+                umma_commit(s_full + w);
             };
-            if (ok) ok = issue_qk(0);
-            for (int j = 0; ok && j < n_tiles; ++j) {
-                const int st = j & 1;
-                const uint32_t ph = (j >> 1) & 1;
-                if (j + 1 < n_tiles && !(ok = issue_qk(j + 1))) break;
-                if (!(ok = mbar_wait(p_ready + st, ph, abort_flag))) break;
-                if (!(ok = mbar_wait(v_full + st, ph, abort_flag))) break;
-                if (!(ok = mbar_wait(o_empty + st, ph ^ 1u, abort_flag))) break;
-                tc_fence_after_sync();
-                const uint32_t v_addr = smem_u32(sV + st * Cfg::KV_BYTES);
-                const uint32_t p_tmem = tmem_base + Cfg::S_COL0 + st * TK;
-                const uint32_t o_tmem = tmem_base + Cfg::O_COL0 + st * HD;
+            auto issue_pv = [&](int w, int j) {
+                const uint32_t v_addr = smem_u32(sV + (j & 1) * Cfg::KV_BYTES);
+                const uint32_t p_tmem = tmem_base + Cfg::S_COL0 + w * TK;
+                const uint32_t o_tmem = tmem_base + Cfg::O_COL0 + w * TK;
 #pragma unroll
                 for (int ks = 0; ks < TK / 16; ++ks) {
                     // 16 keys per step: 8 packed columns of P, two 8-key groups (2 x 1024 bytes) of V
                     umma_bf16_ts(o_tmem, p_tmem + ks * 8,
                                  umma_desc_sw128_mnmajor(v_addr + ks * 2048, Cfg::TILE_BYTES), idesc_pv,
-                                 ks != 0 ? 1u : 0u);
+                                 (j | ks) != 0 ? 1u : 0u);
                 }
+                umma_commit(pv_done + w);
+            };
+            bool ok = mbar_wait(q_full, 0, abort_flag);
+            if (ok && n_max > 0) ok = mbar_wait(k_full + 0, 0, abort_flag);
+            if (ok && n_max > 0) {
+                tc_fence_after_sync();
+                if (n_tiles[0] > 0) issue_qk(0, 0);
+                if (n_tiles[1] > 0) issue_qk(1, 0);
+                umma_commit(k_empty + 0);
+            }
+            for (int j = 0; ok && j < n_max; ++j) {
+                const int st = j & 1;
+                const uint32_t ph = (j >> 1) & 1;
+                const bool next = j + 1 < n_max;
+                if (!(ok = mbar_wait(v_full + st, ph, abort_flag))) break;
+                if (next && !(ok = mbar_wait(k_full + ((j + 1) & 1), ((j + 1) >> 1) & 1, abort_flag))) break;
+#pragma unroll
+                for (int w = 0; w < 2; ++w) {
+                    if (j < n_tiles[w]) {
+                        if (!(ok = mbar_wait(p_ready + w, j & 1, abort_flag))) break;
+                        tc_fence_after_sync();
+                        issue_pv(w, j);
+                    }
+                    if (j + 1 < n_tiles[w]) issue_qk(w, j + 1);
+                }
+                if (!ok) break;
                 umma_commit(v_empty + st);
-                umma_commit(o_full + st);
+                if (next) umma_commit(k_empty + ((j + 1) & 1));
             }
         }
         __syncwarp();
     } else {
+        const int w = (warp - 2) >> 2;                       // query tile of this warp
         const int quarter = warp & 3;
         const int row = quarter * 32 + lane;                 // row of the tile = TMEM lane
-        const int qpos = a.pos0 + q0 + row;                  // position of this query
+        const int tile_q0 = q0 + w * TQ;
+        const int rows_valid = min(TQ, a.seqlen - tile_q0);
+        const int qpos = a.pos0 + tile_q0 + row;             // position of this query
+        const int n_w = n_tiles[w];
         const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
+        const uint32_t s_addr = lane_addr + Cfg::S_COL0 + w * TK;
+        const uint32_t o_addr = lane_addr + Cfg::O_COL0 + w * TK;
         const float sl2 = rsqrtf(static_cast<float>(HD)) * 1.4426950408889634f;
-        float acc[HD];
-#pragma unroll
-        for (int i = 0; i < HD; ++i) acc[i] = 0.f;
-        float m = -INFINITY, l = 0.f;
+        float m_used = -INFINITY, l = 0.f;
         bool ok = true;
 
-        auto add_product = [&](int j) -> bool {              // acc += O_j
-            const int st = j & 1;
-            bool good = mbar_wait(o_full + st, (j >> 1) & 1, abort_flag);
-            good = __all_sync(0xFFFFFFFFu, good);
-            if (!good) return false;
-            tc_fence_after_sync();
-#pragma unroll
-            for (int c = 0; c < HD / 32; ++c) {
-                uint32_t r[32];
-                tmem_ld_32x32(lane_addr + Cfg::O_COL0 + st * HD + c * 32, r);
-                tmem_ld_wait();
-#pragma unroll
-                for (int i = 0; i < 32; ++i) acc[c * 32 + i] += __uint_as_float(r[i]);
-            }
-            tc_fence_before_sync();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(o_empty + st);
-            return true;
-        };
-
-        for (int j = 0; j < n_tiles; ++j) {
-            const int st = j & 1;
-            ok = mbar_wait(s_full + st, (j >> 1) & 1, abort_flag);
+        for (int j = 0; j < n_w; ++j) {
+            ok = mbar_wait(s_full + w, j & 1, abort_flag);
             ok = __all_sync(0xFFFFFFFFu, ok);
             if (!ok) break;
             tc_fence_after_sync();
-            const uint32_t s_addr = lane_addr + Cfg::S_COL0 + st * TK;
-            const bool diag = j * TK + TK - 1 > a.pos0 + q0;  // tile may hold keys beyond some query of this CTA
-            // pass 1: row maximum
-            float mx = -INFINITY;
+            float s[TK];
 #pragma unroll
-            for (int c = 0; c < TK / 32; ++c) {
-                uint32_t r[32];
-                tmem_ld_32x32(s_addr + c * 32, r);
-                tmem_ld_wait();
+            for (int c = 0; c < TK / 32; ++c)
+                tmem_ld_32x32(s_addr + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
+            tmem_ld_wait();
+            if (j * TK + TK - 1 > a.pos0 + tile_q0) {         // tile holds keys beyond some query of this tile
 #pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    float s = __uint_as_float(r[i]);
-                    if (diag && j * TK + c * 32 + i > qpos) s = -INFINITY;
-                    mx = fmaxf(mx, s);
-                }
+                for (int i = 0; i < TK; ++i)
+                    if (j * TK + i > qpos) s[i] = -INFINITY;
             }
-            const float m_new = fmaxf(m, mx);                 // finite: key 0 is visible to every query
-            const float corr = ex2_approx((m - m_new) * sl2);
-            const float ms = m_new * sl2;
-            // pass 2: probabilities, packed to bf16 over the scores they came from
-            float sum = 0.f;
+            float mx = max3f(s[0], s[1], s[2]);
 #pragma unroll
-            for (int c = 0; c < TK / 32; ++c) {
-                uint32_t r[32];
-                tmem_ld_32x32(s_addr + c * 32, r);
-                tmem_ld_wait();
-                uint32_t pk[16];
+            for (int i = 3; i + 1 < TK; i += 2) mx = max3f(mx, s[i], s[i + 1]);
+            mx = fmaxf(mx, s[TK - 1]);
+            if (j == 0) {
+                m_used = mx;                                  // finite: key 0 is visible to every query
+            } else {
+                const bool raise = (mx - m_used) * sl2 > RESCALE_LOG2;
+                if (__any_sync(0xFFFFFFFFu, raise)) {
+                    // O_w must hold every product issued so far before its rows are rescaled
+                    ok = mbar_wait(pv_done + w, (j - 1) & 1, abort_flag);
+                    ok = __all_sync(0xFFFFFFFFu, ok);
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                    const float f = raise ? ex2_approx((m_used - mx) * sl2) : 1.0f;
 #pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                    float s0 = __uint_as_float(r[2 * i]), s1 = __uint_as_float(r[2 * i + 1]);
-                    if (diag) {
-                        if (j * TK + c * 32 + 2 * i > qpos) s0 = -INFINITY;
-                        if (j * TK + c * 32 + 2 * i + 1 > qpos) s1 = -INFINITY;
+                    for (int c = 0; c < HD / 32; ++c) {
+                        uint32_t r[32];
+                        tmem_ld_32x32(o_addr + c * 32, r);
+                        tmem_ld_wait();
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * f);
+                        tmem_st_32x32(o_addr + c * 32, r);
                     }
-                    const float p0 = ex2_approx(fmaf(s0, sl2, -ms));
-                    const float p1 = ex2_approx(fmaf(s1, sl2, -ms));
-                    sum += p0 + p1;
-                    pk[i] = pack_bf16x2(p0, p1);
+                    l *= f;
+                    if (raise) m_used = mx;
                 }
-                tmem_st_32x16(s_addr + c * 16, pk);
             }
+            const float neg_ms = -m_used * sl2;
+            float sum0 = 0.f, sum1 = 0.f;
+            uint32_t pk[TK / 2];
+#pragma unroll
+            for (int i = 0; i < TK / 2; ++i) {
+                float x0 = s[2 * i], x1 = s[2 * i + 1];
+                fma2(x0, x1, sl2, neg_ms);
+                x0 = ex2_approx(x0);
+                x1 = ex2_approx(x1);
+                sum0 += x0;
+                sum1 += x1;
+                pk[i] = pack_bf16x2(x0, x1);
+            }
+#pragma unroll
+            for (int c = 0; c < TK / 64; ++c)
+                tmem_st_32x32(s_addr + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&pk[c * 32]));
             tmem_st_wait();
             tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) mbar_arrive(p_ready + st);
-            l = l * corr + sum;
-            if (j > 0 && !(ok = add_product(j - 1))) break;
-#pragma unroll
-            for (int i = 0; i < HD; ++i) acc[i] *= corr;
-            m = m_new;
+            if (lane == 0) mbar_arrive(p_ready + w);
+            l += sum0 + sum1;
         }
-        if (ok && n_tiles > 0) ok = add_product(n_tiles - 1);
-        if (ok && row < rows_valid) {
+        if (ok && n_w > 0) {
+            ok = mbar_wait(pv_done + w, (n_w - 1) & 1, abort_flag);
+            ok = __all_sync(0xFFFFFFFFu, ok);
+        }
+        if (ok && n_w > 0) {
+            tc_fence_after_sync();
             const float inv = 1.f / l;
             const int d = a.n_head * HD;
-            uint16_t *dst = a.out + g * a.out_gstride + ((long long)b * a.seqlen + q0 + row) * d + h * HD;
+            uint16_t *dst = a.out + g * a.out_gstride + ((long long)b * a.seqlen + tile_q0 + row) * d + h * HD;
 #pragma unroll
-            for (int i = 0; i < HD / 8; ++i) {
-                uint4 u;
-                u.x = pack_bf16x2(acc[8 * i + 0] * inv, acc[8 * i + 1] * inv);
-                u.y = pack_bf16x2(acc[8 * i + 2] * inv, acc[8 * i + 3] * inv);
-                u.z = pack_bf16x2(acc[8 * i + 4] * inv, acc[8 * i + 5] * inv);
-                u.w = pack_bf16x2(acc[8 * i + 6] * inv, acc[8 * i + 7] * inv);
-                reinterpret_cast<uint4 *>(dst)[i] = u;
+            for (int c = 0; c < HD / 32; ++c) {
+                uint32_t r[32];
+                tmem_ld_32x32(o_addr + c * 32, r);
+                tmem_ld_wait();
+                if (row < rows_valid) {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        uint4 u;
+                        u.x = pack_bf16x2(__uint_as_float(r[8 * i + 0]) * inv, __uint_as_float(r[8 * i + 1]) * inv);
+                        u.y = pack_bf16x2(__uint_as_float(r[8 * i + 2]) * inv, __uint_as_float(r[8 * i + 3]) * inv);
+                        u.z = pack_bf16x2(__uint_as_float(r[8 * i + 4]) * inv, __uint_as_float(r[8 * i + 5]) * inv);
+                        u.w = pack_bf16x2(__uint_as_float(r[8 * i + 6]) * inv, __uint_as_float(r[8 * i + 7]) * inv);
+                        reinterpret_cast<uint4 *>(dst + c * 32)[i] = u;
+                    }
+                }
             }
         }
     }
@@ -327,7 +362,7 @@ int launch(const CUtensorMap &tmQ, const CUtensorMap &tmK, const CUtensorMap &tm
             return KRAKEN_ECUDA;
         configured = true;
     }
-    dim3 grid((a.seqlen + TQ - 1) / TQ, a.n_head, a.batch * a.groups);
+    dim3 grid((a.seqlen + 2 * TQ - 1) / (2 * TQ), a.n_head, a.batch * a.groups);
     attn_tc_kernel<HD><<<grid, ATC_THREADS, Cfg::SMEM_BYTES, stream>>>(tmQ, tmK, tmV, a);
     return cudaGetLastError() == cudaSuccess ? KRAKEN_OK : KRAKEN_ECUDA;
 }
