@@ -159,6 +159,8 @@ int kraken_profile_read(kraken_handle *h, double *ms, int64_t *launches);
 int kraken_reset(kraken_handle *h);
 void kraken_destroy(kraken_handle *h);
 const char *kraken_strerror(int status);
+/* Text of the most recent CUDA failure behind a KRAKEN_ECUDA on the calling thread ("" if none). */
+const char *kraken_last_cuda_error(void);
 
 /* ------------------------------------------------------------------------------------------
  * Single steps of the path, exposed so that each kernel can be checked on its own.  All

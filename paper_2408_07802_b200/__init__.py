@@ -31,7 +31,7 @@ PROF_COUNT = len(PROF_CATEGORIES)
 EXPORTS = (
     "kraken_query_sizes", "kraken_create", "kraken_prefill", "kraken_prefill_host",
     "kraken_prefill_all_logits", "kraken_logits_rows", "kraken_decode_step", "kraken_decode_step_host", "kraken_kv_view",
-    "kraken_device_status", "kraken_cur_len", "kraken_profile_enable", "kraken_profile_read", "kraken_reset", "kraken_destroy", "kraken_strerror",
+    "kraken_device_status", "kraken_cur_len", "kraken_profile_enable", "kraken_profile_read", "kraken_reset", "kraken_destroy", "kraken_strerror", "kraken_last_cuda_error",
     "kraken_op_embed", "kraken_op_layernorm", "kraken_op_grouped_gemm", "kraken_op_attention",
     "kraken_op_decode_attention", "kraken_decode_attention_sizes",
     "kraken_op_decode_attention_static", "kraken_decode_attention_static_capacity",
@@ -68,7 +68,8 @@ class GemmArgs(C.Structure):
 class KrakenError(RuntimeError):
     def __init__(self, status: int, what: str):
         self.status = status
-        super().__init__(f"{what}: {strerror(status)} ({status})")
+        detail = lib().kraken_last_cuda_error().decode() if status == ECUDA else ""
+        super().__init__(f"{what}: {strerror(status)} ({status})" + (f" [{detail}]" if detail else ""))
 
 
 _lib = None
@@ -103,6 +104,8 @@ def lib() -> C.CDLL:
         L.kraken_destroy.restype = None
         L.kraken_strerror.argtypes = [C.c_int]
         L.kraken_strerror.restype = C.c_char_p
+        L.kraken_last_cuda_error.argtypes = []
+        L.kraken_last_cuda_error.restype = C.c_char_p
         L.kraken_op_embed.argtypes = [vp, i32, i32, i32, vp, vp, i32, i32, vp, vp, vp]
         L.kraken_op_layernorm.argtypes = [vp, i64, vp, vp, vp, i32, i32, i32, C.c_float, vp, vp]
         L.kraken_op_grouped_gemm.argtypes = [C.POINTER(GemmArgs), vp, vp]

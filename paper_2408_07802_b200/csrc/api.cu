@@ -564,6 +564,8 @@ int kraken_profile_read(kraken_handle *h, double *ms, int64_t *launches) {
     return KRAKEN_OK;
 }
 
+const char *kraken_last_cuda_error(void) { return last_cuda_error(); }
+
 const char *kraken_strerror(int status) {
     switch (status) {
         case KRAKEN_OK: return "ok";

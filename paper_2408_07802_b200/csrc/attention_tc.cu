@@ -53,6 +53,16 @@ __device__ __forceinline__ uint64_t umma_desc_sw128_mnmajor(uint32_t smem_addr, 
     return d;
 }
 
+// 32 lanes x 16 columns store
+__device__ __forceinline__ void tmem_st_32x16(uint32_t taddr, const uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};" ::"r"(taddr),
+        "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+        "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+        : "memory");
+}
+
 __device__ __forceinline__ float max3f(float a, float b, float c) {
     float d;
     asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
@@ -267,51 +277,64 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
 #pragma unroll
             for (int i = 3; i + 1 < TK; i += 2) mx = max3f(mx, s[i], s[i + 1]);
             mx = fmaxf(mx, s[TK - 1]);
+            // raise the maximum in use only when the row's new maximum is far above it
+            bool raise = false;
+            float f = 1.0f;
             if (j == 0) {
                 m_used = mx;                                  // finite: key 0 is visible to every query
             } else {
-                const bool raise = (mx - m_used) * sl2 > RESCALE_LOG2;
-                if (__any_sync(0xFFFFFFFFu, raise)) {
-                    // O_w must hold every product issued so far before its rows are rescaled
-                    ok = mbar_wait(pv_done + w, (j - 1) & 1, abort_flag);
-                    ok = __all_sync(0xFFFFFFFFu, ok);
-                    if (!ok) break;
-                    tc_fence_after_sync();
-                    const float f = raise ? ex2_approx((m_used - mx) * sl2) : 1.0f;
-#pragma unroll
-                    for (int c = 0; c < HD / 32; ++c) {
-                        uint32_t r[32];
-                        tmem_ld_32x32(o_addr + c * 32, r);
-                        tmem_ld_wait();
-#pragma unroll
-                        for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * f);
-                        tmem_st_32x32(o_addr + c * 32, r);
-                    }
-                    l *= f;
-                    if (raise) m_used = mx;
+                raise = (mx - m_used) * sl2 > RESCALE_LOG2;
+                if (raise) {
+                    f = ex2_approx((m_used - mx) * sl2);
+                    m_used = mx;
                 }
             }
             const float neg_ms = -m_used * sl2;
-            float sum0 = 0.f, sum1 = 0.f;
-            uint32_t pk[TK / 2];
+            float sum0 = 0.f, sum1 = 0.f, sum2 = 0.f, sum3 = 0.f;
 #pragma unroll
-            for (int i = 0; i < TK / 2; ++i) {
-                float x0 = s[2 * i], x1 = s[2 * i + 1];
-                fma2(x0, x1, sl2, neg_ms);
-                x0 = ex2_approx(x0);
-                x1 = ex2_approx(x1);
-                sum0 += x0;
-                sum1 += x1;
-                pk[i] = pack_bf16x2(x0, x1);
+            for (int c = 0; c < TK / 32; ++c) {
+                uint32_t pk[16];
+#pragma unroll
+                for (int i = 0; i < 16; i += 2) {
+                    float x0 = s[c * 32 + 2 * i], x1 = s[c * 32 + 2 * i + 1];
+                    float x2 = s[c * 32 + 2 * i + 2], x3 = s[c * 32 + 2 * i + 3];
+                    fma2(x0, x1, sl2, neg_ms);
+                    fma2(x2, x3, sl2, neg_ms);
+                    x0 = ex2_approx(x0);
+                    x1 = ex2_approx(x1);
+                    x2 = ex2_approx(x2);
+                    x3 = ex2_approx(x3);
+                    sum0 += x0;
+                    sum1 += x1;
+                    sum2 += x2;
+                    sum3 += x3;
+                    pk[i] = pack_bf16x2(x0, x1);
+                    pk[i + 1] = pack_bf16x2(x2, x3);
+                }
+                tmem_st_32x16(s_addr + c * 16, pk);   // overwrites scores already consumed
             }
+            l = l * f + ((sum0 + sum1) + (sum2 + sum3));
+            if (__any_sync(0xFFFFFFFFu, raise)) {
+                // (rare) O_w must hold every product issued so far before its rows are rescaled; the
+                // next product is not issued until this warp has released P below
+                ok = mbar_wait(pv_done + w, (j - 1) & 1, abort_flag);
+                ok = __all_sync(0xFFFFFFFFu, ok);
+                if (!ok) break;
+                tc_fence_after_sync();
+#pragma unroll 1
+                for (int c = 0; c < HD / 32; ++c) {
+                    uint32_t r[32];
+                    tmem_ld_32x32(o_addr + c * 32, r);
+                    tmem_ld_wait();
 #pragma unroll
-            for (int c = 0; c < TK / 64; ++c)
-                tmem_st_32x32(s_addr + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&pk[c * 32]));
+                    for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(__uint_as_float(r[i]) * f);
+                    tmem_st_32x32(o_addr + c * 32, r);
+                }
+            }
             tmem_st_wait();
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(p_ready + w);
-            l += sum0 + sum1;
         }
         if (ok && n_w > 0) {
             ok = mbar_wait(pv_done + w, (n_w - 1) & 1, abort_flag);
@@ -357,14 +380,14 @@ int launch(const CUtensorMap &tmQ, const CUtensorMap &tmK, const CUtensorMap &tm
     using Cfg = AtcCfg<HD>;
     static bool configured = false;
     if (!configured) {
-        if (cudaFuncSetAttribute(attn_tc_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES) !=
-            cudaSuccess)
-            return KRAKEN_ECUDA;
+        int rc = cuda_check(cudaFuncSetAttribute(attn_tc_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                 Cfg::SMEM_BYTES), "attention: shared memory opt-in");
+        if (rc) return rc;
         configured = true;
     }
     dim3 grid((a.seqlen + 2 * TQ - 1) / (2 * TQ), a.n_head, a.batch * a.groups);
     attn_tc_kernel<HD><<<grid, ATC_THREADS, Cfg::SMEM_BYTES, stream>>>(tmQ, tmK, tmV, a);
-    return cudaGetLastError() == cudaSuccess ? KRAKEN_OK : KRAKEN_ECUDA;
+    return cuda_check(cudaGetLastError(), "attention: launch");
 }
 
 }  // namespace

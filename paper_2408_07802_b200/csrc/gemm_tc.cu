@@ -238,13 +238,13 @@ int launch_bn(const CUtensorMap &tmA, const CUtensorMap &tmB, const KernelArgs &
     using Cfg = TileCfg<BN>;
     static bool configured = false;
     if (!configured) {
-        if (cudaFuncSetAttribute(gemm_tc_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES) !=
-            cudaSuccess)
-            return KRAKEN_ECUDA;
+        int rc = cuda_check(cudaFuncSetAttribute(gemm_tc_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                 Cfg::SMEM_BYTES), "gemm: shared memory opt-in");
+        if (rc) return rc;
         configured = true;
     }
     gemm_tc_kernel<BN><<<grid, NUM_THREADS, Cfg::SMEM_BYTES, stream>>>(tmA, tmB, ka);
-    return cudaGetLastError() == cudaSuccess ? KRAKEN_OK : KRAKEN_ECUDA;
+    return cuda_check(cudaGetLastError(), "gemm: launch");
 }
 
 }  // namespace

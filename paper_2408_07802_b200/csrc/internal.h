@@ -116,5 +116,8 @@ size_t decode_attention_partial_bytes(int groups, int batch, int n_head, int hea
 int launch_attention_decode(const DecodeAttnParams &p, cudaStream_t stream);
 
 bool env_flag(const char *name);
+// Records the text of a failed CUDA call (per thread) and maps it to KRAKEN_ECUDA.
+int cuda_check(cudaError_t e, const char *where);
+const char *last_cuda_error();
 
 }  // namespace kr

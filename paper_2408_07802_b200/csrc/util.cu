@@ -1,4 +1,5 @@
 // Host utilities: tensor-map encoding through the driver entry point, device queries, env flags.
+#include <stdio.h>
 #include <stdlib.h>
 #include <string.h>
 
@@ -72,6 +73,16 @@ int sm_count() {
     }
     return n;
 }
+
+static thread_local char g_last_error[256] = "";
+
+int cuda_check(cudaError_t e, const char *where) {
+    if (e == cudaSuccess) return KRAKEN_OK;
+    snprintf(g_last_error, sizeof(g_last_error), "%s: %s", where, cudaGetErrorString(e));
+    return KRAKEN_ECUDA;
+}
+
+const char *last_cuda_error() { return g_last_error; }
 
 bool env_flag(const char *name) {
     const char *v = getenv(name);
