@@ -97,7 +97,7 @@ def test_c0_prefill_parity_all_positions_and_cache():
     check_parity(got_all, ref32, refbf, "C0 all positions")
     # the call the benchmark times returns the last position of that same computation
     last = m.prefill(tok).cpu().numpy()
-    assert np.allclose(last[0], got_all[-1], atol=1e-5)
+    assert np.allclose(last[0], got_all[-1], atol=3e-4)
     assert m.device_status() == 0 and m.cur_len == s.seqlen
     # KV cache: the bf16 k, v rows, in [batch, head, position, dim] order
     worst = 0
@@ -240,8 +240,10 @@ def test_c1_full_parity():
     ref32, _ = oracle_all_logits(s, wb, tok[0].cpu().numpy(), False)
     refbf, _ = oracle_all_logits(s, wb, tok[0].cpu().numpy(), True)
     check_parity(got, ref32, refbf, "C1 all positions")
+    # (the few-row tail runs on the weight-streaming GEMM, all positions on the tile GEMM: the two
+    # add the same products in a different order)
     last = m.prefill(tok).cpu().numpy()
-    assert np.allclose(last[0], got[-1], atol=1e-5)
+    assert np.allclose(last[0], got[-1], atol=3e-4)
 
 
 def prefix_parity(name, prefix, seqs):
