@@ -233,6 +233,248 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     if (warp == 1) tmem_dealloc(tmem_base, Cfg::TMEM_COLS);
 }
 
+// ------------------------------------------------------------------------------------------------
+// CTA-pair version: two CTAs of a cluster work on one 256 x 256 output tile.  Each CTA loads its 128
+// rows of A and HALF of the W tile (128 rows), the leader issues tcgen05.mma.cta_group::2 (256 x 256
+// x 16), and each CTA's tensor core reads both halves of W, so every W byte is fetched into shared
+// memory once per pair instead of once per CTA: a third less shared-memory traffic per flop, which
+// is what bounds the single-CTA 128 x 256 tile.  Each CTA drains its own 128 accumulator rows.
+// Barriers: `full` lives in the leader (both CTAs' TMA loads report their bytes to it), `empty` and
+// `acc_full` exist in both CTAs and are signalled by multicast commits, `acc_empty` lives in the
+// leader and collects the epilogue warps of both CTAs.
+// ------------------------------------------------------------------------------------------------
+
+constexpr int BN2 = 256;
+
+struct PairCfg {
+    static constexpr int A_BYTES = BM * BK * 2;            // 128 rows of A
+    static constexpr int B_BYTES = (BN2 / 2) * BK * 2;     // this CTA's half of the W tile
+    static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+    static constexpr int STAGES = 6;
+    static constexpr int TMEM_COLS = 2 * BN2;
+    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 256;
+};
+
+__device__ __forceinline__ bool next_item_pair(const KernelArgs &ka, int it, int cluster_id, int n_clusters,
+                                               int &m_blk, int &n_blk, int &g) {
+    const int G = ka.shape.groups;
+    const int tiles_m = (ka.shape.m + 2 * BM - 1) / (2 * BM);
+    const int num_tiles = tiles_m * ka.tiles_n;
+    int tile;
+    if (ka.group_serial) {
+        tile = cluster_id + (it / G) * n_clusters;
+        g = it % G;
+    } else {
+        const long long idx = cluster_id + (long long)it * n_clusters;
+        g = static_cast<int>(idx / num_tiles);
+        if (g >= G) return false;
+        tile = static_cast<int>(idx % num_tiles);
+    }
+    if (tile >= num_tiles) return false;
+    if (ka.n_fastest) {
+        n_blk = tile % ka.tiles_n;
+        m_blk = tile / ka.tiles_n;
+    } else {
+        m_blk = tile % tiles_m;
+        n_blk = tile / tiles_m;
+    }
+    return true;
+}
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
+gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                    const KernelArgs ka) {
+    using Cfg = PairCfg;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t *tiles = smem;
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem + Cfg::STAGES * Cfg::STAGE_BYTES);
+    uint64_t *full_bar = bars;                         // [STAGES]  used in the leader
+    uint64_t *empty_bar = bars + Cfg::STAGES;          // [STAGES]  both CTAs
+    uint64_t *acc_full = bars + 2 * Cfg::STAGES;       // [2]       both CTAs
+    uint64_t *acc_empty = bars + 2 * Cfg::STAGES + 2;  // [2]       used in the leader
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 2 * Cfg::STAGES + 4);
+    volatile uint32_t *abort_flag = tmem_slot + 1;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();
+    const int cluster_id = blockIdx.x >> 1, n_clusters = gridDim.x >> 1;
+    const int k_blocks = (ka.shape.k + BK - 1) / BK;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < Cfg::STAGES; ++s) {
+            mbar_init(full_bar + s, 1);
+            mbar_init(empty_bar + s, 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(acc_full + a, 1);
+            mbar_init(acc_empty + a, 2 * EPI_WARPS);
+        }
+        *abort_flag = 0;
+        fence_barrier_init();
+        prefetch_tensormap(&tmA);
+        prefetch_tensormap(&tmB);
+    }
+    if (warp == 1) {
+        tmem_alloc_pair(tmem_slot, Cfg::TMEM_COLS);
+        tmem_relinquish_pair();
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    cluster_sync_all();  // both CTAs' barriers exist before anything is signalled across the pair
+    tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            int stage = 0;
+            uint32_t phase = 0;
+            bool ok = true;
+            int m_blk, n_blk, g;
+            for (int it = 0; ok && next_item_pair(ka, it, cluster_id, n_clusters, m_blk, n_blk, g); ++it) {
+                for (int kb = 0; kb < k_blocks; ++kb) {
+                    if (!(ok = mbar_wait(empty_bar + stage, phase ^ 1u, abort_flag))) break;
+                    uint8_t *sa = tiles + stage * Cfg::STAGE_BYTES;
+                    uint8_t *sb = sa + Cfg::A_BYTES;
+                    const uint32_t leader_full = map_to_cta(smem_u32(full_bar + stage), 0);
+                    if (rank == 0) mbar_expect_tx(full_bar + stage, 2 * Cfg::STAGE_BYTES);
+                    tma_load_3d_pair(sa, &tmA, leader_full, kb * BK, m_blk * 2 * BM + (int)rank * BM,
+                                     ka.a_g0 + g * ka.a_gmul);
+                    tma_load_3d_pair(sb, &tmB, leader_full, kb * BK, n_blk * BN2 + (int)rank * (BN2 / 2),
+                                     ka.b_g0 + g * ka.b_gmul);
+                    if (++stage == Cfg::STAGES) {
+                        stage = 0;
+                        phase ^= 1u;
+                    }
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        if (lane == 0 && rank == 0) {
+            constexpr uint32_t idesc = umma_idesc_bf16(2 * BM, BN2);
+            int stage = 0;
+            uint32_t phase = 0;
+            int acc = 0;
+            uint32_t acc_phase = 0;
+            bool ok = true;
+            int m_blk, n_blk, g;
+            for (int it = 0; ok && next_item_pair(ka, it, cluster_id, n_clusters, m_blk, n_blk, g); ++it) {
+                if (!(ok = mbar_wait(acc_empty + acc, acc_phase ^ 1u, abort_flag))) break;
+                tc_fence_after_sync();
+                const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * BN2);
+                for (int kb = 0; kb < k_blocks; ++kb) {
+                    if (!(ok = mbar_wait(full_bar + stage, phase, abort_flag))) break;
+                    tc_fence_after_sync();
+                    const uint32_t sa = smem_u32(tiles + stage * Cfg::STAGE_BYTES);
+                    const uint32_t sb = sa + Cfg::A_BYTES;
+#pragma unroll
+                    for (int k = 0; k < BK / UMMA_K; ++k) {
+                        umma_bf16_ss_pair(d_tmem, umma_desc_sw128_kmajor(sa + k * UMMA_K * 2),
+                                          umma_desc_sw128_kmajor(sb + k * UMMA_K * 2), idesc,
+                                          (kb | k) != 0 ? 1u : 0u);
+                    }
+                    umma_commit_pair(empty_bar + stage, 3);  // frees the stage in both CTAs
+                    if (++stage == Cfg::STAGES) {
+                        stage = 0;
+                        phase ^= 1u;
+                    }
+                }
+                if (!ok) break;
+                umma_commit_pair(acc_full + acc, 3);  // accumulator complete in both CTAs
+                if (++acc == 2) {
+                    acc = 0;
+                    acc_phase ^= 1u;
+                }
+            }
+        }
+        __syncwarp();
+    } else {
+        const int quarter = warp & 3;
+        const int half = (warp - 2) >> 2;
+        constexpr int CHUNKS = BN2 / 32 / 2;
+        int acc = 0;
+        uint32_t acc_phase = 0;
+        bool ok = true;
+        int m_blk, n_blk, g;
+        for (int it = 0; ok && next_item_pair(ka, it, cluster_id, n_clusters, m_blk, n_blk, g); ++it) {
+            ok = mbar_wait(acc_full + acc, acc_phase, abort_flag);
+            ok = __all_sync(0xFFFFFFFFu, ok);
+            if (!ok) break;
+            tc_fence_after_sync();
+            const int row = m_blk * 2 * BM + (int)rank * BM + quarter * 32 + lane;
+            const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
+                                   static_cast<uint32_t>(acc * BN2);
+#pragma unroll 1
+            for (int cc = 0; cc < CHUNKS; ++cc) {
+                const int c = half * CHUNKS + cc;
+                const int col0 = n_blk * BN2 + c * 32;
+                if (col0 >= ka.shape.n_out) break;
+                uint32_t r[32];
+                tmem_ld_32x32(t_row + static_cast<uint32_t>(c * 32), r);
+                tmem_ld_wait();
+                if (row < ka.shape.m) {
+                    float v[32];
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+                    const int ncols = min(32, ka.shape.n_out - col0);
+                    epilogue_chunk(ka.epi, g, row, col0, ncols, v);
+                }
+            }
+            tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(map_to_cta(smem_u32(acc_empty + acc), 0));
+            if (++acc == 2) {
+                acc = 0;
+                acc_phase ^= 1u;
+            }
+        }
+    }
+
+    if (*abort_flag) {
+        for (int i = 0; i < 64; ++i) __nanosleep(10000);
+        if (threadIdx.x == 0 && ka.status) atomicOr(ka.status, STATUS_WAIT_LIMIT);
+    }
+    tc_fence_before_sync();
+    __syncthreads();
+    cluster_sync_all();  // nothing of the pair (remote arrivals, MMA reads of peer memory) is in flight
+    if (warp == 1) tmem_dealloc_pair(tmem_base, Cfg::TMEM_COLS);
+}
+
+int launch_pair(const CUtensorMap &tmA, const CUtensorMap &tmB, const KernelArgs &ka, cudaStream_t stream) {
+    using Cfg = PairCfg;
+    static bool configured = false;
+    static int max_clusters = 0;
+    if (!configured) {
+        int rc = cuda_check(cudaFuncSetAttribute(gemm_tc_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                 Cfg::SMEM_BYTES), "gemm pair: shared memory opt-in");
+        if (rc) return rc;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(2 * 148);
+        cfg.blockDim = dim3(NUM_THREADS);
+        cfg.dynamicSmemBytes = Cfg::SMEM_BYTES;
+        cudaLaunchAttribute attr;
+        attr.id = cudaLaunchAttributeClusterDimension;
+        attr.val.clusterDim.x = 2;
+        attr.val.clusterDim.y = 1;
+        attr.val.clusterDim.z = 1;
+        cfg.attrs = &attr;
+        cfg.numAttrs = 1;
+        int n = 0;
+        if (cudaOccupancyMaxActiveClusters(&n, gemm_tc_pair_kernel, &cfg) != cudaSuccess || n < 1) {
+            cudaGetLastError();
+            n = (sm_count() > 0 ? sm_count() : 148) / 2;
+        }
+        max_clusters = n;
+        configured = true;
+    }
+    const long long tiles = (long long)((ka.shape.m + 2 * BM - 1) / (2 * BM)) * ka.tiles_n;
+    const long long units = ka.group_serial ? tiles : tiles * ka.shape.groups;
+    const int clusters = static_cast<int>(units < max_clusters ? units : max_clusters);
+    gemm_tc_pair_kernel<<<2 * clusters, NUM_THREADS, Cfg::SMEM_BYTES, stream>>>(tmA, tmB, ka);
+    return cuda_check(cudaGetLastError(), "gemm pair: launch");
+}
+
 template <int BN>
 int launch_bn(const CUtensorMap &tmA, const CUtensorMap &tmB, const KernelArgs &ka, int grid, cudaStream_t stream) {
     using Cfg = TileCfg<BN>;
@@ -252,6 +494,11 @@ int launch_bn(const CUtensorMap &tmA, const CUtensorMap &tmB, const KernelArgs &
 int gemm_pick_bn(const GemmShape &s) {
     const int sms = sm_count() > 0 ? sm_count() : 148;
     const long long tiles_m = (s.m + BM - 1) / BM;
+    // CTA pairs on 256 x 256 tiles when that still gives every pair of SMs about two work items
+    {
+        const long long items = ((s.m + 2 * BM - 1) / (2 * BM)) * ((s.n_out + BN2 - 1) / BN2) * s.groups;
+        if (items >= sms && !env_flag("KRAKEN_GEMM_NO_PAIR")) return GEMM_TILE_PAIR;
+    }
     // Largest N tile that still gives every SM about one work item.
     for (int bn : {256, 128}) {
         const long long items = tiles_m * ((s.n_out + bn - 1) / bn) * s.groups;
@@ -267,6 +514,7 @@ int gemm_encode_a(CUtensorMap *map, const GemmOperands &op, const GemmShape &s) 
 }
 
 int gemm_encode_b(CUtensorMap *map, const GemmOperands &op, const GemmShape &s, int bn) {
+    if (bn == GEMM_TILE_PAIR) bn = BN2 / 2;  // each CTA of a pair loads half of the 256-row W tile
     const bool shared = op.w_gstride == 0 || s.groups == 1;
     return encode_tma_3d_bf16(map, op.w, s.k, s.n_out, shared ? 1 : s.groups, op.ldw,
                               shared ? (uint64_t)op.ldw * s.n_out : (uint64_t)op.w_gstride, BK, bn);
@@ -294,13 +542,15 @@ int launch_gemm_tc(const GemmOperands &op, const GemmShape &s, const EpiParams &
     ka.shape = s;
     ka.epi = epi;
     ka.tiles_m = (s.m + BM - 1) / BM;
-    ka.tiles_n = (s.n_out + bn - 1) / bn;
+    const int bn_cols = bn == GEMM_TILE_PAIR ? BN2 : bn;
+    ka.tiles_n = (s.n_out + bn_cols - 1) / bn_cols;
     ka.a_gmul = (op.a_gstride == 0 || s.groups == 1) ? 0 : 1;
     ka.b_gmul = (op.w_gstride == 0 || s.groups == 1) ? 0 : 1;
     ka.a_g0 = 0;
     ka.b_g0 = b_g0;
     ka.group_serial = epi.kind == KRAKEN_EPI_RESID_SUM ? 1 : 0;
     ka.n_fastest = (ka.group_serial && ka.tiles_n <= ka.tiles_m) ? 1 : 0;
+    if (bn == GEMM_TILE_PAIR) return launch_pair(*tmA, *tmB, ka, stream);
     ka.status = d_status;
     const long long tiles = (long long)ka.tiles_m * ka.tiles_n;
     const long long units = ka.group_serial ? tiles : tiles * s.groups;

@@ -55,7 +55,9 @@ struct GemmOperands {
 };
 int launch_gemm_tc(const GemmOperands &op, const GemmShape &shape, const EpiParams &epi, const CUtensorMap *tmA,
                    const CUtensorMap *tmB, int b_g0, int bn_hint, uint32_t *d_status, cudaStream_t stream);
-// Picks the N tile for a shape (64, 128 or 256).
+// Picks the N tile for a shape: 64, 128 or 256 (one CTA per 128-row tile), or GEMM_TILE_PAIR
+// (two CTAs of a cluster share a 256 x 256 tile).
+constexpr int GEMM_TILE_PAIR = 512;
 int gemm_pick_bn(const GemmShape &shape);
 int gemm_encode_a(CUtensorMap *map, const GemmOperands &op, const GemmShape &shape);
 int gemm_encode_b(CUtensorMap *map, const GemmOperands &op, const GemmShape &shape, int bn);
