@@ -77,7 +77,13 @@ def run_case(kind: str, workload: str, reps: int, warmup: int, n_tile: int = 0, 
     hd = d // H
     T = batch * seqlen
     status = torch.zeros(1, dtype=torch.int32, device=DEV)
-    if kind.startswith("gemm_"):
+    if kind.startswith("decode_gemm_"):
+        # the same projection with one row per sequence (decode step): weight streaming
+        g, keep, flops, byts = _gemm_args(kind.replace("decode_", ""), s, batch, 1, 8)
+        if g.epilogue == kr.EPI_RESID_SUM:
+            g.epilogue = kr.EPI_RESID_F32
+        fn = lambda: kr.op_grouped_gemm(g, status)
+    elif kind.startswith("gemm_"):
         g, keep, flops, byts = _gemm_args(kind, s, batch, seqlen, n_tile)
         fn = lambda: kr.op_grouped_gemm(g, status)
     elif kind == "attention":
@@ -128,7 +134,7 @@ def run_case(kind: str, workload: str, reps: int, warmup: int, n_tile: int = 0, 
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("case", help="gemm_qkv | gemm_proj | gemm_up | gemm_down | attention | layernorm | decode_attention | all")
+    ap.add_argument("case", help="gemm_qkv | gemm_proj | gemm_up | gemm_down | attention | layernorm | decode_attention | decode_gemm_{qkv,proj,up,down} | all | decode_all")
     ap.add_argument("--workload", default="C3")
     ap.add_argument("--reps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=2)
@@ -136,7 +142,11 @@ def main():
     ap.add_argument("--batch", type=int, default=None)
     ap.add_argument("--seqlen", type=int, default=None)
     a = ap.parse_args()
-    kinds = ["gemm_qkv", "gemm_proj", "gemm_up", "gemm_down", "attention", "layernorm"] if a.case == "all" else [a.case]
+    kinds = [a.case]
+    if a.case == "all":
+        kinds = ["gemm_qkv", "gemm_proj", "gemm_up", "gemm_down", "attention", "layernorm"]
+    elif a.case == "decode_all":
+        kinds = ["decode_gemm_qkv", "decode_gemm_proj", "decode_gemm_up", "decode_gemm_down", "decode_attention"]
     for k in kinds:
         run_case(k, a.workload, a.reps, a.warmup, a.n_tile, a.batch, a.seqlen)
 

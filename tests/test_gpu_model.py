@@ -281,3 +281,43 @@ def test_c2_full_size_prefix_parity():
 
 def test_c3_full_size_prefix_parity():
     prefix_parity("C3", 32, [0, 3])
+
+
+def test_c4_full_size_prefill_prefix_parity_and_decode_consistency():
+    """C4 at full size (16 sequences x 2048 tokens, then decode steps), in the launch configuration
+    the benchmark times.  Prefill: logits and cache rows of a prefix against an oracle run on that
+    prefix (causality).  Decode: a property that holds at any size - prefill(l) followed by one decode
+    step equals prefill(l + 1) at the last position - plus the cache row the step appended."""
+    s = ki.CONFIGS["C4"]
+    m, w = build(s)
+    wb = host_bits(w)
+    tok = ki.uniform_tokens(1, s.vocab, s.batch, s.seqlen + 1, DEV)
+    first = tok[:, :s.seqlen].contiguous()
+    last = m.prefill(first)
+    assert torch.isfinite(last).all() and m.device_status() == 0
+    prefix = 48
+    for b in (0, s.batch - 1):
+        got = m.logits_rows([b * s.seqlen + t for t in range(prefix)]).cpu().numpy()
+        ids = first[b, :prefix].cpu().numpy()
+        ref32, _ = oracle_all_logits(s, wb, ids, False)
+        refbf, orc = oracle_all_logits(s, wb, ids, True)
+        check_parity(got, ref32, refbf, f"C4 seq {b} first {prefix} positions of the full-size prefill")
+        for layer in (0, s.n_layer - 1):
+            for which in (0, 1):
+                g = m.kv_view(layer, 1, which)[b, :, :prefix].float().cpu().numpy()
+                check_cache(g, orc.cache(layer, 1, which), layer == 0, ("C4", b, layer, which))
+    # decode step at full context against a prefill of one more token
+    step = m.decode_step(tok[:, s.seqlen].contiguous()).cpu().numpy()
+    assert m.cur_len == s.seqlen + 1 and m.device_status() == 0
+    k_after = m.kv_view(s.n_layer - 1, 2, 0)[:, :, s.seqlen].float().cpu().numpy()
+    v_after = m.kv_view(0, 3, 1)[:, :, s.seqlen].float().cpu().numpy()
+    m.reset()
+    longer = m.prefill(tok).cpu().numpy()
+    rel, mx = logits_metrics(step, longer)
+    print(f"[parity] C4 decode step at context {s.seqlen} vs prefill({s.seqlen + 1}): relL2={rel:.3e} maxabs={mx:.3e}")
+    assert rel <= 5e-3 and mx <= 3e-2, (rel, mx)
+    k_ref = m.kv_view(s.n_layer - 1, 2, 0)[:, :, s.seqlen].float().cpu().numpy()
+    v_ref = m.kv_view(0, 3, 1)[:, :, s.seqlen].float().cpu().numpy()
+    assert np.abs(k_after - k_ref).max() <= 0.05 * np.abs(k_ref).max()
+    assert np.array_equal(v_after, v_ref)      # first layer: same inputs, same arithmetic order per row
+    m.close()
