@@ -315,7 +315,7 @@ def test_c4_full_size_prefill_prefix_parity_and_decode_consistency():
     longer = m.prefill(tok).cpu().numpy()
     rel, mx = logits_metrics(step, longer)
     print(f"[parity] C4 decode step at context {s.seqlen} vs prefill({s.seqlen + 1}): relL2={rel:.3e} maxabs={mx:.3e}")
-    assert rel <= 5e-3 and mx <= 3e-2, (rel, mx)
+    assert rel <= REL_L2_MAX and mx <= MAX_ABS_MAX, (rel, mx)   # two bf16 paths, each within the bound of the truth
     k_ref = m.kv_view(s.n_layer - 1, 2, 0)[:, :, s.seqlen].float().cpu().numpy()
     v_ref = m.kv_view(0, 3, 1)[:, :, s.seqlen].float().cpu().numpy()
     assert np.abs(k_after - k_ref).max() <= 0.05 * np.abs(k_ref).max()
