@@ -22,6 +22,15 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of ONE launch of the dominant kernel, from
+# the ncu captures summarised under profiles/ (layer-shaped launches of paper_2408_07802_b200.cases).
+NCU_TRAFFIC = {
+    "C3": {"bytes": 864.1e6, "launch": "FFN up-projection (4 x 8192 x 8192 x 2048)", "algorithmic_bytes": 805.3e6,
+           "source": "profiles/gemm_tc_pair_kernel_C3_gemm_up.md"},
+    "C4": {"bytes": 541.3e6, "launch": "decode attention of one layer (1024 streams x 2048 keys)",
+           "algorithmic_bytes": 537.1e6, "source": "profiles/attn_decode_kernel_C4.md"},
+}
+
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 PAPER_CONTEXT = ("paper: 35.6% geomean TTFT speedup of Kraken over standard Transformers, TensorRT-LLM fp16 on "
                  "8xA100-40GB NVSwitch (another machine and other shapes: context, not a target)")
@@ -258,7 +267,8 @@ def run_decode(args, shape, kr, ki, replicas, torch):
                      "bytes_per_launch": kv_per_layer, "launches_per_step": attn_launch,
                      "avg_launch_ms": attn_ms / shape.n_layer,
                      "timed_in": "separate pass of the same steps with events around every launch",
-                     "traffic": None},
+                     "traffic": NCU_TRAFFIC.get(shape.name, {}).get("bytes"),
+                     "traffic_note": NCU_TRAFFIC.get(shape.name)},
         "weight_streaming": {"ms_per_step": gemm_ms, "gbs": wb_ / (gemm_ms * 1e-3) / 1e9 if gemm_ms > 0 else 0.0},
         "kernels": kernels, "device_status": status,
     }
@@ -431,12 +441,14 @@ def main():
         "e2e": {"value": e2e_value, "unit": "tokens/s", "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": tokens * 4, "d2h_bytes_per_step": shape.batch * shape.vocab * 4},
         "gpu_launches": gpu_launches,
-        "roofline": {"bound": "tensor", "kernel": "gemm_tc_kernel (grouped tcgen05 GEMM: qkv, proj, up, down)",
+        "roofline": {"bound": "tensor", "kernel": "gemm_tc_pair_kernel / gemm_tc_kernel (grouped tcgen05 GEMM: qkv, proj, up, down)",
                      "achieved": achieved, "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
                      "peak_source": f"bf16_tflops_sustained of {peak_kind}",
                      "launches_per_step": int(gemm_launches), "avg_launch_ms": gemm_ms / max(1, gemm_launches),
                      "flops_per_step": fl["gemm"], "timed_in": "separate pass of the same K steps with events "
-                     "around every launch", "traffic": None},
+                     "around every launch",
+                     "traffic": NCU_TRAFFIC.get(shape.name, {}).get("bytes"),
+                     "traffic_note": NCU_TRAFFIC.get(shape.name)},
         "kernels": kernels,
         "device_status": status,
     }
