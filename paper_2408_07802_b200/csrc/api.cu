@@ -217,7 +217,11 @@ int run_layers(const RunCtx &rc, const int32_t *d_tokens) {
     const kraken_config &c = h->cfg;
     const int d = c.d_model, F = c.d_ff, N = c.n_branch, L = c.n_layer, H = c.n_head, hd = d / H, T = rc.T;
     const long long td = (long long)T * d;
-    const bool small_rows = T <= SKINNY_MAX_ROWS && !h->naive;
+    // The down-projection's epilogue can form the cross-branch sum only by running the N groups of an
+    // output tile on one CTA (pair); with too few output tiles that would idle most SMs, so then (and in
+    // decode) LayerNorm-2 of the next layer sums the N branch inputs itself, in the same order.
+    const long long down_tiles = (long long)((T + 255) / 256) * ((d + 255) / 256);
+    const bool small_rows = !h->naive && (T <= SKINNY_MAX_ROWS || down_tiles < (sm_count() > 0 ? sm_count() : 148) / 2);
     float *x0 = at<float>(h, h->lay.x0), *x = at<float>(h, h->lay.x), *a = at<float>(h, h->lay.a),
           *S = at<float>(h, h->lay.s);
     uint16_t *u = at<uint16_t>(h, h->lay.u), *q = at<uint16_t>(h, h->lay.q), *o = at<uint16_t>(h, h->lay.o),

@@ -27,6 +27,29 @@ __device__ __forceinline__ float gelu_f(float x, int tanh_form) {
     return 0.5f * x * (1.0f + erf_as(x * 0.7071067811865476f));
 }
 
+// GELU (erf form) of two values at once on the packed fp32 pipe; same formula as erf_as.
+__device__ __forceinline__ void gelu_erf_pair(float &x0, float &x1) {
+    const uint64_t x = pk2(x0, x1);
+    const uint64_t z = mul2(x, splat2(0.7071067811865476f));
+    const uint64_t az = z & 0x7FFFFFFF7FFFFFFFull;
+    float d0, d1;
+    upk2(fma2(az, splat2(0.3275911f), splat2(1.0f)), d0, d1);
+    const uint64_t t = pk2(rcp_approx(d0), rcp_approx(d1));
+    // -(a1 t + a2 t^2 + a3 t^3 + a4 t^4 + a5 t^5)
+    uint64_t poly = fma2(t, splat2(-1.061405429f), splat2(1.453152027f));
+    poly = fma2(poly, t, splat2(-1.421413741f));
+    poly = fma2(poly, t, splat2(0.284496736f));
+    poly = fma2(poly, t, splat2(-0.254829592f));
+    poly = mul2(poly, t);
+    float e0, e1;
+    upk2(mul2(mul2(az, az), splat2(-1.4426950408889634f)), e0, e1);
+    const uint64_t e = pk2(ex2_approx(e0), ex2_approx(e1));
+    uint64_t erf = fma2(poly, e, splat2(1.0f));                  // erf(|z|) >= 0
+    erf |= z & 0x8000000080000000ull;                            // sign of z
+    const uint64_t phi = fma2(erf, splat2(0.5f), splat2(0.5f));
+    upk2(mul2(x, phi), x0, x1);
+}
+
 __device__ __forceinline__ void store_bf16_chunk(uint16_t *dst, const float (&v)[32], int ncols) {
     if (ncols == 32 && (reinterpret_cast<uintptr_t>(dst) & 15u) == 0) {
         uint4 *d4 = reinterpret_cast<uint4 *>(dst);
@@ -112,8 +135,13 @@ __device__ __forceinline__ void epilogue_chunk(const EpiParams &p, int g, int ro
             store_bf16_chunk(p.out_bf16 + g * p.out_bf16_gstride + (long long)row * p.ld_out_bf16 + col0, v, ncols);
             break;
         case KRAKEN_EPI_GELU_BF16:
+            if (p.gelu_tanh) {
 #pragma unroll
-            for (int i = 0; i < 32; ++i) v[i] = gelu_f(v[i], p.gelu_tanh);
+                for (int i = 0; i < 32; ++i) v[i] = gelu_f(v[i], 1);
+            } else {
+#pragma unroll
+                for (int i = 0; i < 32; i += 2) gelu_erf_pair(v[i], v[i + 1]);
+            }
             store_bf16_chunk(p.out_bf16 + g * p.out_bf16_gstride + (long long)row * p.ld_out_bf16 + col0, v, ncols);
             break;
         case KRAKEN_EPI_RESID_F32:
