@@ -23,6 +23,8 @@ def _gemm_args(kind, s, batch, seqlen, n_tile=0):
     N, d, F, H = s.n_branch, s.d_model, s.d_ff, s.n_head
     hd = d // H
     T = batch * seqlen
+    plain = kind.endswith("_plain")       # same shape, cheapest epilogue (bf16 store): isolates the mainloop
+    kind = kind.replace("_plain", "")
     K, Nout = {"gemm_qkv": (d, 3 * d), "gemm_proj": (d, d), "gemm_up": (d, F), "gemm_down": (F, d)}[kind]
     a = ki.normal_bf16(11, 0, (N, T, K), 1.0, DEV)
     w = ki.normal_bf16(11, 1, (N, Nout, K), 0.02, DEV)
@@ -34,7 +36,13 @@ def _gemm_args(kind, s, batch, seqlen, n_tile=0):
     g.groups, g.m, g.n_out, g.k, g.n_tile = N, T, Nout, K, n_tile
     keep = [a, w, bias]
     out_bytes = 0
-    if kind == "gemm_qkv":
+    if plain:
+        o = torch.empty(N, T, Nout, dtype=torch.bfloat16, device=DEV)
+        g.epilogue = kr.EPI_BF16
+        g.out_bf16, g.out_bf16_gstride, g.ld_out_bf16 = o.data_ptr(), T * Nout, Nout
+        keep += [o]
+        out_bytes = N * T * Nout * 2
+    elif kind == "gemm_qkv":
         q = torch.empty(N, T, d, dtype=torch.bfloat16, device=DEV)
         cache = torch.empty(N, 2, batch, H, seqlen, hd, dtype=torch.bfloat16, device=DEV)
         g.epilogue = kr.EPI_QKV

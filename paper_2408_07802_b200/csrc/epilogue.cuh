@@ -50,8 +50,30 @@ __device__ __forceinline__ void gelu_erf_pair(float &x0, float &x1) {
     upk2(mul2(x, phi), x0, x1);
 }
 
+// 32-byte global accesses (sm_100): half as many memory instructions and L1 wavefronts per row as
+// 16-byte ones.  The address must be 32-byte aligned.
+__device__ __forceinline__ void st_global_32B(void *p, uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                              uint32_t a4, uint32_t a5, uint32_t a6, uint32_t a7) {
+    asm volatile("st.global.v8.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"l"(p), "r"(a0), "r"(a1), "r"(a2),
+                 "r"(a3), "r"(a4), "r"(a5), "r"(a6), "r"(a7)
+                 : "memory");
+}
+__device__ __forceinline__ void ld_global_32B(const void *p, float (&r)[8]) {
+    asm volatile("ld.global.v8.f32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=f"(r[0]), "=f"(r[1]), "=f"(r[2]), "=f"(r[3]), "=f"(r[4]), "=f"(r[5]), "=f"(r[6]), "=f"(r[7])
+                 : "l"(p)
+                 : "memory");
+}
+
 __device__ __forceinline__ void store_bf16_chunk(uint16_t *dst, const float (&v)[32], int ncols) {
-    if (ncols == 32 && (reinterpret_cast<uintptr_t>(dst) & 15u) == 0) {
+    if (ncols == 32 && (reinterpret_cast<uintptr_t>(dst) & 31u) == 0) {
+#pragma unroll
+        for (int i = 0; i < 2; ++i)
+            st_global_32B(dst + 16 * i, pack_bf16x2(v[16 * i + 0], v[16 * i + 1]), pack_bf16x2(v[16 * i + 2], v[16 * i + 3]),
+                          pack_bf16x2(v[16 * i + 4], v[16 * i + 5]), pack_bf16x2(v[16 * i + 6], v[16 * i + 7]),
+                          pack_bf16x2(v[16 * i + 8], v[16 * i + 9]), pack_bf16x2(v[16 * i + 10], v[16 * i + 11]),
+                          pack_bf16x2(v[16 * i + 12], v[16 * i + 13]), pack_bf16x2(v[16 * i + 14], v[16 * i + 15]));
+    } else if (ncols == 32 && (reinterpret_cast<uintptr_t>(dst) & 15u) == 0) {
         uint4 *d4 = reinterpret_cast<uint4 *>(dst);
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
@@ -70,7 +92,13 @@ __device__ __forceinline__ void store_bf16_chunk(uint16_t *dst, const float (&v)
 }
 
 __device__ __forceinline__ void store_f32_chunk(float *dst, const float (&v)[32], int ncols) {
-    if (ncols == 32 && (reinterpret_cast<uintptr_t>(dst) & 15u) == 0) {
+    if (ncols == 32 && (reinterpret_cast<uintptr_t>(dst) & 31u) == 0) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+            st_global_32B(dst + 8 * i, __float_as_uint(v[8 * i]), __float_as_uint(v[8 * i + 1]),
+                          __float_as_uint(v[8 * i + 2]), __float_as_uint(v[8 * i + 3]), __float_as_uint(v[8 * i + 4]),
+                          __float_as_uint(v[8 * i + 5]), __float_as_uint(v[8 * i + 6]), __float_as_uint(v[8 * i + 7]));
+    } else if (ncols == 32 && (reinterpret_cast<uintptr_t>(dst) & 15u) == 0) {
         float4 *d4 = reinterpret_cast<float4 *>(dst);
 #pragma unroll
         for (int i = 0; i < 8; ++i) d4[i] = make_float4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
@@ -82,7 +110,15 @@ __device__ __forceinline__ void store_f32_chunk(float *dst, const float (&v)[32]
 }
 
 __device__ __forceinline__ void add_f32_chunk(const float *src, float (&v)[32], int ncols) {
-    if (ncols == 32 && (reinterpret_cast<uintptr_t>(src) & 15u) == 0) {
+    if (ncols == 32 && (reinterpret_cast<uintptr_t>(src) & 31u) == 0) {
+        float t[4][8];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) ld_global_32B(src + 8 * i, t[i]);
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+            for (int j = 0; j < 8; ++j) v[8 * i + j] += t[i][j];
+    } else if (ncols == 32 && (reinterpret_cast<uintptr_t>(src) & 15u) == 0) {
         const float4 *s4 = reinterpret_cast<const float4 *>(src);
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
@@ -175,6 +211,86 @@ __device__ __forceinline__ void epilogue_chunk(const EpiParams &p, int g, int ro
         default:
             break;
     }
+}
+
+// fp32 epilogues (plain, + residual, + residual and cross-branch sum) of one warp's 32 rows x 32
+// columns with fully coalesced global accesses.  Thread = row cannot coalesce (32 rows per instruction,
+// one L1 wavefront per row piece, and the epilogue warps of an SM share one load/store pipe), so each
+// thread parks its row in a per-warp shared-memory tile (pitch 36 floats: conflict-free 16-byte
+// accesses both ways) and the warp then walks the tile 4 rows x 128 bytes per instruction.
+// The bias has already been added.  Rows must be 16-byte aligned.  The (warp, lane) -> (row, column)
+// mapping is fixed, which keeps the running sum of KRAKEN_EPI_RESID_SUM on the thread that wrote it.
+constexpr int EPI_STAGE_PITCH = 36;
+constexpr int EPI_STAGE_FLOATS = 32 * EPI_STAGE_PITCH;
+
+__device__ __forceinline__ void epilogue_f32_staged(const EpiParams &p, int g, int row_base, int m, int col0,
+                                                    const float (&v)[32], float *stage, int lane) {
+    float4 *mine = reinterpret_cast<float4 *>(stage + lane * EPI_STAGE_PITCH);
+#pragma unroll
+    for (int j = 0; j < 8; ++j) mine[j] = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+    __syncwarp();
+    const int r_in = lane >> 3, c4 = (lane & 7) << 2;
+    const long long col = col0 + c4;
+    // all loads of a phase are issued before any store: the pointers may alias as far as the compiler
+    // knows, so a store in between would serialise the loads behind it
+    float4 x[8];
+#pragma unroll
+    for (int it = 0; it < 8; ++it)
+        x[it] = *reinterpret_cast<const float4 *>(stage + (it * 4 + r_in) * EPI_STAGE_PITCH + c4);
+    if (p.kind != KRAKEN_EPI_F32) {
+        float4 t[8];
+#pragma unroll
+        for (int it = 0; it < 8; ++it) {
+            const int row = row_base + it * 4 + r_in;
+            t[it] = row < m ? *reinterpret_cast<const float4 *>(p.resid + g * p.resid_gstride +
+                                                                (long long)row * p.ld_resid + col)
+                            : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int it = 0; it < 8; ++it) {
+            x[it].x += t[it].x; x[it].y += t[it].y; x[it].z += t[it].z; x[it].w += t[it].w;
+        }
+    }
+    if (p.kind == KRAKEN_EPI_RESID_SUM && g > 0) {
+        float4 t[8];
+#pragma unroll
+        for (int it = 0; it < 8; ++it) {
+            const int row = row_base + it * 4 + r_in;
+            t[it] = row < m ? *reinterpret_cast<const float4 *>(p.sum + (long long)row * p.ld_sum + col)
+                            : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int it = 0; it < 8; ++it) {
+            const int row = row_base + it * 4 + r_in;
+            if (row < m) {
+                *reinterpret_cast<float4 *>(p.out_f32 + g * p.out_f32_gstride + (long long)row * p.ld_out_f32 + col) = x[it];
+                x[it].x += t[it].x; x[it].y += t[it].y; x[it].z += t[it].z; x[it].w += t[it].w;
+                *reinterpret_cast<float4 *>(p.sum + (long long)row * p.ld_sum + col) = x[it];
+            }
+        }
+    } else {
+#pragma unroll
+        for (int it = 0; it < 8; ++it) {
+            const int row = row_base + it * 4 + r_in;
+            if (row < m) {
+                *reinterpret_cast<float4 *>(p.out_f32 + g * p.out_f32_gstride + (long long)row * p.ld_out_f32 + col) = x[it];
+                if (p.kind == KRAKEN_EPI_RESID_SUM)
+                    *reinterpret_cast<float4 *>(p.sum + (long long)row * p.ld_sum + col) = x[it];
+            }
+        }
+    }
+    __syncwarp();
+}
+
+__device__ __forceinline__ bool epilogue_f32_stageable(const EpiParams &p) {
+    if (p.kind != KRAKEN_EPI_F32 && p.kind != KRAKEN_EPI_RESID_F32 && p.kind != KRAKEN_EPI_RESID_SUM) return false;
+    bool ok = (p.ld_out_f32 & 3) == 0 && (reinterpret_cast<uintptr_t>(p.out_f32) & 15) == 0 &&
+              (p.out_f32_gstride & 3) == 0;
+    if (p.kind != KRAKEN_EPI_F32)
+        ok = ok && (p.ld_resid & 3) == 0 && (reinterpret_cast<uintptr_t>(p.resid) & 15) == 0 &&
+             (p.resid_gstride & 3) == 0;
+    if (p.kind == KRAKEN_EPI_RESID_SUM) ok = ok && (p.ld_sum & 3) == 0 && (reinterpret_cast<uintptr_t>(p.sum) & 15) == 0;
+    return ok;
 }
 
 }  // namespace kr

@@ -250,9 +250,10 @@ struct PairCfg {
     static constexpr int A_BYTES = BM * BK * 2;            // 128 rows of A
     static constexpr int B_BYTES = (BN2 / 2) * BK * 2;     // this CTA's half of the W tile
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-    static constexpr int STAGES = 6;
+    static constexpr int STAGES = 5;
     static constexpr int TMEM_COLS = 2 * BN2;
-    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 256;
+    static constexpr int EPI_STAGE_BYTES = EPI_WARPS * EPI_STAGE_FLOATS * 4;  // fp32 epilogue staging tiles
+    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 256 + EPI_STAGE_BYTES;
 };
 
 __device__ __forceinline__ bool next_item_pair(const KernelArgs &ka, int it, int cluster_id, int n_clusters,
@@ -393,6 +394,9 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         const int quarter = warp & 3;
         const int half = (warp - 2) >> 2;
         constexpr int CHUNKS = BN2 / 32 / 2;
+        float *stage = reinterpret_cast<float *>(smem + Cfg::STAGES * Cfg::STAGE_BYTES + 256) +
+                       (warp - 2) * EPI_STAGE_FLOATS;
+        const bool staged = epilogue_f32_stageable(ka.epi);
         int acc = 0;
         uint32_t acc_phase = 0;
         bool ok = true;
@@ -402,7 +406,8 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             ok = __all_sync(0xFFFFFFFFu, ok);
             if (!ok) break;
             tc_fence_after_sync();
-            const int row = m_blk * 2 * BM + (int)rank * BM + quarter * 32 + lane;
+            const int row_base = m_blk * 2 * BM + (int)rank * BM + quarter * 32;
+            const int row = row_base + lane;
             const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
                                    static_cast<uint32_t>(acc * BN2);
 #pragma unroll 1
@@ -413,7 +418,14 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 uint32_t r[32];
                 tmem_ld_32x32(t_row + static_cast<uint32_t>(c * 32), r);
                 tmem_ld_wait();
-                if (row < ka.shape.m) {
+                if (staged && col0 + 32 <= ka.shape.n_out) {
+                    // coalesced path: the whole warp takes part, rows past M are masked inside
+                    float v[32];
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+                    if (ka.epi.bias) add_bias_chunk(ka.epi.bias + g * ka.epi.bias_gstride + col0, v, 32);
+                    epilogue_f32_staged(ka.epi, g, row_base, ka.shape.m, col0, v, stage, lane);
+                } else if (row < ka.shape.m) {
                     float v[32];
 #pragma unroll
                     for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
@@ -550,8 +562,8 @@ int launch_gemm_tc(const GemmOperands &op, const GemmShape &s, const EpiParams &
     ka.b_g0 = b_g0;
     ka.group_serial = epi.kind == KRAKEN_EPI_RESID_SUM ? 1 : 0;
     ka.n_fastest = (ka.group_serial && ka.tiles_n <= ka.tiles_m) ? 1 : 0;
-    if (bn == GEMM_TILE_PAIR) return launch_pair(*tmA, *tmB, ka, stream);
     ka.status = d_status;
+    if (bn == GEMM_TILE_PAIR) return launch_pair(*tmA, *tmB, ka, stream);
     const long long tiles = (long long)ka.tiles_m * ka.tiles_n;
     const long long units = ka.group_serial ? tiles : tiles * s.groups;
     const int sms = sm_count() > 0 ? sm_count() : 148;

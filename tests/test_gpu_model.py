@@ -319,5 +319,7 @@ def test_c4_full_size_prefill_prefix_parity_and_decode_consistency():
     k_ref = m.kv_view(s.n_layer - 1, 2, 0)[:, :, s.seqlen].float().cpu().numpy()
     v_ref = m.kv_view(0, 3, 1)[:, :, s.seqlen].float().cpu().numpy()
     assert np.abs(k_after - k_ref).max() <= 0.05 * np.abs(k_ref).max()
-    assert np.array_equal(v_after, v_ref)      # first layer: same inputs, same arithmetic order per row
+    # first layer: same inputs, but the decode GEMM adds the products in another order than the tile GEMM
+    assert np.abs(v_after - v_ref).max() <= 2.0 ** -6 * np.abs(v_ref).max()
+    assert (v_after == v_ref).mean() > 0.9
     m.close()
