@@ -77,7 +77,8 @@ def _gemm_args(kind, s, batch, seqlen, n_tile=0):
     return g, keep, flops, byts
 
 
-def run_case(kind: str, workload: str, reps: int, warmup: int, n_tile: int = 0, batch=None, seqlen=None):
+def run_case(kind: str, workload: str, reps: int, warmup: int, n_tile: int = 0, batch=None, seqlen=None,
+             graph_launches: int = 0):
     s = ki.CONFIGS[workload]
     batch = batch or s.batch
     seqlen = seqlen or s.seqlen
@@ -124,13 +125,25 @@ def run_case(kind: str, workload: str, reps: int, warmup: int, n_tile: int = 0, 
     for _ in range(warmup):
         fn()
     torch.cuda.synchronize()
+    if graph_launches:
+        # short kernels: replay `graph_launches` back-to-back launches from a CUDA graph, so that the host's
+        # launch pace does not enter the measurement
+        cg = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(cg):
+            for _ in range(graph_launches):
+                fn()
+        cg.replay()
+        torch.cuda.synchronize()
     ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
     for e0, e1 in ev:
         e0.record()
-        fn()
+        if graph_launches:
+            cg.replay()
+        else:
+            fn()
         e1.record()
     torch.cuda.synchronize()
-    ms = sorted(e0.elapsed_time(e1) for e0, e1 in ev)
+    ms = sorted(e0.elapsed_time(e1) / max(1, graph_launches) for e0, e1 in ev)
     med = ms[len(ms) // 2]
     out = {"case": kind, "workload": workload, "batch": batch, "seqlen": seqlen, "n_tile": n_tile,
            "ms_median": med, "ms_min": ms[0], "tflops": flops / (med * 1e-3) / 1e12,
@@ -149,6 +162,7 @@ def main():
     ap.add_argument("--n-tile", type=int, default=0, help="GEMM N tile, or split count for decode_attention")
     ap.add_argument("--batch", type=int, default=None)
     ap.add_argument("--seqlen", type=int, default=None)
+    ap.add_argument("--graph", type=int, default=0, help="time this many launches replayed from one CUDA graph")
     a = ap.parse_args()
     kinds = [a.case]
     if a.case == "all":
@@ -156,7 +170,7 @@ def main():
     elif a.case == "decode_all":
         kinds = ["decode_gemm_qkv", "decode_gemm_proj", "decode_gemm_up", "decode_gemm_down", "decode_attention"]
     for k in kinds:
-        run_case(k, a.workload, a.reps, a.warmup, a.n_tile, a.batch, a.seqlen)
+        run_case(k, a.workload, a.reps, a.warmup, a.n_tile, a.batch, a.seqlen, a.graph)
 
 
 if __name__ == "__main__":

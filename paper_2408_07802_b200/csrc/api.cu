@@ -86,6 +86,14 @@ struct kraken_handle {
     // activation tensor maps, re-encoded when the token count changes
     CUtensorMap tmA[G_COUNT];
     int tmA_rows[G_COUNT];
+    // decode steps replayed as a CUDA graph: positions are read from `pos` in device memory, tokens
+    // and logits go through the staging buffers, so one graph serves every step of a batch size
+    cudaGraphExec_t dec_graph;
+    cudaStream_t cap_stream;                  // capture happens here (the caller's stream may be the legacy default)
+    int dec_graph_batch;
+    int dec_eager_steps;                      // eager steps done for the current batch size (warm-up)
+    long long dec_graph_launches[KRAKEN_PROF_COUNT];
+    bool use_graph;
     // launch accounting and optional per-kernel timing
     long long launches[KRAKEN_PROF_COUNT];
     bool prof_on;
@@ -136,6 +144,8 @@ struct RunCtx {
     kraken_handle *h;
     cudaStream_t st;
     int batch, seqlen, pos0, T;
+    const int *pos_dev;  // decode graph: positions come from device memory
+    int max_keys;        // decode graph: upper bound of the keys a step can see (fixes the split count)
 };
 
 // One grouped GEMM of the model: weights of `kind` at `layer`.
@@ -234,7 +244,7 @@ int run_layers(const RunCtx &rc, const int32_t *d_tokens) {
     {
         LaunchScope scope(h, KRAKEN_PROF_EMBED, rc.st);
         KR_TRY(launch_embed(d_tokens, T, rc.seqlen, rc.pos0, (const uint16_t *)h->w.wte, (const uint16_t *)h->w.wpe, d,
-                            c.vocab, x0, status, rc.st));
+                            c.vocab, x0, status, rc.st, rc.pos_dev));
     }
     for (int l = 0; l < L; ++l) {
         const float *xin = l == 0 ? x0 : x;
@@ -254,6 +264,7 @@ int run_layers(const RunCtx &rc, const int32_t *d_tokens) {
         e.out_bf16 = q; e.out_bf16_gstride = td; e.ld_out_bf16 = d;
         e.k_cache = kc; e.v_cache = kc + cache_kv; e.cache_gstride = 2 * cache_kv;
         e.seqlen = rc.seqlen; e.pos0 = rc.pos0; e.n_head = H; e.head_dim = hd; e.max_pos = c.max_pos; e.d_model = d;
+        e.pos0_dev = rc.pos_dev;
         KR_TRY(model_gemm(rc, G_QKV, l, T, u, td, e));
         // attention over the cached prefix
         AttnParams ap;
@@ -273,7 +284,8 @@ int run_layers(const RunCtx &rc, const int32_t *d_tokens) {
                 dp.cache_gstride = ap.cache_gstride; dp.cache_bstride = ap.cache_bstride;
                 dp.groups = N; dp.batch = rc.batch; dp.n_keys = rc.pos0 + 1; dp.n_head = H; dp.head_dim = hd;
                 dp.max_pos = c.max_pos;
-                dp.splits = decode_attention_splits(N, rc.batch, H, dp.n_keys);
+                dp.pos_dev = rc.pos_dev;
+                dp.splits = decode_attention_splits(N, rc.batch, H, rc.pos_dev ? rc.max_keys : dp.n_keys);
                 dp.partials = at<float>(h, h->lay.dec_part);
                 dp.out = o; dp.out_gstride = td;
                 h->launches[KRAKEN_PROF_ATTENTION] += dp.splits > 1 ? 1 : 0;
@@ -318,7 +330,18 @@ int run_layers(const RunCtx &rc, const int32_t *d_tokens) {
     return KRAKEN_OK;
 }
 
+__global__ void set_pos_kernel(int *pos, int value) {
+    pdl_wait();
+    *pos = value;
+}
+__global__ void advance_pos_kernel(int *pos) {
+    pdl_wait();
+    *pos += 1;
+}
+
 __global__ void make_rows_kernel(int32_t *rows, int n, int mul, int add) {
+    pdl_wait();
+    pdl_trigger();
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i < n) rows[i] = i * mul + add;
 }
@@ -359,12 +382,13 @@ int prefill_common(kraken_handle *h, const int32_t *d_tokens, int batch, int seq
                    bool all_logits) {
     if (!h || !d_tokens || !d_logits || batch < 1 || seqlen < 1) return KRAKEN_EINVAL;
     if (batch > h->cfg.max_batch || seqlen > h->cfg.max_pos) return KRAKEN_ECAPACITY;
-    RunCtx rc{h, static_cast<cudaStream_t>(stream), batch, seqlen, 0, batch * seqlen};
+    RunCtx rc{h, static_cast<cudaStream_t>(stream), batch, seqlen, 0, batch * seqlen, nullptr, 0};
     h->last_stream = rc.st;
     KR_TRY(run_layers(rc, d_tokens));
     h->cur_len = seqlen;
     h->batch = batch;
     h->last_seqlen = seqlen;
+    set_pos_kernel<<<1, 1, 0, rc.st>>>(at<int>(h, h->lay.status + 128), seqlen);
     int32_t *rows = at<int32_t>(h, h->lay.rows);
     const int n_rows = all_logits ? batch * seqlen : batch;
     h->launches[KRAKEN_PROF_TAIL]++;
@@ -413,6 +437,11 @@ int kraken_create(const kraken_config *cfg, const kraken_weights *w, void *d_kv,
     h->last_stream = nullptr;
     h->naive = env_flag("KRAKEN_NAIVE");
     h->prof_on = false;
+    h->dec_graph = nullptr;
+    h->cap_stream = nullptr;
+    h->dec_graph_batch = 0;
+    h->dec_eager_steps = 0;
+    h->use_graph = !env_flag("KRAKEN_NO_GRAPH") && !h->naive;
     h->ev_used = 0;
     for (int i = 0; i < KRAKEN_PROF_COUNT; ++i) h->launches[i] = 0;
     for (int i = 0; i < G_COUNT; ++i) {
@@ -462,24 +491,99 @@ int kraken_logits_rows(kraken_handle *h, const int32_t *h_rows, int32_t n_rows, 
     int32_t *rows = at<int32_t>(h, h->lay.rows);
     if (cudaMemcpyAsync(rows, h_rows, (size_t)n_rows * 4, cudaMemcpyHostToDevice, st) != cudaSuccess)
         return KRAKEN_ECUDA;
-    RunCtx rc{h, st, h->batch, h->last_seqlen, 0, h->last_rows};
+    RunCtx rc{h, st, h->batch, h->last_seqlen, 0, h->last_rows, nullptr, 0};
     h->last_stream = st;
     return run_tail(rc, rows, n_rows, d_logits);
 }
+
+namespace {
+
+// The kernel sequence of one decode step; with from_dev the position is read from device memory.
+int decode_body(kraken_handle *h, cudaStream_t st, const int32_t *d_tokens, int batch, float *d_logits,
+                bool from_dev) {
+    int *d_pos = at<int>(h, h->lay.status + 128);
+    RunCtx rc{h, st, batch, 1, h->cur_len, batch, from_dev ? d_pos : nullptr, h->cfg.max_pos};
+    KR_TRY(run_layers(rc, d_tokens));
+    h->last_seqlen = 1;
+    int32_t *rows = at<int32_t>(h, h->lay.rows);
+    h->launches[KRAKEN_PROF_TAIL]++;
+    make_rows_kernel<<<(batch + 255) / 256, 256, 0, st>>>(rows, batch, 1, 0);
+    if (cudaGetLastError() != cudaSuccess) return KRAKEN_ECUDA;
+    KR_TRY(run_tail(rc, rows, batch, d_logits));
+    advance_pos_kernel<<<1, 1, 0, st>>>(d_pos);
+    return cuda_check(cudaGetLastError(), "decode: position update");
+}
+
+}  // namespace
 
 int kraken_decode_step(kraken_handle *h, const int32_t *d_tokens, int32_t batch, float *d_logits, void *stream) {
     if (!h || !d_tokens || !d_logits || batch < 1) return KRAKEN_EINVAL;
     if (h->cur_len < 1 || batch != h->batch) return KRAKEN_ESTATE;
     if (h->cur_len + 1 > h->cfg.max_pos) return KRAKEN_ECAPACITY;
-    RunCtx rc{h, static_cast<cudaStream_t>(stream), batch, 1, h->cur_len, batch};
-    h->last_stream = rc.st;
-    KR_TRY(run_layers(rc, d_tokens));
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    h->last_stream = st;
+    if (h->dec_graph_batch != batch) {            // a new batch size: forget the old graph, warm up again
+        if (h->dec_graph) cudaGraphExecDestroy(h->dec_graph);
+        h->dec_graph = nullptr;
+        h->dec_graph_batch = batch;
+        h->dec_eager_steps = 0;
+    }
+    if (!h->use_graph || h->prof_on || h->dec_eager_steps < 1) {
+        // eager step (also the first step of a batch size: it performs every one-time set-up call,
+        // none of which may happen inside a stream capture)
+        KR_TRY(decode_body(h, st, d_tokens, batch, d_logits, false));
+        h->dec_eager_steps++;
+        h->cur_len += 1;
+        return KRAKEN_OK;
+    }
+    int32_t *s_tok = at<int32_t>(h, h->lay.tokens);
+    float *s_log = at<float>(h, h->lay.logits);
+    if (d_tokens != s_tok)
+        KR_TRY(cuda_check(cudaMemcpyAsync(s_tok, d_tokens, (size_t)batch * 4, cudaMemcpyDeviceToDevice, st),
+                          "decode: token staging"));
+    if (!h->dec_graph) {
+        long long before[KRAKEN_PROF_COUNT];
+        for (int i = 0; i < KRAKEN_PROF_COUNT; ++i) before[i] = h->launches[i];
+        if (!h->cap_stream)
+            KR_TRY(cuda_check(cudaStreamCreateWithFlags(&h->cap_stream, cudaStreamNonBlocking), "decode: capture stream"));
+        KR_TRY(cuda_check(cudaStreamBeginCapture(h->cap_stream, cudaStreamCaptureModeThreadLocal),
+                          "decode: begin capture"));
+        const int saved_len = h->cur_len, saved_rows = h->last_rows;
+        int rc_body = decode_body(h, h->cap_stream, s_tok, batch, s_log, true);
+        cudaGraph_t graph = nullptr;
+        cudaError_t ce = cudaStreamEndCapture(h->cap_stream, &graph);
+        h->cur_len = saved_len;
+        h->last_rows = saved_rows;
+        for (int i = 0; i < KRAKEN_PROF_COUNT; ++i) {
+            h->dec_graph_launches[i] = h->launches[i] - before[i];
+            h->launches[i] = before[i];
+        }
+        if (rc_body || ce != cudaSuccess || !graph) {
+            if (graph) cudaGraphDestroy(graph);
+            cudaGetLastError();
+            h->use_graph = false;                 // fall back to eager steps for this handle
+            KR_TRY(decode_body(h, st, d_tokens, batch, d_logits, false));
+            h->cur_len += 1;
+            return KRAKEN_OK;
+        }
+        ce = cudaGraphInstantiate(&h->dec_graph, graph, 0);
+        cudaGraphDestroy(graph);
+        if (ce != cudaSuccess) {
+            h->dec_graph = nullptr;
+            h->use_graph = false;
+            cudaGetLastError();
+            KR_TRY(decode_body(h, st, d_tokens, batch, d_logits, false));
+            h->cur_len += 1;
+            return KRAKEN_OK;
+        }
+    }
+    KR_TRY(cuda_check(cudaGraphLaunch(h->dec_graph, st), "decode: graph launch"));
+    for (int i = 0; i < KRAKEN_PROF_COUNT; ++i) h->launches[i] += h->dec_graph_launches[i];
+    h->last_rows = batch;
     h->last_seqlen = 1;
-    int32_t *rows = at<int32_t>(h, h->lay.rows);
-    h->launches[KRAKEN_PROF_TAIL]++;
-    make_rows_kernel<<<(batch + 255) / 256, 256, 0, rc.st>>>(rows, batch, 1, 0);
-    if (cudaGetLastError() != cudaSuccess) return KRAKEN_ECUDA;
-    KR_TRY(run_tail(rc, rows, batch, d_logits));
+    if (d_logits != s_log)
+        KR_TRY(cuda_check(cudaMemcpyAsync(d_logits, s_log, (size_t)batch * h->cfg.vocab * 4,
+                                          cudaMemcpyDeviceToDevice, st), "decode: logits staging"));
     h->cur_len += 1;
     return KRAKEN_OK;
 }
@@ -541,6 +645,8 @@ int kraken_reset(kraken_handle *h) {
 void kraken_destroy(kraken_handle *h) {
     if (!h) return;
     for (cudaEvent_t e : h->ev_pool) cudaEventDestroy(e);
+    if (h->dec_graph) cudaGraphExecDestroy(h->dec_graph);
+    if (h->cap_stream) cudaStreamDestroy(h->cap_stream);
     delete h;
 }
 
@@ -658,7 +764,7 @@ int kraken_op_decode_attention(const void *q, int64_t q_gstride, const void *k_c
     p.k_cache = (const uint16_t *)k_cache; p.v_cache = (const uint16_t *)v_cache;
     p.cache_gstride = cache_gstride; p.cache_bstride = cache_bstride;
     p.groups = groups; p.batch = batch; p.n_keys = n_keys; p.n_head = n_head; p.head_dim = head_dim;
-    p.max_pos = max_pos; p.splits = splits; p.partials = (float *)d_partials;
+    p.max_pos = max_pos; p.pos_dev = nullptr; p.splits = splits; p.partials = (float *)d_partials;
     p.out = (uint16_t *)out; p.out_gstride = out_gstride;
     return launch_attention_decode(p, static_cast<cudaStream_t>(stream));
 }

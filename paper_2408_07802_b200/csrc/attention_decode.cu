@@ -22,6 +22,7 @@ __global__ void __launch_bounds__(DEC_WARPS * 32)
 attn_decode_kernel(const DecodeAttnParams p) {
     constexpr int LPR = HD / 8;       // lanes per cache row (16 bytes each)
     constexpr int RPW = 32 / LPR;     // rows per warp-wide load
+    pdl_wait();
     const int split = blockIdx.x, h = blockIdx.y;
     const int b = blockIdx.z % p.batch, g = blockIdx.z / p.batch;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -29,9 +30,10 @@ attn_decode_kernel(const DecodeAttnParams p) {
     const int d = p.n_head * HD;
 
     // keys of this split
-    const int per = (p.n_keys + p.splits - 1) / p.splits;
+    const int n_keys = p.pos_dev ? *p.pos_dev + 1 : p.n_keys;
+    const int per = (n_keys + p.splits - 1) / p.splits;
     const int k_begin = split * per;
-    const int k_end = min(p.n_keys, k_begin + per);
+    const int k_end = min(n_keys, k_begin + per);
 
     const uint16_t *gq = p.q + g * p.q_gstride + (long long)b * d + h * HD + sub * 8;
     const uint16_t *gk = p.k_cache + g * p.cache_gstride + b * p.cache_bstride + (long long)h * p.max_pos * HD;
@@ -100,6 +102,7 @@ attn_decode_kernel(const DecodeAttnParams p) {
         }
     }
 
+    pdl_trigger();
     // merge the row groups of the warp (lanes with equal `sub`), then the warps through shared memory
 #pragma unroll
     for (int off = LPR; off < 32; off <<= 1) {
@@ -156,6 +159,8 @@ attn_decode_kernel(const DecodeAttnParams p) {
 // out = sum_s o_s 2^(m_s - m) / sum_s l_s 2^(m_s - m)
 template <int HD>
 __global__ void __launch_bounds__(HD) attn_decode_merge_kernel(const DecodeAttnParams p) {
+    pdl_wait();
+    pdl_trigger();
     const int h = blockIdx.x;
     const int b = blockIdx.y % p.batch, g = blockIdx.y / p.batch;
     const int e = threadIdx.x;
@@ -177,14 +182,15 @@ __global__ void __launch_bounds__(HD) attn_decode_merge_kernel(const DecodeAttnP
 template <int HD>
 int launch(const DecodeAttnParams &p, cudaStream_t stream) {
     dim3 grid(p.splits, p.n_head, p.batch * p.groups);
-    attn_decode_kernel<HD><<<grid, DEC_WARPS * 32, 0, stream>>>(p);
-    if (cudaGetLastError() != cudaSuccess) return KRAKEN_ECUDA;
+    int rc = cuda_check(launch_pdl(attn_decode_kernel<HD>, grid, dim3(DEC_WARPS * 32), 0, stream, p),
+                        "decode attention: launch");
+    if (rc) return rc;
     if (p.splits > 1) {
         dim3 g2(p.n_head, p.batch * p.groups);
-        attn_decode_merge_kernel<HD><<<g2, HD, 0, stream>>>(p);
-        if (cudaGetLastError() != cudaSuccess) return KRAKEN_ECUDA;
+        rc = cuda_check(launch_pdl(attn_decode_merge_kernel<HD>, g2, dim3(HD), 0, stream, p),
+                        "decode attention merge: launch");
     }
-    return KRAKEN_OK;
+    return rc;
 }
 
 }  // namespace

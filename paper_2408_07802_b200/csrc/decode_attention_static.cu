@@ -65,6 +65,7 @@ extern "C" int kraken_op_decode_attention_static(const void *q, int64_t q_gstrid
     p.n_head = n_head;
     p.head_dim = head_dim;
     p.max_pos = max_pos;
+    p.pos_dev = nullptr;
     p.splits = splits;
     p.partials = partials;
     p.out = static_cast<uint16_t *>(out);

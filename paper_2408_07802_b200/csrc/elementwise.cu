@@ -12,7 +12,10 @@ constexpr int ROW_WARPS = 8;  // warps (rows) per CTA
 
 __global__ void __launch_bounds__(ROW_WARPS * 32)
 embed_kernel(const int32_t *__restrict__ ids, int n_tokens, int seqlen, int pos0, const uint16_t *__restrict__ wte,
-             const uint16_t *__restrict__ wpe, int d, int vocab, float *__restrict__ out, uint32_t *status) {
+             const uint16_t *__restrict__ wpe, int d, int vocab, float *__restrict__ out, uint32_t *status,
+             const int *__restrict__ pos0_dev) {
+    pdl_wait();
+    pdl_trigger();
     const int t = blockIdx.x * ROW_WARPS + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (t >= n_tokens) return;
@@ -21,7 +24,7 @@ embed_kernel(const int32_t *__restrict__ ids, int n_tokens, int seqlen, int pos0
         if (lane == 0 && status) atomicOr(status, STATUS_BAD_TOKEN);
         id = 0;
     }
-    const int pos = pos0 + t % seqlen;
+    const int pos = (pos0_dev ? *pos0_dev : pos0) + t % seqlen;
     const uint4 *te = reinterpret_cast<const uint4 *>(wte + (size_t)id * d);
     const uint4 *pe = reinterpret_cast<const uint4 *>(wpe + (size_t)pos * d);
     float4 *o = reinterpret_cast<float4 *>(out + (size_t)t * d);
@@ -50,6 +53,7 @@ layernorm_kernel(const float *__restrict__ a, long long a_gstride, const float *
                  const float *__restrict__ ysum, long long ysum_gstride, int ysum_groups,
                  const uint16_t *__restrict__ gamma, const uint16_t *__restrict__ beta, int groups, int rows, int d,
                  float eps, uint16_t *__restrict__ out) {
+    pdl_wait();
     const long long wr = (long long)blockIdx.x * ROW_WARPS + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (wr >= (long long)groups * rows) return;
@@ -108,6 +112,7 @@ layernorm_kernel(const float *__restrict__ a, long long a_gstride, const float *
         sq += (dx * dx + dy * dy) + (dz * dz + dw * dw);
     }
     const float rstd = rsqrtf(warp_sum(sq) / d + eps);
+    pdl_trigger();
 
     const uint2 *pg = reinterpret_cast<const uint2 *>(gamma + (size_t)g * d);
     const uint2 *pb = beta ? reinterpret_cast<const uint2 *>(beta + (size_t)g * d) : nullptr;
@@ -133,6 +138,8 @@ layernorm_kernel(const float *__restrict__ a, long long a_gstride, const float *
 __global__ void __launch_bounds__(ROW_WARPS * 32)
 gather_concat_kernel(const float *__restrict__ x, long long x_gstride, int groups, int d,
                      const int32_t *__restrict__ rows, int n_rows, uint16_t *__restrict__ out) {
+    pdl_wait();
+    pdl_trigger();
     const long long w = (long long)blockIdx.x * ROW_WARPS + (threadIdx.x >> 5);
     const int lane = threadIdx.x & 31;
     if (w >= (long long)n_rows * groups) return;
@@ -157,13 +164,12 @@ int done() { return cudaGetLastError() == cudaSuccess ? KRAKEN_OK : KRAKEN_ECUDA
 }  // namespace
 
 int launch_embed(const int32_t *ids, int n_tokens, int seqlen, int pos0, const uint16_t *wte, const uint16_t *wpe,
-                 int d, int vocab, float *out, uint32_t *status, cudaStream_t stream) {
+                 int d, int vocab, float *out, uint32_t *status, cudaStream_t stream, const int *pos0_dev) {
     if (!ids || !wte || !wpe || !out || n_tokens < 1 || seqlen < 1 || pos0 < 0 || d < 8 || (d & 7) || vocab < 1)
         return KRAKEN_EINVAL;
-    embed_kernel<<<(n_tokens + ROW_WARPS - 1) / ROW_WARPS, ROW_WARPS * 32, 0, stream>>>(ids, n_tokens, seqlen, pos0,
-                                                                                         wte, wpe, d, vocab, out,
-                                                                                         status);
-    return done();
+    return cuda_check(launch_pdl(embed_kernel, dim3((n_tokens + ROW_WARPS - 1) / ROW_WARPS), dim3(ROW_WARPS * 32), 0,
+                                 stream, ids, n_tokens, seqlen, pos0, wte, wpe, d, vocab, out, status, pos0_dev),
+                      "embed: launch");
 }
 
 int launch_layernorm(const float *a, long long a_gstride, const float *y, const uint16_t *gamma,
@@ -172,18 +178,19 @@ int launch_layernorm(const float *a, long long a_gstride, const float *y, const 
     if (!a || !gamma || !out || groups < 1 || rows < 1 || d < 4 || (d & 3)) return KRAKEN_EINVAL;
     if (ysum && (y || ysum_groups < 1 || (ysum_gstride & 3))) return KRAKEN_EINVAL;
     const long long warps = (long long)groups * rows;
-    layernorm_kernel<<<static_cast<unsigned>((warps + ROW_WARPS - 1) / ROW_WARPS), ROW_WARPS * 32, 0, stream>>>(
-        a, a_gstride, y, ysum, ysum_gstride, ysum_groups, gamma, beta, groups, rows, d, eps, out);
-    return done();
+    return cuda_check(launch_pdl(layernorm_kernel, dim3(static_cast<unsigned>((warps + ROW_WARPS - 1) / ROW_WARPS)),
+                                 dim3(ROW_WARPS * 32), 0, stream, a, a_gstride, y, ysum, ysum_gstride, ysum_groups,
+                                 gamma, beta, groups, rows, d, eps, out),
+                      "layernorm: launch");
 }
 
 int launch_gather_concat(const float *x, long long x_gstride, int groups, int d, const int32_t *rows, int n_rows,
                          uint16_t *out, cudaStream_t stream) {
     if (!x || !out || groups < 1 || n_rows < 1 || (d & 3)) return KRAKEN_EINVAL;
     const long long warps = (long long)groups * n_rows;
-    gather_concat_kernel<<<static_cast<unsigned>((warps + ROW_WARPS - 1) / ROW_WARPS), ROW_WARPS * 32, 0, stream>>>(
-        x, x_gstride, groups, d, rows, n_rows, out);
-    return done();
+    return cuda_check(launch_pdl(gather_concat_kernel, dim3(static_cast<unsigned>((warps + ROW_WARPS - 1) / ROW_WARPS)),
+                                 dim3(ROW_WARPS * 32), 0, stream, x, x_gstride, groups, d, rows, n_rows, out),
+                      "gather: launch");
 }
 
 int launch_f32_to_bf16(const float *in, uint16_t *out, long long n, cudaStream_t stream) {

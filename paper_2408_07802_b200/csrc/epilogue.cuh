@@ -201,7 +201,7 @@ __device__ __forceinline__ void epilogue_chunk(const EpiParams &p, int g, int ro
                 const int which = col0 >= 2 * d;
                 const int c = col0 - (1 + which) * d;
                 const int head = c / p.head_dim, e0 = c % p.head_dim;
-                const int b = row / p.seqlen, pos = p.pos0 + row % p.seqlen;
+                const int b = row / p.seqlen, pos = (p.pos0_dev ? *p.pos0_dev : p.pos0) + row % p.seqlen;
                 uint16_t *base = (which ? p.v_cache : p.k_cache) + g * p.cache_gstride;
                 store_bf16_chunk(base + (((long long)b * p.n_head + head) * p.max_pos + pos) * p.head_dim + e0, v,
                                  ncols);

@@ -1,7 +1,7 @@
 // Weight-streaming GEMM for a handful of rows (decode steps and the last-position tail):
 // C_g[M, Nout] = A_g[M, K] . W_g[Nout, K]^T with M <= 32.  Every weight byte is read exactly once,
 // so the kernel is bound by HBM and shaped for bytes in flight, not for the tensor pipe:
-//   - one CTA per strip of 8 output columns of one group, 8 warps splitting K;
+//   - one CTA per strip of 8 output columns of one group, 4 or 8 warps splitting K;
 //   - every lane streams 16-byte pieces of a weight row (4 lanes cover 64 contiguous bytes of each
 //     of 8 rows) and the matching 16-byte pieces of the activation rows (L1/L2 resident);
 //   - products run on m16n8k16 warp MMAs with the K slots permuted identically for both operands,
@@ -16,9 +16,8 @@ namespace kr {
 
 namespace {
 
-constexpr int SK_WARPS = 8;
 constexpr int SK_COLS = 8;
-constexpr int SK_UNROLL = 4;
+constexpr int SK_UNROLL = 8;
 
 __device__ __forceinline__ void mma16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                          uint32_t b0, uint32_t b1) {
@@ -57,7 +56,7 @@ __device__ __forceinline__ void epilogue_elem(const EpiParams &p, int g, int row
             } else {
                 const int which = col >= 2 * d, c = col - (1 + which) * d;
                 const int head = c / p.head_dim, e = c % p.head_dim;
-                const int b = row / p.seqlen, pos = p.pos0 + row % p.seqlen;
+                const int b = row / p.seqlen, pos = (p.pos0_dev ? *p.pos0_dev : p.pos0) + row % p.seqlen;
                 uint16_t *base = (which ? p.v_cache : p.k_cache) + g * p.cache_gstride;
                 base[(((long long)b * p.n_head + head) * p.max_pos + pos) * p.head_dim + e] = to_bf(acc);
             }
@@ -68,9 +67,10 @@ __device__ __forceinline__ void epilogue_elem(const EpiParams &p, int g, int row
     }
 }
 
-template <int MB>  // 16-row blocks of A (1 or 2)
+template <int MB, int SK_WARPS>  // 16-row blocks of A (1 or 2); warps splitting K
 __global__ void __launch_bounds__(SK_WARPS * 32)
 gemm_skinny_kernel(const GemmOperands op, const GemmShape s, const EpiParams epi) {
+    pdl_wait();
     const int g = blockIdx.y;
     const int n0 = blockIdx.x * SK_COLS;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -101,28 +101,31 @@ gemm_skinny_kernel(const GemmOperands op, const GemmShape s, const EpiParams epi
     const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
 
     for (int c0 = c_begin; c0 < c_end; c0 += SK_UNROLL) {
+        // the weight pieces of the whole batch go in flight first (they come from DRAM); the activation
+        // pieces are fetched chunk by chunk right before use (they sit in L1/L2), which keeps the
+        // register count low enough for eight CTAs per SM
         uint4 wv[SK_UNROLL];
-        uint4 av[SK_UNROLL][MB][2];
 #pragma unroll
         for (int u = 0; u < SK_UNROLL; ++u) {
             const int k = (c0 + u) * 32 + kq * 8;
             const bool k_ok = (c0 + u) < c_end && k < s.k;
             wv[u] = (k_ok && n_ok) ? __ldcs(reinterpret_cast<const uint4 *>(wrow + k)) : zero;
-#pragma unroll
-            for (int mb = 0; mb < MB; ++mb)
-#pragma unroll
-                for (int hlf = 0; hlf < 2; ++hlf)
-                    av[u][mb][hlf] = (k_ok && a_ok[mb][hlf]) ? *reinterpret_cast<const uint4 *>(arow[mb][hlf] + k) : zero;
         }
 #pragma unroll
-        for (int u = 0; u < SK_UNROLL; ++u)
+        for (int u = 0; u < SK_UNROLL; ++u) {
+            const int k = (c0 + u) * 32 + kq * 8;
+            const bool k_ok = (c0 + u) < c_end && k < s.k;
 #pragma unroll
             for (int mb = 0; mb < MB; ++mb) {
-                mma16816(acc[mb], av[u][mb][0].x, av[u][mb][1].x, av[u][mb][0].y, av[u][mb][1].y, wv[u].x, wv[u].y);
-                mma16816(acc[mb], av[u][mb][0].z, av[u][mb][1].z, av[u][mb][0].w, av[u][mb][1].w, wv[u].z, wv[u].w);
+                const uint4 a0 = (k_ok && a_ok[mb][0]) ? *reinterpret_cast<const uint4 *>(arow[mb][0] + k) : zero;
+                const uint4 a1 = (k_ok && a_ok[mb][1]) ? *reinterpret_cast<const uint4 *>(arow[mb][1] + k) : zero;
+                mma16816(acc[mb], a0.x, a1.x, a0.y, a1.y, wv[u].x, wv[u].y);
+                mma16816(acc[mb], a0.z, a1.z, a0.w, a1.w, wv[u].z, wv[u].w);
             }
+        }
     }
 
+    pdl_trigger();
     // cross-warp reduction in a fixed order
     __shared__ float part[SK_WARPS][MB * 16][SK_COLS];
 #pragma unroll
@@ -153,11 +156,17 @@ int launch_gemm_skinny(const GemmOperands &op, const GemmShape &s, const EpiPara
         (reinterpret_cast<uintptr_t>(op.w) & 15) || (op.a_gstride & 7) || (op.w_gstride & 7))
         return KRAKEN_EUNSUPPORTED;
     dim3 grid((s.n_out + SK_COLS - 1) / SK_COLS, s.groups);
-    if (s.m <= 16)
-        gemm_skinny_kernel<1><<<grid, SK_WARPS * 32, 0, stream>>>(op, s, epi);
-    else
-        gemm_skinny_kernel<2><<<grid, SK_WARPS * 32, 0, stream>>>(op, s, epi);
-    return cudaGetLastError() == cudaSuccess ? KRAKEN_OK : KRAKEN_ECUDA;
+    // K is split over the warps of a CTA so that each warp still streams a few hundred bytes per lane
+    const bool wide_k = s.k > 2048;
+    cudaError_t ce;
+    if (s.m <= 16) {
+        ce = wide_k ? launch_pdl(gemm_skinny_kernel<1, 8>, grid, dim3(256), 0, stream, op, s, epi)
+                    : launch_pdl(gemm_skinny_kernel<1, 4>, grid, dim3(128), 0, stream, op, s, epi);
+    } else {
+        ce = wide_k ? launch_pdl(gemm_skinny_kernel<2, 8>, grid, dim3(256), 0, stream, op, s, epi)
+                    : launch_pdl(gemm_skinny_kernel<2, 4>, grid, dim3(128), 0, stream, op, s, epi);
+    }
+    return cuda_check(ce, "skinny gemm: launch");
 }
 
 }  // namespace kr

@@ -28,6 +28,7 @@ struct EpiParams {
     long long cache_gstride;
     int seqlen, pos0, n_head, head_dim, max_pos, d_model;
     int gelu_tanh;
+    const int *pos0_dev;  // when set, the first position is read from device memory (replayable decode graph)
 };
 
 struct GemmShape {
@@ -70,7 +71,7 @@ constexpr int SKINNY_MAX_ROWS = 32;
 int launch_gemm_naive(const GemmOperands &op, const GemmShape &shape, const EpiParams &epi, cudaStream_t stream);
 
 int launch_embed(const int32_t *ids, int n_tokens, int seqlen, int pos0, const uint16_t *wte, const uint16_t *wpe,
-                 int d, int vocab, float *out, uint32_t *status, cudaStream_t stream);
+                 int d, int vocab, float *out, uint32_t *status, cudaStream_t stream, const int *pos0_dev = nullptr);
 // y: [rows, d] added before normalisation (or NULL); alternatively ysum: `ysum_groups` tensors
 // [rows, d], ysum_gstride apart, whose sum is added.
 int launch_layernorm(const float *a, long long a_gstride, const float *y, const uint16_t *gamma,
@@ -108,6 +109,7 @@ struct DecodeAttnParams {
     const uint16_t *k_cache, *v_cache;
     long long cache_gstride, cache_bstride;
     int groups, batch, n_keys, n_head, head_dim, max_pos;
+    const int *pos_dev;  // when set, n_keys = *pos_dev + 1 (replayable decode graph)
     int splits;
     float *partials;  // [G*batch*n_head][splits][head_dim + 2] fp32 (max, sum, output); unused when splits == 1
     uint16_t *out;    // [G][batch, d]
@@ -116,6 +118,24 @@ struct DecodeAttnParams {
 int decode_attention_splits(int groups, int batch, int n_head, int n_keys);
 size_t decode_attention_partial_bytes(int groups, int batch, int n_head, int head_dim, int splits);
 int launch_attention_decode(const DecodeAttnParams &p, cudaStream_t stream);
+
+// Launch with programmatic stream serialisation (see pdl_wait / pdl_trigger in ptx.cuh): hides the
+// launch latency between the many short kernels of a decode step.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                              Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
 
 bool env_flag(const char *name);
 // Records the text of a failed CUDA call (per thread) and maps it to KRAKEN_ECUDA.

@@ -292,6 +292,14 @@ __device__ __forceinline__ void umma_commit_pair(uint64_t *bar, uint16_t cta_mas
         : "memory");
 }
 
+// ---------------------------------------------------------------- programmatic dependent launch
+// A kernel launched with the programmatic-serialisation attribute may start while its predecessor in
+// the stream is still draining; it must not touch the predecessor's results before pdl_wait().
+// pdl_trigger() tells the runtime that the dependent kernel may be scheduled (all CTAs must call it or
+// exit).  Both are no-ops for ordinary launches.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ---------------------------------------------------------------- small helpers
 
 __device__ __forceinline__ float ex2_approx(float x) {
