@@ -43,12 +43,14 @@ __device__ __forceinline__ float warp_sum(float v) {
     return v;
 }
 
-constexpr int LN_CACHE = 16;  // float4 per lane kept in registers: rows up to 2048 wide in one pass
 
 // out[g][r, :] = bf16( gamma_g * (v - mean) * rstd + beta_g ),  v = a[g][r, :] + y[r, :]
 // where y is absent, a given [rows, d] tensor, or the sum over `ysum_groups` tensors taken in
 // ascending order (the cross-branch sum computed on the fly when the row count is small).
-__global__ void __launch_bounds__(ROW_WARPS * 32)
+// LN_CACHE: float4 per lane kept in registers (16: rows up to 2048 wide in one pass; 8: up to 1024,
+// with half the registers and twice the resident warps)
+template <int LN_CACHE>
+__global__ void __launch_bounds__(ROW_WARPS * 32, LN_CACHE == 8 ? 3 : 1)
 layernorm_kernel(const float *__restrict__ a, long long a_gstride, const float *__restrict__ y,
                  const float *__restrict__ ysum, long long ysum_gstride, int ysum_groups,
                  const uint16_t *__restrict__ gamma, const uint16_t *__restrict__ beta, int groups, int rows, int d,
@@ -178,10 +180,13 @@ int launch_layernorm(const float *a, long long a_gstride, const float *y, const 
     if (!a || !gamma || !out || groups < 1 || rows < 1 || d < 4 || (d & 3)) return KRAKEN_EINVAL;
     if (ysum && (y || ysum_groups < 1 || (ysum_gstride & 3))) return KRAKEN_EINVAL;
     const long long warps = (long long)groups * rows;
-    return cuda_check(launch_pdl(layernorm_kernel, dim3(static_cast<unsigned>((warps + ROW_WARPS - 1) / ROW_WARPS)),
-                                 dim3(ROW_WARPS * 32), 0, stream, a, a_gstride, y, ysum, ysum_gstride, ysum_groups,
-                                 gamma, beta, groups, rows, d, eps, out),
-                      "layernorm: launch");
+    const dim3 grid(static_cast<unsigned>((warps + ROW_WARPS - 1) / ROW_WARPS)), block(ROW_WARPS * 32);
+    const cudaError_t ce =
+        d <= 1024 ? launch_pdl(layernorm_kernel<8>, grid, block, 0, stream, a, a_gstride, y, ysum, ysum_gstride,
+                               ysum_groups, gamma, beta, groups, rows, d, eps, out)
+                  : launch_pdl(layernorm_kernel<16>, grid, block, 0, stream, a, a_gstride, y, ysum, ysum_gstride,
+                               ysum_groups, gamma, beta, groups, rows, d, eps, out);
+    return cuda_check(ce, "layernorm: launch");
 }
 
 int launch_gather_concat(const float *x, long long x_gstride, int groups, int d, const int32_t *rows, int n_rows,
