@@ -50,7 +50,7 @@ __device__ __forceinline__ float warp_sum(float v) {
 // LN_CACHE: float4 per lane kept in registers (16: rows up to 2048 wide in one pass; 8: up to 1024,
 // with half the registers and twice the resident warps)
 template <int LN_CACHE>
-__global__ void __launch_bounds__(ROW_WARPS * 32, LN_CACHE == 8 ? 3 : 1)
+__global__ void __launch_bounds__(ROW_WARPS * 32, LN_CACHE == 8 ? 3 : 0)
 layernorm_kernel(const float *__restrict__ a, long long a_gstride, const float *__restrict__ y,
                  const float *__restrict__ ysum, long long ysum_gstride, int ysum_groups,
                  const uint16_t *__restrict__ gamma, const uint16_t *__restrict__ beta, int groups, int rows, int d,
