@@ -176,10 +176,12 @@ int kraken_op_embed(const int32_t *d_ids, int32_t n_tokens, int32_t seqlen, int3
 
 /* LayerNorm of Algorithm 1, both placements: out_g = LN(a_g + y; gamma_g, beta_g) -> bf16 [G][rows, d].
  * a: fp32 [G][rows, d] with group stride a_gstride elements (0 = shared); y: fp32 [rows, d] or NULL;
- * gamma/beta bf16 [G][d] (beta may be NULL). */
+ * gamma/beta bf16 [G][d] (beta may be NULL).  d_status: device uint32 or NULL; with a status word
+ * and many rows a persistent kernel with bounded waits is used (bit 1 = a wait ran out), without
+ * one the warp-per-row kernel; both give the same bits. */
 int kraken_op_layernorm(const float *d_a, int64_t a_gstride, const float *d_y, const void *gamma,
                         const void *beta, int32_t groups, int32_t rows, int32_t d_model, float eps,
-                        void *d_out_bf16, void *stream);
+                        void *d_out_bf16, uint32_t *d_status, void *stream);
 
 /* Epilogues of the grouped GEMM  C_g = A_g . W_g^T (+ bias_g) ; A bf16 [G][M, K], W bf16 [G][Nout, K]. */
 typedef enum kraken_epilogue {

@@ -107,7 +107,7 @@ def lib() -> C.CDLL:
         L.kraken_last_cuda_error.argtypes = []
         L.kraken_last_cuda_error.restype = C.c_char_p
         L.kraken_op_embed.argtypes = [vp, i32, i32, i32, vp, vp, i32, i32, vp, vp, vp]
-        L.kraken_op_layernorm.argtypes = [vp, i64, vp, vp, vp, i32, i32, i32, C.c_float, vp, vp]
+        L.kraken_op_layernorm.argtypes = [vp, i64, vp, vp, vp, i32, i32, i32, C.c_float, vp, vp, vp]
         L.kraken_op_grouped_gemm.argtypes = [C.POINTER(GemmArgs), vp, vp]
         L.kraken_op_attention.argtypes = [vp, i64, vp, vp, i64, i64, i32, i32, i32, i32, i32, i32, i32, vp, i64, vp]
         L.kraken_op_decode_attention.argtypes = [vp, i64, vp, vp, i64, i64, i32, i32, i32, i32, i32, i32, i32, vp,
@@ -285,13 +285,15 @@ def op_embed(ids: torch.Tensor, seqlen: int, pos0: int, wte: torch.Tensor, wpe: 
 
 
 def op_layernorm(a: torch.Tensor, y: Optional[torch.Tensor], gamma: torch.Tensor, beta: Optional[torch.Tensor],
-                 eps: float = 1e-5, shared_a: bool = False) -> torch.Tensor:
-    """a fp32 [G, rows, d] (or [rows, d] with shared_a, used by every group); gamma [G, d]."""
+                 eps: float = 1e-5, shared_a: bool = False, status: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """a fp32 [G, rows, d] (or [rows, d] with shared_a, used by every group); gamma [G, d]; status: device
+    uint32 word (with it, many-row calls take the persistent kernel)."""
     G, d = gamma.shape
     rows = a.shape[-2]
     out = torch.empty(G, rows, d, dtype=torch.bfloat16, device=a.device)
     _check(lib().kraken_op_layernorm(a.data_ptr(), 0 if shared_a else rows * d, _ptr(y), gamma.data_ptr(),
-                                     _ptr(beta), G, rows, d, eps, out.data_ptr(), _stream()), "kraken_op_layernorm")
+                                     _ptr(beta), G, rows, d, eps, out.data_ptr(), _ptr(status), _stream()),
+           "kraken_op_layernorm")
     return out
 
 

@@ -117,7 +117,7 @@ def run_case(kind: str, workload: str, reps: int, warmup: int, n_tile: int = 0, 
         y = ki.normal_bf16(13, 1, (T, d), 1.0, DEV).float()
         gamma = torch.ones(N, d, dtype=torch.bfloat16, device=DEV)
         beta = torch.zeros(N, d, dtype=torch.bfloat16, device=DEV)
-        fn = lambda: kr.op_layernorm(a, y, gamma, beta)
+        fn = lambda: kr.op_layernorm(a, y, gamma, beta, status=status)
         flops = 0.0
         byts = N * T * d * 4 + T * d * 4 + N * T * d * 2
     else:

@@ -261,7 +261,7 @@ int run_layers(const RunCtx &rc, const int32_t *d_tokens) {
             LaunchScope scope(h, KRAKEN_PROF_LAYERNORM, rc.st);
             KR_TRY(launch_layernorm(xin, xin_gs, nullptr, (const uint16_t *)h->w.ln1_g + ln_off,
                                     h->w.ln1_b ? (const uint16_t *)h->w.ln1_b + ln_off : nullptr, N, T, d, c.ln_eps,
-                                    u, rc.st));
+                                    u, rc.st, nullptr, 0, 0, status));
         }
         // q | k | v ; K and V go straight into the cache
         uint16_t *kc = kv + (long long)l * N * 2 * cache_kv;
@@ -317,7 +317,7 @@ int run_layers(const RunCtx &rc, const int32_t *d_tokens) {
             KR_TRY(launch_layernorm(a, td, sum_here ? nullptr : (l == 0 ? x0 : S),
                                     (const uint16_t *)h->w.ln2_g + ln_off,
                                     h->w.ln2_b ? (const uint16_t *)h->w.ln2_b + ln_off : nullptr, N, T, d, c.ln_eps,
-                                    u, rc.st, sum_here ? x : nullptr, td, N));
+                                    u, rc.st, sum_here ? x : nullptr, td, N, status));
         }
         // FFN up + GELU
         e = epi_zero();
@@ -764,9 +764,11 @@ int kraken_op_embed(const int32_t *d_ids, int32_t n_tokens, int32_t seqlen, int3
 }
 
 int kraken_op_layernorm(const float *d_a, int64_t a_gstride, const float *d_y, const void *gamma, const void *beta,
-                        int32_t groups, int32_t rows, int32_t d_model, float eps, void *d_out_bf16, void *stream) {
+                        int32_t groups, int32_t rows, int32_t d_model, float eps, void *d_out_bf16,
+                        uint32_t *d_status, void *stream) {
     return launch_layernorm(d_a, a_gstride, d_y, (const uint16_t *)gamma, (const uint16_t *)beta, groups, rows,
-                            d_model, eps, (uint16_t *)d_out_bf16, static_cast<cudaStream_t>(stream));
+                            d_model, eps, (uint16_t *)d_out_bf16, static_cast<cudaStream_t>(stream), nullptr, 0, 0,
+                            d_status);
 }
 
 int kraken_op_grouped_gemm(const kraken_gemm_args *g, uint32_t *d_status, void *stream) {

@@ -137,6 +137,132 @@ layernorm_kernel(const float *__restrict__ a, long long a_gstride, const float *
     for (int v = lane + 32 * LN_CACHE; v < nvec; v += 32) emit(v, load(v));
 }
 
+// The same LayerNorm for many rows, as a persistent producer / consumer kernel: what limits the
+// warp-per-row kernel above is that a warp has nothing in flight while it reduces and writes, so here
+// one thread keeps a ring of whole rows in flight with bulk copies (a stage = the N group rows of one
+// row index plus the shared y row, each fetched from DRAM once) and twelve consumer warps take the rows
+// out of shared memory into registers, release the stage at once and then reduce, normalise and store.
+// Consumer warp c works on group c % groups of every (c / groups)-th stage; the number of stages is a
+// multiple of the number of such warp sets, so a ring slot is always consumed by the same set and every
+// waiter sees every phase of the barriers it waits on.
+constexpr int LNS_CONSUMERS = 12;
+constexpr int LNS_THREADS = (LNS_CONSUMERS + 1) * 32;
+constexpr int LNS_MAX_STAGES = 12;
+constexpr int LNS_SMEM_BUDGET = 226 * 1024;
+
+template <int LN_CACHE>
+__global__ void __launch_bounds__(LNS_THREADS, 1)
+layernorm_stream_kernel(const float *__restrict__ a, long long a_gstride, const float *__restrict__ y,
+                        const uint16_t *__restrict__ gamma, const uint16_t *__restrict__ beta, int groups, int rows,
+                        int d, float eps, uint16_t *__restrict__ out, int stages, uint32_t *status) {
+    extern __shared__ __align__(128) uint8_t lns_smem[];
+    __shared__ uint64_t full[LNS_MAX_STAGES], empty[LNS_MAX_STAGES];
+    __shared__ uint32_t abort_word;
+    volatile uint32_t *abort_flag = &abort_word;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t row_bytes = static_cast<uint32_t>(d) * 4u;
+    const uint32_t stage_bytes = row_bytes * (groups + (y ? 1 : 0));
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < stages; ++s) {
+            mbar_init(full + s, 1);
+            mbar_init(empty + s, groups);
+        }
+        abort_word = 0;
+        fence_barrier_init();
+    }
+    // gamma and beta of every group sit behind the ring: with most of the SM's memory carved out as
+    // shared memory the L1 left over does not hold them, and their latency would sit on every row
+    uint16_t *s_gamma = reinterpret_cast<uint16_t *>(lns_smem + (size_t)stages * stage_bytes);
+    uint16_t *s_beta = s_gamma + (size_t)groups * d;
+    for (int i = threadIdx.x; i < groups * d / 4; i += LNS_THREADS) {
+        reinterpret_cast<uint2 *>(s_gamma)[i] = __ldg(reinterpret_cast<const uint2 *>(gamma) + i);
+        reinterpret_cast<uint2 *>(s_beta)[i] = beta ? __ldg(reinterpret_cast<const uint2 *>(beta) + i) : make_uint2(0u, 0u);
+    }
+    __syncthreads();
+    const int n_units = (rows - static_cast<int>(blockIdx.x) + static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x);
+
+    if (warp == LNS_CONSUMERS) {
+        if (lane == 0) {
+            for (int k = 0; k < n_units; ++k) {
+                const int slot = k % stages;
+                const size_t r = blockIdx.x + (size_t)k * gridDim.x;
+                if (!mbar_wait(empty + slot, ((k / stages) & 1) ^ 1, abort_flag)) break;
+                uint8_t *dst = lns_smem + (size_t)slot * stage_bytes;
+                mbar_expect_tx(full + slot, stage_bytes);
+                for (int g = 0; g < groups; ++g)
+                    bulk_load(dst + g * row_bytes, a + g * a_gstride + r * d, row_bytes, full + slot);
+                if (y) bulk_load(dst + groups * row_bytes, y + r * d, row_bytes, full + slot);
+            }
+        }
+        __syncwarp();
+    } else {
+        const int n_sets = LNS_CONSUMERS / groups;
+        const int set = warp / groups, g = warp % groups;
+        const int nvec = d / 4;
+        const uint2 *pg = reinterpret_cast<const uint2 *>(s_gamma + (size_t)g * d);
+        const uint2 *pb = reinterpret_cast<const uint2 *>(s_beta + (size_t)g * d);
+        for (int k = set; k < n_units; k += n_sets) {
+            const int slot = k % stages;
+            const size_t r = blockIdx.x + (size_t)k * gridDim.x;
+            bool ok = mbar_wait(full + slot, (k / stages) & 1, abort_flag);
+            ok = __all_sync(0xFFFFFFFFu, ok);
+            if (!ok) break;
+            const float4 *sa = reinterpret_cast<const float4 *>(lns_smem + (size_t)slot * stage_bytes + g * row_bytes);
+            const float4 *sy = reinterpret_cast<const float4 *>(lns_smem + (size_t)slot * stage_bytes + groups * row_bytes);
+            float4 cache[LN_CACHE];
+            float sum = 0.f;
+#pragma unroll
+            for (int i = 0; i < LN_CACHE; ++i) {
+                const int v = lane + 32 * i;
+                if (v < nvec) {
+                    float4 t = sa[v];
+                    if (y) {
+                        const float4 u = sy[v];
+                        t.x += u.x; t.y += u.y; t.z += u.z; t.w += u.w;
+                    }
+                    cache[i] = t;
+                    sum += (t.x + t.y) + (t.z + t.w);
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(empty + slot);          // the row is in registers: the stage may be refilled
+            const float mean = warp_sum(sum) / d;
+            float sq = 0.f;
+#pragma unroll
+            for (int i = 0; i < LN_CACHE; ++i) {
+                const int v = lane + 32 * i;
+                if (v < nvec) {
+                    const float4 t = cache[i];
+                    const float dx = t.x - mean, dy = t.y - mean, dz = t.z - mean, dw = t.w - mean;
+                    sq += (dx * dx + dy * dy) + (dz * dz + dw * dw);
+                }
+            }
+            const float rstd = rsqrtf(warp_sum(sq) / d + eps);
+            uint2 *po = reinterpret_cast<uint2 *>(out + ((size_t)g * rows + r) * d);
+#pragma unroll
+            for (int i = 0; i < LN_CACHE; ++i) {
+                const int v = lane + 32 * i;
+                if (v < nvec) {
+                    const float4 t = cache[i];
+                    const uint2 gm = pg[v];
+                    const uint2 bt = pb[v];
+                    const float o0 = (t.x - mean) * rstd * bf16_lo(gm.x) + bf16_lo(bt.x);
+                    const float o1 = (t.y - mean) * rstd * bf16_hi(gm.x) + bf16_hi(bt.x);
+                    const float o2 = (t.z - mean) * rstd * bf16_lo(gm.y) + bf16_lo(bt.y);
+                    const float o3 = (t.w - mean) * rstd * bf16_hi(gm.y) + bf16_hi(bt.y);
+                    po[v] = make_uint2(pack_bf16x2(o0, o1), pack_bf16x2(o2, o3));
+                }
+            }
+        }
+    }
+    __syncthreads();
+    if (*abort_flag) {
+        // a wait ran out: give copies still in flight time to land before the shared memory is released
+        for (int i = 0; i < 64; ++i) __nanosleep(10000);
+        if (threadIdx.x == 0 && status) atomicOr(status, STATUS_WAIT_LIMIT);
+    }
+}
+
 __global__ void __launch_bounds__(ROW_WARPS * 32)
 gather_concat_kernel(const float *__restrict__ x, long long x_gstride, int groups, int d,
                      const int32_t *__restrict__ rows, int n_rows, uint16_t *__restrict__ out) {
@@ -174,11 +300,49 @@ int launch_embed(const int32_t *ids, int n_tokens, int seqlen, int pos0, const u
                       "embed: launch");
 }
 
+// whether the persistent kernel takes the call: enough rows to fill its ring on every SM, a stage
+// that fits at least once per consumer set
+bool layernorm_stream_fits(const float *a, long long a_gstride, const float *y, int groups, int rows, int d,
+                           int *stages_out) {
+    if (groups < 1 || LNS_CONSUMERS % groups != 0) return false;
+    if (d > 2048 || (d & 3) || (a_gstride & 3)) return false;
+    if ((reinterpret_cast<uintptr_t>(a) & 15) || (reinterpret_cast<uintptr_t>(y) & 15)) return false;
+    const int sms = sm_count() > 0 ? sm_count() : 148;
+    if (rows < 8 * sms) return false;
+    const int n_sets = LNS_CONSUMERS / groups;
+    const long long stage_bytes = 4LL * d * (groups + (y ? 1 : 0));
+    long long stages = (LNS_SMEM_BUDGET - 4LL * groups * d) / stage_bytes;   // gamma, beta sit behind the ring
+    if (stages > LNS_MAX_STAGES) stages = LNS_MAX_STAGES;
+    stages -= stages % n_sets;
+    if (stages < 2) return false;
+    *stages_out = static_cast<int>(stages);
+    return true;
+}
+
 int launch_layernorm(const float *a, long long a_gstride, const float *y, const uint16_t *gamma,
                      const uint16_t *beta, int groups, int rows, int d, float eps, uint16_t *out,
-                     cudaStream_t stream, const float *ysum, long long ysum_gstride, int ysum_groups) {
+                     cudaStream_t stream, const float *ysum, long long ysum_gstride, int ysum_groups,
+                     uint32_t *status) {
     if (!a || !gamma || !out || groups < 1 || rows < 1 || d < 4 || (d & 3)) return KRAKEN_EINVAL;
     if (ysum && (y || ysum_groups < 1 || (ysum_gstride & 3))) return KRAKEN_EINVAL;
+    int stages = 0;
+    // the persistent kernel has bounded waits, so it needs a status word to report one that ran out
+    if (status && !ysum && !env_flag("KRAKEN_LN_WARP_ROWS") &&
+        layernorm_stream_fits(a, a_gstride, y, groups, rows, d, &stages)) {
+        const size_t smem = (size_t)stages * 4 * d * (groups + (y ? 1 : 0)) + (size_t)4 * groups * d;
+        const int sms = sm_count() > 0 ? sm_count() : 148;
+        auto kern = d <= 1024 ? layernorm_stream_kernel<8> : layernorm_stream_kernel<16>;
+        static bool configured[2] = {false, false};
+        if (!configured[d <= 1024]) {
+            int rc = cuda_check(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                     LNS_SMEM_BUDGET), "layernorm: shared memory opt-in");
+            if (rc) return rc;
+            configured[d <= 1024] = true;
+        }
+        kern<<<dim3(sms), dim3(LNS_THREADS), smem, stream>>>(a, a_gstride, y, gamma, beta, groups, rows, d, eps, out,
+                                                          stages, status);
+        return cuda_check(cudaGetLastError(), "layernorm: launch");
+    }
     const long long warps = (long long)groups * rows;
     const dim3 grid(static_cast<unsigned>((warps + ROW_WARPS - 1) / ROW_WARPS)), block(ROW_WARPS * 32);
     const cudaError_t ce =

@@ -77,7 +77,7 @@ int launch_embed(const int32_t *ids, int n_tokens, int seqlen, int pos0, const u
 int launch_layernorm(const float *a, long long a_gstride, const float *y, const uint16_t *gamma,
                      const uint16_t *beta, int groups, int rows, int d, float eps, uint16_t *out,
                      cudaStream_t stream, const float *ysum = nullptr, long long ysum_gstride = 0,
-                     int ysum_groups = 0);
+                     int ysum_groups = 0, uint32_t *status = nullptr);
 // rows of N fp32 branch outputs -> bf16 branch-major concatenation [n_rows, N*d]; rows picked by index list
 // (device int32, NULL = identity).
 int launch_gather_concat(const float *x, long long x_gstride, int groups, int d, const int32_t *rows, int n_rows,

@@ -69,6 +69,30 @@ def test_layernorm(d, with_y):
     assert ok, worst
 
 
+@pytest.mark.parametrize("G,d,with_y", [(4, 2048, True), (4, 2048, False), (2, 768, True), (1, 1000, False),
+                                        (3, 512, True), (8, 512, True)])
+def test_layernorm_many_rows_persistent_kernel(G, d, with_y):
+    """With a status word and many rows the persistent ring kernel runs: sampled rows against the oracle,
+    every row bit-equal to the warp-per-row kernel (same operations in the same order); ragged row count."""
+    rows = 8 * torch.cuda.get_device_properties(0).multi_processor_count + 37
+    a = (ki.normal_bf16(4, 0, (G, rows, d), 1.0, DEV).float() * 1.3 - 0.2).contiguous()
+    y = ki.normal_bf16(4, 1, (rows, d), 2.0, DEV).float().contiguous() if with_y else None
+    gamma = (1 + ki.normal_bf16(4, 2, (G, d), 0.3, DEV).float()).to(torch.bfloat16)
+    beta = ki.normal_bf16(4, 3, (G, d), 0.3, DEV)
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    out = kr.op_layernorm(a, y, gamma, beta, status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    plain = kr.op_layernorm(a, y, gamma, beta)
+    assert torch.equal(out.view(torch.int16), plain.view(torch.int16))
+    pick = [0, 1, rows // 2, rows - 38, rows - 1]
+    for g in (0, G - 1):
+        ref = oracle.layernorm(a[g][pick].cpu().numpy(), None if y is None else y[pick].cpu().numpy(),
+                               bits(gamma[g]), bits(beta[g]))
+        ok, worst = bf16_ulp_close(out[g][pick].float().cpu().numpy(), ref, ulps=1.0, atol=1e-5)
+        assert ok, (g, worst)
+
+
 # ------------------------------------------------------------------ grouped GEMM
 
 def gemm_case(G, M, Nout, K, epi, n_tile, seed=0, integer=False, shared_resid=False):
