@@ -84,7 +84,7 @@ int kraken_query_sizes(const kraken_config *cfg, size_t *kv_bytes, size_t *scrat
 /* Build a handle: validates the configuration, records the borrowed weight pointers and
  * the caller's KV and scratch buffers (device, 256-byte aligned, at least the queried
  * sizes), encodes the TMA descriptors of the weights.  Host work only.
- * Supported shapes: head_dim in {64, 128}; d_model and d_ff multiples of 64.
+ * Supported shapes: head_dim in {64, 72, 96, 104, 128}; d_model and d_ff multiples of 8.
  * Errors: EINVAL, EUNSUPPORTED, ECAPACITY (undersized buffers), ECUDA. */
 int kraken_create(const kraken_config *cfg, const kraken_weights *weights, void *d_kv, size_t kv_bytes,
                   void *d_scratch, size_t scratch_bytes, kraken_handle **out);

@@ -68,6 +68,41 @@ CONFIGS: Dict[str, KrakenShape] = {
 }
 
 
+def _engine(name, n_branch, n_layer, d_model, n_head):
+    """Engine shape of the paper's TTFT experiments (Table 3 and Sec. 4.2): FFN width 2 d, vocabulary
+    51,200, input context up to 2048, batch 1.  Heads are per sub-layer."""
+    return KrakenShape(name, n_branch, n_layer, d_model, n_head, 2 * d_model, 51200, 2048, 1, 2048)
+
+
+# Table 3, 4-way and 8-way Kraken columns.  The two largest sizes were run by the paper with a quarter
+# of their layers (80 -> 20, 96 -> 24), which is what the "q" in the name records.
+CONFIGS.update({
+    "K1.3B-4": _engine("K1.3B-4", 4, 24, 1248, 12),       # head dim 104
+    "K1.3B-8": _engine("K1.3B-8", 8, 24, 960, 10),        # 96
+    "K6.7B-4": _engine("K6.7B-4", 4, 32, 2496, 24),       # 104
+    "K6.7B-8": _engine("K6.7B-8", 8, 32, 1920, 20),       # 96
+    "K13B-4": _engine("K13B-4", 4, 40, 3120, 30),         # 104
+    "K13B-8": _engine("K13B-8", 8, 40, 2304, 32),         # 72
+    "K65Bq-4": _engine("K65Bq-4", 4, 20, 4992, 39),       # 128
+    "K65Bq-8": _engine("K65Bq-8", 8, 20, 3648, 38),       # 96
+    "K175Bq-4": _engine("K175Bq-4", 4, 24, 7424, 58),     # 128
+    "K175Bq-8": _engine("K175Bq-8", 8, 24, 5472, 57),     # 96
+    # small models with the same head dims and FFN ratio, for element-by-element parity runs
+    "K0-104": KrakenShape("K0-104", 2, 3, 416, 4, 832, 1024, 320, 2, 300),
+    "K0-96": KrakenShape("K0-96", 4, 2, 192, 2, 384, 1024, 320, 1, 200),
+    "K0-72": KrakenShape("K0-72", 2, 2, 288, 4, 576, 1024, 320, 1, 257),
+})
+
+# TTFT in ms printed by the paper for the Kraken engines (Tables 4 and 5; fp16, batch 1, on as many
+# A100-40GB GPUs as the model has branches): {config: {context: ms}}.  Another machine: context only.
+PAPER_TTFT_MS = {
+    "K1.3B-4": {128: 3.3, 2048: 13.2}, "K6.7B-4": {128: 5.8, 2048: 38.0}, "K13B-4": {128: 10.7, 2048: 66.9},
+    "K65Bq-4": {128: 8.5, 2048: 63.8}, "K175Bq-4": {128: 19.9, 2048: 158.9},
+    "K1.3B-8": {128: 3.2, 2048: 9.7}, "K6.7B-8": {128: 4.7, 2048: 27.6}, "K13B-8": {128: 6.7, 2048: 42.6},
+    "K65Bq-8": {128: 6.2, 2048: 42.9}, "K175Bq-8": {128: 12.4, 2048: 98.0},
+}
+
+
 def weight_shapes(s: KrakenShape) -> Dict[str, tuple]:
     L, N, d, F, V, P = s.n_layer, s.n_branch, s.d_model, s.d_ff, s.vocab, s.max_pos
     return {

@@ -24,6 +24,8 @@ struct Layout {
     size_t status, tokens, rows, logits, x0, x, a, s, u, q, o, g, dec_part, total;
 };
 
+bool decode_head_dim_ok(int hd) { return hd == 64 || hd == 72 || hd == 96 || hd == 104 || hd == 128; }
+
 int check_config(const kraken_config *c) {
     if (!c) return KRAKEN_EINVAL;
     if (c->n_branch < 1 || c->n_layer < 1 || c->d_model < 1 || c->n_head < 1 || c->d_ff < 1 || c->vocab < 1 ||
@@ -31,8 +33,10 @@ int check_config(const kraken_config *c) {
         return KRAKEN_EINVAL;
     if (c->d_model % c->n_head != 0) return KRAKEN_EINVAL;
     const int hd = c->d_model / c->n_head;
-    if (hd != 64 && hd != 128) return KRAKEN_EUNSUPPORTED;
-    if (c->d_model % 64 != 0 || c->d_ff % 64 != 0) return KRAKEN_EUNSUPPORTED;
+    // 64 and 128, and the head dims of the paper's engine shapes (Table 3: 72, 96, 104)
+    if (hd != 64 && hd != 72 && hd != 96 && hd != 104 && hd != 128) return KRAKEN_EUNSUPPORTED;
+    // rows of every operand are multiples of 16 bytes (TMA strides, vector accesses)
+    if (c->d_model % 8 != 0 || c->d_ff % 8 != 0) return KRAKEN_EUNSUPPORTED;
     return KRAKEN_OK;
 }
 
@@ -238,6 +242,8 @@ int run_layers(const RunCtx &rc, const int32_t *d_tokens) {
     // decode) LayerNorm-2 of the next layer sums the N branch inputs itself, in the same order.
     const long long down_tiles = (long long)((T + 255) / 256) * ((d + 255) / 256);
     const bool small_rows = !h->naive && (T <= SKINNY_MAX_ROWS || down_tiles < (sm_count() > 0 ? sm_count() : 148) / 2);
+    // between the two: all groups of the down-projection run side by side and one streaming pass adds the N outputs
+    const bool sum_pass = small_rows && T > SKINNY_MAX_ROWS;
     float *x0 = at<float>(h, h->lay.x0), *x = at<float>(h, h->lay.x), *a = at<float>(h, h->lay.a),
           *S = at<float>(h, h->lay.s);
     uint16_t *u = at<uint16_t>(h, h->lay.u), *q = at<uint16_t>(h, h->lay.q), *o = at<uint16_t>(h, h->lay.o),
@@ -313,7 +319,7 @@ int run_layers(const RunCtx &rc, const int32_t *d_tokens) {
             LaunchScope scope(h, KRAKEN_PROF_LAYERNORM, rc.st);
             // with few rows the cross-branch sum is formed here from the N branch inputs (same order as
             // the down-projection epilogue forms it for long prompts)
-            const bool sum_here = small_rows && l > 0;
+            const bool sum_here = small_rows && !sum_pass && l > 0;
             KR_TRY(launch_layernorm(a, td, sum_here ? nullptr : (l == 0 ? x0 : S),
                                     (const uint16_t *)h->w.ln2_g + ln_off,
                                     h->w.ln2_b ? (const uint16_t *)h->w.ln2_b + ln_off : nullptr, N, T, d, c.ln_eps,
@@ -331,6 +337,10 @@ int run_layers(const RunCtx &rc, const int32_t *d_tokens) {
         e.resid = a; e.resid_gstride = td; e.ld_resid = d;
         e.sum = S; e.ld_sum = d;
         KR_TRY(model_gemm(rc, G_DOWN, l, T, gb, (long long)T * F, e));
+        if (sum_pass && l + 1 < L) {
+            LaunchScope scope(h, KRAKEN_PROF_LAYERNORM, rc.st);
+            KR_TRY(launch_sum_groups(x, td, N, td, S, rc.st));
+        }
     }
     h->last_rows = T;
     return KRAKEN_OK;
@@ -747,7 +757,7 @@ const char *kraken_strerror(int status) {
     switch (status) {
         case KRAKEN_OK: return "ok";
         case KRAKEN_EINVAL: return "invalid argument";
-        case KRAKEN_EUNSUPPORTED: return "unsupported shape (head_dim must be 64 or 128; d_model and d_ff multiples of 64)";
+        case KRAKEN_EUNSUPPORTED: return "unsupported shape (head_dim must be 64, 72, 96, 104 or 128; d_model and d_ff multiples of 8)";
         case KRAKEN_ECAPACITY: return "capacity exceeded (batch, sequence length or buffer size)";
         case KRAKEN_ESTATE: return "call order violated (prefill first; decode batch must equal the prefill batch)";
         case KRAKEN_ECUDA: return "a CUDA call failed";
@@ -782,7 +792,10 @@ int kraken_op_grouped_gemm(const kraken_gemm_args *g, uint32_t *d_status, void *
     if (k == KRAKEN_EPI_RESID_SUM && !g->sum) return KRAKEN_EINVAL;
     if (k == KRAKEN_EPI_QKV) {
         if (!g->k_cache || !g->v_cache || g->seqlen < 1 || g->n_head < 1 || g->pos0 < 0) return KRAKEN_EINVAL;
-        if (g->head_dim % 32 != 0 || g->n_out != 3 * g->n_head * g->head_dim) return KRAKEN_EUNSUPPORTED;
+        // q | k | v and head boundaries fall on 16-byte pieces; the q rows and cache rows must be 16-byte aligned
+        if (g->head_dim % 8 != 0 || g->n_out != 3 * g->n_head * g->head_dim || g->ld_out_bf16 % 8 != 0 ||
+            g->out_bf16_gstride % 8 != 0 || g->cache_gstride % 8 != 0)
+            return KRAKEN_EUNSUPPORTED;
     }
     GemmOperands op{g->a, g->a_gstride, g->lda, g->w, g->w_gstride, g->ldw};
     GemmShape s{g->groups, g->m, g->n_out, g->k};
@@ -823,7 +836,7 @@ int kraken_op_decode_attention(const void *q, int64_t q_gstride, const void *k_c
                                int32_t n_keys, int32_t n_head, int32_t head_dim, int32_t max_pos, int32_t splits,
                                void *d_partials, size_t partial_bytes, void *out, int64_t out_gstride, void *stream) {
     if (groups < 1 || batch < 1 || n_head < 1 || n_keys < 1) return KRAKEN_EINVAL;
-    if (head_dim != 64 && head_dim != 128) return KRAKEN_EUNSUPPORTED;
+    if (!decode_head_dim_ok(head_dim)) return KRAKEN_EUNSUPPORTED;
     if (splits == 0) splits = decode_attention_splits(groups, batch, n_head, n_keys);
     if (splits < 1 || splits > DECODE_MAX_SPLITS) return KRAKEN_EINVAL;
     if (splits > 1 && (!d_partials || partial_bytes < decode_attention_partial_bytes(groups, batch, n_head, head_dim, splits)))
@@ -841,7 +854,7 @@ int kraken_op_decode_attention(const void *q, int64_t q_gstride, const void *k_c
 int kraken_decode_attention_sizes(int32_t groups, int32_t batch, int32_t n_keys, int32_t n_head, int32_t head_dim,
                                   int32_t *splits, size_t *partial_bytes) {
     if (groups < 1 || batch < 1 || n_head < 1 || n_keys < 1 || !splits || !partial_bytes) return KRAKEN_EINVAL;
-    if (head_dim != 64 && head_dim != 128) return KRAKEN_EUNSUPPORTED;
+    if (!decode_head_dim_ok(head_dim)) return KRAKEN_EUNSUPPORTED;
     if (*splits == 0) *splits = decode_attention_splits(groups, batch, n_head, n_keys);
     if (*splits < 1 || *splits > DECODE_MAX_SPLITS) return KRAKEN_EINVAL;
     *partial_bytes = *splits > 1 ? decode_attention_partial_bytes(groups, batch, n_head, head_dim, *splits) : 0;

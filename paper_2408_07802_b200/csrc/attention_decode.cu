@@ -20,13 +20,15 @@ constexpr int UNROLL = 4;
 template <int HD>
 __global__ void __launch_bounds__(DEC_WARPS * 32)
 attn_decode_kernel(const DecodeAttnParams p) {
-    constexpr int LPR = HD / 8;       // lanes per cache row (16 bytes each)
-    constexpr int RPW = 32 / LPR;     // rows per warp-wide load
+    constexpr int LPR = HD / 8;       // lanes that hold one cache row (16 bytes each)
+    constexpr int GRP = LPR <= 8 ? 8 : 16;   // lanes set aside per row: the next power of two (the rest idle)
+    constexpr int RPW = 32 / GRP;     // rows per warp-wide load
     pdl_wait();
     const int split = blockIdx.x, h = blockIdx.y;
     const int b = blockIdx.z % p.batch, g = blockIdx.z / p.batch;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int sub = lane % LPR, rg = lane / LPR;
+    const int sub = lane % GRP, rg = lane / GRP;
+    const bool active = sub < LPR;
     const int d = p.n_head * HD;
 
     // keys of this split
@@ -35,7 +37,7 @@ attn_decode_kernel(const DecodeAttnParams p) {
     const int k_begin = split * per;
     const int k_end = min(n_keys, k_begin + per);
 
-    const uint16_t *gq = p.q + g * p.q_gstride + (long long)b * d + h * HD + sub * 8;
+    const uint16_t *gq = p.q + g * p.q_gstride + (long long)b * d + h * HD + (active ? sub : 0) * 8;
     const uint16_t *gk = p.k_cache + g * p.cache_gstride + b * p.cache_bstride + (long long)h * p.max_pos * HD;
     const uint16_t *gv = p.v_cache + g * p.cache_gstride + b * p.cache_bstride + (long long)h * p.max_pos * HD;
 
@@ -60,8 +62,8 @@ attn_decode_kernel(const DecodeAttnParams p) {
             const int key = r0 + u * RPW + rg;
             valid[u] = key < k_end;
             const long long off = (long long)(valid[u] ? key : k_begin) * HD + sub * 8;
-            kk[u] = *reinterpret_cast<const uint4 *>(gk + off);
-            vv[u] = *reinterpret_cast<const uint4 *>(gv + off);
+            kk[u] = active ? *reinterpret_cast<const uint4 *>(gk + off) : make_uint4(0u, 0u, 0u, 0u);
+            vv[u] = active ? *reinterpret_cast<const uint4 *>(gv + off) : make_uint4(0u, 0u, 0u, 0u);
         }
         float s[UNROLL];
         float mx = m;
@@ -76,7 +78,7 @@ attn_decode_kernel(const DecodeAttnParams p) {
             acc = fmaf(qf[6], bf16_lo(kk[u].w), acc);
             acc = fmaf(qf[7], bf16_hi(kk[u].w), acc);
 #pragma unroll
-            for (int off = 1; off < LPR; off <<= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, off);
+            for (int off = 1; off < GRP; off <<= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, off);
             s[u] = valid[u] ? acc : -INFINITY;
             mx = fmaxf(mx, s[u]);
         }
@@ -105,7 +107,7 @@ attn_decode_kernel(const DecodeAttnParams p) {
     pdl_trigger();
     // merge the row groups of the warp (lanes with equal `sub`), then the warps through shared memory
 #pragma unroll
-    for (int off = LPR; off < 32; off <<= 1) {
+    for (int off = GRP; off < 32; off <<= 1) {
         const float m2 = __shfl_xor_sync(0xFFFFFFFFu, m, off);
         const float l2 = __shfl_xor_sync(0xFFFFFFFFu, l, off);
         const float mn = fmaxf(m, m2);
@@ -120,7 +122,7 @@ attn_decode_kernel(const DecodeAttnParams p) {
         m = mn;
     }
     __shared__ float sm_m[DEC_WARPS], sm_l[DEC_WARPS], sm_o[DEC_WARPS][HD];
-    if (rg == 0) {
+    if (rg == 0 && active) {
 #pragma unroll
         for (int i = 0; i < 8; ++i) sm_o[warp][sub * 8 + i] = o[i];
         if (sub == 0) {
@@ -215,9 +217,14 @@ int launch_attention_decode(const DecodeAttnParams &p, cudaStream_t stream) {
     if (!p.q || !p.k_cache || !p.v_cache || !p.out || p.groups < 1 || p.batch < 1 || p.n_head < 1 || p.n_keys < 1 ||
         p.n_keys > p.max_pos || p.splits < 1 || p.splits > DECODE_MAX_SPLITS || (p.splits > 1 && !p.partials))
         return KRAKEN_EINVAL;
-    if (p.head_dim == 64) return launch<64>(p, stream);
-    if (p.head_dim == 128) return launch<128>(p, stream);
-    return KRAKEN_EUNSUPPORTED;
+    switch (p.head_dim) {   // 64 and 128, and the head dims of the paper's engine shapes (Table 3)
+        case 64: return launch<64>(p, stream);
+        case 72: return launch<72>(p, stream);
+        case 96: return launch<96>(p, stream);
+        case 104: return launch<104>(p, stream);
+        case 128: return launch<128>(p, stream);
+        default: return KRAKEN_EUNSUPPORTED;
+    }
 }
 
 }  // namespace kr

@@ -40,6 +40,7 @@ constexpr bool POLY_EXP2 = false;
 
 struct AttnTcArgs {
     int groups, batch, seqlen, pos0, n_head;
+    int head_dim;      // <= HD of the kernel instance, a multiple of 8 (columns past it are zero-filled by TMA)
     uint16_t *out;
     long long out_gstride;
     uint32_t *status;
@@ -232,7 +233,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 for (int w = 0; w < q_tiles; ++w)
 #pragma unroll
                     for (int hf = 0; hf < Cfg::HALVES; ++hf)
-                        tma_load_3d(sQ + w * Cfg::Q_BYTES + hf * Cfg::TILE_BYTES, &tmQ, q_full, it.h * HD + hf * 64,
+                        tma_load_3d(sQ + w * Cfg::Q_BYTES + hf * Cfg::TILE_BYTES, &tmQ, q_full, it.h * a.head_dim + hf * 64,
                                     it.b * a.seqlen + it.q0 + w * TQ, it.g);
                 for (int j = 0; ok && j < it.n_max; ++j, ++kv_cnt) {
                     const int st = kv_cnt & 1;
@@ -255,14 +256,18 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         __syncwarp();
     } else if (warp == 1) {
         if (lane == 0) {
+            // head dims below HD: the scores need ceil(head_dim / 16) steps (K is zero beyond head_dim, so
+            // whatever Q holds there does not count), the output ceil(head_dim / 16) * 16 columns
+            const int qk_steps = (a.head_dim + 15) / 16;
             constexpr uint32_t idesc_qk = umma_idesc_bf16(TQ, TK);
-            constexpr uint32_t idesc_pv = umma_idesc_bf16(TQ, HD) | (1u << 16);  // B (V) is MN-major
+            const uint32_t idesc_pv = umma_idesc_bf16(TQ, qk_steps * 16) | (1u << 16);  // B (V) is MN-major
             auto issue_qk = [&](int w, int st) {
                 const uint32_t q_addr = smem_u32(sQ + w * Cfg::Q_BYTES);
                 const uint32_t k_addr = smem_u32(sK + st * Cfg::KV_BYTES);
                 const uint32_t d_tmem = tmem_base + Cfg::S_COL0 + w * TK;
 #pragma unroll
                 for (int ks = 0; ks < HD / 16; ++ks) {
+                    if (ks >= qk_steps) break;
                     const uint32_t off = (ks >> 2) * Cfg::TILE_BYTES + (ks & 3) * 32;
                     umma_bf16_ss(d_tmem, umma_desc_sw128_kmajor(q_addr + off), umma_desc_sw128_kmajor(k_addr + off),
                                  idesc_qk, ks != 0 ? 1u : 0u);
@@ -327,7 +332,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
         const uint32_t s_addr = lane_addr + Cfg::S_COL0 + w * TK;
         const uint32_t o_addr = lane_addr + Cfg::O_COL0 + w * TK;
-        const float sl2 = rsqrtf(static_cast<float>(HD)) * 1.4426950408889634f;
+        const float sl2 = rsqrtf(static_cast<float>(a.head_dim)) * 1.4426950408889634f;
         bool ok = true;
         uint32_t tile_cnt = 0;                               // tiles this warp group has consumed so far
         AtcItem it;
@@ -432,8 +437,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 if (!ok) break;
                 tc_fence_after_sync();
                 const float inv = 1.f / l;
-                const int d = a.n_head * HD;
-                uint16_t *dst = a.out + it.g * a.out_gstride + ((long long)it.b * a.seqlen + tile_q0 + row) * d + it.h * HD;
+                const int d = a.n_head * a.head_dim;
+                uint16_t *dst = a.out + it.g * a.out_gstride + ((long long)it.b * a.seqlen + tile_q0 + row) * d +
+                                it.h * a.head_dim;
 #pragma unroll
                 for (int c = 0; c < HD / 32; ++c) {
                     uint32_t r[32];
@@ -442,6 +448,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     if (row < rows_valid) {
 #pragma unroll
                         for (int i = 0; i < 4; ++i) {
+                            if (c * 32 + 8 * i >= a.head_dim) break;
                             uint4 u;
                             u.x = pack_bf16x2(__uint_as_float(r[8 * i + 0]) * inv, __uint_as_float(r[8 * i + 1]) * inv);
                             u.y = pack_bf16x2(__uint_as_float(r[8 * i + 2]) * inv, __uint_as_float(r[8 * i + 3]) * inv);
@@ -492,7 +499,9 @@ int launch(const CUtensorMap &tmQ, const CUtensorMap &tmK, const CUtensorMap &tm
 }  // namespace
 
 bool attention_tc_supported(const AttnParams &p) {
-    if (p.head_dim != 64 && p.head_dim != 128) return false;
+    // any head dim that is a multiple of 8 (16-byte rows for TMA) up to 128: the 64- or 128-wide kernel
+    // instance runs it with the missing columns zero-filled by the tensor maps
+    if (p.head_dim < 16 || p.head_dim > 128 || (p.head_dim & 7)) return false;
     // the cache of one group must be [batch][head][max_pos][head_dim] without gaps
     if (p.cache_bstride != (long long)p.n_head * p.max_pos * p.head_dim) return false;
     const int d = p.n_head * p.head_dim;
@@ -540,10 +549,11 @@ int launch_attention_tc(const AttnParams &p, const CUtensorMap *tmQ, const CUten
     a.seqlen = p.seqlen;
     a.pos0 = p.pos0;
     a.n_head = p.n_head;
+    a.head_dim = p.head_dim;
     a.out = p.out;
     a.out_gstride = p.out_gstride;
     a.status = d_status;
-    return p.head_dim == 64 ? launch<64>(*tmQ, *tmK, *tmV, a, stream) : launch<128>(*tmQ, *tmK, *tmV, a, stream);
+    return p.head_dim <= 64 ? launch<64>(*tmQ, *tmK, *tmV, a, stream) : launch<128>(*tmQ, *tmK, *tmV, a, stream);
 }
 
 }  // namespace kr

@@ -281,6 +281,25 @@ gather_concat_kernel(const float *__restrict__ x, long long x_gstride, int group
     }
 }
 
+// out = x_0 + x_1 + ... + x_{G-1} element by element, added in ascending group order (the order the
+// down-projection epilogue and LayerNorm-2 use when they form the same cross-branch sum themselves)
+__global__ void __launch_bounds__(256)
+sum_groups_kernel(const float *__restrict__ x, long long gstride, int groups, long long n4, float *__restrict__ out) {
+    pdl_wait();
+    pdl_trigger();
+    const float4 *px = reinterpret_cast<const float4 *>(x);
+    float4 *po = reinterpret_cast<float4 *>(out);
+    const long long stride = (long long)gridDim.x * blockDim.x, gs4 = gstride / 4;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += stride) {
+        float4 acc = px[i];
+        for (int g = 1; g < groups; ++g) {
+            const float4 t = px[g * gs4 + i];
+            acc.x += t.x; acc.y += t.y; acc.z += t.z; acc.w += t.w;
+        }
+        po[i] = acc;
+    }
+}
+
 __global__ void f32_to_bf16_kernel(const float *__restrict__ in, uint16_t *__restrict__ out, long long n) {
     long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     const long long stride = (long long)gridDim.x * blockDim.x;
@@ -360,6 +379,19 @@ int launch_gather_concat(const float *x, long long x_gstride, int groups, int d,
     return cuda_check(launch_pdl(gather_concat_kernel, dim3(static_cast<unsigned>((warps + ROW_WARPS - 1) / ROW_WARPS)),
                                  dim3(ROW_WARPS * 32), 0, stream, x, x_gstride, groups, d, rows, n_rows, out),
                       "gather: launch");
+}
+
+int launch_sum_groups(const float *x, long long gstride, int groups, long long n, float *out, cudaStream_t stream) {
+    if (!x || !out || groups < 1 || n < 4 || (n & 3) || (gstride & 3) || (reinterpret_cast<uintptr_t>(x) & 15) ||
+        (reinterpret_cast<uintptr_t>(out) & 15))
+        return KRAKEN_EINVAL;
+    const long long n4 = n / 4;
+    const int sms = sm_count() > 0 ? sm_count() : 148;
+    long long blocks = (n4 + 255) / 256;
+    if (blocks > 8LL * sms) blocks = 8LL * sms;
+    return cuda_check(launch_pdl(sum_groups_kernel, dim3(static_cast<unsigned>(blocks)), dim3(256), 0, stream, x, gstride,
+                                 groups, n4, out),
+                      "sum over groups: launch");
 }
 
 int launch_f32_to_bf16(const float *in, uint16_t *out, long long n, cudaStream_t stream) {

@@ -78,6 +78,8 @@ int launch_layernorm(const float *a, long long a_gstride, const float *y, const 
                      const uint16_t *beta, int groups, int rows, int d, float eps, uint16_t *out,
                      cudaStream_t stream, const float *ysum = nullptr, long long ysum_gstride = 0,
                      int ysum_groups = 0, uint32_t *status = nullptr);
+// out[i] = sum over groups of x[g * gstride + i], ascending g; n elements (a multiple of 4), 16-byte aligned
+int launch_sum_groups(const float *x, long long gstride, int groups, long long n, float *out, cudaStream_t stream);
 // rows of N fp32 branch outputs -> bf16 branch-major concatenation [n_rows, N*d]; rows picked by index list
 // (device int32, NULL = identity).
 int launch_gather_concat(const float *x, long long x_gstride, int groups, int d, const int32_t *rows, int n_rows,

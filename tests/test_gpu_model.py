@@ -275,6 +275,47 @@ def prefix_parity(name, prefix, seqs):
     m.close()
 
 
+@pytest.mark.parametrize("name", ["K0-104", "K0-96", "K0-72"])
+def test_engine_head_dims_small_models_all_positions_cache_and_decode(name):
+    """Small models with the head dims (104, 96, 72) and the 2 d FFN of the paper's engine shapes (Table 3):
+    every position and the cache element by element, then teacher-forced decode steps."""
+    s = ki.CONFIGS[name]
+    m, w = build(s)
+    wb = host_bits(w)
+    steps = 4
+    tok = ki.uniform_tokens(5, s.vocab, s.batch, s.seqlen + steps, DEV)
+    first = tok[:, :s.seqlen].contiguous()
+    got_all = m.prefill_all_logits(first).cpu().numpy()
+    orcs = []
+    for b in range(s.batch):
+        ids = tok[b, :s.seqlen].cpu().numpy()
+        ref32, _ = oracle_all_logits(s, wb, ids, False)
+        refbf, orc = oracle_all_logits(s, wb, ids, True)
+        check_parity(got_all[b], ref32, refbf, f"{name} seq {b} all positions")
+        for layer in range(s.n_layer):
+            for n in range(s.n_branch):
+                for which in (0, 1):
+                    g = m.kv_view(layer, n, which)[b, :, :s.seqlen].float().cpu().numpy()
+                    check_cache(g, orc.cache(layer, n, which), layer == 0, (name, b, layer, n, which))
+        orcs.append(oracle.Oracle(s, wb, bf16_store=False))
+        orcs[-1].prefill(ids)
+    assert m.device_status() == 0
+    for t in range(steps):
+        got = m.decode_step(tok[:, s.seqlen + t].contiguous()).cpu().numpy()
+        for b in range(s.batch):
+            ref = orcs[b].decode_step(int(tok[b, s.seqlen + t]))
+            rel, mx = logits_metrics(got[b], ref)
+            assert rel <= REL_L2_MAX and mx <= MAX_ABS_MAX, (name, t, b, rel, mx)
+    assert m.device_status() == 0 and m.cur_len == s.seqlen + steps
+    m.close()
+
+
+def test_engine_shape_1p3b_4way_full_size_prefix_parity():
+    """The paper's 1.3B 4-way engine shape (d 1248 = 12 heads of 104, FFN 2496, vocabulary 51,200) at its full
+    2048-token context, in the launch configuration the benchmark times."""
+    prefix_parity("K1.3B-4", 40, [0])
+
+
 def test_c2_full_size_prefix_parity():
     prefix_parity("C2", 128, [0])
 

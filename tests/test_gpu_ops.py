@@ -187,9 +187,10 @@ def test_gemm_cross_branch_sum(n_tile):
     assert np.array_equal(r["sum"], r["ref"].sum(0))
 
 
-@pytest.mark.parametrize("hd,H", [(64, 2), (128, 1)])
+@pytest.mark.parametrize("hd,H", [(64, 2), (128, 1), (104, 3), (72, 2), (96, 1), (96, 3)])
 def test_gemm_qkv_scatter_is_index_exact(hd, H):
-    """One-hot activations times integer-coded weights: every cache element names its source."""
+    """One-hot activations times integer-coded weights: every cache element names its source.  Head dims that
+    are not multiples of 32 (and widths that are not) take the path that stores 16-byte pieces."""
     d = H * hd
     G, batch, seqlen, pos0, P, K = 2, 3, 50, 7, 64, 64
     M = batch * seqlen
@@ -244,10 +245,12 @@ def test_gemm_rejects_unaligned():
 # ------------------------------------------------------------------ attention
 
 @pytest.mark.parametrize("kernel", ["tcgen05", "warp_mma"])
-@pytest.mark.parametrize("hd", [64, 128])
+@pytest.mark.parametrize("hd", [64, 128, 72, 96, 104])
 @pytest.mark.parametrize("seqlen,pos0", [(200, 0), (100, 37), (1, 90), (64, 0), (300, 0), (129, 127)])
 def test_attention_matches_oracle(hd, seqlen, pos0, kernel, monkeypatch):
     if kernel == "warp_mma":
+        if hd not in (64, 128):
+            pytest.skip("the warp-MMA kernel covers head dims 64 and 128 only")
         monkeypatch.setenv("KRAKEN_ATTN_WARP_MMA", "1")   # the m16n8k16 kernel kept for odd cache strides
     G, B, H, P = 2, 2, 2, 512
     d = H * hd
@@ -274,7 +277,7 @@ def test_attention_matches_oracle(hd, seqlen, pos0, kernel, monkeypatch):
     assert np.sqrt(num / den) < 6e-3, np.sqrt(num / den)
 
 
-@pytest.mark.parametrize("hd", [64, 128])
+@pytest.mark.parametrize("hd", [64, 128, 72, 96, 104])
 @pytest.mark.parametrize("n_keys,splits", [(1, 1), (2, 0), (131, 3), (700, 0), (2049, 32), (300, 1)])
 def test_decode_attention_matches_oracle(hd, n_keys, splits):
     G, B, H, P = 2, 3, 2, 2112
