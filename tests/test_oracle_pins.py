@@ -244,6 +244,18 @@ def test_matches_library_composition(final_ln):
         assert np.max(np.abs(lo[-1, n] - ref_x[n])) < 2e-5
 
 
+@pytest.mark.parametrize("d_model,n_head", [(144, 2), (208, 2), (96, 1)])
+def test_engine_head_dims_match_library_composition(d_model, n_head):
+    """Head dims of the paper's engine shapes (Table 3: 72, 104, 96) with the 2 d FFN: the oracle against the
+    same composition written with library routines."""
+    shape = small_shape(d_model=d_model, n_head=n_head, d_ff=2 * d_model, n_branch=2)
+    w = rand_weights(shape)
+    ids = ki.uniform_tokens(11, shape.vocab, 1, shape.seqlen)[0].numpy()
+    ref, _ = torch_kraken(shape, w, ids, final_ln=True)
+    got, _ = oracle.Oracle(shape, wbits(w)).prefill(ids)
+    assert np.max(np.abs(got - ref)) < 2e-5 * max(1.0, np.max(np.abs(ref)))
+
+
 def test_c0_matches_library_composition():
     shape = ki.CONFIGS["C0"]
     w = ki.make_weights(shape, seed=0)
@@ -455,3 +467,19 @@ def test_parameter_counts_match_paper_tables():
             d, printed = int(r[2]), float(r[3])
             got = ki.param_count(1, 1, d, 0, 4 * d) / 1e6
             assert abs(got - printed) / printed < 3e-3, (r, got)
+
+
+def test_engine_configs_follow_table3():
+    """The K* workloads are the Kraken columns of Table 3: (degree, width) pairs as printed, FFN 2 d, vocabulary
+    51,200, 2048-token context, batch 1 (Sec. 4.2), and the TTFT table names only those workloads."""
+    rows = [ln.split() for ln in open(os.path.join(GOLDEN, "paper_param_tables.txt"))
+            if ln.strip() and not ln.startswith("#")]
+    printed = {(int(r[1]), int(r[2])) for r in rows if r[0] == "table3"}
+    engines = {k: s for k, s in ki.CONFIGS.items() if k.startswith("K") and not k.startswith("K0")}
+    assert {(s.n_branch, s.d_model) for s in engines.values()} == printed
+    for s in engines.values():
+        assert s.d_ff == 2 * s.d_model and s.vocab == 51200 and s.max_pos == 2048 and s.batch == 1
+        assert s.d_model % s.n_head == 0 and s.head_dim in (72, 96, 104, 128)
+    assert set(ki.PAPER_TTFT_MS) == set(engines)
+    assert all(set(v) == {128, 2048} for v in ki.PAPER_TTFT_MS.values())
+
