@@ -50,10 +50,20 @@ class KrakenShape:
     ln_eps: float = 1e-5
     gelu_tanh: int = 0
     final_ln: int = 1
+    n_kv_head: int = 0      # key/value heads per sub-layer; 0 = n_head (multi-head), 1 = multi-query
 
     @property
     def head_dim(self) -> int:
         return self.d_model // self.n_head
+
+    @property
+    def kv_heads(self) -> int:
+        return self.n_kv_head or self.n_head
+
+    @property
+    def qkv_width(self) -> int:
+        """Output width of the fused q | k | v projection: d + 2 * kv_heads * head_dim."""
+        return self.d_model + 2 * self.kv_heads * self.head_dim
 
     def asdict(self):
         return asdict(self)
@@ -65,6 +75,12 @@ CONFIGS: Dict[str, KrakenShape] = {
     "C2": KrakenShape("C2", 4, 24, 1024, 16, 4096, 50257, 1024, 1, 1024),
     "C3": KrakenShape("C3", 4, 32, 2048, 16, 8192, 50257, 2048, 4, 2048),
     "C4": KrakenShape("C4", 4, 24, 1024, 16, 4096, 50257, 2176, 16, 2048, decode_steps=128),
+    # C4 with grouped-query (4 query heads per key/value head) and multi-query attention: the mitigation
+    # the paper names for the KV cache that grows with the number of branches (Sec. 4.2)
+    "C4-gqa4": KrakenShape("C4-gqa4", 4, 24, 1024, 16, 4096, 50257, 2176, 16, 2048, decode_steps=128, n_kv_head=4),
+    "C4-mqa": KrakenShape("C4-mqa", 4, 24, 1024, 16, 4096, 50257, 2176, 16, 2048, decode_steps=128, n_kv_head=1),
+    "C0-gqa": KrakenShape("C0-gqa", 2, 4, 256, 4, 512, 4096, 160, 2, 128, n_kv_head=2),
+    "C0-mqa": KrakenShape("C0-mqa", 2, 3, 256, 4, 512, 4096, 160, 1, 150, n_kv_head=1),
 }
 
 
@@ -108,7 +124,7 @@ def weight_shapes(s: KrakenShape) -> Dict[str, tuple]:
     return {
         "wte": (V, d), "wpe": (P, d),
         "ln1_g": (L, N, d), "ln1_b": (L, N, d),
-        "w_qkv": (L, N, 3 * d, d), "b_qkv": (L, N, 3 * d),
+        "w_qkv": (L, N, s.qkv_width, d), "b_qkv": (L, N, s.qkv_width),
         "w_proj": (L, N, d, d), "b_proj": (L, N, d),
         "ln2_g": (L, N, d), "ln2_b": (L, N, d),
         "w_up": (L, N, F, d), "b_up": (L, N, F),
@@ -248,7 +264,7 @@ def algorithmic_flops(s: KrakenShape, batch: Optional[int] = None, seqlen: Optio
     l = s.seqlen if seqlen is None else seqlen
     T = B * l
     N, L, d, F, H, hd, V = s.n_branch, s.n_layer, s.d_model, s.d_ff, s.n_head, s.head_dim, s.vocab
-    gemm = 2.0 * T * N * L * (4 * d * d + 2 * d * F)
+    gemm = 2.0 * T * N * L * (d * s.qkv_width + d * d + 2 * d * F)
     attn = float(N * L * B * H) * 4 * hd * (l * (l + 1) / 2)
     tail = 2.0 * B * (N * d * d + V * d)
     return {"gemm": gemm, "attn": attn, "tail": tail, "total": gemm + attn + tail}

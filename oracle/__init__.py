@@ -36,7 +36,7 @@ class KoConfig(C.Structure):
     _fields_ = [(n, C.c_int32) for n in
                 ("n_branch", "n_layer", "d_model", "n_head", "d_ff", "vocab", "max_pos")] + [
         ("ln_eps", C.c_float), ("gelu_tanh", C.c_int32), ("final_ln", C.c_int32),
-        ("bf16_store", C.c_int32), ("y_zero", C.c_int32)]
+        ("bf16_store", C.c_int32), ("y_zero", C.c_int32), ("n_kv_head", C.c_int32)]
 
 
 class KoWeights(C.Structure):
@@ -148,7 +148,7 @@ class Oracle:
             d_ff=shape.d_ff, vocab=shape.vocab, max_pos=shape.max_pos, ln_eps=shape.ln_eps,
             gelu_tanh=int(shape.gelu_tanh if gelu_tanh is None else gelu_tanh),
             final_ln=int(shape.final_ln if final_ln is None else final_ln),
-            bf16_store=int(bf16_store), y_zero=int(y_zero))
+            bf16_store=int(bf16_store), y_zero=int(y_zero), n_kv_head=int(getattr(shape, "n_kv_head", 0)))
         self._keep = {k: _bits(v) for k, v in weights_bits.items()}
         self.w = KoWeights(**{k: _ptr(self._keep.get(k)) for k in WEIGHT_FIELDS})
         self.shape = shape
@@ -188,11 +188,12 @@ class Oracle:
         return logits
 
     def cache(self, layer: int, branch: int, which: int) -> np.ndarray:
-        """K (which=0) or V (which=1) rows as [H, cur_len, hd] fp32 (copy)."""
+        """K (which=0) or V (which=1) rows as [key/value heads, cur_len, hd] fp32 (copy)."""
         s = self.shape
         hd = s.head_dim
-        out = np.empty((s.n_head, self.cur_len, hd), dtype=np.float32)
-        for h in range(s.n_head):
+        n_kv = getattr(s, "n_kv_head", 0) or s.n_head
+        out = np.empty((n_kv, self.cur_len, hd), dtype=np.float32)
+        for h in range(n_kv):
             p = lib().ko_cache_ptr(self._h, layer, branch, which, h)
             arr = np.ctypeslib.as_array(p, shape=(s.max_pos, hd))
             out[h] = arr[: self.cur_len]

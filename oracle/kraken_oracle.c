@@ -47,6 +47,10 @@ typedef struct ko_config {
     int32_t final_ln;    /* 1: LayerNorm between W_concat and the unembedding */
     int32_t bf16_store;  /* 1: round activations to bf16 at the store points */
     int32_t y_zero;      /* test-only: drop the y term (reduces N = 1 to a GPT-2 stack) */
+    int32_t n_kv_head;   /* key/value heads per sub-layer: 0 or n_head = multi-head attention; fewer =
+                            grouped-query attention, 1 = multi-query (the KV-cache mitigation of Sec. 4.2
+                            and the KV-cache appendix): query head h reads key/value head
+                            h / (n_head / n_kv_head) */
 } ko_config;
 
 typedef struct ko_weights { /* host pointers to bf16 bit patterns; bias / beta may be NULL */
@@ -60,7 +64,7 @@ typedef struct ko_state {
     ko_config cfg;
     ko_weights w;
     int32_t cur_len;
-    float *kcache; /* [L][N][H][max_pos][hd] */
+    float *kcache; /* [L][N][H_kv][max_pos][hd] */
     float *vcache;
 } ko_state;
 
@@ -202,8 +206,10 @@ void ko_attention_head(const float *q, int64_t q_stride, const float *k, const f
 
 /* ---------------------------------------------------------------- model */
 
+static int kv_heads(const ko_config *c) { return c->n_kv_head > 0 ? c->n_kv_head : c->n_head; }
+
 size_t ko_cache_floats(const ko_config *c) {
-    return (size_t)c->n_layer * c->n_branch * (size_t)c->max_pos * c->d_model;
+    return (size_t)c->n_layer * c->n_branch * (size_t)c->max_pos * kv_heads(c) * (c->d_model / c->n_head);
 }
 
 ko_state *ko_create(const ko_config *cfg, const ko_weights *w) {
@@ -211,6 +217,7 @@ ko_state *ko_create(const ko_config *cfg, const ko_weights *w) {
     if (cfg->n_branch < 1 || cfg->n_layer < 1 || cfg->d_model < 1 || cfg->n_head < 1 ||
         cfg->d_model % cfg->n_head != 0 || cfg->d_ff < 1 || cfg->vocab < 1 || cfg->max_pos < 1)
         return NULL;
+    if (cfg->n_kv_head < 0 || (cfg->n_kv_head > 0 && cfg->n_head % cfg->n_kv_head != 0)) return NULL;
     ko_state *s = (ko_state *)calloc(1, sizeof(ko_state));
     if (!s) return NULL;
     s->cfg = *cfg;
@@ -235,12 +242,12 @@ void ko_destroy(ko_state *s) {
 
 int ko_cur_len(const ko_state *s) { return s ? s->cur_len : -1; }
 
-/* Pointer to the cached K (which = 0) or V (which = 1) rows of (layer, branch, head):
+/* Pointer to the cached K (which = 0) or V (which = 1) rows of (layer, branch, key/value head):
  * [max_pos, hd] contiguous. */
 const float *ko_cache_ptr(const ko_state *s, int layer, int branch, int which, int head) {
     const ko_config *c = &s->cfg;
     int hd = c->d_model / c->n_head;
-    size_t off = ((((size_t)layer * c->n_branch + branch) * c->n_head + head) * (size_t)c->max_pos) * hd;
+    size_t off = ((((size_t)layer * c->n_branch + branch) * kv_heads(c) + head) * (size_t)c->max_pos) * hd;
     return (which ? s->vcache : s->kcache) + off;
 }
 
@@ -263,6 +270,7 @@ static int forward(ko_state *s, const int32_t *ids, int n, int pos0, float *logi
     const ko_weights *w = &s->w;
     const int N = c->n_branch, L = c->n_layer, d = c->d_model, H = c->n_head, F = c->d_ff, V = c->vocab;
     const int hd = d / H, rb = c->bf16_store;
+    const int Hkv = kv_heads(c), kvd = Hkv * hd, qw = d + 2 * kvd; /* q | k | v row: d + 2 H_kv hd columns */
     if (!ids || n < 1 || pos0 < 0) return -1;
     if (pos0 + n > c->max_pos) return -2;
     for (int t = 0; t < n; ++t)
@@ -274,7 +282,7 @@ static int forward(ko_state *s, const int32_t *ids, int n, int pos0, float *logi
     float *xn = (float *)malloc(sizeof(float) * nd * N);    /* next layer's inputs    */
     float *y = (float *)malloc(sizeof(float) * nd);
     float *u = (float *)malloc(sizeof(float) * nd);
-    float *qkv = (float *)malloc(sizeof(float) * nd * 3);
+    float *qkv = (float *)malloc(sizeof(float) * (size_t)n * qw);
     float *o = (float *)malloc(sizeof(float) * nd);
     float *a = (float *)malloc(sizeof(float) * nd);
     float *hh = (float *)malloc(sizeof(float) * nd);
@@ -312,23 +320,25 @@ static int forward(ko_state *s, const int32_t *ids, int n, int pos0, float *logi
             ko_layernorm(xb, NULL, n, d, w->ln1_g + ln * d, w->ln1_b ? w->ln1_b + ln * d : NULL,
                          c->ln_eps, rb, u);
             /* q | k | v */
-            ko_linear(u, n, d, w->w_qkv + ln * 3 * (size_t)d * d, d,
-                      w->b_qkv ? w->b_qkv + ln * 3 * d : NULL, 3 * d, qkv);
-            maybe_round(qkv, nd * 3, rb);
-            /* memoise k, v */
-            for (int h = 0; h < H; ++h) {
+            ko_linear(u, n, d, w->w_qkv + ln * (size_t)qw * d, d,
+                      w->b_qkv ? w->b_qkv + ln * qw : NULL, qw, qkv);
+            maybe_round(qkv, (size_t)n * qw, rb);
+            /* memoise k, v (one row per key/value head) */
+            for (int h = 0; h < Hkv; ++h) {
                 float *kc = (float *)ko_cache_ptr(s, l, b, 0, h);
                 float *vc = (float *)ko_cache_ptr(s, l, b, 1, h);
                 for (int t = 0; t < n; ++t)
                     for (int e = 0; e < hd; ++e) {
-                        kc[(size_t)(pos0 + t) * hd + e] = qkv[(size_t)t * 3 * d + d + h * hd + e];
-                        vc[(size_t)(pos0 + t) * hd + e] = qkv[(size_t)t * 3 * d + 2 * d + h * hd + e];
+                        kc[(size_t)(pos0 + t) * hd + e] = qkv[(size_t)t * qw + d + h * hd + e];
+                        vc[(size_t)(pos0 + t) * hd + e] = qkv[(size_t)t * qw + d + kvd + h * hd + e];
                     }
             }
-            /* attention per head over the cached rows */
-            for (int h = 0; h < H; ++h)
-                ko_attention_head(qkv + h * hd, 3 * (int64_t)d, ko_cache_ptr(s, l, b, 0, h),
-                                  ko_cache_ptr(s, l, b, 1, h), hd, n, pos0, hd, o + h * hd, d);
+            /* attention per query head over the cached rows of its key/value head */
+            for (int h = 0; h < H; ++h) {
+                const int hk = h / (H / Hkv);
+                ko_attention_head(qkv + h * hd, (int64_t)qw, ko_cache_ptr(s, l, b, 0, hk),
+                                  ko_cache_ptr(s, l, b, 1, hk), hd, n, pos0, hd, o + h * hd, d);
+            }
             maybe_round(o, nd, rb);
             /* x = res + MHA */
             ko_linear(o, n, d, w->w_proj + ln * (size_t)d * d, d, w->b_proj ? w->b_proj + ln * d : NULL, d, tmp);

@@ -483,3 +483,52 @@ def test_engine_configs_follow_table3():
     assert set(ki.PAPER_TTFT_MS) == set(engines)
     assert all(set(v) == {128, 2048} for v in ki.PAPER_TTFT_MS.values())
 
+
+# ------------------------------------------------------------------ grouped-query / multi-query attention
+
+@pytest.mark.parametrize("n_head,n_kv", [(4, 2), (4, 1), (6, 3), (2, 2)])
+def test_grouped_query_attention_equals_multi_head_with_repeated_kv(n_head, n_kv):
+    """Grouped-query attention (the KV-cache mitigation named in Sec. 4.2) is multi-head attention whose
+    key / value projections are shared by the query heads of a group: copying each shared K and V
+    projection to every query head of its group gives a multi-head model with the same logits, and the
+    grouped cache holds one row set per key/value head."""
+    hd = 8
+    d = n_head * hd
+    g_shape = small_shape(d_model=d, n_head=n_head, d_ff=2 * d, n_kv_head=n_kv)
+    m_shape = small_shape(d_model=d, n_head=n_head, d_ff=2 * d)
+    wg = rand_weights(g_shape)
+    assert wg["w_qkv"].shape[2] == d + 2 * n_kv * hd
+    rep = n_head // n_kv
+    kvd = n_kv * hd
+    idx = torch.arange(n_head * hd)
+    src = (idx // hd // rep) * hd + idx % hd                      # column of the shared head for each MHA column
+    wm = dict(wg)
+    wq, wk, wv = wg["w_qkv"][:, :, :d], wg["w_qkv"][:, :, d:d + kvd], wg["w_qkv"][:, :, d + kvd:]
+    wm["w_qkv"] = torch.cat([wq, wk[:, :, src], wv[:, :, src]], dim=2).contiguous()
+    bq, bk, bv = wg["b_qkv"][:, :, :d], wg["b_qkv"][:, :, d:d + kvd], wg["b_qkv"][:, :, d + kvd:]
+    wm["b_qkv"] = torch.cat([bq, bk[:, :, src], bv[:, :, src]], dim=2).contiguous()
+    ids = ki.uniform_tokens(9, g_shape.vocab, 1, g_shape.seqlen)[0].numpy()
+    og, om = oracle.Oracle(g_shape, wbits(wg)), oracle.Oracle(m_shape, wbits(wm))
+    lg, _ = og.prefill(ids[:-2])
+    lm, _ = om.prefill(ids[:-2])
+    assert np.array_equal(lg, lm)
+    for t in ids[-2:]:                                            # and through decode steps
+        assert np.array_equal(og.decode_step(int(t)), om.decode_step(int(t)))
+    for layer in range(g_shape.n_layer):
+        for which in (0, 1):
+            cg, cm = og.cache(layer, 1, which), om.cache(layer, 1, which)
+            assert cg.shape == (n_kv, len(ids), hd) and cm.shape == (n_head, len(ids), hd)
+            for h in range(n_head):
+                assert np.array_equal(cm[h], cg[h // rep])
+
+
+def test_kv_heads_equal_to_heads_is_plain_multi_head():
+    a, b = small_shape(), small_shape(n_kv_head=2)
+    w = rand_weights(a)
+    ids = ki.uniform_tokens(9, a.vocab, 1, a.seqlen)[0].numpy()
+    la, _ = oracle.Oracle(a, wbits(w)).prefill(ids)
+    lb, _ = oracle.Oracle(b, wbits(w)).prefill(ids)
+    assert np.array_equal(la, lb)
+    with pytest.raises(ValueError):
+        oracle.Oracle(small_shape(n_kv_head=3), wbits(w))       # 2 heads cannot share 3 key/value heads
+
