@@ -147,7 +147,8 @@ def run_reference(args, shape):
 def workload_config(shape, args):
     what = "decode after prefill" if shape.decode_steps else "prefill"
     cfg = {"workload": f"{shape.name} {what}", "n_branch": shape.n_branch, "n_layer": shape.n_layer,
-           "d_model": shape.d_model, "n_head": shape.n_head, "d_ff": shape.d_ff, "vocab": shape.vocab,
+           "d_model": shape.d_model, "n_head": shape.n_head, "n_kv_head": shape.kv_heads, "d_ff": shape.d_ff,
+           "vocab": shape.vocab,
            "batch": shape.batch, "seqlen": shape.seqlen, "tokens_per_step": shape.batch * shape.seqlen,
            "parallelism": f"replicas x{args.gpus}" if args.gpus > 1 else "single GPU",
            "l2": "inputs larger than L2 (weights read every step exceed 126 MB)"
@@ -170,15 +171,16 @@ def paper_ttft_ms(shape):
 
 
 def weight_bytes(s):
-    return 2 * (s.n_layer * s.n_branch * (4 * s.d_model ** 2 + 2 * s.d_model * s.d_ff) + s.vocab * s.d_model)
+    return 2 * (s.n_layer * s.n_branch * (s.d_model * s.qkv_width + s.d_model ** 2 + 2 * s.d_model * s.d_ff)
+                + s.vocab * s.d_model)
 
 
 def decode_bytes(shape, t):
     """Bytes one decode step must move at cache length t: every weight once, K and V rows 0..t."""
     s = shape
-    w = 2 * (s.n_layer * s.n_branch * (4 * s.d_model ** 2 + 2 * s.d_model * s.d_ff) + s.vocab * s.d_model
-             + s.n_branch * s.d_model ** 2)
-    kv = 2 * s.n_layer * s.n_branch * s.batch * (t + 1) * s.d_model * 2
+    w = 2 * (s.n_layer * s.n_branch * (s.d_model * s.qkv_width + s.d_model ** 2 + 2 * s.d_model * s.d_ff)
+             + s.vocab * s.d_model + s.n_branch * s.d_model ** 2)
+    kv = 2 * s.n_layer * s.n_branch * s.batch * (t + 1) * s.kv_heads * s.head_dim * 2
     return w, kv
 
 

@@ -54,18 +54,22 @@ typedef struct kraken_config {
     float ln_eps;      /* LayerNorm epsilon (1e-5)                                            */
     int32_t gelu_tanh; /* 0: GELU by erf (default), 1: tanh approximation                     */
     int32_t final_ln;  /* 1: LayerNorm between W_concat and the unembedding (default), 0: none */
-    int32_t reserved[5];
+    int32_t n_kv_head; /* key/value heads per sub-layer: 0 or n_head = multi-head attention; a divisor of
+                          n_head = grouped-query attention, 1 = multi-query attention (the KV-cache
+                          mitigation of Sec. 4.2): query head h reads key/value head h / (n_head / n_kv_head) */
+    int32_t reserved[4];
 } kraken_config;
 
 /* Device pointers to bf16 weights, row-major [out_features, in_features]; BORROWED until
  * kraken_destroy.  Any bias or LayerNorm-beta pointer may be NULL (= zeros).
- * w_qkv rows 0..d-1 produce Q, d..2d-1 K, 2d..3d-1 V; head h owns rows h*hd..(h+1)*hd-1 of each.
+ * w_qkv rows 0..d-1 produce Q, the next kvd = n_kv_head*hd rows K, the last kvd rows V (kvd = d for
+ * multi-head attention); head h owns rows h*hd..(h+1)*hd-1 of each part.
  * w_concat input index n*d + j is feature j of branch n (branch-major concatenation). */
 typedef struct kraken_weights {
     const void *wte;                /* [V, d] token embedding, also the unembedding (tied) */
     const void *wpe;                /* [max_pos, d] learned positions                     */
     const void *ln1_g, *ln1_b;      /* [L][N][d]                                          */
-    const void *w_qkv, *b_qkv;      /* [L][N][3d][d], [L][N][3d]                          */
+    const void *w_qkv, *b_qkv;      /* [L][N][d+2kvd][d], [L][N][d+2kvd]                  */
     const void *w_proj, *b_proj;    /* [L][N][d][d],  [L][N][d]                           */
     const void *ln2_g, *ln2_b;      /* [L][N][d]                                          */
     const void *w_up, *b_up;        /* [L][N][F][d],  [L][N][F]                           */
@@ -77,7 +81,7 @@ typedef struct kraken_weights {
 typedef struct kraken_handle kraken_handle;
 
 /* Bytes of KV cache and scratch a handle of this configuration needs.  Pure host
- * arithmetic, usable without a GPU.  KV layout: [L][N][2 (K,V)][max_batch][n_head][max_pos][head_dim] bf16.
+ * arithmetic, usable without a GPU.  KV layout: [L][N][2 (K,V)][max_batch][n_kv_head][max_pos][head_dim] bf16.
  * Errors: EINVAL (null, non-positive field, d % n_head != 0), EUNSUPPORTED (see kraken_create). */
 int kraken_query_sizes(const kraken_config *cfg, size_t *kv_bytes, size_t *scratch_bytes);
 
@@ -211,7 +215,9 @@ typedef struct kraken_gemm_args {
     int32_t n_tile;                                           /* N tile: 0 = automatic, 64 / 128 / 256, 512 = CTA
                                                                  pairs on 256 x 256 tiles, or 8 = the
                                                                  weight-streaming kernel for m <= 32 (no RESID_SUM) */
-    int32_t reserved[2];
+    int32_t n_kv_head;                                        /* QKV only: key/value heads (0 = n_head); the K and V
+                                                                 parts of n_out are n_kv_head * head_dim wide each */
+    int32_t reserved[1];
 } kraken_gemm_args;
 
 /* Grouped bf16 GEMM on the tensor cores (tcgen05 + TMEM accumulators, TMA operand loads).
@@ -222,24 +228,28 @@ int kraken_op_grouped_gemm(const kraken_gemm_args *args, uint32_t *d_status, voi
 /* Causal multi-head attention over a prefix held in the cache layout (Sec. 2.1):
  * for sequence b, head h, query row t (position pos0 + t): softmax over keys 0..pos0+t of
  * q.k / sqrt(head_dim), times V.  q, out: bf16 [G][batch*seqlen, n_head*head_dim];
- * k_cache, v_cache: bf16 [G][.][batch_stride][n_head][max_pos][head_dim] as described by
- * cache_gstride / cache_bstride (elements). */
+ * k_cache, v_cache: bf16 [G][.][batch_stride][n_kv_head][max_pos][head_dim] as described by
+ * cache_gstride / cache_bstride (elements).  n_kv_head: key/value heads in the cache, 0 = n_head;
+ * with fewer (grouped-query / multi-query attention) query head h reads key/value head
+ * h / (n_head / n_kv_head). */
 int kraken_op_attention(const void *q, int64_t q_gstride, const void *k_cache, const void *v_cache,
                         int64_t cache_gstride, int64_t cache_bstride, int32_t groups, int32_t batch,
-                        int32_t seqlen, int32_t pos0, int32_t n_head, int32_t head_dim, int32_t max_pos,
-                        void *out, int64_t out_gstride, void *stream);
+                        int32_t seqlen, int32_t pos0, int32_t n_head, int32_t n_kv_head, int32_t head_dim,
+                        int32_t max_pos, void *out, int64_t out_gstride, void *stream);
 
 /* Decode-step attention (Sec. 2.1: the decode step reads the whole KV cache): one query row per
  * (group, sequence, head) at position n_keys - 1 against cache rows 0..n_keys-1.  The keys are split
  * over `splits` CTAs per (group, sequence, head); each split leaves an unnormalised partial in
  * d_partials (device scratch, fp32 [groups*batch*n_head][splits][head_dim + 2]) and a second kernel
  * merges them.  splits = 0 lets the library choose; splits = 1 needs no scratch (d_partials may be NULL).
- * q, out: bf16 [G][batch, n_head*head_dim].  Errors: EINVAL, EUNSUPPORTED (head_dim), ECAPACITY
- * (partial_bytes too small). */
+ * q, out: bf16 [G][batch, n_head*head_dim].  n_kv_head as in kraken_op_attention: the query heads of a
+ * group are served together, so each cache row is fetched once per group.  Errors: EINVAL,
+ * EUNSUPPORTED (head_dim), ECAPACITY (partial_bytes too small). */
 int kraken_op_decode_attention(const void *q, int64_t q_gstride, const void *k_cache, const void *v_cache,
                                int64_t cache_gstride, int64_t cache_bstride, int32_t groups, int32_t batch,
-                               int32_t n_keys, int32_t n_head, int32_t head_dim, int32_t max_pos, int32_t splits,
-                               void *d_partials, size_t partial_bytes, void *out, int64_t out_gstride, void *stream);
+                               int32_t n_keys, int32_t n_head, int32_t n_kv_head, int32_t head_dim, int32_t max_pos,
+                               int32_t splits, void *d_partials, size_t partial_bytes, void *out,
+                               int64_t out_gstride, void *stream);
 
 /* Split count the library would choose (when *splits == 0 on entry; otherwise *splits is validated and kept)
  * and the scratch bytes kraken_op_decode_attention needs for it.  Pure host arithmetic. */

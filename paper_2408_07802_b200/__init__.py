@@ -41,7 +41,8 @@ EXPORTS = (
 class KrakenConfig(C.Structure):
     _fields_ = [(n, C.c_int32) for n in
                 ("n_branch", "n_layer", "d_model", "n_head", "d_ff", "vocab", "max_pos", "max_batch")] + [
-        ("ln_eps", C.c_float), ("gelu_tanh", C.c_int32), ("final_ln", C.c_int32), ("reserved", C.c_int32 * 5)]
+        ("ln_eps", C.c_float), ("gelu_tanh", C.c_int32), ("final_ln", C.c_int32), ("n_kv_head", C.c_int32),
+        ("reserved", C.c_int32 * 4)]
 
 
 class KrakenWeights(C.Structure):
@@ -61,7 +62,8 @@ class GemmArgs(C.Structure):
         ("sum", C.c_void_p), ("ld_sum", C.c_int32),
         ("k_cache", C.c_void_p), ("v_cache", C.c_void_p), ("cache_gstride", C.c_int64),
         ("seqlen", C.c_int32), ("pos0", C.c_int32), ("n_head", C.c_int32), ("head_dim", C.c_int32),
-        ("max_pos", C.c_int32), ("gelu_tanh", C.c_int32), ("n_tile", C.c_int32), ("reserved", C.c_int32 * 2),
+        ("max_pos", C.c_int32), ("gelu_tanh", C.c_int32), ("n_tile", C.c_int32), ("n_kv_head", C.c_int32),
+        ("reserved", C.c_int32 * 1),
     ]
 
 
@@ -109,8 +111,8 @@ def lib() -> C.CDLL:
         L.kraken_op_embed.argtypes = [vp, i32, i32, i32, vp, vp, i32, i32, vp, vp, vp]
         L.kraken_op_layernorm.argtypes = [vp, i64, vp, vp, vp, i32, i32, i32, C.c_float, vp, vp, vp]
         L.kraken_op_grouped_gemm.argtypes = [C.POINTER(GemmArgs), vp, vp]
-        L.kraken_op_attention.argtypes = [vp, i64, vp, vp, i64, i64, i32, i32, i32, i32, i32, i32, i32, vp, i64, vp]
-        L.kraken_op_decode_attention.argtypes = [vp, i64, vp, vp, i64, i64, i32, i32, i32, i32, i32, i32, i32, vp,
+        L.kraken_op_attention.argtypes = [vp, i64, vp, vp, i64, i64, i32, i32, i32, i32, i32, i32, i32, i32, vp, i64, vp]
+        L.kraken_op_decode_attention.argtypes = [vp, i64, vp, vp, i64, i64, i32, i32, i32, i32, i32, i32, i32, i32, vp,
                                                  C.c_size_t, vp, i64, vp]
         L.kraken_decode_attention_sizes.argtypes = [i32, i32, i32, i32, i32, C.POINTER(i32), C.POINTER(C.c_size_t)]
         L.kraken_op_decode_attention_static.argtypes = [vp, i64, vp, vp, i64, i64, i32, i32, i32, i32, i32, i32, i32,
@@ -144,7 +146,7 @@ def make_config(shape, max_batch: Optional[int] = None, max_pos: Optional[int] =
         n_branch=shape.n_branch, n_layer=shape.n_layer, d_model=shape.d_model, n_head=shape.n_head,
         d_ff=shape.d_ff, vocab=shape.vocab, max_pos=max_pos or shape.max_pos,
         max_batch=max_batch or shape.batch, ln_eps=shape.ln_eps, gelu_tanh=shape.gelu_tanh,
-        final_ln=shape.final_ln)
+        final_ln=shape.final_ln, n_kv_head=int(getattr(shape, "n_kv_head", 0) or 0))
     for k, v in over.items():
         setattr(cfg, k, v)
     return cfg
@@ -237,7 +239,7 @@ class KrakenModel:
 
     # -------- inspection
     def kv_view(self, layer: int, branch: int, which: int) -> torch.Tensor:
-        """bf16 view [max_batch, n_head, max_pos, head_dim] of the K (0) or V (1) cache of (layer, branch)."""
+        """bf16 view [max_batch, key/value heads, max_pos, head_dim] of the K (0) or V (1) cache of (layer, branch)."""
         p = C.c_void_p()
         st = (C.c_int64 * 4)()
         _check(lib().kraken_kv_view(self._h, layer, branch, which, C.byref(p), C.byref(st)), "kraken_kv_view")
@@ -245,7 +247,7 @@ class KrakenModel:
         hd = c.d_model // c.n_head
         off = (p.value - self.kv.data_ptr()) // 2
         flat = self.kv.view(torch.bfloat16)
-        return flat.as_strided((c.max_batch, c.n_head, c.max_pos, hd), tuple(st), off)
+        return flat.as_strided((c.max_batch, c.n_kv_head or c.n_head, c.max_pos, hd), tuple(st), off)
 
     def device_status(self) -> int:
         f = C.c_uint32(0)
@@ -303,13 +305,14 @@ def op_grouped_gemm(args: GemmArgs, status: Optional[torch.Tensor] = None):
 
 def op_attention(q: torch.Tensor, k_cache: torch.Tensor, v_cache: torch.Tensor, batch: int, seqlen: int, pos0: int,
                  n_head: int) -> torch.Tensor:
-    """q bf16 [G, batch*seqlen, d]; k_cache / v_cache bf16 [G, batch, n_head, max_pos, head_dim]."""
+    """q bf16 [G, batch*seqlen, d]; k_cache / v_cache bf16 [G, batch, key/value heads, max_pos, head_dim]
+    (fewer key/value heads than n_head = grouped-query attention)."""
     G, _, d = q.shape
-    _, _, H, P, hd = k_cache.shape
-    assert H == n_head and H * hd == d
+    _, _, Hkv, P, hd = k_cache.shape
+    assert n_head % Hkv == 0 and n_head * hd == d
     out = torch.empty_like(q)
     _check(lib().kraken_op_attention(q.data_ptr(), q.stride(0), k_cache.data_ptr(), v_cache.data_ptr(),
-                                     k_cache.stride(0), k_cache.stride(1), G, batch, seqlen, pos0, H, hd, P,
+                                     k_cache.stride(0), k_cache.stride(1), G, batch, seqlen, pos0, n_head, Hkv, hd, P,
                                      out.data_ptr(), out.stride(0), _stream()), "kraken_op_attention")
     return out
 
@@ -324,15 +327,17 @@ def decode_attention_sizes(groups: int, batch: int, n_keys: int, n_head: int, he
 
 def op_decode_attention(q: torch.Tensor, k_cache: torch.Tensor, v_cache: torch.Tensor, n_keys: int,
                         splits: int = 0, partials: Optional[torch.Tensor] = None) -> torch.Tensor:
-    """q bf16 [G, batch, d]; caches bf16 [G, batch, n_head, max_pos, head_dim]; attends to rows 0..n_keys-1."""
+    """q bf16 [G, batch, d]; caches bf16 [G, batch, key/value heads, max_pos, head_dim]; attends to rows
+    0..n_keys-1.  The number of query heads is d / head_dim."""
     G, B, d = q.shape
-    _, _, H, P, hd = k_cache.shape
+    _, _, Hkv, P, hd = k_cache.shape
+    H = d // hd
     splits, nbytes = decode_attention_sizes(G, B, n_keys, H, hd, splits)
     if partials is None and nbytes:
         partials = torch.empty(nbytes, dtype=torch.uint8, device=q.device)
     out = torch.empty_like(q)
     _check(lib().kraken_op_decode_attention(q.data_ptr(), q.stride(0), k_cache.data_ptr(), v_cache.data_ptr(),
-                                            k_cache.stride(0), k_cache.stride(1), G, B, n_keys, H, hd, P, splits,
+                                            k_cache.stride(0), k_cache.stride(1), G, B, n_keys, H, Hkv, hd, P, splits,
                                             _ptr(partials), 0 if partials is None else partials.numel(),
                                             out.data_ptr(), out.stride(0), _stream()), "kraken_op_decode_attention")
     return out

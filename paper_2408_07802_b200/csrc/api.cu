@@ -24,6 +24,8 @@ struct Layout {
     size_t status, tokens, rows, logits, x0, x, a, s, u, q, o, g, dec_part, total;
 };
 
+int kv_heads_of(const kraken_config &c) { return c.n_kv_head > 0 ? c.n_kv_head : c.n_head; }
+
 bool decode_head_dim_ok(int hd) { return hd == 64 || hd == 72 || hd == 96 || hd == 104 || hd == 128; }
 
 int check_config(const kraken_config *c) {
@@ -32,6 +34,7 @@ int check_config(const kraken_config *c) {
         c->max_pos < 1 || c->max_batch < 1 || !(c->ln_eps > 0.f))
         return KRAKEN_EINVAL;
     if (c->d_model % c->n_head != 0) return KRAKEN_EINVAL;
+    if (c->n_kv_head < 0 || (c->n_kv_head > 0 && c->n_head % c->n_kv_head != 0)) return KRAKEN_EINVAL;
     const int hd = c->d_model / c->n_head;
     // 64 and 128, and the head dims of the paper's engine shapes (Table 3: 72, 96, 104)
     if (hd != 64 && hd != 72 && hd != 96 && hd != 104 && hd != 128) return KRAKEN_EUNSUPPORTED;
@@ -41,7 +44,8 @@ int check_config(const kraken_config *c) {
 }
 
 size_t kv_bytes_of(const kraken_config *c) {
-    return (size_t)c->n_layer * c->n_branch * 2 * c->max_batch * c->max_pos * (size_t)c->d_model * 2;
+    return (size_t)c->n_layer * c->n_branch * 2 * c->max_batch * c->max_pos *
+           (size_t)(kv_heads_of(*c) * (c->d_model / c->n_head)) * 2;
 }
 
 Layout layout_of(const kraken_config *c) {
@@ -170,7 +174,7 @@ int model_gemm(const RunCtx &rc, GemmKind kind, int layer, int m_rows, const uin
     const uint16_t *wbase;
     const uint16_t *bias = nullptr;
     switch (kind) {
-        case G_QKV: s = {N, m_rows, 3 * d, d}; wbase = (const uint16_t *)h->w.w_qkv; bias = (const uint16_t *)h->w.b_qkv; break;
+        case G_QKV: s = {N, m_rows, d + 2 * kv_heads_of(c) * (d / c.n_head), d}; wbase = (const uint16_t *)h->w.w_qkv; bias = (const uint16_t *)h->w.b_qkv; break;
         case G_PROJ: s = {N, m_rows, d, d}; wbase = (const uint16_t *)h->w.w_proj; bias = (const uint16_t *)h->w.b_proj; break;
         case G_UP: s = {N, m_rows, F, d}; wbase = (const uint16_t *)h->w.w_up; bias = (const uint16_t *)h->w.b_up; break;
         case G_DOWN: s = {N, m_rows, d, F}; wbase = (const uint16_t *)h->w.w_down; bias = (const uint16_t *)h->w.b_down; break;
@@ -249,7 +253,8 @@ int run_layers(const RunCtx &rc, const int32_t *d_tokens) {
     uint16_t *u = at<uint16_t>(h, h->lay.u), *q = at<uint16_t>(h, h->lay.q), *o = at<uint16_t>(h, h->lay.o),
              *gb = at<uint16_t>(h, h->lay.g);
     uint32_t *status = at<uint32_t>(h, h->lay.status);
-    const long long cache_b = (long long)H * c.max_pos * hd;      // one sequence of one of K / V
+    const int Hkv = kv_heads_of(c);
+    const long long cache_b = (long long)Hkv * c.max_pos * hd;    // one sequence of one of K / V
     const long long cache_kv = (long long)c.max_batch * cache_b;  // all of K (or V) of one (layer, branch)
     uint16_t *kv = reinterpret_cast<uint16_t *>(h->kv);
 
@@ -276,6 +281,7 @@ int run_layers(const RunCtx &rc, const int32_t *d_tokens) {
         e.out_bf16 = q; e.out_bf16_gstride = td; e.ld_out_bf16 = d;
         e.k_cache = kc; e.v_cache = kc + cache_kv; e.cache_gstride = 2 * cache_kv;
         e.seqlen = rc.seqlen; e.pos0 = rc.pos0; e.n_head = H; e.head_dim = hd; e.max_pos = c.max_pos; e.d_model = d;
+        e.n_kv_head = Hkv;
         e.pos0_dev = rc.pos_dev;
         KR_TRY(model_gemm(rc, G_QKV, l, T, u, td, e));
         // attention over the cached prefix
@@ -283,6 +289,7 @@ int run_layers(const RunCtx &rc, const int32_t *d_tokens) {
         ap.q = q; ap.q_gstride = td;
         ap.k_cache = kc; ap.v_cache = kc + cache_kv; ap.cache_gstride = 2 * cache_kv; ap.cache_bstride = cache_b;
         ap.groups = N; ap.batch = rc.batch; ap.seqlen = rc.seqlen; ap.pos0 = rc.pos0; ap.n_head = H; ap.head_dim = hd;
+        ap.n_kv_head = Hkv;
         ap.max_pos = c.max_pos; ap.out = o; ap.out_gstride = td;
         {
             LaunchScope scope(h, KRAKEN_PROF_ATTENTION, rc.st);
@@ -295,6 +302,7 @@ int run_layers(const RunCtx &rc, const int32_t *d_tokens) {
                 dp.k_cache = ap.k_cache; dp.v_cache = ap.v_cache;
                 dp.cache_gstride = ap.cache_gstride; dp.cache_bstride = ap.cache_bstride;
                 dp.groups = N; dp.batch = rc.batch; dp.n_keys = rc.pos0 + 1; dp.n_head = H; dp.head_dim = hd;
+                dp.n_kv_head = Hkv;
                 dp.max_pos = c.max_pos;
                 dp.pos_dev = rc.pos_dev;
                 dp.splits = decode_attention_splits(N, rc.batch, H, rc.pos_dev ? rc.max_keys : dp.n_keys);
@@ -685,7 +693,7 @@ int kraken_kv_view(kraken_handle *h, int32_t layer, int32_t branch, int32_t whic
     if (layer < 0 || layer >= c.n_layer || branch < 0 || branch >= c.n_branch || which < 0 || which > 1)
         return KRAKEN_EINVAL;
     const int hd = c.d_model / c.n_head;
-    const long long cache_b = (long long)c.n_head * c.max_pos * hd, cache_kv = (long long)c.max_batch * cache_b;
+    const long long cache_b = (long long)kv_heads_of(c) * c.max_pos * hd, cache_kv = (long long)c.max_batch * cache_b;
     *ptr = reinterpret_cast<uint16_t *>(h->kv) + (((long long)layer * c.n_branch + branch) * 2 + which) * cache_kv;
     strides[0] = cache_b;
     strides[1] = (long long)c.max_pos * hd;
@@ -793,7 +801,9 @@ int kraken_op_grouped_gemm(const kraken_gemm_args *g, uint32_t *d_status, void *
     if (k == KRAKEN_EPI_QKV) {
         if (!g->k_cache || !g->v_cache || g->seqlen < 1 || g->n_head < 1 || g->pos0 < 0) return KRAKEN_EINVAL;
         // q | k | v and head boundaries fall on 16-byte pieces; the q rows and cache rows must be 16-byte aligned
-        if (g->head_dim % 8 != 0 || g->n_out != 3 * g->n_head * g->head_dim || g->ld_out_bf16 % 8 != 0 ||
+        if (g->n_kv_head < 0 || (g->n_kv_head > 0 && g->n_head % g->n_kv_head != 0)) return KRAKEN_EINVAL;
+        const int n_kv = g->n_kv_head > 0 ? g->n_kv_head : g->n_head;
+        if (g->head_dim % 8 != 0 || g->n_out != (g->n_head + 2 * n_kv) * g->head_dim || g->ld_out_bf16 % 8 != 0 ||
             g->out_bf16_gstride % 8 != 0 || g->cache_gstride % 8 != 0)
             return KRAKEN_EUNSUPPORTED;
     }
@@ -809,6 +819,7 @@ int kraken_op_grouped_gemm(const kraken_gemm_args *g, uint32_t *d_status, void *
     e.k_cache = (uint16_t *)g->k_cache; e.v_cache = (uint16_t *)g->v_cache; e.cache_gstride = g->cache_gstride;
     e.seqlen = g->seqlen; e.pos0 = g->pos0; e.n_head = g->n_head; e.head_dim = g->head_dim; e.max_pos = g->max_pos;
     e.d_model = g->n_head * g->head_dim;
+    e.n_kv_head = g->n_kv_head > 0 ? g->n_kv_head : g->n_head;
     e.gelu_tanh = g->gelu_tanh;
     if (env_flag("KRAKEN_NAIVE")) return launch_gemm_naive(op, s, e, static_cast<cudaStream_t>(stream));
     if (g->n_tile == 8) return launch_gemm_skinny(op, s, e, static_cast<cudaStream_t>(stream));
@@ -817,9 +828,11 @@ int kraken_op_grouped_gemm(const kraken_gemm_args *g, uint32_t *d_status, void *
 
 int kraken_op_attention(const void *q, int64_t q_gstride, const void *k_cache, const void *v_cache,
                         int64_t cache_gstride, int64_t cache_bstride, int32_t groups, int32_t batch, int32_t seqlen,
-                        int32_t pos0, int32_t n_head, int32_t head_dim, int32_t max_pos, void *out,
-                        int64_t out_gstride, void *stream) {
+                        int32_t pos0, int32_t n_head, int32_t n_kv_head, int32_t head_dim, int32_t max_pos,
+                        void *out, int64_t out_gstride, void *stream) {
+    if (n_head < 1 || n_kv_head < 0 || (n_kv_head > 0 && n_head % n_kv_head != 0)) return KRAKEN_EINVAL;
     AttnParams p;
+    p.n_kv_head = n_kv_head;
     p.q = (const uint16_t *)q; p.q_gstride = q_gstride;
     p.k_cache = (const uint16_t *)k_cache; p.v_cache = (const uint16_t *)v_cache;
     p.cache_gstride = cache_gstride; p.cache_bstride = cache_bstride;
@@ -833,9 +846,11 @@ int kraken_op_attention(const void *q, int64_t q_gstride, const void *k_cache, c
 
 int kraken_op_decode_attention(const void *q, int64_t q_gstride, const void *k_cache, const void *v_cache,
                                int64_t cache_gstride, int64_t cache_bstride, int32_t groups, int32_t batch,
-                               int32_t n_keys, int32_t n_head, int32_t head_dim, int32_t max_pos, int32_t splits,
-                               void *d_partials, size_t partial_bytes, void *out, int64_t out_gstride, void *stream) {
+                               int32_t n_keys, int32_t n_head, int32_t n_kv_head, int32_t head_dim, int32_t max_pos,
+                               int32_t splits, void *d_partials, size_t partial_bytes, void *out,
+                               int64_t out_gstride, void *stream) {
     if (groups < 1 || batch < 1 || n_head < 1 || n_keys < 1) return KRAKEN_EINVAL;
+    if (n_kv_head < 0 || (n_kv_head > 0 && n_head % n_kv_head != 0)) return KRAKEN_EINVAL;
     if (!decode_head_dim_ok(head_dim)) return KRAKEN_EUNSUPPORTED;
     if (splits == 0) splits = decode_attention_splits(groups, batch, n_head, n_keys);
     if (splits < 1 || splits > DECODE_MAX_SPLITS) return KRAKEN_EINVAL;
@@ -848,6 +863,7 @@ int kraken_op_decode_attention(const void *q, int64_t q_gstride, const void *k_c
     p.groups = groups; p.batch = batch; p.n_keys = n_keys; p.n_head = n_head; p.head_dim = head_dim;
     p.max_pos = max_pos; p.pos_dev = nullptr; p.splits = splits; p.partials = (float *)d_partials;
     p.out = (uint16_t *)out; p.out_gstride = out_gstride;
+    p.n_kv_head = n_kv_head;
     return launch_attention_decode(p, static_cast<cudaStream_t>(stream));
 }
 

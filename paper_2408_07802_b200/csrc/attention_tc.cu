@@ -40,6 +40,7 @@ constexpr bool POLY_EXP2 = false;
 
 struct AttnTcArgs {
     int groups, batch, seqlen, pos0, n_head;
+    int n_kv_head, kv_rep;   // key/value heads in the cache; query heads per key/value head
     int head_dim;      // <= HD of the kernel instance, a multiple of 8 (columns past it are zero-filled by TMA)
     uint16_t *out;
     long long out_gstride;
@@ -243,13 +244,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
 #pragma unroll
                     for (int hf = 0; hf < Cfg::HALVES; ++hf)
                         tma_load_4d(sK + st * Cfg::KV_BYTES + hf * Cfg::TILE_BYTES, &tmK, k_full + st, hf * 64,
-                                    j * TK, it.b * a.n_head + it.h, it.g);
+                                    j * TK, it.b * a.n_kv_head + it.h / a.kv_rep, it.g);
                     if (!(ok = mbar_wait(v_empty + st, ph ^ 1u, abort_flag))) break;
                     mbar_expect_tx(v_full + st, Cfg::KV_BYTES);
 #pragma unroll
                     for (int hf = 0; hf < Cfg::HALVES; ++hf)
                         tma_load_4d(sV + st * Cfg::KV_BYTES + hf * Cfg::TILE_BYTES, &tmV, v_full + st, hf * 64,
-                                    j * TK, it.b * a.n_head + it.h, it.g);
+                                    j * TK, it.b * a.n_kv_head + it.h / a.kv_rep, it.g);
                 }
             }
         }
@@ -503,7 +504,9 @@ bool attention_tc_supported(const AttnParams &p) {
     // instance runs it with the missing columns zero-filled by the tensor maps
     if (p.head_dim < 16 || p.head_dim > 128 || (p.head_dim & 7)) return false;
     // the cache of one group must be [batch][head][max_pos][head_dim] without gaps
-    if (p.cache_bstride != (long long)p.n_head * p.max_pos * p.head_dim) return false;
+    const int n_kv = p.n_kv_head > 0 ? p.n_kv_head : p.n_head;
+    if (p.n_head % n_kv != 0) return false;
+    if (p.cache_bstride != (long long)n_kv * p.max_pos * p.head_dim) return false;
     const int d = p.n_head * p.head_dim;
     if ((reinterpret_cast<uintptr_t>(p.q) & 15) || (reinterpret_cast<uintptr_t>(p.k_cache) & 15) ||
         (reinterpret_cast<uintptr_t>(p.v_cache) & 15) || (reinterpret_cast<uintptr_t>(p.out) & 15) ||
@@ -520,7 +523,8 @@ int attention_tc_encode(const AttnParams &p, CUtensorMap *tmQ, CUtensorMap *tmK,
     if (rc) return rc;
     // rows past the keys written so far are out of bounds of the map and read as zeros
     const uint64_t kv_len = (uint64_t)p.pos0 + p.seqlen;
-    const uint64_t dims[4] = {(uint64_t)p.head_dim, kv_len, (uint64_t)p.batch * p.n_head, (uint64_t)p.groups};
+    const int n_kv = p.n_kv_head > 0 ? p.n_kv_head : p.n_head;
+    const uint64_t dims[4] = {(uint64_t)p.head_dim, kv_len, (uint64_t)p.batch * n_kv, (uint64_t)p.groups};
     const uint64_t strides[3] = {(uint64_t)p.head_dim, (uint64_t)p.max_pos * p.head_dim,
                                  one ? (uint64_t)p.cache_bstride * p.batch : (uint64_t)p.cache_gstride};
     const uint32_t box[4] = {64, TK, 1, 1};
@@ -549,6 +553,8 @@ int launch_attention_tc(const AttnParams &p, const CUtensorMap *tmQ, const CUten
     a.seqlen = p.seqlen;
     a.pos0 = p.pos0;
     a.n_head = p.n_head;
+    a.n_kv_head = p.n_kv_head > 0 ? p.n_kv_head : p.n_head;
+    a.kv_rep = p.n_head / a.n_kv_head;
     a.head_dim = p.head_dim;
     a.out = p.out;
     a.out_gstride = p.out_gstride;

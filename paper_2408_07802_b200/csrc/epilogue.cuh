@@ -193,20 +193,21 @@ __device__ __forceinline__ void epilogue_chunk(const EpiParams &p, int g, int ro
             break;
         }
         case KRAKEN_EPI_QKV: {
-            // columns [0, d) are q, [d, 2d) the key row, [2d, 3d) the value row of this token; keys and
-            // values go to their (sequence, head, position) row of the cache
+            // columns [0, d) are q, the next n_kv_head * head_dim the key row, the last n_kv_head * head_dim the
+            // value row of this token; keys and values go to their (sequence, head, position) row of the cache
             const int d = p.d_model;
+            const int kvd = p.n_kv_head * p.head_dim;      // width of the k part and of the v part
             const int b = row / p.seqlen, pos = (p.pos0_dev ? *p.pos0_dev : p.pos0) + row % p.seqlen;
             if (((d | p.head_dim) & 31) == 0) {            // the 32 columns lie inside q or inside one head
                 if (col0 < d) {
                     store_bf16_chunk(p.out_bf16 + g * p.out_bf16_gstride + (long long)row * p.ld_out_bf16 + col0, v,
                                      ncols);
                 } else {
-                    const int which = col0 >= 2 * d;
-                    const int c = col0 - (1 + which) * d;
+                    const int which = col0 >= d + kvd;
+                    const int c = col0 - d - which * kvd;
                     const int head = c / p.head_dim, e0 = c % p.head_dim;
                     uint16_t *base = (which ? p.v_cache : p.k_cache) + g * p.cache_gstride;
-                    store_bf16_chunk(base + (((long long)b * p.n_head + head) * p.max_pos + pos) * p.head_dim + e0, v,
+                    store_bf16_chunk(base + (((long long)b * p.n_kv_head + head) * p.max_pos + pos) * p.head_dim + e0, v,
                                      ncols);
                 }
             } else {
@@ -220,11 +221,11 @@ __device__ __forceinline__ void epilogue_chunk(const EpiParams &p, int g, int ro
                     if (col < d) {
                         dst = p.out_bf16 + g * p.out_bf16_gstride + (long long)row * p.ld_out_bf16 + col;
                     } else {
-                        const int which = col >= 2 * d;
-                        const int c = col - (1 + which) * d;
+                        const int which = col >= d + kvd;
+                        const int c = col - d - which * kvd;
                         const int head = c / p.head_dim, e0 = c % p.head_dim;
                         dst = (which ? p.v_cache : p.k_cache) + g * p.cache_gstride +
-                              (((long long)b * p.n_head + head) * p.max_pos + pos) * p.head_dim + e0;
+                              (((long long)b * p.n_kv_head + head) * p.max_pos + pos) * p.head_dim + e0;
                     }
                     uint4 u;
                     u.x = pack_bf16x2(v[8 * i + 0], v[8 * i + 1]);

@@ -54,11 +54,12 @@ __device__ __forceinline__ void epilogue_elem(const EpiParams &p, int g, int row
             if (col < d) {
                 p.out_bf16[g * p.out_bf16_gstride + (long long)row * p.ld_out_bf16 + col] = to_bf(acc);
             } else {
-                const int which = col >= 2 * d, c = col - (1 + which) * d;
+                const int kvd = p.n_kv_head * p.head_dim;
+                const int which = col >= d + kvd, c = col - d - which * kvd;
                 const int head = c / p.head_dim, e = c % p.head_dim;
                 const int b = row / p.seqlen, pos = (p.pos0_dev ? *p.pos0_dev : p.pos0) + row % p.seqlen;
                 uint16_t *base = (which ? p.v_cache : p.k_cache) + g * p.cache_gstride;
-                base[(((long long)b * p.n_head + head) * p.max_pos + pos) * p.head_dim + e] = to_bf(acc);
+                base[(((long long)b * p.n_kv_head + head) * p.max_pos + pos) * p.head_dim + e] = to_bf(acc);
             }
             break;
         }

@@ -27,6 +27,7 @@ struct EpiParams {
     uint16_t *k_cache, *v_cache;
     long long cache_gstride;
     int seqlen, pos0, n_head, head_dim, max_pos, d_model;
+    int n_kv_head;  // key/value heads (grouped-query attention); the k and v parts are n_kv_head * head_dim wide
     int gelu_tanh;
     const int *pos0_dev;  // when set, the first position is read from device memory (replayable decode graph)
 };
@@ -94,6 +95,7 @@ struct AttnParams {
     int groups, batch, seqlen, pos0, n_head, head_dim, max_pos;
     uint16_t *out;
     long long out_gstride;
+    int n_kv_head = 0;  // key/value heads in the cache (0 = n_head); query head h reads head h / (n_head / n_kv_head)
 };
 int launch_attention_prefill(const AttnParams &p, cudaStream_t stream);
 int launch_attention_naive(const AttnParams &p, cudaStream_t stream);
@@ -111,6 +113,7 @@ struct DecodeAttnParams {
     const uint16_t *k_cache, *v_cache;
     long long cache_gstride, cache_bstride;
     int groups, batch, n_keys, n_head, head_dim, max_pos;
+    int n_kv_head = 0;   // key/value heads in the cache (0 = n_head)
     const int *pos_dev;  // when set, n_keys = *pos_dev + 1 (replayable decode graph)
     int splits;
     float *partials;  // [G*batch*n_head][splits][head_dim + 2] fp32 (max, sum, output); unused when splits == 1

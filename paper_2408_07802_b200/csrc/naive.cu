@@ -48,11 +48,12 @@ __global__ void gemm_naive_kernel(GemmOperands op, GemmShape s, EpiParams p) {
                 if (col < d) {
                     p.out_bf16[g * p.out_bf16_gstride + (long long)row * p.ld_out_bf16 + col] = to_bf(acc);
                 } else {
-                    const int which = col >= 2 * d, c = col - (1 + which) * d;
+                    const int kvd = p.n_kv_head * p.head_dim;
+                    const int which = col >= d + kvd, c = col - d - which * kvd;
                     const int head = c / p.head_dim, e = c % p.head_dim;
                     const int b = row / p.seqlen, pos = p.pos0 + row % p.seqlen;
                     uint16_t *base = (which ? p.v_cache : p.k_cache) + g * p.cache_gstride;
-                    base[(((long long)b * p.n_head + head) * p.max_pos + pos) * p.head_dim + e] = to_bf(acc);
+                    base[(((long long)b * p.n_kv_head + head) * p.max_pos + pos) * p.head_dim + e] = to_bf(acc);
                 }
                 break;
             }
@@ -73,8 +74,9 @@ __global__ void attention_naive_kernel(AttnParams p) {
     const int hd = p.head_dim, d = p.n_head * hd;
     const int per = hd / 32;  // 2 or 4 dims per lane
     const uint16_t *q = p.q + g * p.q_gstride + ((long long)b * p.seqlen + t) * d + h * hd;
-    const uint16_t *kc = p.k_cache + g * p.cache_gstride + b * p.cache_bstride + (long long)h * p.max_pos * hd;
-    const uint16_t *vc = p.v_cache + g * p.cache_gstride + b * p.cache_bstride + (long long)h * p.max_pos * hd;
+    const int hk = h / (p.n_head / (p.n_kv_head > 0 ? p.n_kv_head : p.n_head));   // key/value head of this query head
+    const uint16_t *kc = p.k_cache + g * p.cache_gstride + b * p.cache_bstride + (long long)hk * p.max_pos * hd;
+    const uint16_t *vc = p.v_cache + g * p.cache_gstride + b * p.cache_bstride + (long long)hk * p.max_pos * hd;
     float qv[4], o[4] = {0.f, 0.f, 0.f, 0.f};
     for (int i = 0; i < per; ++i) qv[i] = bf(q[lane * per + i]);
     const float scale = rsqrtf(static_cast<float>(hd));

@@ -29,7 +29,7 @@ def test_exports_match_header(L):
 
 
 def test_struct_sizes_match_header():
-    # 8 int32 + float + 2 int32 + 5 reserved = 16 words; 18 pointers
+    # 8 int32 + float + 3 int32 + 4 reserved = 16 words; 18 pointers
     assert C.sizeof(kr.KrakenConfig) == 64
     assert C.sizeof(kr.KrakenWeights) == 18 * 8
 
@@ -38,10 +38,14 @@ def test_query_sizes_arithmetic(L):
     for name, s in ki.CONFIGS.items():
         cfg = kr.make_config(s)
         kv, scratch = kr.query_sizes(cfg)
-        assert kv == s.n_layer * s.n_branch * 2 * s.batch * s.max_pos * s.d_model * 2
+        assert kv == s.n_layer * s.n_branch * 2 * s.batch * s.max_pos * s.kv_heads * s.head_dim * 2
         T = s.batch * s.max_pos
         floor = T * s.d_model * 4 * (2 + 2 * s.n_branch) + T * s.n_branch * 2 * (3 * s.d_model + s.d_ff)
         assert floor <= scratch < floor * 1.05 + (1 << 22)
+    # grouped-query attention shrinks the cache by the group size (the mitigation of Sec. 4.2)
+    full = kr.query_sizes(kr.make_config(ki.CONFIGS["C4"]))[0]
+    assert kr.query_sizes(kr.make_config(ki.CONFIGS["C4-gqa4"]))[0] * 4 == full
+    assert kr.query_sizes(kr.make_config(ki.CONFIGS["C4-mqa"]))[0] * 16 == full
     # C3's cache is the 8.59 GB the shape implies
     assert abs(kr.query_sizes(kr.make_config(ki.CONFIGS["C3"]))[0] / 1e9 - 8.59) < 0.01
 
@@ -58,6 +62,8 @@ def test_config_validation(L):
     assert q(kr.make_config(s, n_head=4)) == kr.EUNSUPPORTED      # head_dim 32
     assert q(kr.make_config(s, d_ff=100)) == kr.EUNSUPPORTED
     assert q(kr.make_config(s, ln_eps=0.0)) == kr.EINVAL
+    assert q(kr.make_config(s, n_kv_head=3)) == kr.EINVAL         # 2 heads cannot share 3 key/value heads
+    assert q(kr.make_config(s, n_kv_head=1)) == kr.OK             # multi-query attention
 
 
 def test_create_rejects_bad_arguments_before_touching_the_device(L):

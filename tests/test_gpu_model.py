@@ -275,10 +275,11 @@ def prefix_parity(name, prefix, seqs):
     m.close()
 
 
-@pytest.mark.parametrize("name", ["K0-104", "K0-96", "K0-72"])
-def test_engine_head_dims_small_models_all_positions_cache_and_decode(name):
-    """Small models with the head dims (104, 96, 72) and the 2 d FFN of the paper's engine shapes (Table 3):
-    every position and the cache element by element, then teacher-forced decode steps."""
+@pytest.mark.parametrize("name", ["K0-104", "K0-96", "K0-72", "C0-gqa", "C0-mqa"])
+def test_engine_head_dims_and_shared_kv_heads_small_models_all_positions_cache_and_decode(name):
+    """Small models with the head dims (104, 96, 72) and the 2 d FFN of the paper's engine shapes (Table 3), and
+    with grouped-query / multi-query attention (Sec. 4.2): every position and the cache element by element,
+    then teacher-forced decode steps."""
     s = ki.CONFIGS[name]
     m, w = build(s)
     wb = host_bits(w)
@@ -324,12 +325,14 @@ def test_c3_full_size_prefix_parity():
     prefix_parity("C3", 32, [0, 3])
 
 
-def test_c4_full_size_prefill_prefix_parity_and_decode_consistency():
+@pytest.mark.parametrize("name", ["C4", "C4-gqa4"])
+def test_c4_full_size_prefill_prefix_parity_and_decode_consistency(name):
     """C4 at full size (16 sequences x 2048 tokens, then decode steps), in the launch configuration
-    the benchmark times.  Prefill: logits and cache rows of a prefix against an oracle run on that
-    prefix (causality).  Decode: a property that holds at any size - prefill(l) followed by one decode
-    step equals prefill(l + 1) at the last position - plus the cache row the step appended."""
-    s = ki.CONFIGS["C4"]
+    the benchmark times; also with 4 query heads per key/value head.  Prefill: logits and cache rows of a
+    prefix against an oracle run on that prefix (causality).  Decode: a property that holds at any size -
+    prefill(l) followed by one decode step equals prefill(l + 1) at the last position - plus the cache row
+    the step appended."""
+    s = ki.CONFIGS[name]
     m, w = build(s)
     wb = host_bits(w)
     tok = ki.uniform_tokens(1, s.vocab, s.batch, s.seqlen + 1, DEV)

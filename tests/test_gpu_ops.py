@@ -187,8 +187,9 @@ def test_gemm_cross_branch_sum(n_tile):
     assert np.array_equal(r["sum"], r["ref"].sum(0))
 
 
-@pytest.mark.parametrize("hd,H", [(64, 2), (128, 1), (104, 3), (72, 2), (96, 1), (96, 3)])
-def test_gemm_qkv_scatter_is_index_exact(hd, H):
+@pytest.mark.parametrize("hd,H,Hkv", [(64, 2, 2), (128, 1, 1), (104, 3, 3), (72, 2, 2), (96, 1, 1), (96, 3, 3),
+                                       (64, 4, 2), (64, 4, 1), (104, 4, 2), (128, 2, 1)])
+def test_gemm_qkv_scatter_is_index_exact(hd, H, Hkv):
     """One-hot activations times integer-coded weights: every cache element names its source.  Head dims that
     are not multiples of 32 (and widths that are not) take the path that stores 16-byte pieces."""
     d = H * hd
@@ -197,16 +198,19 @@ def test_gemm_qkv_scatter_is_index_exact(hd, H):
     t = torch.arange(M, device=DEV)
     a = torch.zeros(G, M, K, dtype=torch.bfloat16, device=DEV)
     a[:, t, t % K] = 1.0
-    o = torch.arange(3 * d, device=DEV)[:, None]
+    kvd = Hkv * hd                                                  # width of the K part and of the V part
+    nout = d + 2 * kvd
+    o = torch.arange(nout, device=DEV)[:, None]
     k = torch.arange(K, device=DEV)[None, :]
     w = torch.stack([((o * 7 + k * 13 + g * 29) % 251 - 125) for g in range(G)]).to(torch.bfloat16).contiguous()
     qbuf = torch.zeros(G, M, d, dtype=torch.bfloat16, device=DEV)
-    cache = torch.full((G, 2, batch, H, P, hd), -7.0, dtype=torch.bfloat16, device=DEV)
+    cache = torch.full((G, 2, batch, Hkv, P, hd), -7.0, dtype=torch.bfloat16, device=DEV)
     args = kr.GemmArgs()
     args.a, args.a_gstride, args.lda = a.data_ptr(), M * K, K
-    args.w, args.w_gstride, args.ldw = w.data_ptr(), 3 * d * K, K
-    args.groups, args.m, args.n_out, args.k = G, M, 3 * d, K
+    args.w, args.w_gstride, args.ldw = w.data_ptr(), nout * K, K
+    args.groups, args.m, args.n_out, args.k = G, M, nout, K
     args.epilogue = kr.EPI_QKV
+    args.n_kv_head = Hkv if Hkv != H else 0
     args.out_bf16, args.out_bf16_gstride, args.ld_out_bf16 = qbuf.data_ptr(), M * d, d
     args.k_cache, args.v_cache = cache[0, 0].data_ptr(), cache[0, 1].data_ptr()
     args.cache_gstride = cache.stride(0)
@@ -220,8 +224,8 @@ def test_gemm_qkv_scatter_is_index_exact(hd, H):
         assert np.array_equal(got_q[g], wf[g][:d, tk].T)
         for which in (0, 1):
             for b in range(batch):
-                for h in range(H):
-                    rows = wf[g][d * (1 + which) + h * hd: d * (1 + which) + (h + 1) * hd]  # [hd, K]
+                for h in range(Hkv):
+                    rows = wf[g][d + which * kvd + h * hd: d + which * kvd + (h + 1) * hd]    # [hd, K]
                     want = rows[:, tk[b * seqlen:(b + 1) * seqlen]].T                          # [seqlen, hd]
                     assert np.array_equal(got_c[g, which, b, h, pos0:pos0 + seqlen], want)
                     # rows outside the written range are untouched
@@ -275,6 +279,58 @@ def test_attention_matches_oracle(hd, seqlen, pos0, kernel, monkeypatch):
                 den += (ref ** 2).sum()
     assert worst < 3e-2, worst
     assert np.sqrt(num / den) < 6e-3, np.sqrt(num / den)
+
+
+@pytest.mark.parametrize("hd,H,Hkv", [(64, 4, 2), (64, 8, 1), (128, 4, 1), (96, 6, 2), (64, 6, 2), (128, 2, 2)])
+@pytest.mark.parametrize("seqlen,pos0", [(300, 0), (100, 37)])
+def test_grouped_query_attention_matches_oracle(hd, H, Hkv, seqlen, pos0):
+    """Query head h attends over key/value head h / (H / Hkv) (prefill kernel), against the oracle's
+    single-head attention on the corresponding cache rows."""
+    G, B, P = 2, 2, 512
+    d = H * hd
+    q = ki.normal_bf16(17, 0, (G, B * seqlen, d), 1.0, DEV)
+    kc = ki.normal_bf16(17, 1, (G, B, Hkv, P, hd), 1.0, DEV)
+    vc = ki.normal_bf16(17, 2, (G, B, Hkv, P, hd), 1.0, DEV)
+    kc[:, :, :, pos0 + seqlen:] = float("nan")
+    vc[:, :, :, pos0 + seqlen:] = float("nan")
+    out = kr.op_attention(q, kc, vc, B, seqlen, pos0, H).float().cpu().numpy()
+    assert not np.isnan(out).any()
+    qn, kn, vn = q.float().cpu().numpy(), kc.float().cpu().numpy(), vc.float().cpu().numpy()
+    worst = 0.0
+    for g in range(G):
+        for b in range(B):
+            for h in range(H):
+                hk = h // (H // Hkv)
+                ref = oracle.attention_head(qn[g, b * seqlen:(b + 1) * seqlen, h * hd:(h + 1) * hd],
+                                            kn[g, b, hk, :pos0 + seqlen], vn[g, b, hk, :pos0 + seqlen], q_pos0=pos0)
+                worst = max(worst, np.abs(out[g, b * seqlen:(b + 1) * seqlen, h * hd:(h + 1) * hd] - ref).max())
+    assert worst < 3e-2, worst
+
+
+@pytest.mark.parametrize("hd,H,Hkv", [(64, 4, 2), (64, 8, 1), (128, 4, 1), (96, 6, 2), (64, 6, 2), (128, 16, 4)])
+@pytest.mark.parametrize("n_keys,splits", [(1, 1), (131, 3), (700, 0), (2049, 32)])
+def test_grouped_query_decode_attention_matches_oracle(hd, H, Hkv, n_keys, splits):
+    """Decode step with shared key/value heads: the query heads of a group are served by one CTA (4, 2 or
+    1 of them at a time)."""
+    G, B, P = 2, 3, 2112
+    d = H * hd
+    q = ki.normal_bf16(18, 0, (G, B, d), 1.0, DEV)
+    kc = ki.normal_bf16(18, 1, (G, B, Hkv, P, hd), 1.0, DEV)
+    vc = ki.normal_bf16(18, 2, (G, B, Hkv, P, hd), 1.0, DEV)
+    kc[:, :, :, n_keys:] = float("nan")
+    vc[:, :, :, n_keys:] = float("nan")
+    out = kr.op_decode_attention(q, kc, vc, n_keys, splits).float().cpu().numpy()
+    assert not np.isnan(out).any()
+    qn, kn, vn = q.float().cpu().numpy(), kc.float().cpu().numpy(), vc.float().cpu().numpy()
+    worst = 0.0
+    for g in range(G):
+        for b in range(B):
+            for h in range(H):
+                hk = h // (H // Hkv)
+                ref = oracle.attention_head(qn[g, b:b + 1, h * hd:(h + 1) * hd], kn[g, b, hk, :n_keys],
+                                            vn[g, b, hk, :n_keys], q_pos0=n_keys - 1)
+                worst = max(worst, np.abs(out[g, b, h * hd:(h + 1) * hd] - ref[0]).max())
+    assert worst < 2e-2, worst
 
 
 @pytest.mark.parametrize("hd", [64, 128, 72, 96, 104])
