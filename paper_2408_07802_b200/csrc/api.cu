@@ -305,7 +305,8 @@ int run_layers(const RunCtx &rc, const int32_t *d_tokens) {
                 dp.n_kv_head = Hkv;
                 dp.max_pos = c.max_pos;
                 dp.pos_dev = rc.pos_dev;
-                dp.splits = decode_attention_splits(N, rc.batch, H, rc.pos_dev ? rc.max_keys : dp.n_keys);
+                dp.splits = decode_attention_splits(N, rc.batch, (hd == 64 || hd == 128) && decode_gqa_tile(H, Hkv) ? Hkv : H,
+                                                    rc.pos_dev ? rc.max_keys : dp.n_keys);
                 dp.partials = at<float>(h, h->lay.dec_part);
                 dp.out = o; dp.out_gstride = td;
                 h->launches[KRAKEN_PROF_ATTENTION] += dp.splits > 1 ? 1 : 0;

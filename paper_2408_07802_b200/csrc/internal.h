@@ -121,6 +121,9 @@ struct DecodeAttnParams {
     long long out_gstride;
 };
 int decode_attention_splits(int groups, int batch, int n_head, int n_keys);
+// whether the query heads of a key/value head are served together by the tensor-core tile kernel (then the
+// number of CTA streams, which the split count should be chosen for, is the number of key/value heads)
+bool decode_gqa_tile(int n_head, int n_kv_head);
 size_t decode_attention_partial_bytes(int groups, int batch, int n_head, int head_dim, int splits);
 int launch_attention_decode(const DecodeAttnParams &p, cudaStream_t stream);
 
