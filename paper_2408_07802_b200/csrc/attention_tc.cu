@@ -19,7 +19,8 @@
 // 2^8 in the exponent; then (rarely) the warp rescales its rows of O in TMEM before releasing P.
 // Using a stale maximum is exact: numerator and denominator carry the same factor.
 // Every role walks a list of work items with running barrier phases, so a CTA can take several items
-// without draining its pipeline; by default the grid has one CTA per item (see launch()).
+// without draining its pipeline: with enough work each SM gets one CTA and a fixed list of couples of items
+// of equal total length (atc_next), else the grid has one CTA per item (see launch()).
 // TMEM: S/P of tile w at column 128 w, O of tile w at 256 + 128 w.  All waits are time-bounded.
 #include <math.h>
 
@@ -41,6 +42,7 @@ constexpr bool POLY_EXP2 = false;
 struct AttnTcArgs {
     int groups, batch, seqlen, pos0, n_head;
     int n_kv_head, kv_rep;   // key/value heads in the cache; query heads per key/value head
+    int balanced;            // 1: a fixed list of work per CTA, built from pairs of items of equal total length
     int head_dim;      // <= HD of the kernel instance, a multiple of 8 (columns past it are zero-filled by TMA)
     uint16_t *out;
     long long out_gstride;
@@ -168,6 +170,35 @@ __device__ __forceinline__ bool atc_item(const AttnTcArgs &a, int idx, AtcItem &
     return true;
 }
 
+// The j-th work item of this CTA (j = 0, 1, ...; advanced here), false when the CTA is done.
+//   one CTA per item:  item blockIdx.x only.
+//   balanced list:     the work of a causal item grows linearly with its place in the sequence, so the k-th
+//                      longest and the k-th shortest pair of query tiles of one head together always cost the
+//                      same.  Such couples are dealt round-robin to the CTAs (couple c, c + grid, ...), long
+//                      half first, which gives every CTA the same work without a queue, keeps a head's K/V on
+//                      neighbouring CTAs, and lets a CTA start the next item while the last one drains.
+__device__ __forceinline__ bool atc_next(const AttnTcArgs &a, int &j, AtcItem &it) {
+    if (!a.balanced) {
+        if (j != 0) return false;
+        ++j;
+        return atc_item(a, blockIdx.x, it);
+    }
+    const int n_pairs = (a.seqlen + 2 * TQ - 1) / (2 * TQ);
+    const int couples = (n_pairs + 1) / 2;                    // per head; the middle pair stands alone when odd
+    const long long total = (long long)couples * a.n_head * a.batch * a.groups;
+    for (;;) {
+        const long long c = blockIdx.x + (long long)(j >> 1) * gridDim.x;
+        if (c >= total) return false;
+        const int k = static_cast<int>(c % couples);
+        const int hb = static_cast<int>(c / couples);
+        const bool second = j & 1;
+        ++j;
+        if (second && k == n_pairs - 1 - k) continue;         // the middle pair has no partner
+        // atc_item numbers the pairs of a head longest first: index k is the (k+1)-th longest
+        return atc_item(a, hb * n_pairs + (second ? n_pairs - 1 - k : k), it);
+    }
+}
+
 template <int HD>
 __global__ void __launch_bounds__(ATC_THREADS, 1)
 attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
@@ -227,7 +258,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             bool ok = true;
             uint32_t kv_cnt = 0, item_cnt = 0;
             AtcItem it;
-            for (int idx = blockIdx.x; ok && atc_item(a, idx, it); idx += gridDim.x, ++item_cnt) {
+            for (int jj = 0; ok && atc_next(a, jj, it); ++item_cnt) {
                 if (!(ok = mbar_wait(q_empty, (item_cnt & 1u) ^ 1u, abort_flag))) break;
                 const int q_tiles = it.n_tiles[1] > 0 ? 2 : 1;
                 mbar_expect_tx(q_full, q_tiles * Cfg::Q_BYTES);
@@ -291,7 +322,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             bool ok = true;
             uint32_t kv_cnt = 0, item_cnt = 0, tile_cnt[2] = {0, 0};
             AtcItem it;
-            for (int idx = blockIdx.x; ok && atc_item(a, idx, it); idx += gridDim.x, ++item_cnt) {
+            for (int jj = 0; ok && atc_next(a, jj, it); ++item_cnt) {
                 if (!(ok = mbar_wait(q_full, item_cnt & 1u, abort_flag))) break;
                 if (!(ok = mbar_wait(k_full + (kv_cnt & 1), (kv_cnt >> 1) & 1, abort_flag))) break;
                 tc_fence_after_sync();
@@ -337,7 +368,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         bool ok = true;
         uint32_t tile_cnt = 0;                               // tiles this warp group has consumed so far
         AtcItem it;
-        for (int idx = blockIdx.x; ok && atc_item(a, idx, it); idx += gridDim.x) {
+        for (int jj = 0; ok && atc_next(a, jj, it);) {
             const int tile_q0 = it.q0 + w * TQ;
             const int rows_valid = min(TQ, a.seqlen - tile_q0);
             const int qpos = a.pos0 + tile_q0 + row;         // position of this query
@@ -487,13 +518,18 @@ int launch(const CUtensorMap &tmQ, const CUtensorMap &tmK, const CUtensorMap &tm
         configured = true;
     }
     const long long items = (long long)((a.seqlen + 2 * TQ - 1) / (2 * TQ)) * a.n_head * a.batch * a.groups;
-    // One CTA per item lets the hardware scheduler balance the very unequal items (a pair of query
-    // tiles near the end of a sequence has ten times the keys of the first pair); a fixed list per SM
-    // measured slower (0.38 vs 0.35 ms at 4 x 2048 x 16 heads x 128) because of that imbalance.
+    // With enough work, one CTA per SM walks a fixed list of couples of equal total length (atc_next); a plain
+    // round-robin list of single items measured slower than one CTA per item (0.38 vs 0.35 ms at 4 x 2048 x 16
+    // heads x 128) because the items are so unequal.  KRAKEN_ATTN_ONE_CTA_PER_ITEM=1 keeps the hardware scheduler.
     const int sms = sm_count() > 0 ? sm_count() : 148;
-    const bool persistent = env_flag("KRAKEN_ATTN_PERSISTENT");
-    dim3 grid(static_cast<unsigned>(persistent && items > sms ? sms : items));
-    attn_tc_kernel<HD><<<grid, ATC_THREADS, Cfg::SMEM_BYTES, stream>>>(tmQ, tmK, tmV, a);
+    const long long couples = (long long)(((a.seqlen + 2 * TQ - 1) / (2 * TQ) + 1) / 2) * a.n_head * a.batch * a.groups;
+    AttnTcArgs b = a;
+    // the list pays when its rounds fill the machine: couples / (SMs x rounds) >= 0.85 (measured: 0.87 gains 7 %,
+    // 0.72 loses 3 % against one CTA per item)
+    const long long rounds = (couples + sms - 1) / sms;
+    b.balanced = couples >= 2LL * sms && couples * 100 >= 85LL * sms * rounds && !env_flag("KRAKEN_ATTN_ONE_CTA_PER_ITEM");
+    dim3 grid(static_cast<unsigned>(b.balanced ? sms : items));
+    attn_tc_kernel<HD><<<grid, ATC_THREADS, Cfg::SMEM_BYTES, stream>>>(tmQ, tmK, tmV, b);
     return cuda_check(cudaGetLastError(), "attention: launch");
 }
 
