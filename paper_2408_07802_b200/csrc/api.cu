@@ -21,7 +21,7 @@ constexpr size_t ALIGN = 256;
 size_t align_up(size_t v) { return (v + ALIGN - 1) / ALIGN * ALIGN; }
 
 struct Layout {
-    size_t status, tokens, rows, logits, x0, x, a, s, u, q, o, g, dec_part, total;
+    size_t status, tokens, rows, logits, x0, x, a, s, u, q, o, g, dec_part, x_alt, total;
 };
 
 int kv_heads_of(const kraken_config &c) { return c.n_kv_head > 0 ? c.n_kv_head : c.n_head; }
@@ -71,6 +71,7 @@ Layout layout_of(const kraken_config *c) {
     l.g = take(N * T * F * 2);
     l.dec_part = take(decode_attention_partial_bytes(c->n_branch, c->max_batch, c->n_head, c->d_model / c->n_head,
                                                      DECODE_MAX_SPLITS));
+    l.x_alt = take((size_t)N * c->max_batch * d * 4);   // second copy of the branch outputs of a decode step
     l.total = off;
     return l;
 }
@@ -78,6 +79,8 @@ Layout layout_of(const kraken_config *c) {
 enum GemmKind { G_QKV = 0, G_PROJ, G_UP, G_DOWN, G_CONCAT, G_HEAD, G_COUNT };
 
 }  // namespace
+
+constexpr int MAX_CHAINS = 8;
 
 struct kraken_handle {
     kraken_config cfg;
@@ -108,6 +111,10 @@ struct kraken_handle {
     int dec_eager_steps;                      // eager steps done for the current batch size (warm-up)
     long long dec_graph_launches[KRAKEN_PROF_COUNT];
     bool use_graph;
+    // decode steps run the branches as concurrent chains, one stream each (see run_layers_decode_branches)
+    cudaStream_t br_stream[MAX_CHAINS];
+    cudaEvent_t ev_fork, ev_join[MAX_CHAINS], ev_down[2][MAX_CHAINS];
+    bool br_ready;
     // launch accounting and optional per-kernel timing
     long long launches[KRAKEN_PROF_COUNT];
     bool prof_on;
@@ -163,8 +170,10 @@ struct RunCtx {
 };
 
 // One grouped GEMM of the model: weights of `kind` at `layer`.
+// g0 / gcnt: a run of branches (gcnt = 0: all of them; the caller then passes A and the epilogue's pointers
+// already moved to branch g0); st: the stream (null: the call's stream).
 int model_gemm(const RunCtx &rc, GemmKind kind, int layer, int m_rows, const uint16_t *a, long long a_gstride,
-               EpiParams epi) {
+               EpiParams epi, int g0 = 0, int gcnt = 0, cudaStream_t st = nullptr) {
     kraken_handle *h = rc.h;
     const kraken_config &c = h->cfg;
     const int d = c.d_model, F = c.d_ff, N = c.n_branch;
@@ -183,15 +192,17 @@ int model_gemm(const RunCtx &rc, GemmKind kind, int layer, int m_rows, const uin
     }
     const bool layered = kind <= G_DOWN;
     total_groups = layered ? c.n_layer * N : 1;
+    if (gcnt > 0) s.groups = gcnt;
+    if (!st) st = rc.st;
     const long long w_gstride = (long long)s.n_out * s.k;
     op.a = a;
     op.a_gstride = a_gstride;
     op.lda = s.k;
     op.ldw = s.k;
     op.w_gstride = w_gstride;
-    op.w = wbase + (layered ? (long long)layer * N * w_gstride : 0);
+    op.w = wbase + (layered ? ((long long)layer * N + g0) * w_gstride : 0);
     if (bias) {
-        epi.bias = bias + (layered ? (long long)layer * N * s.n_out : 0);
+        epi.bias = bias + (layered ? ((long long)layer * N + g0) * s.n_out : 0);
         epi.bias_gstride = s.n_out;
     } else {
         epi.bias = nullptr;
@@ -199,9 +210,9 @@ int model_gemm(const RunCtx &rc, GemmKind kind, int layer, int m_rows, const uin
     }
     static const int cat_of[G_COUNT] = {KRAKEN_PROF_GEMM_QKV, KRAKEN_PROF_GEMM_PROJ, KRAKEN_PROF_GEMM_UP,
                                         KRAKEN_PROF_GEMM_DOWN, KRAKEN_PROF_TAIL, KRAKEN_PROF_TAIL};
-    LaunchScope scope(h, cat_of[kind], rc.st);
-    if (h->naive) return launch_gemm_naive(op, s, epi, rc.st);
-    if (m_rows <= SKINNY_MAX_ROWS && epi.kind != KRAKEN_EPI_RESID_SUM) return launch_gemm_skinny(op, s, epi, rc.st);
+    LaunchScope scope(h, cat_of[kind], st);
+    if (h->naive) return launch_gemm_naive(op, s, epi, st);
+    if (m_rows <= SKINNY_MAX_ROWS && epi.kind != KRAKEN_EPI_RESID_SUM) return launch_gemm_skinny(op, s, epi, st);
 
     const int bn = gemm_pick_bn(s);
     if (h->tmB_bn[kind] != bn) {
@@ -219,8 +230,8 @@ int model_gemm(const RunCtx &rc, GemmKind kind, int layer, int m_rows, const uin
         if (r) return r;
         h->tmA_rows[kind] = m_rows;
     }
-    return launch_gemm_tc(op, s, epi, &h->tmA[kind], &h->tmB[kind], layered ? layer * N : 0, bn,
-                          at<uint32_t>(h, h->lay.status), rc.st);
+    return launch_gemm_tc(op, s, epi, &h->tmA[kind], &h->tmB[kind], layered ? layer * N + g0 : 0, bn,
+                          at<uint32_t>(h, h->lay.status), st);
 }
 
 EpiParams epi_zero() {
@@ -351,6 +362,154 @@ int run_layers(const RunCtx &rc, const int32_t *d_tokens) {
             KR_TRY(launch_sum_groups(x, td, N, td, S, rc.st));
         }
     }
+    h->last_rows = T;
+    return KRAKEN_OK;
+}
+
+// Streams and events of the branch chains, created on first use.
+int branch_streams(kraken_handle *h) {
+    if (h->br_ready) return KRAKEN_OK;
+    for (int b = 0; b < MAX_CHAINS; ++b) {
+        if (cudaStreamCreateWithFlags(&h->br_stream[b], cudaStreamNonBlocking) != cudaSuccess) return KRAKEN_ECUDA;
+        if (cudaEventCreateWithFlags(&h->ev_join[b], cudaEventDisableTiming) != cudaSuccess) return KRAKEN_ECUDA;
+        for (int p = 0; p < 2; ++p)
+            if (cudaEventCreateWithFlags(&h->ev_down[p][b], cudaEventDisableTiming) != cudaSuccess) return KRAKEN_ECUDA;
+    }
+    if (cudaEventCreateWithFlags(&h->ev_fork, cudaEventDisableTiming) != cudaSuccess) return KRAKEN_ECUDA;
+    h->br_ready = true;
+    return KRAKEN_OK;
+}
+
+// The layers of one decode step (one new token per sequence) with every branch as its own chain of
+// launches on its own stream.  A decode layer alternates a bandwidth-bound kernel (attention streaming the
+// KV cache) with a run of short latency-bound ones (LayerNorms, weight-streaming GEMMs of a few MB);
+// launched for all branches at once the two kinds take turns and HBM idles during the second.  The
+// branches of a Kraken layer depend on each other only through the cross-branch sum that LayerNorm-2
+// reads (Algorithm 1), so here branch b's chain  LN1 -> qkv -> attention -> proj  runs ahead on its own
+// and only its LN2 waits for the other branches' previous-layer outputs; the chains drift apart by
+// themselves, so one branch's cache streaming overlaps the others' short kernels (starting them a kernel
+// or more apart on purpose measured the same or worse).
+// Branch outputs alternate between two buffers by layer: a chain that runs ahead writes layer l while
+// another chain's LN2 still sums the outputs of layer l-1.
+int run_layers_decode_branches(const RunCtx &rc, const int32_t *d_tokens) {
+    kraken_handle *h = rc.h;
+    const kraken_config &c = h->cfg;
+    const int d = c.d_model, F = c.d_ff, N = c.n_branch, L = c.n_layer, H = c.n_head, hd = d / H, T = rc.T;
+    const long long td = (long long)T * d;
+    KR_TRY(branch_streams(h));
+    float *x0 = at<float>(h, h->lay.x0), *a = at<float>(h, h->lay.a);
+    float *xbuf[2] = {at<float>(h, h->lay.x), at<float>(h, h->lay.x_alt)};
+    uint16_t *u = at<uint16_t>(h, h->lay.u), *q = at<uint16_t>(h, h->lay.q), *o = at<uint16_t>(h, h->lay.o),
+             *gb = at<uint16_t>(h, h->lay.g);
+    uint32_t *status = at<uint32_t>(h, h->lay.status);
+    const int Hkv = kv_heads_of(c);
+    const long long cache_b = (long long)Hkv * c.max_pos * hd;
+    const long long cache_kv = (long long)c.max_batch * cache_b;
+    uint16_t *kv = reinterpret_cast<uint16_t *>(h->kv);
+    auto stream_of = [&](int b) { return b == 0 ? rc.st : h->br_stream[b]; };
+    auto out_of = [&](int l) { return xbuf[(L - 1 - l) & 1]; };   // the last layer lands in the main buffer
+#define KR_CU(x)                                              \
+    do {                                                      \
+        if ((x) != cudaSuccess) return cuda_check(cudaGetLastError(), "decode branch chains"); \
+    } while (0)
+
+    {
+        LaunchScope scope(h, KRAKEN_PROF_EMBED, rc.st);
+        KR_TRY(launch_embed(d_tokens, T, rc.seqlen, rc.pos0, (const uint16_t *)h->w.wte, (const uint16_t *)h->w.wpe, d,
+                            c.vocab, x0, status, rc.st, rc.pos_dev));
+    }
+    KR_CU(cudaEventRecord(h->ev_fork, rc.st));
+    for (int b = 1; b < N; ++b) KR_CU(cudaStreamWaitEvent(h->br_stream[b], h->ev_fork, 0));
+
+    const int tile = (hd == 64 || hd == 128) && decode_gqa_tile(H, Hkv);
+    // splits per (sequence, head) of one branch: about six CTAs per SM per branch launch, rounded to nearest
+    // (measured at 16 x 16 streams of 2100 keys: 3 splits 2.98 ms per step, 2: 3.11, 4: 3.16, 1: 3.36)
+    int splits;
+    {
+        const long long streams = (long long)rc.batch * (tile ? Hkv : H);
+        const int n_keys = rc.pos_dev ? rc.max_keys : rc.pos0 + 1;
+        const long long want = 6LL * (sm_count() > 0 ? sm_count() : 148);
+        long long sp = (want + streams / 2) / streams;
+        const long long by_len = (n_keys + 127) / 128;
+        if (sp > by_len) sp = by_len;
+        if (sp > DECODE_MAX_SPLITS) sp = DECODE_MAX_SPLITS;
+        if (sp < 1) sp = 1;
+        splits = static_cast<int>(sp);
+    }
+    const long long part_b = (long long)rc.batch * H * splits * (hd + 2);   // floats of partials per branch
+
+    for (int l = 0; l < L; ++l) {
+        const long long ln_off = (long long)l * N * d;
+        float *xout = out_of(l);
+        const float *xprev = l == 0 ? nullptr : out_of(l - 1);
+        uint16_t *kc = kv + (long long)l * N * 2 * cache_kv;
+        for (int b = 0; b < N; ++b) {
+            cudaStream_t st = stream_of(b);
+            const float *xin = l == 0 ? x0 : xprev + b * td;
+            {
+                LaunchScope scope(h, KRAKEN_PROF_LAYERNORM, st);
+                KR_TRY(launch_layernorm(xin, 0, nullptr, (const uint16_t *)h->w.ln1_g + ln_off + (long long)b * d,
+                                        h->w.ln1_b ? (const uint16_t *)h->w.ln1_b + ln_off + (long long)b * d : nullptr,
+                                        1, T, d, c.ln_eps, u + b * td, st));
+            }
+            EpiParams e = epi_zero();
+            e.kind = KRAKEN_EPI_QKV;
+            e.out_bf16 = q + b * td; e.out_bf16_gstride = td; e.ld_out_bf16 = d;
+            e.k_cache = kc + (long long)b * 2 * cache_kv; e.v_cache = e.k_cache + cache_kv; e.cache_gstride = 2 * cache_kv;
+            e.seqlen = rc.seqlen; e.pos0 = rc.pos0; e.n_head = H; e.head_dim = hd; e.max_pos = c.max_pos; e.d_model = d;
+            e.n_kv_head = Hkv;
+            e.pos0_dev = rc.pos_dev;
+            KR_TRY(model_gemm(rc, G_QKV, l, T, u + b * td, td, e, b, 1, st));
+            {
+                LaunchScope scope(h, KRAKEN_PROF_ATTENTION, st);
+                DecodeAttnParams dp;
+                dp.q = q + b * td; dp.q_gstride = td;
+                dp.k_cache = e.k_cache; dp.v_cache = e.v_cache;
+                dp.cache_gstride = 2 * cache_kv; dp.cache_bstride = cache_b;
+                dp.groups = 1; dp.batch = rc.batch; dp.n_keys = rc.pos0 + 1; dp.n_head = H; dp.head_dim = hd;
+                dp.n_kv_head = Hkv;
+                dp.max_pos = c.max_pos;
+                dp.pos_dev = rc.pos_dev;
+                dp.splits = splits;
+                dp.partials = at<float>(h, h->lay.dec_part) + b * part_b;
+                dp.out = o + b * td; dp.out_gstride = td;
+                h->launches[KRAKEN_PROF_ATTENTION] += dp.splits > 1 ? 1 : 0;
+                KR_TRY(launch_attention_decode(dp, st));
+            }
+            e = epi_zero();
+            e.kind = KRAKEN_EPI_RESID_F32;
+            e.out_f32 = a + b * td; e.out_f32_gstride = td; e.ld_out_f32 = d;
+            e.resid = xin; e.resid_gstride = 0; e.ld_resid = d;
+            KR_TRY(model_gemm(rc, G_PROJ, l, T, o + b * td, td, e, b, 1, st));
+            // LayerNorm-2 sums the previous layer's outputs of every branch
+            if (l > 0)
+                for (int j = 0; j < N; ++j)
+                    if (j != b) KR_CU(cudaStreamWaitEvent(st, h->ev_down[(l - 1) & 1][j], 0));
+            {
+                LaunchScope scope(h, KRAKEN_PROF_LAYERNORM, st);
+                KR_TRY(launch_layernorm(a + b * td, 0, l == 0 ? x0 : nullptr,
+                                        (const uint16_t *)h->w.ln2_g + ln_off + (long long)b * d,
+                                        h->w.ln2_b ? (const uint16_t *)h->w.ln2_b + ln_off + (long long)b * d : nullptr,
+                                        1, T, d, c.ln_eps, u + b * td, st, l == 0 ? nullptr : xprev, td, N));
+            }
+            e = epi_zero();
+            e.kind = KRAKEN_EPI_GELU_BF16;
+            e.out_bf16 = gb + b * (long long)T * F; e.out_bf16_gstride = (long long)T * F; e.ld_out_bf16 = F;
+            e.gelu_tanh = c.gelu_tanh;
+            KR_TRY(model_gemm(rc, G_UP, l, T, u + b * td, td, e, b, 1, st));
+            e = epi_zero();
+            e.kind = KRAKEN_EPI_RESID_F32;
+            e.out_f32 = xout + b * td; e.out_f32_gstride = td; e.ld_out_f32 = d;
+            e.resid = a + b * td; e.resid_gstride = td; e.ld_resid = d;
+            KR_TRY(model_gemm(rc, G_DOWN, l, T, gb + b * (long long)T * F, (long long)T * F, e, b, 1, st));
+            KR_CU(cudaEventRecord(h->ev_down[l & 1][b], st));
+        }
+    }
+    for (int b = 1; b < N; ++b) {
+        KR_CU(cudaEventRecord(h->ev_join[b], h->br_stream[b]));
+        KR_CU(cudaStreamWaitEvent(rc.st, h->ev_join[b], 0));
+    }
+#undef KR_CU
     h->last_rows = T;
     return KRAKEN_OK;
 }
@@ -524,6 +683,7 @@ int kraken_create(const kraken_config *cfg, const kraken_weights *w, void *d_kv,
     h->pre_tokens = h->pre_logits = nullptr;
     h->pre_batch = h->pre_seqlen = h->pre_all = h->pre_seen = 0;
     h->cap_stream = nullptr;
+    h->br_ready = false;
     h->dec_graph_batch = 0;
     h->dec_eager_steps = 0;
     h->use_graph = !env_flag("KRAKEN_NO_GRAPH") && !h->naive;
@@ -583,12 +743,22 @@ int kraken_logits_rows(kraken_handle *h, const int32_t *h_rows, int32_t n_rows, 
 
 namespace {
 
+// Whether decode steps of this handle run the branches as concurrent chains.
+bool decode_chains(const kraken_handle *h) {
+    return !h->naive && h->cfg.n_branch >= 2 && h->cfg.n_branch <= MAX_CHAINS && !env_flag("KRAKEN_DECODE_ONE_CHAIN");
+}
+
 // The kernel sequence of one decode step; with from_dev the position is read from device memory.
 int decode_body(kraken_handle *h, cudaStream_t st, const int32_t *d_tokens, int batch, float *d_logits,
                 bool from_dev) {
     int *d_pos = at<int>(h, h->lay.status + 128);
     RunCtx rc{h, st, batch, 1, h->cur_len, batch, from_dev ? d_pos : nullptr, h->cfg.max_pos};
-    KR_TRY(run_layers(rc, d_tokens));
+    // per-kernel timing wants the kernels one after the other, so profiled steps keep all branches in one chain
+    if (decode_chains(h) && !h->prof_on) {
+        KR_TRY(run_layers_decode_branches(rc, d_tokens));
+    } else {
+        KR_TRY(run_layers(rc, d_tokens));
+    }
     h->last_seqlen = 1;
     int32_t *rows = at<int32_t>(h, h->lay.rows);
     h->launches[KRAKEN_PROF_TAIL]++;
@@ -607,6 +777,7 @@ int kraken_decode_step(kraken_handle *h, const int32_t *d_tokens, int32_t batch,
     if (h->cur_len + 1 > h->cfg.max_pos) return KRAKEN_ECAPACITY;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     h->last_stream = st;
+    if (decode_chains(h)) KR_TRY(branch_streams(h));   // created outside any capture
     if (h->dec_graph_batch != batch) {            // a new batch size: forget the old graph, warm up again
         if (h->dec_graph) cudaGraphExecDestroy(h->dec_graph);
         h->dec_graph = nullptr;
@@ -733,6 +904,15 @@ void kraken_destroy(kraken_handle *h) {
     if (h->dec_graph) cudaGraphExecDestroy(h->dec_graph);
     if (h->pre_graph) cudaGraphExecDestroy(h->pre_graph);
     if (h->cap_stream) cudaStreamDestroy(h->cap_stream);
+    if (h->br_ready) {
+        for (int b = 0; b < MAX_CHAINS; ++b) {
+            cudaStreamDestroy(h->br_stream[b]);
+            cudaEventDestroy(h->ev_join[b]);
+            cudaEventDestroy(h->ev_down[0][b]);
+            cudaEventDestroy(h->ev_down[1][b]);
+        }
+        cudaEventDestroy(h->ev_fork);
+    }
     delete h;
 }
 
