@@ -229,6 +229,44 @@ def test_decode_teacher_forced_matches_oracle():
         assert (a - b_).abs().max() <= 2.0 ** -6 * b_.abs().max()
 
 
+@pytest.mark.parametrize("n_branch", [1, 3, 8, 9])
+@pytest.mark.parametrize("one_chain", [False, True])
+def test_decode_branch_chains_any_branch_count(n_branch, one_chain, monkeypatch):
+    """Decode steps run the branches as concurrent chains of launches (up to 8; more, or one branch, fall back
+    to the single chain): teacher-forced steps against the oracle for odd and large branch counts, replayed
+    graph steps included, and the same bits from the single-chain path."""
+    if one_chain:
+        monkeypatch.setenv("KRAKEN_DECODE_ONE_CHAIN", "1")
+    s = ki.KrakenShape(f"chains{n_branch}", n_branch, 3, 128, 2, 256, 512, 64, 2, 20)
+    steps = 5
+    m, w = build(s)
+    wb = host_bits(w)
+    tok = ki.uniform_tokens(21, s.vocab, s.batch, s.seqlen + steps, DEV)
+    m.prefill(tok[:, :s.seqlen].contiguous())
+    orcs = [oracle.Oracle(s, wb, bf16_store=False) for _ in range(s.batch)]
+    for b in range(s.batch):
+        orcs[b].prefill(tok[b, :s.seqlen].cpu().numpy())
+    outs = []
+    for t in range(s.seqlen, s.seqlen + steps):
+        got = m.decode_step(tok[:, t].contiguous()).cpu().numpy()
+        outs.append(got)
+        for b in range(s.batch):
+            ref = orcs[b].decode_step(int(tok[b, t]))
+            rel, mx = logits_metrics(got[b], ref)
+            assert rel <= REL_L2_MAX and mx <= MAX_ABS_MAX, (n_branch, t, b, rel, mx)
+    assert m.device_status() == 0 and m.cur_len == s.seqlen + steps
+    if not one_chain:
+        # the chains change the order of launches, not the arithmetic
+        monkeypatch.setenv("KRAKEN_DECODE_ONE_CHAIN", "1")
+        m2, _ = build(s)
+        m2.prefill(tok[:, :s.seqlen].contiguous())
+        for i, t in enumerate(range(s.seqlen, s.seqlen + steps)):
+            again = m2.decode_step(tok[:, t].contiguous()).cpu().numpy()
+            assert np.array_equal(again, outs[i]), (n_branch, t)
+        m2.close()
+    m.close()
+
+
 # ------------------------------------------------------------------ C1 .. C3 at full size
 
 def test_c1_full_parity():
