@@ -98,10 +98,13 @@ def host_weight_bits(w):
     return {k: (None if v is None else ki.bf16_tensor_to_bits(v)) for k, v in w.items()}
 
 
+HALF = False   # set from --dtype: the oracle then reads the weight patterns as IEEE half
+
+
 def oracle_tokens_per_s(shape, wb, ids, n_tokens):
     """Oracle prefill of the first n_tokens of one sequence (last-position logits only)."""
     import oracle
-    orc = oracle.Oracle(shape, wb)
+    orc = oracle.Oracle(shape, wb, half=HALF)
     t0 = time.perf_counter()
     orc.prefill(ids[:n_tokens], logits_from=n_tokens - 1)
     dt = time.perf_counter() - t0
@@ -118,7 +121,7 @@ def run_reference(args, shape):
     if rank != 0:
         return
     dev = "cuda:0" if torch.cuda.is_available() else "cpu"
-    w = ki.make_weights(shape, seed=0, device=dev)
+    w = ki.make_weights(shape, seed=0, device=dev, dtype=args.dtype)
     wb = host_weight_bits(w)
     del w
     ids = ki.uniform_tokens(1, shape.vocab, shape.batch, shape.seqlen)[0].numpy()
@@ -190,8 +193,8 @@ def run_decode(args, shape, kr, ki, replicas, torch):
     rank, local_rank, world = replicas.rank_env()
     dev = f"cuda:{local_rank}"
     steps = min(args.steps, shape.decode_steps)
-    w = ki.make_weights(shape, seed=0, device=dev)
-    model = kr.KrakenModel(kr.make_config(shape), w, dev)
+    w = ki.make_weights(shape, seed=0, device=dev, dtype=args.dtype)
+    model = kr.KrakenModel(kr.make_config(shape), w, dev, dtype=args.dtype)
     tok = ki.uniform_tokens(replicas.token_seed(rank), shape.vocab, shape.batch, shape.seqlen, dev)
     logits = torch.empty(shape.batch, shape.vocab, dtype=torch.float32, device=dev)
 
@@ -268,7 +271,7 @@ def run_decode(args, shape, kr, ki, replicas, torch):
     line = {
         "metric": "decode_tokens_per_s", "value": value, "unit": "tokens/s", "n_gpus": world, "steps": steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "bf16", "data": "synthetic", "config": workload_config(shape, args),
+        "vs_baseline": None, "dtype": args.dtype, "data": "synthetic", "config": workload_config(shape, args),
         "hbm_gbs": total_bytes / (ms_per_step * 1e-3) / 1e9,
         "frac_of_measured_hbm": total_bytes / (ms_per_step * 1e-3) / 1e9 / peaks["hbm_gbs"],
         "bytes_per_step": {"weights": wb_, "kv_cache": kvb, "at_cache_length": t_mid},
@@ -292,7 +295,7 @@ def run_decode(args, shape, kr, ki, replicas, torch):
         import oracle
         hb = host_weight_bits(w)
         ctx, n_dec = 256, 8
-        orc = oracle.Oracle(shape, hb)
+        orc = oracle.Oracle(shape, hb, half=HALF)
         ids = tok[0].cpu().numpy()
         orc.prefill(ids[:ctx], logits_from=ctx - 1)
         t0 = time.perf_counter()
@@ -316,6 +319,8 @@ def main():
     ap.add_argument("--seqlen", type=int, default=0,
                     help="prompt length override (the paper's engine shapes K* were timed at 128 and 2048)")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--dtype", default="bf16", choices=["bf16", "f16"],
+                    help="16-bit storage type: bf16 (libkraken.so) or IEEE half (libkraken_f16.so, the paper's precision)")
     ap.add_argument("--ref-tokens", type=int, default=8, help="tokens per step of the reference arm")
     ap.add_argument("--cpu-baseline-seconds", type=float, default=15.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -323,6 +328,8 @@ def main():
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
     import kraken_inputs as ki
+    global HALF
+    HALF = args.dtype == "f16"
     shape = ki.CONFIGS[args.workload]
     if args.seqlen:
         import dataclasses
@@ -345,10 +352,10 @@ def main():
     if world > 1:
         dist = replicas.init_process_group("nccl", torch.device(dev))
     if rank == 0:
-        kbuild.build()
+        kbuild.build(dtype=args.dtype)
     if dist:
         dist.barrier()
-    kr.lib()
+    kr.lib(args.dtype)
     if shape.decode_steps:
         if args.steps == 10:
             args.steps = shape.decode_steps
@@ -357,8 +364,8 @@ def main():
             dist.destroy_process_group()
         return
 
-    w = ki.make_weights(shape, seed=0, device=dev)
-    model = kr.KrakenModel(kr.make_config(shape), w, dev)
+    w = ki.make_weights(shape, seed=0, device=dev, dtype=args.dtype)
+    model = kr.KrakenModel(kr.make_config(shape), w, dev, dtype=args.dtype)
     tok = ki.uniform_tokens(replicas.token_seed(rank), shape.vocab, shape.batch, shape.seqlen, dev)
     logits = torch.empty(shape.batch, shape.vocab, dtype=torch.float32, device=dev)
     flush = None
@@ -457,7 +464,7 @@ def main():
         # tokens/s against the paper's figure for the same engine shape and context, where it prints one
         "vs_baseline": (value / (shape.seqlen / (paper_ttft_ms(shape) * 1e-3))
                         if paper_ttft_ms(shape) is not None and world == 1 else None),
-        "dtype": "bf16",
+        "dtype": args.dtype,
         "data": "synthetic", "config": workload_config(shape, args),
         "model_tflops": fl["total"] / (ms_per_step * 1e-3) / 1e12,
         "frac_of_nominal_2250": fl["total"] / (ms_per_step * 1e-3) / 2.25e15,

@@ -16,7 +16,12 @@
  *   - "device" pointers are CUDA device memory of the current device; "host" pointers
  *     are ordinary (preferably pinned) host memory.  The library never allocates device
  *     memory: weights, KV cache, scratch, tokens and logits are caller-owned.
- *   - bf16 tensors are raw 16-bit patterns, row-major, innermost dimension contiguous.
+ *   - 16-bit tensors ("bf16" below) are raw 16-bit patterns, row-major, innermost dimension
+ *     contiguous.  The library comes as two images of the same ABI: libkraken.so stores weights,
+ *     activations and the KV cache as bfloat16, libkraken_f16.so as IEEE half (the precision of the
+ *     paper's engines, Sec. 4.2); wherever this header says bf16 the second image means half.
+ *     kraken_storage_dtype() tells which one is loaded.  Accumulation, the residual stream and the
+ *     logits are fp32 in both.
  *   - Calls only enqueue work on the given stream (a cudaStream_t passed as void*; NULL
  *     is the legacy default stream) unless stated otherwise.
  *   - Every call returns 0 or a negative kraken_status.  Nothing aborts, throws across
@@ -165,6 +170,8 @@ void kraken_destroy(kraken_handle *h);
 const char *kraken_strerror(int status);
 /* Text of the most recent CUDA failure behind a KRAKEN_ECUDA on the calling thread ("" if none). */
 const char *kraken_last_cuda_error(void);
+/* 16-bit storage type this image was built for: 0 = bfloat16, 1 = IEEE half. */
+int kraken_storage_dtype(void);
 
 /* ------------------------------------------------------------------------------------------
  * Single steps of the path, exposed so that each kernel can be checked on its own.  All

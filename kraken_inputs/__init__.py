@@ -231,29 +231,36 @@ def uniform_tokens(seed: int, vocab: int, batch: int, seqlen: int, device="cpu")
     return ((h * vocab) >> 32).to(torch.int32).reshape(batch, seqlen)
 
 
+def normal_f16(seed: int, tensor_id: int, shape, std: float = 0.02, device="cpu") -> torch.Tensor:
+    """The same draws as normal_bf16, held as IEEE half (every table value converts exactly except the few
+    below 2^-14, which round to half's subnormal grid)."""
+    return normal_bf16(seed, tensor_id, shape, std, device).to(torch.float16)
+
+
 def make_weights(s: KrakenShape, seed: int = 0, device="cpu", std: float = 0.02,
-                 bias: bool = True) -> Dict[str, Optional[torch.Tensor]]:
-    """All weight tensors of a Kraken model as bf16 torch tensors.
+                 bias: bool = True, dtype: str = "bf16") -> Dict[str, Optional[torch.Tensor]]:
+    """All weight tensors of a Kraken model as 16-bit torch tensors (dtype "bf16" or "f16").
 
     Linear weights and (if bias) linear biases ~ N(0, std^2); LayerNorm gamma = 1,
     beta = 0.  With bias=False the bias entries are None (the ABI's NULL = zeros).
     """
+    tdt = {"bf16": torch.bfloat16, "f16": torch.float16}[dtype]
     out: Dict[str, Optional[torch.Tensor]] = {}
     for tid, (name, shape) in enumerate(weight_shapes(s).items()):
         assert WEIGHT_FIELDS[tid] == name
         if name.endswith("_g") and name.startswith("ln"):
-            out[name] = torch.ones(shape, dtype=torch.bfloat16, device=device)
+            out[name] = torch.ones(shape, dtype=tdt, device=device)
         elif name.endswith("_b") and name.startswith("ln"):
-            out[name] = torch.zeros(shape, dtype=torch.bfloat16, device=device)
+            out[name] = torch.zeros(shape, dtype=tdt, device=device)
         elif name.startswith("b_") and not bias:
             out[name] = None
         else:
-            out[name] = normal_bf16(seed, tid, shape, std, device)
+            out[name] = normal_bf16(seed, tid, shape, std, device).to(tdt)
     return out
 
 
 def bf16_tensor_to_bits(t: torch.Tensor) -> np.ndarray:
-    """Host uint16 view of a bf16 tensor (copied to CPU if needed)."""
+    """Host uint16 view of a 16-bit (bf16 or half) tensor (copied to CPU if needed)."""
     return t.detach().cpu().contiguous().view(torch.int16).numpy().view(np.uint16)
 
 

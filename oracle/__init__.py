@@ -36,7 +36,7 @@ class KoConfig(C.Structure):
     _fields_ = [(n, C.c_int32) for n in
                 ("n_branch", "n_layer", "d_model", "n_head", "d_ff", "vocab", "max_pos")] + [
         ("ln_eps", C.c_float), ("gelu_tanh", C.c_int32), ("final_ln", C.c_int32),
-        ("bf16_store", C.c_int32), ("y_zero", C.c_int32), ("n_kv_head", C.c_int32)]
+        ("bf16_store", C.c_int32), ("y_zero", C.c_int32), ("half", C.c_int32), ("n_kv_head", C.c_int32)]
 
 
 class KoWeights(C.Structure):
@@ -66,6 +66,11 @@ def lib():
         L.ko_gelu.argtypes = [C.c_float, C.c_int]
         L.ko_round_bf16.restype = C.c_float
         L.ko_round_bf16.argtypes = [C.c_float]
+        L.ko_round_f16.restype = C.c_float
+        L.ko_round_f16.argtypes = [C.c_float]
+        L.ko_f16_to_f32.restype = C.c_float
+        L.ko_f16_to_f32.argtypes = [C.c_uint16]
+        L.ko_set_half.argtypes = [C.c_int]
         L.ko_num_threads.restype = C.c_int
         L.ko_layernorm.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_void_p,
                                    C.c_float, C.c_int, C.c_void_p]
@@ -102,28 +107,42 @@ def round_bf16(x: float) -> float:
     return float(lib().ko_round_bf16(float(x)))
 
 
+def round_f16(x: float) -> float:
+    """fp32 -> nearest IEEE half (ties to even), as a float."""
+    return float(lib().ko_round_f16(float(x)))
+
+
+def f16_to_f32(bits: int) -> float:
+    return float(lib().ko_f16_to_f32(int(bits)))
+
+
 def num_threads() -> int:
     return int(lib().ko_num_threads())
 
 
-def layernorm(a, b, gamma_bits, beta_bits, eps=1e-5, round_out=False) -> np.ndarray:
+def layernorm(a, b, gamma_bits, beta_bits, eps=1e-5, round_out=False, half=False) -> np.ndarray:
+    """half: the bit patterns (and the rounding of the output) are IEEE half instead of bfloat16."""
     a = _f32(a)
     b = None if b is None else _f32(b)
     rows, d = a.shape
     out = np.empty_like(a)
     g, be = _bits(gamma_bits), _bits(beta_bits)
+    lib().ko_set_half(int(half))
     lib().ko_layernorm(_ptr(a), _ptr(b), rows, d, _ptr(g), _ptr(be), eps, int(round_out), _ptr(out))
+    lib().ko_set_half(0)
     return out
 
 
-def linear(x, w_bits, bias_bits=None) -> np.ndarray:
+def linear(x, w_bits, bias_bits=None, half=False) -> np.ndarray:
     x = _f32(x)
     w = _bits(w_bits)
     rows, n_in = x.shape
     n_out = w.shape[0]
     assert w.shape[1] == n_in
     out = np.empty((rows, n_out), dtype=np.float32)
+    lib().ko_set_half(int(half))
     lib().ko_linear(_ptr(x), rows, n_in, _ptr(w), n_in, _ptr(_bits(bias_bits)), n_out, _ptr(out))
+    lib().ko_set_half(0)
     return out
 
 
@@ -142,13 +161,15 @@ class Oracle:
     """One sequence's Kraken forward state (weights borrowed, KV cache owned)."""
 
     def __init__(self, shape, weights_bits: Dict[str, Optional[np.ndarray]], bf16_store: bool = False,
-                 y_zero: bool = False, final_ln: Optional[bool] = None, gelu_tanh: Optional[bool] = None):
+                 y_zero: bool = False, final_ln: Optional[bool] = None, gelu_tanh: Optional[bool] = None,
+                 half: bool = False):
         self.cfg = KoConfig(
             n_branch=shape.n_branch, n_layer=shape.n_layer, d_model=shape.d_model, n_head=shape.n_head,
             d_ff=shape.d_ff, vocab=shape.vocab, max_pos=shape.max_pos, ln_eps=shape.ln_eps,
             gelu_tanh=int(shape.gelu_tanh if gelu_tanh is None else gelu_tanh),
             final_ln=int(shape.final_ln if final_ln is None else final_ln),
-            bf16_store=int(bf16_store), y_zero=int(y_zero), n_kv_head=int(getattr(shape, "n_kv_head", 0)))
+            bf16_store=int(bf16_store), y_zero=int(y_zero), half=int(half),
+            n_kv_head=int(getattr(shape, "n_kv_head", 0)))
         self._keep = {k: _bits(v) for k, v in weights_bits.items()}
         self.w = KoWeights(**{k: _ptr(self._keep.get(k)) for k in WEIGHT_FIELDS})
         self.shape = shape

@@ -26,6 +26,9 @@
  * (round-to-nearest-even) at those points: both LayerNorm outputs, q/k/v (hence
  * the cache), the attention output, the GELU output, the W_concat input and the
  * final LayerNorm output.  The residual stream and y always stay fp32.
+ * The 16-bit type is bfloat16 unless half = 1 in the configuration (IEEE half, the
+ * precision of the paper's engines, Sec. 4.2): then the weight patterns are read as
+ * half and the store points round to half.
  *
  * Parity status: every step is pinned by the CPU tests (closed forms, brute
  * force, a library composition for the N = 1 reduction, invariants).  The
@@ -47,6 +50,7 @@ typedef struct ko_config {
     int32_t final_ln;    /* 1: LayerNorm between W_concat and the unembedding */
     int32_t bf16_store;  /* 1: round activations to bf16 at the store points */
     int32_t y_zero;      /* test-only: drop the y term (reduces N = 1 to a GPT-2 stack) */
+    int32_t half;        /* 16-bit type of weights and store points: 0 = bfloat16, 1 = IEEE half */
     int32_t n_kv_head;   /* key/value heads per sub-layer: 0 or n_head = multi-head attention; fewer =
                             grouped-query attention, 1 = multi-query (the KV-cache mitigation of Sec. 4.2
                             and the KV-cache appendix): query head h reads key/value head
@@ -87,6 +91,30 @@ static inline float round_bf16(float f) { /* RNE to bf16, returned as fp32 */
 
 float ko_round_bf16(float f) { return round_bf16(f); }
 
+/* IEEE half (1 sign, 5 exponent, 10 fraction bits) widened exactly. */
+static inline float f16_to_f32(uint16_t b) {
+    const int sign = b >> 15, e = (b >> 10) & 31, m = b & 1023;
+    double v;
+    if (e == 0) v = ldexp((double)m, -24);                    /* zero and subnormals: m * 2^-24 */
+    else if (e == 31) v = m ? NAN : INFINITY;
+    else v = ldexp(1.0 + m / 1024.0, e - 15);
+    return (float)(sign ? -v : v);
+}
+
+/* fp32 -> nearest half (ties to even, overflow to infinity), returned as fp32: the compiler's IEEE
+ * half type does the rounding; the pins check it against an independent implementation. */
+static inline float round_f16(float f) { return (float)(_Float16)f; }
+
+float ko_f16_to_f32(uint16_t b) { return f16_to_f32(b); }
+float ko_round_f16(float f) { return round_f16(f); }
+
+/* The 16-bit type in force: set from the configuration at the start of every forward pass, or by
+ * ko_set_half for the single-step wrappers.  (The oracle is driven from one thread.) */
+static int g_half = 0;
+void ko_set_half(int on) { g_half = on != 0; }
+static inline float h16_to_f32(uint16_t b) { return g_half ? f16_to_f32(b) : bf16_to_f32(b); }
+static inline float round_h16(float f) { return g_half ? round_f16(f) : round_bf16(f); }
+
 float ko_gelu(float x, int tanh_form) {
     double v = x;
     if (tanh_form) {
@@ -126,10 +154,10 @@ void ko_layernorm(const float *a, const float *b, int rows, int d, const uint16_
         double rstd = 1.0 / sqrt(var + (double)eps);
         for (int j = 0; j < d; ++j) {
             double v = ((double)(pb ? pa[j] + pb[j] : pa[j]) - mean) * rstd;
-            double g = gamma ? bf16_to_f32(gamma[j]) : 1.0;
-            double be = beta ? bf16_to_f32(beta[j]) : 0.0;
+            double g = gamma ? h16_to_f32(gamma[j]) : 1.0;
+            double be = beta ? h16_to_f32(beta[j]) : 0.0;
             float o = (float)(v * g + be);
-            out[(size_t)r * d + j] = round_out ? round_bf16(o) : o;
+            out[(size_t)r * d + j] = round_out ? round_h16(o) : o;
         }
     }
 }
@@ -145,8 +173,8 @@ void ko_linear(const float *in, int rows, int n_in, const uint16_t *W, int64_t w
 #pragma omp for schedule(static)
         for (int o = 0; o < n_out; ++o) {
             const uint16_t *wp = W + (size_t)o * (size_t)w_stride;
-            for (int i = 0; i < n_in; ++i) wrow[i] = bf16_to_f32(wp[i]);
-            double bo = bias ? (double)bf16_to_f32(bias[o]) : 0.0;
+            for (int i = 0; i < n_in; ++i) wrow[i] = h16_to_f32(wp[i]);
+            double bo = bias ? (double)h16_to_f32(bias[o]) : 0.0;
             for (int t = 0; t < rows; ++t) {
                 const float *x = in + (size_t)t * n_in;
                 double acc = 0.0;
@@ -254,7 +282,7 @@ const float *ko_cache_ptr(const ko_state *s, int layer, int branch, int which, i
 static void maybe_round(float *x, size_t n, int on) {
     if (!on) return;
 #pragma omp parallel for schedule(static)
-    for (size_t i = 0; i < n; ++i) x[i] = round_bf16(x[i]);
+    for (size_t i = 0; i < n; ++i) x[i] = round_h16(x[i]);
 }
 
 /* Evaluate positions pos0 .. pos0 + n - 1 of the sequence whose first pos0 positions
@@ -268,6 +296,7 @@ static int forward(ko_state *s, const int32_t *ids, int n, int pos0, float *logi
                    int logits_from, float *layer_out) {
     const ko_config *c = &s->cfg;
     const ko_weights *w = &s->w;
+    g_half = c->half != 0;
     const int N = c->n_branch, L = c->n_layer, d = c->d_model, H = c->n_head, F = c->d_ff, V = c->vocab;
     const int hd = d / H, rb = c->bf16_store;
     const int Hkv = kv_heads(c), kvd = Hkv * hd, qw = d + 2 * kvd; /* q | k | v row: d + 2 H_kv hd columns */
@@ -296,8 +325,8 @@ static int forward(ko_state *s, const int32_t *ids, int n, int pos0, float *logi
     /* shared embedding: token row + position row */
     for (int t = 0; t < n; ++t)
         for (int j = 0; j < d; ++j)
-            x0[(size_t)t * d + j] = bf16_to_f32(w->wte[(size_t)ids[t] * d + j]) +
-                                    bf16_to_f32(w->wpe[(size_t)(pos0 + t) * d + j]);
+            x0[(size_t)t * d + j] = h16_to_f32(w->wte[(size_t)ids[t] * d + j]) +
+                                    h16_to_f32(w->wpe[(size_t)(pos0 + t) * d + j]);
     for (int b = 0; b < N; ++b) memcpy(x + nd * b, x0, sizeof(float) * nd);
 
     for (int l = 0; l < L; ++l) {
@@ -349,7 +378,7 @@ static int forward(ko_state *s, const int32_t *ids, int n, int pos0, float *logi
             ko_linear(hh, n, d, w->w_up + ln * (size_t)F * d, d, w->b_up ? w->b_up + ln * F : NULL, F, g);
             for (size_t i = 0; i < (size_t)n * F; ++i) {
                 float v = ko_gelu(g[i], c->gelu_tanh);
-                g[i] = rb ? round_bf16(v) : v;
+                g[i] = rb ? round_h16(v) : v;
             }
             ko_linear(g, n, F, w->w_down + ln * (size_t)d * F, F, w->b_down ? w->b_down + ln * d : NULL, d, tmp);
             float *ob = xn + nd * b;
@@ -371,7 +400,7 @@ static int forward(ko_state *s, const int32_t *ids, int n, int pos0, float *logi
                 for (int b = 0; b < N; ++b)
                     for (int j = 0; j < d; ++j) {
                         float v = x[nd * b + (size_t)(logits_from + t) * d + j];
-                        cat[((size_t)t * N + b) * d + j] = rb ? round_bf16(v) : v;
+                        cat[((size_t)t * N + b) * d + j] = rb ? round_h16(v) : v;
                     }
             ko_linear(cat, nr, N * d, w->w_concat, (int64_t)N * d, w->b_concat, d, z);
             if (c->final_ln)

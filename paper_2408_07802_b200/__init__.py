@@ -7,11 +7,14 @@ call raises.
 """
 from __future__ import annotations
 
+import contextlib
 import ctypes as C
 import os
 from typing import Dict, Optional
 
 import torch
+
+from . import build as kbuild
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libkraken.so")
@@ -34,7 +37,7 @@ EXPORTS = (
     "kraken_device_status", "kraken_cur_len", "kraken_profile_enable", "kraken_profile_read", "kraken_reset", "kraken_destroy", "kraken_strerror", "kraken_last_cuda_error",
     "kraken_op_embed", "kraken_op_layernorm", "kraken_op_grouped_gemm", "kraken_op_attention",
     "kraken_op_decode_attention", "kraken_decode_attention_sizes",
-    "kraken_op_decode_attention_static", "kraken_decode_attention_static_capacity",
+    "kraken_op_decode_attention_static", "kraken_decode_attention_static_capacity", "kraken_storage_dtype",
 )
 
 
@@ -74,18 +77,35 @@ class KrakenError(RuntimeError):
         super().__init__(f"{what}: {strerror(status)} ({status})" + (f" [{detail}]" if detail else ""))
 
 
-_lib = None
+_libs: Dict[str, C.CDLL] = {}
+_current_dtype = "bf16"
+TORCH_DTYPE = {"bf16": torch.bfloat16, "f16": torch.float16}
 
 
-def lib() -> C.CDLL:
-    """Loads libkraken.so; raises if it has not been built."""
-    global _lib
-    if _lib is None:
-        if not os.path.exists(LIB_PATH):
+@contextlib.contextmanager
+def storage_dtype(dtype: str):
+    """Within the block, calls that do not name a dtype go to that image ('bf16': libkraken.so, 'f16':
+    libkraken_f16.so, the same ABI with IEEE half as the 16-bit storage type)."""
+    global _current_dtype
+    if dtype not in TORCH_DTYPE:
+        raise ValueError("storage dtype must be 'bf16' or 'f16'")
+    old, _current_dtype = _current_dtype, dtype
+    try:
+        yield
+    finally:
+        _current_dtype = old
+
+
+def lib(dtype: Optional[str] = None) -> C.CDLL:
+    """Loads the library image of the storage dtype; raises if it has not been built."""
+    dtype = dtype or _current_dtype
+    if dtype not in _libs:
+        path = kbuild.lib_path(dtype)
+        if not os.path.exists(path):
             raise RuntimeError(
-                f"{LIB_PATH} is missing: build it with `python -m paper_2408_07802_b200.build` "
+                f"{path} is missing: build it with `python -m paper_2408_07802_b200.build` "
                 "(there is no CPU or PyTorch fallback)")
-        L = C.CDLL(LIB_PATH)
+        L = C.CDLL(path)
         vp, i32, i64 = C.c_void_p, C.c_int32, C.c_int64
         L.kraken_query_sizes.argtypes = [C.POINTER(KrakenConfig), C.POINTER(C.c_size_t), C.POINTER(C.c_size_t)]
         L.kraken_create.argtypes = [C.POINTER(KrakenConfig), C.POINTER(KrakenWeights), vp, C.c_size_t, vp,
@@ -119,8 +139,11 @@ def lib() -> C.CDLL:
                                                         vp, i64, vp]
         L.kraken_decode_attention_static_capacity.argtypes = []
         L.kraken_decode_attention_static_capacity.restype = C.c_size_t
-        _lib = L
-    return _lib
+        L.kraken_storage_dtype.argtypes = []
+        if L.kraken_storage_dtype() != (1 if dtype == "f16" else 0):
+            raise RuntimeError(f"{path} was not built for storage dtype {dtype}")
+        _libs[dtype] = L
+    return _libs[dtype]
 
 
 def strerror(status: int) -> str:
@@ -161,13 +184,15 @@ def query_sizes(cfg: KrakenConfig):
 class KrakenModel:
     """Owns the device buffers (through torch) and a kraken_handle."""
 
-    def __init__(self, cfg: KrakenConfig, weights: Dict[str, Optional[torch.Tensor]], device="cuda:0"):
+    def __init__(self, cfg: KrakenConfig, weights: Dict[str, Optional[torch.Tensor]], device="cuda:0",
+                 dtype: Optional[str] = None):
         self.cfg = cfg
         self.device = torch.device(device)
+        self.dtype = dtype or _current_dtype
         for k in WEIGHT_FIELDS:
             t = weights.get(k)
             if t is not None:
-                assert t.dtype == torch.bfloat16 and t.is_contiguous() and t.device == self.device, k
+                assert t.dtype == TORCH_DTYPE[self.dtype] and t.is_contiguous() and t.device == self.device, k
         self.weights = dict(weights)
         kv_bytes, scratch_bytes = query_sizes(cfg)
         self.kv = torch.empty(kv_bytes, dtype=torch.uint8, device=self.device)
@@ -175,13 +200,13 @@ class KrakenModel:
         w = KrakenWeights(**{k: _ptr(weights.get(k)) for k in WEIGHT_FIELDS})
         h = C.c_void_p()
         with torch.cuda.device(self.device):
-            _check(lib().kraken_create(C.byref(cfg), C.byref(w), self.kv.data_ptr(), kv_bytes,
+            _check(lib(self.dtype).kraken_create(C.byref(cfg), C.byref(w), self.kv.data_ptr(), kv_bytes,
                                        self.scratch.data_ptr(), scratch_bytes, C.byref(h)), "kraken_create")
         self._h = h
 
     def close(self):
         if getattr(self, "_h", None):
-            lib().kraken_destroy(self._h)
+            lib(self.dtype).kraken_destroy(self._h)
             self._h = None
 
     def __del__(self):
@@ -194,14 +219,14 @@ class KrakenModel:
         assert tokens.dtype == torch.int32 and tokens.is_contiguous() and tokens.device == self.device
         if logits is None:
             logits = torch.empty(b, self.cfg.vocab, dtype=torch.float32, device=self.device)
-        _check(lib().kraken_prefill(self._h, tokens.data_ptr(), b, l, logits.data_ptr(), _stream()), "kraken_prefill")
+        _check(lib(self.dtype).kraken_prefill(self._h, tokens.data_ptr(), b, l, logits.data_ptr(), _stream()), "kraken_prefill")
         return logits
 
     def prefill_host(self, tokens: torch.Tensor, logits: torch.Tensor) -> torch.Tensor:
         """tokens / logits: HOST tensors (pinned for full-rate copies); blocks until the logits are there."""
         b, l = tokens.shape
         assert tokens.dtype == torch.int32 and tokens.device.type == "cpu" and logits.device.type == "cpu"
-        _check(lib().kraken_prefill_host(self._h, tokens.data_ptr(), b, l, logits.data_ptr(), _stream()),
+        _check(lib(self.dtype).kraken_prefill_host(self._h, tokens.data_ptr(), b, l, logits.data_ptr(), _stream()),
                "kraken_prefill_host")
         return logits
 
@@ -209,14 +234,14 @@ class KrakenModel:
         b, l = tokens.shape
         assert tokens.dtype == torch.int32 and tokens.is_contiguous() and tokens.device == self.device
         logits = torch.empty(b, l, self.cfg.vocab, dtype=torch.float32, device=self.device)
-        _check(lib().kraken_prefill_all_logits(self._h, tokens.data_ptr(), b, l, logits.data_ptr(), _stream()),
+        _check(lib(self.dtype).kraken_prefill_all_logits(self._h, tokens.data_ptr(), b, l, logits.data_ptr(), _stream()),
                "kraken_prefill_all_logits")
         return logits
 
     def logits_rows(self, rows) -> torch.Tensor:
         rows_t = torch.as_tensor(rows, dtype=torch.int32).contiguous()
         out = torch.empty(rows_t.numel(), self.cfg.vocab, dtype=torch.float32, device=self.device)
-        _check(lib().kraken_logits_rows(self._h, rows_t.data_ptr(), rows_t.numel(), out.data_ptr(), _stream()),
+        _check(lib(self.dtype).kraken_logits_rows(self._h, rows_t.data_ptr(), rows_t.numel(), out.data_ptr(), _stream()),
                "kraken_logits_rows")
         torch.cuda.current_stream().synchronize()  # rows_t (host) must outlive the copy
         return out
@@ -226,14 +251,14 @@ class KrakenModel:
         b = tokens.numel()
         if logits is None:
             logits = torch.empty(b, self.cfg.vocab, dtype=torch.float32, device=self.device)
-        _check(lib().kraken_decode_step(self._h, tokens.data_ptr(), b, logits.data_ptr(), _stream()),
+        _check(lib(self.dtype).kraken_decode_step(self._h, tokens.data_ptr(), b, logits.data_ptr(), _stream()),
                "kraken_decode_step")
         return logits
 
     def decode_step_host(self, tokens: torch.Tensor, logits: torch.Tensor) -> torch.Tensor:
         """tokens [batch] / logits [batch, V]: HOST tensors; blocks until the logits are there."""
         assert tokens.dtype == torch.int32 and tokens.device.type == "cpu" and logits.device.type == "cpu"
-        _check(lib().kraken_decode_step_host(self._h, tokens.data_ptr(), tokens.numel(), logits.data_ptr(),
+        _check(lib(self.dtype).kraken_decode_step_host(self._h, tokens.data_ptr(), tokens.numel(), logits.data_ptr(),
                                              _stream()), "kraken_decode_step_host")
         return logits
 
@@ -242,36 +267,36 @@ class KrakenModel:
         """bf16 view [max_batch, key/value heads, max_pos, head_dim] of the K (0) or V (1) cache of (layer, branch)."""
         p = C.c_void_p()
         st = (C.c_int64 * 4)()
-        _check(lib().kraken_kv_view(self._h, layer, branch, which, C.byref(p), C.byref(st)), "kraken_kv_view")
+        _check(lib(self.dtype).kraken_kv_view(self._h, layer, branch, which, C.byref(p), C.byref(st)), "kraken_kv_view")
         c = self.cfg
         hd = c.d_model // c.n_head
         off = (p.value - self.kv.data_ptr()) // 2
-        flat = self.kv.view(torch.bfloat16)
+        flat = self.kv.view(TORCH_DTYPE[self.dtype])
         return flat.as_strided((c.max_batch, c.n_kv_head or c.n_head, c.max_pos, hd), tuple(st), off)
 
     def device_status(self) -> int:
         f = C.c_uint32(0)
-        _check(lib().kraken_device_status(self._h, C.byref(f)), "kraken_device_status")
+        _check(lib(self.dtype).kraken_device_status(self._h, C.byref(f)), "kraken_device_status")
         return f.value
 
     @property
     def cur_len(self) -> int:
         v = C.c_int32(0)
-        _check(lib().kraken_cur_len(self._h, C.byref(v)), "kraken_cur_len")
+        _check(lib(self.dtype).kraken_cur_len(self._h, C.byref(v)), "kraken_cur_len")
         return v.value
 
     def profile_enable(self, on: bool):
-        _check(lib().kraken_profile_enable(self._h, int(on)), "kraken_profile_enable")
+        _check(lib(self.dtype).kraken_profile_enable(self._h, int(on)), "kraken_profile_enable")
 
     def profile_read(self):
         """({category: device ms}, {category: launches}) since the last read; synchronises."""
         ms = (C.c_double * PROF_COUNT)()
         n = (C.c_int64 * PROF_COUNT)()
-        _check(lib().kraken_profile_read(self._h, C.byref(ms), C.byref(n)), "kraken_profile_read")
+        _check(lib(self.dtype).kraken_profile_read(self._h, C.byref(ms), C.byref(n)), "kraken_profile_read")
         return dict(zip(PROF_CATEGORIES, list(ms))), dict(zip(PROF_CATEGORIES, list(n)))
 
     def reset(self):
-        _check(lib().kraken_reset(self._h), "kraken_reset")
+        _check(lib(self.dtype).kraken_reset(self._h), "kraken_reset")
 
 
 # ------------------------------------------------------------------ single steps
@@ -292,7 +317,7 @@ def op_layernorm(a: torch.Tensor, y: Optional[torch.Tensor], gamma: torch.Tensor
     uint32 word (with it, many-row calls take the persistent kernel)."""
     G, d = gamma.shape
     rows = a.shape[-2]
-    out = torch.empty(G, rows, d, dtype=torch.bfloat16, device=a.device)
+    out = torch.empty(G, rows, d, dtype=gamma.dtype, device=a.device)
     _check(lib().kraken_op_layernorm(a.data_ptr(), 0 if shared_a else rows * d, _ptr(y), gamma.data_ptr(),
                                      _ptr(beta), G, rows, d, eps, out.data_ptr(), _ptr(status), _stream()),
            "kraken_op_layernorm")

@@ -942,6 +942,8 @@ int kraken_profile_read(kraken_handle *h, double *ms, int64_t *launches) {
 
 const char *kraken_last_cuda_error(void) { return last_cuda_error(); }
 
+int kraken_storage_dtype(void) { return KRAKEN_F16 ? 1 : 0; }
+
 const char *kraken_strerror(int status) {
     switch (status) {
         case KRAKEN_OK: return "ok";

@@ -54,9 +54,9 @@ attn_decode_kernel(const DecodeAttnParams p) {
 #pragma unroll
     for (int qh = 0; qh < QH; ++qh) {
         const uint4 u = *reinterpret_cast<const uint4 *>(gq + qh * HD);
-        qf[qh][0] = bf16_lo(u.x) * sl2; qf[qh][1] = bf16_hi(u.x) * sl2; qf[qh][2] = bf16_lo(u.y) * sl2;
-        qf[qh][3] = bf16_hi(u.y) * sl2; qf[qh][4] = bf16_lo(u.z) * sl2; qf[qh][5] = bf16_hi(u.z) * sl2;
-        qf[qh][6] = bf16_lo(u.w) * sl2; qf[qh][7] = bf16_hi(u.w) * sl2;
+        qf[qh][0] = h16_lo(u.x) * sl2; qf[qh][1] = h16_hi(u.x) * sl2; qf[qh][2] = h16_lo(u.y) * sl2;
+        qf[qh][3] = h16_hi(u.y) * sl2; qf[qh][4] = h16_lo(u.z) * sl2; qf[qh][5] = h16_hi(u.z) * sl2;
+        qf[qh][6] = h16_lo(u.w) * sl2; qf[qh][7] = h16_hi(u.w) * sl2;
         m[qh] = -INFINITY;
         l[qh] = 0.f;
 #pragma unroll
@@ -81,14 +81,14 @@ attn_decode_kernel(const DecodeAttnParams p) {
             float mx = m[qh];
 #pragma unroll
             for (int u = 0; u < UNROLL; ++u) {
-                float acc = qf[qh][0] * bf16_lo(kk[u].x);
-                acc = fmaf(qf[qh][1], bf16_hi(kk[u].x), acc);
-                acc = fmaf(qf[qh][2], bf16_lo(kk[u].y), acc);
-                acc = fmaf(qf[qh][3], bf16_hi(kk[u].y), acc);
-                acc = fmaf(qf[qh][4], bf16_lo(kk[u].z), acc);
-                acc = fmaf(qf[qh][5], bf16_hi(kk[u].z), acc);
-                acc = fmaf(qf[qh][6], bf16_lo(kk[u].w), acc);
-                acc = fmaf(qf[qh][7], bf16_hi(kk[u].w), acc);
+                float acc = qf[qh][0] * h16_lo(kk[u].x);
+                acc = fmaf(qf[qh][1], h16_hi(kk[u].x), acc);
+                acc = fmaf(qf[qh][2], h16_lo(kk[u].y), acc);
+                acc = fmaf(qf[qh][3], h16_hi(kk[u].y), acc);
+                acc = fmaf(qf[qh][4], h16_lo(kk[u].z), acc);
+                acc = fmaf(qf[qh][5], h16_hi(kk[u].z), acc);
+                acc = fmaf(qf[qh][6], h16_lo(kk[u].w), acc);
+                acc = fmaf(qf[qh][7], h16_hi(kk[u].w), acc);
 #pragma unroll
                 for (int off = 1; off < GRP; off <<= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, off);
                 s[u] = valid[u] ? acc : -INFINITY;
@@ -103,14 +103,14 @@ attn_decode_kernel(const DecodeAttnParams p) {
                 for (int u = 0; u < UNROLL; ++u) {
                     const float pu = ex2_approx(s[u] - mx);
                     l[qh] += pu;
-                    o[qh][0] = fmaf(pu, bf16_lo(vv[u].x), o[qh][0]);
-                    o[qh][1] = fmaf(pu, bf16_hi(vv[u].x), o[qh][1]);
-                    o[qh][2] = fmaf(pu, bf16_lo(vv[u].y), o[qh][2]);
-                    o[qh][3] = fmaf(pu, bf16_hi(vv[u].y), o[qh][3]);
-                    o[qh][4] = fmaf(pu, bf16_lo(vv[u].z), o[qh][4]);
-                    o[qh][5] = fmaf(pu, bf16_hi(vv[u].z), o[qh][5]);
-                    o[qh][6] = fmaf(pu, bf16_lo(vv[u].w), o[qh][6]);
-                    o[qh][7] = fmaf(pu, bf16_hi(vv[u].w), o[qh][7]);
+                    o[qh][0] = fmaf(pu, h16_lo(vv[u].x), o[qh][0]);
+                    o[qh][1] = fmaf(pu, h16_hi(vv[u].x), o[qh][1]);
+                    o[qh][2] = fmaf(pu, h16_lo(vv[u].y), o[qh][2]);
+                    o[qh][3] = fmaf(pu, h16_hi(vv[u].y), o[qh][3]);
+                    o[qh][4] = fmaf(pu, h16_lo(vv[u].z), o[qh][4]);
+                    o[qh][5] = fmaf(pu, h16_hi(vv[u].z), o[qh][5]);
+                    o[qh][6] = fmaf(pu, h16_lo(vv[u].w), o[qh][6]);
+                    o[qh][7] = fmaf(pu, h16_hi(vv[u].w), o[qh][7]);
                 }
                 m[qh] = mx;
             }
@@ -165,7 +165,7 @@ attn_decode_kernel(const DecodeAttnParams p) {
             const long long stream = ((long long)blockIdx.z * p.n_head + h);
             if (p.splits == 1) {
                 p.out[g * p.out_gstride + (long long)b * d + h * HD + e] =
-                    __bfloat16_as_ushort(__float2bfloat16_rn(ot / lt));
+                    to_h16((ot / lt));
             } else {
                 float *part = p.partials + (stream * p.splits + split) * (HD + 2);
                 part[2 + e] = ot;
@@ -194,7 +194,7 @@ attn_decode_kernel(const DecodeAttnParams p) {
 __device__ __forceinline__ void mma16816_dec(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                              uint32_t b0, uint32_t b1) {
     asm volatile(
-        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+        "mma.sync.aligned.m16n8k16.row.col.f32." KRAKEN_MMA_T "." KRAKEN_MMA_T ".f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
         "{%0, %1, %2, %3};"
         : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
@@ -289,8 +289,8 @@ attn_decode_gqa_kernel(const DecodeAttnParams p) {
             const float p00 = ex2_approx(s[0][2 * hl] - mx), p01 = ex2_approx(s[0][2 * hl + 1] - mx);
             const float p10 = ex2_approx(s[1][2 * hl] - mx), p11 = ex2_approx(s[1][2 * hl + 1] - mx);
             l[hl] = l[hl] * corr + ((p00 + p01) + (p10 + p11));    // this lane's columns; summed over the quad at the end
-            pa[hl] = pack_bf16x2(p00, p01);
-            pa[2 + hl] = pack_bf16x2(p10, p11);
+            pa[hl] = pack_h16x2(p00, p01);
+            pa[2 + hl] = pack_h16x2(p10, p11);
 #pragma unroll
             for (int j = 0; j < HF * 8; ++j) {
                 o[j][2 * hl] *= corr;
@@ -352,7 +352,7 @@ attn_decode_gqa_kernel(const DecodeAttnParams p) {
         const int h = h0 + row;
         const long long stream = ((long long)blockIdx.z * p.n_head + h);
         if (p.splits == 1) {
-            p.out[g * p.out_gstride + (long long)b * d + h * HD + e] = __bfloat16_as_ushort(__float2bfloat16_rn(ot / lt));
+            p.out[g * p.out_gstride + (long long)b * d + h * HD + e] = to_h16((ot / lt));
         } else {
             float *part = p.partials + (stream * p.splits + split) * (HD + 2);
             part[2 + e] = ot;
@@ -384,7 +384,7 @@ __global__ void __launch_bounds__(HD) attn_decode_merge_kernel(const DecodeAttnP
         ot += part[s * (HD + 2) + 2 + e] * c;
     }
     const int d = p.n_head * HD;
-    p.out[g * p.out_gstride + (long long)b * d + h * HD + e] = __bfloat16_as_ushort(__float2bfloat16_rn(ot / lt));
+    p.out[g * p.out_gstride + (long long)b * d + h * HD + e] = to_h16((ot / lt));
 }
 
 template <int HD>

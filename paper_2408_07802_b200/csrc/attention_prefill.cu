@@ -39,7 +39,7 @@ __device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t add
 }
 __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
     asm volatile(
-        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+        "mma.sync.aligned.m16n8k16.row.col.f32." KRAKEN_MMA_T "." KRAKEN_MMA_T ".f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
         "{%0, %1, %2, %3};"
         : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
         : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
@@ -178,10 +178,10 @@ __global__ void __launch_bounds__(128) attn_prefill_kernel(const AttnParams p) {
 #pragma unroll
         for (int kk = 0; kk < ABN / 16; ++kk) {
             uint32_t pf[4];
-            pf[0] = pack_bf16x2(s[2 * kk][0], s[2 * kk][1]);
-            pf[1] = pack_bf16x2(s[2 * kk][2], s[2 * kk][3]);
-            pf[2] = pack_bf16x2(s[2 * kk + 1][0], s[2 * kk + 1][1]);
-            pf[3] = pack_bf16x2(s[2 * kk + 1][2], s[2 * kk + 1][3]);
+            pf[0] = pack_h16x2(s[2 * kk][0], s[2 * kk][1]);
+            pf[1] = pack_h16x2(s[2 * kk][2], s[2 * kk][3]);
+            pf[2] = pack_h16x2(s[2 * kk + 1][0], s[2 * kk + 1][1]);
+            pf[3] = pack_h16x2(s[2 * kk + 1][2], s[2 * kk + 1][3]);
 #pragma unroll
             for (int dp = 0; dp < KS; ++dp) {
                 uint32_t vf[4];
@@ -207,9 +207,9 @@ __global__ void __launch_bounds__(128) attn_prefill_kernel(const AttnParams p) {
     for (int nt = 0; nt < HD / 8; ++nt) {
         const int col = nt * 8 + ((lane & 3) << 1);
         if (r0 < rows_valid)
-            *reinterpret_cast<uint32_t *>(go + (long long)r0 * d + col) = pack_bf16x2(acc[nt][0] * inv0, acc[nt][1] * inv0);
+            *reinterpret_cast<uint32_t *>(go + (long long)r0 * d + col) = pack_h16x2(acc[nt][0] * inv0, acc[nt][1] * inv0);
         if (r1 < rows_valid)
-            *reinterpret_cast<uint32_t *>(go + (long long)r1 * d + col) = pack_bf16x2(acc[nt][2] * inv1, acc[nt][3] * inv1);
+            *reinterpret_cast<uint32_t *>(go + (long long)r1 * d + col) = pack_h16x2(acc[nt][2] * inv1, acc[nt][3] * inv1);
     }
 }
 

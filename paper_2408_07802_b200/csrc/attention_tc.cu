@@ -291,8 +291,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             // head dims below HD: the scores need ceil(head_dim / 16) steps (K is zero beyond head_dim, so
             // whatever Q holds there does not count), the output ceil(head_dim / 16) * 16 columns
             const int qk_steps = (a.head_dim + 15) / 16;
-            constexpr uint32_t idesc_qk = umma_idesc_bf16(TQ, TK);
-            const uint32_t idesc_pv = umma_idesc_bf16(TQ, qk_steps * 16) | (1u << 16);  // B (V) is MN-major
+            constexpr uint32_t idesc_qk = umma_idesc_h16(TQ, TK);
+            const uint32_t idesc_pv = umma_idesc_h16(TQ, qk_steps * 16) | (1u << 16);  // B (V) is MN-major
             auto issue_qk = [&](int w, int st) {
                 const uint32_t q_addr = smem_u32(sQ + w * Cfg::Q_BYTES);
                 const uint32_t k_addr = smem_u32(sK + st * Cfg::KV_BYTES);
@@ -434,8 +434,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                         sum1 += x1;
                         sum2 += x2;
                         sum3 += x3;
-                        pk[i] = pack_bf16x2(x0, x1);
-                        pk[i + 1] = pack_bf16x2(x2, x3);
+                        pk[i] = pack_h16x2(x0, x1);
+                        pk[i + 1] = pack_h16x2(x2, x3);
                     }
                     tmem_st_32x16(s_addr + c * 16, pk);       // overwrites scores already consumed
                 }
@@ -482,10 +482,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                         for (int i = 0; i < 4; ++i) {
                             if (c * 32 + 8 * i >= a.head_dim) break;
                             uint4 u;
-                            u.x = pack_bf16x2(__uint_as_float(r[8 * i + 0]) * inv, __uint_as_float(r[8 * i + 1]) * inv);
-                            u.y = pack_bf16x2(__uint_as_float(r[8 * i + 2]) * inv, __uint_as_float(r[8 * i + 3]) * inv);
-                            u.z = pack_bf16x2(__uint_as_float(r[8 * i + 4]) * inv, __uint_as_float(r[8 * i + 5]) * inv);
-                            u.w = pack_bf16x2(__uint_as_float(r[8 * i + 6]) * inv, __uint_as_float(r[8 * i + 7]) * inv);
+                            u.x = pack_h16x2(__uint_as_float(r[8 * i + 0]) * inv, __uint_as_float(r[8 * i + 1]) * inv);
+                            u.y = pack_h16x2(__uint_as_float(r[8 * i + 2]) * inv, __uint_as_float(r[8 * i + 3]) * inv);
+                            u.z = pack_h16x2(__uint_as_float(r[8 * i + 4]) * inv, __uint_as_float(r[8 * i + 5]) * inv);
+                            u.w = pack_h16x2(__uint_as_float(r[8 * i + 6]) * inv, __uint_as_float(r[8 * i + 7]) * inv);
                             reinterpret_cast<uint4 *>(dst + c * 32)[i] = u;
                         }
                     }

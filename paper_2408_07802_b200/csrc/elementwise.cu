@@ -30,10 +30,10 @@ embed_kernel(const int32_t *__restrict__ ids, int n_tokens, int seqlen, int pos0
     float4 *o = reinterpret_cast<float4 *>(out + (size_t)t * d);
     for (int v = lane; v < d / 8; v += 32) {
         const uint4 a = __ldg(te + v), b = __ldg(pe + v);
-        o[2 * v] = make_float4(bf16_lo(a.x) + bf16_lo(b.x), bf16_hi(a.x) + bf16_hi(b.x),
-                               bf16_lo(a.y) + bf16_lo(b.y), bf16_hi(a.y) + bf16_hi(b.y));
-        o[2 * v + 1] = make_float4(bf16_lo(a.z) + bf16_lo(b.z), bf16_hi(a.z) + bf16_hi(b.z),
-                                   bf16_lo(a.w) + bf16_lo(b.w), bf16_hi(a.w) + bf16_hi(b.w));
+        o[2 * v] = make_float4(h16_lo(a.x) + h16_lo(b.x), h16_hi(a.x) + h16_hi(b.x),
+                               h16_lo(a.y) + h16_lo(b.y), h16_hi(a.y) + h16_hi(b.y));
+        o[2 * v + 1] = make_float4(h16_lo(a.z) + h16_lo(b.z), h16_hi(a.z) + h16_hi(b.z),
+                                   h16_lo(a.w) + h16_lo(b.w), h16_hi(a.w) + h16_hi(b.w));
     }
 }
 
@@ -123,11 +123,11 @@ layernorm_kernel(const float *__restrict__ a, long long a_gstride, const float *
         const uint2 gm = __ldg(pg + v);
         uint2 bt = make_uint2(0u, 0u);
         if (pb) bt = __ldg(pb + v);
-        const float o0 = (t.x - mean) * rstd * bf16_lo(gm.x) + bf16_lo(bt.x);
-        const float o1 = (t.y - mean) * rstd * bf16_hi(gm.x) + bf16_hi(bt.x);
-        const float o2 = (t.z - mean) * rstd * bf16_lo(gm.y) + bf16_lo(bt.y);
-        const float o3 = (t.w - mean) * rstd * bf16_hi(gm.y) + bf16_hi(bt.y);
-        po[v] = make_uint2(pack_bf16x2(o0, o1), pack_bf16x2(o2, o3));
+        const float o0 = (t.x - mean) * rstd * h16_lo(gm.x) + h16_lo(bt.x);
+        const float o1 = (t.y - mean) * rstd * h16_hi(gm.x) + h16_hi(bt.x);
+        const float o2 = (t.z - mean) * rstd * h16_lo(gm.y) + h16_lo(bt.y);
+        const float o3 = (t.w - mean) * rstd * h16_hi(gm.y) + h16_hi(bt.y);
+        po[v] = make_uint2(pack_h16x2(o0, o1), pack_h16x2(o2, o3));
     };
 #pragma unroll
     for (int i = 0; i < LN_CACHE; ++i) {
@@ -246,11 +246,11 @@ layernorm_stream_kernel(const float *__restrict__ a, long long a_gstride, const 
                     const float4 t = cache[i];
                     const uint2 gm = pg[v];
                     const uint2 bt = pb[v];
-                    const float o0 = (t.x - mean) * rstd * bf16_lo(gm.x) + bf16_lo(bt.x);
-                    const float o1 = (t.y - mean) * rstd * bf16_hi(gm.x) + bf16_hi(bt.x);
-                    const float o2 = (t.z - mean) * rstd * bf16_lo(gm.y) + bf16_lo(bt.y);
-                    const float o3 = (t.w - mean) * rstd * bf16_hi(gm.y) + bf16_hi(bt.y);
-                    po[v] = make_uint2(pack_bf16x2(o0, o1), pack_bf16x2(o2, o3));
+                    const float o0 = (t.x - mean) * rstd * h16_lo(gm.x) + h16_lo(bt.x);
+                    const float o1 = (t.y - mean) * rstd * h16_hi(gm.x) + h16_hi(bt.x);
+                    const float o2 = (t.z - mean) * rstd * h16_lo(gm.y) + h16_lo(bt.y);
+                    const float o3 = (t.w - mean) * rstd * h16_hi(gm.y) + h16_hi(bt.y);
+                    po[v] = make_uint2(pack_h16x2(o0, o1), pack_h16x2(o2, o3));
                 }
             }
         }
@@ -277,7 +277,7 @@ gather_concat_kernel(const float *__restrict__ x, long long x_gstride, int group
     uint2 *dst = reinterpret_cast<uint2 *>(out + ((size_t)r * groups + g) * d);
     for (int v = lane; v < d / 4; v += 32) {
         const float4 t = src[v];
-        dst[v] = make_uint2(pack_bf16x2(t.x, t.y), pack_bf16x2(t.z, t.w));
+        dst[v] = make_uint2(pack_h16x2(t.x, t.y), pack_h16x2(t.z, t.w));
     }
 }
 
@@ -303,7 +303,7 @@ sum_groups_kernel(const float *__restrict__ x, long long gstride, int groups, lo
 __global__ void f32_to_bf16_kernel(const float *__restrict__ in, uint16_t *__restrict__ out, long long n) {
     long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     const long long stride = (long long)gridDim.x * blockDim.x;
-    for (; i < n; i += stride) out[i] = __bfloat16_as_ushort(__float2bfloat16_rn(in[i]));
+    for (; i < n; i += stride) out[i] = to_h16((in[i]));
 }
 
 int done() { return cudaGetLastError() == cudaSuccess ? KRAKEN_OK : KRAKEN_ECUDA; }

@@ -69,25 +69,25 @@ __device__ __forceinline__ void store_bf16_chunk(uint16_t *dst, const float (&v)
     if (ncols == 32 && (reinterpret_cast<uintptr_t>(dst) & 31u) == 0) {
 #pragma unroll
         for (int i = 0; i < 2; ++i)
-            st_global_32B(dst + 16 * i, pack_bf16x2(v[16 * i + 0], v[16 * i + 1]), pack_bf16x2(v[16 * i + 2], v[16 * i + 3]),
-                          pack_bf16x2(v[16 * i + 4], v[16 * i + 5]), pack_bf16x2(v[16 * i + 6], v[16 * i + 7]),
-                          pack_bf16x2(v[16 * i + 8], v[16 * i + 9]), pack_bf16x2(v[16 * i + 10], v[16 * i + 11]),
-                          pack_bf16x2(v[16 * i + 12], v[16 * i + 13]), pack_bf16x2(v[16 * i + 14], v[16 * i + 15]));
+            st_global_32B(dst + 16 * i, pack_h16x2(v[16 * i + 0], v[16 * i + 1]), pack_h16x2(v[16 * i + 2], v[16 * i + 3]),
+                          pack_h16x2(v[16 * i + 4], v[16 * i + 5]), pack_h16x2(v[16 * i + 6], v[16 * i + 7]),
+                          pack_h16x2(v[16 * i + 8], v[16 * i + 9]), pack_h16x2(v[16 * i + 10], v[16 * i + 11]),
+                          pack_h16x2(v[16 * i + 12], v[16 * i + 13]), pack_h16x2(v[16 * i + 14], v[16 * i + 15]));
     } else if (ncols == 32 && (reinterpret_cast<uintptr_t>(dst) & 15u) == 0) {
         uint4 *d4 = reinterpret_cast<uint4 *>(dst);
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             uint4 u;
-            u.x = pack_bf16x2(v[8 * i + 0], v[8 * i + 1]);
-            u.y = pack_bf16x2(v[8 * i + 2], v[8 * i + 3]);
-            u.z = pack_bf16x2(v[8 * i + 4], v[8 * i + 5]);
-            u.w = pack_bf16x2(v[8 * i + 6], v[8 * i + 7]);
+            u.x = pack_h16x2(v[8 * i + 0], v[8 * i + 1]);
+            u.y = pack_h16x2(v[8 * i + 2], v[8 * i + 3]);
+            u.z = pack_h16x2(v[8 * i + 4], v[8 * i + 5]);
+            u.w = pack_h16x2(v[8 * i + 6], v[8 * i + 7]);
             d4[i] = u;
         }
     } else {
 #pragma unroll
         for (int i = 0; i < 32; ++i)
-            if (i < ncols) dst[i] = __bfloat16_as_ushort(__float2bfloat16_rn(v[i]));
+            if (i < ncols) dst[i] = to_h16((v[i]));
     }
 }
 
@@ -141,19 +141,19 @@ __device__ __forceinline__ void add_bias_chunk(const uint16_t *bias, float (&v)[
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             uint4 u = __ldg(b4 + i);
-            v[8 * i + 0] += bf16_lo(u.x);
-            v[8 * i + 1] += bf16_hi(u.x);
-            v[8 * i + 2] += bf16_lo(u.y);
-            v[8 * i + 3] += bf16_hi(u.y);
-            v[8 * i + 4] += bf16_lo(u.z);
-            v[8 * i + 5] += bf16_hi(u.z);
-            v[8 * i + 6] += bf16_lo(u.w);
-            v[8 * i + 7] += bf16_hi(u.w);
+            v[8 * i + 0] += h16_lo(u.x);
+            v[8 * i + 1] += h16_hi(u.x);
+            v[8 * i + 2] += h16_lo(u.y);
+            v[8 * i + 3] += h16_hi(u.y);
+            v[8 * i + 4] += h16_lo(u.z);
+            v[8 * i + 5] += h16_hi(u.z);
+            v[8 * i + 6] += h16_lo(u.w);
+            v[8 * i + 7] += h16_hi(u.w);
         }
     } else {
 #pragma unroll
         for (int i = 0; i < 32; ++i)
-            if (i < ncols) v[i] += __uint_as_float(static_cast<uint32_t>(bias[i]) << 16);
+            if (i < ncols) v[i] += from_h16(bias[i]);
     }
 }
 
@@ -228,10 +228,10 @@ __device__ __forceinline__ void epilogue_chunk(const EpiParams &p, int g, int ro
                               (((long long)b * p.n_kv_head + head) * p.max_pos + pos) * p.head_dim + e0;
                     }
                     uint4 u;
-                    u.x = pack_bf16x2(v[8 * i + 0], v[8 * i + 1]);
-                    u.y = pack_bf16x2(v[8 * i + 2], v[8 * i + 3]);
-                    u.z = pack_bf16x2(v[8 * i + 4], v[8 * i + 5]);
-                    u.w = pack_bf16x2(v[8 * i + 6], v[8 * i + 7]);
+                    u.x = pack_h16x2(v[8 * i + 0], v[8 * i + 1]);
+                    u.y = pack_h16x2(v[8 * i + 2], v[8 * i + 3]);
+                    u.z = pack_h16x2(v[8 * i + 4], v[8 * i + 5]);
+                    u.w = pack_h16x2(v[8 * i + 6], v[8 * i + 7]);
                     *reinterpret_cast<uint4 *>(dst) = u;
                 }
             }

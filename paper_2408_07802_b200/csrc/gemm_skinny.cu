@@ -22,28 +22,26 @@ constexpr int SK_UNROLL = 8;
 __device__ __forceinline__ void mma16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                          uint32_t b0, uint32_t b1) {
     asm volatile(
-        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+        "mma.sync.aligned.m16n8k16.row.col.f32." KRAKEN_MMA_T "." KRAKEN_MMA_T ".f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
         "{%0, %1, %2, %3};"
         : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-__device__ __forceinline__ float bf(uint16_t v) { return __uint_as_float(static_cast<uint32_t>(v) << 16); }
-__device__ __forceinline__ uint16_t to_bf(float v) { return __bfloat16_as_ushort(__float2bfloat16_rn(v)); }
 
 // Epilogue of one output element (same semantics as the tile epilogue of the tensor-core GEMM,
 // except KRAKEN_EPI_RESID_SUM, which this kernel does not take: callers sum small tensors elsewhere).
 __device__ __forceinline__ void epilogue_elem(const EpiParams &p, int g, int row, int col, float acc) {
-    if (p.bias) acc += bf(p.bias[g * p.bias_gstride + col]);
+    if (p.bias) acc += from_h16(p.bias[g * p.bias_gstride + col]);
     switch (p.kind) {
         case KRAKEN_EPI_F32:
             p.out_f32[g * p.out_f32_gstride + (long long)row * p.ld_out_f32 + col] = acc;
             break;
         case KRAKEN_EPI_BF16:
-            p.out_bf16[g * p.out_bf16_gstride + (long long)row * p.ld_out_bf16 + col] = to_bf(acc);
+            p.out_bf16[g * p.out_bf16_gstride + (long long)row * p.ld_out_bf16 + col] = to_h16(acc);
             break;
         case KRAKEN_EPI_GELU_BF16:
-            p.out_bf16[g * p.out_bf16_gstride + (long long)row * p.ld_out_bf16 + col] = to_bf(gelu_f(acc, p.gelu_tanh));
+            p.out_bf16[g * p.out_bf16_gstride + (long long)row * p.ld_out_bf16 + col] = to_h16(gelu_f(acc, p.gelu_tanh));
             break;
         case KRAKEN_EPI_RESID_F32:
             p.out_f32[g * p.out_f32_gstride + (long long)row * p.ld_out_f32 + col] =
@@ -52,14 +50,14 @@ __device__ __forceinline__ void epilogue_elem(const EpiParams &p, int g, int row
         case KRAKEN_EPI_QKV: {
             const int d = p.d_model;
             if (col < d) {
-                p.out_bf16[g * p.out_bf16_gstride + (long long)row * p.ld_out_bf16 + col] = to_bf(acc);
+                p.out_bf16[g * p.out_bf16_gstride + (long long)row * p.ld_out_bf16 + col] = to_h16(acc);
             } else {
                 const int kvd = p.n_kv_head * p.head_dim;
                 const int which = col >= d + kvd, c = col - d - which * kvd;
                 const int head = c / p.head_dim, e = c % p.head_dim;
                 const int b = row / p.seqlen, pos = (p.pos0_dev ? *p.pos0_dev : p.pos0) + row % p.seqlen;
                 uint16_t *base = (which ? p.v_cache : p.k_cache) + g * p.cache_gstride;
-                base[(((long long)b * p.n_kv_head + head) * p.max_pos + pos) * p.head_dim + e] = to_bf(acc);
+                base[(((long long)b * p.n_kv_head + head) * p.max_pos + pos) * p.head_dim + e] = to_h16(acc);
             }
             break;
         }

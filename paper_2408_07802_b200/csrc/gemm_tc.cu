@@ -144,7 +144,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         __syncwarp();
     } else if (warp == 1) {
         if (lane == 0) {
-            constexpr uint32_t idesc = umma_idesc_bf16(BM, BN);
+            constexpr uint32_t idesc = umma_idesc_h16(BM, BN);
             int stage = 0;
             uint32_t phase = 0;
             int acc = 0;
@@ -353,7 +353,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         __syncwarp();
     } else if (warp == 1) {
         if (lane == 0 && rank == 0) {
-            constexpr uint32_t idesc = umma_idesc_bf16(2 * BM, BN2);
+            constexpr uint32_t idesc = umma_idesc_h16(2 * BM, BN2);
             int stage = 0;
             uint32_t phase = 0;
             int acc = 0;

@@ -10,8 +10,6 @@ namespace kr {
 
 namespace {
 
-__device__ __forceinline__ float bf(uint16_t v) { return __uint_as_float(static_cast<uint32_t>(v) << 16); }
-__device__ __forceinline__ uint16_t to_bf(float v) { return __bfloat16_as_ushort(__float2bfloat16_rn(v)); }
 
 __global__ void gemm_naive_kernel(GemmOperands op, GemmShape s, EpiParams p) {
     const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
@@ -22,18 +20,18 @@ __global__ void gemm_naive_kernel(GemmOperands op, GemmShape s, EpiParams p) {
         const uint16_t *a = static_cast<const uint16_t *>(op.a) + g * op.a_gstride + (long long)row * op.lda;
         const uint16_t *w = static_cast<const uint16_t *>(op.w) + g * op.w_gstride + (long long)col * op.ldw;
         float acc = 0.f;
-        for (int k = 0; k < s.k; ++k) acc = fmaf(bf(a[k]), bf(w[k]), acc);
-        if (p.bias) acc += bf(p.bias[g * p.bias_gstride + col]);
+        for (int k = 0; k < s.k; ++k) acc = fmaf(from_h16(a[k]), from_h16(w[k]), acc);
+        if (p.bias) acc += from_h16(p.bias[g * p.bias_gstride + col]);
         switch (p.kind) {
             case KRAKEN_EPI_F32:
                 p.out_f32[g * p.out_f32_gstride + (long long)row * p.ld_out_f32 + col] = acc;
                 break;
             case KRAKEN_EPI_BF16:
-                p.out_bf16[g * p.out_bf16_gstride + (long long)row * p.ld_out_bf16 + col] = to_bf(acc);
+                p.out_bf16[g * p.out_bf16_gstride + (long long)row * p.ld_out_bf16 + col] = to_h16(acc);
                 break;
             case KRAKEN_EPI_GELU_BF16:
                 p.out_bf16[g * p.out_bf16_gstride + (long long)row * p.ld_out_bf16 + col] =
-                    to_bf(gelu_f(acc, p.gelu_tanh));
+                    to_h16(gelu_f(acc, p.gelu_tanh));
                 break;
             case KRAKEN_EPI_RESID_F32:
             case KRAKEN_EPI_RESID_SUM: {
@@ -46,14 +44,14 @@ __global__ void gemm_naive_kernel(GemmOperands op, GemmShape s, EpiParams p) {
             case KRAKEN_EPI_QKV: {
                 const int d = p.d_model;
                 if (col < d) {
-                    p.out_bf16[g * p.out_bf16_gstride + (long long)row * p.ld_out_bf16 + col] = to_bf(acc);
+                    p.out_bf16[g * p.out_bf16_gstride + (long long)row * p.ld_out_bf16 + col] = to_h16(acc);
                 } else {
                     const int kvd = p.n_kv_head * p.head_dim;
                     const int which = col >= d + kvd, c = col - d - which * kvd;
                     const int head = c / p.head_dim, e = c % p.head_dim;
                     const int b = row / p.seqlen, pos = p.pos0 + row % p.seqlen;
                     uint16_t *base = (which ? p.v_cache : p.k_cache) + g * p.cache_gstride;
-                    base[(((long long)b * p.n_kv_head + head) * p.max_pos + pos) * p.head_dim + e] = to_bf(acc);
+                    base[(((long long)b * p.n_kv_head + head) * p.max_pos + pos) * p.head_dim + e] = to_h16(acc);
                 }
                 break;
             }
@@ -78,22 +76,22 @@ __global__ void attention_naive_kernel(AttnParams p) {
     const uint16_t *kc = p.k_cache + g * p.cache_gstride + b * p.cache_bstride + (long long)hk * p.max_pos * hd;
     const uint16_t *vc = p.v_cache + g * p.cache_gstride + b * p.cache_bstride + (long long)hk * p.max_pos * hd;
     float qv[4], o[4] = {0.f, 0.f, 0.f, 0.f};
-    for (int i = 0; i < per; ++i) qv[i] = bf(q[lane * per + i]);
+    for (int i = 0; i < per; ++i) qv[i] = from_h16(q[lane * per + i]);
     const float scale = rsqrtf(static_cast<float>(hd));
     float m = -INFINITY, l = 0.f;
     for (int j = 0; j <= p.pos0 + t; ++j) {
         float s = 0.f;
-        for (int i = 0; i < per; ++i) s += qv[i] * bf(kc[(long long)j * hd + lane * per + i]);
+        for (int i = 0; i < per; ++i) s += qv[i] * from_h16(kc[(long long)j * hd + lane * per + i]);
         for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, off);
         s *= scale;
         const float mn = fmaxf(m, s);
         const float corr = __expf(m - mn), e = __expf(s - mn);
         l = l * corr + e;
-        for (int i = 0; i < per; ++i) o[i] = o[i] * corr + e * bf(vc[(long long)j * hd + lane * per + i]);
+        for (int i = 0; i < per; ++i) o[i] = o[i] * corr + e * from_h16(vc[(long long)j * hd + lane * per + i]);
         m = mn;
     }
     uint16_t *out = p.out + g * p.out_gstride + ((long long)b * p.seqlen + t) * d + h * hd;
-    for (int i = 0; i < per; ++i) out[lane * per + i] = to_bf(o[i] / l);
+    for (int i = 0; i < per; ++i) out[lane * per + i] = to_h16(o[i] / l);
 }
 
 }  // namespace

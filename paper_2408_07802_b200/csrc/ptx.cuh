@@ -3,6 +3,16 @@
 #pragma once
 #include <cuda.h>
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
+
+#ifndef KRAKEN_F16
+#define KRAKEN_F16 0
+#endif
+#if KRAKEN_F16
+#define KRAKEN_MMA_T "f16"
+#else
+#define KRAKEN_MMA_T "bf16"
+#endif
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -150,9 +160,11 @@ __device__ __forceinline__ uint64_t umma_desc_sw128_kmajor(uint32_t smem_addr) {
     return d;
 }
 
-// Instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M x N tile.
-__host__ __device__ constexpr uint32_t umma_idesc_bf16(int m, int n) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(n >> 3) << 17) |
+// Instruction descriptor: h16 x h16 -> fp32, both operands K-major, M x N tile (operand format field:
+// 0 = half, 1 = bfloat16).
+__host__ __device__ constexpr uint32_t umma_idesc_h16(int m, int n) {
+    constexpr uint32_t fmt = KRAKEN_F16 ? 0u : 1u;
+    return (1u << 4) | (fmt << 7) | (fmt << 10) | (static_cast<uint32_t>(n >> 3) << 17) |
            (static_cast<uint32_t>(m >> 4) << 24);
 }
 
@@ -344,12 +356,27 @@ __device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
 }
 __device__ __forceinline__ uint64_t splat2(float v) { return pk2(v, v); }
 
-__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+// The 16-bit storage type of weights, activations and the KV cache ("h16") is fixed when the library is
+// built: bfloat16 (the default build) or IEEE half (KRAKEN_F16 = 1, the precision of the paper's engines,
+// Sec. 4.2).  Everything else - fp32 accumulation, fp32 residual stream, layouts - is the same.
+#if KRAKEN_F16
+__device__ __forceinline__ uint32_t pack_h16x2(float lo, float hi) {
+    __half2 v = __floats2half2_rn(lo, hi);
+    return *reinterpret_cast<uint32_t *>(&v);
+}
+__device__ __forceinline__ float h16_lo(uint32_t v) { return __half2float(__ushort_as_half(static_cast<unsigned short>(v & 0xFFFFu))); }
+__device__ __forceinline__ float h16_hi(uint32_t v) { return __half2float(__ushort_as_half(static_cast<unsigned short>(v >> 16))); }
+__device__ __forceinline__ uint16_t to_h16(float v) { return __half_as_ushort(__float2half_rn(v)); }
+__device__ __forceinline__ float from_h16(uint16_t v) { return __half2float(__ushort_as_half(v)); }
+#else
+__device__ __forceinline__ uint32_t pack_h16x2(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t *>(&v);
 }
-
-__device__ __forceinline__ float bf16_lo(uint32_t v) { return __uint_as_float(v << 16); }
-__device__ __forceinline__ float bf16_hi(uint32_t v) { return __uint_as_float(v & 0xFFFF0000u); }
+__device__ __forceinline__ float h16_lo(uint32_t v) { return __uint_as_float(v << 16); }
+__device__ __forceinline__ float h16_hi(uint32_t v) { return __uint_as_float(v & 0xFFFF0000u); }
+__device__ __forceinline__ uint16_t to_h16(float v) { return __bfloat16_as_ushort(__float2bfloat16_rn(v)); }
+__device__ __forceinline__ float from_h16(uint16_t v) { return __uint_as_float(static_cast<uint32_t>(v) << 16); }
+#endif
 
 }  // namespace kr

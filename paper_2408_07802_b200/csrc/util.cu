@@ -7,6 +7,10 @@
 
 #include "internal.h"
 
+#ifndef KRAKEN_F16
+#define KRAKEN_F16 0
+#endif
+
 namespace kr {
 
 namespace {
@@ -40,7 +44,7 @@ int encode(CUtensorMap *map, const void *base, int rank, const uint64_t *dims, c
         estride[i] = 1;
     }
     for (int i = 0; i + 1 < rank; ++i) gstride[i] = strides_elems[i] * 2;  // bytes
-    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, rank, const_cast<void *>(base), gdim, gstride, bdim,
+    CUresult r = fn(map, (KRAKEN_F16 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16), rank, const_cast<void *>(base), gdim, gstride, bdim,
                     estride, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                     CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS ? KRAKEN_OK : KRAKEN_ECUDA;

@@ -26,6 +26,12 @@ def test_exports_match_header(L):
     assert declared == set(kr.EXPORTS)
     for name in declared:
         assert hasattr(L, name), name
+    # the IEEE-half image has the same ABI and says which one it is
+    kbuild.build(dtype="f16")
+    L16 = kr.lib("f16")
+    for name in declared:
+        assert hasattr(L16, name), name
+    assert L.kraken_storage_dtype() == 0 and L16.kraken_storage_dtype() == 1
 
 
 def test_struct_sizes_match_header():

@@ -267,6 +267,64 @@ def test_decode_branch_chains_any_branch_count(n_branch, one_chain, monkeypatch)
     m.close()
 
 
+# ------------------------------------------------------------------ IEEE half as the 16-bit storage type
+
+@pytest.mark.parametrize("name", ["C0", "K0-104", "C0-gqa"])
+def test_half_storage_image_all_positions_cache_and_decode(name):
+    """libkraken_f16.so (weights, activations and KV cache in IEEE half, the precision of the paper's engines,
+    Sec. 4.2) against the oracle in half mode: every position, the cache, teacher-forced decode steps."""
+    s = ki.CONFIGS[name]
+    w = ki.make_weights(s, seed=0, device=DEV, dtype="f16")
+    m = kr.KrakenModel(kr.make_config(s), w, DEV, dtype="f16")
+    wb = host_bits(w)
+    steps = 4
+    l0 = min(s.seqlen, s.max_pos - steps)
+    tok = ki.uniform_tokens(6, s.vocab, s.batch, l0 + steps, DEV)
+    first = tok[:, :l0].contiguous()
+    got_all = m.prefill_all_logits(first).cpu().numpy()
+    orcs = []
+    for b in range(s.batch):
+        ids = tok[b, :l0].cpu().numpy()
+        ref32, _ = oracle.Oracle(s, wb, half=True).prefill(ids)
+        orc = oracle.Oracle(s, wb, bf16_store=True, half=True)
+        refh, _ = orc.prefill(ids)
+        check_parity(got_all[b], ref32, refh, f"{name} half storage, seq {b}, all positions")
+        for layer in range(s.n_layer):
+            for n in (0, s.n_branch - 1):
+                for which in (0, 1):
+                    g = m.kv_view(layer, n, which)[b, :, :l0].float().cpu().numpy()
+                    check_cache(g, orc.cache(layer, n, which), False, (name, b, layer, n, which))
+        o2 = oracle.Oracle(s, wb, half=True)
+        o2.prefill(ids)
+        orcs.append(o2)
+    for t in range(steps):
+        got = m.decode_step(tok[:, l0 + t].contiguous()).cpu().numpy()
+        for b in range(s.batch):
+            ref = orcs[b].decode_step(int(tok[b, l0 + t]))
+            rel, mx = logits_metrics(got[b], ref)
+            assert rel <= REL_L2_MAX and mx <= MAX_ABS_MAX, (name, t, b, rel, mx)
+    assert m.device_status() == 0
+    m.close()
+
+
+def test_half_storage_engine_shape_prefix_parity():
+    """The paper's 1.3B 4-way engine shape in its own precision (IEEE half), full 2048-token context."""
+    s = ki.CONFIGS["K1.3B-4"]
+    w = ki.make_weights(s, seed=0, device=DEV, dtype="f16")
+    m = kr.KrakenModel(kr.make_config(s), w, DEV, dtype="f16")
+    wb = host_bits(w)
+    tok = ki.uniform_tokens(1, s.vocab, s.batch, s.seqlen, DEV)
+    last = m.prefill(tok)
+    assert torch.isfinite(last).all() and m.device_status() == 0
+    prefix = 32
+    got = m.logits_rows(list(range(prefix))).cpu().numpy()
+    ids = tok[0, :prefix].cpu().numpy()
+    ref32, _ = oracle.Oracle(s, wb, half=True).prefill(ids)
+    refh, _ = oracle.Oracle(s, wb, bf16_store=True, half=True).prefill(ids)
+    check_parity(got, ref32, refh, "K1.3B-4 half storage, first 32 positions of the full-size run")
+    m.close()
+
+
 # ------------------------------------------------------------------ C1 .. C3 at full size
 
 def test_c1_full_parity():

@@ -398,3 +398,58 @@ def test_skinny_gemm_unaligned_output_rows():
     kr.op_grouped_gemm(args)
     ref = oracle.linear(a[0].float().cpu().numpy(), bits(w[0]))
     assert np.abs(out.cpu().numpy() - ref).max() < 2e-4
+
+
+# ------------------------------------------------------------------ IEEE half image, single steps
+
+def test_half_image_gemm_layernorm_and_attention():
+    """The single steps of libkraken_f16.so on half tensors against the oracle's steps in half mode."""
+    with kr.storage_dtype("f16"):
+        G, M, K, Nout = 2, 300, 256, 384
+        a = ki.normal_f16(31, 0, (G, M, K), 1.0, DEV)
+        w = ki.normal_f16(31, 1, (G, Nout, K), 0.05, DEV)
+        bias = ki.normal_f16(31, 2, (G, Nout), 0.1, DEV)
+        out = torch.empty(G, M, Nout, dtype=torch.float32, device=DEV)
+        args = kr.GemmArgs()
+        args.a, args.a_gstride, args.lda = a.data_ptr(), M * K, K
+        args.w, args.w_gstride, args.ldw = w.data_ptr(), Nout * K, K
+        args.bias, args.bias_gstride = bias.data_ptr(), Nout
+        args.groups, args.m, args.n_out, args.k = G, M, Nout, K
+        args.epilogue = kr.EPI_F32
+        args.out_f32, args.out_f32_gstride, args.ld_out_f32 = out.data_ptr(), M * Nout, Nout
+        kr.op_grouped_gemm(args)
+        torch.cuda.synchronize()
+        for g in range(G):
+            ref = oracle.linear(a[g].float().cpu().numpy(), bits(w[g]), bits(bias[g]), half=True)
+            assert np.abs(out[g].cpu().numpy() - ref).max() < 2e-4 * max(1.0, np.abs(ref).max())
+        # LayerNorm with half gamma / beta and half output
+        x = (ki.normal_bf16(32, 0, (G, 40, 256), 1.0, DEV).float() * 1.5 + 0.2).contiguous()
+        gamma = (1 + ki.normal_bf16(32, 1, (G, 256), 0.3, DEV).float()).to(torch.float16)
+        beta = ki.normal_f16(32, 2, (G, 256), 0.3, DEV)
+        ln = kr.op_layernorm(x, None, gamma, beta)
+        assert ln.dtype == torch.float16
+        for g in range(G):
+            ref = oracle.layernorm(x[g].cpu().numpy(), None, bits(gamma[g]), bits(beta[g]), round_out=True, half=True)
+            got = ln[g].float().cpu().numpy()
+            assert (np.abs(got - ref) <= 2.0 ** -10 * np.maximum(np.abs(ref), 0.05)).all()
+        # attention on half q, k, v
+        B, H, hd, P, seqlen = 2, 2, 64, 256, 200
+        q = ki.normal_f16(33, 0, (G, B * seqlen, H * hd), 1.0, DEV)
+        kc = ki.normal_f16(33, 1, (G, B, H, P, hd), 1.0, DEV)
+        vc = ki.normal_f16(33, 2, (G, B, H, P, hd), 1.0, DEV)
+        o = kr.op_attention(q, kc, vc, B, seqlen, 0, H).float().cpu().numpy()
+        qn, kn, vn = q.float().cpu().numpy(), kc.float().cpu().numpy(), vc.float().cpu().numpy()
+        for g in range(G):
+            for b in range(B):
+                for h in range(H):
+                    ref = oracle.attention_head(qn[g, b * seqlen:(b + 1) * seqlen, h * hd:(h + 1) * hd],
+                                                kn[g, b, h, :seqlen], vn[g, b, h, :seqlen])
+                    assert np.abs(o[g, b * seqlen:(b + 1) * seqlen, h * hd:(h + 1) * hd] - ref).max() < 1e-2
+        od = kr.op_decode_attention(q[:, :B].contiguous(), kc, vc, 150).float().cpu().numpy()
+        for g in range(G):
+            for b in range(B):
+                for h in range(H):
+                    ref = oracle.attention_head(qn[g, b:b + 1, h * hd:(h + 1) * hd], kn[g, b, h, :150], vn[g, b, h, :150],
+                                                q_pos0=149)
+                    assert np.abs(od[g, b, h * hd:(h + 1) * hd] - ref[0]).max() < 1e-2
+

@@ -532,3 +532,47 @@ def test_kv_heads_equal_to_heads_is_plain_multi_head():
     with pytest.raises(ValueError):
         oracle.Oracle(small_shape(n_kv_head=3), wbits(w))       # 2 heads cannot share 3 key/value heads
 
+
+# ------------------------------------------------------------------ IEEE half as the 16-bit type
+
+def test_half_rounding_and_widening_against_numpy():
+    """The oracle's half conversions against numpy's float16 (an independent implementation): every bit
+    pattern widens to the same value; rounding agrees on ties, subnormals, overflow and a random sweep."""
+    pats = np.arange(65536, dtype=np.uint16)
+    want = pats.view(np.float16).astype(np.float32)
+    got = np.array([oracle.f16_to_f32(int(b)) for b in pats[::7]], dtype=np.float32)
+    w = want[::7]
+    assert np.array_equal(np.isnan(got), np.isnan(w))
+    assert np.array_equal(got[~np.isnan(w)], w[~np.isnan(w)])
+    cases = [1.0 + 2.0 ** -11, 1.0 + 3 * 2.0 ** -11, 2049.0, 2051.0, 65504.0, 65519.9, 65520.0, 70000.0, -70000.0,
+             6e-8, 5.96e-8, 2.98e-8, 2.9e-8, 1e-7, -1e-7, 6.1e-5, 0.1, -0.3333, 0.0]
+    rng = np.random.default_rng(0)
+    cases += list(rng.normal(0, 1, 2000).astype(np.float32)) + list(rng.normal(0, 1e-5, 500).astype(np.float32))
+    for x in cases:
+        with np.errstate(over="ignore"):
+            ref = float(np.float32(x).astype(np.float16).astype(np.float32))
+        assert oracle.round_f16(float(np.float32(x))) == ref, x
+
+
+def test_half_mode_matches_library_composition_and_rounds_stores_to_half():
+    shape = small_shape()
+    w = {k: (None if v is None else v.to(torch.float16)) for k, v in rand_weights(shape).items()}
+    ids = ki.uniform_tokens(7, shape.vocab, 1, shape.seqlen)[0].numpy()
+    ref, _ = torch_kraken(shape, w, ids, final_ln=True)
+    got, _ = oracle.Oracle(shape, wbits(w), half=True).prefill(ids)
+    assert np.max(np.abs(got - ref)) < 2e-5 * max(1.0, np.max(np.abs(ref)))
+    # the same patterns read as bfloat16 are a different model
+    other, _ = oracle.Oracle(shape, wbits(w), half=False).prefill(ids)
+    assert np.max(np.abs(other - ref)) > 1e-2
+    # store points round to half: LayerNorm output
+    a = np.random.default_rng(1).normal(0, 1, (5, 32)).astype(np.float32)
+    g = bits(torch.ones(32, dtype=torch.float16))
+    plain = oracle.layernorm(a, None, g, None, half=True)
+    rounded = oracle.layernorm(a, None, g, None, round_out=True, half=True)
+    assert np.array_equal(rounded, plain.astype(np.float16).astype(np.float32))
+    # and the cache of a store-rounding run holds values exactly representable in half
+    orc = oracle.Oracle(shape, wbits(w), bf16_store=True, half=True)
+    orc.prefill(ids)
+    k = orc.cache(0, 0, 0)
+    assert np.array_equal(k, k.astype(np.float16).astype(np.float32))
+
