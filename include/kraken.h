@@ -219,8 +219,9 @@ typedef struct kraken_gemm_args {
     void *k_cache, *v_cache; int64_t cache_gstride;           /* QKV only: bases of this layer's K and V      */
     int32_t seqlen, pos0, n_head, head_dim, max_pos;          /* QKV only                                     */
     int32_t gelu_tanh;
-    int32_t n_tile;                                           /* N tile: 0 = automatic, 64 / 128 / 256, 512 = CTA
-                                                                 pairs on 256 x 256 tiles, or 8 = the
+    int32_t n_tile;                                           /* N tile: 0 = automatic; 32, 64, ... 256 (multiples of
+                                                                 32) = one CTA per 128 x n_tile tile; 512 = CTA
+                                                                 pairs on 256 x 256 tiles; 8 = the
                                                                  weight-streaming kernel for m <= 32 (no RESID_SUM) */
     int32_t n_kv_head;                                        /* QKV only: key/value heads (0 = n_head); the K and V
                                                                  parts of n_out are n_kv_head * head_dim wide each */

@@ -39,7 +39,8 @@ struct TileCfg {
     static constexpr int B_BYTES = BN * BK * 2;
     static constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
     static constexpr int STAGES = SMEM_BUDGET / STAGE_BYTES > 8 ? 8 : SMEM_BUDGET / STAGE_BYTES;
-    static constexpr int TMEM_COLS = 2 * BN;  // two accumulators; 128, 256 or 512 columns
+    // two accumulators; TMEM is allocated in powers of two of at least 32 columns
+    static constexpr int TMEM_COLS = 2 * BN <= 64 ? 64 : (2 * BN <= 128 ? 128 : (2 * BN <= 256 ? 256 : 512));
     static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 };
 
@@ -183,7 +184,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     } else {
         const int quarter = warp & 3;          // TMEM lanes this warp may read
         const int half = (warp - 2) >> 2;      // which half of the tile's columns it drains
-        constexpr int CHUNKS = BN / 32 / 2;    // 32-column chunks per warp
+        constexpr int CHUNKS = BN / 32;        // 32-column chunks of the tile: `half` takes every second one
         int acc = 0;
         uint32_t acc_phase = 0;
         bool ok = true;
@@ -197,8 +198,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
                                    static_cast<uint32_t>(acc * BN);
 #pragma unroll 1
-            for (int cc = 0; cc < CHUNKS; ++cc) {
-                const int c = half * CHUNKS + cc;
+            for (int c = half; c < CHUNKS; c += 2) {
                 const int col0 = n_blk * BN + c * 32;
                 if (col0 >= ka.shape.n_out) break;  // uniform across the warp
                 uint32_t r[32];
@@ -511,12 +511,26 @@ int gemm_pick_bn(const GemmShape &s) {
         const long long items = ((s.m + 2 * BM - 1) / (2 * BM)) * ((s.n_out + BN2 - 1) / BN2) * s.groups;
         if (items >= sms && !env_flag("KRAKEN_GEMM_NO_PAIR")) return GEMM_TILE_PAIR;
     }
-    // Largest N tile that still gives every SM about one work item.
+    // Plenty of tiles: the largest N tile that still gives every SM about two work items.
     for (int bn : {256, 128}) {
         const long long items = tiles_m * ((s.n_out + bn - 1) / bn) * s.groups;
-        if (items >= sms) return bn;
+        if (items >= 2LL * sms) return bn;
     }
-    return 64;
+    // Few tiles (short prompts: the weights stream through once): the tile width decides how many rounds the
+    // SMs need, and a round costs about its width plus a fixed part (the A tile, set-up, drain).  156 tiles
+    // of 64 columns are two rounds on 148 SMs where 104 tiles of 96 columns are one.
+    int best = 64;
+    long long best_cost = -1;
+    for (int bn = 256; bn >= 32; bn -= 32) {
+        const long long items = tiles_m * ((s.n_out + bn - 1) / bn) * s.groups;
+        const long long rounds = (items + sms - 1) / sms;
+        const long long cost = rounds * (bn + 64);
+        if (best_cost < 0 || cost < best_cost) {
+            best_cost = cost;
+            best = bn;
+        }
+    }
+    return best;
 }
 
 int gemm_encode_a(CUtensorMap *map, const GemmOperands &op, const GemmShape &s) {
@@ -570,8 +584,13 @@ int launch_gemm_tc(const GemmOperands &op, const GemmShape &s, const EpiParams &
     const int grid = static_cast<int>(units < sms ? units : sms);
     switch (bn) {
         case 256: return launch_bn<256>(*tmA, *tmB, ka, grid, stream);
+        case 224: return launch_bn<224>(*tmA, *tmB, ka, grid, stream);
+        case 192: return launch_bn<192>(*tmA, *tmB, ka, grid, stream);
+        case 160: return launch_bn<160>(*tmA, *tmB, ka, grid, stream);
         case 128: return launch_bn<128>(*tmA, *tmB, ka, grid, stream);
+        case 96: return launch_bn<96>(*tmA, *tmB, ka, grid, stream);
         case 64: return launch_bn<64>(*tmA, *tmB, ka, grid, stream);
+        case 32: return launch_bn<32>(*tmA, *tmB, ka, grid, stream);
         default: return KRAKEN_EINVAL;
     }
 }

@@ -146,21 +146,21 @@ def gemm_case(G, M, Nout, K, epi, n_tile, seed=0, integer=False, shared_resid=Fa
                 sum=None if ssum is None else ssum.cpu().numpy(), ref=ref, keep=keep)
 
 
-@pytest.mark.parametrize("n_tile", [64, 128, 256, 512])
+@pytest.mark.parametrize("n_tile", [32, 64, 96, 128, 160, 192, 224, 256, 512])
 def test_gemm_integer_exact_ragged(n_tile):
     """Small integers make every product and partial sum exact: any mis-placed element shows."""
     r = gemm_case(2, 300, 200, 136, kr.EPI_F32, n_tile, integer=True)
     assert np.array_equal(r["out_f32"], r["ref"])
 
 
-@pytest.mark.parametrize("n_tile", [0, 64, 128, 256, 512])
+@pytest.mark.parametrize("n_tile", [0, 32, 64, 96, 128, 160, 192, 224, 256, 512])
 def test_gemm_f32_many_tiles(n_tile):
     r = gemm_case(2, 2048, 2304, 768, kr.EPI_F32, n_tile, seed=1)
     err = np.abs(r["out_f32"] - r["ref"])
     assert err.max() < 2e-4, err.max()
 
 
-@pytest.mark.parametrize("n_tile", [0, 512])
+@pytest.mark.parametrize("n_tile", [0, 96, 160, 512])
 @pytest.mark.parametrize("epi", [kr.EPI_BF16, kr.EPI_GELU_BF16])
 def test_gemm_bf16_epilogues(epi, n_tile):
     r = gemm_case(3, 200, 320, 256, epi, n_tile, seed=2)
