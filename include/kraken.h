@@ -62,7 +62,10 @@ typedef struct kraken_config {
     int32_t n_kv_head; /* key/value heads per sub-layer: 0 or n_head = multi-head attention; a divisor of
                           n_head = grouped-query attention, 1 = multi-query attention (the KV-cache
                           mitigation of Sec. 4.2): query head h reads key/value head h / (n_head / n_kv_head) */
-    int32_t reserved[4];
+    int32_t no_combine;/* 1: no cross-branch term (y = 0 in every layer).  With n_branch = 1 the layers are those
+                          of the standard pre-LayerNorm Transformer the paper compares against (Sec. 4.2), on
+                          the same kernels; 0 (default): Algorithm 1 */
+    int32_t reserved[3];
 } kraken_config;
 
 /* Device pointers to bf16 weights, row-major [out_features, in_features]; BORROWED until

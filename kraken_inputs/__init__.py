@@ -51,6 +51,7 @@ class KrakenShape:
     gelu_tanh: int = 0
     final_ln: int = 1
     n_kv_head: int = 0      # key/value heads per sub-layer; 0 = n_head (multi-head), 1 = multi-query
+    no_combine: int = 0     # 1: no cross-branch term; with one branch, the standard pre-LN Transformer's layers
 
     @property
     def head_dim(self) -> int:
@@ -107,6 +108,11 @@ CONFIGS.update({
     "K0-104": KrakenShape("K0-104", 2, 3, 416, 4, 832, 1024, 320, 2, 300),
     "K0-96": KrakenShape("K0-96", 4, 2, 192, 2, 384, 1024, 320, 1, 200),
     "K0-72": KrakenShape("K0-72", 2, 2, 288, 4, 576, 1024, 320, 1, 257),
+    # the standard Transformers of the same table (one branch, no cross-branch term, FFN 4 d): the architecture
+    # the paper compares Kraken against, here on the same kernels and the same single GPU
+    "S1.3B": KrakenShape("S1.3B", 1, 24, 2048, 16, 8192, 51200, 2048, 1, 2048, no_combine=1),
+    "S6.7B": KrakenShape("S6.7B", 1, 32, 4096, 32, 16384, 51200, 2048, 1, 2048, no_combine=1),
+    "S0": KrakenShape("S0", 1, 3, 256, 4, 1024, 1024, 160, 2, 100, no_combine=1),
 })
 
 # TTFT in ms printed by the paper for the Kraken engines (Tables 4 and 5; fp16, batch 1, on as many

@@ -168,7 +168,7 @@ class Oracle:
             d_ff=shape.d_ff, vocab=shape.vocab, max_pos=shape.max_pos, ln_eps=shape.ln_eps,
             gelu_tanh=int(shape.gelu_tanh if gelu_tanh is None else gelu_tanh),
             final_ln=int(shape.final_ln if final_ln is None else final_ln),
-            bf16_store=int(bf16_store), y_zero=int(y_zero), half=int(half),
+            bf16_store=int(bf16_store), y_zero=int(y_zero or getattr(shape, "no_combine", 0)), half=int(half),
             n_kv_head=int(getattr(shape, "n_kv_head", 0)))
         self._keep = {k: _bits(v) for k, v in weights_bits.items()}
         self.w = KoWeights(**{k: _ptr(self._keep.get(k)) for k in WEIGHT_FIELDS})

@@ -49,7 +49,8 @@ typedef struct ko_config {
     int32_t gelu_tanh;   /* 0: erf form, 1: tanh approximation */
     int32_t final_ln;    /* 1: LayerNorm between W_concat and the unembedding */
     int32_t bf16_store;  /* 1: round activations to bf16 at the store points */
-    int32_t y_zero;      /* test-only: drop the y term (reduces N = 1 to a GPT-2 stack) */
+    int32_t y_zero;      /* drop the y term: with N = 1 the layers are a standard pre-LN Transformer's
+                            (the comparison architecture of Sec. 4.2) */
     int32_t half;        /* 16-bit type of weights and store points: 0 = bfloat16, 1 = IEEE half */
     int32_t n_kv_head;   /* key/value heads per sub-layer: 0 or n_head = multi-head attention; fewer =
                             grouped-query attention, 1 = multi-query (the KV-cache mitigation of Sec. 4.2

@@ -45,7 +45,7 @@ class KrakenConfig(C.Structure):
     _fields_ = [(n, C.c_int32) for n in
                 ("n_branch", "n_layer", "d_model", "n_head", "d_ff", "vocab", "max_pos", "max_batch")] + [
         ("ln_eps", C.c_float), ("gelu_tanh", C.c_int32), ("final_ln", C.c_int32), ("n_kv_head", C.c_int32),
-        ("reserved", C.c_int32 * 4)]
+        ("no_combine", C.c_int32), ("reserved", C.c_int32 * 3)]
 
 
 class KrakenWeights(C.Structure):
@@ -169,7 +169,8 @@ def make_config(shape, max_batch: Optional[int] = None, max_pos: Optional[int] =
         n_branch=shape.n_branch, n_layer=shape.n_layer, d_model=shape.d_model, n_head=shape.n_head,
         d_ff=shape.d_ff, vocab=shape.vocab, max_pos=max_pos or shape.max_pos,
         max_batch=max_batch or shape.batch, ln_eps=shape.ln_eps, gelu_tanh=shape.gelu_tanh,
-        final_ln=shape.final_ln, n_kv_head=int(getattr(shape, "n_kv_head", 0) or 0))
+        final_ln=shape.final_ln, n_kv_head=int(getattr(shape, "n_kv_head", 0) or 0),
+        no_combine=int(getattr(shape, "no_combine", 0) or 0))
     for k, v in over.items():
         setattr(cfg, k, v)
     return cfg

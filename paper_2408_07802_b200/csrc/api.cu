@@ -339,8 +339,8 @@ int run_layers(const RunCtx &rc, const int32_t *d_tokens) {
             LaunchScope scope(h, KRAKEN_PROF_LAYERNORM, rc.st);
             // with few rows the cross-branch sum is formed here from the N branch inputs (same order as
             // the down-projection epilogue forms it for long prompts)
-            const bool sum_here = small_rows && !sum_pass && l > 0;
-            KR_TRY(launch_layernorm(a, td, sum_here ? nullptr : (l == 0 ? x0 : S),
+            const bool sum_here = small_rows && !sum_pass && l > 0 && !c.no_combine;
+            KR_TRY(launch_layernorm(a, td, (sum_here || c.no_combine) ? nullptr : (l == 0 ? x0 : S),
                                     (const uint16_t *)h->w.ln2_g + ln_off,
                                     h->w.ln2_b ? (const uint16_t *)h->w.ln2_b + ln_off : nullptr, N, T, d, c.ln_eps,
                                     u, rc.st, sum_here ? x : nullptr, td, N, status));
@@ -352,12 +352,12 @@ int run_layers(const RunCtx &rc, const int32_t *d_tokens) {
         KR_TRY(model_gemm(rc, G_UP, l, T, u, td, e));
         // out = res + FFN ; the sum over branches (the AllReduce feeding the next layer) in the epilogue
         e = epi_zero();
-        e.kind = (l + 1 < L && !small_rows) ? KRAKEN_EPI_RESID_SUM : KRAKEN_EPI_RESID_F32;
+        e.kind = (l + 1 < L && !small_rows && !c.no_combine) ? KRAKEN_EPI_RESID_SUM : KRAKEN_EPI_RESID_F32;
         e.out_f32 = x; e.out_f32_gstride = td; e.ld_out_f32 = d;
         e.resid = a; e.resid_gstride = td; e.ld_resid = d;
         e.sum = S; e.ld_sum = d;
         KR_TRY(model_gemm(rc, G_DOWN, l, T, gb, (long long)T * F, e));
-        if (sum_pass && l + 1 < L) {
+        if (sum_pass && l + 1 < L && !c.no_combine) {
             LaunchScope scope(h, KRAKEN_PROF_LAYERNORM, rc.st);
             KR_TRY(launch_sum_groups(x, td, N, td, S, rc.st));
         }
@@ -482,15 +482,16 @@ int run_layers_decode_branches(const RunCtx &rc, const int32_t *d_tokens) {
             e.resid = xin; e.resid_gstride = 0; e.ld_resid = d;
             KR_TRY(model_gemm(rc, G_PROJ, l, T, o + b * td, td, e, b, 1, st));
             // LayerNorm-2 sums the previous layer's outputs of every branch
-            if (l > 0)
+            if (l > 0 && !c.no_combine)
                 for (int j = 0; j < N; ++j)
                     if (j != b) KR_CU(cudaStreamWaitEvent(st, h->ev_down[(l - 1) & 1][j], 0));
             {
                 LaunchScope scope(h, KRAKEN_PROF_LAYERNORM, st);
-                KR_TRY(launch_layernorm(a + b * td, 0, l == 0 ? x0 : nullptr,
+                KR_TRY(launch_layernorm(a + b * td, 0, (l == 0 && !c.no_combine) ? x0 : nullptr,
                                         (const uint16_t *)h->w.ln2_g + ln_off + (long long)b * d,
                                         h->w.ln2_b ? (const uint16_t *)h->w.ln2_b + ln_off + (long long)b * d : nullptr,
-                                        1, T, d, c.ln_eps, u + b * td, st, l == 0 ? nullptr : xprev, td, N));
+                                        1, T, d, c.ln_eps, u + b * td, st,
+                                        (l == 0 || c.no_combine) ? nullptr : xprev, td, N));
             }
             e = epi_zero();
             e.kind = KRAKEN_EPI_GELU_BF16;
