@@ -65,7 +65,10 @@ typedef struct kraken_config {
     int32_t no_combine;/* 1: no cross-branch term (y = 0 in every layer).  With n_branch = 1 the layers are those
                           of the standard pre-LayerNorm Transformer the paper compares against (Sec. 4.2), on
                           the same kernels; 0 (default): Algorithm 1 */
-    int32_t reserved[3];
+    int32_t parallel_ffn; /* 1: the FFN reads the first LayerNorm's output, in parallel with attention:
+                          out = x + MHA(LN(x)) + FFN(LN(x)) - the "Parallel Attention + FeedForward"
+                          comparison architecture of Sec. 4.2; ln2 weights are then unused and there is no y */
+    int32_t reserved[2];
 } kraken_config;
 
 /* Device pointers to bf16 weights, row-major [out_features, in_features]; BORROWED until

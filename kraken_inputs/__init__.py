@@ -52,6 +52,7 @@ class KrakenShape:
     final_ln: int = 1
     n_kv_head: int = 0      # key/value heads per sub-layer; 0 = n_head (multi-head), 1 = multi-query
     no_combine: int = 0     # 1: no cross-branch term; with one branch, the standard pre-LN Transformer's layers
+    parallel_ffn: int = 0   # 1: out = x + MHA(LN(x)) + FFN(LN(x)): the parallel Attention + FeedForward variant
 
     @property
     def head_dim(self) -> int:
@@ -113,6 +114,10 @@ CONFIGS.update({
     "S1.3B": KrakenShape("S1.3B", 1, 24, 2048, 16, 8192, 51200, 2048, 1, 2048, no_combine=1),
     "S6.7B": KrakenShape("S6.7B", 1, 32, 4096, 32, 16384, 51200, 2048, 1, 2048, no_combine=1),
     "S0": KrakenShape("S0", 1, 3, 256, 4, 1024, 1024, 160, 2, 100, no_combine=1),
+    # and the parallel Attention + FeedForward variants of the same sizes (GPT-J-like dataflow, Sec. 4.2)
+    "P1.3B": KrakenShape("P1.3B", 1, 24, 2048, 16, 8192, 51200, 2048, 1, 2048, no_combine=1, parallel_ffn=1),
+    "P6.7B": KrakenShape("P6.7B", 1, 32, 4096, 32, 16384, 51200, 2048, 1, 2048, no_combine=1, parallel_ffn=1),
+    "P0": KrakenShape("P0", 1, 3, 256, 4, 1024, 1024, 160, 2, 100, no_combine=1, parallel_ffn=1),
 })
 
 # TTFT in ms printed by the paper for the Kraken engines (Tables 4 and 5; fp16, batch 1, on as many

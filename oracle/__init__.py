@@ -36,7 +36,8 @@ class KoConfig(C.Structure):
     _fields_ = [(n, C.c_int32) for n in
                 ("n_branch", "n_layer", "d_model", "n_head", "d_ff", "vocab", "max_pos")] + [
         ("ln_eps", C.c_float), ("gelu_tanh", C.c_int32), ("final_ln", C.c_int32),
-        ("bf16_store", C.c_int32), ("y_zero", C.c_int32), ("half", C.c_int32), ("n_kv_head", C.c_int32)]
+        ("bf16_store", C.c_int32), ("y_zero", C.c_int32), ("half", C.c_int32), ("parallel_ffn", C.c_int32),
+        ("n_kv_head", C.c_int32)]
 
 
 class KoWeights(C.Structure):
@@ -169,7 +170,7 @@ class Oracle:
             gelu_tanh=int(shape.gelu_tanh if gelu_tanh is None else gelu_tanh),
             final_ln=int(shape.final_ln if final_ln is None else final_ln),
             bf16_store=int(bf16_store), y_zero=int(y_zero or getattr(shape, "no_combine", 0)), half=int(half),
-            n_kv_head=int(getattr(shape, "n_kv_head", 0)))
+            parallel_ffn=int(getattr(shape, "parallel_ffn", 0)), n_kv_head=int(getattr(shape, "n_kv_head", 0)))
         self._keep = {k: _bits(v) for k, v in weights_bits.items()}
         self.w = KoWeights(**{k: _ptr(self._keep.get(k)) for k in WEIGHT_FIELDS})
         self.shape = shape

@@ -52,6 +52,9 @@ typedef struct ko_config {
     int32_t y_zero;      /* drop the y term: with N = 1 the layers are a standard pre-LN Transformer's
                             (the comparison architecture of Sec. 4.2) */
     int32_t half;        /* 16-bit type of weights and store points: 0 = bfloat16, 1 = IEEE half */
+    int32_t parallel_ffn;/* 1: the FFN reads the first LayerNorm's output, in parallel with attention:
+                            out = x + MHA(LN(x)) + FFN(LN(x)), the "Parallel Attention + FeedForward"
+                            comparison architecture of Sec. 4.2 (no second LayerNorm, no y) */
     int32_t n_kv_head;   /* key/value heads per sub-layer: 0 or n_head = multi-head attention; fewer =
                             grouped-query attention, 1 = multi-query (the KV-cache mitigation of Sec. 4.2
                             and the KV-cache appendix): query head h reads key/value head
@@ -373,8 +376,11 @@ static int forward(ko_state *s, const int32_t *ids, int n, int pos0, float *logi
             /* x = res + MHA */
             ko_linear(o, n, d, w->w_proj + ln * (size_t)d * d, d, w->b_proj ? w->b_proj + ln * d : NULL, d, tmp);
             for (size_t i = 0; i < nd; ++i) a[i] = xb[i] + tmp[i];
-            /* x = LN(x + y) */
-            ko_layernorm(a, y, n, d, w->ln2_g + ln * d, w->ln2_b ? w->ln2_b + ln * d : NULL, c->ln_eps, rb, hh);
+            /* x = LN(x + y); in the parallel variant the FFN takes the first LayerNorm's output instead */
+            if (c->parallel_ffn)
+                memcpy(hh, u, sizeof(float) * nd);
+            else
+                ko_layernorm(a, y, n, d, w->ln2_g + ln * d, w->ln2_b ? w->ln2_b + ln * d : NULL, c->ln_eps, rb, hh);
             /* out = res + FFN(x) */
             ko_linear(hh, n, d, w->w_up + ln * (size_t)F * d, d, w->b_up ? w->b_up + ln * F : NULL, F, g);
             for (size_t i = 0; i < (size_t)n * F; ++i) {

@@ -45,7 +45,7 @@ class KrakenConfig(C.Structure):
     _fields_ = [(n, C.c_int32) for n in
                 ("n_branch", "n_layer", "d_model", "n_head", "d_ff", "vocab", "max_pos", "max_batch")] + [
         ("ln_eps", C.c_float), ("gelu_tanh", C.c_int32), ("final_ln", C.c_int32), ("n_kv_head", C.c_int32),
-        ("no_combine", C.c_int32), ("reserved", C.c_int32 * 3)]
+        ("no_combine", C.c_int32), ("parallel_ffn", C.c_int32), ("reserved", C.c_int32 * 2)]
 
 
 class KrakenWeights(C.Structure):
@@ -170,7 +170,8 @@ def make_config(shape, max_batch: Optional[int] = None, max_pos: Optional[int] =
         d_ff=shape.d_ff, vocab=shape.vocab, max_pos=max_pos or shape.max_pos,
         max_batch=max_batch or shape.batch, ln_eps=shape.ln_eps, gelu_tanh=shape.gelu_tanh,
         final_ln=shape.final_ln, n_kv_head=int(getattr(shape, "n_kv_head", 0) or 0),
-        no_combine=int(getattr(shape, "no_combine", 0) or 0))
+        no_combine=int(getattr(shape, "no_combine", 0) or 0),
+        parallel_ffn=int(getattr(shape, "parallel_ffn", 0) or 0))
     for k, v in over.items():
         setattr(cfg, k, v)
     return cfg

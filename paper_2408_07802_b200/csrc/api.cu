@@ -35,6 +35,7 @@ int check_config(const kraken_config *c) {
         return KRAKEN_EINVAL;
     if (c->d_model % c->n_head != 0) return KRAKEN_EINVAL;
     if (c->n_kv_head < 0 || (c->n_kv_head > 0 && c->n_head % c->n_kv_head != 0)) return KRAKEN_EINVAL;
+    if (c->parallel_ffn && !c->no_combine) return KRAKEN_EINVAL;   // the parallel variant has no cross-branch term
     const int hd = c->d_model / c->n_head;
     // 64 and 128, and the head dims of the paper's engine shapes (Table 3: 72, 96, 104)
     if (hd != 64 && hd != 72 && hd != 96 && hd != 104 && hd != 128) return KRAKEN_EUNSUPPORTED;
@@ -335,7 +336,8 @@ int run_layers(const RunCtx &rc, const int32_t *d_tokens) {
         e.resid = xin; e.resid_gstride = xin_gs; e.ld_resid = d;
         KR_TRY(model_gemm(rc, G_PROJ, l, T, o, td, e));
         // x = LN(x + y): y is the shared embedding in the first layer, the cross-branch sum afterwards
-        {
+        // (the parallel variant feeds the FFN with the first LayerNorm's output, still in u)
+        if (!c.parallel_ffn) {
             LaunchScope scope(h, KRAKEN_PROF_LAYERNORM, rc.st);
             // with few rows the cross-branch sum is formed here from the N branch inputs (same order as
             // the down-projection epilogue forms it for long prompts)
@@ -482,10 +484,10 @@ int run_layers_decode_branches(const RunCtx &rc, const int32_t *d_tokens) {
             e.resid = xin; e.resid_gstride = 0; e.ld_resid = d;
             KR_TRY(model_gemm(rc, G_PROJ, l, T, o + b * td, td, e, b, 1, st));
             // LayerNorm-2 sums the previous layer's outputs of every branch
-            if (l > 0 && !c.no_combine)
+            if (l > 0 && !c.no_combine && !c.parallel_ffn)
                 for (int j = 0; j < N; ++j)
                     if (j != b) KR_CU(cudaStreamWaitEvent(st, h->ev_down[(l - 1) & 1][j], 0));
-            {
+            if (!c.parallel_ffn) {
                 LaunchScope scope(h, KRAKEN_PROF_LAYERNORM, st);
                 KR_TRY(launch_layernorm(a + b * td, 0, (l == 0 && !c.no_combine) ? x0 : nullptr,
                                         (const uint16_t *)h->w.ln2_g + ln_off + (long long)b * d,

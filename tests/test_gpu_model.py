@@ -371,13 +371,14 @@ def prefix_parity(name, prefix, seqs):
     m.close()
 
 
-@pytest.mark.parametrize("name", ["K0-104", "K0-96", "K0-72", "C0-gqa", "C0-mqa", "S0", "S0x2"])
+@pytest.mark.parametrize("name", ["K0-104", "K0-96", "K0-72", "C0-gqa", "C0-mqa", "S0", "S0x2", "P0"])
 def test_engine_head_dims_and_shared_kv_heads_small_models_all_positions_cache_and_decode(name):
     """Small models with the head dims (104, 96, 72) and the 2 d FFN of the paper's engine shapes (Table 3), and
     with grouped-query / multi-query attention (Sec. 4.2): every position and the cache element by element,
     then teacher-forced decode steps."""
     # S0: one branch without the cross-branch term = the standard pre-LN Transformer's layers (the paper's
-    # comparison architecture); S0x2: two such independent stacks joined only by W_concat
+    # comparison architecture); S0x2: two such independent stacks joined only by W_concat; P0: the parallel
+    # Attention + FeedForward variant (the FFN reads the first LayerNorm's output)
     s = ki.KrakenShape("S0x2", 2, 3, 256, 4, 1024, 1024, 160, 2, 100, no_combine=1) if name == "S0x2" else ki.CONFIGS[name]
     m, w = build(s)
     wb = host_bits(w)

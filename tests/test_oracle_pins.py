@@ -576,3 +576,34 @@ def test_half_mode_matches_library_composition_and_rounds_stores_to_half():
     k = orc.cache(0, 0, 0)
     assert np.array_equal(k, k.astype(np.float16).astype(np.float32))
 
+
+# ------------------------------------------------------------------ comparison architectures of Sec. 4.2
+
+def test_parallel_attention_feedforward_variant_is_a_gptj_style_stack():
+    """parallel_ffn = 1 (with one branch and no cross-branch term): out = x + MHA(LN(x)) + FFN(LN(x)), one
+    LayerNorm per layer, written here from library routines without any Kraken notion."""
+    shape = small_shape(n_branch=1, n_layer=3, no_combine=1, parallel_ffn=1)
+    w = rand_weights(shape)
+    w["w_concat"] = torch.eye(shape.d_model, dtype=torch.bfloat16)
+    w["b_concat"] = None
+    ids = ki.uniform_tokens(5, shape.vocab, 1, shape.seqlen)[0].numpy()
+    W = {k: (None if v is None else v.double()) for k, v in w.items()}
+    d, H = shape.d_model, shape.n_head
+    l = len(ids)
+    x = W["wte"][torch.as_tensor(ids, dtype=torch.long)] + W["wpe"][:l]
+    for layer in range(shape.n_layer):
+        u = F.layer_norm(x, (d,), W["ln1_g"][layer, 0], W["ln1_b"][layer, 0], 1e-5)
+        qkv = F.linear(u, W["w_qkv"][layer, 0], W["b_qkv"][layer, 0])
+        q, k, v = [t.reshape(l, H, d // H).transpose(0, 1) for t in qkv.split(d, dim=1)]
+        o = F.scaled_dot_product_attention(q[None], k[None], v[None], is_causal=True)[0].transpose(0, 1).reshape(l, d)
+        attn = F.linear(o, W["w_proj"][layer, 0], W["b_proj"][layer, 0])
+        ffn = F.linear(F.gelu(F.linear(u, W["w_up"][layer, 0], W["b_up"][layer, 0])),
+                       W["w_down"][layer, 0], W["b_down"][layer, 0])
+        x = x + attn + ffn
+    ref = (F.layer_norm(x, (d,), W["lnf_g"], W["lnf_b"], 1e-5) @ W["wte"].T).numpy()
+    got, _ = oracle.Oracle(shape, wbits(w)).prefill(ids)
+    assert np.max(np.abs(got - ref)) < 2e-5 * max(1.0, np.max(np.abs(ref)))
+    # it is a different function from the sequential stack on the same weights
+    seq, _ = oracle.Oracle(small_shape(n_branch=1, n_layer=3, no_combine=1), wbits(w)).prefill(ids)
+    assert np.max(np.abs(seq - ref)) > 1e-3
+
