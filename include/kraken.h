@@ -119,6 +119,20 @@ int kraken_prefill(kraken_handle *h, const int32_t *d_tokens, int32_t batch, int
 int kraken_prefill_host(kraken_handle *h, const int32_t *h_tokens, int32_t batch, int32_t seqlen,
                         float *h_logits, void *stream);
 
+/* Prefill of a batch whose sequences have different lengths, without padding ("packed" input): d_tokens
+ * holds the sequences back to back (device int32, sum of the lengths), h_seq_lens their lengths (HOST,
+ * read before the call returns), d_logits device fp32 [batch, V] = the logits of every sequence's last
+ * position.  Sequence b fills rows 0 .. len_b - 1 of its own slice of the KV cache (kraken_kv_view), and the
+ * decode steps that follow continue every sequence at its own position.  kraken_logits_rows then counts
+ * rows in the packed order.  Errors: EINVAL (a length < 1), ECAPACITY (batch > max_batch, a length >
+ * max_pos). */
+int kraken_prefill_packed(kraken_handle *h, const int32_t *d_tokens, const int32_t *h_seq_lens, int32_t batch,
+                          float *d_logits, void *stream);
+
+/* Current length of every cached sequence (host array of `batch` entries; kraken_cur_len is their maximum).
+ * ESTATE when batch differs from the cached batch. */
+int kraken_seq_lens(kraken_handle *h, int32_t *h_seq_lens, int32_t batch);
+
 /* Prefill that returns the logits of EVERY position: d_logits device fp32 [batch, seqlen, V].
  * Same cache side effects as kraken_prefill.  Meant for tests and evaluation. */
 int kraken_prefill_all_logits(kraken_handle *h, const int32_t *d_tokens, int32_t batch, int32_t seqlen,

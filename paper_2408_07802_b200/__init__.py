@@ -33,7 +33,7 @@ PROF_COUNT = len(PROF_CATEGORIES)
 
 EXPORTS = (
     "kraken_query_sizes", "kraken_create", "kraken_prefill", "kraken_prefill_host",
-    "kraken_prefill_all_logits", "kraken_logits_rows", "kraken_decode_step", "kraken_decode_step_host", "kraken_kv_view",
+    "kraken_prefill_all_logits", "kraken_prefill_packed", "kraken_seq_lens", "kraken_logits_rows", "kraken_decode_step", "kraken_decode_step_host", "kraken_kv_view",
     "kraken_device_status", "kraken_cur_len", "kraken_profile_enable", "kraken_profile_read", "kraken_reset", "kraken_destroy", "kraken_strerror", "kraken_last_cuda_error",
     "kraken_op_embed", "kraken_op_layernorm", "kraken_op_grouped_gemm", "kraken_op_attention",
     "kraken_op_decode_attention", "kraken_decode_attention_sizes",
@@ -113,6 +113,8 @@ def lib(dtype: Optional[str] = None) -> C.CDLL:
         L.kraken_prefill.argtypes = [vp, vp, i32, i32, vp, vp]
         L.kraken_prefill_host.argtypes = [vp, vp, i32, i32, vp, vp]
         L.kraken_prefill_all_logits.argtypes = [vp, vp, i32, i32, vp, vp]
+        L.kraken_prefill_packed.argtypes = [vp, vp, vp, i32, vp, vp]
+        L.kraken_seq_lens.argtypes = [vp, vp, i32]
         L.kraken_logits_rows.argtypes = [vp, vp, i32, vp, vp]
         L.kraken_decode_step.argtypes = [vp, vp, i32, vp, vp]
         L.kraken_decode_step_host.argtypes = [vp, vp, i32, vp, vp]
@@ -239,6 +241,24 @@ class KrakenModel:
         _check(lib(self.dtype).kraken_prefill_all_logits(self._h, tokens.data_ptr(), b, l, logits.data_ptr(), _stream()),
                "kraken_prefill_all_logits")
         return logits
+
+    def prefill_packed(self, tokens: torch.Tensor, seq_lens, logits: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """tokens: device int32 [sum(seq_lens)], the sequences back to back -> fp32 [batch, V] logits of every
+        sequence's last position."""
+        lens = torch.as_tensor(seq_lens, dtype=torch.int32).contiguous()
+        b = lens.numel()
+        assert tokens.dtype == torch.int32 and tokens.is_contiguous() and tokens.device == self.device
+        assert tokens.numel() == int(lens.sum())
+        if logits is None:
+            logits = torch.empty(b, self.cfg.vocab, dtype=torch.float32, device=self.device)
+        _check(lib(self.dtype).kraken_prefill_packed(self._h, tokens.data_ptr(), lens.data_ptr(), b, logits.data_ptr(),
+                                                     _stream()), "kraken_prefill_packed")
+        return logits
+
+    def seq_lens(self, batch: int):
+        out = torch.zeros(batch, dtype=torch.int32)
+        _check(lib(self.dtype).kraken_seq_lens(self._h, out.data_ptr(), batch), "kraken_seq_lens")
+        return out.tolist()
 
     def logits_rows(self, rows) -> torch.Tensor:
         rows_t = torch.as_tensor(rows, dtype=torch.int32).contiguous()

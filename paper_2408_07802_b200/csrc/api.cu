@@ -21,7 +21,7 @@ constexpr size_t ALIGN = 256;
 size_t align_up(size_t v) { return (v + ALIGN - 1) / ALIGN * ALIGN; }
 
 struct Layout {
-    size_t status, tokens, rows, logits, x0, x, a, s, u, q, o, g, dec_part, x_alt, total;
+    size_t status, tokens, rows, logits, x0, x, a, s, u, q, o, g, dec_part, x_alt, row_seq, row_pos, pos_arr, total;
 };
 
 int kv_heads_of(const kraken_config &c) { return c.n_kv_head > 0 ? c.n_kv_head : c.n_head; }
@@ -73,6 +73,9 @@ Layout layout_of(const kraken_config *c) {
     l.dec_part = take(decode_attention_partial_bytes(c->n_branch, c->max_batch, c->n_head, c->d_model / c->n_head,
                                                      DECODE_MAX_SPLITS));
     l.x_alt = take((size_t)N * c->max_batch * d * 4);   // second copy of the branch outputs of a decode step
+    l.row_seq = take(T * 4);                            // packed prefill: sequence and position of every row
+    l.row_pos = take(T * 4);
+    l.pos_arr = take((size_t)c->max_batch * 4);         // next position of every sequence (device copy)
     l.total = off;
     return l;
 }
@@ -90,6 +93,10 @@ struct kraken_handle {
     uint8_t *scratch;
     Layout lay;
     int cur_len, batch, last_seqlen, last_rows;  // last_rows: token rows of the last model run
+    // length of every cached sequence (cur_len is their maximum); ragged = they differ, set by a packed prefill
+    std::vector<int> seq_len;
+    bool ragged;
+    std::vector<int> host_rows, host_row_seq, host_row_pos;   // staging of the packed-prefill tables
     cudaStream_t last_stream;
     bool naive;
     // weight tensor maps, one per GEMM kind, re-encoded when the N tile changes
@@ -166,8 +173,12 @@ struct RunCtx {
     kraken_handle *h;
     cudaStream_t st;
     int batch, seqlen, pos0, T;
-    const int *pos_dev;  // decode graph: positions come from device memory
-    int max_keys;        // decode graph: upper bound of the keys a step can see (fixes the split count)
+    const int *pos_dev;  // decode: the next position of every sequence, in device memory
+    int max_keys;        // decode: upper bound of the keys a step can see (fixes the split count)
+    // packed prefill of sequences of different lengths (h->seq_len): sequence and position of every row;
+    // seqlen is then the longest length
+    bool packed;
+    const int *row_seq, *row_pos;
 };
 
 // One grouped GEMM of the model: weights of `kind` at `layer`.
@@ -273,7 +284,7 @@ int run_layers(const RunCtx &rc, const int32_t *d_tokens) {
     {
         LaunchScope scope(h, KRAKEN_PROF_EMBED, rc.st);
         KR_TRY(launch_embed(d_tokens, T, rc.seqlen, rc.pos0, (const uint16_t *)h->w.wte, (const uint16_t *)h->w.wpe, d,
-                            c.vocab, x0, status, rc.st, rc.pos_dev));
+                            c.vocab, x0, status, rc.st, rc.pos_dev, rc.row_pos));
     }
     for (int l = 0; l < L; ++l) {
         const float *xin = l == 0 ? x0 : x;
@@ -295,6 +306,7 @@ int run_layers(const RunCtx &rc, const int32_t *d_tokens) {
         e.seqlen = rc.seqlen; e.pos0 = rc.pos0; e.n_head = H; e.head_dim = hd; e.max_pos = c.max_pos; e.d_model = d;
         e.n_kv_head = Hkv;
         e.pos0_dev = rc.pos_dev;
+        e.row_seq = rc.row_seq; e.row_pos = rc.row_pos;
         KR_TRY(model_gemm(rc, G_QKV, l, T, u, td, e));
         // attention over the cached prefix
         AttnParams ap;
@@ -305,7 +317,28 @@ int run_layers(const RunCtx &rc, const int32_t *d_tokens) {
         ap.max_pos = c.max_pos; ap.out = o; ap.out_gstride = td;
         {
             LaunchScope scope(h, KRAKEN_PROF_ATTENTION, rc.st);
-            if (h->naive) {
+            if (rc.packed) {
+                // sequences of different lengths: one launch per sequence on its rows of the packed tensors
+                long long row0 = 0;
+                for (int b = 0; b < rc.batch; ++b) {
+                    AttnParams sp = ap;
+                    sp.batch = 1;
+                    sp.seqlen = h->seq_len[b];
+                    sp.q = q + row0 * d;
+                    sp.out = o + row0 * d;
+                    sp.k_cache = ap.k_cache + b * cache_b;
+                    sp.v_cache = ap.v_cache + b * cache_b;
+                    if (b > 0) h->launches[KRAKEN_PROF_ATTENTION]++;
+                    if (h->naive) {
+                        KR_TRY(launch_attention_naive(sp, rc.st));
+                    } else if (attention_tc_supported(sp) && !env_flag("KRAKEN_ATTN_WARP_MMA")) {
+                        KR_TRY(launch_attention_tc(sp, nullptr, nullptr, nullptr, status, rc.st));
+                    } else {
+                        KR_TRY(launch_attention_prefill(sp, rc.st));
+                    }
+                    row0 += h->seq_len[b];
+                }
+            } else if (h->naive) {
                 KR_TRY(launch_attention_naive(ap, rc.st));
             } else if (rc.seqlen == 1) {
                 // decode step: stream the cache with the split-KV kernel
@@ -418,7 +451,7 @@ int run_layers_decode_branches(const RunCtx &rc, const int32_t *d_tokens) {
     {
         LaunchScope scope(h, KRAKEN_PROF_EMBED, rc.st);
         KR_TRY(launch_embed(d_tokens, T, rc.seqlen, rc.pos0, (const uint16_t *)h->w.wte, (const uint16_t *)h->w.wpe, d,
-                            c.vocab, x0, status, rc.st, rc.pos_dev));
+                            c.vocab, x0, status, rc.st, rc.pos_dev, rc.row_pos));
     }
     KR_CU(cudaEventRecord(h->ev_fork, rc.st));
     for (int b = 1; b < N; ++b) KR_CU(cudaStreamWaitEvent(h->br_stream[b], h->ev_fork, 0));
@@ -517,13 +550,14 @@ int run_layers_decode_branches(const RunCtx &rc, const int32_t *d_tokens) {
     return KRAKEN_OK;
 }
 
-__global__ void set_pos_kernel(int *pos, int value) {
+// The next position of every sequence lives in device memory (the decode graph reads it there).
+__global__ void set_pos_kernel(int *pos, int value, int batch) {
     pdl_wait();
-    *pos = value;
+    for (int b = threadIdx.x; b < batch; b += blockDim.x) pos[b] = value;
 }
-__global__ void advance_pos_kernel(int *pos) {
+__global__ void advance_pos_kernel(int *pos, int batch) {
     pdl_wait();
-    *pos += 1;
+    for (int b = threadIdx.x; b < batch; b += blockDim.x) pos[b] += 1;
 }
 
 __global__ void make_rows_kernel(int32_t *rows, int n, int mul, int add) {
@@ -570,7 +604,7 @@ int prefill_body(kraken_handle *h, cudaStream_t st, const int32_t *d_tokens, int
                  bool all_logits) {
     RunCtx rc{h, st, batch, seqlen, 0, batch * seqlen, nullptr, 0};
     KR_TRY(run_layers(rc, d_tokens));
-    set_pos_kernel<<<1, 1, 0, st>>>(at<int>(h, h->lay.status + 128), seqlen);
+    set_pos_kernel<<<1, 64, 0, st>>>(at<int>(h, h->lay.pos_arr), seqlen, batch);
     int32_t *rows = at<int32_t>(h, h->lay.rows);
     const int n_rows = all_logits ? batch * seqlen : batch;
     h->launches[KRAKEN_PROF_TAIL]++;
@@ -639,6 +673,62 @@ int prefill_common(kraken_handle *h, const int32_t *d_tokens, int batch, int seq
     h->cur_len = seqlen;
     h->batch = batch;
     h->last_seqlen = seqlen;
+    h->seq_len.assign(batch, seqlen);
+    h->ragged = false;
+    return KRAKEN_OK;
+}
+
+// Packed prefill: the sequences of the batch have their own lengths and their tokens follow each other
+// without padding.  Everything that works on token rows (LayerNorms, GEMMs) sees one [sum of lengths, d]
+// tensor; the embedding and the K/V scatter take a row's sequence and position from two small tables;
+// attention runs once per sequence on that sequence's rows.
+int prefill_packed(kraken_handle *h, const int32_t *d_tokens, const int32_t *h_seq_lens, int batch, float *d_logits,
+                   void *stream) {
+    if (!h || !d_tokens || !h_seq_lens || !d_logits || batch < 1) return KRAKEN_EINVAL;
+    if (batch > h->cfg.max_batch) return KRAKEN_ECAPACITY;
+    long long total = 0;
+    int longest = 0;
+    for (int b = 0; b < batch; ++b) {
+        if (h_seq_lens[b] < 1) return KRAKEN_EINVAL;
+        if (h_seq_lens[b] > h->cfg.max_pos) return KRAKEN_ECAPACITY;
+        total += h_seq_lens[b];
+        longest = h_seq_lens[b] > longest ? h_seq_lens[b] : longest;
+    }
+    if (total > (long long)h->cfg.max_batch * h->cfg.max_pos) return KRAKEN_ECAPACITY;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    h->last_stream = st;
+    if (h->pre_graph) cudaGraphExecDestroy(h->pre_graph);     // the cached prefill graph belongs to another shape
+    h->pre_graph = nullptr;
+    h->pre_tokens = nullptr;
+    h->pre_seen = 0;
+    const int T = static_cast<int>(total);
+    h->seq_len.assign(h_seq_lens, h_seq_lens + batch);
+    h->host_row_seq.resize(T);
+    h->host_row_pos.resize(T);
+    h->host_rows.resize(batch);
+    int r = 0;
+    for (int b = 0; b < batch; ++b) {
+        for (int t = 0; t < h_seq_lens[b]; ++t, ++r) {
+            h->host_row_seq[r] = b;
+            h->host_row_pos[r] = t;
+        }
+        h->host_rows[b] = r - 1;                              // last position of the sequence
+    }
+    int *d_row_seq = at<int>(h, h->lay.row_seq), *d_row_pos = at<int>(h, h->lay.row_pos);
+    int32_t *rows = at<int32_t>(h, h->lay.rows);
+    int *d_pos = at<int>(h, h->lay.pos_arr);
+    if (cudaMemcpyAsync(d_row_seq, h->host_row_seq.data(), (size_t)T * 4, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaMemcpyAsync(d_row_pos, h->host_row_pos.data(), (size_t)T * 4, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaMemcpyAsync(rows, h->host_rows.data(), (size_t)batch * 4, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+        cudaMemcpyAsync(d_pos, h->seq_len.data(), (size_t)batch * 4, cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return cuda_check(cudaGetLastError(), "packed prefill: table upload");
+    RunCtx rc{h, st, batch, longest, 0, T, nullptr, 0, true, d_row_seq, d_row_pos};
+    KR_TRY(run_layers(rc, d_tokens));
+    KR_TRY(run_tail(rc, rows, batch, d_logits));
+    h->cur_len = longest;
+    h->batch = batch;
+    h->last_seqlen = longest;
+    h->ragged = true;
     return KRAKEN_OK;
 }
 
@@ -687,6 +777,7 @@ int kraken_create(const kraken_config *cfg, const kraken_weights *w, void *d_kv,
     h->pre_batch = h->pre_seqlen = h->pre_all = h->pre_seen = 0;
     h->cap_stream = nullptr;
     h->br_ready = false;
+    h->ragged = false;
     h->dec_graph_batch = 0;
     h->dec_eager_steps = 0;
     h->use_graph = !env_flag("KRAKEN_NO_GRAPH") && !h->naive;
@@ -707,6 +798,18 @@ int kraken_create(const kraken_config *cfg, const kraken_weights *w, void *d_kv,
 int kraken_prefill(kraken_handle *h, const int32_t *d_tokens, int32_t batch, int32_t seqlen, float *d_logits,
                    void *stream) {
     return prefill_common(h, d_tokens, batch, seqlen, d_logits, stream, false);
+}
+
+int kraken_prefill_packed(kraken_handle *h, const int32_t *d_tokens, const int32_t *h_seq_lens, int32_t batch,
+                          float *d_logits, void *stream) {
+    return prefill_packed(h, d_tokens, h_seq_lens, batch, d_logits, stream);
+}
+
+int kraken_seq_lens(kraken_handle *h, int32_t *h_seq_lens, int32_t batch) {
+    if (!h || !h_seq_lens || batch < 1) return KRAKEN_EINVAL;
+    if (batch != h->batch || (int)h->seq_len.size() != batch) return KRAKEN_ESTATE;
+    for (int b = 0; b < batch; ++b) h_seq_lens[b] = h->seq_len[b];
+    return KRAKEN_OK;
 }
 
 int kraken_prefill_all_logits(kraken_handle *h, const int32_t *d_tokens, int32_t batch, int32_t seqlen,
@@ -746,6 +849,11 @@ int kraken_logits_rows(kraken_handle *h, const int32_t *h_rows, int32_t n_rows, 
 
 namespace {
 
+void advance_lengths(kraken_handle *h) {
+    h->cur_len += 1;
+    for (int &v : h->seq_len) v += 1;
+}
+
 // Whether decode steps of this handle run the branches as concurrent chains.
 bool decode_chains(const kraken_handle *h) {
     return !h->naive && h->cfg.n_branch >= 2 && h->cfg.n_branch <= MAX_CHAINS && !env_flag("KRAKEN_DECODE_ONE_CHAIN");
@@ -754,8 +862,10 @@ bool decode_chains(const kraken_handle *h) {
 // The kernel sequence of one decode step; with from_dev the position is read from device memory.
 int decode_body(kraken_handle *h, cudaStream_t st, const int32_t *d_tokens, int batch, float *d_logits,
                 bool from_dev) {
-    int *d_pos = at<int>(h, h->lay.status + 128);
-    RunCtx rc{h, st, batch, 1, h->cur_len, batch, from_dev ? d_pos : nullptr, h->cfg.max_pos};
+    // positions always come from the device array: the sequences of a batch may differ in length
+    int *d_pos = at<int>(h, h->lay.pos_arr);
+    (void)from_dev;
+    RunCtx rc{h, st, batch, 1, h->cur_len, batch, d_pos, h->cfg.max_pos};
     // per-kernel timing wants the kernels one after the other, so profiled steps keep all branches in one chain
     if (decode_chains(h) && !h->prof_on) {
         KR_TRY(run_layers_decode_branches(rc, d_tokens));
@@ -768,7 +878,7 @@ int decode_body(kraken_handle *h, cudaStream_t st, const int32_t *d_tokens, int 
     make_rows_kernel<<<(batch + 255) / 256, 256, 0, st>>>(rows, batch, 1, 0);
     if (cudaGetLastError() != cudaSuccess) return KRAKEN_ECUDA;
     KR_TRY(run_tail(rc, rows, batch, d_logits));
-    advance_pos_kernel<<<1, 1, 0, st>>>(d_pos);
+    advance_pos_kernel<<<1, 64, 0, st>>>(d_pos, batch);
     return cuda_check(cudaGetLastError(), "decode: position update");
 }
 
@@ -792,7 +902,7 @@ int kraken_decode_step(kraken_handle *h, const int32_t *d_tokens, int32_t batch,
         // none of which may happen inside a stream capture)
         KR_TRY(decode_body(h, st, d_tokens, batch, d_logits, false));
         h->dec_eager_steps++;
-        h->cur_len += 1;
+        advance_lengths(h);
         return KRAKEN_OK;
     }
     int32_t *s_tok = at<int32_t>(h, h->lay.tokens);
@@ -822,7 +932,7 @@ int kraken_decode_step(kraken_handle *h, const int32_t *d_tokens, int32_t batch,
             cudaGetLastError();
             h->use_graph = false;                 // fall back to eager steps for this handle
             KR_TRY(decode_body(h, st, d_tokens, batch, d_logits, false));
-            h->cur_len += 1;
+            advance_lengths(h);
             return KRAKEN_OK;
         }
         ce = cudaGraphInstantiate(&h->dec_graph, graph, 0);
@@ -832,7 +942,7 @@ int kraken_decode_step(kraken_handle *h, const int32_t *d_tokens, int32_t batch,
             h->use_graph = false;
             cudaGetLastError();
             KR_TRY(decode_body(h, st, d_tokens, batch, d_logits, false));
-            h->cur_len += 1;
+            advance_lengths(h);
             return KRAKEN_OK;
         }
     }
@@ -843,7 +953,7 @@ int kraken_decode_step(kraken_handle *h, const int32_t *d_tokens, int32_t batch,
     if (d_logits != s_log)
         KR_TRY(cuda_check(cudaMemcpyAsync(d_logits, s_log, (size_t)batch * h->cfg.vocab * 4,
                                           cudaMemcpyDeviceToDevice, st), "decode: logits staging"));
-    h->cur_len += 1;
+    advance_lengths(h);
     return KRAKEN_OK;
 }
 
@@ -898,6 +1008,8 @@ int kraken_reset(kraken_handle *h) {
     h->batch = 0;
     h->last_rows = 0;
     h->last_seqlen = 0;
+    h->seq_len.clear();
+    h->ragged = false;
     return KRAKEN_OK;
 }
 

@@ -39,7 +39,7 @@ attn_decode_kernel(const DecodeAttnParams p) {
     const int d = p.n_head * HD;
 
     // keys of this split
-    const int n_keys = p.pos_dev ? *p.pos_dev + 1 : p.n_keys;
+    const int n_keys = p.pos_dev ? p.pos_dev[b] + 1 : p.n_keys;
     const int per = (n_keys + p.splits - 1) / p.splits;
     const int k_begin = split * per;
     const int k_end = min(n_keys, k_begin + per);
@@ -219,7 +219,7 @@ attn_decode_gqa_kernel(const DecodeAttnParams p) {
     const int kq = lane & 3, nq = lane >> 2;
     const int d = p.n_head * HD;
 
-    const int n_keys = p.pos_dev ? *p.pos_dev + 1 : p.n_keys;
+    const int n_keys = p.pos_dev ? p.pos_dev[b] + 1 : p.n_keys;
     const int per = (n_keys + p.splits - 1) / p.splits;
     const int k_begin = split * per;
     const int k_end = min(n_keys, k_begin + per);

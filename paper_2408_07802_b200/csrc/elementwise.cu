@@ -13,7 +13,7 @@ constexpr int ROW_WARPS = 8;  // warps (rows) per CTA
 __global__ void __launch_bounds__(ROW_WARPS * 32)
 embed_kernel(const int32_t *__restrict__ ids, int n_tokens, int seqlen, int pos0, const uint16_t *__restrict__ wte,
              const uint16_t *__restrict__ wpe, int d, int vocab, float *__restrict__ out, uint32_t *status,
-             const int *__restrict__ pos0_dev) {
+             const int *__restrict__ pos0_dev, const int *__restrict__ row_pos) {
     pdl_wait();
     pdl_trigger();
     const int t = blockIdx.x * ROW_WARPS + (threadIdx.x >> 5);
@@ -24,7 +24,9 @@ embed_kernel(const int32_t *__restrict__ ids, int n_tokens, int seqlen, int pos0
         if (lane == 0 && status) atomicOr(status, STATUS_BAD_TOKEN);
         id = 0;
     }
-    const int pos = (pos0_dev ? *pos0_dev : pos0) + t % seqlen;
+    // position: from the packed-batch table, else the sequence's first position (device array or host value)
+    // plus the offset inside the sequence
+    const int pos = row_pos ? row_pos[t] : (pos0_dev ? pos0_dev[t / seqlen] : pos0) + t % seqlen;
     const uint4 *te = reinterpret_cast<const uint4 *>(wte + (size_t)id * d);
     const uint4 *pe = reinterpret_cast<const uint4 *>(wpe + (size_t)pos * d);
     float4 *o = reinterpret_cast<float4 *>(out + (size_t)t * d);
@@ -311,11 +313,12 @@ int done() { return cudaGetLastError() == cudaSuccess ? KRAKEN_OK : KRAKEN_ECUDA
 }  // namespace
 
 int launch_embed(const int32_t *ids, int n_tokens, int seqlen, int pos0, const uint16_t *wte, const uint16_t *wpe,
-                 int d, int vocab, float *out, uint32_t *status, cudaStream_t stream, const int *pos0_dev) {
+                 int d, int vocab, float *out, uint32_t *status, cudaStream_t stream, const int *pos0_dev,
+                 const int *row_pos) {
     if (!ids || !wte || !wpe || !out || n_tokens < 1 || seqlen < 1 || pos0 < 0 || d < 8 || (d & 7) || vocab < 1)
         return KRAKEN_EINVAL;
     return cuda_check(launch_pdl(embed_kernel, dim3((n_tokens + ROW_WARPS - 1) / ROW_WARPS), dim3(ROW_WARPS * 32), 0,
-                                 stream, ids, n_tokens, seqlen, pos0, wte, wpe, d, vocab, out, status, pos0_dev),
+                                 stream, ids, n_tokens, seqlen, pos0, wte, wpe, d, vocab, out, status, pos0_dev, row_pos),
                       "embed: launch");
 }
 

@@ -197,7 +197,8 @@ __device__ __forceinline__ void epilogue_chunk(const EpiParams &p, int g, int ro
             // value row of this token; keys and values go to their (sequence, head, position) row of the cache
             const int d = p.d_model;
             const int kvd = p.n_kv_head * p.head_dim;      // width of the k part and of the v part
-            const int b = row / p.seqlen, pos = (p.pos0_dev ? *p.pos0_dev : p.pos0) + row % p.seqlen;
+            const int b = p.row_seq ? p.row_seq[row] : row / p.seqlen;
+            const int pos = p.row_pos ? p.row_pos[row] : (p.pos0_dev ? p.pos0_dev[b] : p.pos0) + row % p.seqlen;
             if (((d | p.head_dim) & 31) == 0) {            // the 32 columns lie inside q or inside one head
                 if (col0 < d) {
                     store_bf16_chunk(p.out_bf16 + g * p.out_bf16_gstride + (long long)row * p.ld_out_bf16 + col0, v,

@@ -55,7 +55,8 @@ __device__ __forceinline__ void epilogue_elem(const EpiParams &p, int g, int row
                 const int kvd = p.n_kv_head * p.head_dim;
                 const int which = col >= d + kvd, c = col - d - which * kvd;
                 const int head = c / p.head_dim, e = c % p.head_dim;
-                const int b = row / p.seqlen, pos = (p.pos0_dev ? *p.pos0_dev : p.pos0) + row % p.seqlen;
+                const int b = p.row_seq ? p.row_seq[row] : row / p.seqlen;
+                const int pos = p.row_pos ? p.row_pos[row] : (p.pos0_dev ? p.pos0_dev[b] : p.pos0) + row % p.seqlen;
                 uint16_t *base = (which ? p.v_cache : p.k_cache) + g * p.cache_gstride;
                 base[(((long long)b * p.n_kv_head + head) * p.max_pos + pos) * p.head_dim + e] = to_h16(acc);
             }

@@ -29,7 +29,11 @@ struct EpiParams {
     int seqlen, pos0, n_head, head_dim, max_pos, d_model;
     int n_kv_head;  // key/value heads (grouped-query attention); the k and v parts are n_kv_head * head_dim wide
     int gelu_tanh;
-    const int *pos0_dev;  // when set, the first position is read from device memory (replayable decode graph)
+    // when set, the first position of sequence b is pos0_dev[b] in device memory (replayable decode graph,
+    // sequences of different lengths)
+    const int *pos0_dev;
+    // packed (ragged) prefill: row r belongs to sequence row_seq[r] at position row_pos[r]
+    const int *row_seq, *row_pos;
 };
 
 struct GemmShape {
@@ -72,7 +76,8 @@ constexpr int SKINNY_MAX_ROWS = 32;
 int launch_gemm_naive(const GemmOperands &op, const GemmShape &shape, const EpiParams &epi, cudaStream_t stream);
 
 int launch_embed(const int32_t *ids, int n_tokens, int seqlen, int pos0, const uint16_t *wte, const uint16_t *wpe,
-                 int d, int vocab, float *out, uint32_t *status, cudaStream_t stream, const int *pos0_dev = nullptr);
+                 int d, int vocab, float *out, uint32_t *status, cudaStream_t stream, const int *pos0_dev = nullptr,
+                 const int *row_pos = nullptr);
 // y: [rows, d] added before normalisation (or NULL); alternatively ysum: `ysum_groups` tensors
 // [rows, d], ysum_gstride apart, whose sum is added.
 int launch_layernorm(const float *a, long long a_gstride, const float *y, const uint16_t *gamma,
@@ -114,7 +119,7 @@ struct DecodeAttnParams {
     long long cache_gstride, cache_bstride;
     int groups, batch, n_keys, n_head, head_dim, max_pos;
     int n_kv_head = 0;   // key/value heads in the cache (0 = n_head)
-    const int *pos_dev;  // when set, n_keys = *pos_dev + 1 (replayable decode graph)
+    const int *pos_dev;  // when set, sequence b has n_keys = pos_dev[b] + 1 (replayable decode graph, ragged batches)
     int splits;
     float *partials;  // [G*batch*n_head][splits][head_dim + 2] fp32 (max, sum, output); unused when splits == 1
     uint16_t *out;    // [G][batch, d]

@@ -267,6 +267,74 @@ def test_decode_branch_chains_any_branch_count(n_branch, one_chain, monkeypatch)
     m.close()
 
 
+# ------------------------------------------------------------------ packed batches (sequences of different lengths)
+
+@pytest.mark.parametrize("name,lens", [("C0", [37, 128 - 6, 1, 64]), ("K0-104", [300, 5]), ("C0-gqa", [129, 130])])
+def test_packed_prefill_and_ragged_decode(name, lens):
+    """Sequences of different lengths, packed without padding: every position of every sequence and its cache
+    rows against the oracle (which runs one sequence at a time), then teacher-forced decode steps that continue
+    every sequence at its own position; index work (which cache row a token lands in) is exact."""
+    s = ki.CONFIGS[name]
+    B = len(lens)
+    m, w = build(s, max_batch=B)
+    wb = host_bits(w)
+    steps = 5
+    seqs = [ki.uniform_tokens(30 + b, s.vocab, 1, L + steps, DEV)[0] for b, L in enumerate(lens)]
+    packed = torch.cat([q[:L] for q, L in zip(seqs, lens)]).contiguous()
+    last = m.prefill_packed(packed, lens).cpu().numpy()
+    assert m.device_status() == 0 and m.seq_lens(B) == lens and m.cur_len == max(lens)
+    allrows = m.logits_rows(list(range(sum(lens)))).cpu().numpy()
+    orcs, r0 = [], 0
+    for b, L in enumerate(lens):
+        ids = seqs[b][:L].cpu().numpy()
+        ref32, _ = oracle_all_logits(s, wb, ids, False)
+        refbf, orc = oracle_all_logits(s, wb, ids, True)
+        got = allrows[r0:r0 + L]
+        if L >= 16:
+            check_parity(got, ref32, refbf, f"{name} packed seq {b} (length {L})")
+        else:
+            rel, mx = logits_metrics(got, ref32)
+            assert rel <= REL_L2_MAX and mx <= MAX_ABS_MAX, (b, rel, mx)
+        assert np.allclose(last[b], got[-1], atol=3e-4)
+        for layer in (0, s.n_layer - 1):
+            for which in (0, 1):
+                g = m.kv_view(layer, s.n_branch - 1, which)[b, :, :L].float().cpu().numpy()
+                check_cache(g, orc.cache(layer, s.n_branch - 1, which), layer == 0 and L >= 16, (name, b, layer, which))
+        o2 = oracle.Oracle(s, wb, bf16_store=False)
+        o2.prefill(ids)
+        orcs.append(o2)
+        r0 += L
+    for t in range(steps):
+        toks = torch.stack([seqs[b][lens[b] + t] for b in range(B)]).contiguous()
+        got = m.decode_step(toks).cpu().numpy()
+        for b in range(B):
+            ref = orcs[b].decode_step(int(toks[b]))
+            rel, mx = logits_metrics(got[b], ref)
+            assert rel <= REL_L2_MAX and mx <= MAX_ABS_MAX, (name, t, b, rel, mx)
+    assert m.seq_lens(B) == [L + steps for L in lens] and m.device_status() == 0
+    m.close()
+
+
+def test_packed_prefill_of_equal_lengths_equals_the_uniform_call():
+    s = ki.CONFIGS["C0"]
+    B, L = 3, 70
+    tok = ki.uniform_tokens(9, s.vocab, B, L, DEV)
+    m, _ = build(s, max_batch=B)
+    uni = m.prefill(tok).clone()
+    ku = m.kv_view(s.n_layer - 1, 1, 0)[:, :, :L].clone()
+    m.reset()
+    pk = m.prefill_packed(tok.reshape(-1).contiguous(), [L] * B)
+    assert torch.equal(pk, uni)
+    assert torch.equal(m.kv_view(s.n_layer - 1, 1, 0)[:, :, :L], ku)
+    # a uniform call afterwards works as before
+    m.reset()
+    assert torch.equal(m.prefill(tok), uni)
+    with pytest.raises(kr.KrakenError) as e:
+        m.prefill_packed(tok.reshape(-1).contiguous()[:L], [L, 0])   # a zero length
+    assert e.value.status == kr.EINVAL
+    m.close()
+
+
 # ------------------------------------------------------------------ IEEE half as the 16-bit storage type
 
 @pytest.mark.parametrize("name", ["C0", "K0-104", "C0-gqa"])
