@@ -129,6 +129,39 @@ int kraken_prefill_host(kraken_handle *h, const int32_t *h_tokens, int32_t batch
 int kraken_prefill_packed(kraken_handle *h, const int32_t *d_tokens, const int32_t *h_seq_lens, int32_t batch,
                           float *d_logits, void *stream);
 
+/* ------------------------------------------------------------------------------------------
+ * Branch-parallel deployment (the paper's own: each device holds some of the N branches of every
+ * layer, Fig. 3 and App. A.2).  A handle created with the LOCAL branches' weights (n_branch = the
+ * number held here, w_concat = the columns of W_concat that multiply those branches, b_concat only
+ * on one device) is driven in pieces, so that the caller can sum the layer outputs over all devices
+ * (the AllReduce of Algorithm 1) while the next layer's attention half is already running - the
+ * overlap the paper builds its latency claim on (Sec. 3.1):
+ *
+ *   kraken_stage_begin(tokens)                      shared embedding x0 (identical on every device)
+ *   for layer l = 0 .. L-1:
+ *       kraken_stage_attention(l)                   LN1, qkv, attention, proj + residual
+ *       kraken_stage_ffn(l, y)                      LN2(. + y), up, GELU, down + residual; then the sum
+ *                                                   of this device's layer outputs is in d_local_sum
+ *           y = x0 for l = 0, else the sum over ALL devices of the d_local_sum of layer l-1
+ *           (the caller's all-reduce; it must be complete before kraken_stage_ffn(l) is enqueued
+ *           and may run while kraken_stage_attention(l) does)
+ *   kraken_stage_concat(z)                          this device's part of W_concat at the last positions
+ *   (caller: sum z over all devices)
+ *   kraken_stage_head(z, logits)                    final LayerNorm, unembedding; the prefill is then
+ *                                                   complete (cur_len = seqlen) and kraken_kv_view valid
+ *
+ * d_y, d_z: device fp32 [batch*seqlen, d] and [batch, d]; kraken_stage_buffers returns the device
+ * addresses of x0 and of the local-sum buffer ([batch*seqlen, d] fp32, overwritten by every
+ * kraken_stage_ffn).  Calls out of order return ESTATE.  With one device holding all branches the
+ * sequence computes exactly what kraken_prefill computes.  Decode steps in this mode are not built.
+ * ------------------------------------------------------------------------------------------ */
+int kraken_stage_begin(kraken_handle *h, const int32_t *d_tokens, int32_t batch, int32_t seqlen, void *stream);
+int kraken_stage_attention(kraken_handle *h, int32_t layer, void *stream);
+int kraken_stage_ffn(kraken_handle *h, int32_t layer, const float *d_y, void *stream);
+int kraken_stage_buffers(kraken_handle *h, float **d_x0, float **d_local_sum);
+int kraken_stage_concat(kraken_handle *h, float *d_z, void *stream);
+int kraken_stage_head(kraken_handle *h, const float *d_z, float *d_logits, void *stream);
+
 /* Current length of every cached sequence (host array of `batch` entries; kraken_cur_len is their maximum).
  * ESTATE when batch differs from the cached batch. */
 int kraken_seq_lens(kraken_handle *h, int32_t *h_seq_lens, int32_t batch);

@@ -33,7 +33,9 @@ PROF_COUNT = len(PROF_CATEGORIES)
 
 EXPORTS = (
     "kraken_query_sizes", "kraken_create", "kraken_prefill", "kraken_prefill_host",
-    "kraken_prefill_all_logits", "kraken_prefill_packed", "kraken_seq_lens", "kraken_logits_rows", "kraken_decode_step", "kraken_decode_step_host", "kraken_kv_view",
+    "kraken_prefill_all_logits", "kraken_prefill_packed", "kraken_seq_lens", "kraken_logits_rows",
+    "kraken_stage_begin", "kraken_stage_attention", "kraken_stage_ffn", "kraken_stage_buffers", "kraken_stage_concat",
+    "kraken_stage_head", "kraken_decode_step", "kraken_decode_step_host", "kraken_kv_view",
     "kraken_device_status", "kraken_cur_len", "kraken_profile_enable", "kraken_profile_read", "kraken_reset", "kraken_destroy", "kraken_strerror", "kraken_last_cuda_error",
     "kraken_op_embed", "kraken_op_layernorm", "kraken_op_grouped_gemm", "kraken_op_attention",
     "kraken_op_decode_attention", "kraken_decode_attention_sizes",
@@ -115,6 +117,12 @@ def lib(dtype: Optional[str] = None) -> C.CDLL:
         L.kraken_prefill_all_logits.argtypes = [vp, vp, i32, i32, vp, vp]
         L.kraken_prefill_packed.argtypes = [vp, vp, vp, i32, vp, vp]
         L.kraken_seq_lens.argtypes = [vp, vp, i32]
+        L.kraken_stage_begin.argtypes = [vp, vp, i32, i32, vp]
+        L.kraken_stage_attention.argtypes = [vp, i32, vp]
+        L.kraken_stage_ffn.argtypes = [vp, i32, vp, vp]
+        L.kraken_stage_buffers.argtypes = [vp, C.POINTER(vp), C.POINTER(vp)]
+        L.kraken_stage_concat.argtypes = [vp, vp, vp]
+        L.kraken_stage_head.argtypes = [vp, vp, vp, vp]
         L.kraken_logits_rows.argtypes = [vp, vp, i32, vp, vp]
         L.kraken_decode_step.argtypes = [vp, vp, i32, vp, vp]
         L.kraken_decode_step_host.argtypes = [vp, vp, i32, vp, vp]
@@ -253,6 +261,46 @@ class KrakenModel:
             logits = torch.empty(b, self.cfg.vocab, dtype=torch.float32, device=self.device)
         _check(lib(self.dtype).kraken_prefill_packed(self._h, tokens.data_ptr(), lens.data_ptr(), b, logits.data_ptr(),
                                                      _stream()), "kraken_prefill_packed")
+        return logits
+
+    # -------- the path in pieces, for the branch-parallel deployment (see branch_parallel.py)
+    def stage_begin(self, tokens: torch.Tensor):
+        b, l = tokens.shape
+        assert tokens.dtype == torch.int32 and tokens.is_contiguous() and tokens.device == self.device
+        _check(lib(self.dtype).kraken_stage_begin(self._h, tokens.data_ptr(), b, l, _stream()), "kraken_stage_begin")
+        self._stage_shape = (b, l)
+
+    def stage_attention(self, layer: int):
+        _check(lib(self.dtype).kraken_stage_attention(self._h, layer, _stream()), "kraken_stage_attention")
+
+    def stage_ffn(self, layer: int, y: torch.Tensor):
+        assert y.dtype == torch.float32 and y.is_contiguous() and y.device == self.device
+        _check(lib(self.dtype).kraken_stage_ffn(self._h, layer, y.data_ptr(), _stream()), "kraken_stage_ffn")
+
+    def stage_buffers(self):
+        """(x0, local_sum): fp32 [batch*seqlen, d] views of the shared embedding and of the sum of this
+        handle's layer outputs (rewritten by every stage_ffn)."""
+        p0, p1 = C.c_void_p(), C.c_void_p()
+        _check(lib(self.dtype).kraken_stage_buffers(self._h, C.byref(p0), C.byref(p1)), "kraken_stage_buffers")
+        b, l = self._stage_shape
+        flat = self.scratch.view(torch.float32)
+        base = self.scratch.data_ptr()
+        n = b * l * self.cfg.d_model
+        return (flat[(p0.value - base) // 4:(p0.value - base) // 4 + n].view(b * l, self.cfg.d_model),
+                flat[(p1.value - base) // 4:(p1.value - base) // 4 + n].view(b * l, self.cfg.d_model))
+
+    def stage_concat(self) -> torch.Tensor:
+        b, _ = self._stage_shape
+        z = torch.empty(b, self.cfg.d_model, dtype=torch.float32, device=self.device)
+        _check(lib(self.dtype).kraken_stage_concat(self._h, z.data_ptr(), _stream()), "kraken_stage_concat")
+        return z
+
+    def stage_head(self, z: torch.Tensor, logits: Optional[torch.Tensor] = None) -> torch.Tensor:
+        b, _ = self._stage_shape
+        assert z.dtype == torch.float32 and z.is_contiguous() and z.device == self.device
+        if logits is None:
+            logits = torch.empty(b, self.cfg.vocab, dtype=torch.float32, device=self.device)
+        _check(lib(self.dtype).kraken_stage_head(self._h, z.data_ptr(), logits.data_ptr(), _stream()), "kraken_stage_head")
         return logits
 
     def seq_lens(self, batch: int):

@@ -96,6 +96,7 @@ struct kraken_handle {
     // length of every cached sequence (cur_len is their maximum); ragged = they differ, set by a packed prefill
     std::vector<int> seq_len;
     bool ragged;
+    int stage_layer_done;   // branch-parallel driving: the last layer whose FFN half has run (-1: none)
     std::vector<int> host_rows, host_row_seq, host_row_pos;   // staging of the packed-prefill tables
     cudaStream_t last_stream;
     bool naive;
@@ -179,7 +180,12 @@ struct RunCtx {
     // seqlen is then the longest length
     bool packed;
     const int *row_seq, *row_pos;
+    // branch-parallel deployment: the path is driven in pieces (kraken_stage_*): 0 = the whole path,
+    // STAGE_EMBED, STAGE_ATTN / STAGE_FFN = one half of layer stage_layer; y_ext = the cross-device sum for LN2
+    int stage, stage_layer;
+    const float *y_ext;
 };
+enum { STAGE_ALL = 0, STAGE_EMBED = 1, STAGE_ATTN = 2, STAGE_FFN = 3 };
 
 // One grouped GEMM of the model: weights of `kind` at `layer`.
 // g0 / gcnt: a run of branches (gcnt = 0: all of them; the caller then passes A and the epilogue's pointers
@@ -281,15 +287,19 @@ int run_layers(const RunCtx &rc, const int32_t *d_tokens) {
     const long long cache_kv = (long long)c.max_batch * cache_b;  // all of K (or V) of one (layer, branch)
     uint16_t *kv = reinterpret_cast<uint16_t *>(h->kv);
 
-    {
+    if (rc.stage == STAGE_ALL || rc.stage == STAGE_EMBED) {
         LaunchScope scope(h, KRAKEN_PROF_EMBED, rc.st);
         KR_TRY(launch_embed(d_tokens, T, rc.seqlen, rc.pos0, (const uint16_t *)h->w.wte, (const uint16_t *)h->w.wpe, d,
                             c.vocab, x0, status, rc.st, rc.pos_dev, rc.row_pos));
     }
-    for (int l = 0; l < L; ++l) {
+    if (rc.stage == STAGE_EMBED) return KRAKEN_OK;
+    const int l_begin = rc.stage ? rc.stage_layer : 0, l_end = rc.stage ? rc.stage_layer + 1 : L;
+    for (int l = l_begin; l < l_end; ++l) {
         const float *xin = l == 0 ? x0 : x;
         const long long xin_gs = l == 0 ? 0 : td;
         const long long ln_off = (long long)l * N * d;
+        EpiParams e = epi_zero();
+        if (rc.stage != STAGE_FFN) {
         // x = LN(x)
         {
             LaunchScope scope(h, KRAKEN_PROF_LAYERNORM, rc.st);
@@ -299,7 +309,7 @@ int run_layers(const RunCtx &rc, const int32_t *d_tokens) {
         }
         // q | k | v ; K and V go straight into the cache
         uint16_t *kc = kv + (long long)l * N * 2 * cache_kv;
-        EpiParams e = epi_zero();
+        e = epi_zero();
         e.kind = KRAKEN_EPI_QKV;
         e.out_bf16 = q; e.out_bf16_gstride = td; e.ld_out_bf16 = d;
         e.k_cache = kc; e.v_cache = kc + cache_kv; e.cache_gstride = 2 * cache_kv;
@@ -368,9 +378,17 @@ int run_layers(const RunCtx &rc, const int32_t *d_tokens) {
         e.out_f32 = a; e.out_f32_gstride = td; e.ld_out_f32 = d;
         e.resid = xin; e.resid_gstride = xin_gs; e.ld_resid = d;
         KR_TRY(model_gemm(rc, G_PROJ, l, T, o, td, e));
+        }  // attention half
+        if (rc.stage == STAGE_ATTN) continue;
         // x = LN(x + y): y is the shared embedding in the first layer, the cross-branch sum afterwards
         // (the parallel variant feeds the FFN with the first LayerNorm's output, still in u)
-        if (!c.parallel_ffn) {
+        if (rc.stage == STAGE_FFN) {
+            // driven from outside: y is whatever the caller summed over all devices (layer 1: the embedding)
+            LaunchScope scope(h, KRAKEN_PROF_LAYERNORM, rc.st);
+            KR_TRY(launch_layernorm(a, td, rc.y_ext, (const uint16_t *)h->w.ln2_g + ln_off,
+                                    h->w.ln2_b ? (const uint16_t *)h->w.ln2_b + ln_off : nullptr, N, T, d, c.ln_eps,
+                                    u, rc.st, nullptr, 0, 0, status));
+        } else if (!c.parallel_ffn) {
             LaunchScope scope(h, KRAKEN_PROF_LAYERNORM, rc.st);
             // with few rows the cross-branch sum is formed here from the N branch inputs (same order as
             // the down-projection epilogue forms it for long prompts)
@@ -387,12 +405,13 @@ int run_layers(const RunCtx &rc, const int32_t *d_tokens) {
         KR_TRY(model_gemm(rc, G_UP, l, T, u, td, e));
         // out = res + FFN ; the sum over branches (the AllReduce feeding the next layer) in the epilogue
         e = epi_zero();
-        e.kind = (l + 1 < L && !small_rows && !c.no_combine) ? KRAKEN_EPI_RESID_SUM : KRAKEN_EPI_RESID_F32;
+        e.kind = (l + 1 < L && !small_rows && !c.no_combine && !rc.stage) ? KRAKEN_EPI_RESID_SUM : KRAKEN_EPI_RESID_F32;
         e.out_f32 = x; e.out_f32_gstride = td; e.ld_out_f32 = d;
         e.resid = a; e.resid_gstride = td; e.ld_resid = d;
         e.sum = S; e.ld_sum = d;
         KR_TRY(model_gemm(rc, G_DOWN, l, T, gb, (long long)T * F, e));
-        if (sum_pass && l + 1 < L && !c.no_combine) {
+        if ((sum_pass && l + 1 < L && !c.no_combine) || rc.stage == STAGE_FFN) {
+            // (driven from outside: the sum of this device's branches, for the caller's all-reduce)
             LaunchScope scope(h, KRAKEN_PROF_LAYERNORM, rc.st);
             KR_TRY(launch_sum_groups(x, td, N, td, S, rc.st));
         }
@@ -568,13 +587,14 @@ __global__ void make_rows_kernel(int32_t *rows, int n, int mul, int add) {
 }
 
 // W_concat, final LayerNorm and the tied unembedding for n_rows token rows (device index list).
-int run_tail(const RunCtx &rc, const int32_t *d_rows, int n_rows, float *d_logits) {
+// W_concat over the chosen rows of the last layer's outputs: z [n_rows, d] fp32.
+int tail_concat(const RunCtx &rc, const int32_t *d_rows, int n_rows, float *z) {
     kraken_handle *h = rc.h;
     const kraken_config &c = h->cfg;
     const int d = c.d_model, N = c.n_branch;
     const long long td = (long long)h->last_rows * d;
-    float *x = at<float>(h, h->lay.x), *z = at<float>(h, h->lay.s);
-    uint16_t *cat = at<uint16_t>(h, h->lay.u), *zf = at<uint16_t>(h, h->lay.q);
+    float *x = at<float>(h, h->lay.x);
+    uint16_t *cat = at<uint16_t>(h, h->lay.u);
     {
         LaunchScope scope(h, KRAKEN_PROF_TAIL, rc.st);
         KR_TRY(launch_gather_concat(x, td, N, d, d_rows, n_rows, cat, rc.st));
@@ -582,7 +602,15 @@ int run_tail(const RunCtx &rc, const int32_t *d_rows, int n_rows, float *d_logit
     EpiParams e = epi_zero();
     e.kind = KRAKEN_EPI_F32;
     e.out_f32 = z; e.ld_out_f32 = d;
-    KR_TRY(model_gemm(rc, G_CONCAT, 0, n_rows, cat, 0, e));
+    return model_gemm(rc, G_CONCAT, 0, n_rows, cat, 0, e);
+}
+
+// Final LayerNorm (if configured) and the tied unembedding of z [n_rows, d].
+int tail_head(const RunCtx &rc, const float *z, int n_rows, float *d_logits) {
+    kraken_handle *h = rc.h;
+    const kraken_config &c = h->cfg;
+    const int d = c.d_model;
+    uint16_t *zf = at<uint16_t>(h, h->lay.q);
     {
         LaunchScope scope(h, KRAKEN_PROF_TAIL, rc.st);
         if (c.final_ln) {
@@ -592,11 +620,16 @@ int run_tail(const RunCtx &rc, const int32_t *d_rows, int n_rows, float *d_logit
             KR_TRY(launch_f32_to_bf16(z, zf, (long long)n_rows * d, rc.st));
         }
     }
-    e = epi_zero();
+    EpiParams e = epi_zero();
     e.kind = KRAKEN_EPI_F32;
     e.out_f32 = d_logits; e.ld_out_f32 = c.vocab;
-    KR_TRY(model_gemm(rc, G_HEAD, 0, n_rows, zf, 0, e));
-    return KRAKEN_OK;
+    return model_gemm(rc, G_HEAD, 0, n_rows, zf, 0, e);
+}
+
+int run_tail(const RunCtx &rc, const int32_t *d_rows, int n_rows, float *d_logits) {
+    float *z = at<float>(rc.h, rc.h->lay.s);
+    KR_TRY(tail_concat(rc, d_rows, n_rows, z));
+    return tail_head(rc, z, n_rows, d_logits);
 }
 
 // The kernel sequence of one prefill on stream st.
@@ -778,6 +811,7 @@ int kraken_create(const kraken_config *cfg, const kraken_weights *w, void *d_kv,
     h->cap_stream = nullptr;
     h->br_ready = false;
     h->ragged = false;
+    h->stage_layer_done = -1;
     h->dec_graph_batch = 0;
     h->dec_eager_steps = 0;
     h->use_graph = !env_flag("KRAKEN_NO_GRAPH") && !h->naive;
@@ -803,6 +837,85 @@ int kraken_prefill(kraken_handle *h, const int32_t *d_tokens, int32_t batch, int
 int kraken_prefill_packed(kraken_handle *h, const int32_t *d_tokens, const int32_t *h_seq_lens, int32_t batch,
                           float *d_logits, void *stream) {
     return prefill_packed(h, d_tokens, h_seq_lens, batch, d_logits, stream);
+}
+
+// ---- branch-parallel deployment: the path in pieces (see kraken.h)
+
+int kraken_stage_begin(kraken_handle *h, const int32_t *d_tokens, int32_t batch, int32_t seqlen, void *stream) {
+    if (!h || !d_tokens || batch < 1 || seqlen < 1) return KRAKEN_EINVAL;
+    if (batch > h->cfg.max_batch || seqlen > h->cfg.max_pos) return KRAKEN_ECAPACITY;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    h->last_stream = st;
+    if (h->pre_graph) cudaGraphExecDestroy(h->pre_graph);
+    h->pre_graph = nullptr;
+    h->pre_tokens = nullptr;
+    h->pre_seen = 0;
+    h->cur_len = 0;                       // nothing is cached until kraken_stage_head has run
+    h->batch = batch;
+    h->last_seqlen = seqlen;
+    h->stage_layer_done = -1;
+    RunCtx rc{h, st, batch, seqlen, 0, batch * seqlen, nullptr, 0, false, nullptr, nullptr, STAGE_EMBED, 0, nullptr};
+    KR_TRY(run_layers(rc, d_tokens));
+    h->last_rows = batch * seqlen;
+    return KRAKEN_OK;
+}
+
+int kraken_stage_attention(kraken_handle *h, int32_t layer, void *stream) {
+    if (!h || layer < 0 || layer >= h->cfg.n_layer) return KRAKEN_EINVAL;
+    if (h->batch < 1 || h->last_seqlen < 1 || layer != h->stage_layer_done + 1) return KRAKEN_ESTATE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    h->last_stream = st;
+    RunCtx rc{h, st, h->batch, h->last_seqlen, 0, h->batch * h->last_seqlen, nullptr, 0, false, nullptr, nullptr,
+              STAGE_ATTN, layer, nullptr};
+    return run_layers(rc, nullptr);
+}
+
+int kraken_stage_ffn(kraken_handle *h, int32_t layer, const float *d_y, void *stream) {
+    if (!h || layer < 0 || layer >= h->cfg.n_layer || !d_y) return KRAKEN_EINVAL;
+    if (h->batch < 1 || h->last_seqlen < 1 || layer != h->stage_layer_done + 1) return KRAKEN_ESTATE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    h->last_stream = st;
+    RunCtx rc{h, st, h->batch, h->last_seqlen, 0, h->batch * h->last_seqlen, nullptr, 0, false, nullptr, nullptr,
+              STAGE_FFN, layer, d_y};
+    KR_TRY(run_layers(rc, nullptr));
+    h->stage_layer_done = layer;
+    return KRAKEN_OK;
+}
+
+int kraken_stage_buffers(kraken_handle *h, float **d_x0, float **d_local_sum) {
+    if (!h || !d_x0 || !d_local_sum) return KRAKEN_EINVAL;
+    *d_x0 = at<float>(h, h->lay.x0);
+    *d_local_sum = at<float>(h, h->lay.s);
+    return KRAKEN_OK;
+}
+
+int kraken_stage_concat(kraken_handle *h, float *d_z, void *stream) {
+    if (!h || !d_z) return KRAKEN_EINVAL;
+    if (h->batch < 1 || h->stage_layer_done != h->cfg.n_layer - 1) return KRAKEN_ESTATE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    h->last_stream = st;
+    RunCtx rc{h, st, h->batch, h->last_seqlen, 0, h->batch * h->last_seqlen, nullptr, 0, false, nullptr, nullptr, 0, 0,
+              nullptr};
+    int32_t *rows = at<int32_t>(h, h->lay.rows);
+    h->launches[KRAKEN_PROF_TAIL]++;
+    make_rows_kernel<<<(h->batch + 255) / 256, 256, 0, st>>>(rows, h->batch, h->last_seqlen, h->last_seqlen - 1);
+    if (cudaGetLastError() != cudaSuccess) return KRAKEN_ECUDA;
+    return tail_concat(rc, rows, h->batch, d_z);
+}
+
+int kraken_stage_head(kraken_handle *h, const float *d_z, float *d_logits, void *stream) {
+    if (!h || !d_z || !d_logits) return KRAKEN_EINVAL;
+    if (h->batch < 1 || h->stage_layer_done != h->cfg.n_layer - 1) return KRAKEN_ESTATE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    h->last_stream = st;
+    RunCtx rc{h, st, h->batch, h->last_seqlen, 0, h->batch * h->last_seqlen, nullptr, 0, false, nullptr, nullptr, 0, 0,
+              nullptr};
+    KR_TRY(tail_head(rc, d_z, h->batch, d_logits));
+    set_pos_kernel<<<1, 64, 0, st>>>(at<int>(h, h->lay.pos_arr), h->last_seqlen, h->batch);
+    h->cur_len = h->last_seqlen;
+    h->seq_len.assign(h->batch, h->last_seqlen);
+    h->ragged = false;
+    return cuda_check(cudaGetLastError(), "stage head: position update");
 }
 
 int kraken_seq_lens(kraken_handle *h, int32_t *h_seq_lens, int32_t batch) {
