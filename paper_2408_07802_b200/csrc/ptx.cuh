@@ -93,7 +93,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volati
     return true;
 }
 
-// ---------------------------------------------------------------- TMA (tile mode, no multicast)
+// ---------------------------------------------------------------- TMA (tile mode; every load is for the issuing CTA alone)
 
 __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap *map) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
