@@ -335,6 +335,46 @@ def test_packed_prefill_of_equal_lengths_equals_the_uniform_call():
     m.close()
 
 
+def test_call_sequences_on_one_handle_match_fresh_handles():
+    """One handle driven through uniform prefill, decode steps, a packed prefill, more decode steps, a reset and
+    a repeated prefill (graph replay) gives at every point what a fresh handle gives for the same call."""
+    s = ki.CONFIGS["C0-gqa"]
+    B = 2
+    w = ki.make_weights(s, seed=0, device=DEV)
+    tok = ki.uniform_tokens(40, s.vocab, B, 90, DEV)
+
+    def fresh():
+        return kr.KrakenModel(kr.make_config(s, max_batch=B), w, DEV)
+
+    m = fresh()
+    a1 = m.prefill(tok[:, :60].contiguous()).clone()
+    d1 = [m.decode_step(tok[:, 60 + i].contiguous()).clone() for i in range(3)]
+    lens = [50, 17]
+    packed = torch.cat([tok[0, :50], tok[1, :17]]).contiguous()
+    p1 = m.prefill_packed(packed, lens).clone()
+    d2 = [m.decode_step(torch.stack([tok[0, 50 + i], tok[1, 17 + i]]).contiguous()).clone() for i in range(3)]
+    m.reset()
+    a2 = [m.prefill(tok[:, :60].contiguous()).clone() for _ in range(3)]      # third call replays the graph
+    d3 = m.decode_step(tok[:, 60].contiguous()).clone()
+    assert m.device_status() == 0
+
+    f = fresh()
+    assert torch.equal(f.prefill(tok[:, :60].contiguous()), a1)
+    for i in range(3):
+        assert torch.equal(f.decode_step(tok[:, 60 + i].contiguous()), d1[i]), i
+    f.close()
+    f = fresh()
+    assert torch.equal(f.prefill_packed(packed, lens), p1)
+    for i in range(3):
+        got = f.decode_step(torch.stack([tok[0, 50 + i], tok[1, 17 + i]]).contiguous())
+        assert torch.equal(got, d2[i]), i
+    f.close()
+    for x in a2:
+        assert torch.equal(x, a1)
+    assert torch.equal(d3, d1[0])
+    m.close()
+
+
 # ------------------------------------------------------------------ IEEE half as the 16-bit storage type
 
 @pytest.mark.parametrize("name", ["C0", "K0-104", "C0-gqa"])
