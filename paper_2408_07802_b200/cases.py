@@ -78,7 +78,7 @@ def _gemm_args(kind, s, batch, seqlen, n_tile=0):
 
 
 def run_case(kind: str, workload: str, reps: int, warmup: int, n_tile: int = 0, batch=None, seqlen=None,
-             graph_launches: int = 0):
+             graph_launches: int = 0, kv_heads: int = 0):
     s = ki.CONFIGS[workload]
     batch = batch or s.batch
     seqlen = seqlen or s.seqlen
@@ -104,14 +104,15 @@ def run_case(kind: str, workload: str, reps: int, warmup: int, n_tile: int = 0, 
         byts = 4 * N * T * d * 2
     elif kind == "decode_attention":
         ctx = seqlen
+        Hkv = kv_heads or s.kv_heads          # fewer key/value heads than heads: grouped-query attention
         q = ki.normal_bf16(12, 0, (N, batch, d), 1.0, DEV)
-        kc = ki.normal_bf16(12, 1, (N, batch, H, ctx, hd), 1.0, DEV)
-        vc = ki.normal_bf16(12, 2, (N, batch, H, ctx, hd), 1.0, DEV)
+        kc = ki.normal_bf16(12, 1, (N, batch, Hkv, ctx, hd), 1.0, DEV)
+        vc = ki.normal_bf16(12, 2, (N, batch, Hkv, ctx, hd), 1.0, DEV)
         sp, nb = kr.decode_attention_sizes(N, batch, ctx, H, hd, n_tile)
         part = torch.empty(max(nb, 16), dtype=torch.uint8, device=DEV)
         fn = lambda: kr.op_decode_attention(q, kc, vc, ctx, sp, part)
         flops = 4.0 * N * batch * ctx * d
-        byts = 2 * N * batch * ctx * d * 2 + 2 * N * batch * d * 2
+        byts = 2 * N * batch * ctx * Hkv * hd * 2 + 2 * N * batch * d * 2
     elif kind == "layernorm":
         a = ki.normal_bf16(13, 0, (N, T, d), 1.0, DEV).float()
         y = ki.normal_bf16(13, 1, (T, d), 1.0, DEV).float()
@@ -163,6 +164,7 @@ def main():
     ap.add_argument("--batch", type=int, default=None)
     ap.add_argument("--seqlen", type=int, default=None)
     ap.add_argument("--graph", type=int, default=0, help="time this many launches replayed from one CUDA graph")
+    ap.add_argument("--kv-heads", type=int, default=0, help="key/value heads of decode_attention (default: the workload's)")
     a = ap.parse_args()
     kinds = [a.case]
     if a.case == "all":
@@ -170,7 +172,7 @@ def main():
     elif a.case == "decode_all":
         kinds = ["decode_gemm_qkv", "decode_gemm_proj", "decode_gemm_up", "decode_gemm_down", "decode_attention"]
     for k in kinds:
-        run_case(k, a.workload, a.reps, a.warmup, a.n_tile, a.batch, a.seqlen, a.graph)
+        run_case(k, a.workload, a.reps, a.warmup, a.n_tile, a.batch, a.seqlen, a.graph, a.kv_heads)
 
 
 if __name__ == "__main__":
