@@ -153,9 +153,12 @@ int kraken_prefill_packed(kraken_handle *h, const int32_t *d_tokens, const int32
  * d_y, d_z: device fp32 [batch*seqlen, d] and [batch, d]; kraken_stage_buffers returns the device
  * addresses of x0 and of the local-sum buffer ([batch*seqlen, d] fp32, overwritten by every
  * kraken_stage_ffn).  Calls out of order return ESTATE.  With one device holding all branches the
- * sequence computes exactly what kraken_prefill computes.  Decode steps in this mode are not built.
+ * sequence computes exactly what kraken_prefill computes.  A decode step is driven the same way after
+ * kraken_stage_begin_decode(tokens [batch]) (one new token per sequence; d_y and the local sum are then
+ * [batch, d]); its kraken_stage_head advances every sequence by one position.
  * ------------------------------------------------------------------------------------------ */
 int kraken_stage_begin(kraken_handle *h, const int32_t *d_tokens, int32_t batch, int32_t seqlen, void *stream);
+int kraken_stage_begin_decode(kraken_handle *h, const int32_t *d_tokens, int32_t batch, void *stream);
 int kraken_stage_attention(kraken_handle *h, int32_t layer, void *stream);
 int kraken_stage_ffn(kraken_handle *h, int32_t layer, const float *d_y, void *stream);
 int kraken_stage_buffers(kraken_handle *h, float **d_x0, float **d_local_sum);

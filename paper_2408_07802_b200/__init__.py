@@ -34,7 +34,7 @@ PROF_COUNT = len(PROF_CATEGORIES)
 EXPORTS = (
     "kraken_query_sizes", "kraken_create", "kraken_prefill", "kraken_prefill_host",
     "kraken_prefill_all_logits", "kraken_prefill_packed", "kraken_seq_lens", "kraken_logits_rows",
-    "kraken_stage_begin", "kraken_stage_attention", "kraken_stage_ffn", "kraken_stage_buffers", "kraken_stage_concat",
+    "kraken_stage_begin", "kraken_stage_begin_decode", "kraken_stage_attention", "kraken_stage_ffn", "kraken_stage_buffers", "kraken_stage_concat",
     "kraken_stage_head", "kraken_decode_step", "kraken_decode_step_host", "kraken_kv_view",
     "kraken_device_status", "kraken_cur_len", "kraken_profile_enable", "kraken_profile_read", "kraken_reset", "kraken_destroy", "kraken_strerror", "kraken_last_cuda_error",
     "kraken_op_embed", "kraken_op_layernorm", "kraken_op_grouped_gemm", "kraken_op_attention",
@@ -118,6 +118,7 @@ def lib(dtype: Optional[str] = None) -> C.CDLL:
         L.kraken_prefill_packed.argtypes = [vp, vp, vp, i32, vp, vp]
         L.kraken_seq_lens.argtypes = [vp, vp, i32]
         L.kraken_stage_begin.argtypes = [vp, vp, i32, i32, vp]
+        L.kraken_stage_begin_decode.argtypes = [vp, vp, i32, vp]
         L.kraken_stage_attention.argtypes = [vp, i32, vp]
         L.kraken_stage_ffn.argtypes = [vp, i32, vp, vp]
         L.kraken_stage_buffers.argtypes = [vp, C.POINTER(vp), C.POINTER(vp)]
@@ -269,6 +270,12 @@ class KrakenModel:
         assert tokens.dtype == torch.int32 and tokens.is_contiguous() and tokens.device == self.device
         _check(lib(self.dtype).kraken_stage_begin(self._h, tokens.data_ptr(), b, l, _stream()), "kraken_stage_begin")
         self._stage_shape = (b, l)
+
+    def stage_begin_decode(self, tokens: torch.Tensor):
+        assert tokens.dtype == torch.int32 and tokens.is_contiguous() and tokens.device == self.device
+        _check(lib(self.dtype).kraken_stage_begin_decode(self._h, tokens.data_ptr(), tokens.numel(), _stream()),
+               "kraken_stage_begin_decode")
+        self._stage_shape = (tokens.numel(), 1)
 
     def stage_attention(self, layer: int):
         _check(lib(self.dtype).kraken_stage_attention(self._h, layer, _stream()), "kraken_stage_attention")

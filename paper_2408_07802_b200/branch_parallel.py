@@ -66,8 +66,16 @@ class BranchParallelPrefill:
         self.n_layer = n_layer
 
     def prefill(self, tokens: torch.Tensor) -> torch.Tensor:
+        self.engine.stage_begin(tokens)
+        return self._run()
+
+    def decode_step(self, tokens: torch.Tensor) -> torch.Tensor:
+        """One new token per sequence, after a prefill: the same order of pieces on [batch, d] tensors."""
+        self.engine.stage_begin_decode(tokens)
+        return self._run()
+
+    def _run(self) -> torch.Tensor:
         e, g = self.engine, self.group
-        e.stage_begin(tokens)
         x0, local_sum = e.stage_buffers()
         bufs = [torch.empty_like(local_sum), torch.empty_like(local_sum)]
         y, pending = x0, None                       # layer 1: the AllReduce is the identity (Algorithm 1)
@@ -86,12 +94,15 @@ class BranchParallelPrefill:
         return e.stage_head(z)
 
 
-def lockstep_prefill(engines, n_layer: int, tokens: torch.Tensor) -> List[torch.Tensor]:
+def lockstep_prefill(engines, n_layer: int, tokens: torch.Tensor, decode: bool = False) -> List[torch.Tensor]:
     """The same order of pieces as BranchParallelPrefill, for all ranks in one process: every piece is run for
     rank 0, 1, ... in turn and the all-reduce is an in-order sum (rank 0 first, the order in which a single
-    device adds its branches)."""
+    device adds its branches).  decode: `tokens` is one new token per sequence after a prefill."""
     for e in engines:
-        e.stage_begin(tokens)
+        if decode:
+            e.stage_begin_decode(tokens)
+        else:
+            e.stage_begin(tokens)
     bufs = [e.stage_buffers() for e in engines]
     ys = [x0 for x0, _ in bufs]
     for layer in range(n_layer):

@@ -97,6 +97,7 @@ struct kraken_handle {
     std::vector<int> seq_len;
     bool ragged;
     int stage_layer_done;   // branch-parallel driving: the last layer whose FFN half has run (-1: none)
+    bool stage_decode;      // the pieces being driven are a decode step (one new token per sequence)
     std::vector<int> host_rows, host_row_seq, host_row_pos;   // staging of the packed-prefill tables
     cudaStream_t last_stream;
     bool naive;
@@ -569,6 +570,11 @@ int run_layers_decode_branches(const RunCtx &rc, const int32_t *d_tokens) {
     return KRAKEN_OK;
 }
 
+void advance_lengths(kraken_handle *h) {
+    h->cur_len += 1;
+    for (int &v : h->seq_len) v += 1;
+}
+
 // The next position of every sequence lives in device memory (the decode graph reads it there).
 __global__ void set_pos_kernel(int *pos, int value, int batch) {
     pdl_wait();
@@ -812,6 +818,7 @@ int kraken_create(const kraken_config *cfg, const kraken_weights *w, void *d_kv,
     h->br_ready = false;
     h->ragged = false;
     h->stage_layer_done = -1;
+    h->stage_decode = false;
     h->dec_graph_batch = 0;
     h->dec_eager_steps = 0;
     h->use_graph = !env_flag("KRAKEN_NO_GRAPH") && !h->naive;
@@ -841,6 +848,16 @@ int kraken_prefill_packed(kraken_handle *h, const int32_t *d_tokens, const int32
 
 // ---- branch-parallel deployment: the path in pieces (see kraken.h)
 
+// Run context of one piece: a prefill of batch x last_seqlen tokens at position 0, or a decode step whose
+// positions come from the device array.
+static RunCtx stage_ctx(kraken_handle *h, cudaStream_t st, int stage, int layer, const float *y) {
+    if (h->stage_decode)
+        return RunCtx{h, st, h->batch, 1, h->cur_len, h->batch, at<int>(h, h->lay.pos_arr), h->cfg.max_pos,
+                      false, nullptr, nullptr, stage, layer, y};
+    return RunCtx{h, st, h->batch, h->last_seqlen, 0, h->batch * h->last_seqlen, nullptr, 0,
+                  false, nullptr, nullptr, stage, layer, y};
+}
+
 int kraken_stage_begin(kraken_handle *h, const int32_t *d_tokens, int32_t batch, int32_t seqlen, void *stream) {
     if (!h || !d_tokens || batch < 1 || seqlen < 1) return KRAKEN_EINVAL;
     if (batch > h->cfg.max_batch || seqlen > h->cfg.max_pos) return KRAKEN_ECAPACITY;
@@ -854,9 +871,25 @@ int kraken_stage_begin(kraken_handle *h, const int32_t *d_tokens, int32_t batch,
     h->batch = batch;
     h->last_seqlen = seqlen;
     h->stage_layer_done = -1;
+    h->stage_decode = false;
     RunCtx rc{h, st, batch, seqlen, 0, batch * seqlen, nullptr, 0, false, nullptr, nullptr, STAGE_EMBED, 0, nullptr};
     KR_TRY(run_layers(rc, d_tokens));
     h->last_rows = batch * seqlen;
+    return KRAKEN_OK;
+}
+
+int kraken_stage_begin_decode(kraken_handle *h, const int32_t *d_tokens, int32_t batch, void *stream) {
+    if (!h || !d_tokens || batch < 1) return KRAKEN_EINVAL;
+    if (h->cur_len < 1 || batch != h->batch) return KRAKEN_ESTATE;
+    if (h->cur_len + 1 > h->cfg.max_pos) return KRAKEN_ECAPACITY;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    h->last_stream = st;
+    h->last_seqlen = 1;
+    h->stage_layer_done = -1;
+    h->stage_decode = true;
+    RunCtx rc = stage_ctx(h, st, STAGE_EMBED, 0, nullptr);
+    KR_TRY(run_layers(rc, d_tokens));
+    h->last_rows = batch;
     return KRAKEN_OK;
 }
 
@@ -865,8 +898,7 @@ int kraken_stage_attention(kraken_handle *h, int32_t layer, void *stream) {
     if (h->batch < 1 || h->last_seqlen < 1 || layer != h->stage_layer_done + 1) return KRAKEN_ESTATE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     h->last_stream = st;
-    RunCtx rc{h, st, h->batch, h->last_seqlen, 0, h->batch * h->last_seqlen, nullptr, 0, false, nullptr, nullptr,
-              STAGE_ATTN, layer, nullptr};
+    RunCtx rc = stage_ctx(h, st, STAGE_ATTN, layer, nullptr);
     return run_layers(rc, nullptr);
 }
 
@@ -875,8 +907,7 @@ int kraken_stage_ffn(kraken_handle *h, int32_t layer, const float *d_y, void *st
     if (h->batch < 1 || h->last_seqlen < 1 || layer != h->stage_layer_done + 1) return KRAKEN_ESTATE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     h->last_stream = st;
-    RunCtx rc{h, st, h->batch, h->last_seqlen, 0, h->batch * h->last_seqlen, nullptr, 0, false, nullptr, nullptr,
-              STAGE_FFN, layer, d_y};
+    RunCtx rc = stage_ctx(h, st, STAGE_FFN, layer, d_y);
     KR_TRY(run_layers(rc, nullptr));
     h->stage_layer_done = layer;
     return KRAKEN_OK;
@@ -894,8 +925,7 @@ int kraken_stage_concat(kraken_handle *h, float *d_z, void *stream) {
     if (h->batch < 1 || h->stage_layer_done != h->cfg.n_layer - 1) return KRAKEN_ESTATE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     h->last_stream = st;
-    RunCtx rc{h, st, h->batch, h->last_seqlen, 0, h->batch * h->last_seqlen, nullptr, 0, false, nullptr, nullptr, 0, 0,
-              nullptr};
+    RunCtx rc = stage_ctx(h, st, STAGE_ALL, 0, nullptr);
     int32_t *rows = at<int32_t>(h, h->lay.rows);
     h->launches[KRAKEN_PROF_TAIL]++;
     make_rows_kernel<<<(h->batch + 255) / 256, 256, 0, st>>>(rows, h->batch, h->last_seqlen, h->last_seqlen - 1);
@@ -908,13 +938,18 @@ int kraken_stage_head(kraken_handle *h, const float *d_z, float *d_logits, void 
     if (h->batch < 1 || h->stage_layer_done != h->cfg.n_layer - 1) return KRAKEN_ESTATE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     h->last_stream = st;
-    RunCtx rc{h, st, h->batch, h->last_seqlen, 0, h->batch * h->last_seqlen, nullptr, 0, false, nullptr, nullptr, 0, 0,
-              nullptr};
+    RunCtx rc = stage_ctx(h, st, STAGE_ALL, 0, nullptr);
     KR_TRY(tail_head(rc, d_z, h->batch, d_logits));
-    set_pos_kernel<<<1, 64, 0, st>>>(at<int>(h, h->lay.pos_arr), h->last_seqlen, h->batch);
-    h->cur_len = h->last_seqlen;
-    h->seq_len.assign(h->batch, h->last_seqlen);
-    h->ragged = false;
+    h->stage_layer_done = -1;
+    if (h->stage_decode) {
+        advance_pos_kernel<<<1, 64, 0, st>>>(at<int>(h, h->lay.pos_arr), h->batch);
+        advance_lengths(h);
+    } else {
+        set_pos_kernel<<<1, 64, 0, st>>>(at<int>(h, h->lay.pos_arr), h->last_seqlen, h->batch);
+        h->cur_len = h->last_seqlen;
+        h->seq_len.assign(h->batch, h->last_seqlen);
+        h->ragged = false;
+    }
     return cuda_check(cudaGetLastError(), "stage head: position update");
 }
 
@@ -961,11 +996,6 @@ int kraken_logits_rows(kraken_handle *h, const int32_t *h_rows, int32_t n_rows, 
 }
 
 namespace {
-
-void advance_lengths(kraken_handle *h) {
-    h->cur_len += 1;
-    for (int &v : h->seq_len) v += 1;
-}
 
 // Whether decode steps of this handle run the branches as concurrent chains.
 bool decode_chains(const kraken_handle *h) {

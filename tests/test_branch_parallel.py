@@ -135,7 +135,8 @@ def test_stage_calls_in_lockstep_equal_the_single_gpu_prefill(name, split):
     s = ki.CONFIGS[name]
     w = ki.make_weights(s, seed=0, device=dev)
     whole = kr.KrakenModel(kr.make_config(s), w, dev)
-    tok = ki.uniform_tokens(2, s.vocab, s.batch, s.seqlen, dev)
+    l0 = min(s.seqlen, s.max_pos - 4)               # room for the decode steps below
+    tok = ki.uniform_tokens(2, s.vocab, s.batch, l0, dev)
     ref = whole.prefill(tok)
     engines = []
     for first, count in split:
@@ -147,12 +148,21 @@ def test_stage_calls_in_lockstep_equal_the_single_gpu_prefill(name, split):
         assert err <= 2e-3 * max(1.0, ref.abs().max().item()), err
     # every rank's cache holds exactly its branches' rows of the whole model's cache
     for (first, count), e in zip(split, engines):
-        assert e.cur_len == s.seqlen and e.device_status() == 0
+        assert e.cur_len == l0 and e.device_status() == 0
         for n in range(count):
             for which in (0, 1):
-                a = e.kv_view(s.n_layer - 1, n, which)[:, :, :s.seqlen].float()
-                b = whole.kv_view(s.n_layer - 1, first + n, which)[:, :, :s.seqlen].float()
+                a = e.kv_view(s.n_layer - 1, n, which)[:, :, :l0].float()
+                b = whole.kv_view(s.n_layer - 1, first + n, which)[:, :, :l0].float()
                 assert (a - b).abs().max().item() <= 2.0 ** -6 * b.abs().max().item()
+    # decode steps driven the same way continue from the caches
+    nxt = ki.uniform_tokens(3, s.vocab, 1, s.batch, dev)[0].contiguous()
+    for step in range(2):
+        want = whole.decode_step(nxt)
+        outs = bp.lockstep_prefill(engines, s.n_layer, nxt, decode=True)
+        for o in outs:
+            err = (o - want).abs().max().item()
+            assert err <= 2e-3 * max(1.0, want.abs().max().item()), (step, err)
+    assert all(e.cur_len == l0 + 2 for e in engines)
     # out-of-order calls are refused
     with pytest.raises(kr.KrakenError) as ex:
         engines[0].stage_attention(1)
