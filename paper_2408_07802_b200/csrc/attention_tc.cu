@@ -518,17 +518,21 @@ int launch(const CUtensorMap &tmQ, const CUtensorMap &tmK, const CUtensorMap &tm
         configured = true;
     }
     const long long items = (long long)((a.seqlen + 2 * TQ - 1) / (2 * TQ)) * a.n_head * a.batch * a.groups;
-    // With enough work, one CTA per SM walks a fixed list of couples of equal total length (atc_next); a plain
+    // With more items than SMs, each CTA walks a fixed list of couples of equal total length (atc_next); a plain
     // round-robin list of single items measured slower than one CTA per item (0.38 vs 0.35 ms at 4 x 2048 x 16
     // heads x 128) because the items are so unequal.  KRAKEN_ATTN_ONE_CTA_PER_ITEM=1 keeps the hardware scheduler.
     const int sms = sm_count() > 0 ? sm_count() : 148;
     const long long couples = (long long)(((a.seqlen + 2 * TQ - 1) / (2 * TQ) + 1) / 2) * a.n_head * a.batch * a.groups;
     AttnTcArgs b = a;
-    // the list pays when its rounds fill the machine: couples / (SMs x rounds) >= 0.85 (measured: 0.87 gains 7 %,
-    // 0.72 loses 3 % against one CTA per item)
+    // The list pays when its rounds fill the machine.  One round (couples <= SMs < items): every couple has an
+    // SM of its own and ends together, where the hardware scheduler hands late CTAs the long items (measured at
+    // 64 heads x 1024: 29.5 vs 36.1 us).  Several rounds: couples / (SMs x rounds) >= 0.85 (measured: 0.87 gains
+    // 7 %, 0.72 loses 3 % against one CTA per item).  With no more items than SMs every item has its own SM and
+    // the longest item alone sets the time, which a couple would only lengthen.
     const long long rounds = (couples + sms - 1) / sms;
-    b.balanced = couples >= 2LL * sms && couples * 100 >= 85LL * sms * rounds && !env_flag("KRAKEN_ATTN_ONE_CTA_PER_ITEM");
-    dim3 grid(static_cast<unsigned>(b.balanced ? sms : items));
+    b.balanced = items > sms && (rounds == 1 || couples * 100 >= 85LL * sms * rounds) &&
+                 !env_flag("KRAKEN_ATTN_ONE_CTA_PER_ITEM");
+    dim3 grid(static_cast<unsigned>(b.balanced ? (couples < sms ? couples : sms) : items));
     attn_tc_kernel<HD><<<grid, ATC_THREADS, Cfg::SMEM_BYTES, stream>>>(tmQ, tmK, tmV, b);
     return cuda_check(cudaGetLastError(), "attention: launch");
 }

@@ -281,6 +281,31 @@ def test_attention_matches_oracle(hd, seqlen, pos0, kernel, monkeypatch):
     assert np.sqrt(num / den) < 6e-3, np.sqrt(num / den)
 
 
+@pytest.mark.parametrize("G,B,H,hd,seqlen", [(4, 1, 16, 64, 768),     # one round of couples, a middle pair alone
+                                              (4, 1, 16, 64, 1024),    # one round, every pair has a partner
+                                              (4, 2, 16, 64, 1300),    # several rounds, ragged last tile
+                                              (3, 2, 12, 128, 520)])   # fewer couples than SMs, ragged
+def test_attention_fixed_work_lists_match_one_cta_per_item(G, B, H, hd, seqlen, monkeypatch):
+    """With more work items than SMs the kernel walks per-CTA lists of couples of items; each item's arithmetic
+    is the same as with one CTA per item, so the outputs are equal bit for bit, and sampled heads match the
+    oracle."""
+    d = H * hd
+    q = ki.normal_bf16(17, 0, (G, B * seqlen, d), 1.0, DEV)
+    kc = ki.normal_bf16(17, 1, (G, B, H, seqlen, hd), 1.0, DEV)
+    vc = ki.normal_bf16(17, 2, (G, B, H, seqlen, hd), 1.0, DEV)
+    got = kr.op_attention(q, kc, vc, B, seqlen, 0, H)
+    monkeypatch.setenv("KRAKEN_ATTN_ONE_CTA_PER_ITEM", "1")
+    plain = kr.op_attention(q, kc, vc, B, seqlen, 0, H)
+    torch.cuda.synchronize()
+    assert torch.equal(got, plain)
+    out = got.float().cpu().numpy()
+    qn, kn, vn = q.float().cpu().numpy(), kc.float().cpu().numpy(), vc.float().cpu().numpy()
+    for g, b, h in [(0, 0, 0), (G - 1, B - 1, H - 1), (1, 0, H // 2)]:
+        ref = oracle.attention_head(qn[g, b * seqlen:(b + 1) * seqlen, h * hd:(h + 1) * hd], kn[g, b, h], vn[g, b, h])
+        err = np.abs(out[g, b * seqlen:(b + 1) * seqlen, h * hd:(h + 1) * hd] - ref)
+        assert err.max() < 3e-2, (g, b, h, err.max())
+
+
 @pytest.mark.parametrize("hd,H,Hkv", [(64, 4, 2), (64, 8, 1), (128, 4, 1), (96, 6, 2), (64, 6, 2), (128, 2, 2)])
 @pytest.mark.parametrize("seqlen,pos0", [(300, 0), (100, 37)])
 def test_grouped_query_attention_matches_oracle(hd, H, Hkv, seqlen, pos0):
