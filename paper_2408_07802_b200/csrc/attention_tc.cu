@@ -4,8 +4,9 @@
 // 128 keys by TMA; the two query tiles share every K/V tile and take turns on the tensor pipe, so
 // that while one tile's scores are in the softmax the other tile's matrix products run.
 //
-//   warp 0      TMA producer: both Q tiles once, then K and V tiles into two-stage rings
-//               (128-byte swizzle; rows past the keys written so far are out of bounds = zeros);
+//   warp 0      TMA producer: both Q tiles once, then K and V tiles into a two-stage ring whose stage
+//               holds what one step of the issuer reads, V_j and K_{j+1} (one barrier wait and one release
+//               per step; 128-byte swizzle; rows past the keys written so far are out of bounds = zeros);
 //   warp 1      MMA issuer, per K/V tile j and query tile w:
 //                   S_w = Q_w K_j^T          both operands K-major in shared memory -> TMEM
 //                   O_w (+)= P_w V_j         P_w read from TMEM (it overwrites S_w in place as packed
@@ -136,7 +137,8 @@ struct AtcCfg {
     static constexpr int Q_BYTES = HALVES * TILE_BYTES;    // one Q tile
     static constexpr int KV_BYTES = HALVES * TILE_BYTES;   // one K (or V) tile
     static constexpr int STAGES = 2;
-    static constexpr int SMEM_BYTES = 2 * Q_BYTES + 2 * STAGES * KV_BYTES + 1024 + 256;
+    static constexpr int BUNDLE_BYTES = 2 * KV_BYTES;      // a ring stage: V_j, then K_{j+1}
+    static constexpr int SMEM_BYTES = 2 * Q_BYTES + STAGES * BUNDLE_BYTES + 1024 + 256;
     static constexpr int S_COL0 = 0;                       // S / P of query tile w at 128 w
     static constexpr int O_COL0 = 256;                     // O of query tile w at 256 + 128 w
     static constexpr int TMEM_COLS = 512;
@@ -207,19 +209,16 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     extern __shared__ uint8_t smem_raw_atc[];
     uint8_t *smem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw_atc) + 1023) & ~uintptr_t(1023));
     uint8_t *sQ = smem;                                    // [2][Q_BYTES]
-    uint8_t *sK = sQ + 2 * Cfg::Q_BYTES;                   // [STAGES][KV_BYTES]
-    uint8_t *sV = sK + Cfg::STAGES * Cfg::KV_BYTES;        // [STAGES][KV_BYTES]
-    uint64_t *bars = reinterpret_cast<uint64_t *>(sV + Cfg::STAGES * Cfg::KV_BYTES);
+    uint8_t *sB = sQ + 2 * Cfg::Q_BYTES;                   // [STAGES][V tile | K tile]
+    uint64_t *bars = reinterpret_cast<uint64_t *>(sB + Cfg::STAGES * Cfg::BUNDLE_BYTES);
     uint64_t *q_full = bars;            // 1    Q tiles of the current item loaded
     uint64_t *q_empty = bars + 1;       // 1    every S = Q K^T of the item has finished reading Q
-    uint64_t *k_full = bars + 2;        // [2]
-    uint64_t *k_empty = bars + 4;       // [2]
-    uint64_t *v_full = bars + 6;        // [2]
-    uint64_t *v_empty = bars + 8;       // [2]
-    uint64_t *s_full = bars + 10;       // [2]  scores of query tile w ready      (MMA -> softmax w)
-    uint64_t *p_ready = bars + 12;      // [2]  probabilities of tile w in TMEM   (softmax w -> MMA)
-    uint64_t *pv_done = bars + 14;      // [2]  O_w holds every product issued so far (MMA -> softmax w)
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 16);
+    uint64_t *b_full = bars + 2;        // [2]  V_j and K_{j+1} loaded
+    uint64_t *b_empty = bars + 4;       // [2]  every product that reads them has finished
+    uint64_t *s_full = bars + 6;        // [2]  scores of query tile w ready      (MMA -> softmax w)
+    uint64_t *p_ready = bars + 8;       // [2]  probabilities of tile w in TMEM   (softmax w -> MMA)
+    uint64_t *pv_done = bars + 10;      // [2]  O_w of the item is complete       (MMA -> softmax w)
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 12);
     volatile uint32_t *abort_flag = tmem_slot + 1;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -228,10 +227,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         mbar_init(q_full, 1);
         mbar_init(q_empty, 1);
         for (int s = 0; s < 2; ++s) {
-            mbar_init(k_full + s, 1);
-            mbar_init(k_empty + s, 1);
-            mbar_init(v_full + s, 1);
-            mbar_init(v_empty + s, 1);
+            mbar_init(b_full + s, 1);
+            mbar_init(b_empty + s, 1);
             mbar_init(s_full + s, 1);
             mbar_init(p_ready + s, 4);
             mbar_init(pv_done + s, 1);
@@ -267,21 +264,25 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                     for (int hf = 0; hf < Cfg::HALVES; ++hf)
                         tma_load_3d(sQ + w * Cfg::Q_BYTES + hf * Cfg::TILE_BYTES, &tmQ, q_full, it.h * a.head_dim + hf * 64,
                                     it.b * a.seqlen + it.q0 + w * TQ, it.g);
-                for (int j = 0; ok && j < it.n_max; ++j, ++kv_cnt) {
+                // stage -1 of the item holds K_0 alone; stage j holds V_j and, unless it is the last, K_{j+1}
+                const int kvh = it.b * a.n_kv_head + it.h / a.kv_rep;
+                for (int j = -1; ok && j < it.n_max; ++j, ++kv_cnt) {
                     const int st = kv_cnt & 1;
                     const uint32_t ph = (kv_cnt >> 1) & 1;
-                    if (!(ok = mbar_wait(k_empty + st, ph ^ 1u, abort_flag))) break;
-                    mbar_expect_tx(k_full + st, Cfg::KV_BYTES);
+                    if (!(ok = mbar_wait(b_empty + st, ph ^ 1u, abort_flag))) break;
+                    const bool has_v = j >= 0, has_k = j + 1 < it.n_max;
+                    mbar_expect_tx(b_full + st, ((has_v ? 1 : 0) + (has_k ? 1 : 0)) * Cfg::KV_BYTES);
+                    uint8_t *sV = sB + st * Cfg::BUNDLE_BYTES, *sK = sV + Cfg::KV_BYTES;
+                    if (has_v) {
 #pragma unroll
-                    for (int hf = 0; hf < Cfg::HALVES; ++hf)
-                        tma_load_4d(sK + st * Cfg::KV_BYTES + hf * Cfg::TILE_BYTES, &tmK, k_full + st, hf * 64,
-                                    j * TK, it.b * a.n_kv_head + it.h / a.kv_rep, it.g);
-                    if (!(ok = mbar_wait(v_empty + st, ph ^ 1u, abort_flag))) break;
-                    mbar_expect_tx(v_full + st, Cfg::KV_BYTES);
+                        for (int hf = 0; hf < Cfg::HALVES; ++hf)
+                            tma_load_4d(sV + hf * Cfg::TILE_BYTES, &tmV, b_full + st, hf * 64, j * TK, kvh, it.g);
+                    }
+                    if (has_k) {
 #pragma unroll
-                    for (int hf = 0; hf < Cfg::HALVES; ++hf)
-                        tma_load_4d(sV + st * Cfg::KV_BYTES + hf * Cfg::TILE_BYTES, &tmV, v_full + st, hf * 64,
-                                    j * TK, it.b * a.n_kv_head + it.h / a.kv_rep, it.g);
+                        for (int hf = 0; hf < Cfg::HALVES; ++hf)
+                            tma_load_4d(sK + hf * Cfg::TILE_BYTES, &tmK, b_full + st, hf * 64, (j + 1) * TK, kvh, it.g);
+                    }
                 }
             }
         }
@@ -295,7 +296,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             const uint32_t idesc_pv = umma_idesc_h16(TQ, qk_steps * 16) | (1u << 16);  // B (V) is MN-major
             auto issue_qk = [&](int w, int st) {
                 const uint32_t q_addr = smem_u32(sQ + w * Cfg::Q_BYTES);
-                const uint32_t k_addr = smem_u32(sK + st * Cfg::KV_BYTES);
+                const uint32_t k_addr = smem_u32(sB + st * Cfg::BUNDLE_BYTES + Cfg::KV_BYTES);
                 const uint32_t d_tmem = tmem_base + Cfg::S_COL0 + w * TK;
 #pragma unroll
                 for (int ks = 0; ks < HD / 16; ++ks) {
@@ -306,8 +307,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 }
                 umma_commit(s_full + w);
             };
-            auto issue_pv = [&](int w, int st, bool first) {
-                const uint32_t v_addr = smem_u32(sV + st * Cfg::KV_BYTES);
+            auto issue_pv = [&](int w, int st, bool first, bool last) {
+                const uint32_t v_addr = smem_u32(sB + st * Cfg::BUNDLE_BYTES);
                 const uint32_t p_tmem = tmem_base + Cfg::S_COL0 + w * TK;
                 const uint32_t o_tmem = tmem_base + Cfg::O_COL0 + w * TK;
 #pragma unroll
@@ -317,42 +318,38 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                                  umma_desc_sw128_mnmajor(v_addr + ks * 2048, Cfg::TILE_BYTES), idesc_pv,
                                  (first && ks == 0) ? 0u : 1u);
                 }
-                umma_commit(pv_done + w);
+                // the softmax warps need no signal for the products in between: the scores they wait for next
+                // are committed after this product, and a commit covers everything issued before it
+                if (last) umma_commit(pv_done + w);
             };
             bool ok = true;
             uint32_t kv_cnt = 0, item_cnt = 0, tile_cnt[2] = {0, 0};
             AtcItem it;
             for (int jj = 0; ok && atc_next(a, jj, it); ++item_cnt) {
                 if (!(ok = mbar_wait(q_full, item_cnt & 1u, abort_flag))) break;
-                if (!(ok = mbar_wait(k_full + (kv_cnt & 1), (kv_cnt >> 1) & 1, abort_flag))) break;
+                if (!(ok = mbar_wait(b_full + (kv_cnt & 1), (kv_cnt >> 1) & 1, abort_flag))) break;
                 tc_fence_after_sync();
                 if (it.n_tiles[0] > 0) issue_qk(0, kv_cnt & 1);
                 if (it.n_tiles[1] > 0) issue_qk(1, kv_cnt & 1);
-                umma_commit(k_empty + (kv_cnt & 1));
+                umma_commit(b_empty + (kv_cnt & 1));
+                ++kv_cnt;
                 if (it.n_max == 1) umma_commit(q_empty);
                 for (int j = 0; ok && j < it.n_max; ++j, ++kv_cnt) {
                     const int st = kv_cnt & 1;
-                    const uint32_t ph = (kv_cnt >> 1) & 1;
-                    const bool next = j + 1 < it.n_max;
-                    const int st_n = (kv_cnt + 1) & 1;
-                    if (!(ok = mbar_wait(v_full + st, ph, abort_flag))) break;
-                    if (next && !(ok = mbar_wait(k_full + st_n, ((kv_cnt + 1) >> 1) & 1, abort_flag))) break;
+                    if (!(ok = mbar_wait(b_full + st, (kv_cnt >> 1) & 1, abort_flag))) break;
 #pragma unroll
                     for (int w = 0; w < 2; ++w) {
                         if (j < it.n_tiles[w]) {
                             if (!(ok = mbar_wait(p_ready + w, tile_cnt[w] & 1u, abort_flag))) break;
                             ++tile_cnt[w];
                             tc_fence_after_sync();
-                            issue_pv(w, st, j == 0);
+                            issue_pv(w, st, j == 0, j + 1 == it.n_tiles[w]);
                         }
-                        if (j + 1 < it.n_tiles[w]) issue_qk(w, st_n);
+                        if (j + 1 < it.n_tiles[w]) issue_qk(w, st);
                     }
                     if (!ok) break;
-                    umma_commit(v_empty + st);
-                    if (next) {
-                        umma_commit(k_empty + st_n);
-                        if (j + 2 == it.n_max) umma_commit(q_empty);   // the item's last scores are issued
-                    }
+                    umma_commit(b_empty + st);
+                    if (j + 2 == it.n_max) umma_commit(q_empty);   // the item's last scores are issued
                 }
             }
         }
@@ -367,6 +364,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         const float sl2 = rsqrtf(static_cast<float>(a.head_dim)) * 1.4426950408889634f;
         bool ok = true;
         uint32_t tile_cnt = 0;                               // tiles this warp group has consumed so far
+        uint32_t done_cnt = 0;                               // items this warp group has finished
         AtcItem it;
         for (int jj = 0; ok && atc_next(a, jj, it);) {
             const int tile_q0 = it.q0 + w * TQ;
@@ -441,12 +439,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 }
                 l = l * f + ((sum0 + sum1) + (sum2 + sum3));
                 if (__any_sync(0xFFFFFFFFu, raise)) {
-                    // (rare) O_w must hold every product issued so far before its rows are rescaled; the
-                    // next product is not issued until this warp has released P below
-                    ok = mbar_wait(pv_done + w, (tile_cnt - 1u) & 1u, abort_flag);
-                    ok = __all_sync(0xFFFFFFFFu, ok);
-                    if (!ok) break;
-                    tc_fence_after_sync();
+                    // (rare) O_w holds every product issued so far: these scores were committed after the last
+                    // one, and a commit covers all that was issued before it.  The next product is not issued
+                    // until this warp has released P below.
 #pragma unroll 1
                     for (int c = 0; c < HD / 32; ++c) {
                         uint32_t r[32];
@@ -464,9 +459,10 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             }
             if (!ok) break;
             if (n_w > 0) {
-                ok = mbar_wait(pv_done + w, (tile_cnt - 1u) & 1u, abort_flag);
+                ok = mbar_wait(pv_done + w, done_cnt & 1u, abort_flag);   // one arrival per item of this tile slot
                 ok = __all_sync(0xFFFFFFFFu, ok);
                 if (!ok) break;
+                ++done_cnt;
                 tc_fence_after_sync();
                 const float inv = 1.f / l;
                 const int d = a.n_head * a.head_dim;
