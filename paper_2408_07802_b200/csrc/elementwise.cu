@@ -139,6 +139,95 @@ layernorm_kernel(const float *__restrict__ a, long long a_gstride, const float *
     for (int v = lane + 32 * LN_CACHE; v < nvec; v += 32) emit(v, load(v));
 }
 
+// The same LayerNorm with one CTA per row: for rows wider than a warp can keep in registers (d > 2048, where the
+// kernel above goes over the tail of the row three times) and for few, wide rows, where eight warps on one row
+// shorten the chain of dependent memory round trips that a single warp would walk alone.  Thread t holds elements
+// 4 (t + 256 i) .. + 3; partial sums go through a warp shuffle tree and then through shared memory, added in warp
+// order by every thread, so the result does not depend on timing.
+constexpr int LNB_THREADS = 256;
+constexpr int LNB_CACHE = 8;   // float4 per thread: rows up to 8192 wide
+
+__global__ void __launch_bounds__(LNB_THREADS)
+layernorm_block_kernel(const float *__restrict__ a, long long a_gstride, const float *__restrict__ y,
+                       const uint16_t *__restrict__ gamma, const uint16_t *__restrict__ beta, int groups, int rows,
+                       int d, float eps, uint16_t *__restrict__ out) {
+    __shared__ float red[2][LNB_THREADS / 32];
+    pdl_wait();
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int nvec = d / 4;
+    bool triggered = false;
+    for (long long wr = blockIdx.x; wr < (long long)groups * rows; wr += gridDim.x) {
+        // neighbouring CTAs take the groups of one row, so the shared y row is fetched from DRAM once
+        const int r = static_cast<int>(wr / groups), g = static_cast<int>(wr % groups);
+        const float4 *pa = reinterpret_cast<const float4 *>(a + g * a_gstride + (size_t)r * d);
+        const float4 *py = y ? reinterpret_cast<const float4 *>(y + (size_t)r * d) : nullptr;
+        float4 cache[LNB_CACHE];
+        float sum = 0.f;
+#pragma unroll
+        for (int i = 0; i < LNB_CACHE; ++i) {
+            const int v = tid + LNB_THREADS * i;
+            if (v < nvec) {
+                float4 t = pa[v];
+                if (py) {
+                    const float4 u = py[v];
+                    t.x += u.x; t.y += u.y; t.z += u.z; t.w += u.w;
+                }
+                cache[i] = t;
+                sum += (t.x + t.y) + (t.z + t.w);
+            }
+        }
+        sum = warp_sum(sum);
+        if (lane == 0) red[0][warp] = sum;
+        __syncthreads();
+        float tot = 0.f;
+#pragma unroll
+        for (int w = 0; w < LNB_THREADS / 32; ++w) tot += red[0][w];
+        const float mean = tot / d;
+        float sq = 0.f;
+#pragma unroll
+        for (int i = 0; i < LNB_CACHE; ++i) {
+            const int v = tid + LNB_THREADS * i;
+            if (v < nvec) {
+                const float4 t = cache[i];
+                const float dx = t.x - mean, dy = t.y - mean, dz = t.z - mean, dw = t.w - mean;
+                sq += (dx * dx + dy * dy) + (dz * dz + dw * dw);
+            }
+        }
+        sq = warp_sum(sq);
+        if (lane == 0) red[1][warp] = sq;
+        __syncthreads();
+        float tot2 = 0.f;
+#pragma unroll
+        for (int w = 0; w < LNB_THREADS / 32; ++w) tot2 += red[1][w];
+        const float rstd = rsqrtf(tot2 / d + eps);
+        if (!triggered) {
+            pdl_trigger();
+            triggered = true;
+        }
+        const uint2 *pg = reinterpret_cast<const uint2 *>(gamma + (size_t)g * d);
+        const uint2 *pb = beta ? reinterpret_cast<const uint2 *>(beta + (size_t)g * d) : nullptr;
+        uint2 *po = reinterpret_cast<uint2 *>(out + ((size_t)g * rows + r) * d);
+#pragma unroll
+        for (int i = 0; i < LNB_CACHE; ++i) {
+            const int v = tid + LNB_THREADS * i;
+            if (v < nvec) {
+                const float4 t = cache[i];
+                const uint2 gm = __ldg(pg + v);
+                uint2 bt = make_uint2(0u, 0u);
+                if (pb) bt = __ldg(pb + v);
+                const float o0 = (t.x - mean) * rstd * h16_lo(gm.x) + h16_lo(bt.x);
+                const float o1 = (t.y - mean) * rstd * h16_hi(gm.x) + h16_hi(bt.x);
+                const float o2 = (t.z - mean) * rstd * h16_lo(gm.y) + h16_lo(bt.y);
+                const float o3 = (t.w - mean) * rstd * h16_hi(gm.y) + h16_hi(bt.y);
+                po[v] = make_uint2(pack_h16x2(o0, o1), pack_h16x2(o2, o3));
+            }
+        }
+        // red[] is written again by the next row only after every thread has passed the second barrier of
+        // this one; its first barrier then keeps the two rows' partial sums apart
+    }
+    if (!triggered) pdl_trigger();
+}
+
 // The same LayerNorm for many rows, as a persistent producer / consumer kernel: what limits the
 // warp-per-row kernel above is that a warp has nothing in flight while it reduces and writes, so here
 // one thread keeps a ring of whole rows in flight with bulk copies (a stage = the N group rows of one
@@ -366,6 +455,23 @@ int launch_layernorm(const float *a, long long a_gstride, const float *y, const 
         return cuda_check(cudaGetLastError(), "layernorm: launch");
     }
     const long long warps = (long long)groups * rows;
+    // One CTA per row (layernorm_block_kernel) for up to 24 rows per SM of more than 1024 elements, and for rows
+    // of more than 4096 elements whatever their number.  Measured, 4 groups, us per launch, warp / CTA per row:
+    // 128 tokens d 2496 9.0 / 5.5, d 3120 11.3 / 6.2, d 7424 29.1 / 8.9; 512 tokens d 2496 16.0 / 11.4; 2048 tokens
+    // d 2496 48.0 / 56.7, d 3120 61.2 / 62.4, d 4992 121.7 / 80.3, d 7424 216.8 / 105.5 (a warp keeps 2048 elements
+    // in registers and goes over the rest of a wider row three times; keeping 4096 costs it more in occupancy).
+    // KRAKEN_LN_BLOCK=0/1 forces the choice.
+    const int sms_b = sm_count() > 0 ? sm_count() : 148;
+    const char *force_b = getenv("KRAKEN_LN_BLOCK");
+    const bool block_auto = d > 4096 || (d > 1024 && warps <= 24LL * sms_b);
+    const bool block_rows = !ysum && d <= 4 * LNB_THREADS * LNB_CACHE &&
+                            (force_b && (force_b[0] == '0' || force_b[0] == '1') ? force_b[0] == '1' : block_auto);
+    if (block_rows) {
+        const long long ctas = warps < 8LL * sms_b ? warps : 8LL * sms_b;
+        return cuda_check(launch_pdl(layernorm_block_kernel, dim3(static_cast<unsigned>(ctas)), dim3(LNB_THREADS), 0,
+                                     stream, a, a_gstride, y, gamma, beta, groups, rows, d, eps, out),
+                          "layernorm: launch");
+    }
     const dim3 grid(static_cast<unsigned>((warps + ROW_WARPS - 1) / ROW_WARPS)), block(ROW_WARPS * 32);
     const cudaError_t ce =
         d <= 1024 ? launch_pdl(layernorm_kernel<8>, grid, block, 0, stream, a, a_gstride, y, ysum, ysum_gstride,

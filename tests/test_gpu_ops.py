@@ -48,7 +48,7 @@ def test_embed_and_bad_token_flag():
 
 # ------------------------------------------------------------------ LayerNorm
 
-@pytest.mark.parametrize("d", [128, 768, 2048, 4096])
+@pytest.mark.parametrize("d", [128, 768, 2048, 2496, 4096, 7424])
 @pytest.mark.parametrize("with_y", [False, True])
 def test_layernorm(d, with_y):
     G, rows = 3, 37
@@ -89,6 +89,26 @@ def test_layernorm_many_rows_persistent_kernel(G, d, with_y):
     for g in (0, G - 1):
         ref = oracle.layernorm(a[g][pick].cpu().numpy(), None if y is None else y[pick].cpu().numpy(),
                                bits(gamma[g]), bits(beta[g]))
+        ok, worst = bf16_ulp_close(out[g][pick].float().cpu().numpy(), ref, ulps=1.0, atol=1e-5)
+        assert ok, (g, worst)
+
+
+@pytest.mark.parametrize("force", ["0", "1"])
+def test_layernorm_one_cta_per_row_walks_many_rows(force, monkeypatch):
+    """Rows wider than 4096 take the one-CTA-per-row kernel, whose grid is smaller than the number of rows here, so
+    every CTA walks several rows; the same call forced onto the warp-per-row kernel agrees within one bf16 step
+    (the two sum in different orders)."""
+    monkeypatch.setenv("KRAKEN_LN_BLOCK", force)
+    G, d = 2, 4992
+    rows = 5 * torch.cuda.get_device_properties(0).multi_processor_count + 3
+    a = (ki.normal_bf16(5, 0, (G, rows, d), 1.0, DEV).float() * 0.9 + 0.1).contiguous()
+    y = ki.normal_bf16(5, 1, (rows, d), 2.0, DEV).float().contiguous()
+    gamma = (1 + ki.normal_bf16(5, 2, (G, d), 0.3, DEV).float()).to(torch.bfloat16)
+    beta = ki.normal_bf16(5, 3, (G, d), 0.3, DEV)
+    out = kr.op_layernorm(a, y, gamma, beta)
+    pick = [0, 1, rows // 3, rows - 2, rows - 1]
+    for g in range(G):
+        ref = oracle.layernorm(a[g][pick].cpu().numpy(), y[pick].cpu().numpy(), bits(gamma[g]), bits(beta[g]))
         ok, worst = bf16_ulp_close(out[g][pick].float().cpu().numpy(), ref, ulps=1.0, atol=1e-5)
         assert ok, (g, worst)
 
