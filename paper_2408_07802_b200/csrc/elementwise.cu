@@ -231,21 +231,21 @@ layernorm_block_kernel(const float *__restrict__ a, long long a_gstride, const f
 // The same LayerNorm for many rows, as a persistent producer / consumer kernel: what limits the
 // warp-per-row kernel above is that a warp has nothing in flight while it reduces and writes, so here
 // one thread keeps a ring of whole rows in flight with bulk copies (a stage = the N group rows of one
-// row index plus the shared y row, each fetched from DRAM once) and twelve consumer warps take the rows
+// row index plus the shared y row, each fetched from DRAM once) and twelve (or up to sixteen) consumer warps take the rows
 // out of shared memory into registers, release the stage at once and then reduce, normalise and store.
 // Consumer warp c works on group c % groups of every (c / groups)-th stage; the number of stages is a
 // multiple of the number of such warp sets, so a ring slot is always consumed by the same set and every
 // waiter sees every phase of the barriers it waits on.
-constexpr int LNS_CONSUMERS = 12;
-constexpr int LNS_THREADS = (LNS_CONSUMERS + 1) * 32;
+constexpr int LNS_CONSUMERS = 12;       // group counts that divide 12 (1, 2, 3, 4, 6, 12)
+constexpr int LNS_CONSUMERS_WIDE = 16;  // other group counts up to 16: the largest multiple of the count <= 16
 constexpr int LNS_MAX_STAGES = 12;
 constexpr int LNS_SMEM_BUDGET = 226 * 1024;
 
-template <int LN_CACHE>
-__global__ void __launch_bounds__(LNS_THREADS, 1)
+template <int LN_CACHE, int MAX_CONSUMERS>
+__global__ void __launch_bounds__((MAX_CONSUMERS + 1) * 32, 1)
 layernorm_stream_kernel(const float *__restrict__ a, long long a_gstride, const float *__restrict__ y,
                         const uint16_t *__restrict__ gamma, const uint16_t *__restrict__ beta, int groups, int rows,
-                        int d, float eps, uint16_t *__restrict__ out, int stages, uint32_t *status) {
+                        int d, float eps, uint16_t *__restrict__ out, int stages, int n_consumers, uint32_t *status) {
     extern __shared__ __align__(128) uint8_t lns_smem[];
     __shared__ uint64_t full[LNS_MAX_STAGES], empty[LNS_MAX_STAGES];
     __shared__ uint32_t abort_word;
@@ -265,14 +265,14 @@ layernorm_stream_kernel(const float *__restrict__ a, long long a_gstride, const 
     // shared memory the L1 left over does not hold them, and their latency would sit on every row
     uint16_t *s_gamma = reinterpret_cast<uint16_t *>(lns_smem + (size_t)stages * stage_bytes);
     uint16_t *s_beta = s_gamma + (size_t)groups * d;
-    for (int i = threadIdx.x; i < groups * d / 4; i += LNS_THREADS) {
+    for (int i = threadIdx.x; i < groups * d / 4; i += blockDim.x) {
         reinterpret_cast<uint2 *>(s_gamma)[i] = __ldg(reinterpret_cast<const uint2 *>(gamma) + i);
         reinterpret_cast<uint2 *>(s_beta)[i] = beta ? __ldg(reinterpret_cast<const uint2 *>(beta) + i) : make_uint2(0u, 0u);
     }
     __syncthreads();
     const int n_units = (rows - static_cast<int>(blockIdx.x) + static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x);
 
-    if (warp == LNS_CONSUMERS) {
+    if (warp == n_consumers) {
         if (lane == 0) {
             for (int k = 0; k < n_units; ++k) {
                 const int slot = k % stages;
@@ -287,7 +287,7 @@ layernorm_stream_kernel(const float *__restrict__ a, long long a_gstride, const 
         }
         __syncwarp();
     } else {
-        const int n_sets = LNS_CONSUMERS / groups;
+        const int n_sets = n_consumers / groups;
         const int set = warp / groups, g = warp % groups;
         const int nvec = d / 4;
         const uint2 *pg = reinterpret_cast<const uint2 *>(s_gamma + (size_t)g * d);
@@ -413,14 +413,23 @@ int launch_embed(const int32_t *ids, int n_tokens, int seqlen, int pos0, const u
 
 // whether the persistent kernel takes the call: enough rows to fill its ring on every SM, a stage
 // that fits at least once per consumer set
+// consumer warps of the persistent kernel for a group count: 12 where the count divides 12, else the largest
+// multiple of the count up to 16 (0: more than 16 groups)
+static int layernorm_stream_consumers(int groups) {
+    if (groups < 1 || groups > LNS_CONSUMERS_WIDE) return 0;
+    if (LNS_CONSUMERS % groups == 0) return LNS_CONSUMERS;
+    return LNS_CONSUMERS_WIDE / groups * groups;
+}
+
 bool layernorm_stream_fits(const float *a, long long a_gstride, const float *y, int groups, int rows, int d,
                            int *stages_out) {
-    if (groups < 1 || LNS_CONSUMERS % groups != 0) return false;
+    const int n_consumers = layernorm_stream_consumers(groups);
+    if (n_consumers == 0) return false;
     if (d > 2048 || (d & 3) || (a_gstride & 3)) return false;
     if ((reinterpret_cast<uintptr_t>(a) & 15) || (reinterpret_cast<uintptr_t>(y) & 15)) return false;
     const int sms = sm_count() > 0 ? sm_count() : 148;
     if (rows < 8 * sms) return false;
-    const int n_sets = LNS_CONSUMERS / groups;
+    const int n_sets = n_consumers / groups;
     const long long stage_bytes = 4LL * d * (groups + (y ? 1 : 0));
     long long stages = (LNS_SMEM_BUDGET - 4LL * groups * d) / stage_bytes;   // gamma, beta sit behind the ring
     if (stages > LNS_MAX_STAGES) stages = LNS_MAX_STAGES;
@@ -442,16 +451,20 @@ int launch_layernorm(const float *a, long long a_gstride, const float *y, const 
         layernorm_stream_fits(a, a_gstride, y, groups, rows, d, &stages)) {
         const size_t smem = (size_t)stages * 4 * d * (groups + (y ? 1 : 0)) + (size_t)4 * groups * d;
         const int sms = sm_count() > 0 ? sm_count() : 148;
-        auto kern = d <= 1024 ? layernorm_stream_kernel<8> : layernorm_stream_kernel<16>;
-        static bool configured[2] = {false, false};
-        if (!configured[d <= 1024]) {
+        const int n_consumers = layernorm_stream_consumers(groups);
+        const bool wide = n_consumers > LNS_CONSUMERS;
+        auto kern = wide ? (d <= 1024 ? layernorm_stream_kernel<8, LNS_CONSUMERS_WIDE> : layernorm_stream_kernel<16, LNS_CONSUMERS_WIDE>)
+                         : (d <= 1024 ? layernorm_stream_kernel<8, LNS_CONSUMERS> : layernorm_stream_kernel<16, LNS_CONSUMERS>);
+        static bool configured[4] = {false, false, false, false};
+        const int which = (wide ? 2 : 0) + (d <= 1024 ? 1 : 0);
+        if (!configured[which]) {
             int rc = cuda_check(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                      LNS_SMEM_BUDGET), "layernorm: shared memory opt-in");
             if (rc) return rc;
-            configured[d <= 1024] = true;
+            configured[which] = true;
         }
-        kern<<<dim3(sms), dim3(LNS_THREADS), smem, stream>>>(a, a_gstride, y, gamma, beta, groups, rows, d, eps, out,
-                                                          stages, status);
+        kern<<<dim3(sms), dim3((n_consumers + 1) * 32), smem, stream>>>(a, a_gstride, y, gamma, beta, groups, rows, d, eps,
+                                                                     out, stages, n_consumers, status);
         return cuda_check(cudaGetLastError(), "layernorm: launch");
     }
     const long long warps = (long long)groups * rows;

@@ -70,7 +70,7 @@ def test_layernorm(d, with_y):
 
 
 @pytest.mark.parametrize("G,d,with_y", [(4, 2048, True), (4, 2048, False), (2, 768, True), (1, 1000, False),
-                                        (3, 512, True), (8, 512, True)])
+                                        (3, 512, True), (8, 512, True), (8, 1920, True), (5, 768, True), (16, 256, False)])
 def test_layernorm_many_rows_persistent_kernel(G, d, with_y):
     """With a status word and many rows the persistent ring kernel runs: sampled rows against the oracle,
     every row bit-equal to the warp-per-row kernel (same operations in the same order); ragged row count."""
