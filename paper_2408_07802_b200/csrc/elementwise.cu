@@ -413,19 +413,23 @@ int launch_embed(const int32_t *ids, int n_tokens, int seqlen, int pos0, const u
 
 // whether the persistent kernel takes the call: enough rows to fill its ring on every SM, a stage
 // that fits at least once per consumer set
-// consumer warps of the persistent kernel for a group count: 12 where the count divides 12, else the largest
-// multiple of the count up to 16 (0: more than 16 groups)
-static int layernorm_stream_consumers(int groups) {
+// consumer warps of the persistent kernel: rows up to 2048 wide, 12 where the group count divides 12, else the
+// largest multiple of the count up to 16; rows up to 4096 wide need twice the registers per consumer, so 8 warps
+// (group counts 1, 2, 4, 8).  0: the kernel does not take the shape.
+constexpr int LNS_CONSUMERS_4K = 8;
+static int layernorm_stream_consumers(int groups, int d) {
     if (groups < 1 || groups > LNS_CONSUMERS_WIDE) return 0;
+    if (d > 4096) return 0;
+    if (d > 2048) return LNS_CONSUMERS_4K % groups == 0 ? LNS_CONSUMERS_4K : 0;
     if (LNS_CONSUMERS % groups == 0) return LNS_CONSUMERS;
     return LNS_CONSUMERS_WIDE / groups * groups;
 }
 
 bool layernorm_stream_fits(const float *a, long long a_gstride, const float *y, int groups, int rows, int d,
                            int *stages_out) {
-    const int n_consumers = layernorm_stream_consumers(groups);
+    const int n_consumers = layernorm_stream_consumers(groups, d);
     if (n_consumers == 0) return false;
-    if (d > 2048 || (d & 3) || (a_gstride & 3)) return false;
+    if ((d & 3) || (a_gstride & 3)) return false;
     if ((reinterpret_cast<uintptr_t>(a) & 15) || (reinterpret_cast<uintptr_t>(y) & 15)) return false;
     const int sms = sm_count() > 0 ? sm_count() : 148;
     if (rows < 8 * sms) return false;
@@ -451,12 +455,15 @@ int launch_layernorm(const float *a, long long a_gstride, const float *y, const 
         layernorm_stream_fits(a, a_gstride, y, groups, rows, d, &stages)) {
         const size_t smem = (size_t)stages * 4 * d * (groups + (y ? 1 : 0)) + (size_t)4 * groups * d;
         const int sms = sm_count() > 0 ? sm_count() : 148;
-        const int n_consumers = layernorm_stream_consumers(groups);
+        const int n_consumers = layernorm_stream_consumers(groups, d);
         const bool wide = n_consumers > LNS_CONSUMERS;
-        auto kern = wide ? (d <= 1024 ? layernorm_stream_kernel<8, LNS_CONSUMERS_WIDE> : layernorm_stream_kernel<16, LNS_CONSUMERS_WIDE>)
-                         : (d <= 1024 ? layernorm_stream_kernel<8, LNS_CONSUMERS> : layernorm_stream_kernel<16, LNS_CONSUMERS>);
-        static bool configured[4] = {false, false, false, false};
-        const int which = (wide ? 2 : 0) + (d <= 1024 ? 1 : 0);
+        auto kern = d > 2048 ? layernorm_stream_kernel<32, LNS_CONSUMERS_4K>
+                    : wide   ? (d <= 1024 ? layernorm_stream_kernel<8, LNS_CONSUMERS_WIDE>
+                                          : layernorm_stream_kernel<16, LNS_CONSUMERS_WIDE>)
+                             : (d <= 1024 ? layernorm_stream_kernel<8, LNS_CONSUMERS>
+                                          : layernorm_stream_kernel<16, LNS_CONSUMERS>);
+        static bool configured[5] = {false, false, false, false, false};
+        const int which = d > 2048 ? 4 : (wide ? 2 : 0) + (d <= 1024 ? 1 : 0);
         if (!configured[which]) {
             int rc = cuda_check(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                      LNS_SMEM_BUDGET), "layernorm: shared memory opt-in");

@@ -70,8 +70,9 @@ def test_layernorm(d, with_y):
 
 
 @pytest.mark.parametrize("G,d,with_y", [(4, 2048, True), (4, 2048, False), (2, 768, True), (1, 1000, False),
-                                        (3, 512, True), (8, 512, True), (8, 1920, True), (5, 768, True), (16, 256, False)])
-def test_layernorm_many_rows_persistent_kernel(G, d, with_y):
+                                        (3, 512, True), (8, 512, True), (8, 1920, True), (5, 768, True), (16, 256, False),
+                                        (4, 2496, True), (4, 3120, False), (2, 4096, True)])
+def test_layernorm_many_rows_persistent_kernel(G, d, with_y, monkeypatch):
     """With a status word and many rows the persistent ring kernel runs: sampled rows against the oracle,
     every row bit-equal to the warp-per-row kernel (same operations in the same order); ragged row count."""
     rows = 8 * torch.cuda.get_device_properties(0).multi_processor_count + 37
@@ -83,6 +84,7 @@ def test_layernorm_many_rows_persistent_kernel(G, d, with_y):
     out = kr.op_layernorm(a, y, gamma, beta, status=status)
     torch.cuda.synchronize()
     assert int(status.item()) == 0
+    monkeypatch.setenv("KRAKEN_LN_BLOCK", "0")       # the warp-per-row kernel, not one CTA per row
     plain = kr.op_layernorm(a, y, gamma, beta)
     assert torch.equal(out.view(torch.int16), plain.view(torch.int16))
     pick = [0, 1, rows // 2, rows - 38, rows - 1]
