@@ -147,7 +147,7 @@ layernorm_kernel(const float *__restrict__ a, long long a_gstride, const float *
 constexpr int LNB_THREADS = 256;
 constexpr int LNB_CACHE = 8;   // float4 per thread: rows up to 8192 wide
 
-__global__ void __launch_bounds__(LNB_THREADS)
+__global__ void __launch_bounds__(LNB_THREADS, 4)
 layernorm_block_kernel(const float *__restrict__ a, long long a_gstride, const float *__restrict__ y,
                        const uint16_t *__restrict__ gamma, const uint16_t *__restrict__ beta, int groups, int rows,
                        int d, float eps, uint16_t *__restrict__ out) {
@@ -475,19 +475,30 @@ int launch_layernorm(const float *a, long long a_gstride, const float *y, const 
         return cuda_check(cudaGetLastError(), "layernorm: launch");
     }
     const long long warps = (long long)groups * rows;
-    // One CTA per row (layernorm_block_kernel) for up to 24 rows per SM of more than 1024 elements, and for rows
-    // of more than 4096 elements whatever their number.  Measured, 4 groups, us per launch, warp / CTA per row:
-    // 128 tokens d 2496 9.0 / 5.5, d 3120 11.3 / 6.2, d 7424 29.1 / 8.9; 512 tokens d 2496 16.0 / 11.4; 2048 tokens
-    // d 2496 48.0 / 56.7, d 3120 61.2 / 62.4, d 4992 121.7 / 80.3, d 7424 216.8 / 105.5 (a warp keeps 2048 elements
-    // in registers and goes over the rest of a wider row three times; keeping 4096 costs it more in occupancy).
-    // KRAKEN_LN_BLOCK=0/1 forces the choice.
+    // One CTA per row (layernorm_block_kernel) for rows of more than 2048 elements (a warp keeps 2048 in registers
+    // and would go over the rest of the row three times) and for up to 24 rows per SM of more than 1024 elements.
+    // Measured, 4 groups, us per launch, warp per row / CTA per row: 128 tokens d 2496 9.0 / 4.0, d 3120 11.3 / 4.5,
+    // d 7424 29.1 / 6.3; 512 tokens d 2496 16.0 / 11.2; 2048 tokens d 2496 48.2 / 45.5, d 3120 61.2 / 50.3,
+    // d 4992 121.7 / 66.7, d 7424 216.8 / 90.7; 8 groups d 3648 130.5 / 100.1; but d 2048 31.3 / 38.5 and 8 groups
+    // d 1920 53.1 / 71.9.  KRAKEN_LN_BLOCK=0/1 forces the choice.
     const int sms_b = sm_count() > 0 ? sm_count() : 148;
     const char *force_b = getenv("KRAKEN_LN_BLOCK");
-    const bool block_auto = d > 4096 || (d > 1024 && warps <= 24LL * sms_b);
+    const bool block_auto = d > 2048 || (d > 1024 && warps <= 24LL * sms_b);
     const bool block_rows = !ysum && d <= 4 * LNB_THREADS * LNB_CACHE &&
                             (force_b && (force_b[0] == '0' || force_b[0] == '1') ? force_b[0] == '1' : block_auto);
     if (block_rows) {
-        const long long ctas = warps < 8LL * sms_b ? warps : 8LL * sms_b;
+        // a grid of resident CTAs that walk the rows: no second wave with a ragged tail
+        static int per_sm = 0;
+        if (per_sm == 0) {
+            int n = 0;
+            if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, layernorm_block_kernel, LNB_THREADS, 0) != cudaSuccess || n < 1) {
+                cudaGetLastError();
+                n = 4;
+            }
+            per_sm = n;
+        }
+        const long long resident = (long long)per_sm * sms_b;
+        const long long ctas = warps < resident ? warps : resident;
         return cuda_check(launch_pdl(layernorm_block_kernel, dim3(static_cast<unsigned>(ctas)), dim3(LNB_THREADS), 0,
                                      stream, a, a_gstride, y, gamma, beta, groups, rows, d, eps, out),
                           "layernorm: launch");
