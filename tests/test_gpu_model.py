@@ -532,6 +532,49 @@ def test_c3_full_size_prefix_parity():
     prefix_parity("C3", 32, [0, 3])
 
 
+def test_c3_full_size_late_positions_agree_across_launch_configurations():
+    """C3 at full size, where the oracle can only afford a prefix: properties that hold at any size tie the late
+    positions down.  (1) A sequence run alone (other GEMM tile counts, attention with one CTA per item instead of
+    per-CTA work lists) gives the logits and cache rows it gives inside the batch of four.  (2) prefill(l - 1)
+    followed by one decode step (the cache-streaming kernels) gives the last-position logits of prefill(l).
+    (3) Equal sequences in different batch slots give equal results."""
+    s = ki.CONFIGS["C3"]
+    m, _ = build(s)
+    tok = ki.uniform_tokens(7, s.vocab, s.batch, s.seqlen, DEV)
+    tok[1] = tok[3]                                   # slots 1 and 3 hold the same sequence
+    full = m.prefill(tok).clone()
+    assert torch.isfinite(full).all() and m.device_status() == 0
+    assert torch.equal(full[1], full[3])
+    picks = [0, 127, 128, 1000, 1535, 1536, s.seqlen - 2, s.seqlen - 1]
+    keys = [(0, 0, 0), (s.n_layer // 2, 1, 1), (s.n_layer - 1, s.n_branch - 1, 0), (s.n_layer - 1, 2, 1)]
+    kv_full = {k: m.kv_view(*k)[2][:, picks].float().clone() for k in keys}
+    for k in keys:
+        assert torch.equal(m.kv_view(*k)[1][:, :s.seqlen], m.kv_view(*k)[3][:, :s.seqlen])
+    # (1) sequence 2 alone
+    m.reset()
+    one = m.prefill(tok[2:3].contiguous()).clone()
+    rel, mx = logits_metrics(one[0].cpu().numpy(), full[2].cpu().numpy())
+    print(f"[parity] C3 sequence alone vs inside the batch: relL2={rel:.3e} maxabs={mx:.3e}")
+    assert rel <= 1e-3 and mx <= 5e-3, (rel, mx)
+    for k in keys:
+        a, b = m.kv_view(*k)[0][:, picks].float(), kv_full[k]
+        assert (a - b).abs().max().item() <= 2.0 ** -6 * b.abs().max().item(), k
+        assert (a == b).float().mean().item() > 0.9, k
+    # (2) one token less, then a decode step
+    m.reset()
+    m.prefill(tok[:, :s.seqlen - 1].contiguous())
+    step = m.decode_step(tok[:, s.seqlen - 1].contiguous())
+    assert m.cur_len == s.seqlen and m.device_status() == 0
+    rel, mx = logits_metrics(step.cpu().numpy(), full.cpu().numpy())
+    print(f"[parity] C3 prefill({s.seqlen - 1}) + decode step vs prefill({s.seqlen}): relL2={rel:.3e} maxabs={mx:.3e}")
+    assert rel <= REL_L2_MAX and mx <= MAX_ABS_MAX, (rel, mx)   # two bf16 paths, each within the bound of the truth
+    # the token either path would pick scores within the two paths' distance of the other path's best
+    # (random-init logits are nearly flat, so the arg max itself may differ)
+    for b in range(s.batch):
+        assert full[b, step[b].argmax()].item() >= full[b].max().item() - 2 * mx, b
+    m.close()
+
+
 @pytest.mark.parametrize("name", ["C4", "C4-gqa4"])
 def test_c4_full_size_prefill_prefix_parity_and_decode_consistency(name):
     """C4 at full size (16 sequences x 2048 tokens, then decode steps), in the launch configuration
