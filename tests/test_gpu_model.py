@@ -518,6 +518,35 @@ def test_engine_head_dims_and_shared_kv_heads_small_models_all_positions_cache_a
     m.close()
 
 
+def test_long_context_8192_tokens_small_model_all_positions_and_decode():
+    """A context four times the benchmark's: 64 key tiles per head in the prefill attention (per-CTA work lists over
+    32 pairs of query tiles), a cache of 8192 rows for the split decode attention.  The model is small enough for the
+    oracle to run the whole prompt: logits at every position, the last cache rows, then decode steps."""
+    s = ki.KrakenShape("L8K", 2, 2, 128, 2, 256, 512, 8200, 1, 8192)
+    m, w = build(s)
+    wb = host_bits(w)
+    steps = 3
+    tok = ki.uniform_tokens(9, s.vocab, 1, s.seqlen + steps, DEV)
+    first = tok[:, :s.seqlen].contiguous()
+    got_all = m.prefill_all_logits(first).cpu().numpy()[0]
+    ids = first[0].cpu().numpy()
+    ref32, orc = oracle_all_logits(s, wb, ids, False)
+    refbf, orcbf = oracle_all_logits(s, wb, ids, True)
+    check_parity(got_all, ref32, refbf, "8192-token prompt, all positions")
+    for layer in range(s.n_layer):
+        for which in (0, 1):
+            g = m.kv_view(layer, 1, which)[0, :, :s.seqlen].float().cpu().numpy()
+            check_cache(g, orcbf.cache(layer, 1, which), layer == 0, ("L8K", layer, which))
+    assert m.device_status() == 0
+    for t in range(steps):
+        got = m.decode_step(tok[:, s.seqlen + t].contiguous()).cpu().numpy()
+        ref = orc.decode_step(int(tok[0, s.seqlen + t]))
+        rel, mx = logits_metrics(got[0], ref)
+        assert rel <= REL_L2_MAX and mx <= MAX_ABS_MAX, (t, rel, mx)
+    assert m.device_status() == 0 and m.cur_len == s.seqlen + steps
+    m.close()
+
+
 def test_engine_shape_1p3b_4way_full_size_prefix_parity():
     """The paper's 1.3B 4-way engine shape (d 1248 = 12 heads of 104, FFN 2496, vocabulary 51,200) at its full
     2048-token context, in the launch configuration the benchmark times."""
