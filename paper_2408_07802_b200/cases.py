@@ -25,6 +25,8 @@ def _gemm_args(kind, s, batch, seqlen, n_tile=0):
     T = batch * seqlen
     plain = kind.endswith("_plain")       # same shape, cheapest epilogue (bf16 store): isolates the mainloop
     kind = kind.replace("_plain", "")
+    resid_only = kind == "gemm_down_resid"   # the down-projection without the cross-branch sum (short prompts)
+    kind = kind.replace("_resid", "")
     K, Nout = {"gemm_qkv": (d, 3 * d), "gemm_proj": (d, d), "gemm_up": (d, F), "gemm_down": (F, d)}[kind]
     a = ki.normal_bf16(11, 0, (N, T, K), 1.0, DEV)
     w = ki.normal_bf16(11, 1, (N, Nout, K), 0.02, DEV)
@@ -64,7 +66,7 @@ def _gemm_args(kind, s, batch, seqlen, n_tile=0):
         g.resid, g.resid_gstride, g.ld_resid = r.data_ptr(), T * d, d
         keep += [o, r]
         out_bytes = N * T * d * 8
-        if kind == "gemm_down":
+        if kind == "gemm_down" and not resid_only:
             ssum = torch.empty(T, d, dtype=torch.float32, device=DEV)
             g.epilogue = kr.EPI_RESID_SUM
             g.sum, g.ld_sum = ssum.data_ptr(), d
@@ -156,7 +158,7 @@ def run_case(kind: str, workload: str, reps: int, warmup: int, n_tile: int = 0, 
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("case", help="gemm_qkv | gemm_proj | gemm_up | gemm_down | attention | layernorm | decode_attention | decode_gemm_{qkv,proj,up,down} | all | decode_all")
+    ap.add_argument("case", help="gemm_qkv | gemm_proj | gemm_up | gemm_down | gemm_down_resid | attention | layernorm | decode_attention | decode_gemm_{qkv,proj,up,down} | all | decode_all")
     ap.add_argument("--workload", default="C3")
     ap.add_argument("--reps", type=int, default=5)
     ap.add_argument("--warmup", type=int, default=2)

@@ -506,19 +506,13 @@ int launch_bn(const CUtensorMap &tmA, const CUtensorMap &tmB, const KernelArgs &
 int gemm_pick_bn(const GemmShape &s) {
     const int sms = sm_count() > 0 ? sm_count() : 148;
     const long long tiles_m = (s.m + BM - 1) / BM;
-    // CTA pairs on 256 x 256 tiles when that still gives every pair of SMs about two work items
-    {
-        const long long items = ((s.m + 2 * BM - 1) / (2 * BM)) * ((s.n_out + BN2 - 1) / BN2) * s.groups;
-        if (items >= sms && !env_flag("KRAKEN_GEMM_NO_PAIR")) return GEMM_TILE_PAIR;
-    }
-    // Plenty of tiles: the largest N tile that still gives every SM about two work items.
-    for (int bn : {256, 128}) {
-        const long long items = tiles_m * ((s.n_out + bn - 1) / bn) * s.groups;
-        if (items >= 2LL * sms) return bn;
-    }
-    // Few tiles (short prompts: the weights stream through once): the tile width decides how many rounds the
-    // SMs need, and a round costs about its width plus a fixed part (the A tile, set-up, drain).  156 tiles
-    // of 64 columns are two rounds on 148 SMs where 104 tiles of 96 columns are one.
+    const bool pairs_ok = !env_flag("KRAKEN_GEMM_NO_PAIR");
+    // CTA pairs on 256 x 256 tiles when that gives every pair of SMs about two work items
+    const long long pair_items = ((s.m + 2 * BM - 1) / (2 * BM)) * ((s.n_out + BN2 - 1) / BN2) * s.groups;
+    if (pair_items >= sms && pairs_ok) return GEMM_TILE_PAIR;
+    // Fewer tiles: the tile width decides how many rounds the SMs need, and a round costs about its width plus a
+    // fixed part (the A tile, set-up, drain).  156 tiles of 64 columns are two rounds on 148 SMs where 104 tiles
+    // of 96 columns are one.
     int best = 64;
     long long best_cost = -1;
     for (int bn = 256; bn >= 32; bn -= 32) {
@@ -529,6 +523,13 @@ int gemm_pick_bn(const GemmShape &s) {
             best_cost = cost;
             best = bn;
         }
+    }
+    // A pair's 256 x 256 tile is a 128 x 256 tile per SM that needs a third less operand fill, measured 0.92 of the
+    // single CTA's time at equal rounds (4 x 1024 x 1024 x 1024: 15.5 against 16.9 us; 4 x 512 x 2496 x 4992:
+    // 64.6 against 75.3).  Not with a single M tile, where half of every pair would idle.
+    if (pairs_ok && s.m > BM) {
+        const long long pair_rounds = (pair_items + sms / 2 - 1) / (sms / 2);
+        if (pair_rounds * 295 < best_cost) return GEMM_TILE_PAIR;
     }
     return best;
 }
