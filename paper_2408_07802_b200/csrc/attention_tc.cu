@@ -247,6 +247,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
+    pdl_wait();   // launched ahead of the end of its predecessor: nothing of the predecessor's is touched before here
 
     // Every role walks the same item sequence (blockIdx.x, + gridDim.x, ...) and keeps running
     // counters for the barrier phases, so the pipeline never drains between items.
@@ -529,8 +530,8 @@ int launch(const CUtensorMap &tmQ, const CUtensorMap &tmK, const CUtensorMap &tm
     b.balanced = items > sms && (rounds == 1 || couples * 100 >= 85LL * sms * rounds) &&
                  !env_flag("KRAKEN_ATTN_ONE_CTA_PER_ITEM");
     dim3 grid(static_cast<unsigned>(b.balanced ? (couples < sms ? couples : sms) : items));
-    attn_tc_kernel<HD><<<grid, ATC_THREADS, Cfg::SMEM_BYTES, stream>>>(tmQ, tmK, tmV, b);
-    return cuda_check(cudaGetLastError(), "attention: launch");
+    return cuda_check(launch_pdl(attn_tc_kernel<HD>, grid, dim3(ATC_THREADS), Cfg::SMEM_BYTES, stream, tmQ, tmK, tmV, b),
+                      "attention: launch");
 }
 
 }  // namespace

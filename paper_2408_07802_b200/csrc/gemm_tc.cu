@@ -120,6 +120,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
+    pdl_wait();   // launched ahead of the end of its predecessor: nothing of the predecessor's is touched before here
 
     if (warp == 0) {
         if (lane == 0) {
@@ -325,6 +326,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     cluster_sync_all();  // both CTAs' barriers exist before anything is signalled across the pair
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
+    pdl_wait();
 
     if (warp == 0) {
         if (lane == 0) {
@@ -483,8 +485,8 @@ int launch_pair(const CUtensorMap &tmA, const CUtensorMap &tmB, const KernelArgs
     const long long tiles = (long long)((ka.shape.m + 2 * BM - 1) / (2 * BM)) * ka.tiles_n;
     const long long units = ka.group_serial ? tiles : tiles * ka.shape.groups;
     const int clusters = static_cast<int>(units < max_clusters ? units : max_clusters);
-    gemm_tc_pair_kernel<<<2 * clusters, NUM_THREADS, Cfg::SMEM_BYTES, stream>>>(tmA, tmB, ka);
-    return cuda_check(cudaGetLastError(), "gemm pair: launch");
+    return cuda_check(launch_pdl(gemm_tc_pair_kernel, dim3(2 * clusters), dim3(NUM_THREADS), Cfg::SMEM_BYTES, stream, tmA, tmB, ka),
+                      "gemm pair: launch");
 }
 
 template <int BN>
@@ -497,8 +499,8 @@ int launch_bn(const CUtensorMap &tmA, const CUtensorMap &tmB, const KernelArgs &
         if (rc) return rc;
         configured = true;
     }
-    gemm_tc_kernel<BN><<<grid, NUM_THREADS, Cfg::SMEM_BYTES, stream>>>(tmA, tmB, ka);
-    return cuda_check(cudaGetLastError(), "gemm: launch");
+    return cuda_check(launch_pdl(gemm_tc_kernel<BN>, dim3(grid), dim3(NUM_THREADS), Cfg::SMEM_BYTES, stream, tmA, tmB, ka),
+                      "gemm: launch");
 }
 
 }  // namespace
