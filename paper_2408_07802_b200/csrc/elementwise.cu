@@ -270,6 +270,7 @@ layernorm_stream_kernel(const float *__restrict__ a, long long a_gstride, const 
         reinterpret_cast<uint2 *>(s_beta)[i] = beta ? __ldg(reinterpret_cast<const uint2 *>(beta) + i) : make_uint2(0u, 0u);
     }
     __syncthreads();
+    pdl_wait();   // gamma and beta are weights; everything below touches what the predecessor wrote
     const int n_units = (rows - static_cast<int>(blockIdx.x) + static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x);
 
     if (warp == n_consumers) {
@@ -470,8 +471,9 @@ int launch_layernorm(const float *a, long long a_gstride, const float *y, const 
             if (rc) return rc;
             configured[which] = true;
         }
-        kern<<<dim3(sms), dim3((n_consumers + 1) * 32), smem, stream>>>(a, a_gstride, y, gamma, beta, groups, rows, d, eps,
-                                                                     out, stages, n_consumers, status);
+        const cudaError_t ce = launch_pdl(kern, dim3(sms), dim3((n_consumers + 1) * 32), smem, stream, a, a_gstride, y, gamma,
+                                          beta, groups, rows, d, eps, out, stages, n_consumers, status);
+        if (ce != cudaSuccess) return cuda_check(ce, "layernorm: launch");
         return cuda_check(cudaGetLastError(), "layernorm: launch");
     }
     const long long warps = (long long)groups * rows;
