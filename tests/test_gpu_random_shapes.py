@@ -175,3 +175,14 @@ def test_whole_model_random_configurations(seed):
             assert rel <= REL_L2_MAX and mx <= MAX_ABS_MAX, (s, t, b, rel, mx)
     assert m.device_status() == 0 and m.cur_len == seqlen + steps
     m.close()
+
+
+@pytest.mark.parametrize("seed", range(6))
+def test_packed_prefill_random_lengths(seed):
+    """Packed (ragged) batches with random numbers of sequences and random lengths, then ragged decode steps."""
+    from test_gpu_model import test_packed_prefill_and_ragged_decode as packed_case
+    rng = np.random.default_rng(7000 + seed)
+    name = str(rng.choice(["C0", "K0-104", "C0-gqa", "K0-72"]))
+    s = ki.CONFIGS[name]
+    lens = [int(x) for x in rng.integers(1, s.max_pos - 5, size=int(rng.integers(1, 7)))]
+    packed_case(name, lens)
