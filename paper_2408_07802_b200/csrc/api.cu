@@ -265,6 +265,13 @@ EpiParams epi_zero() {
         if (_rc) return _rc; \
     } while (0)
 
+int branch_streams(kraken_handle *h);
+
+#define KR_CU(x)                                              \
+    do {                                                      \
+        if ((x) != cudaSuccess) return cuda_check(cudaGetLastError(), "streams and events"); \
+    } while (0)
+
 // Runs the L layers on `T = batch * seqlen` new tokens at positions pos0 .. pos0 + seqlen - 1.
 int run_layers(const RunCtx &rc, const int32_t *d_tokens) {
     kraken_handle *h = rc.h;
@@ -278,6 +285,8 @@ int run_layers(const RunCtx &rc, const int32_t *d_tokens) {
     const bool small_rows = !h->naive && (T <= SKINNY_MAX_ROWS || down_tiles < (sm_count() > 0 ? sm_count() : 148) / 2);
     // between the two: all groups of the down-projection run side by side and one streaming pass adds the N outputs
     const bool sum_pass = small_rows && T > SKINNY_MAX_ROWS;
+    const bool sum_beside = sum_pass && !rc.stage && !env_flag("KRAKEN_SUM_IN_LINE") && branch_streams(h) == KRAKEN_OK;
+    bool sum_pending = false;
     float *x0 = at<float>(h, h->lay.x0), *x = at<float>(h, h->lay.x), *a = at<float>(h, h->lay.a),
           *S = at<float>(h, h->lay.s);
     uint16_t *u = at<uint16_t>(h, h->lay.u), *q = at<uint16_t>(h, h->lay.q), *o = at<uint16_t>(h, h->lay.o),
@@ -390,6 +399,10 @@ int run_layers(const RunCtx &rc, const int32_t *d_tokens) {
                                     h->w.ln2_b ? (const uint16_t *)h->w.ln2_b + ln_off : nullptr, N, T, d, c.ln_eps,
                                     u, rc.st, nullptr, 0, 0, status));
         } else if (!c.parallel_ffn) {
+            if (sum_pending) {
+                KR_CU(cudaStreamWaitEvent(rc.st, h->ev_join[1], 0));
+                sum_pending = false;
+            }
             LaunchScope scope(h, KRAKEN_PROF_LAYERNORM, rc.st);
             // with few rows the cross-branch sum is formed here from the N branch inputs (same order as
             // the down-projection epilogue forms it for long prompts)
@@ -411,10 +424,26 @@ int run_layers(const RunCtx &rc, const int32_t *d_tokens) {
         e.resid = a; e.resid_gstride = td; e.ld_resid = d;
         e.sum = S; e.ld_sum = d;
         KR_TRY(model_gemm(rc, G_DOWN, l, T, gb, (long long)T * F, e));
-        if ((sum_pass && l + 1 < L && !c.no_combine) || rc.stage == STAGE_FFN) {
-            // (driven from outside: the sum of this device's branches, for the caller's all-reduce)
+        if (rc.stage == STAGE_FFN) {
+            // driven from outside: the sum of this device's branches, for the caller's all-reduce
             LaunchScope scope(h, KRAKEN_PROF_LAYERNORM, rc.st);
             KR_TRY(launch_sum_groups(x, td, N, td, S, rc.st));
+        } else if (sum_pass && l + 1 < L && !c.no_combine) {
+            // The sum is first read by the next layer's second LayerNorm, so it runs beside that layer's
+            // attention half on a stream of its own (x is not written again, nor S read, before the join).
+            if (sum_beside) {
+                KR_CU(cudaEventRecord(h->ev_fork, rc.st));
+                KR_CU(cudaStreamWaitEvent(h->br_stream[1], h->ev_fork, 0));
+            }
+            cudaStream_t ss = sum_beside ? h->br_stream[1] : rc.st;
+            {
+                LaunchScope scope(h, KRAKEN_PROF_LAYERNORM, ss);
+                KR_TRY(launch_sum_groups(x, td, N, td, S, ss));
+            }
+            if (sum_beside) {
+                KR_CU(cudaEventRecord(h->ev_join[1], ss));
+                sum_pending = true;
+            }
         }
     }
     h->last_rows = T;
@@ -463,10 +492,6 @@ int run_layers_decode_branches(const RunCtx &rc, const int32_t *d_tokens) {
     uint16_t *kv = reinterpret_cast<uint16_t *>(h->kv);
     auto stream_of = [&](int b) { return b == 0 ? rc.st : h->br_stream[b]; };
     auto out_of = [&](int l) { return xbuf[(L - 1 - l) & 1]; };   // the last layer lands in the main buffer
-#define KR_CU(x)                                              \
-    do {                                                      \
-        if ((x) != cudaSuccess) return cuda_check(cudaGetLastError(), "decode branch chains"); \
-    } while (0)
 
     {
         LaunchScope scope(h, KRAKEN_PROF_EMBED, rc.st);
