@@ -55,7 +55,7 @@ __device__ __forceinline__ float warp_sum(float v) {
 // launches of more CTAs than three per SM (4096 rows of 1024: 8.8 -> 5.7 us).  Launches of few rows keep the full
 // build: a decode step measured 4 % slower with the trimmed one.
 template <int LN_CACHE, bool YSUM, bool DENSE = false>
-__global__ void __launch_bounds__(ROW_WARPS * 32, LN_CACHE == 8 ? (DENSE ? 4 : 3) : 0)
+__global__ void __launch_bounds__(ROW_WARPS * 32, LN_CACHE == 8 ? (DENSE ? 4 : 2) : 0)
 layernorm_kernel(const float *__restrict__ a, long long a_gstride, const float *__restrict__ y,
                  const float *__restrict__ ysum, long long ysum_gstride, int ysum_groups,
                  const uint16_t *__restrict__ gamma, const uint16_t *__restrict__ beta, int groups, int rows, int d,
@@ -87,6 +87,21 @@ layernorm_kernel(const float *__restrict__ a, long long a_gstride, const float *
         return t;
     };
 
+    // Launches of few rows (a decode step) are a chain of dependent round trips to L2; there gamma and beta are
+    // requested together with the row instead of after the statistics.
+    constexpr bool EARLY_GB = LN_CACHE == 8 && !DENSE;
+    const uint2 *pg = nullptr, *pb = nullptr;
+    uint2 gmc[EARLY_GB ? LN_CACHE : 1], btc[EARLY_GB ? LN_CACHE : 1];
+    if (EARLY_GB) {
+        pg = reinterpret_cast<const uint2 *>(gamma + (size_t)g * d);
+        pb = beta ? reinterpret_cast<const uint2 *>(beta + (size_t)g * d) : nullptr;
+#pragma unroll
+        for (int i = 0; i < LN_CACHE; ++i) {
+            const int v = lane + 32 * i;
+            gmc[EARLY_GB ? i : 0] = v < nvec ? __ldg(pg + v) : make_uint2(0u, 0u);
+            btc[EARLY_GB ? i : 0] = (pb && v < nvec) ? __ldg(pb + v) : make_uint2(0u, 0u);
+        }
+    }
     float4 cache[LN_CACHE];
     float sum = 0.f;
 #pragma unroll
@@ -121,23 +136,28 @@ layernorm_kernel(const float *__restrict__ a, long long a_gstride, const float *
     const float rstd = rsqrtf(warp_sum(sq) / d + eps);
     pdl_trigger();
 
-    const uint2 *pg = reinterpret_cast<const uint2 *>(gamma + (size_t)g * d);
-    const uint2 *pb = beta ? reinterpret_cast<const uint2 *>(beta + (size_t)g * d) : nullptr;
+    if (!EARLY_GB) {
+        pg = reinterpret_cast<const uint2 *>(gamma + (size_t)g * d);
+        pb = beta ? reinterpret_cast<const uint2 *>(beta + (size_t)g * d) : nullptr;
+    }
     uint2 *po = reinterpret_cast<uint2 *>(out + ((size_t)g * rows + r) * d);
-    auto emit = [&](int v, const float4 &t) {
-        const uint2 gm = __ldg(pg + v);
-        uint2 bt = make_uint2(0u, 0u);
-        if (pb) bt = __ldg(pb + v);
+    auto emit_gb = [&](int v, const float4 &t, const uint2 gm, const uint2 bt) {
         const float o0 = (t.x - mean) * rstd * h16_lo(gm.x) + h16_lo(bt.x);
         const float o1 = (t.y - mean) * rstd * h16_hi(gm.x) + h16_hi(bt.x);
         const float o2 = (t.z - mean) * rstd * h16_lo(gm.y) + h16_lo(bt.y);
         const float o3 = (t.w - mean) * rstd * h16_hi(gm.y) + h16_hi(bt.y);
         po[v] = make_uint2(pack_h16x2(o0, o1), pack_h16x2(o2, o3));
     };
+    auto emit = [&](int v, const float4 &t) {
+        emit_gb(v, t, __ldg(pg + v), pb ? __ldg(pb + v) : make_uint2(0u, 0u));
+    };
 #pragma unroll
     for (int i = 0; i < LN_CACHE; ++i) {
         const int v = lane + 32 * i;
-        if (v < nvec) emit(v, cache[i]);
+        if (v < nvec) {
+            if (EARLY_GB) emit_gb(v, cache[i], gmc[EARLY_GB ? i : 0], btc[EARLY_GB ? i : 0]);
+            else emit(v, cache[i]);
+        }
     }
     for (int v = lane + 32 * LN_CACHE; v < nvec; v += 32) emit(v, load(v));
 }
