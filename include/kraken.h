@@ -229,6 +229,26 @@ const char *kraken_last_cuda_error(void);
 /* 16-bit storage type this image was built for: 0 = bfloat16, 1 = IEEE half. */
 int kraken_storage_dtype(void);
 
+/* Hooks for tests and measurements (not part of the model's arithmetic).  Where the library has two kernels
+ * for one step that give the same result and picks by shape, a test can force either one, process-wide:
+ * value 0 restores the library's own choice.  Nothing on the launch path reads the environment; the two
+ * environment switches of a handle (KRAKEN_NO_GRAPH, KRAKEN_DECODE_ONE_CHAIN) are read once by kraken_create.
+ * Errors: EINVAL (unknown key, value outside 0..2). */
+typedef enum kraken_tuning_key {
+    KRAKEN_TUNE_LN_ROW_KERNEL = 0,   /* LayerNorm of few or wide rows: 1 = one warp per row, 2 = one CTA per row */
+    KRAKEN_TUNE_ATTN_SCHEDULE = 1,   /* prefill attention: 1 = one CTA per work item (no per-CTA work lists)     */
+    KRAKEN_TUNE_COUNT = 2
+} kraken_tuning_key;
+int kraken_tuning_set(int32_t key, int32_t value);
+
+/* Makes one bounded wait run out, harmlessly: a single small CTA waits, with the library's own wait routine
+ * and a limit of limit_us microseconds (1 .. 1,000,000), on a barrier that nothing ever signals and that has
+ * no copy in flight, then takes the same way out as the model kernels do: it returns normally and raises
+ * bit 1 of *d_status (device uint32).  Asynchronous on `stream`; the context stays usable.  This is how
+ * the failure path of the kernels' waits (Sec. 3.1's steps never block forever here) is exercised
+ * without starving a real kernel.  Errors: EINVAL, ECUDA. */
+int kraken_test_wait_limit(uint32_t *d_status, uint32_t limit_us, void *stream);
+
 /* ------------------------------------------------------------------------------------------
  * Single steps of the path, exposed so that each kernel can be checked on its own.  All
  * pointers are device pointers.  G is the number of groups (branches); a group stride of 0
@@ -328,12 +348,16 @@ int kraken_decode_attention_sizes(int32_t groups, int32_t batch, int32_t n_keys,
  * implies.  The split-KV partials go to a fixed 8 MiB array inside the library image (held by every
  * GPU that loads the library, until the process exits); the call itself allocates nothing, on the
  * host side of CUDA or on the device.
- *   - Same arguments, layouts and results as kraken_op_decode_attention (q, out: device bf16
- *     [G][batch, n_head*head_dim]; caches as there; splits = 0 lets the library choose).
+ *   - Same layouts and results as kraken_op_decode_attention with n_kv_head = n_head (q, out: device bf16
+ *     [G][batch, n_head*head_dim]; caches as there with one key/value head per query head: there is no
+ *     grouped-query form of this call; splits = 0 lets the library choose); the same head dims are
+ *     accepted (64, 72, 96, 104, 128; EUNSUPPORTED otherwise).
  *   - ECAPACITY when groups * batch * n_head * splits * (head_dim + 2) * 4 bytes exceeds
  *     kraken_decode_attention_static_capacity(); pass a smaller `splits` (1 needs no partials).
  *   - The first call on each device looks up the array's device address (once per device, with that
- *     device current); make that first call before starting any stream capture.
+ *     device current); make that first call before starting any stream capture.  On EVERY call the
+ *     current device must be the one that owns `stream`, q and out: the array is per device, and
+ *     the call checks where q lives and returns EINVAL when that is another device.
  *   - All calls share the one array and it keeps whatever the previous call left.  Nothing in it has
  *     to start at zero: each call overwrites every partial it later reads.  Two calls whose kernels
  *     may overlap on the GPU (different streams) race on it; serialise them. */

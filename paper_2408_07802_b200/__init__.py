@@ -40,7 +40,11 @@ EXPORTS = (
     "kraken_op_embed", "kraken_op_layernorm", "kraken_op_grouped_gemm", "kraken_op_attention",
     "kraken_op_decode_attention", "kraken_decode_attention_sizes",
     "kraken_op_decode_attention_static", "kraken_decode_attention_static_capacity", "kraken_storage_dtype",
+    "kraken_tuning_set", "kraken_test_wait_limit",
 )
+
+TUNE_LN_ROW_KERNEL, TUNE_ATTN_SCHEDULE = 0, 1
+STATUS_BAD_TOKEN, STATUS_WAIT_LIMIT = 1, 2
 
 
 class KrakenConfig(C.Structure):
@@ -151,6 +155,8 @@ def lib(dtype: Optional[str] = None) -> C.CDLL:
         L.kraken_decode_attention_static_capacity.argtypes = []
         L.kraken_decode_attention_static_capacity.restype = C.c_size_t
         L.kraken_storage_dtype.argtypes = []
+        L.kraken_tuning_set.argtypes = [i32, i32]
+        L.kraken_test_wait_limit.argtypes = [vp, C.c_uint32, vp]
         if L.kraken_storage_dtype() != (1 if dtype == "f16" else 0):
             raise RuntimeError(f"{path} was not built for storage dtype {dtype}")
         _libs[dtype] = L
@@ -446,13 +452,17 @@ def op_decode_attention(q: torch.Tensor, k_cache: torch.Tensor, v_cache: torch.T
 
 
 def op_decode_attention_static(q: torch.Tensor, k_cache: torch.Tensor, v_cache: torch.Tensor, n_keys: int,
-                               splits: int = 0) -> torch.Tensor:
+                               splits: int = 0, out: Optional[torch.Tensor] = None) -> torch.Tensor:
     """op_decode_attention for callers that cannot provide scratch: the partials live in a fixed
     array inside the library (see kraken_op_decode_attention_static).  The output tensor is still the
-    caller's; this wrapper creates it with torch only for convenience."""
+    caller's; this wrapper creates it with torch only when `out` is not given."""
     G, B, d = q.shape
     _, _, H, P, hd = k_cache.shape
-    out = torch.empty_like(q)
+    if H * hd != d:
+        raise ValueError("kraken_op_decode_attention_static has no grouped-query form: the cache must hold one "
+                         f"key/value head per query head (cache heads {H} x head_dim {hd} != d {d})")
+    if out is None:
+        out = torch.empty_like(q)
     _check(lib().kraken_op_decode_attention_static(q.data_ptr(), q.stride(0), k_cache.data_ptr(), v_cache.data_ptr(),
                                                    k_cache.stride(0), k_cache.stride(1), G, B, n_keys, H, hd, P,
                                                    splits, out.data_ptr(), out.stride(0), _stream()),
@@ -462,3 +472,26 @@ def op_decode_attention_static(q: torch.Tensor, k_cache: torch.Tensor, v_cache: 
 
 def decode_attention_static_capacity() -> int:
     return int(lib().kraken_decode_attention_static_capacity())
+
+
+def set_tuning(key: int, value: int) -> None:
+    """Test / measurement hook: forces one of two equivalent kernels for a step (0 = the library's choice)."""
+    _check(lib().kraken_tuning_set(int(key), int(value)), "kraken_tuning_set")
+
+
+@contextlib.contextmanager
+def tuning(key: int, value: int):
+    set_tuning(key, value)
+    try:
+        yield
+    finally:
+        set_tuning(key, 0)
+
+
+def test_wait_limit(status: torch.Tensor, limit_us: int) -> None:
+    """Launches the probe whose bounded wait runs out after limit_us microseconds and raises bit 1 of `status`
+    (a device int32/uint32 word)."""
+    _check(lib().kraken_test_wait_limit(status.data_ptr(), int(limit_us), _stream()), "kraken_test_wait_limit")
+
+
+test_wait_limit.__test__ = False   # not a pytest case

@@ -26,8 +26,6 @@ struct Layout {
 
 int kv_heads_of(const kraken_config &c) { return c.n_kv_head > 0 ? c.n_kv_head : c.n_head; }
 
-bool decode_head_dim_ok(int hd) { return hd == 64 || hd == 72 || hd == 96 || hd == 104 || hd == 128; }
-
 int check_config(const kraken_config *c) {
     if (!c) return KRAKEN_EINVAL;
     if (c->n_branch < 1 || c->n_layer < 1 || c->d_model < 1 || c->n_head < 1 || c->d_ff < 1 || c->vocab < 1 ||
@@ -100,13 +98,13 @@ struct kraken_handle {
     bool stage_decode;      // the pieces being driven are a decode step (one new token per sequence)
     std::vector<int> host_rows, host_row_seq, host_row_pos;   // staging of the packed-prefill tables
     cudaStream_t last_stream;
-    bool naive;
+    bool one_chain;   // decode steps keep all branches in one chain of launches (KRAKEN_DECODE_ONE_CHAIN at create)
     // weight tensor maps, one per GEMM kind, re-encoded when the N tile changes
     CUtensorMap tmB[G_COUNT];
     int tmB_bn[G_COUNT];
-    // activation tensor maps, re-encoded when the token count changes
+    // activation tensor maps, re-encoded when anything they describe changes (base, rows, groups, group stride)
     CUtensorMap tmA[G_COUNT];
-    int tmA_rows[G_COUNT];
+    struct AKey { const void *base; int rows, groups; long long gstride; } tmA_key[G_COUNT];
     // decode steps replayed as a CUDA graph: positions are read from `pos` in device memory, tokens
     // and logits go through the staging buffers, so one graph serves every step of a batch size
     // a prefill with the same shape and buffers as the previous one is replayed as a graph too (it has a
@@ -230,7 +228,6 @@ int model_gemm(const RunCtx &rc, GemmKind kind, int layer, int m_rows, const uin
     static const int cat_of[G_COUNT] = {KRAKEN_PROF_GEMM_QKV, KRAKEN_PROF_GEMM_PROJ, KRAKEN_PROF_GEMM_UP,
                                         KRAKEN_PROF_GEMM_DOWN, KRAKEN_PROF_TAIL, KRAKEN_PROF_TAIL};
     LaunchScope scope(h, cat_of[kind], st);
-    if (h->naive) return launch_gemm_naive(op, s, epi, st);
     if (m_rows <= SKINNY_MAX_ROWS && epi.kind != KRAKEN_EPI_RESID_SUM) return launch_gemm_skinny(op, s, epi, st);
 
     const int bn = gemm_pick_bn(s);
@@ -244,10 +241,13 @@ int model_gemm(const RunCtx &rc, GemmKind kind, int layer, int m_rows, const uin
         h->tmB_bn[kind] = bn;
     }
     // A maps: the up-projection reads the same buffer as qkv but after LN2, same shape -> same map works.
-    if (h->tmA_rows[kind] != m_rows) {
+    // (a run of branches starting at g0 > 0 has its own base pointer, so it never reuses another run's map)
+    const kraken_handle::AKey key{a, m_rows, s.groups, a_gstride};
+    kraken_handle::AKey &have = h->tmA_key[kind];
+    if (have.base != key.base || have.rows != key.rows || have.groups != key.groups || have.gstride != key.gstride) {
         int r = gemm_encode_a(&h->tmA[kind], op, s);
         if (r) return r;
-        h->tmA_rows[kind] = m_rows;
+        have = key;
     }
     return launch_gemm_tc(op, s, epi, &h->tmA[kind], &h->tmB[kind], layered ? layer * N + g0 : 0, bn,
                           at<uint32_t>(h, h->lay.status), st);
@@ -282,10 +282,10 @@ int run_layers(const RunCtx &rc, const int32_t *d_tokens) {
     // output tile on one CTA (pair); with too few output tiles that would idle most SMs, so then (and in
     // decode) LayerNorm-2 of the next layer sums the N branch inputs itself, in the same order.
     const long long down_tiles = (long long)((T + 255) / 256) * ((d + 255) / 256);
-    const bool small_rows = !h->naive && (T <= SKINNY_MAX_ROWS || down_tiles < (sm_count() > 0 ? sm_count() : 148) / 2);
+    const bool small_rows = (T <= SKINNY_MAX_ROWS || down_tiles < (sm_count() > 0 ? sm_count() : 148) / 2);
     // between the two: all groups of the down-projection run side by side and one streaming pass adds the N outputs
     const bool sum_pass = small_rows && T > SKINNY_MAX_ROWS;
-    const bool sum_beside = sum_pass && !rc.stage && !env_flag("KRAKEN_SUM_IN_LINE") && branch_streams(h) == KRAKEN_OK;
+    const bool sum_beside = sum_pass && !rc.stage && branch_streams(h) == KRAKEN_OK;
     bool sum_pending = false;
     float *x0 = at<float>(h, h->lay.x0), *x = at<float>(h, h->lay.x), *a = at<float>(h, h->lay.a),
           *S = at<float>(h, h->lay.s);
@@ -349,17 +349,9 @@ int run_layers(const RunCtx &rc, const int32_t *d_tokens) {
                     sp.k_cache = ap.k_cache + b * cache_b;
                     sp.v_cache = ap.v_cache + b * cache_b;
                     if (b > 0) h->launches[KRAKEN_PROF_ATTENTION]++;
-                    if (h->naive) {
-                        KR_TRY(launch_attention_naive(sp, rc.st));
-                    } else if (attention_tc_supported(sp) && !env_flag("KRAKEN_ATTN_WARP_MMA")) {
-                        KR_TRY(launch_attention_tc(sp, nullptr, nullptr, nullptr, status, rc.st));
-                    } else {
-                        KR_TRY(launch_attention_prefill(sp, rc.st));
-                    }
+                    KR_TRY(launch_attention_tc(sp, nullptr, nullptr, nullptr, status, rc.st));
                     row0 += h->seq_len[b];
                 }
-            } else if (h->naive) {
-                KR_TRY(launch_attention_naive(ap, rc.st));
             } else if (rc.seqlen == 1) {
                 // decode step: stream the cache with the split-KV kernel
                 DecodeAttnParams dp;
@@ -376,10 +368,8 @@ int run_layers(const RunCtx &rc, const int32_t *d_tokens) {
                 dp.out = o; dp.out_gstride = td;
                 h->launches[KRAKEN_PROF_ATTENTION] += dp.splits > 1 ? 1 : 0;
                 KR_TRY(launch_attention_decode(dp, rc.st));
-            } else if (attention_tc_supported(ap) && !env_flag("KRAKEN_ATTN_WARP_MMA")) {
-                KR_TRY(launch_attention_tc(ap, nullptr, nullptr, nullptr, status, rc.st));
             } else {
-                KR_TRY(launch_attention_prefill(ap, rc.st));
+                KR_TRY(launch_attention_tc(ap, nullptr, nullptr, nullptr, status, rc.st));
             }
         }
         // x = res + MHA(x)
@@ -833,7 +823,8 @@ int kraken_create(const kraken_config *cfg, const kraken_weights *w, void *d_kv,
     h->last_seqlen = 0;
     h->last_rows = 0;
     h->last_stream = nullptr;
-    h->naive = env_flag("KRAKEN_NAIVE");
+    // the two environment switches of a handle are read here, once; nothing on the launch path reads the environment
+    h->one_chain = env_flag("KRAKEN_DECODE_ONE_CHAIN");
     h->prof_on = false;
     h->dec_graph = nullptr;
     h->pre_graph = nullptr;
@@ -846,12 +837,12 @@ int kraken_create(const kraken_config *cfg, const kraken_weights *w, void *d_kv,
     h->stage_decode = false;
     h->dec_graph_batch = 0;
     h->dec_eager_steps = 0;
-    h->use_graph = !env_flag("KRAKEN_NO_GRAPH") && !h->naive;
+    h->use_graph = !env_flag("KRAKEN_NO_GRAPH");
     h->ev_used = 0;
     for (int i = 0; i < KRAKEN_PROF_COUNT; ++i) h->launches[i] = 0;
     for (int i = 0; i < G_COUNT; ++i) {
         h->tmB_bn[i] = 0;
-        h->tmA_rows[i] = 0;
+        h->tmA_key[i] = {nullptr, 0, 0, 0};
     }
     if (cudaMemset(h->scratch + lay.status, 0, 256) != cudaSuccess) {
         delete h;
@@ -1024,7 +1015,7 @@ namespace {
 
 // Whether decode steps of this handle run the branches as concurrent chains.
 bool decode_chains(const kraken_handle *h) {
-    return !h->naive && h->cfg.n_branch >= 2 && h->cfg.n_branch <= MAX_CHAINS && !env_flag("KRAKEN_DECODE_ONE_CHAIN");
+    return h->cfg.n_branch >= 2 && h->cfg.n_branch <= MAX_CHAINS && !h->one_chain;
 }
 
 // The kernel sequence of one decode step; with from_dev the position is read from device memory.
@@ -1225,6 +1216,8 @@ int kraken_profile_read(kraken_handle *h, double *ms, int64_t *launches) {
 
 const char *kraken_last_cuda_error(void) { return last_cuda_error(); }
 
+int kraken_tuning_set(int32_t key, int32_t value) { return set_tuning(key, value); }
+
 int kraken_storage_dtype(void) { return KRAKEN_F16 ? 1 : 0; }
 
 const char *kraken_strerror(int status) {
@@ -1287,7 +1280,6 @@ int kraken_op_grouped_gemm(const kraken_gemm_args *g, uint32_t *d_status, void *
     e.d_model = g->n_head * g->head_dim;
     e.n_kv_head = g->n_kv_head > 0 ? g->n_kv_head : g->n_head;
     e.gelu_tanh = g->gelu_tanh;
-    if (env_flag("KRAKEN_NAIVE")) return launch_gemm_naive(op, s, e, static_cast<cudaStream_t>(stream));
     if (g->n_tile == 8) return launch_gemm_skinny(op, s, e, static_cast<cudaStream_t>(stream));
     return launch_gemm_tc(op, s, e, nullptr, nullptr, 0, g->n_tile, d_status, static_cast<cudaStream_t>(stream));
 }
@@ -1304,10 +1296,8 @@ int kraken_op_attention(const void *q, int64_t q_gstride, const void *k_cache, c
     p.cache_gstride = cache_gstride; p.cache_bstride = cache_bstride;
     p.groups = groups; p.batch = batch; p.seqlen = seqlen; p.pos0 = pos0; p.n_head = n_head; p.head_dim = head_dim;
     p.max_pos = max_pos; p.out = (uint16_t *)out; p.out_gstride = out_gstride;
-    if (env_flag("KRAKEN_NAIVE")) return launch_attention_naive(p, static_cast<cudaStream_t>(stream));
-    if (attention_tc_supported(p) && !env_flag("KRAKEN_ATTN_WARP_MMA"))
-        return launch_attention_tc(p, nullptr, nullptr, nullptr, nullptr, static_cast<cudaStream_t>(stream));
-    return launch_attention_prefill(p, static_cast<cudaStream_t>(stream));
+    // one kernel serves every supported layout; a cache with gaps between its rows or heads is refused
+    return launch_attention_tc(p, nullptr, nullptr, nullptr, nullptr, static_cast<cudaStream_t>(stream));
 }
 
 int kraken_op_decode_attention(const void *q, int64_t q_gstride, const void *k_cache, const void *v_cache,

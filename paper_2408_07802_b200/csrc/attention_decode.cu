@@ -396,7 +396,7 @@ int launch(const DecodeAttnParams &p, cudaStream_t stream) {
     dim3 grid(p.splits, n_kv * (rep / qh), p.batch * p.groups);
     cudaError_t ce;
     if constexpr (HD == 64 || HD == 128) {
-        if (decode_gqa_tile(p.n_head, n_kv) && !env_flag("KRAKEN_DECODE_GQA_SIMT")) {
+        if (decode_gqa_tile(p.n_head, n_kv)) {
             DecodeAttnParams q = p;
             q.n_kv_head = n_kv;
             ce = launch_pdl(attn_decode_gqa_kernel<HD>, dim3(p.splits, n_kv, p.batch * p.groups), dim3(DEC_WARPS * 32), 0,

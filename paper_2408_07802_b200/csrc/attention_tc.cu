@@ -507,17 +507,17 @@ template <int HD>
 int launch(const CUtensorMap &tmQ, const CUtensorMap &tmK, const CUtensorMap &tmV, const AttnTcArgs &a,
            cudaStream_t stream) {
     using Cfg = AtcCfg<HD>;
-    static bool configured = false;
-    if (!configured) {
+    static DeviceOnce configured;
+    if (!configured.done()) {
         int rc = cuda_check(cudaFuncSetAttribute(attn_tc_kernel<HD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                  Cfg::SMEM_BYTES), "attention: shared memory opt-in");
         if (rc) return rc;
-        configured = true;
+        configured.set();
     }
     const long long items = (long long)((a.seqlen + 2 * TQ - 1) / (2 * TQ)) * a.n_head * a.batch * a.groups;
     // With more items than SMs, each CTA walks a fixed list of couples of equal total length (atc_next); a plain
     // round-robin list of single items measured slower than one CTA per item (0.38 vs 0.35 ms at 4 x 2048 x 16
-    // heads x 128) because the items are so unequal.  KRAKEN_ATTN_ONE_CTA_PER_ITEM=1 keeps the hardware scheduler.
+    // heads x 128) because the items are so unequal.  KRAKEN_TUNE_ATTN_SCHEDULE = 1 keeps the hardware scheduler.
     const int sms = sm_count() > 0 ? sm_count() : 148;
     const long long couples = (long long)(((a.seqlen + 2 * TQ - 1) / (2 * TQ) + 1) / 2) * a.n_head * a.batch * a.groups;
     AttnTcArgs b = a;
@@ -528,7 +528,7 @@ int launch(const CUtensorMap &tmQ, const CUtensorMap &tmK, const CUtensorMap &tm
     // the longest item alone sets the time, which a couple would only lengthen.
     const long long rounds = (couples + sms - 1) / sms;
     b.balanced = items > sms && (rounds == 1 || couples * 100 >= 85LL * sms * rounds) &&
-                 !env_flag("KRAKEN_ATTN_ONE_CTA_PER_ITEM");
+                 tuning(KRAKEN_TUNE_ATTN_SCHEDULE) != 1;
     dim3 grid(static_cast<unsigned>(b.balanced ? (couples < sms ? couples : sms) : items));
     return cuda_check(launch_pdl(attn_tc_kernel<HD>, grid, dim3(ATC_THREADS), Cfg::SMEM_BYTES, stream, tmQ, tmK, tmV, b),
                       "attention: launch");

@@ -16,15 +16,23 @@ namespace {
 constexpr size_t STATIC_PARTIAL_FLOATS = size_t(2) << 20;
 static __device__ __align__(256) float g_decode_partials[STATIC_PARTIAL_FLOATS];
 
-constexpr int MAX_DEVICES = 64;
 std::mutex g_setup_mutex;
-float *g_partials_addr[MAX_DEVICES] = {};  // device address of the array, per device ordinal
+float *g_partials_addr[kr::MAX_DEVICES] = {};  // device address of the array, per device ordinal
 
 // In host code `g_decode_partials` is only a handle for the runtime, never a device address: the
 // address a kernel can use must be asked for, once per device, with that device current.
-int partials_address(float **out) {
-    int dev = -1;
-    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return KRAKEN_ECUDA;
+// The array belongs to the current device, so the tensors of the call must live there too: `q` is
+// looked up and a pointer into another device's memory is refused instead of being paired with
+// this device's array.
+int partials_address(const void *q, float **out) {
+    const int dev = kr::device_slot();
+    if (dev < 0) return KRAKEN_ECUDA;
+    cudaPointerAttributes attr;
+    if (cudaPointerGetAttributes(&attr, q) != cudaSuccess) {
+        cudaGetLastError();
+        return KRAKEN_EINVAL;
+    }
+    if (attr.type == cudaMemoryTypeDevice && attr.device != dev) return KRAKEN_EINVAL;
     std::lock_guard<std::mutex> lock(g_setup_mutex);
     if (!g_partials_addr[dev]) {
         void *p = nullptr;
@@ -44,13 +52,14 @@ extern "C" int kraken_op_decode_attention_static(const void *q, int64_t q_gstrid
                                                  int64_t out_gstride, void *stream) {
     using namespace kr;
     if (groups < 1 || batch < 1 || n_head < 1 || n_keys < 1) return KRAKEN_EINVAL;
-    if (head_dim != 64 && head_dim != 128) return KRAKEN_EUNSUPPORTED;
+    if (!q || !k_cache || !v_cache || !out) return KRAKEN_EINVAL;
+    if (!decode_head_dim_ok(head_dim)) return KRAKEN_EUNSUPPORTED;
     if (splits == 0) splits = decode_attention_splits(groups, batch, n_head, n_keys);
     if (splits < 1 || splits > DECODE_MAX_SPLITS) return KRAKEN_EINVAL;
     const size_t need = decode_attention_partial_bytes(groups, batch, n_head, head_dim, splits);
     if (splits > 1 && need > STATIC_PARTIAL_FLOATS * sizeof(float)) return KRAKEN_ECAPACITY;
     float *partials = nullptr;
-    int rc = partials_address(&partials);
+    int rc = partials_address(q, &partials);
     if (rc) return rc;
     DecodeAttnParams p;
     p.q = static_cast<const uint16_t *>(q);

@@ -475,8 +475,7 @@ int launch_layernorm(const float *a, long long a_gstride, const float *y, const 
     if (ysum && (y || ysum_groups < 1 || (ysum_gstride & 3))) return KRAKEN_EINVAL;
     int stages = 0;
     // the persistent kernel has bounded waits, so it needs a status word to report one that ran out
-    if (status && !ysum && !env_flag("KRAKEN_LN_WARP_ROWS") &&
-        layernorm_stream_fits(a, a_gstride, y, groups, rows, d, &stages)) {
+    if (status && !ysum && layernorm_stream_fits(a, a_gstride, y, groups, rows, d, &stages)) {
         const size_t smem = (size_t)stages * 4 * d * (groups + (y ? 1 : 0)) + (size_t)4 * groups * d;
         const int sms = sm_count() > 0 ? sm_count() : 148;
         const int n_consumers = layernorm_stream_consumers(groups, d);
@@ -486,13 +485,13 @@ int launch_layernorm(const float *a, long long a_gstride, const float *y, const 
                                           : layernorm_stream_kernel<16, LNS_CONSUMERS_WIDE>)
                              : (d <= 1024 ? layernorm_stream_kernel<8, LNS_CONSUMERS>
                                           : layernorm_stream_kernel<16, LNS_CONSUMERS>);
-        static bool configured[5] = {false, false, false, false, false};
+        static DeviceOnce configured[5];
         const int which = d > 2048 ? 4 : (wide ? 2 : 0) + (d <= 1024 ? 1 : 0);
-        if (!configured[which]) {
+        if (!configured[which].done()) {
             int rc = cuda_check(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                      LNS_SMEM_BUDGET), "layernorm: shared memory opt-in");
             if (rc) return rc;
-            configured[which] = true;
+            configured[which].set();
         }
         const cudaError_t ce = launch_pdl(kern, dim3(sms), dim3((n_consumers + 1) * 32), smem, stream, a, a_gstride, y, gamma,
                                           beta, groups, rows, d, eps, out, stages, n_consumers, status);
@@ -505,22 +504,24 @@ int launch_layernorm(const float *a, long long a_gstride, const float *y, const 
     // Measured, 4 groups, us per launch, warp per row / CTA per row: 128 tokens d 2496 9.0 / 4.0, d 3120 11.3 / 4.5,
     // d 7424 29.1 / 6.3; 512 tokens d 2496 16.0 / 11.2; 2048 tokens d 2496 48.2 / 45.5, d 3120 61.2 / 50.3,
     // d 4992 121.7 / 66.7, d 7424 216.8 / 90.7; 8 groups d 3648 130.5 / 100.1; but d 2048 31.3 / 38.5 and 8 groups
-    // d 1920 53.1 / 71.9.  KRAKEN_LN_BLOCK=0/1 forces the choice.
+    // d 1920 53.1 / 71.9.  KRAKEN_TUNE_LN_ROW_KERNEL = 1 / 2 forces the warp / the CTA per row.
     const int sms_b = sm_count() > 0 ? sm_count() : 148;
-    const char *force_b = getenv("KRAKEN_LN_BLOCK");
+    const int force_b = tuning(KRAKEN_TUNE_LN_ROW_KERNEL);
     const bool block_auto = d > 2048 || (d > 1024 && warps <= 24LL * sms_b);
-    const bool block_rows = !ysum && d <= 4 * LNB_THREADS * LNB_CACHE &&
-                            (force_b && (force_b[0] == '0' || force_b[0] == '1') ? force_b[0] == '1' : block_auto);
+    const bool block_rows = !ysum && d <= 4 * LNB_THREADS * LNB_CACHE && (force_b ? force_b == 2 : block_auto);
     if (block_rows) {
         // a grid of resident CTAs that walk the rows: no second wave with a ragged tail
-        static int per_sm = 0;
+        static std::atomic<int> per_sm_of[MAX_DEVICES];
+        const int dev = device_slot();
+        if (dev < 0) return KRAKEN_ECUDA;
+        int per_sm = per_sm_of[dev].load();
         if (per_sm == 0) {
             int n = 0;
             if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, layernorm_block_kernel, LNB_THREADS, 0) != cudaSuccess || n < 1) {
                 cudaGetLastError();
                 n = 4;
             }
-            per_sm = n;
+            per_sm_of[dev].store(per_sm = n);
         }
         const long long resident = (long long)per_sm * sms_b;
         const long long ctas = warps < resident ? warps : resident;

@@ -457,9 +457,11 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 
 int launch_pair(const CUtensorMap &tmA, const CUtensorMap &tmB, const KernelArgs &ka, cudaStream_t stream) {
     using Cfg = PairCfg;
-    static bool configured = false;
-    static int max_clusters = 0;
-    if (!configured) {
+    static DeviceOnce configured;
+    static std::atomic<int> max_clusters_of[MAX_DEVICES];
+    const int dev = device_slot();
+    if (dev < 0) return KRAKEN_ECUDA;
+    if (!configured.done()) {
         int rc = cuda_check(cudaFuncSetAttribute(gemm_tc_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                  Cfg::SMEM_BYTES), "gemm pair: shared memory opt-in");
         if (rc) return rc;
@@ -479,9 +481,10 @@ int launch_pair(const CUtensorMap &tmA, const CUtensorMap &tmB, const KernelArgs
             cudaGetLastError();
             n = (sm_count() > 0 ? sm_count() : 148) / 2;
         }
-        max_clusters = n;
-        configured = true;
+        max_clusters_of[dev].store(n);
+        configured.set();
     }
+    const int max_clusters = max_clusters_of[dev].load();
     const long long tiles = (long long)((ka.shape.m + 2 * BM - 1) / (2 * BM)) * ka.tiles_n;
     const long long units = ka.group_serial ? tiles : tiles * ka.shape.groups;
     const int clusters = static_cast<int>(units < max_clusters ? units : max_clusters);
@@ -492,12 +495,12 @@ int launch_pair(const CUtensorMap &tmA, const CUtensorMap &tmB, const KernelArgs
 template <int BN>
 int launch_bn(const CUtensorMap &tmA, const CUtensorMap &tmB, const KernelArgs &ka, int grid, cudaStream_t stream) {
     using Cfg = TileCfg<BN>;
-    static bool configured = false;
-    if (!configured) {
+    static DeviceOnce configured;
+    if (!configured.done()) {
         int rc = cuda_check(cudaFuncSetAttribute(gemm_tc_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                  Cfg::SMEM_BYTES), "gemm: shared memory opt-in");
         if (rc) return rc;
-        configured = true;
+        configured.set();
     }
     return cuda_check(launch_pdl(gemm_tc_kernel<BN>, dim3(grid), dim3(NUM_THREADS), Cfg::SMEM_BYTES, stream, tmA, tmB, ka),
                       "gemm: launch");
@@ -508,7 +511,7 @@ int launch_bn(const CUtensorMap &tmA, const CUtensorMap &tmB, const KernelArgs &
 int gemm_pick_bn(const GemmShape &s) {
     const int sms = sm_count() > 0 ? sm_count() : 148;
     const long long tiles_m = (s.m + BM - 1) / BM;
-    const bool pairs_ok = !env_flag("KRAKEN_GEMM_NO_PAIR");
+    const bool pairs_ok = true;
     // CTA pairs on 256 x 256 tiles when that gives every pair of SMs about two work items
     const long long pair_items = ((s.m + 2 * BM - 1) / (2 * BM)) * ((s.n_out + BN2 - 1) / BN2) * s.groups;
     if (pair_items >= sms && pairs_ok) return GEMM_TILE_PAIR;

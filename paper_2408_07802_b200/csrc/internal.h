@@ -4,6 +4,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "../../include/kraken.h"
 
 namespace kr {
@@ -46,7 +48,20 @@ int encode_tma_3d_bf16(CUtensorMap *map, const void *base, uint64_t dim0, uint64
 int encode_tma_4d_bf16(CUtensorMap *map, const void *base, const uint64_t dims[4], const uint64_t strides_elems[3],
                        const uint32_t box[4]);
 
-int sm_count();
+// Launch set-up (shared-memory opt-ins, occupancy queries, the SM count) belongs to a device, not to the
+// process: a host may drive several GPUs.  State is kept per device ordinal of the current device.
+constexpr int MAX_DEVICES = 64;
+int device_slot();   // ordinal of the current device, -1 if it cannot be had or is out of range
+struct DeviceOnce {  // zero-initialised static: "this set-up has been done on the current device"
+    std::atomic<unsigned char> flag[MAX_DEVICES];
+    bool done() const;
+    void set();
+};
+int sm_count();      // of the current device; 0 on failure
+
+// Process-wide kernel choices for tests and measurements (kraken_tuning_set); 0 = the library's own choice.
+int tuning(int key);
+int set_tuning(int key, int value);
 
 // Tensor-core grouped GEMM.  tmA / tmB may be NULL: they are then encoded from the operands.
 // b_g0: index of the first group along the outermost dimension of a caller-made tmB (a map
@@ -71,9 +86,6 @@ int gemm_encode_b(CUtensorMap *map, const GemmOperands &op, const GemmShape &sha
 // Weight-streaming GEMM for M <= 32 rows (decode, last-position tail); every epilogue except RESID_SUM.
 int launch_gemm_skinny(const GemmOperands &op, const GemmShape &shape, const EpiParams &epi, cudaStream_t stream);
 constexpr int SKINNY_MAX_ROWS = 32;
-
-// One thread per output element; for bring-up comparisons only (KRAKEN_NAIVE=1).
-int launch_gemm_naive(const GemmOperands &op, const GemmShape &shape, const EpiParams &epi, cudaStream_t stream);
 
 int launch_embed(const int32_t *ids, int n_tokens, int seqlen, int pos0, const uint16_t *wte, const uint16_t *wpe,
                  int d, int vocab, float *out, uint32_t *status, cudaStream_t stream, const int *pos0_dev = nullptr,
@@ -102,8 +114,6 @@ struct AttnParams {
     long long out_gstride;
     int n_kv_head = 0;  // key/value heads in the cache (0 = n_head); query head h reads head h / (n_head / n_kv_head)
 };
-int launch_attention_prefill(const AttnParams &p, cudaStream_t stream);
-int launch_attention_naive(const AttnParams &p, cudaStream_t stream);
 // tcgen05 / TMEM attention for tiles of 128 queries x 128 keys; tensor maps may be NULL (encoded per call).
 bool attention_tc_supported(const AttnParams &p);
 int attention_tc_encode(const AttnParams &p, CUtensorMap *tmQ, CUtensorMap *tmK, CUtensorMap *tmV);
@@ -125,6 +135,7 @@ struct DecodeAttnParams {
     uint16_t *out;    // [G][batch, d]
     long long out_gstride;
 };
+inline bool decode_head_dim_ok(int hd) { return hd == 64 || hd == 72 || hd == 96 || hd == 104 || hd == 128; }
 int decode_attention_splits(int groups, int batch, int n_head, int n_keys);
 // whether the query heads of a key/value head are served together by the tensor-core tile kernel (then the
 // number of CTA streams, which the split count should be chosen for, is the number of key/value heads)

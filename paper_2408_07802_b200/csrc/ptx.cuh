@@ -75,7 +75,8 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
 // Wait for the given phase parity.  Returns false when the wait limit ran out or another
 // thread of the CTA already gave up (abort_flag, in shared memory, is then set): the caller
 // must leave its loop and fall through to the common teardown.
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile uint32_t *abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile uint32_t *abort_flag,
+                                          unsigned long long limit_ns = WAIT_LIMIT_NS) {
     if (mbar_try_wait(bar, parity)) return true;
     unsigned long long t0 = 0;
     uint32_t polls = 0;
@@ -84,7 +85,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volati
             if (*abort_flag) return false;
             unsigned long long now = global_timer_ns();
             if (t0 == 0) t0 = now;
-            else if (now - t0 > WAIT_LIMIT_NS) {
+            else if (now - t0 > limit_ns) {
                 *abort_flag = 1u;
                 return false;
             }

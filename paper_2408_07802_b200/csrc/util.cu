@@ -3,6 +3,7 @@
 #include <stdlib.h>
 #include <string.h>
 
+#include <atomic>
 #include <mutex>
 
 #include "internal.h"
@@ -65,17 +66,44 @@ int encode_tma_4d_bf16(CUtensorMap *map, const void *base, const uint64_t dims[4
     return encode(map, base, 4, dims, strides_elems, box);
 }
 
+int device_slot() {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) return -1;
+    return dev;
+}
+
+bool DeviceOnce::done() const {
+    const int dev = device_slot();
+    return dev >= 0 && flag[dev].load(std::memory_order_acquire) != 0;
+}
+
+void DeviceOnce::set() {
+    const int dev = device_slot();
+    if (dev >= 0) flag[dev].store(1, std::memory_order_release);
+}
+
 int sm_count() {
-    static int n = -1;
-    if (n < 0) {
-        int dev = 0, v = 0;
-        if (cudaGetDevice(&dev) == cudaSuccess &&
-            cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) == cudaSuccess)
-            n = v;
-        else
-            return 0;
+    static std::atomic<int> n[MAX_DEVICES];
+    const int dev = device_slot();
+    if (dev < 0) return 0;
+    int v = n[dev].load(std::memory_order_relaxed);
+    if (v <= 0) {
+        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return 0;
+        n[dev].store(v, std::memory_order_relaxed);
     }
-    return n;
+    return v;
+}
+
+namespace {
+std::atomic<int> g_tuning[KRAKEN_TUNE_COUNT];
+}
+
+int tuning(int key) { return key >= 0 && key < KRAKEN_TUNE_COUNT ? g_tuning[key].load(std::memory_order_relaxed) : 0; }
+
+int set_tuning(int key, int value) {
+    if (key < 0 || key >= KRAKEN_TUNE_COUNT || value < 0 || value > 2) return KRAKEN_EINVAL;
+    g_tuning[key].store(value, std::memory_order_relaxed);
+    return KRAKEN_OK;
 }
 
 static thread_local char g_last_error[256] = "";

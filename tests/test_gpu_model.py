@@ -138,21 +138,6 @@ def test_ragged_lengths_and_batches():
             assert rel <= REL_L2_MAX and mx <= MAX_ABS_MAX, (seqlen, b, rel, mx)
 
 
-def test_naive_kernels_agree_with_tensor_core_path():
-    s = ki.CONFIGS["C0"]
-    tok = ki.uniform_tokens(1, s.vocab, 1, 100, DEV)
-    m, _ = build(s)
-    fast = m.prefill_all_logits(tok).cpu().numpy()
-    os.environ["KRAKEN_NAIVE"] = "1"
-    try:
-        m2, _ = build(s)
-        slow = m2.prefill_all_logits(tok).cpu().numpy()
-    finally:
-        del os.environ["KRAKEN_NAIVE"]
-    rel, mx = logits_metrics(fast[0], slow[0])
-    assert rel < 5e-3 and mx < 3e-2, (rel, mx)
-
-
 def test_prefill_host_matches_device_call():
     s = ki.CONFIGS["C0"]
     m, _ = build(s)
@@ -264,6 +249,40 @@ def test_decode_branch_chains_any_branch_count(n_branch, one_chain, monkeypatch)
             again = m2.decode_step(tok[:, t].contiguous()).cpu().numpy()
             assert np.array_equal(again, outs[i]), (n_branch, t)
         m2.close()
+    m.close()
+
+
+def test_decode_branch_chains_with_more_rows_than_the_weight_streaming_gemm_takes(monkeypatch):
+    """A decode batch above 32 rows leaves the weight-streaming GEMM for the tensor-core tile kernel, launched
+    once per branch chain on that branch's slice of the activations: every branch must read its own rows
+    (teacher-forced steps against the oracle on sampled sequences), and the chains give the same bits as the
+    single chain, whose launches cover all branches at once."""
+    s = ki.KrakenShape("chains3x40", 3, 2, 128, 2, 256, 512, 48, 40, 9)
+    steps = 3
+    m, w = build(s)
+    wb = host_bits(w)
+    tok = ki.uniform_tokens(23, s.vocab, s.batch, s.seqlen + steps, DEV)
+    m.prefill(tok[:, :s.seqlen].contiguous())
+    pick = [0, 17, 33, 39]
+    orcs = {b: oracle.Oracle(s, wb, bf16_store=False) for b in pick}
+    for b in pick:
+        orcs[b].prefill(tok[b, :s.seqlen].cpu().numpy())
+    outs = []
+    for t in range(s.seqlen, s.seqlen + steps):
+        got = m.decode_step(tok[:, t].contiguous()).cpu().numpy()
+        outs.append(got)
+        for b in pick:
+            ref = orcs[b].decode_step(int(tok[b, t]))
+            rel, mx = logits_metrics(got[b], ref)
+            assert rel <= REL_L2_MAX and mx <= MAX_ABS_MAX, (t, b, rel, mx)
+    assert m.device_status() == 0
+    monkeypatch.setenv("KRAKEN_DECODE_ONE_CHAIN", "1")
+    m2, _ = build(s)
+    m2.prefill(tok[:, :s.seqlen].contiguous())
+    for i, t in enumerate(range(s.seqlen, s.seqlen + steps)):
+        again = m2.decode_step(tok[:, t].contiguous()).cpu().numpy()
+        assert np.array_equal(again, outs[i]), t
+    m2.close()
     m.close()
 
 

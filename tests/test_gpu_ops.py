@@ -72,7 +72,7 @@ def test_layernorm(d, with_y):
 @pytest.mark.parametrize("G,d,with_y", [(4, 2048, True), (4, 2048, False), (2, 768, True), (1, 1000, False),
                                         (3, 512, True), (8, 512, True), (8, 1920, True), (5, 768, True), (16, 256, False),
                                         (4, 2496, True), (4, 3120, False), (2, 4096, True)])
-def test_layernorm_many_rows_persistent_kernel(G, d, with_y, monkeypatch):
+def test_layernorm_many_rows_persistent_kernel(G, d, with_y):
     """With a status word and many rows the persistent ring kernel runs: sampled rows against the oracle,
     every row bit-equal to the warp-per-row kernel (same operations in the same order); ragged row count."""
     rows = 8 * torch.cuda.get_device_properties(0).multi_processor_count + 37
@@ -84,8 +84,8 @@ def test_layernorm_many_rows_persistent_kernel(G, d, with_y, monkeypatch):
     out = kr.op_layernorm(a, y, gamma, beta, status=status)
     torch.cuda.synchronize()
     assert int(status.item()) == 0
-    monkeypatch.setenv("KRAKEN_LN_BLOCK", "0")       # the warp-per-row kernel, not one CTA per row
-    plain = kr.op_layernorm(a, y, gamma, beta)
+    with kr.tuning(kr.TUNE_LN_ROW_KERNEL, 1):          # the warp-per-row kernel, not one CTA per row
+        plain = kr.op_layernorm(a, y, gamma, beta)
     assert torch.equal(out.view(torch.int16), plain.view(torch.int16))
     pick = [0, 1, rows // 2, rows - 38, rows - 1]
     for g in (0, G - 1):
@@ -95,12 +95,20 @@ def test_layernorm_many_rows_persistent_kernel(G, d, with_y, monkeypatch):
         assert ok, (g, worst)
 
 
-@pytest.mark.parametrize("force", ["0", "1"])
-def test_layernorm_one_cta_per_row_walks_many_rows(force, monkeypatch):
+@pytest.fixture(autouse=True)
+def _library_choices_restored():
+    """Every test starts and ends with the library's own kernel choices."""
+    yield
+    for key in (kr.TUNE_LN_ROW_KERNEL, kr.TUNE_ATTN_SCHEDULE):
+        kr.set_tuning(key, 0)
+
+
+@pytest.mark.parametrize("force", [1, 2])
+def test_layernorm_one_cta_per_row_walks_many_rows(force):
     """Rows wider than 4096 take the one-CTA-per-row kernel, whose grid is smaller than the number of rows here, so
     every CTA walks several rows; the same call forced onto the warp-per-row kernel agrees within one bf16 step
     (the two sum in different orders)."""
-    monkeypatch.setenv("KRAKEN_LN_BLOCK", force)
+    kr.set_tuning(kr.TUNE_LN_ROW_KERNEL, force)      # 1: one warp per row, 2: one CTA per row
     G, d = 2, 4992
     rows = 5 * torch.cuda.get_device_properties(0).multi_processor_count + 3
     a = (ki.normal_bf16(5, 0, (G, rows, d), 1.0, DEV).float() * 0.9 + 0.1).contiguous()
@@ -270,14 +278,9 @@ def test_gemm_rejects_unaligned():
 
 # ------------------------------------------------------------------ attention
 
-@pytest.mark.parametrize("kernel", ["tcgen05", "warp_mma"])
 @pytest.mark.parametrize("hd", [64, 128, 72, 96, 104])
 @pytest.mark.parametrize("seqlen,pos0", [(200, 0), (100, 37), (1, 90), (64, 0), (300, 0), (129, 127)])
-def test_attention_matches_oracle(hd, seqlen, pos0, kernel, monkeypatch):
-    if kernel == "warp_mma":
-        if hd not in (64, 128):
-            pytest.skip("the warp-MMA kernel covers head dims 64 and 128 only")
-        monkeypatch.setenv("KRAKEN_ATTN_WARP_MMA", "1")   # the m16n8k16 kernel kept for odd cache strides
+def test_attention_matches_oracle(hd, seqlen, pos0):
     G, B, H, P = 2, 2, 2, 512
     d = H * hd
     q = ki.normal_bf16(7, 0, (G, B * seqlen, d), 1.0, DEV)
@@ -303,11 +306,49 @@ def test_attention_matches_oracle(hd, seqlen, pos0, kernel, monkeypatch):
     assert np.sqrt(num / den) < 6e-3, np.sqrt(num / den)
 
 
+def test_attention_refuses_a_cache_with_gaps():
+    """One kernel serves prefill attention; a cache whose sequences are further apart than heads x max_pos x
+    head_dim (a view into a larger buffer) is refused with EUNSUPPORTED, not handed to a second kernel."""
+    G, B, H, P, hd, seqlen = 1, 2, 2, 128, 64, 40
+    q = ki.normal_bf16(9, 0, (G, B * seqlen, H * hd), 1.0, DEV)
+    big = ki.normal_bf16(9, 1, (G, B, H + 1, P, hd), 1.0, DEV)
+    kc = big[:, :, :H]                                       # sequences H + 1 heads apart
+    with pytest.raises(kr.KrakenError) as e:
+        kr.op_attention(q, kc, kc, B, seqlen, 0, H)
+    assert e.value.status == kr.EUNSUPPORTED
+
+
+def test_bounded_wait_runs_out_and_the_context_stays_usable():
+    """Every device-side wait of the library has a limit; when it runs out the kernel leaves its loop, raises
+    bit 1 of the status word and returns.  The probe waits, with that same routine, on a barrier that nothing
+    signals: the status bit must appear, the kernel must return (no hang, no fault), and ordinary work on the
+    same context afterwards must be correct."""
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    t0 = torch.cuda.Event(enable_timing=True)
+    t1 = torch.cuda.Event(enable_timing=True)
+    t0.record()
+    kr.test_wait_limit(status, 3000)                         # 3 ms
+    t1.record()
+    torch.cuda.synchronize()
+    assert int(status.item()) == kr.STATUS_WAIT_LIMIT
+    ms = t0.elapsed_time(t1)
+    assert 2.0 <= ms <= 500.0, ms                            # it really waited, and it really stopped
+    with pytest.raises(kr.KrakenError):
+        kr.test_wait_limit(status, 0)
+    # the context is intact: a LayerNorm launch right after gives the oracle's result
+    a = ki.normal_bf16(31, 0, (1, 64, 256), 1.0, DEV).float().contiguous()
+    gamma = (1 + ki.normal_bf16(31, 1, (1, 256), 0.3, DEV).float()).to(torch.bfloat16)
+    out = kr.op_layernorm(a, None, gamma, None)
+    ref = oracle.layernorm(a[0].cpu().numpy(), None, bits(gamma[0]), None)
+    ok, worst = bf16_ulp_close(out[0].float().cpu().numpy(), ref, ulps=1.0, atol=1e-5)
+    assert ok, worst
+
+
 @pytest.mark.parametrize("G,B,H,hd,seqlen", [(4, 1, 16, 64, 768),     # one round of couples, a middle pair alone
                                               (4, 1, 16, 64, 1024),    # one round, every pair has a partner
                                               (4, 2, 16, 64, 1300),    # several rounds, ragged last tile
                                               (3, 2, 12, 128, 520)])   # fewer couples than SMs, ragged
-def test_attention_fixed_work_lists_match_one_cta_per_item(G, B, H, hd, seqlen, monkeypatch):
+def test_attention_fixed_work_lists_match_one_cta_per_item(G, B, H, hd, seqlen):
     """With more work items than SMs the kernel walks per-CTA lists of couples of items; each item's arithmetic
     is the same as with one CTA per item, so the outputs are equal bit for bit, and sampled heads match the
     oracle."""
@@ -316,8 +357,8 @@ def test_attention_fixed_work_lists_match_one_cta_per_item(G, B, H, hd, seqlen, 
     kc = ki.normal_bf16(17, 1, (G, B, H, seqlen, hd), 1.0, DEV)
     vc = ki.normal_bf16(17, 2, (G, B, H, seqlen, hd), 1.0, DEV)
     got = kr.op_attention(q, kc, vc, B, seqlen, 0, H)
-    monkeypatch.setenv("KRAKEN_ATTN_ONE_CTA_PER_ITEM", "1")
-    plain = kr.op_attention(q, kc, vc, B, seqlen, 0, H)
+    with kr.tuning(kr.TUNE_ATTN_SCHEDULE, 1):
+        plain = kr.op_attention(q, kc, vc, B, seqlen, 0, H)
     torch.cuda.synchronize()
     assert torch.equal(got, plain)
     out = got.float().cpu().numpy()

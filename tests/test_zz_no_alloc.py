@@ -4,12 +4,12 @@ Runs last in the suite (file name) so that a failure here cannot hide another te
 passes on its own in a fresh process, where its first call is the one that looks up the address of
 the library's built-in partials array.
 """
-import ctypes as C
-
+import numpy as np
 import pytest
 import torch
 
 import kraken_inputs as ki
+import oracle
 import paper_2408_07802_b200 as kr
 
 pytestmark = pytest.mark.gpu
@@ -24,22 +24,48 @@ def _inputs(G, B, H, hd, P, seed):
 
 
 def test_static_scratch_matches_caller_scratch_twice_in_a_row():
-    """Two back-to-back calls with different shapes share the built-in array; each must equal the
+    """Back-to-back calls with different shapes share the built-in array; each must equal the
     existing entry point run on the same inputs (same kernels, same split count: bit for bit, which is
-    inside the 2e-2 absolute bound the attention tests use against the oracle)."""
-    cases = [(2, 3, 2, 64, 600, 577, 5, 21), (1, 2, 4, 128, 300, 300, 3, 22)]
-    for G, B, H, hd, P, n_keys, splits, seed in cases:
+    inside the 2e-2 absolute bound the attention tests use against the oracle), and sampled heads must
+    match the oracle's attention over the same cache rows.  From the second call on (the first one may
+    look up the array's address) the device's free memory and torch's allocation count do not move."""
+    cases = [(2, 3, 2, 64, 600, 577, 5, 21), (1, 2, 4, 128, 300, 300, 3, 22), (2, 2, 2, 96, 200, 150, 2, 23)]
+    for i, (G, B, H, hd, P, n_keys, splits, seed) in enumerate(cases):
         q, kc, vc = _inputs(G, B, H, hd, P, seed)
         out = torch.empty_like(q)           # inputs and output stay the caller's
+        torch.cuda.synchronize()
+        free0, used0 = torch.cuda.mem_get_info()[0], torch.cuda.memory_allocated()
         rc = kr.lib().kraken_op_decode_attention_static(
             q.data_ptr(), q.stride(0), kc.data_ptr(), vc.data_ptr(), kc.stride(0), kc.stride(1), G, B, n_keys, H,
             hd, P, splits, out.data_ptr(), out.stride(0), torch.cuda.current_stream().cuda_stream)
         assert rc == kr.OK, kr.strerror(rc)
+        torch.cuda.synchronize()
+        if i > 0:
+            assert torch.cuda.mem_get_info()[0] >= free0 and torch.cuda.memory_allocated() == used0
         ref = kr.op_decode_attention(q, kc, vc, n_keys, splits)
         torch.cuda.synchronize()
         assert torch.isfinite(out.float()).all()
         assert (out.float() - ref.float()).abs().max().item() <= 2e-2
         assert torch.equal(out, ref)
+        qn, kn, vn, on = (t.float().cpu().numpy() for t in (q, kc, vc, out))
+        for g, b, h in [(0, 0, 0), (G - 1, B - 1, H - 1)]:
+            want = oracle.attention_head(qn[g, b:b + 1, h * hd:(h + 1) * hd], kn[g, b, h, :n_keys], vn[g, b, h, :n_keys],
+                                         q_pos0=n_keys - 1)
+            assert np.abs(on[g, b, h * hd:(h + 1) * hd] - want[0]).max() <= 2e-2, (i, g, b, h)
+
+
+def test_static_scratch_has_no_grouped_query_form():
+    """The call takes no key/value head count: the binding refuses a cache with fewer heads than d / head_dim
+    instead of reading it with the wrong head layout, and head dims outside the supported set are an error."""
+    q = torch.zeros(1, 2, 4 * 64, dtype=torch.bfloat16, device=DEV)
+    kc = torch.zeros(1, 2, 2, 32, 64, dtype=torch.bfloat16, device=DEV)      # 2 key/value heads for 4 query heads
+    with pytest.raises(ValueError):
+        kr.op_decode_attention_static(q, kc, kc, 16)
+    q = torch.zeros(1, 2, 2 * 80, dtype=torch.bfloat16, device=DEV)
+    kc = torch.zeros(1, 2, 2, 32, 80, dtype=torch.bfloat16, device=DEV)
+    with pytest.raises(kr.KrakenError) as e:
+        kr.op_decode_attention_static(q, kc, kc, 16)
+    assert e.value.status == kr.EUNSUPPORTED
 
 
 def test_static_scratch_rejects_what_does_not_fit():
