@@ -402,7 +402,11 @@ static int forward(ko_state *s, const int32_t *ids, int n, int pos0, float *logi
             float *cat = (float *)malloc(sizeof(float) * (size_t)nr * N * d);
             float *z = (float *)malloc(sizeof(float) * (size_t)nr * d);
             float *zf = (float *)malloc(sizeof(float) * (size_t)nr * d);
-            if (!cat || !z || !zf) { free(cat); free(z); free(zf); return -4; }
+            if (!cat || !z || !zf) {
+                free(cat); free(z); free(zf);
+                free(x0); free(x); free(xn); free(y); free(u); free(qkv); free(o); free(a); free(hh); free(g); free(tmp);
+                return -4;
+            }
             for (int t = 0; t < nr; ++t)
                 for (int b = 0; b < N; ++b)
                     for (int j = 0; j < d; ++j) {

@@ -607,3 +607,92 @@ def test_parallel_attention_feedforward_variant_is_a_gptj_style_stack():
     seq, _ = oracle.Oracle(small_shape(n_branch=1, n_layer=3, no_combine=1), wbits(w)).prefill(ids)
     assert np.max(np.abs(seq - ref)) > 1e-3
 
+
+
+# ------------------------------------------------------------------ the store points of the rounding mode
+
+STORE_POINTS = ("ln1", "qkv", "o", "ln2", "gelu", "concat_in", "zf")
+
+
+def forward_with_explicit_rounding(shape, w, ids, half, final_ln, skip=None):
+    """Algorithm 1 plus the tail, assembled from the individually pinned step functions, with a round-to-16-bit
+    written out after each store point of a "16-bit activations, fp32 accumulate" implementation: the two
+    LayerNorm outputs, q | k | v (hence the cache), the attention output, the GELU output, the rows that
+    W_concat reads and the rows that the unembedding reads.  The residual stream (x0, a, x_n, y) is never
+    rounded.  The rounding itself is numpy's / torch's conversion, not the oracle's.  `skip` leaves one
+    store point unrounded (the negative controls)."""
+    def rnd(name, x):
+        if name == skip:
+            return x
+        x = np.ascontiguousarray(x, dtype=np.float32)
+        if half:
+            return x.astype(np.float16).astype(np.float32)
+        return torch.from_numpy(x).to(torch.bfloat16).float().numpy()
+
+    N, L, d, H = shape.n_branch, shape.n_layer, shape.d_model, shape.n_head
+    hd = d // H
+    n = len(ids)
+    x0 = (w["wte"].float()[torch.as_tensor(ids, dtype=torch.long)] + w["wpe"].float()[:n]).numpy()
+    x = [x0.copy() for _ in range(N)]
+    layer_out = np.zeros((L, N, n, d), dtype=np.float32)
+    caches = {}
+    for l in range(L):
+        y = x0 if l == 0 else np.sum(np.stack(x).astype(np.float64), axis=0).astype(np.float32)
+        nxt = []
+        for b in range(N):
+            g = lambda k: bits(w[k][l, b])
+            u = rnd("ln1", oracle.layernorm(x[b], None, g("ln1_g"), g("ln1_b"), half=half))
+            qkv = rnd("qkv", oracle.linear(u, g("w_qkv"), g("b_qkv"), half=half))
+            caches[(l, b, 0)] = qkv[:, d:2 * d].reshape(n, H, hd).transpose(1, 0, 2)
+            caches[(l, b, 1)] = qkv[:, 2 * d:].reshape(n, H, hd).transpose(1, 0, 2)
+            o = np.zeros((n, d), dtype=np.float32)
+            for h in range(H):
+                sl = slice(h * hd, (h + 1) * hd)
+                o[:, sl] = oracle.attention_head(qkv[:, sl], qkv[:, d:2 * d][:, sl], qkv[:, 2 * d:][:, sl])
+            o = rnd("o", o)
+            a = x[b] + oracle.linear(o, g("w_proj"), g("b_proj"), half=half)
+            hh = rnd("ln2", oracle.layernorm(a, y, g("ln2_g"), g("ln2_b"), half=half))
+            up = oracle.linear(hh, g("w_up"), g("b_up"), half=half)
+            gl = rnd("gelu", np.vectorize(lambda t: oracle.gelu(float(t)))(up).astype(np.float32))
+            out = a + oracle.linear(gl, g("w_down"), g("b_down"), half=half)
+            layer_out[l, b] = out
+            nxt.append(out)
+        x = nxt
+    cat = rnd("concat_in", np.concatenate(x, axis=1))                        # branch-major
+    z = oracle.linear(cat, bits(w["w_concat"]), bits(w["b_concat"]), half=half)
+    if final_ln:
+        zf = rnd("zf", oracle.layernorm(z, None, bits(w["lnf_g"]), bits(w["lnf_b"]), half=half))
+    else:
+        zf = rnd("zf", z)
+    logits = oracle.linear(zf, bits(w["wte"]), None, half=half)
+    return logits, layer_out, caches
+
+
+@pytest.mark.parametrize("half", [False, True])
+@pytest.mark.parametrize("final_ln", [True, False])
+def test_rounding_mode_rounds_exactly_at_the_store_points(half, final_ln):
+    """The mode that decides the arg-max criterion and the cache comparison: its sub-layer outputs, cache rows
+    and logits equal, bit for bit, the composition above with every rounding written out; leaving any single
+    rounding out gives different logits, so none of the store points is missing from (or extra in) the oracle."""
+    shape = small_shape(n_branch=2, n_layer=2, seqlen=10)
+    w = rand_weights(shape)
+    if half:
+        w = {k: (None if v is None else v.to(torch.float16)) for k, v in w.items()}
+    ids = ki.uniform_tokens(13, shape.vocab, 1, shape.seqlen)[0].numpy()
+    orc = oracle.Oracle(shape, wbits(w), bf16_store=True, half=half, final_ln=final_ln)
+    got, lo = orc.prefill(ids, want_layer_out=True)
+    want, want_lo, want_cache = forward_with_explicit_rounding(shape, w, ids, half, final_ln)
+    assert np.array_equal(lo, want_lo)
+    for (l, b, which), rows in want_cache.items():
+        assert np.array_equal(orc.cache(l, b, which), rows), (l, b, which)
+    assert np.array_equal(got, want)
+    # the unrounded mode is a different function at every one of these outputs
+    plain, plain_lo = oracle.Oracle(shape, wbits(w), half=half, final_ln=final_ln).prefill(ids, want_layer_out=True)
+    assert not np.array_equal(plain, got) and not np.array_equal(plain_lo, lo)
+    for point in STORE_POINTS:
+        other, other_lo, _ = forward_with_explicit_rounding(shape, w, ids, half, final_ln, skip=point)
+        assert not np.array_equal(other, got), point
+        if point in ("concat_in", "zf"):
+            assert np.array_equal(other_lo, lo), point           # the tail's roundings do not touch the layers
+        else:
+            assert not np.array_equal(other_lo, lo), point
