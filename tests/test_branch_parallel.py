@@ -3,7 +3,8 @@
 CPU: the ordering of pieces and collectives in `BranchParallelPrefill`, run as two gloo ranks whose "engine"
 is built from the oracle's single steps, against the oracle's whole-model forward pass.
 GPU: the library's stage calls, with several ranks standing in one process on one GPU and driven in lockstep
-(no kernel ever waits for another rank), against the ordinary single-GPU prefill of the same model.
+(no kernel ever waits for another rank), against the ordinary single-GPU prefill of the same model and against
+the oracle's logits.
 """
 import os
 import socket
@@ -146,6 +147,17 @@ def test_stage_calls_in_lockstep_equal_the_single_gpu_prefill(name, split):
     for o in outs:
         err = (o - ref).abs().max().item()
         assert err <= 2e-3 * max(1.0, ref.abs().max().item()), err
+    # and against the oracle's whole-model forward pass, within the bounds stated for the logits
+    wb = {k: bits(v) for k, v in w.items()}
+    orcs = []
+    for b in range(s.batch):
+        orc = oracle.Oracle(s, wb)
+        want, _ = orc.prefill(tok[b].cpu().numpy(), logits_from=l0 - 1)
+        orcs.append(orc)
+        for o in outs:
+            got = o[b].float().cpu().numpy()
+            assert np.linalg.norm(got - want[0]) / np.linalg.norm(want[0]) <= 1e-2
+            assert np.abs(got - want[0]).max() <= 5e-2
     # every rank's cache holds exactly its branches' rows of the whole model's cache
     for (first, count), e in zip(split, engines):
         assert e.cur_len == l0 and e.device_status() == 0
@@ -162,6 +174,11 @@ def test_stage_calls_in_lockstep_equal_the_single_gpu_prefill(name, split):
         for o in outs:
             err = (o - want).abs().max().item()
             assert err <= 2e-3 * max(1.0, want.abs().max().item()), (step, err)
+        for b in range(s.batch):
+            truth = orcs[b].decode_step(int(nxt[b]))
+            got = outs[0][b].float().cpu().numpy()
+            assert np.linalg.norm(got - truth) / np.linalg.norm(truth) <= 1e-2, (step, b)
+            assert np.abs(got - truth).max() <= 5e-2, (step, b)
     assert all(e.cur_len == l0 + 2 for e in engines)
     # out-of-order calls are refused
     with pytest.raises(kr.KrakenError) as ex:

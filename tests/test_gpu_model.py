@@ -51,11 +51,20 @@ def argmax_agreement(got, ref):
     return same.mean(), (same | tie).mean()
 
 
+def record(line):
+    """Parity figures go to stdout (pytest -s) and, when KRAKEN_PARITY_LOG names a file, are appended there."""
+    print(line)
+    path = os.environ.get("KRAKEN_PARITY_LOG")
+    if path:
+        with open(path, "a") as f:
+            f.write(line + "\n")
+
+
 def check_parity(got, ref32, refbf, what):
     assert not np.isnan(got).any(), what
     rel, mx = logits_metrics(got, ref32)
     raw, adj = argmax_agreement(got, refbf)
-    print(f"[parity] {what}: relL2={rel:.3e} maxabs={mx:.3e} argmax raw={raw:.4f} tie-adjusted={adj:.4f}")
+    record(f"[parity] {what}: rows={len(got)} relL2={rel:.3e} maxabs={mx:.3e} argmax raw={raw:.4f} tie-adjusted={adj:.4f}")
     assert rel <= REL_L2_MAX, (what, rel)
     assert mx <= MAX_ABS_MAX, (what, mx)
     assert adj >= ARGMAX_MIN, (what, raw, adj)
@@ -572,12 +581,63 @@ def test_engine_shape_1p3b_4way_full_size_prefix_parity():
     prefix_parity("K1.3B-4", 40, [0])
 
 
-def test_c2_full_size_prefix_parity():
-    prefix_parity("C2", 128, [0])
+def test_c2_full_parity():
+    """C2 as the benchmark runs it (one sequence of 1024 tokens): every position against both oracle modes."""
+    s = ki.CONFIGS["C2"]
+    m, w = build(s)
+    wb = host_bits(w)
+    tok = ki.uniform_tokens(1, s.vocab, s.batch, s.seqlen, DEV)
+    last = m.prefill(tok).cpu().numpy()
+    assert m.device_status() == 0
+    got = m.logits_rows(list(range(s.seqlen))).cpu().numpy()
+    ref32, _ = oracle_all_logits(s, wb, tok[0].cpu().numpy(), False)
+    refbf, orc = oracle_all_logits(s, wb, tok[0].cpu().numpy(), True)
+    check_parity(got, ref32, refbf, "C2 all positions")
+    rel, mx = logits_metrics(last[0], ref32[-1])
+    record(f"[parity] C2 last position of the timed call: relL2={rel:.3e} maxabs={mx:.3e}")
+    assert rel <= REL_L2_MAX and mx <= MAX_ABS_MAX
+    for layer in (0, s.n_layer // 2, s.n_layer - 1):
+        for n in (0, s.n_branch - 1):
+            for which in (0, 1):
+                g = m.kv_view(layer, n, which)[0, :, :s.seqlen].float().cpu().numpy()
+                check_cache(g, orc.cache(layer, n, which), layer == 0, ("C2", layer, n, which))
+    m.close()
 
 
 def test_c3_full_size_prefix_parity():
     prefix_parity("C3", 32, [0, 3])
+
+
+def test_c3_full_size_one_whole_sequence_against_the_oracle():
+    """C3 in the launch configuration the benchmark times (4 x 2048 tokens): one whole sequence goes through the
+    oracle (minutes of host time), so the numbers the benchmark reports, the last-position logits, and the late
+    positions and cache rows behind them are compared with the oracle directly, not only through a prefix."""
+    s = ki.CONFIGS["C3"]
+    m, w = build(s)
+    wb = host_bits(w)
+    tok = ki.uniform_tokens(1, s.vocab, s.batch, s.seqlen, DEV)
+    last = m.prefill(tok).cpu().numpy()
+    assert m.device_status() == 0
+    b, first = 2, 1536                                     # rows 1536 .. 2047: the last four key tiles
+    orc = oracle.Oracle(s, wb, bf16_store=False)
+    ref, _ = orc.prefill(tok[b].cpu().numpy(), logits_from=first)
+    got = m.logits_rows([b * s.seqlen + t for t in range(first, s.seqlen)]).cpu().numpy()
+    check_parity(got, ref, ref, f"C3 seq {b} positions {first}..{s.seqlen - 1} of the full-size run (fp32 oracle)")
+    rel, mx = logits_metrics(last[b], ref[-1])
+    record(f"[parity] C3 seq {b} last position of the timed call: relL2={rel:.3e} maxabs={mx:.3e}")
+    assert rel <= REL_L2_MAX and mx <= MAX_ABS_MAX
+    # cache rows at late positions, every head, against the unrounded oracle: one bf16 step of the value plus the
+    # logits' relative bound for what the layers above have accumulated
+    late = [1000, 1535, 1536, 2046, 2047]
+    for layer in (0, s.n_layer // 2, s.n_layer - 1):
+        for n in (0, s.n_branch - 1):
+            for which in (0, 1):
+                g = m.kv_view(layer, n, which)[b][:, late].float().cpu().numpy()
+                r = orc.cache(layer, n, which)[:, late]
+                rel = np.linalg.norm(g - r) / np.linalg.norm(r)
+                assert rel <= REL_L2_MAX, (layer, n, which, rel)
+                assert np.abs(g - r).max() <= 0.05 * np.abs(r).max(), (layer, n, which)
+    m.close()
 
 
 def test_c3_full_size_late_positions_agree_across_launch_configurations():
@@ -620,6 +680,41 @@ def test_c3_full_size_late_positions_agree_across_launch_configurations():
     # (random-init logits are nearly flat, so the arg max itself may differ)
     for b in range(s.batch):
         assert full[b, step[b].argmax()].item() >= full[b].max().item() - 2 * mx, b
+    m.close()
+
+
+def test_c4_full_size_one_whole_sequence_and_decode_steps_against_the_oracle():
+    """C4 as the benchmark runs it (16 sequences x 2048 tokens, then decode steps at batch 16): one whole
+    sequence goes through the oracle, then four teacher-forced decode steps at context 2048 .. 2051, so the
+    cache-streaming kernels are compared with the oracle at the context length the benchmark times."""
+    s = ki.CONFIGS["C4"]
+    steps = 4
+    m, w = build(s)
+    wb = host_bits(w)
+    tok = ki.uniform_tokens(1, s.vocab, s.batch, s.seqlen + steps, DEV)
+    last = m.prefill(tok[:, :s.seqlen].contiguous()).cpu().numpy()
+    assert m.device_status() == 0
+    b, first = 5, s.seqlen - 128
+    orc = oracle.Oracle(s, wb, bf16_store=False)
+    ref, _ = orc.prefill(tok[b, :s.seqlen].cpu().numpy(), logits_from=first)
+    got = m.logits_rows([b * s.seqlen + t for t in range(first, s.seqlen)]).cpu().numpy()
+    check_parity(got, ref, ref, f"C4 seq {b} positions {first}..{s.seqlen - 1} of the full-size prefill (fp32 oracle)")
+    rel, mx = logits_metrics(last[b], ref[-1])
+    assert rel <= REL_L2_MAX and mx <= MAX_ABS_MAX
+    for layer in (0, s.n_layer - 1):
+        for which in (0, 1):
+            g = m.kv_view(layer, 2, which)[b][:, first:s.seqlen].float().cpu().numpy()
+            r = orc.cache(layer, 2, which)[:, first:]
+            assert np.linalg.norm(g - r) / np.linalg.norm(r) <= REL_L2_MAX, (layer, which)
+    for i in range(steps):
+        t = s.seqlen + i
+        got = m.decode_step(tok[:, t].contiguous()).cpu().numpy()
+        want = orc.decode_step(int(tok[b, t]))
+        rel, mx = logits_metrics(got[b], want)
+        record(f"[parity] C4 decode step at context {t}, seq {b} (fp32 oracle): relL2={rel:.3e} maxabs={mx:.3e} "
+               f"argmax equal={int(got[b].argmax() == want.argmax())}")
+        assert rel <= REL_L2_MAX and mx <= MAX_ABS_MAX, (t, rel, mx)
+    assert m.device_status() == 0 and m.cur_len == s.seqlen + steps
     m.close()
 
 
