@@ -310,6 +310,129 @@ def run_decode(args, shape, kr, ki, replicas, torch):
     print(json.dumps(line))
 
 
+def prefill_leg(name, args, kr, ki, torch, dev, local_rank, steps=20):
+    """A short prefill measurement of another BASELINE config, for the `other_configs` key of the default line:
+    same protocol as the headline (warm-up, events on the launching stream, L2 flushed between steps when the
+    weights fit in it, clock samples during the timed steps, a second pass with events around every launch)."""
+    shape = ki.CONFIGS[name]
+    w = ki.make_weights(shape, seed=0, device=dev, dtype=args.dtype)
+    model = kr.KrakenModel(kr.make_config(shape), w, dev, dtype=args.dtype)
+    tok = ki.uniform_tokens(1, shape.vocab, shape.batch, shape.seqlen, dev)
+    logits = torch.empty(shape.batch, shape.vocab, dtype=torch.float32, device=dev)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev) if weight_bytes(shape) <= 126e6 else None
+    for _ in range(5):
+        model.prefill(tok, logits)
+    torch.cuda.synchronize()
+    model.profile_read()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    time.sleep(0.25)
+    e0 = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+    e1 = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+    for i in range(steps):
+        if flush is not None:
+            flush.zero_()
+        e0[i].record()
+        model.prefill(tok, logits)
+        e1[i].record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    per_step = sorted(a.elapsed_time(b) for a, b in zip(e0, e1))
+    _, launches = model.profile_read()
+    ms = sum(per_step) / steps
+    model.profile_enable(True)
+    for _ in range(steps):
+        if flush is not None:
+            flush.zero_()
+        model.prefill(tok, logits)
+    prof_ms, prof_n = model.profile_read()
+    model.profile_enable(False)
+    status = model.device_status()
+    model.close()
+    peaks, _ = load_peaks()
+    fl = ki.algorithmic_flops(shape)
+    tokens = shape.batch * shape.seqlen
+    return {
+        "workload": f"{name} prefill", "batch": shape.batch, "seqlen": shape.seqlen, "steps": steps,
+        "ttft_ms": ms, "ttft_ms_median": per_step[len(per_step) // 2], "ttft_ms_min": per_step[0],
+        "tokens_per_s": tokens / (ms * 1e-3),
+        "model_tflops": fl["total"] / (ms * 1e-3) / 1e12,
+        "frac_of_nominal_2250": fl["total"] / (ms * 1e-3) / 2.25e15,
+        "frac_of_measured_sustained": fl["total"] / (ms * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"],
+        "gpu_launches_per_step": int(sum(launches.values())) // steps,
+        "l2": "flushed between steps" if flush is not None else "weights exceed L2",
+        "kernels_ms_per_step": {k: v / steps for k, v in prof_ms.items()},
+        "clocks": clocks, "device_status": status,
+    }
+
+
+def decode_leg(name, args, kr, ki, torch, dev, local_rank):
+    """The decode config for the `other_configs` key: prefill once, then all of the config's greedy decode steps
+    (events around every step), then the same steps with events around every launch (single chain)."""
+    shape = ki.CONFIGS[name]
+    steps = shape.decode_steps
+    w = ki.make_weights(shape, seed=0, device=dev, dtype=args.dtype)
+    model = kr.KrakenModel(kr.make_config(shape), w, dev, dtype=args.dtype)
+    tok = ki.uniform_tokens(1, shape.vocab, shape.batch, shape.seqlen, dev)
+    logits = torch.empty(shape.batch, shape.vocab, dtype=torch.float32, device=dev)
+
+    def start():
+        model.prefill(tok, logits)
+        return logits.argmax(1).to(torch.int32)
+
+    nxt = start()
+    for _ in range(3):
+        model.decode_step(nxt, logits)
+        nxt = logits.argmax(1).to(torch.int32)
+    p0, p1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    p0.record()
+    nxt = start()
+    p1.record()
+    torch.cuda.synchronize()
+    prefill_ms = p0.elapsed_time(p1)
+    model.profile_read()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    time.sleep(0.25)
+    e0 = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+    e1 = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+    for i in range(steps):
+        e0[i].record()
+        model.decode_step(nxt, logits)
+        e1[i].record()
+        nxt = logits.argmax(1).to(torch.int32)
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms = sum(a.elapsed_time(b) for a, b in zip(e0, e1)) / steps
+    _, launches = model.profile_read()
+    nxt = start()
+    model.profile_read()
+    model.profile_enable(True)
+    for _ in range(steps):
+        model.decode_step(nxt, logits)
+        nxt = logits.argmax(1).to(torch.int32)
+    prof_ms, prof_n = model.profile_read()
+    model.profile_enable(False)
+    status = model.device_status()
+    model.close()
+    peaks, _ = load_peaks()
+    wb_, kvb = decode_bytes(shape, shape.seqlen + steps // 2)
+    gbs = (wb_ + kvb) / (ms * 1e-3) / 1e9
+    attn_ms = prof_ms["attention"] / steps
+    gemm_ms = sum(prof_ms[k] for k in ("gemm_qkv", "gemm_proj", "gemm_up", "gemm_down", "tail")) / steps
+    return {
+        "workload": f"{name} decode after prefill", "batch": shape.batch, "context": shape.seqlen, "steps": steps,
+        "prefill_ms": prefill_ms, "ms_per_step": ms, "tokens_per_s": shape.batch / (ms * 1e-3),
+        "hbm_gbs": gbs, "frac_of_measured_hbm": gbs / peaks["hbm_gbs"], "frac_of_nominal_8000": gbs / 8000.0,
+        "bytes_per_step": {"weights": wb_, "kv_cache": kvb},
+        "attention_gbs_single_chain": kvb / (attn_ms * 1e-3) / 1e9 if attn_ms > 0 else None,
+        "weight_streaming_gbs_single_chain": wb_ / (gemm_ms * 1e-3) / 1e9 if gemm_ms > 0 else None,
+        "gpu_launches_per_step": int(sum(launches.values())) // steps,
+        "kernels_ms_per_step_single_chain": {k: v / steps for k, v in prof_ms.items()},
+        "clocks": clocks, "device_status": status,
+    }
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -324,6 +447,8 @@ def main():
     ap.add_argument("--ref-tokens", type=int, default=8, help="tokens per step of the reference arm")
     ap.add_argument("--cpu-baseline-seconds", type=float, default=15.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--headline-only", action="store_true",
+                    help="skip the short legs of the other BASELINE configs that the default C3 run appends")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
 
@@ -494,6 +619,17 @@ def main():
         rate, dt = oracle_tokens_per_s(shape, wb, ids, n)
         line["cpu_baseline"] = {"value": rate, "unit": "tokens/s", "cores": oracle.num_threads(), "kind": "oracle",
                                 "sample": f"oracle prefill of the first {n} tokens of sequence 0 ({dt:.1f} s)"}
+    if world == 1 and args.workload == "C3" and not args.seqlen and not args.headline_only:
+        # the other four BASELINE configs, measured in the same run (each leg builds and frees its own model)
+        model.close()
+        del model, w, tok, logits
+        torch.cuda.empty_cache()
+        others = {}
+        for name in ("C0", "C1", "C2"):
+            others[name] = prefill_leg(name, args, kr, ki, torch, dev, local_rank)
+            torch.cuda.empty_cache()
+        others["C4"] = decode_leg("C4", args, kr, ki, torch, dev, local_rank)
+        line["other_configs"] = others
     print(json.dumps(line))
     if dist:
         dist.destroy_process_group()
