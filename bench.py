@@ -447,6 +447,9 @@ def main():
     ap.add_argument("--ref-tokens", type=int, default=8, help="tokens per step of the reference arm")
     ap.add_argument("--cpu-baseline-seconds", type=float, default=15.0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--layernorm", default="auto", choices=["auto", "fused", "fused-down"],
+                    help="fused: every LayerNorm inside the GEMM kernel that finishes its rows; fused-down: only behind "
+                         "the FFN down-projection (for comparison with the default, separate LayerNorm launches)")
     ap.add_argument("--headline-only", action="store_true",
                     help="skip the short legs of the other BASELINE configs that the default C3 run appends")
     args = ap.parse_args()
@@ -473,6 +476,9 @@ def main():
         raise SystemExit("bench.py needs a CUDA device: the product path has no CPU fallback")
     torch.cuda.set_device(local_rank)
     dev = f"cuda:{local_rank}"
+    if args.layernorm != "auto":
+        with kr.storage_dtype(args.dtype):
+            kr.set_tuning(kr.TUNE_LN_FUSION, 2 if args.layernorm == "fused" else 3)
     dist = None
     if world > 1:
         dist = replicas.init_process_group("nccl", torch.device(dev))

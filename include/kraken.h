@@ -233,11 +233,14 @@ int kraken_storage_dtype(void);
  * for one step that give the same result and picks by shape, a test can force either one, process-wide:
  * value 0 restores the library's own choice.  Nothing on the launch path reads the environment; the two
  * environment switches of a handle (KRAKEN_NO_GRAPH, KRAKEN_DECODE_ONE_CHAIN) are read once by kraken_create.
- * Errors: EINVAL (unknown key, value outside 0..2). */
+ * Errors: EINVAL (unknown key, value outside 0..3). */
 typedef enum kraken_tuning_key {
     KRAKEN_TUNE_LN_ROW_KERNEL = 0,   /* LayerNorm of few or wide rows: 1 = one warp per row, 2 = one CTA per row */
     KRAKEN_TUNE_ATTN_SCHEDULE = 1,   /* prefill attention: 1 = one CTA per work item (no per-CTA work lists)     */
-    KRAKEN_TUNE_COUNT = 2
+    KRAKEN_TUNE_LN_FUSION = 2,       /* LayerNorm inside the kernel that finishes its input rows (kraken_op_grouped_gemm_ln):
+                                        2 = wherever it fits, 3 = behind the FFN down-projection only; 0, 1 = every
+                                        LayerNorm its own launch (the default: see the measurements in the source)   */
+    KRAKEN_TUNE_COUNT = 3
 } kraken_tuning_key;
 int kraken_tuning_set(int32_t key, int32_t value);
 
@@ -248,6 +251,20 @@ int kraken_tuning_set(int32_t key, int32_t value);
  * the failure path of the kernels' waits (Sec. 3.1's steps never block forever here) is exercised
  * without starving a real kernel.  Errors: EINVAL, ECUDA. */
 int kraken_test_wait_limit(uint32_t *d_status, uint32_t limit_us, void *stream);
+
+/* Issue-rate probe for the tensor-core products of the attention step (Sec. 2.1's softmax(Q K^T) V on 128 x 128
+ * tiles): n_ctas CTAs (one per SM at most) each issue `iters` blocks of `tcgen05.mma` instructions of M 128,
+ * K 16 from one thread (issuers = 1) or from two threads in different warps (issuers = 2, each on its own
+ * accumulator) and record the SM clock cycles from the first issue to the completion of the last product in
+ * d_cycles[cta] (device int64; -1 if a bounded wait gave up, then bit 1 of *d_status is raised too).
+ * form: 0 = S = Q K^T (both operands in shared memory, N 128); 1 = O += P V (A from tensor memory, V MN-major in
+ * shared memory, N 128); 2 = 8 of the first then 8 of the second, alternating (the attention kernel's pattern);
+ * 3 = form 2 with a commit after every 8; 4 = form 3 with a barrier wait that succeeds at once after every 8;
+ * 5 = form 0 with N 64; 6 = form 0 with N 256.  *products_per_iter (host, may be NULL) receives the products one
+ * thread issues per iteration, so cycles per product = d_cycles / (iters * products_per_iter) for one issuer and
+ * half of that for two.  A measurement tool, not part of the model's arithmetic.  Errors: EINVAL, ECUDA. */
+int kraken_test_mma_issue_rate(int32_t form, int32_t issuers, int32_t iters, int64_t *d_cycles, int32_t n_ctas,
+                               int32_t *products_per_iter, uint32_t *d_status, void *stream);
 
 /* ------------------------------------------------------------------------------------------
  * Single steps of the path, exposed so that each kernel can be checked on its own.  All
@@ -308,6 +325,30 @@ typedef struct kraken_gemm_args {
  * Requirements: a, w 16-byte aligned; lda, ldw multiples of 8; k >= 8.  d_status as above (bit 1).
  * Errors: EINVAL, EUNSUPPORTED, ECUDA. */
 int kraken_op_grouped_gemm(const kraken_gemm_args *args, uint32_t *d_status, void *stream);
+
+/* LayerNorm of the finished rows in the same kernel as a RESID_F32 or RESID_SUM grouped GEMM (Algorithm 1:
+ * `x = LN(x)` follows `out = res + FFN(x)`, `x = LN(x + y)` follows `x = res + MHA(x)`):
+ *     ln_out[g] = LN(out_f32[g] + y; gamma[g], beta[g])      over the n_out columns of every row,
+ * biased variance, statistics in fp32, result stored in the library's 16-bit type.  A row is spread over the
+ * N tiles of its row block, i.e. over several CTAs: every epilogue warp leaves the statistics of its part in
+ * d_scratch, waits (bounded; status bit 1 if it gives up) for the other parts and normalises the values it kept
+ * in tensor memory.  out_f32 (and sum) are written as without the LayerNorm.
+ * d_scratch: device memory of kraken_gemm_ln_scratch_bytes() bytes, zeroed ONCE by the caller before its first
+ * use; every launch leaves its counters at zero again, so launches on one stream can share it (launches that
+ * overlap on the device cannot).  gamma, beta: [G][n_out] (beta may be NULL = zeros); y: fp32 [M, n_out] added
+ * to every group's rows before the statistics, or NULL.  Errors: EINVAL (other epilogues, missing pointers),
+ * EUNSUPPORTED (m <= 32 rows with n_tile = 8; a row block of more N tiles than CTAs run at once),
+ * ECAPACITY (scratch_bytes too small). */
+typedef struct kraken_gemm_ln_args {
+    void *ln_out;        int64_t ln_out_gstride; int32_t ld_ln_out;   /* 16-bit [G][M, n_out]                 */
+    const void *gamma;   const void *beta;       int64_t gb_gstride;  /* 16-bit [G][n_out]                    */
+    const float *y;      int32_t ld_y;
+    float eps;
+    void *d_scratch;     size_t scratch_bytes;
+} kraken_gemm_ln_args;
+int kraken_gemm_ln_scratch_bytes(int32_t groups, int32_t m, int32_t n_out, int32_t k, int32_t n_tile, size_t *bytes);
+int kraken_op_grouped_gemm_ln(const kraken_gemm_args *args, const kraken_gemm_ln_args *ln, uint32_t *d_status,
+                              void *stream);
 
 /* Causal multi-head attention over a prefix held in the cache layout (Sec. 2.1):
  * for sequence b, head h, query row t (position pos0 + t): softmax over keys 0..pos0+t of

@@ -38,12 +38,13 @@ EXPORTS = (
     "kraken_stage_head", "kraken_decode_step", "kraken_decode_step_host", "kraken_kv_view",
     "kraken_device_status", "kraken_cur_len", "kraken_profile_enable", "kraken_profile_read", "kraken_reset", "kraken_destroy", "kraken_strerror", "kraken_last_cuda_error",
     "kraken_op_embed", "kraken_op_layernorm", "kraken_op_grouped_gemm", "kraken_op_attention",
+    "kraken_op_grouped_gemm_ln", "kraken_gemm_ln_scratch_bytes",
     "kraken_op_decode_attention", "kraken_decode_attention_sizes",
     "kraken_op_decode_attention_static", "kraken_decode_attention_static_capacity", "kraken_storage_dtype",
-    "kraken_tuning_set", "kraken_test_wait_limit",
+    "kraken_tuning_set", "kraken_test_wait_limit", "kraken_test_mma_issue_rate",
 )
 
-TUNE_LN_ROW_KERNEL, TUNE_ATTN_SCHEDULE = 0, 1
+TUNE_LN_ROW_KERNEL, TUNE_ATTN_SCHEDULE, TUNE_LN_FUSION = 0, 1, 2
 STATUS_BAD_TOKEN, STATUS_WAIT_LIMIT = 1, 2
 
 
@@ -73,6 +74,16 @@ class GemmArgs(C.Structure):
         ("seqlen", C.c_int32), ("pos0", C.c_int32), ("n_head", C.c_int32), ("head_dim", C.c_int32),
         ("max_pos", C.c_int32), ("gelu_tanh", C.c_int32), ("n_tile", C.c_int32), ("n_kv_head", C.c_int32),
         ("reserved", C.c_int32 * 1),
+    ]
+
+
+class GemmLnArgs(C.Structure):
+    _fields_ = [
+        ("ln_out", C.c_void_p), ("ln_out_gstride", C.c_int64), ("ld_ln_out", C.c_int32),
+        ("gamma", C.c_void_p), ("beta", C.c_void_p), ("gb_gstride", C.c_int64),
+        ("y", C.c_void_p), ("ld_y", C.c_int32),
+        ("eps", C.c_float),
+        ("d_scratch", C.c_void_p), ("scratch_bytes", C.c_size_t),
     ]
 
 
@@ -146,6 +157,8 @@ def lib(dtype: Optional[str] = None) -> C.CDLL:
         L.kraken_op_embed.argtypes = [vp, i32, i32, i32, vp, vp, i32, i32, vp, vp, vp]
         L.kraken_op_layernorm.argtypes = [vp, i64, vp, vp, vp, i32, i32, i32, C.c_float, vp, vp, vp]
         L.kraken_op_grouped_gemm.argtypes = [C.POINTER(GemmArgs), vp, vp]
+        L.kraken_op_grouped_gemm_ln.argtypes = [C.POINTER(GemmArgs), C.POINTER(GemmLnArgs), vp, vp]
+        L.kraken_gemm_ln_scratch_bytes.argtypes = [i32, i32, i32, i32, i32, C.POINTER(C.c_size_t)]
         L.kraken_op_attention.argtypes = [vp, i64, vp, vp, i64, i64, i32, i32, i32, i32, i32, i32, i32, i32, vp, i64, vp]
         L.kraken_op_decode_attention.argtypes = [vp, i64, vp, vp, i64, i64, i32, i32, i32, i32, i32, i32, i32, i32, vp,
                                                  C.c_size_t, vp, i64, vp]
@@ -157,6 +170,7 @@ def lib(dtype: Optional[str] = None) -> C.CDLL:
         L.kraken_storage_dtype.argtypes = []
         L.kraken_tuning_set.argtypes = [i32, i32]
         L.kraken_test_wait_limit.argtypes = [vp, C.c_uint32, vp]
+        L.kraken_test_mma_issue_rate.argtypes = [i32, i32, i32, vp, i32, C.POINTER(C.c_int32), vp, vp]
         if L.kraken_storage_dtype() != (1 if dtype == "f16" else 0):
             raise RuntimeError(f"{path} was not built for storage dtype {dtype}")
         _libs[dtype] = L
@@ -411,6 +425,18 @@ def op_grouped_gemm(args: GemmArgs, status: Optional[torch.Tensor] = None):
     _check(lib().kraken_op_grouped_gemm(C.byref(args), _ptr(status), _stream()), "kraken_op_grouped_gemm")
 
 
+def gemm_ln_scratch_bytes(groups: int, m: int, n_out: int, k: int, n_tile: int = 0) -> int:
+    n = C.c_size_t(0)
+    _check(lib().kraken_gemm_ln_scratch_bytes(groups, m, n_out, k, n_tile, C.byref(n)), "kraken_gemm_ln_scratch_bytes")
+    return int(n.value)
+
+
+def op_grouped_gemm_ln(args: GemmArgs, ln: GemmLnArgs, status: Optional[torch.Tensor] = None):
+    """A RESID_F32 / RESID_SUM grouped GEMM with the LayerNorm of the finished rows in the same kernel."""
+    _check(lib().kraken_op_grouped_gemm_ln(C.byref(args), C.byref(ln), _ptr(status), _stream()),
+           "kraken_op_grouped_gemm_ln")
+
+
 def op_attention(q: torch.Tensor, k_cache: torch.Tensor, v_cache: torch.Tensor, batch: int, seqlen: int, pos0: int,
                  n_head: int) -> torch.Tensor:
     """q bf16 [G, batch*seqlen, d]; k_cache / v_cache bf16 [G, batch, key/value heads, max_pos, head_dim]
@@ -495,3 +521,18 @@ def test_wait_limit(status: torch.Tensor, limit_us: int) -> None:
 
 
 test_wait_limit.__test__ = False   # not a pytest case
+
+
+def mma_issue_rate(form: int, issuers: int = 1, iters: int = 2000, n_ctas: int = 148) -> float:
+    """SM clock cycles per tcgen05.mma (M 128, K 16) of the issue-rate probe, averaged over the CTAs
+    (see kraken_test_mma_issue_rate for the forms)."""
+    dev = torch.device("cuda", torch.cuda.current_device())
+    cycles = torch.zeros(n_ctas, dtype=torch.int64, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    per = C.c_int32(0)
+    _check(lib().kraken_test_mma_issue_rate(form, issuers, iters, cycles.data_ptr(), n_ctas, C.byref(per),
+                                            status.data_ptr(), _stream()), "kraken_test_mma_issue_rate")
+    torch.cuda.synchronize()
+    if int(status.item()) != 0 or bool((cycles < 0).any()):
+        raise KrakenError(ECUDA, "kraken_test_mma_issue_rate: a bounded wait gave up")
+    return float(cycles.double().mean().item()) / (iters * per.value * issuers)

@@ -7,6 +7,8 @@
 //   -> gather of the wanted rows -> GEMM W_concat -> final LN -> GEMM unembedding -> fp32 logits.
 #include <string.h>
 
+#include <algorithm>
+
 #include <new>
 #include <vector>
 
@@ -21,7 +23,8 @@ constexpr size_t ALIGN = 256;
 size_t align_up(size_t v) { return (v + ALIGN - 1) / ALIGN * ALIGN; }
 
 struct Layout {
-    size_t status, tokens, rows, logits, x0, x, a, s, u, q, o, g, dec_part, x_alt, row_seq, row_pos, pos_arr, total;
+    size_t status, tokens, rows, logits, x0, x, a, s, u, q, o, g, dec_part, x_alt, row_seq, row_pos, pos_arr, ln_parts,
+        ln_parts_bytes, ln_cnt, ln_cnt_bytes, total;
 };
 
 int kv_heads_of(const kraken_config &c) { return c.n_kv_head > 0 ? c.n_kv_head : c.n_head; }
@@ -74,6 +77,13 @@ Layout layout_of(const kraken_config *c) {
     l.row_seq = take(T * 4);                            // packed prefill: sequence and position of every row
     l.row_pos = take(T * 4);
     l.pos_arr = take((size_t)c->max_batch * 4);         // next position of every sequence (device copy)
+    // LayerNorm behind the GEMM epilogues: per row and N tile two (mean, M2, count) entries, and two counters per
+    // 32 rows.  Sized for 256-wide tiles on every row; narrower tiles (short prompts) fit into the 4 MiB floor or
+    // the LayerNorm runs as its own launch.
+    l.ln_parts_bytes = std::max<size_t>(gemm_ln_parts_bytes((int)N, (int)T, (int)d, GEMM_TILE_PAIR), size_t(4) << 20);
+    l.ln_parts = take(l.ln_parts_bytes);
+    l.ln_cnt_bytes = gemm_ln_cnt_bytes((int)N, (int)T);
+    l.ln_cnt = take(l.ln_cnt_bytes);
     l.total = off;
     return l;
 }
@@ -287,6 +297,39 @@ int run_layers(const RunCtx &rc, const int32_t *d_tokens) {
     const bool sum_pass = small_rows && T > SKINNY_MAX_ROWS;
     const bool sum_beside = sum_pass && !rc.stage && branch_streams(h) == KRAKEN_OK;
     bool sum_pending = false;
+    uint16_t *const u_ = at<uint16_t>(h, h->lay.u);
+    // A LayerNorm can run behind the epilogue of the GEMM that finishes its input rows (LN-2 behind the attention
+    // output projection, the next layer's LN-1 behind the down-projection) when that GEMM goes to the tensor-core
+    // kernels, the statistics scratch holds its tiling and the path is not driven in pieces (there y comes from
+    // outside after the projection).  It is not the default: measured, it pays only behind the down-projection of
+    // long prompts (K = d_ff per tile leaves the epilogue time to spare: C3 109.4 -> 108.9 ms), costs time behind
+    // the output projection (its epilogue already bounds it: 8.2 -> 18.6 ms per step) and for short prompts (one
+    // tile per CTA, the wait for the row block's other tiles is exposed: C1 0.98 -> 1.04 ms), and the statistics
+    // are summed in another order than the LayerNorm kernel's, so a sequence would no longer give the same 16-bit
+    // activations alone and inside a batch that takes the other route.  KRAKEN_TUNE_LN_FUSION: 2 = wherever it
+    // fits, 3 = behind the down-projection only.  The first layer's LN-1 reads the embedding and is always a
+    // launch of its own.
+    auto ln_fits = [&](const GemmShape &gs) {
+        const int bn = gemm_pick_bn(gs);
+        const int cols = bn == GEMM_TILE_PAIR ? 256 : bn;
+        const int sms = sm_count() > 0 ? sm_count() : 148;
+        return gemm_ln_parts_bytes(N, T, d, bn) <= h->lay.ln_parts_bytes &&
+               (d + cols - 1) / cols <= (bn == GEMM_TILE_PAIR ? sms / 2 : sms);
+    };
+    const int ln_mode = tuning(KRAKEN_TUNE_LN_FUSION);
+    const bool ln_fuse = !rc.stage && T > SKINNY_MAX_ROWS && (ln_mode == 2 || ln_mode == 3);
+    const bool fuse_ln2 = ln_fuse && ln_mode == 2 && !c.parallel_ffn && ln_fits(GemmShape{N, T, d, d});
+    const bool fuse_ln1 = ln_fuse && ln_fits(GemmShape{N, T, d, F});
+    auto ln_epi = [&](EpiParams &e, const void *gamma, const void *beta, long long off, const float *y) {
+        e.ln_out = u_; e.ln_out_gstride = td; e.ln_ld_out = d;
+        e.ln_gamma = (const uint16_t *)gamma + off;
+        e.ln_beta = beta ? (const uint16_t *)beta + off : nullptr;
+        e.ln_gb_gstride = d;
+        e.ln_y = y; e.ln_ld_y = d;
+        e.ln_eps = c.ln_eps;
+        e.ln_parts = at<float4>(h, h->lay.ln_parts);
+        e.ln_cnt = at<uint32_t>(h, h->lay.ln_cnt);
+    };
     float *x0 = at<float>(h, h->lay.x0), *x = at<float>(h, h->lay.x), *a = at<float>(h, h->lay.a),
           *S = at<float>(h, h->lay.s);
     uint16_t *u = at<uint16_t>(h, h->lay.u), *q = at<uint16_t>(h, h->lay.q), *o = at<uint16_t>(h, h->lay.o),
@@ -310,8 +353,8 @@ int run_layers(const RunCtx &rc, const int32_t *d_tokens) {
         const long long ln_off = (long long)l * N * d;
         EpiParams e = epi_zero();
         if (rc.stage != STAGE_FFN) {
-        // x = LN(x)
-        {
+        // x = LN(x)   (already done behind the previous layer's down-projection when fused)
+        if (!(fuse_ln1 && l > l_begin)) {
             LaunchScope scope(h, KRAKEN_PROF_LAYERNORM, rc.st);
             KR_TRY(launch_layernorm(xin, xin_gs, nullptr, (const uint16_t *)h->w.ln1_g + ln_off,
                                     h->w.ln1_b ? (const uint16_t *)h->w.ln1_b + ln_off : nullptr, N, T, d, c.ln_eps,
@@ -377,6 +420,15 @@ int run_layers(const RunCtx &rc, const int32_t *d_tokens) {
         e.kind = KRAKEN_EPI_RESID_F32;
         e.out_f32 = a; e.out_f32_gstride = td; e.ld_out_f32 = d;
         e.resid = xin; e.resid_gstride = xin_gs; e.ld_resid = d;
+        if (fuse_ln2) {
+            // x = LN(x + y) behind this epilogue: y is the shared embedding in the first layer, the cross-branch sum
+            // afterwards (formed by the previous down-projection, or by the pass beside it, joined here)
+            if (sum_pending) {
+                KR_CU(cudaStreamWaitEvent(rc.st, h->ev_join[1], 0));
+                sum_pending = false;
+            }
+            ln_epi(e, h->w.ln2_g, h->w.ln2_b, ln_off, c.no_combine ? nullptr : (l == 0 ? x0 : S));
+        }
         KR_TRY(model_gemm(rc, G_PROJ, l, T, o, td, e));
         }  // attention half
         if (rc.stage == STAGE_ATTN) continue;
@@ -388,7 +440,7 @@ int run_layers(const RunCtx &rc, const int32_t *d_tokens) {
             KR_TRY(launch_layernorm(a, td, rc.y_ext, (const uint16_t *)h->w.ln2_g + ln_off,
                                     h->w.ln2_b ? (const uint16_t *)h->w.ln2_b + ln_off : nullptr, N, T, d, c.ln_eps,
                                     u, rc.st, nullptr, 0, 0, status));
-        } else if (!c.parallel_ffn) {
+        } else if (!c.parallel_ffn && !fuse_ln2) {
             if (sum_pending) {
                 KR_CU(cudaStreamWaitEvent(rc.st, h->ev_join[1], 0));
                 sum_pending = false;
@@ -413,6 +465,8 @@ int run_layers(const RunCtx &rc, const int32_t *d_tokens) {
         e.out_f32 = x; e.out_f32_gstride = td; e.ld_out_f32 = d;
         e.resid = a; e.resid_gstride = td; e.ld_resid = d;
         e.sum = S; e.ld_sum = d;
+        if (fuse_ln1 && l + 1 < l_end)   // the next layer's x = LN(x) behind this epilogue
+            ln_epi(e, h->w.ln1_g, h->w.ln1_b, ln_off + (long long)N * d, nullptr);
         KR_TRY(model_gemm(rc, G_DOWN, l, T, gb, (long long)T * F, e));
         if (rc.stage == STAGE_FFN) {
             // driven from outside: the sum of this device's branches, for the caller's all-reduce
@@ -844,7 +898,8 @@ int kraken_create(const kraken_config *cfg, const kraken_weights *w, void *d_kv,
         h->tmB_bn[i] = 0;
         h->tmA_key[i] = {nullptr, 0, 0, 0};
     }
-    if (cudaMemset(h->scratch + lay.status, 0, 256) != cudaSuccess) {
+    if (cudaMemset(h->scratch + lay.ln_cnt, 0, lay.ln_cnt_bytes) != cudaSuccess ||
+        cudaMemset(h->scratch + lay.status, 0, 256) != cudaSuccess) {
         delete h;
         return KRAKEN_ECUDA;
     }
@@ -1163,6 +1218,7 @@ int kraken_reset(kraken_handle *h) {
     if (!h) return KRAKEN_EINVAL;
     if (cudaStreamSynchronize(h->last_stream) != cudaSuccess) return KRAKEN_ECUDA;
     if (cudaMemset(h->scratch + h->lay.status, 0, 256) != cudaSuccess) return KRAKEN_ECUDA;
+    if (cudaMemset(h->scratch + h->lay.ln_cnt, 0, h->lay.ln_cnt_bytes) != cudaSuccess) return KRAKEN_ECUDA;
     h->cur_len = 0;
     h->batch = 0;
     h->last_rows = 0;
@@ -1248,7 +1304,35 @@ int kraken_op_layernorm(const float *d_a, int64_t a_gstride, const float *d_y, c
                             d_status);
 }
 
+namespace {
+int op_grouped_gemm(const kraken_gemm_args *g, const kraken_gemm_ln_args *ln, uint32_t *d_status, void *stream);
+size_t ln_cnt_region(int groups, int m) { return align_up(gemm_ln_cnt_bytes(groups, m)); }
+int ln_tile_of(const kraken_gemm_args *g) {
+    return g->n_tile ? g->n_tile : gemm_pick_bn(GemmShape{g->groups, g->m, g->n_out, g->k});
+}
+}  // namespace
+
 int kraken_op_grouped_gemm(const kraken_gemm_args *g, uint32_t *d_status, void *stream) {
+    return op_grouped_gemm(g, nullptr, d_status, stream);
+}
+
+int kraken_gemm_ln_scratch_bytes(int32_t groups, int32_t m, int32_t n_out, int32_t k, int32_t n_tile, size_t *bytes) {
+    if (!bytes || groups < 1 || m < 1 || n_out < 1 || k < 1) return KRAKEN_EINVAL;
+    if (n_tile == 8 || (n_tile && n_tile != GEMM_TILE_PAIR && (n_tile < 32 || n_tile > 256 || n_tile % 32)))
+        return KRAKEN_EUNSUPPORTED;
+    const int bn = n_tile ? n_tile : gemm_pick_bn(GemmShape{groups, m, n_out, k});
+    *bytes = ln_cnt_region(groups, m) + gemm_ln_parts_bytes(groups, m, n_out, bn);
+    return KRAKEN_OK;
+}
+
+int kraken_op_grouped_gemm_ln(const kraken_gemm_args *g, const kraken_gemm_ln_args *ln, uint32_t *d_status,
+                              void *stream) {
+    if (!ln) return KRAKEN_EINVAL;
+    return op_grouped_gemm(g, ln, d_status, stream);
+}
+
+namespace {
+int op_grouped_gemm(const kraken_gemm_args *g, const kraken_gemm_ln_args *ln, uint32_t *d_status, void *stream) {
     if (!g || !g->a || !g->w) return KRAKEN_EINVAL;
     if (g->epilogue < KRAKEN_EPI_F32 || g->epilogue > KRAKEN_EPI_QKV) return KRAKEN_EINVAL;
     const int k = g->epilogue;
@@ -1280,9 +1364,25 @@ int kraken_op_grouped_gemm(const kraken_gemm_args *g, uint32_t *d_status, void *
     e.d_model = g->n_head * g->head_dim;
     e.n_kv_head = g->n_kv_head > 0 ? g->n_kv_head : g->n_head;
     e.gelu_tanh = g->gelu_tanh;
-    if (g->n_tile == 8) return launch_gemm_skinny(op, s, e, static_cast<cudaStream_t>(stream));
-    return launch_gemm_tc(op, s, e, nullptr, nullptr, 0, g->n_tile, d_status, static_cast<cudaStream_t>(stream));
+    int n_tile = g->n_tile;
+    if (ln) {
+        if (k != KRAKEN_EPI_RESID_F32 && k != KRAKEN_EPI_RESID_SUM) return KRAKEN_EINVAL;
+        if (!ln->ln_out || !ln->gamma || !ln->d_scratch || !(ln->eps > 0.f)) return KRAKEN_EINVAL;
+        if (n_tile == 8) return KRAKEN_EUNSUPPORTED;
+        n_tile = ln_tile_of(g);
+        const size_t cnt_bytes = ln_cnt_region(g->groups, g->m);
+        if (ln->scratch_bytes < cnt_bytes + gemm_ln_parts_bytes(g->groups, g->m, g->n_out, n_tile)) return KRAKEN_ECAPACITY;
+        e.ln_out = (uint16_t *)ln->ln_out; e.ln_out_gstride = ln->ln_out_gstride; e.ln_ld_out = ln->ld_ln_out;
+        e.ln_gamma = (const uint16_t *)ln->gamma; e.ln_beta = (const uint16_t *)ln->beta; e.ln_gb_gstride = ln->gb_gstride;
+        e.ln_y = ln->y; e.ln_ld_y = ln->ld_y;
+        e.ln_eps = ln->eps;
+        e.ln_cnt = reinterpret_cast<uint32_t *>(ln->d_scratch);
+        e.ln_parts = reinterpret_cast<float4 *>(static_cast<uint8_t *>(ln->d_scratch) + cnt_bytes);
+    }
+    if (n_tile == 8) return launch_gemm_skinny(op, s, e, static_cast<cudaStream_t>(stream));
+    return launch_gemm_tc(op, s, e, nullptr, nullptr, 0, n_tile, d_status, static_cast<cudaStream_t>(stream));
 }
+}  // namespace
 
 int kraken_op_attention(const void *q, int64_t q_gstride, const void *k_cache, const void *v_cache,
                         int64_t cache_gstride, int64_t cache_bstride, int32_t groups, int32_t batch, int32_t seqlen,

@@ -253,8 +253,10 @@ __device__ __forceinline__ void epilogue_chunk(const EpiParams &p, int g, int ro
 constexpr int EPI_STAGE_PITCH = 36;
 constexpr int EPI_STAGE_FLOATS = 32 * EPI_STAGE_PITCH;
 
+// With `ln` set (LayerNorm fused behind the epilogue) the finished row, plus ln_y, comes back in v in the
+// thread = row mapping, for the row statistics and for the copy kept in tensor memory.
 __device__ __forceinline__ void epilogue_f32_staged(const EpiParams &p, int g, int row_base, int m, int col0,
-                                                    const float (&v)[32], float *stage, int lane) {
+                                                    float (&v)[32], float *stage, int lane, bool ln = false) {
     float4 *mine = reinterpret_cast<float4 *>(stage + lane * EPI_STAGE_PITCH);
 #pragma unroll
     for (int j = 0; j < 8; ++j) mine[j] = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
@@ -294,8 +296,8 @@ __device__ __forceinline__ void epilogue_f32_staged(const EpiParams &p, int g, i
             const int row = row_base + it * 4 + r_in;
             if (row < m) {
                 *reinterpret_cast<float4 *>(p.out_f32 + g * p.out_f32_gstride + (long long)row * p.ld_out_f32 + col) = x[it];
-                x[it].x += t[it].x; x[it].y += t[it].y; x[it].z += t[it].z; x[it].w += t[it].w;
-                *reinterpret_cast<float4 *>(p.sum + (long long)row * p.ld_sum + col) = x[it];
+                t[it].x += x[it].x; t[it].y += x[it].y; t[it].z += x[it].z; t[it].w += x[it].w;
+                *reinterpret_cast<float4 *>(p.sum + (long long)row * p.ld_sum + col) = t[it];
             }
         }
     } else {
@@ -310,6 +312,175 @@ __device__ __forceinline__ void epilogue_f32_staged(const EpiParams &p, int g, i
         }
     }
     __syncwarp();
+    if (ln) {
+        if (p.ln_y) {
+#pragma unroll
+            for (int it = 0; it < 8; ++it) {
+                const int row = row_base + it * 4 + r_in;
+                if (row < m) {
+                    const float4 y = *reinterpret_cast<const float4 *>(p.ln_y + (long long)row * p.ln_ld_y + col);
+                    x[it].x += y.x; x[it].y += y.y; x[it].z += y.z; x[it].w += y.w;
+                }
+            }
+        }
+#pragma unroll
+        for (int it = 0; it < 8; ++it)
+            *reinterpret_cast<float4 *>(stage + (it * 4 + r_in) * EPI_STAGE_PITCH + c4) = x[it];
+        __syncwarp();
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const float4 r = mine[j];
+            v[4 * j] = r.x; v[4 * j + 1] = r.y; v[4 * j + 2] = r.z; v[4 * j + 3] = r.w;
+        }
+        __syncwarp();
+    }
+}
+
+// ---------------------------------------------------------------- LayerNorm fused behind the fp32 epilogues
+// (Algorithm 1: x = LN(x) after `out = res + FFN(x)`, x = LN(x + y) after `x = res + MHA(x)`.)
+
+// Running (mean, M2, count) of one row, updated with up to 32 new values: the values are centred on
+// their own mean first and the two sets are joined with the pairwise update, so nothing cancels.
+struct RowStats {
+    float mean, m2, cnt;
+};
+
+__device__ __forceinline__ void stats_join(RowStats &s, float mean_b, float m2_b, float n_b) {
+    if (n_b == 0.f) return;
+    const float tot = s.cnt + n_b;
+    const float delta = mean_b - s.mean;
+    const float w = n_b / tot;
+    s.mean = fmaf(delta, w, s.mean);
+    s.m2 += m2_b + delta * delta * s.cnt * w;
+    s.cnt = tot;
+}
+
+__device__ __forceinline__ void stats_add_chunk(RowStats &s, const float (&z)[32], int ncols) {
+    float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll
+    for (int i = 0; i < 32; i += 4) {
+        a0 += i < ncols ? z[i] : 0.f;
+        a1 += i + 1 < ncols ? z[i + 1] : 0.f;
+        a2 += i + 2 < ncols ? z[i + 2] : 0.f;
+        a3 += i + 3 < ncols ? z[i + 3] : 0.f;
+    }
+    const float cm = ((a0 + a1) + (a2 + a3)) / static_cast<float>(ncols);
+    float q0 = 0.f, q1 = 0.f, q2 = 0.f, q3 = 0.f;
+#pragma unroll
+    for (int i = 0; i < 32; i += 4) {
+        const float d0 = z[i] - cm, d1 = z[i + 1] - cm, d2 = z[i + 2] - cm, d3 = z[i + 3] - cm;
+        q0 = i < ncols ? fmaf(d0, d0, q0) : q0;
+        q1 = i + 1 < ncols ? fmaf(d1, d1, q1) : q1;
+        q2 = i + 2 < ncols ? fmaf(d2, d2, q2) : q2;
+        q3 = i + 3 < ncols ? fmaf(d3, d3, q3) : q3;
+    }
+    stats_join(s, cm, (q0 + q1) + (q2 + q3), static_cast<float>(ncols));
+}
+
+__device__ __forceinline__ void load_h16_chunk(const uint16_t *src, float (&o)[32], int ncols, float fill) {
+    if (ncols == 32 && (reinterpret_cast<uintptr_t>(src) & 15u) == 0) {
+        const uint4 *b4 = reinterpret_cast<const uint4 *>(src);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            uint4 u = __ldg(b4 + i);
+            o[8 * i + 0] = h16_lo(u.x); o[8 * i + 1] = h16_hi(u.x);
+            o[8 * i + 2] = h16_lo(u.y); o[8 * i + 3] = h16_hi(u.y);
+            o[8 * i + 4] = h16_lo(u.z); o[8 * i + 5] = h16_hi(u.z);
+            o[8 * i + 6] = h16_lo(u.w); o[8 * i + 7] = h16_hi(u.w);
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) o[i] = i < ncols ? from_h16(src[i]) : fill;
+    }
+}
+
+__device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t *p) {
+    uint32_t v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
+// The warp has left its part of 32 rows in ln_parts: count it in, then wait until all `need` parts of those
+// rows are there.  Bounded like every other wait; false = gave up (abort flag raised).
+__device__ __forceinline__ bool ln_arrive_and_wait(uint32_t *cnt, uint32_t need, int lane, volatile uint32_t *abort_flag) {
+    __threadfence();
+    __syncwarp();
+    bool ok = true;
+    if (lane == 0) {
+        atomicAdd(cnt, 1u);
+        unsigned long long t0 = 0;
+        uint32_t polls = 0;
+        while (ld_acquire_u32(cnt) < need) {
+            __nanosleep(40);
+            if ((++polls & 63u) == 0u) {
+                if (*abort_flag) { ok = false; break; }
+                const unsigned long long now = global_timer_ns();
+                if (t0 == 0) t0 = now;
+                else if (now - t0 > WAIT_LIMIT_NS) { *abort_flag = 1u; ok = false; break; }
+            }
+        }
+    }
+    // lane 0's acquire and the warp barrier order the other lanes' reads of the parts (which bypass L1) behind it
+    ok = __all_sync(0xFFFFFFFFu, ok);
+    return ok;
+}
+
+// The last of the `need` warps to leave a slab of rows puts its two counters back to zero for the next launch.
+__device__ __forceinline__ void ln_depart(uint32_t *cnt, uint32_t need, int lane) {
+    __syncwarp();
+    if (lane == 0) {
+        if (atomicAdd(cnt + 1, 1u) == need - 1u) {
+            cnt[0] = 0u;
+            cnt[1] = 0u;
+        }
+    }
+}
+
+// Joins the parts of one row in their fixed order: mean and 1 / sqrt(var + eps) of the whole row.
+__device__ __forceinline__ void ln_row_stats(const float4 *parts, int n_parts, float eps, float &mean, float &rstd) {
+    RowStats s{0.f, 0.f, 0.f};
+    for (int p0 = 0; p0 < n_parts; p0 += 8) {      // eight loads in flight, then joined in order
+        float4 v[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) v[i] = p0 + i < n_parts ? __ldcg(parts + p0 + i) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) stats_join(s, v[i].x, v[i].y, v[i].z);
+    }
+    mean = s.mean;
+    rstd = rsqrtf(s.m2 / s.cnt + eps);
+}
+
+// Second pass over one 32-column chunk of one row (the thread's own TMEM lane): normalise and store 16-bit.
+__device__ __forceinline__ void ln_store_chunk(const EpiParams &p, int g, int row, int col0, int ncols, float (&z)[32],
+                                               float mean, float rstd) {
+    float gam[32], bet[32];
+    load_h16_chunk(p.ln_gamma + g * p.ln_gb_gstride + col0, gam, ncols, 0.f);
+    if (p.ln_beta) load_h16_chunk(p.ln_beta + g * p.ln_gb_gstride + col0, bet, ncols, 0.f);
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+        const float n = (z[i] - mean) * rstd;
+        z[i] = p.ln_beta ? fmaf(n, gam[i], bet[i]) : n * gam[i];
+    }
+    store_bf16_chunk(p.ln_out + g * p.ln_out_gstride + (long long)row * p.ln_ld_out + col0, z, ncols);
+}
+
+// The thread = row form of the fp32 epilogues with a LayerNorm behind them (one thread finishes 32 columns of
+// its row): bias, residual, the fp32 output, the running cross-branch sum; v comes back as the row the
+// LayerNorm sees (out + ln_y).
+__device__ __forceinline__ void epilogue_chunk_ln(const EpiParams &p, int g, int row, int col0, int ncols,
+                                                  float (&v)[32]) {
+    if (p.bias) add_bias_chunk(p.bias + g * p.bias_gstride + col0, v, ncols);
+    add_f32_chunk(p.resid + g * p.resid_gstride + (long long)row * p.ld_resid + col0, v, ncols);
+    store_f32_chunk(p.out_f32 + g * p.out_f32_gstride + (long long)row * p.ld_out_f32 + col0, v, ncols);
+    if (p.kind == KRAKEN_EPI_RESID_SUM) {
+        float t[32];
+#pragma unroll
+        for (int i = 0; i < 32; ++i) t[i] = v[i];
+        float *sp = p.sum + (long long)row * p.ld_sum + col0;
+        if (g > 0) add_f32_chunk(sp, t, ncols);
+        store_f32_chunk(sp, t, ncols);
+    }
+    if (p.ln_y) add_f32_chunk(p.ln_y + (long long)row * p.ln_ld_y + col0, v, ncols);
 }
 
 __device__ __forceinline__ bool epilogue_f32_stageable(const EpiParams &p) {
@@ -320,6 +491,7 @@ __device__ __forceinline__ bool epilogue_f32_stageable(const EpiParams &p) {
         ok = ok && (p.ld_resid & 3) == 0 && (reinterpret_cast<uintptr_t>(p.resid) & 15) == 0 &&
              (p.resid_gstride & 3) == 0;
     if (p.kind == KRAKEN_EPI_RESID_SUM) ok = ok && (p.ld_sum & 3) == 0 && (reinterpret_cast<uintptr_t>(p.sum) & 15) == 0;
+    if (p.ln_out && p.ln_y) ok = ok && (p.ln_ld_y & 3) == 0 && (reinterpret_cast<uintptr_t>(p.ln_y) & 15) == 0;
     return ok;
 }
 

@@ -44,6 +44,9 @@ struct TileCfg {
     static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 };
 
+// 32-row slabs of one group as the fused LayerNorm counts them: every tile row, also past M, has its counters
+__host__ __device__ constexpr int ln_slabs(int m) { return (m + 2 * BM - 1) / (2 * BM) * (2 * BM / 32); }
+
 struct KernelArgs {
     GemmShape shape;
     EpiParams epi;
@@ -186,6 +189,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         const int quarter = warp & 3;          // TMEM lanes this warp may read
         const int half = (warp - 2) >> 2;      // which half of the tile's columns it drains
         constexpr int CHUNKS = BN / 32;        // 32-column chunks of the tile: `half` takes every second one
+        const bool ln = ka.epi.ln_out != nullptr;
         int acc = 0;
         uint32_t acc_phase = 0;
         bool ok = true;
@@ -198,6 +202,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const int row = m_blk * BM + quarter * 32 + lane;
             const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
                                    static_cast<uint32_t>(acc * BN);
+            RowStats rs{0.f, 0.f, 0.f};
 #pragma unroll 1
             for (int c = half; c < CHUNKS; c += 2) {
                 const int col0 = n_blk * BN + c * 32;
@@ -205,13 +210,48 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 uint32_t r[32];
                 tmem_ld_32x32(t_row + static_cast<uint32_t>(c * 32), r);
                 tmem_ld_wait();
+                const int ncols = min(32, ka.shape.n_out - col0);
                 if (row < ka.shape.m) {
                     float v[32];
 #pragma unroll
                     for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
-                    const int ncols = min(32, ka.shape.n_out - col0);
-                    epilogue_chunk(ka.epi, g, row, col0, ncols, v);
+                    if (ln) {
+                        epilogue_chunk_ln(ka.epi, g, row, col0, ncols, v);
+                        stats_add_chunk(rs, v, ncols);
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(v[i]);
+                    } else {
+                        epilogue_chunk(ka.epi, g, row, col0, ncols, v);
+                    }
                 }
+                if (ln) tmem_st_32x32(t_row + static_cast<uint32_t>(c * 32), r);   // the row the LayerNorm sees
+            }
+            if (ln) {
+                // the row's other columns are other CTAs' tiles: leave this part's statistics, wait for the rest
+                tmem_st_wait();
+                const int n_parts = ka.epi.ln_n_parts;
+                float4 *parts = ka.epi.ln_parts + ((long long)g * ka.shape.m + row) * n_parts;
+                if (row < ka.shape.m) parts[n_blk * 2 + half] = make_float4(rs.mean, rs.m2, rs.cnt, 0.f);
+                uint32_t *cnt = ka.epi.ln_cnt + ((long long)g * ln_slabs(ka.shape.m) + m_blk * (BM / 32) + quarter) * 2;
+                ok = ln_arrive_and_wait(cnt, n_parts, lane, abort_flag);
+                if (!ok) break;
+                float mean = 0.f, rstd = 0.f;
+                if (row < ka.shape.m) ln_row_stats(parts, n_parts, ka.epi.ln_eps, mean, rstd);
+#pragma unroll 1
+                for (int c = half; c < CHUNKS; c += 2) {
+                    const int col0 = n_blk * BN + c * 32;
+                    if (col0 >= ka.shape.n_out) break;
+                    uint32_t r[32];
+                    tmem_ld_32x32(t_row + static_cast<uint32_t>(c * 32), r);
+                    tmem_ld_wait();
+                    if (row < ka.shape.m) {
+                        float z[32];
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) z[i] = __uint_as_float(r[i]);
+                        ln_store_chunk(ka.epi, g, row, col0, min(32, ka.shape.n_out - col0), z, mean, rstd);
+                    }
+                }
+                ln_depart(cnt, n_parts, lane);
             }
             tc_fence_before_sync();
             __syncwarp();
@@ -399,6 +439,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         float *stage = reinterpret_cast<float *>(smem + Cfg::STAGES * Cfg::STAGE_BYTES + 256) +
                        (warp - 2) * EPI_STAGE_FLOATS;
         const bool staged = epilogue_f32_stageable(ka.epi);
+        const bool ln = ka.epi.ln_out != nullptr;
         int acc = 0;
         uint32_t acc_phase = 0;
         bool ok = true;
@@ -412,6 +453,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             const int row = row_base + lane;
             const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
                                    static_cast<uint32_t>(acc * BN2);
+            RowStats rs{0.f, 0.f, 0.f};
 #pragma unroll 1
             for (int cc = 0; cc < CHUNKS; ++cc) {
                 const int c = half * CHUNKS + cc;
@@ -420,20 +462,60 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 uint32_t r[32];
                 tmem_ld_32x32(t_row + static_cast<uint32_t>(c * 32), r);
                 tmem_ld_wait();
+                const int ncols = min(32, ka.shape.n_out - col0);
                 if (staged && col0 + 32 <= ka.shape.n_out) {
                     // coalesced path: the whole warp takes part, rows past M are masked inside
                     float v[32];
 #pragma unroll
                     for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
                     if (ka.epi.bias) add_bias_chunk(ka.epi.bias + g * ka.epi.bias_gstride + col0, v, 32);
-                    epilogue_f32_staged(ka.epi, g, row_base, ka.shape.m, col0, v, stage, lane);
+                    epilogue_f32_staged(ka.epi, g, row_base, ka.shape.m, col0, v, stage, lane, ln);
+                    if (ln) {
+                        if (row < ka.shape.m) stats_add_chunk(rs, v, 32);
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(v[i]);
+                    }
                 } else if (row < ka.shape.m) {
                     float v[32];
 #pragma unroll
                     for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
-                    const int ncols = min(32, ka.shape.n_out - col0);
-                    epilogue_chunk(ka.epi, g, row, col0, ncols, v);
+                    if (ln) {
+                        epilogue_chunk_ln(ka.epi, g, row, col0, ncols, v);
+                        stats_add_chunk(rs, v, ncols);
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(v[i]);
+                    } else {
+                        epilogue_chunk(ka.epi, g, row, col0, ncols, v);
+                    }
                 }
+                if (ln) tmem_st_32x32(t_row + static_cast<uint32_t>(c * 32), r);   // the row the LayerNorm sees
+            }
+            if (ln) {
+                tmem_st_wait();
+                const int n_parts = ka.epi.ln_n_parts;
+                float4 *parts = ka.epi.ln_parts + ((long long)g * ka.shape.m + row) * n_parts;
+                if (row < ka.shape.m) parts[n_blk * 2 + half] = make_float4(rs.mean, rs.m2, rs.cnt, 0.f);
+                uint32_t *cnt = ka.epi.ln_cnt + ((long long)g * ln_slabs(ka.shape.m) + row_base / 32) * 2;
+                ok = ln_arrive_and_wait(cnt, n_parts, lane, abort_flag);
+                if (!ok) break;
+                float mean = 0.f, rstd = 0.f;
+                if (row < ka.shape.m) ln_row_stats(parts, n_parts, ka.epi.ln_eps, mean, rstd);
+#pragma unroll 1
+                for (int cc = 0; cc < CHUNKS; ++cc) {
+                    const int c = half * CHUNKS + cc;
+                    const int col0 = n_blk * BN2 + c * 32;
+                    if (col0 >= ka.shape.n_out) break;
+                    uint32_t r[32];
+                    tmem_ld_32x32(t_row + static_cast<uint32_t>(c * 32), r);
+                    tmem_ld_wait();
+                    if (row < ka.shape.m) {
+                        float z[32];
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) z[i] = __uint_as_float(r[i]);
+                        ln_store_chunk(ka.epi, g, row, col0, min(32, ka.shape.n_out - col0), z, mean, rstd);
+                    }
+                }
+                ln_depart(cnt, n_parts, lane);
             }
             tc_fence_before_sync();
             __syncwarp();
@@ -487,7 +569,10 @@ int launch_pair(const CUtensorMap &tmA, const CUtensorMap &tmB, const KernelArgs
     const int max_clusters = max_clusters_of[dev].load();
     const long long tiles = (long long)((ka.shape.m + 2 * BM - 1) / (2 * BM)) * ka.tiles_n;
     const long long units = ka.group_serial ? tiles : tiles * ka.shape.groups;
-    const int clusters = static_cast<int>(units < max_clusters ? units : max_clusters);
+    int clusters = static_cast<int>(units < max_clusters ? units : max_clusters);
+    // LayerNorm behind the epilogue: the N tiles of a row block wait for each other, so a round of clusters must
+    // hold whole row blocks (a block split over two rounds stalls its first part for a whole tile, every round)
+    if (ka.epi.ln_out && clusters > ka.tiles_n) clusters -= clusters % ka.tiles_n;
     return cuda_check(launch_pdl(gemm_tc_pair_kernel, dim3(2 * clusters), dim3(NUM_THREADS), Cfg::SMEM_BYTES, stream, tmA, tmB, ka),
                       "gemm pair: launch");
 }
@@ -582,12 +667,24 @@ int launch_gemm_tc(const GemmOperands &op, const GemmShape &s, const EpiParams &
     ka.b_g0 = b_g0;
     ka.group_serial = epi.kind == KRAKEN_EPI_RESID_SUM ? 1 : 0;
     ka.n_fastest = (ka.group_serial && ka.tiles_n <= ka.tiles_m) ? 1 : 0;
+    if (epi.ln_out) {
+        // LayerNorm behind the epilogue: the N tiles of a row block wait for each other, so they must be in
+        // flight together: N tiles run fastest (neighbouring CTAs take one row block), and a row block may not be
+        // wider than the grid
+        if (epi.kind != KRAKEN_EPI_RESID_F32 && epi.kind != KRAKEN_EPI_RESID_SUM) return KRAKEN_EINVAL;
+        if (!epi.ln_gamma || !epi.ln_parts || !epi.ln_cnt || !epi.resid || !epi.out_f32) return KRAKEN_EINVAL;
+        ka.epi.ln_n_parts = 2 * ka.tiles_n;
+        ka.n_fastest = 1;
+        const int sms_ = sm_count() > 0 ? sm_count() : 148;
+        if (ka.tiles_n > (bn == GEMM_TILE_PAIR ? sms_ / 2 : sms_)) return KRAKEN_EUNSUPPORTED;
+    }
     ka.status = d_status;
     if (bn == GEMM_TILE_PAIR) return launch_pair(*tmA, *tmB, ka, stream);
     const long long tiles = (long long)ka.tiles_m * ka.tiles_n;
     const long long units = ka.group_serial ? tiles : tiles * s.groups;
     const int sms = sm_count() > 0 ? sm_count() : 148;
-    const int grid = static_cast<int>(units < sms ? units : sms);
+    int grid = static_cast<int>(units < sms ? units : sms);
+    if (epi.ln_out && grid > ka.tiles_n) grid -= grid % ka.tiles_n;   // whole row blocks per round, as for the pairs
     switch (bn) {
         case 256: return launch_bn<256>(*tmA, *tmB, ka, grid, stream);
         case 224: return launch_bn<224>(*tmA, *tmB, ka, grid, stream);
@@ -600,5 +697,12 @@ int launch_gemm_tc(const GemmOperands &op, const GemmShape &s, const EpiParams &
         default: return KRAKEN_EINVAL;
     }
 }
+
+size_t gemm_ln_parts_bytes(int groups, int m, int n_out, int bn) {
+    const int cols = bn == GEMM_TILE_PAIR ? BN2 : bn;
+    return (size_t)groups * m * 2 * ((n_out + cols - 1) / cols) * sizeof(float4);
+}
+
+size_t gemm_ln_cnt_bytes(int groups, int m) { return (size_t)groups * ln_slabs(m) * 2 * sizeof(uint32_t); }
 
 }  // namespace kr

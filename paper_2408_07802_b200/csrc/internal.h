@@ -36,7 +36,28 @@ struct EpiParams {
     const int *pos0_dev;
     // packed (ragged) prefill: row r belongs to sequence row_seq[r] at position row_pos[r]
     const int *row_seq, *row_pos;
+    // LayerNorm of the finished rows in the same kernel (RESID_F32 and RESID_SUM only; ln_out != NULL turns it on):
+    //   ln_out[g] = LN(out_f32[g] + ln_y; gamma[g], beta[g])   over the whole row of n_out columns.
+    // A row is spread over the N tiles of its row block, i.e. over several CTAs, so every epilogue warp leaves
+    // the (mean, M2, count) of its part of each row in ln_parts, counts itself in ln_cnt, waits (bounded) for the
+    // other parts of its 32 rows and then normalises the values it kept in tensor memory.
+    uint16_t *ln_out;
+    long long ln_out_gstride;
+    int ln_ld_out;
+    const uint16_t *ln_gamma, *ln_beta;   // [G][n_out]; beta may be NULL
+    long long ln_gb_gstride;
+    const float *ln_y;                    // [M, n_out] added before the statistics, or NULL
+    int ln_ld_y;
+    float ln_eps;
+    float4 *ln_parts;                     // [G][M][ln_n_parts]
+    uint32_t *ln_cnt;                     // [G][ceil(M / 32)][2]: arrivals, departures; zero between launches
+    int ln_n_parts;                       // 2 * N tiles, filled in by the launcher
 };
+
+// Scratch of the fused LayerNorm for a launch of `groups` x `m` rows whose rows are `n_out` wide and cut into
+// tiles of `bn` columns (GEMM_TILE_PAIR: 256): bytes of the parts array and of the counters.
+size_t gemm_ln_parts_bytes(int groups, int m, int n_out, int bn);
+size_t gemm_ln_cnt_bytes(int groups, int m);
 
 struct GemmShape {
     int groups, m, n_out, k;

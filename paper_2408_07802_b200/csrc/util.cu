@@ -101,7 +101,7 @@ std::atomic<int> g_tuning[KRAKEN_TUNE_COUNT];
 int tuning(int key) { return key >= 0 && key < KRAKEN_TUNE_COUNT ? g_tuning[key].load(std::memory_order_relaxed) : 0; }
 
 int set_tuning(int key, int value) {
-    if (key < 0 || key >= KRAKEN_TUNE_COUNT || value < 0 || value > 2) return KRAKEN_EINVAL;
+    if (key < 0 || key >= KRAKEN_TUNE_COUNT || value < 0 || value > 3) return KRAKEN_EINVAL;
     g_tuning[key].store(value, std::memory_order_relaxed);
     return KRAKEN_OK;
 }

@@ -47,7 +47,8 @@ def test_query_sizes_arithmetic(L):
         assert kv == s.n_layer * s.n_branch * 2 * s.batch * s.max_pos * s.kv_heads * s.head_dim * 2
         T = s.batch * s.max_pos
         floor = T * s.d_model * 4 * (2 + 2 * s.n_branch) + T * s.n_branch * 2 * (3 * s.d_model + s.d_ff)
-        assert floor <= scratch < floor * 1.05 + (1 << 22)
+        # small fixed parts on top: staging, split-KV partials, and the 4 MiB floor of the fused LayerNorm's statistics
+        assert floor <= scratch < floor * 1.05 + (1 << 23)
     # grouped-query attention shrinks the cache by the group size (the mitigation of Sec. 4.2)
     full = kr.query_sizes(kr.make_config(ki.CONFIGS["C4"]))[0]
     assert kr.query_sizes(kr.make_config(ki.CONFIGS["C4-gqa4"]))[0] * 4 == full

@@ -760,3 +760,40 @@ def test_c4_full_size_prefill_prefix_parity_and_decode_consistency(name):
     assert np.abs(v_after - v_ref).max() <= 2.0 ** -6 * np.abs(v_ref).max()
     assert (v_after == v_ref).mean() > 0.9
     m.close()
+
+
+@pytest.mark.parametrize("name", ["C0", "K0-72", "C0-gqa", "S0", "P0"])
+@pytest.mark.parametrize("mode", [2, 3])
+def test_layernorm_behind_the_gemm_epilogues_whole_model(name, mode):
+    """Algorithm 1's two LayerNorm lines inside the kernels that finish their input rows (mode 2: LN-2 behind the
+    attention output projection and the next layer's LN-1 behind the down-projection; mode 3: the latter only):
+    every position against the oracle, then a decode step continuing from the cache; in mode 2 only the first
+    layer's LN-1 is left as a LayerNorm launch."""
+    s = ki.CONFIGS[name]
+    with kr.tuning(kr.TUNE_LN_FUSION, mode):
+        m, w = build(s)
+        wb = host_bits(w)
+        l0 = s.seqlen - 1            # leaves room in the cache for the decode step
+        tok = ki.uniform_tokens(7, s.vocab, s.batch, l0 + 1, DEV)
+        first = tok[:, :l0].contiguous()
+        m.profile_read()
+        got_all = m.prefill_all_logits(first).cpu().numpy()
+        _, launches = m.profile_read()
+        for b in range(s.batch):
+            ids = tok[b, :l0].cpu().numpy()
+            ref32, _ = oracle_all_logits(s, wb, ids, False)
+            refbf, _ = oracle_all_logits(s, wb, ids, True)
+            check_parity(got_all[b], ref32, refbf, f"{name} LayerNorm mode {mode} seq {b} all positions")
+        if mode == 2 and not s.parallel_ffn and s.batch * l0 > 32:
+            # embed .. tail categories: LayerNorm launches = the first layer's LN-1 (+ the cross-branch sum passes
+            # of short prompts, which are counted with the LayerNorms)
+            assert launches["layernorm"] <= 1 + s.n_layer, launches
+        got = m.decode_step(tok[:, l0].contiguous()).cpu().numpy()
+        for b in range(s.batch):
+            orc = oracle.Oracle(s, wb, bf16_store=False)
+            orc.prefill(tok[b, :l0].cpu().numpy())
+            ref = orc.decode_step(int(tok[b, l0]))
+            rel, mx = logits_metrics(got[b], ref)
+            assert rel <= REL_L2_MAX and mx <= MAX_ABS_MAX, (b, rel, mx)
+        assert m.device_status() == 0
+        m.close()

@@ -263,6 +263,100 @@ def test_gemm_qkv_scatter_is_index_exact(hd, H, Hkv):
                     assert np.all(got_c[g, which, b, h, pos0 + seqlen:] == -7.0)
 
 
+@pytest.mark.parametrize("G,M,Nout,K,epi,n_tile,with_y", [
+    (2, 300, 768, 256, "resid", 64, True),        # twelve N tiles per row block, ragged last M tile
+    (3, 700, 1024, 128, "sum", 512, False),       # CTA pairs, cross-branch sum and LayerNorm in one epilogue
+    (1, 129, 520, 64, "resid", 256, True),        # ragged last N tile (8 columns), one row in the second M tile
+    (2, 64, 96, 64, "resid", 32, False),          # one 32-column chunk per tile: half of the epilogue warps hold nothing
+    (2, 512, 768, 192, "sum", 0, True),           # the library's own tile choice
+    (4, 1024, 512, 64, "resid", 32, True),        # 512 tiles on 148 CTAs: row blocks straddle the rounds
+    (4, 4096, 1024, 64, "sum", 512, False),       # 256 pair tiles on 74 pairs: the same for CTA pairs and the sum
+])
+def test_gemm_with_layernorm_behind_the_epilogue(G, M, Nout, K, epi, n_tile, with_y):
+    """x = LN(out + y) in the kernel that produces `out` (Algorithm 1's two LayerNorm lines): the fp32 output and
+    the cross-branch sum equal the oracle's linear step as without the LayerNorm, and the 16-bit LayerNorm output
+    is within one bf16 step of the oracle's LayerNorm of those very rows.  Two launches in a row share the scratch."""
+    kind = kr.EPI_RESID_F32 if epi == "resid" else kr.EPI_RESID_SUM
+    a = ki.normal_bf16(5, 60, (G, M, K), 1.0, DEV)
+    w = ki.normal_bf16(5, 61, (G, Nout, K), 1.0 / np.sqrt(K), DEV)
+    bias = ki.normal_bf16(5, 62, (G, Nout), 0.5, DEV)
+    resid = (ki.normal_bf16(5, 63, (G, M, Nout), 1.0, DEV).float() * 1.37 + 0.4).contiguous()
+    y = (ki.normal_bf16(5, 64, (M, Nout), 2.0, DEV).float() - 0.7).contiguous() if with_y else None
+    gamma = (1 + ki.normal_bf16(5, 65, (G, Nout), 0.3, DEV).float()).to(torch.bfloat16)
+    beta = ki.normal_bf16(5, 66, (G, Nout), 0.3, DEV)
+    args = kr.GemmArgs()
+    args.a, args.a_gstride, args.lda = a.data_ptr(), M * K, K
+    args.w, args.w_gstride, args.ldw = w.data_ptr(), Nout * K, K
+    args.bias, args.bias_gstride = bias.data_ptr(), Nout
+    args.groups, args.m, args.n_out, args.k = G, M, Nout, K
+    args.epilogue, args.n_tile = kind, n_tile
+    args.resid, args.resid_gstride, args.ld_resid = resid.data_ptr(), M * Nout, Nout
+    nbytes = kr.gemm_ln_scratch_bytes(G, M, Nout, K, n_tile)
+    scratch = torch.zeros(nbytes, dtype=torch.uint8, device=DEV)       # zeroed once, shared by both launches
+    status = torch.zeros(1, dtype=torch.int32, device=DEV)
+    for rep in range(2):
+        out = torch.full((G, M, Nout), float("nan"), dtype=torch.float32, device=DEV)
+        ssum = torch.full((M, Nout), float("nan"), dtype=torch.float32, device=DEV)
+        ln_out = torch.full((G, M, Nout), float("nan"), dtype=torch.bfloat16, device=DEV)
+        args.out_f32, args.out_f32_gstride, args.ld_out_f32 = out.data_ptr(), M * Nout, Nout
+        if kind == kr.EPI_RESID_SUM:
+            args.sum, args.ld_sum = ssum.data_ptr(), Nout
+        ln = kr.GemmLnArgs()
+        ln.ln_out, ln.ln_out_gstride, ln.ld_ln_out = ln_out.data_ptr(), M * Nout, Nout
+        ln.gamma, ln.beta, ln.gb_gstride = gamma.data_ptr(), beta.data_ptr() if rep == 0 else None, Nout
+        ln.y, ln.ld_y = (y.data_ptr() if with_y else None), Nout
+        ln.eps = 1e-5
+        ln.d_scratch, ln.scratch_bytes = scratch.data_ptr(), nbytes
+        kr.op_grouped_gemm_ln(args, ln, status)
+        torch.cuda.synchronize()
+        assert int(status.item()) == 0
+        assert int(scratch[:G * ((M + 255) // 256) * 8 * 8].view(torch.int32).abs().sum().item()) == 0   # counters back at zero
+        got = out.cpu().numpy()
+        for g in ([0, G - 1] if rep == 0 else [G // 2]):
+            ref = oracle.linear(a[g].float().cpu().numpy(), bits(w[g]), bits(bias[g])) + resid[g].cpu().numpy()
+            assert np.abs(got[g] - ref).max() < 3e-4, (g, np.abs(got[g] - ref).max())
+            want = oracle.layernorm(got[g], y.cpu().numpy() if with_y else None, bits(gamma[g]),
+                                    bits(beta[g]) if rep == 0 else None)
+            ok, worst = bf16_ulp_close(ln_out[g].float().cpu().numpy(), want, ulps=1.0, atol=1e-5)
+            assert ok, (rep, g, worst)
+        if kind == kr.EPI_RESID_SUM:
+            assert np.abs(ssum.cpu().numpy() - got.astype(np.float64).sum(0)).max() < 1e-4 * G
+
+
+def test_gemm_with_layernorm_rejects_other_epilogues_and_small_scratch():
+    G, M, Nout, K = 1, 64, 64, 64
+    a = torch.zeros(G, M, K, dtype=torch.bfloat16, device=DEV)
+    w = torch.zeros(G, Nout, K, dtype=torch.bfloat16, device=DEV)
+    out = torch.zeros(G, M, Nout, dtype=torch.float32, device=DEV)
+    lo = torch.zeros(G, M, Nout, dtype=torch.bfloat16, device=DEV)
+    gamma = torch.ones(G, Nout, dtype=torch.bfloat16, device=DEV)
+    args = kr.GemmArgs()
+    args.a, args.a_gstride, args.lda = a.data_ptr(), M * K, K
+    args.w, args.w_gstride, args.ldw = w.data_ptr(), Nout * K, K
+    args.groups, args.m, args.n_out, args.k = G, M, Nout, K
+    args.out_f32, args.out_f32_gstride, args.ld_out_f32 = out.data_ptr(), M * Nout, Nout
+    args.resid, args.resid_gstride, args.ld_resid = out.data_ptr(), M * Nout, Nout
+    args.n_tile = 64
+    nbytes = kr.gemm_ln_scratch_bytes(G, M, Nout, K, 64)
+    scratch = torch.zeros(nbytes, dtype=torch.uint8, device=DEV)
+    ln = kr.GemmLnArgs()
+    ln.ln_out, ln.ln_out_gstride, ln.ld_ln_out = lo.data_ptr(), M * Nout, Nout
+    ln.gamma, ln.gb_gstride, ln.eps = gamma.data_ptr(), Nout, 1e-5
+    ln.d_scratch, ln.scratch_bytes = scratch.data_ptr(), nbytes
+    args.epilogue = kr.EPI_F32
+    with pytest.raises(kr.KrakenError) as e:
+        kr.op_grouped_gemm_ln(args, ln)
+    assert e.value.status == kr.EINVAL
+    args.epilogue = kr.EPI_RESID_F32
+    ln.scratch_bytes = nbytes - 16
+    with pytest.raises(kr.KrakenError) as e:
+        kr.op_grouped_gemm_ln(args, ln)
+    assert e.value.status == kr.ECAPACITY
+    ln.scratch_bytes = nbytes
+    kr.op_grouped_gemm_ln(args, ln)
+    torch.cuda.synchronize()
+
+
 def test_gemm_rejects_unaligned():
     a = torch.zeros(1, 8, 68, dtype=torch.bfloat16, device=DEV)
     args = kr.GemmArgs()
@@ -342,6 +436,19 @@ def test_bounded_wait_runs_out_and_the_context_stays_usable():
     ref = oracle.layernorm(a[0].cpu().numpy(), None, bits(gamma[0]), None)
     ok, worst = bf16_ulp_close(out[0].float().cpu().numpy(), ref, ulps=1.0, atol=1e-5)
     assert ok, worst
+
+
+def test_tensor_core_issue_rate_one_and_two_issuing_threads():
+    """The probe behind the attention kernel's roofline argument: 128 x 128 x 16 products issued by one thread
+    cost clearly more than their 64 tensor cycles, 128 x 256 x 16 products run at the tensor rate (128), and two
+    issuing threads in different warps reach the tensor rate with the small products too."""
+    one = {f: kr.mma_issue_rate(f, 1) for f in range(7)}
+    two = {f: kr.mma_issue_rate(f, 2) for f in (0, 1, 2, 3)}
+    print("[probe] cycles per product, one issuing thread:", {k: round(v, 1) for k, v in one.items()},
+          "two issuing threads:", {k: round(v, 1) for k, v in two.items()})
+    assert 126 <= one[6] <= 134
+    assert all(72 <= one[f] <= 130 for f in (0, 1, 2, 3, 4, 5)), one
+    assert all(62 <= two[f] <= 70 for f in two), two
 
 
 @pytest.mark.parametrize("G,B,H,hd,seqlen", [(4, 1, 16, 64, 768),     # one round of couples, a middle pair alone
