@@ -57,13 +57,48 @@ class TorchDistGroup:
         handle.wait()
 
 
-class BranchParallelPrefill:
-    """One rank of a branch-parallel Kraken prefill."""
+class _Clock:
+    """Times the pieces of one rank: CUDA events on the current stream for device tensors, wall clock otherwise."""
 
-    def __init__(self, engine, group, n_layer: int):
+    def __init__(self, on_device: bool):
+        self.on_device = on_device
+        self.marks = []
+
+    def mark(self, label: str):
+        if self.on_device:
+            ev = torch.cuda.Event(enable_timing=True)
+            ev.record()
+            self.marks.append((label, ev))
+        else:
+            import time
+            self.marks.append((label, time.perf_counter()))
+
+    def spans(self) -> List[tuple]:
+        """[(label of the piece that ended at the mark, milliseconds)] between consecutive marks."""
+        if self.on_device:
+            torch.cuda.synchronize()
+        out = []
+        for (_, a), (label, b) in zip(self.marks, self.marks[1:]):
+            out.append((label, a.elapsed_time(b) if self.on_device else (b - a) * 1e3))
+        return out
+
+
+class BranchParallelPrefill:
+    """One rank of a branch-parallel Kraken prefill.
+
+    overlap=False waits for every all-reduce right where it is started (the blocking placement of a standard
+    tensor-parallel layer): the difference to the default shows what the overlap hides.
+    timing=True fills `last_timing` after every run: per layer the milliseconds of the attention half, of the
+    time this rank's stream then still had to wait for the previous layer's all-reduce (what the attention half
+    did NOT hide), and of the FFN half; plus the W_concat part with its blocking reduction and the head."""
+
+    def __init__(self, engine, group, n_layer: int, overlap: bool = True, timing: bool = False):
         self.engine = engine
         self.group = group
         self.n_layer = n_layer
+        self.overlap = overlap
+        self.timing = timing
+        self.last_timing = None
 
     def prefill(self, tokens: torch.Tensor) -> torch.Tensor:
         self.engine.stage_begin(tokens)
@@ -77,21 +112,43 @@ class BranchParallelPrefill:
     def _run(self) -> torch.Tensor:
         e, g = self.engine, self.group
         x0, local_sum = e.stage_buffers()
+        clock = _Clock(local_sum.is_cuda) if self.timing else None
+        mark = clock.mark if clock else (lambda label: None)
         bufs = [torch.empty_like(local_sum), torch.empty_like(local_sum)]
         y, pending = x0, None                       # layer 1: the AllReduce is the identity (Algorithm 1)
+        mark("start")
         for layer in range(self.n_layer):
             e.stage_attention(layer)                # overlaps the all-reduce started after the previous layer
+            mark("attention")
             if pending is not None:
                 g.wait(pending)
                 pending = None
+            mark("exposed_wait")
             e.stage_ffn(layer, y)
             if layer + 1 < self.n_layer:
                 y = bufs[layer & 1]
                 y.copy_(local_sum)                  # the next stage_ffn overwrites local_sum
                 pending = g.all_reduce_start(y)
+                if not self.overlap:
+                    g.wait(pending)
+                    pending = None
+            mark("ffn")
         z = e.stage_concat()
         g.wait(g.all_reduce_start(z))               # nothing left to overlap: the logits need the full z
-        return e.stage_head(z)
+        mark("concat")
+        logits = e.stage_head(z)
+        mark("head")
+        if clock:
+            per = {"attention": [], "exposed_wait": [], "ffn": []}
+            rest = {}
+            for label, ms in clock.spans():
+                if label in per:
+                    per[label].append(ms)
+                else:
+                    rest[label] = ms
+            self.last_timing = {"per_layer_ms": per, "concat_ms": rest.get("concat"), "head_ms": rest.get("head"),
+                                "total_ms": sum(ms for _, ms in clock.spans()), "overlap": self.overlap}
+        return logits
 
 
 def lockstep_prefill(engines, n_layer: int, tokens: torch.Tensor, decode: bool = False) -> List[torch.Tensor]:

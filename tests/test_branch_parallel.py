@@ -97,8 +97,14 @@ def _worker(rank, world, port, out):
     mine = bp.slice_weights(w, SHAPE.n_branch, first, count, with_concat_bias=rank == 0)
     eng = OracleStageEngine(SHAPE, mine)
     tok = ki.uniform_tokens(8, SHAPE.vocab, 1, SHAPE.seqlen)
-    logits = bp.BranchParallelPrefill(eng, bp.TorchDistGroup(), SHAPE.n_layer).prefill(tok)
+    runner = bp.BranchParallelPrefill(eng, bp.TorchDistGroup(), SHAPE.n_layer, timing=True)
+    logits = runner.prefill(tok)
     out[rank] = logits.numpy()
+    t = runner.last_timing
+    assert len(t["per_layer_ms"]["attention"]) == SHAPE.n_layer and t["total_ms"] > 0 and t["overlap"]
+    # the blocking placement of the all-reduce gives the same logits (same sums in the same order)
+    blocking = bp.BranchParallelPrefill(eng, bp.TorchDistGroup(), SHAPE.n_layer, overlap=False).prefill(tok)
+    assert np.array_equal(blocking.numpy(), out[rank])
     dist.barrier()
     dist.destroy_process_group()
 
@@ -205,7 +211,10 @@ def test_one_nccl_rank_through_the_collective_path_equals_prefill():
         m = kr.KrakenModel(kr.make_config(s), w, dev)
         tok = ki.uniform_tokens(2, s.vocab, s.batch, s.seqlen, dev)
         ref = m.prefill(tok).clone()
-        got = bp.BranchParallelPrefill(m, bp.TorchDistGroup(), s.n_layer).prefill(tok)
+        runner = bp.BranchParallelPrefill(m, bp.TorchDistGroup(), s.n_layer, timing=True)
+        got = runner.prefill(tok)
+        t = runner.last_timing
+        assert len(t["per_layer_ms"]["ffn"]) == s.n_layer and all(v >= 0 for v in t["per_layer_ms"]["exposed_wait"])
         torch.cuda.synchronize()
         err = (got - ref).abs().max().item()
         assert err <= 2e-3 * max(1.0, ref.abs().max().item()), err
