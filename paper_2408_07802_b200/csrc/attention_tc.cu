@@ -9,9 +9,13 @@
 //               per step; 128-byte swizzle; rows past the keys written so far are out of bounds = zeros);
 //   warp 1      MMA issuer, per K/V tile j and query tile w:
 //                   S_w = Q_w K_j^T          both operands K-major in shared memory -> TMEM
-//                   O_w (+)= P_w V_j         P_w read from TMEM (it overwrites S_w in place as packed
-//                                            bf16), V_j MN-major in shared memory, O_w accumulates in TMEM
-//               issued in the order PV_0(j), QK_0(j+1), PV_1(j), QK_1(j+1);
+//                   O_w (+)= P_w V_j         P_w read from TMEM (packed 16-bit), V_j MN-major in shared memory,
+//                                            O_w accumulates in TMEM
+//               With 128-wide O tensor memory is full and P_w overwrites S_w in place: the products are issued in
+//               the order PV_0(j), QK_0(j+1), PV_1(j), QK_1(j+1).  With head dims up to 64 P_w has columns of its
+//               own and the order is QK_0(j+1), QK_1(j+1) as soon as the softmax warps hold S_w(j) in registers,
+//               then PV_0(j), PV_1(j): the softmax of a query tile never waits for its next scores
+//               (64 heads x 1024 tokens 34.9 -> 31.2 us, 16 x 64 heads x 2048 tokens 1080 -> 1006 us);
 //   warps 2-5   softmax of query tile 0, warps 6-9 of query tile 1: one thread per query row (TMEM
 //               lane = row: row max and row sum need no shuffles).  The whole score row is pulled into
 //               registers with tcgen05.ld, masked on diagonal tiles, exponentiated with the scale folded
@@ -22,7 +26,10 @@
 // Every role walks a list of work items with running barrier phases, so a CTA can take several items
 // without draining its pipeline: with enough work each SM gets one CTA and a fixed list of couples of items
 // of equal total length (atc_next), else the grid has one CTA per item (see launch()).
-// TMEM: S/P of tile w at column 128 w, O of tile w at 256 + 128 w.  All waits are time-bounded.
+// TMEM: head dim 128: S/P of tile w at column 128 w, O of tile w at 256 + 128 w; head dim 64: S at 128 w, P at
+// 256 + 64 w, O at 384 + 64 w.  All waits are time-bounded.  Exponentials as a polynomial on the FMA pipe (a quarter
+// or half of them) measured slower in both layouts (1241 / 1276 against 1006 us): the softmax warps are bound by
+// instruction issue, not by the exp unit.
 #include <math.h>
 
 #include "internal.h"
@@ -36,10 +43,6 @@ constexpr int TQ = 128;   // query rows per tile (two tiles per CTA)
 constexpr int TK = 128;   // keys per tile
 constexpr int ATC_THREADS = 320;
 constexpr float RESCALE_LOG2 = 8.0f;
-// Measured: the softmax warps are bound by instruction issue, not by the special-function unit, so
-// moving exponentials to the FMA pipe costs time (0.39 vs 0.35 ms at 4 x 2048 x 16 heads x 128).
-constexpr bool POLY_EXP2 = false;
-
 struct AttnTcArgs {
     int groups, batch, seqlen, pos0, n_head;
     int n_kv_head, kv_rep;   // key/value heads in the cache; query heads per key/value head
@@ -93,43 +96,6 @@ __device__ __forceinline__ void fma2(float &x0, float &x1, float a, float b) {
         : "f"(a), "f"(b));
 }
 
-// 2^x for two values on the FMA pipe (no special-function unit): x = n + f with n = round(x),
-// f in [-0.5, 0.5]; 2^f by a cubic (relative error 1e-4, far below a bf16 step); n goes straight into
-// the exponent bits.  Inputs below -126 (masked scores) come out as 2^-126 ~ 0.
-__device__ __forceinline__ void exp2_poly_pair(float &x0, float &x1) {
-    uint32_t r0, r1;
-    asm("{\n"
-        ".reg .b64 x, t, f, p, c;\n"
-        ".reg .b32 t0, t1, p0, p1, lo, hi;\n"
-        "max.f32 lo, %2, 0fC2FC0000;\n"            // -126
-        "max.f32 hi, %3, 0fC2FC0000;\n"
-        "mov.b64 x, {lo, hi};\n"
-        "mov.b64 c, {0f4B400000, 0f4B400000};\n"   // 1.5 * 2^23: adding it rounds to an integer
-        "add.rn.f32x2 t, x, c;\n"
-        "mov.b64 c, {0fCB400000, 0fCB400000};\n"
-        "add.rn.f32x2 f, t, c;\n"                  // n = round(x)
-        "mov.b64 c, {0fBF800000, 0fBF800000};\n"
-        "fma.rn.f32x2 f, f, c, x;\n"               // f = x - n
-        "mov.b64 p, {0f3D650E81, 0f3D650E81};\n"   // 0.055922035
-        "mov.b64 c, {0f3E7876A4, 0f3E7876A4};\n"   // 0.24264008
-        "fma.rn.f32x2 p, p, f, c;\n"
-        "mov.b64 c, {0f3F317061, 0f3F317061};\n"   // 0.69312102
-        "fma.rn.f32x2 p, p, f, c;\n"
-        "mov.b64 c, {0f3F7FFB0D, 0f3F7FFB0D};\n"   // 0.99992448
-        "fma.rn.f32x2 p, p, f, c;\n"
-        "mov.b64 {t0, t1}, t;\n"
-        "mov.b64 {p0, p1}, p;\n"
-        "shl.b32 t0, t0, 23;\n"
-        "shl.b32 t1, t1, 23;\n"
-        "add.s32 %0, p0, t0;\n"
-        "add.s32 %1, p1, t1;\n"
-        "}\n"
-        : "=r"(r0), "=r"(r1)
-        : "f"(x0), "f"(x1));
-    x0 = __uint_as_float(r0);
-    x1 = __uint_as_float(r1);
-}
-
 template <int HD>
 struct AtcCfg {
     static constexpr int HALVES = HD / 64;                 // 64-column (128-byte) pieces of the head dim
@@ -139,8 +105,16 @@ struct AtcCfg {
     static constexpr int STAGES = 2;
     static constexpr int BUNDLE_BYTES = 2 * KV_BYTES;      // a ring stage: V_j, then K_{j+1}
     static constexpr int SMEM_BYTES = 2 * Q_BYTES + STAGES * BUNDLE_BYTES + 1024 + 256;
-    static constexpr int S_COL0 = 0;                       // S / P of query tile w at 128 w
-    static constexpr int O_COL0 = 256;                     // O of query tile w at 256 + 128 w
+    static constexpr int S_COL0 = 0;                       // S of query tile w at 128 w
+    // Head dims up to 64 leave tensor-memory columns free (O is 64 wide): P then gets columns of its own, so the
+    // next scores of a query tile are issued as soon as its softmax warps hold the current ones in registers,
+    // instead of after the product that reads P.  With 128-wide O the 512 columns are full and P overwrites S.
+    static constexpr bool SEPARATE_P = HD <= 64;
+    static constexpr int P_COLS = TK / 2;                  // packed 16-bit probabilities of one tile
+    static constexpr int P_COL0 = SEPARATE_P ? 256 : S_COL0;
+    static constexpr int P_STRIDE = SEPARATE_P ? P_COLS : TK;
+    static constexpr int O_COL0 = SEPARATE_P ? 384 : 256;  // O of query tile w at O_COL0 + HD w (128 w when P overwrites S)
+    static constexpr int O_STRIDE = SEPARATE_P ? HD : TK;
     static constexpr int TMEM_COLS = 512;
 };
 
@@ -218,7 +192,9 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     uint64_t *s_full = bars + 6;        // [2]  scores of query tile w ready      (MMA -> softmax w)
     uint64_t *p_ready = bars + 8;       // [2]  probabilities of tile w in TMEM   (softmax w -> MMA)
     uint64_t *pv_done = bars + 10;      // [2]  O_w of the item is complete       (MMA -> softmax w)
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 12);
+    uint64_t *s_free = bars + 12;       // [2]  scores of tile w are in registers (softmax w -> MMA; separate P only)
+    uint64_t *p_free = bars + 14;       // [2]  the product that read P_w is done (MMA -> softmax w; separate P only)
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(bars + 16);
     volatile uint32_t *abort_flag = tmem_slot + 1;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -232,6 +208,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             mbar_init(s_full + s, 1);
             mbar_init(p_ready + s, 4);
             mbar_init(pv_done + s, 1);
+            mbar_init(s_free + s, 4);
+            mbar_init(p_free + s, 1);
         }
         *abort_flag = 0;
         fence_barrier_init();
@@ -310,8 +288,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
             };
             auto issue_pv = [&](int w, int st, bool first, bool last) {
                 const uint32_t v_addr = smem_u32(sB + st * Cfg::BUNDLE_BYTES);
-                const uint32_t p_tmem = tmem_base + Cfg::S_COL0 + w * TK;
-                const uint32_t o_tmem = tmem_base + Cfg::O_COL0 + w * TK;
+                const uint32_t p_tmem = tmem_base + Cfg::P_COL0 + w * Cfg::P_STRIDE;
+                const uint32_t o_tmem = tmem_base + Cfg::O_COL0 + w * Cfg::O_STRIDE;
 #pragma unroll
                 for (int ks = 0; ks < TK / 16; ++ks) {
                     // 16 keys per step: 8 packed columns of P, two 8-key groups (2 x 1024 bytes) of V
@@ -322,6 +300,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 // the softmax warps need no signal for the products in between: the scores they wait for next
                 // are committed after this product, and a commit covers everything issued before it
                 if (last) umma_commit(pv_done + w);
+                else if (Cfg::SEPARATE_P) umma_commit(p_free + w);   // the softmax may write the next P
             };
             bool ok = true;
             uint32_t kv_cnt = 0, item_cnt = 0, tile_cnt[2] = {0, 0};
@@ -338,15 +317,37 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 for (int j = 0; ok && j < it.n_max; ++j, ++kv_cnt) {
                     const int st = kv_cnt & 1;
                     if (!(ok = mbar_wait(b_full + st, (kv_cnt >> 1) & 1, abort_flag))) break;
+                    if (Cfg::SEPARATE_P) {
+                        // the next scores first: S_w is free as soon as its softmax warps have read it
 #pragma unroll
-                    for (int w = 0; w < 2; ++w) {
-                        if (j < it.n_tiles[w]) {
-                            if (!(ok = mbar_wait(p_ready + w, tile_cnt[w] & 1u, abort_flag))) break;
-                            ++tile_cnt[w];
-                            tc_fence_after_sync();
-                            issue_pv(w, st, j == 0, j + 1 == it.n_tiles[w]);
+                        for (int w = 0; w < 2; ++w) {
+                            if (j + 1 < it.n_tiles[w]) {
+                                if (!(ok = mbar_wait(s_free + w, tile_cnt[w] & 1u, abort_flag))) break;
+                                tc_fence_after_sync();
+                                issue_qk(w, st);
+                            }
                         }
-                        if (j + 1 < it.n_tiles[w]) issue_qk(w, st);
+                        if (!ok) break;
+#pragma unroll
+                        for (int w = 0; w < 2; ++w) {
+                            if (j < it.n_tiles[w]) {
+                                if (!(ok = mbar_wait(p_ready + w, tile_cnt[w] & 1u, abort_flag))) break;
+                                ++tile_cnt[w];
+                                tc_fence_after_sync();
+                                issue_pv(w, st, j == 0, j + 1 == it.n_tiles[w]);
+                            }
+                        }
+                    } else {
+#pragma unroll
+                        for (int w = 0; w < 2; ++w) {
+                            if (j < it.n_tiles[w]) {
+                                if (!(ok = mbar_wait(p_ready + w, tile_cnt[w] & 1u, abort_flag))) break;
+                                ++tile_cnt[w];
+                                tc_fence_after_sync();
+                                issue_pv(w, st, j == 0, j + 1 == it.n_tiles[w]);
+                            }
+                            if (j + 1 < it.n_tiles[w]) issue_qk(w, st);
+                        }
                     }
                     if (!ok) break;
                     umma_commit(b_empty + st);
@@ -361,11 +362,13 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
         const int row = quarter * 32 + lane;                 // row of the tile = TMEM lane
         const uint32_t lane_addr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);
         const uint32_t s_addr = lane_addr + Cfg::S_COL0 + w * TK;
-        const uint32_t o_addr = lane_addr + Cfg::O_COL0 + w * TK;
+        const uint32_t p_addr = lane_addr + Cfg::P_COL0 + w * Cfg::P_STRIDE;
+        const uint32_t o_addr = lane_addr + Cfg::O_COL0 + w * Cfg::O_STRIDE;
         const float sl2 = rsqrtf(static_cast<float>(a.head_dim)) * 1.4426950408889634f;
         bool ok = true;
         uint32_t tile_cnt = 0;                               // tiles this warp group has consumed so far
         uint32_t done_cnt = 0;                               // items this warp group has finished
+        uint32_t pf_cnt = 0;                                 // waits on p_free so far (one per tile but an item's first)
         AtcItem it;
         for (int jj = 0; ok && atc_next(a, jj, it);) {
             const int tile_q0 = it.q0 + w * TQ;
@@ -384,6 +387,12 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                 for (int c = 0; c < TK / 32; ++c)
                     tmem_ld_32x32(s_addr + c * 32, *reinterpret_cast<uint32_t(*)[32]>(&s[c * 32]));
                 tmem_ld_wait();
+                if (Cfg::SEPARATE_P) {
+                    // the scores are in registers: S_w may take the next tile's scores
+                    tc_fence_before_sync();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(s_free + w);
+                }
                 if (j * TK + TK - 1 > a.pos0 + tile_q0) {     // tile holds keys beyond some query of this tile
 #pragma unroll
                     for (int i = 0; i < TK; ++i)
@@ -410,6 +419,16 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                         m_used = mx;
                     }
                 }
+                if (Cfg::SEPARATE_P && j > 0) {
+                    // P_w and (for a rescale) O_w are touched next: the product that read the previous P_w must be
+                    // done.  It was issued a whole softmax ago, so this wait succeeds at once.  (The item's first
+                    // tile follows the wait for pv_done at the end of the previous item.)
+                    ok = mbar_wait(p_free + w, pf_cnt & 1u, abort_flag);
+                    ++pf_cnt;
+                    ok = __all_sync(0xFFFFFFFFu, ok);
+                    if (!ok) break;
+                    tc_fence_after_sync();
+                }
                 const float neg_ms = -m_used * sl2;
                 float sum0 = 0.f, sum1 = 0.f, sum2 = 0.f, sum3 = 0.f;
 #pragma unroll
@@ -423,12 +442,8 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                         fma2(x2, x3, sl2, neg_ms);
                         x0 = ex2_approx(x0);
                         x1 = ex2_approx(x1);
-                        if (POLY_EXP2) {                      // optionally half of the exponentials on the FMA pipe
-                            exp2_poly_pair(x2, x3);
-                        } else {
-                            x2 = ex2_approx(x2);
-                            x3 = ex2_approx(x3);
-                        }
+                        x2 = ex2_approx(x2);
+                        x3 = ex2_approx(x3);
                         sum0 += x0;
                         sum1 += x1;
                         sum2 += x2;
@@ -436,7 +451,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
                         pk[i] = pack_h16x2(x0, x1);
                         pk[i + 1] = pack_h16x2(x2, x3);
                     }
-                    tmem_st_32x16(s_addr + c * 16, pk);       // overwrites scores already consumed
+                    tmem_st_32x16(p_addr + c * 16, pk);       // (overwrites scores already consumed when P shares S's columns)
                 }
                 l = l * f + ((sum0 + sum1) + (sum2 + sum3));
                 if (__any_sync(0xFFFFFFFFu, raise)) {
