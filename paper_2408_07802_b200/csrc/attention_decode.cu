@@ -72,8 +72,8 @@ attn_decode_kernel(const DecodeAttnParams p) {
             const int key = r0 + u * RPW + rg;
             valid[u] = key < k_end;
             const long long off = (long long)(valid[u] ? key : k_begin) * HD + sub * 8;
-            kk[u] = active ? *reinterpret_cast<const uint4 *>(gk + off) : make_uint4(0u, 0u, 0u, 0u);
-            vv[u] = active ? *reinterpret_cast<const uint4 *>(gv + off) : make_uint4(0u, 0u, 0u, 0u);
+            kk[u] = active ? __ldcs(reinterpret_cast<const uint4 *>(gk + off)) : make_uint4(0u, 0u, 0u, 0u);
+            vv[u] = active ? __ldcs(reinterpret_cast<const uint4 *>(gv + off)) : make_uint4(0u, 0u, 0u, 0u);
         }
 #pragma unroll
         for (int qh = 0; qh < QH; ++qh) {
@@ -252,14 +252,14 @@ attn_decode_gqa_kernel(const DecodeAttnParams p) {
             const int key = r0 + kb * 8 + nq;
 #pragma unroll
             for (int c = 0; c < CH; ++c)
-                kk[kb][c] = key < k_end ? *reinterpret_cast<const uint4 *>(gk + (long long)key * HD + c * 32 + kq * 8) : zero;
+                kk[kb][c] = key < k_end ? __ldcs(reinterpret_cast<const uint4 *>(gk + (long long)key * HD + c * 32 + kq * 8)) : zero;
         }
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             const int key = r0 + (i >> 1) * 8 + kq * 2 + (i & 1);
 #pragma unroll
             for (int hf = 0; hf < HF; ++hf)
-                vv[i][hf] = key < k_end ? *reinterpret_cast<const uint4 *>(gv + (long long)key * HD + hf * 64 + nq * 8) : zero;
+                vv[i][hf] = key < k_end ? __ldcs(reinterpret_cast<const uint4 *>(gv + (long long)key * HD + hf * 64 + nq * 8)) : zero;
         }
         float s[2][4];
 #pragma unroll
