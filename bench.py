@@ -157,6 +157,9 @@ def workload_config(shape, args):
            "l2": "inputs larger than L2 (weights read every step exceed 126 MB)"
                  if weight_bytes(shape) > 126e6 else "L2 flushed between steps",
            "context": PAPER_CONTEXT}
+    if not shape.decode_steps and shape.batch * shape.seqlen > 32:
+        cfg["last_layer"] = ("past its qkv GEMM the last layer runs for the last position of every sequence only (the "
+                             "logits of the other positions are not part of the call); that work is not in the FLOP counts")
     paper_ms = paper_ttft_ms(shape)
     if paper_ms is not None:
         cfg["paper_ttft_ms"] = paper_ms
@@ -350,7 +353,7 @@ def prefill_leg(name, args, kr, ki, torch, dev, local_rank, steps=20):
     status = model.device_status()
     model.close()
     peaks, _ = load_peaks()
-    fl = ki.algorithmic_flops(shape)
+    fl = ki.algorithmic_flops(shape, last_positions_only=shape.batch * shape.seqlen > 32)
     tokens = shape.batch * shape.seqlen
     return {
         "workload": f"{name} prefill", "batch": shape.batch, "seqlen": shape.seqlen, "steps": steps,
@@ -573,14 +576,18 @@ def main():
         return
 
     peaks, peak_kind = load_peaks()
-    fl = ki.algorithmic_flops(shape)
+    # the call returns last-position logits, so the last layer runs on one row per sequence past its qkv GEMM: the
+    # work that is thereby not needed is not counted (kraken_inputs.algorithmic_flops)
+    short_last = tokens > 32
+    fl = ki.algorithmic_flops(shape, last_positions_only=short_last)
     gemm_ms = sum(prof_ms[k] for k in ("gemm_qkv", "gemm_proj", "gemm_up", "gemm_down")) / args.steps
     gemm_launches = sum(prof_n[k] for k in ("gemm_qkv", "gemm_proj", "gemm_up", "gemm_down")) // args.steps
     achieved = fl["gemm"] / (gemm_ms * 1e-3) / 1e12 if gemm_ms > 0 else 0.0
     peak = peaks["bf16_tflops_sustained"]
     T, N, L, d, F = tokens, shape.n_branch, shape.n_layer, shape.d_model, shape.d_ff
-    kind_flops = {"gemm_qkv": 2.0 * T * N * L * 3 * d * d, "gemm_proj": 2.0 * T * N * L * d * d,
-                  "gemm_up": 2.0 * T * N * L * d * F, "gemm_down": 2.0 * T * N * L * d * F,
+    rows_rest = T * (L - 1) + shape.batch if short_last else T * L      # token rows past the qkv GEMMs, over all layers
+    kind_flops = {"gemm_qkv": 2.0 * T * N * L * 3 * d * d, "gemm_proj": 2.0 * rows_rest * N * d * d,
+                  "gemm_up": 2.0 * rows_rest * N * d * F, "gemm_down": 2.0 * rows_rest * N * d * F,
                   "attention": fl["attn"]}
     kernels = {}
     for k, ms in prof_ms.items():

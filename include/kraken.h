@@ -109,6 +109,11 @@ int kraken_create(const kraken_config *cfg, const kraken_weights *weights, void 
  * d_logits: device fp32 [batch, V], logits of the LAST position of each sequence.
  * Fills the KV cache rows 0..seqlen-1 of sequences 0..batch-1 and sets the handle's
  * length to seqlen.  Token ids outside [0, V) are read as 0 and raise status bit 0.
+ * Only the last position's logits are returned, so past its Q_K_V product (whose K and V rows the cache needs
+ * for every position) the LAST layer runs for the last position of every sequence only: its queries attend over
+ * the cache like a decode step, and the output projection, the second LayerNorm and the FFN see batch rows.
+ * The results are those of Algorithm 1 for these rows; the work for the other rows of that layer is not done
+ * (kraken_logits_rows does it when asked for them).  kraken_prefill_packed does the same.
  * Errors: EINVAL, ECAPACITY (batch > max_batch, seqlen > max_pos), ECUDA. */
 int kraken_prefill(kraken_handle *h, const int32_t *d_tokens, int32_t batch, int32_t seqlen,
                    float *d_logits, void *stream);
@@ -175,7 +180,9 @@ int kraken_prefill_all_logits(kraken_handle *h, const int32_t *d_tokens, int32_t
                               float *d_logits, void *stream);
 
 /* Logits of chosen token rows of the most recent prefill (its last-layer outputs stay in
- * scratch until the next call that runs the model).  h_rows: HOST int32 [n_rows], row = b*seqlen + t;
+ * scratch until the next call that runs the model; after a prefill that ran its last layer for the last
+ * positions only, this call first runs that layer on every row, from the inputs the prefill left in scratch).
+ * h_rows: HOST int32 [n_rows], row = b*seqlen + t;
  * d_logits: device fp32 [n_rows, V].  Errors: EINVAL, ESTATE (no prefill yet), ECAPACITY (n_rows
  * larger than max_batch * max_pos). */
 int kraken_logits_rows(kraken_handle *h, const int32_t *h_rows, int32_t n_rows, float *d_logits, void *stream);
@@ -240,7 +247,8 @@ typedef enum kraken_tuning_key {
     KRAKEN_TUNE_LN_FUSION = 2,       /* LayerNorm inside the kernel that finishes its input rows (kraken_op_grouped_gemm_ln):
                                         2 = wherever it fits, 3 = behind the FFN down-projection only; 0, 1 = every
                                         LayerNorm its own launch (the default: see the measurements in the source)   */
-    KRAKEN_TUNE_COUNT = 3
+    KRAKEN_TUNE_LAST_LAYER = 3,      /* prefill that returns last-position logits: 1 = the last layer runs on every row too */
+    KRAKEN_TUNE_COUNT = 4
 } kraken_tuning_key;
 int kraken_tuning_set(int32_t key, int32_t value);
 

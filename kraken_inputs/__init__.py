@@ -275,15 +275,23 @@ def bf16_tensor_to_bits(t: torch.Tensor) -> np.ndarray:
     return t.detach().cpu().contiguous().view(torch.int16).numpy().view(np.uint16)
 
 
-def algorithmic_flops(s: KrakenShape, batch: Optional[int] = None, seqlen: Optional[int] = None) -> Dict[str, float]:
+def algorithmic_flops(s: KrakenShape, batch: Optional[int] = None, seqlen: Optional[int] = None,
+                      last_positions_only: bool = False) -> Dict[str, float]:
     """FLOPs the prefill must perform: dense contractions, causal half of attention,
-    last-position tail.  Masked attention work is not counted."""
+    last-position tail.  Masked attention work is not counted.
+    last_positions_only: the count for a prefill that returns the logits of the last position of every sequence
+    and therefore runs the last layer, past its qkv GEMM (the cache still needs every K and V row), on those B rows
+    only: the last layer's output projection and FFN on the other T - B rows and its attention for every query but
+    the last are not part of what has to be computed, and are not counted."""
     B = s.batch if batch is None else batch
     l = s.seqlen if seqlen is None else seqlen
     T = B * l
     N, L, d, F, H, hd, V = s.n_branch, s.n_layer, s.d_model, s.d_ff, s.n_head, s.head_dim, s.vocab
     gemm = 2.0 * T * N * L * (d * s.qkv_width + d * d + 2 * d * F)
     attn = float(N * L * B * H) * 4 * hd * (l * (l + 1) / 2)
+    if last_positions_only:
+        gemm -= 2.0 * (T - B) * N * (d * d + 2 * d * F)
+        attn -= float(N * B * H) * 4 * hd * (l * (l + 1) / 2 - l)
     tail = 2.0 * B * (N * d * d + V * d)
     return {"gemm": gemm, "attn": attn, "tail": tail, "total": gemm + attn + tail}
 

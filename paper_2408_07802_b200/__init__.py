@@ -44,7 +44,7 @@ EXPORTS = (
     "kraken_tuning_set", "kraken_test_wait_limit", "kraken_test_mma_issue_rate",
 )
 
-TUNE_LN_ROW_KERNEL, TUNE_ATTN_SCHEDULE, TUNE_LN_FUSION = 0, 1, 2
+TUNE_LN_ROW_KERNEL, TUNE_ATTN_SCHEDULE, TUNE_LN_FUSION, TUNE_LAST_LAYER = 0, 1, 2, 3
 STATUS_BAD_TOKEN, STATUS_WAIT_LIMIT = 1, 2
 
 

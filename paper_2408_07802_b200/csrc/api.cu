@@ -24,7 +24,7 @@ size_t align_up(size_t v) { return (v + ALIGN - 1) / ALIGN * ALIGN; }
 
 struct Layout {
     size_t status, tokens, rows, logits, x0, x, a, s, u, q, o, g, dec_part, x_alt, row_seq, row_pos, pos_arr, ln_parts,
-        ln_parts_bytes, ln_cnt, ln_cnt_bytes, total;
+        ln_parts_bytes, ln_cnt, ln_cnt_bytes, last_q, last_o, last_a, last_x, last_y, last_u, last_g, last_r, last_len, total;
 };
 
 int kv_heads_of(const kraken_config &c) { return c.n_kv_head > 0 ? c.n_kv_head : c.n_head; }
@@ -84,6 +84,17 @@ Layout layout_of(const kraken_config *c) {
     l.ln_parts = take(l.ln_parts_bytes);
     l.ln_cnt_bytes = gemm_ln_cnt_bytes((int)N, (int)T);
     l.ln_cnt = take(l.ln_cnt_bytes);
+    // the last layer of a prefill that only returns last-position logits: one row per sequence past the qkv GEMM
+    const size_t Bm = c->max_batch;
+    l.last_q = take(N * Bm * d * 2);
+    l.last_o = take(N * Bm * d * 2);
+    l.last_a = take(N * Bm * d * 4);
+    l.last_x = take(N * Bm * d * 4);
+    l.last_y = take(Bm * d * 4);
+    l.last_u = take(N * Bm * d * 2);
+    l.last_g = take(N * Bm * F * 2);
+    l.last_r = take(N * Bm * d * 4);
+    l.last_len = take(Bm * 4);
     l.total = off;
     return l;
 }
@@ -101,12 +112,15 @@ struct kraken_handle {
     uint8_t *scratch;
     Layout lay;
     int cur_len, batch, last_seqlen, last_rows;  // last_rows: token rows of the last model run
+    // the last prefill ran its last layer, past the qkv GEMM, for the last position of every sequence only: the
+    // layer outputs of the other rows are not there (kraken_logits_rows completes the layer first)
+    bool x_partial;
     // length of every cached sequence (cur_len is their maximum); ragged = they differ, set by a packed prefill
     std::vector<int> seq_len;
     bool ragged;
     int stage_layer_done;   // branch-parallel driving: the last layer whose FFN half has run (-1: none)
     bool stage_decode;      // the pieces being driven are a decode step (one new token per sequence)
-    std::vector<int> host_rows, host_row_seq, host_row_pos;   // staging of the packed-prefill tables
+    std::vector<int> host_rows, host_row_seq, host_row_pos, host_len_m1;   // staging of the packed-prefill tables
     cudaStream_t last_stream;
     bool one_chain;   // decode steps keep all branches in one chain of launches (KRAKEN_DECODE_ONE_CHAIN at create)
     // weight tensor maps, one per GEMM kind, re-encoded when the N tile changes
@@ -193,6 +207,13 @@ struct RunCtx {
     // STAGE_EMBED, STAGE_ATTN / STAGE_FFN = one half of layer stage_layer; y_ext = the cross-device sum for LN2
     int stage, stage_layer;
     const float *y_ext;
+    // TTFT needs the logits of the last position of every sequence only, so the last layer's attention queries and
+    // everything after them (output projection, LN-2, FFN) are needed for those rows only; K and V of the last layer
+    // are still computed for every position (the cache).  last_rows: device list of those rows, one per sequence.
+    bool last_only = false;
+    const int32_t *last_rows = nullptr;
+    const int *last_len_m1 = nullptr;   // packed prefill: length - 1 of every sequence (device), else all are seqlen - 1
+    int only_layer = -1;   // >= 0: run this layer alone, on every row (completing a last_only prefill)
 };
 enum { STAGE_ALL = 0, STAGE_EMBED = 1, STAGE_ATTN = 2, STAGE_FFN = 3 };
 
@@ -282,6 +303,13 @@ int branch_streams(kraken_handle *h);
         if ((x) != cudaSuccess) return cuda_check(cudaGetLastError(), "streams and events"); \
     } while (0)
 
+// Whether this run takes the short form of the last layer (see RunCtx::last_only): a whole-path prefill with more
+// than 32 rows (shorter prompts do not form the cross-branch sum as a tensor).
+bool short_last_of(const RunCtx &rc) {
+    return rc.last_only && !rc.stage && rc.only_layer < 0 && rc.T > SKINNY_MAX_ROWS && rc.last_rows != nullptr &&
+           (!rc.packed || rc.last_len_m1 != nullptr);
+}
+
 // Runs the L layers on `T = batch * seqlen` new tokens at positions pos0 .. pos0 + seqlen - 1.
 int run_layers(const RunCtx &rc, const int32_t *d_tokens) {
     kraken_handle *h = rc.h;
@@ -340,13 +368,16 @@ int run_layers(const RunCtx &rc, const int32_t *d_tokens) {
     const long long cache_kv = (long long)c.max_batch * cache_b;  // all of K (or V) of one (layer, branch)
     uint16_t *kv = reinterpret_cast<uint16_t *>(h->kv);
 
-    if (rc.stage == STAGE_ALL || rc.stage == STAGE_EMBED) {
+    if ((rc.stage == STAGE_ALL && rc.only_layer < 0) || rc.stage == STAGE_EMBED) {
         LaunchScope scope(h, KRAKEN_PROF_EMBED, rc.st);
         KR_TRY(launch_embed(d_tokens, T, rc.seqlen, rc.pos0, (const uint16_t *)h->w.wte, (const uint16_t *)h->w.wpe, d,
                             c.vocab, x0, status, rc.st, rc.pos_dev, rc.row_pos));
     }
     if (rc.stage == STAGE_EMBED) return KRAKEN_OK;
-    const int l_begin = rc.stage ? rc.stage_layer : 0, l_end = rc.stage ? rc.stage_layer + 1 : L;
+    const int l_begin = rc.stage ? rc.stage_layer : (rc.only_layer >= 0 ? rc.only_layer : 0);
+    const int l_end = rc.stage ? rc.stage_layer + 1 : (rc.only_layer >= 0 ? rc.only_layer + 1 : L);
+    // (the short last layer needs the cross-branch sum as a tensor, which prompts of up to 32 rows do not form)
+    const bool short_last = short_last_of(rc);
     for (int l = l_begin; l < l_end; ++l) {
         const float *xin = l == 0 ? x0 : x;
         const long long xin_gs = l == 0 ? 0 : td;
@@ -371,6 +402,75 @@ int run_layers(const RunCtx &rc, const int32_t *d_tokens) {
         e.pos0_dev = rc.pos_dev;
         e.row_seq = rc.row_seq; e.row_pos = rc.row_pos;
         KR_TRY(model_gemm(rc, G_QKV, l, T, u, td, e));
+        if (short_last && l == L - 1) {
+            // Last layer, last position of every sequence only (K and V of every position are in the cache by now):
+            // the rows' queries are gathered, attend over the cache like a decode step, and the rest of the layer
+            // runs on batch rows.
+            const int n = rc.batch;
+            const long long nd = (long long)n * d;
+            uint16_t *ql = at<uint16_t>(h, h->lay.last_q), *ol = at<uint16_t>(h, h->lay.last_o),
+                     *ul = at<uint16_t>(h, h->lay.last_u), *gl = at<uint16_t>(h, h->lay.last_g);
+            float *al = at<float>(h, h->lay.last_a), *xl = at<float>(h, h->lay.last_x), *yl = at<float>(h, h->lay.last_y),
+                  *rl = at<float>(h, h->lay.last_r);
+            {
+                LaunchScope scope(h, KRAKEN_PROF_ATTENTION, rc.st);
+                KR_TRY(launch_gather_rows(q, td * 2, N, d * 2, rc.last_rows, n, ql, rc.st));
+            }
+            {
+                LaunchScope scope(h, KRAKEN_PROF_ATTENTION, rc.st);
+                DecodeAttnParams dp;
+                dp.q = ql; dp.q_gstride = nd;
+                dp.k_cache = kc; dp.v_cache = kc + cache_kv;
+                dp.cache_gstride = 2 * cache_kv; dp.cache_bstride = cache_b;
+                dp.groups = N; dp.batch = n; dp.n_keys = rc.pos0 + rc.seqlen; dp.n_head = H; dp.head_dim = hd;
+                dp.n_kv_head = Hkv;
+                dp.max_pos = c.max_pos;
+                dp.pos_dev = rc.packed ? rc.last_len_m1 : nullptr;   // sequences of different lengths: their own key counts
+                dp.splits = decode_attention_splits(N, n, (hd == 64 || hd == 128) && decode_gqa_tile(H, Hkv) ? Hkv : H,
+                                                    dp.n_keys);
+                dp.partials = at<float>(h, h->lay.dec_part);
+                dp.out = ol; dp.out_gstride = nd;
+                h->launches[KRAKEN_PROF_ATTENTION] += dp.splits > 1 ? 1 : 0;
+                KR_TRY(launch_attention_decode(dp, rc.st));
+            }
+            e = epi_zero();
+            e.kind = KRAKEN_EPI_RESID_F32;
+            e.out_f32 = al; e.out_f32_gstride = nd; e.ld_out_f32 = d;
+            {
+                LaunchScope scope(h, KRAKEN_PROF_GEMM_PROJ, rc.st);   // the residual rows of the output projection
+                KR_TRY(launch_gather_rows(xin, xin_gs * 4, xin_gs ? N : 1, d * 4, rc.last_rows, n, rl, rc.st));
+            }
+            e.resid = rl; e.resid_gstride = xin_gs ? nd : 0; e.ld_resid = d;
+            KR_TRY(model_gemm(rc, G_PROJ, l, n, ol, nd, e));
+            if (c.parallel_ffn) {
+                LaunchScope scope(h, KRAKEN_PROF_LAYERNORM, rc.st);
+                KR_TRY(launch_gather_rows(u, td * 2, N, d * 2, rc.last_rows, n, ul, rc.st));
+            } else {
+                if (sum_pending) {
+                    KR_CU(cudaStreamWaitEvent(rc.st, h->ev_join[1], 0));
+                    sum_pending = false;
+                }
+                const float *ysrc = c.no_combine ? nullptr : (l == 0 ? x0 : S);
+                if (ysrc) {
+                    LaunchScope scope(h, KRAKEN_PROF_LAYERNORM, rc.st);
+                    KR_TRY(launch_gather_rows(ysrc, 0, 1, d * 4, rc.last_rows, n, yl, rc.st));
+                }
+                LaunchScope scope(h, KRAKEN_PROF_LAYERNORM, rc.st);
+                KR_TRY(launch_layernorm(al, nd, ysrc ? yl : nullptr, (const uint16_t *)h->w.ln2_g + ln_off,
+                                        h->w.ln2_b ? (const uint16_t *)h->w.ln2_b + ln_off : nullptr, N, n, d, c.ln_eps,
+                                        ul, rc.st, nullptr, 0, 0, status));
+            }
+            e = epi_zero();
+            e.kind = KRAKEN_EPI_GELU_BF16;
+            e.out_bf16 = gl; e.out_bf16_gstride = (long long)n * F; e.ld_out_bf16 = F; e.gelu_tanh = c.gelu_tanh;
+            KR_TRY(model_gemm(rc, G_UP, l, n, ul, nd, e));
+            e = epi_zero();
+            e.kind = KRAKEN_EPI_RESID_F32;
+            e.out_f32 = xl; e.out_f32_gstride = nd; e.ld_out_f32 = d;
+            e.resid = al; e.resid_gstride = nd; e.ld_resid = d;
+            KR_TRY(model_gemm(rc, G_DOWN, l, n, gl, (long long)n * F, e));
+            continue;
+        }
         // attention over the cached prefix
         AttnParams ap;
         ap.q = q; ap.q_gstride = td;
@@ -672,7 +772,10 @@ int tail_concat(const RunCtx &rc, const int32_t *d_rows, int n_rows, float *z) {
     uint16_t *cat = at<uint16_t>(h, h->lay.u);
     {
         LaunchScope scope(h, KRAKEN_PROF_TAIL, rc.st);
-        KR_TRY(launch_gather_concat(x, td, N, d, d_rows, n_rows, cat, rc.st));
+        if (short_last_of(rc))   // the last layer left one row per sequence, in sequence order: exactly the rows asked for
+            KR_TRY(launch_gather_concat(at<float>(h, h->lay.last_x), (long long)n_rows * d, N, d, nullptr, n_rows, cat, rc.st));
+        else
+            KR_TRY(launch_gather_concat(x, td, N, d, d_rows, n_rows, cat, rc.st));
     }
     EpiParams e = epi_zero();
     e.kind = KRAKEN_EPI_F32;
@@ -702,7 +805,9 @@ int tail_head(const RunCtx &rc, const float *z, int n_rows, float *d_logits) {
 }
 
 int run_tail(const RunCtx &rc, const int32_t *d_rows, int n_rows, float *d_logits) {
-    float *z = at<float>(rc.h, rc.h->lay.s);
+    // z normally borrows the cross-branch sum's buffer; after a short last layer that sum (and q) must survive, in
+    // case kraken_logits_rows runs the layer on every row later, so z then goes where the gathered y rows were
+    float *z = short_last_of(rc) ? at<float>(rc.h, rc.h->lay.last_y) : at<float>(rc.h, rc.h->lay.s);
     KR_TRY(tail_concat(rc, d_rows, n_rows, z));
     return tail_head(rc, z, n_rows, d_logits);
 }
@@ -711,14 +816,16 @@ int run_tail(const RunCtx &rc, const int32_t *d_rows, int n_rows, float *d_logit
 int prefill_body(kraken_handle *h, cudaStream_t st, const int32_t *d_tokens, int batch, int seqlen, float *d_logits,
                  bool all_logits) {
     RunCtx rc{h, st, batch, seqlen, 0, batch * seqlen, nullptr, 0};
-    KR_TRY(run_layers(rc, d_tokens));
-    set_pos_kernel<<<1, 64, 0, st>>>(at<int>(h, h->lay.pos_arr), seqlen, batch);
     int32_t *rows = at<int32_t>(h, h->lay.rows);
     const int n_rows = all_logits ? batch * seqlen : batch;
     h->launches[KRAKEN_PROF_TAIL]++;
     make_rows_kernel<<<(n_rows + 255) / 256, 256, 0, st>>>(rows, n_rows, all_logits ? 1 : seqlen,
                                                            all_logits ? 0 : seqlen - 1);
     if (cudaGetLastError() != cudaSuccess) return KRAKEN_ECUDA;
+    rc.last_only = !all_logits && tuning(KRAKEN_TUNE_LAST_LAYER) != 1;
+    rc.last_rows = rows;
+    KR_TRY(run_layers(rc, d_tokens));
+    set_pos_kernel<<<1, 64, 0, st>>>(at<int>(h, h->lay.pos_arr), seqlen, batch);
     return run_tail(rc, rows, n_rows, d_logits);
 }
 
@@ -739,6 +846,12 @@ int prefill_common(kraken_handle *h, const int32_t *d_tokens, int batch, int seq
         h->pre_seqlen = seqlen;
         h->pre_all = all_logits ? 1 : 0;
         h->pre_seen = 0;
+    }
+    {
+        RunCtx probe{h, st, batch, seqlen, 0, batch * seqlen, nullptr, 0};
+        probe.last_only = !all_logits && tuning(KRAKEN_TUNE_LAST_LAYER) != 1;
+        probe.last_rows = at<int32_t>(h, h->lay.rows);
+        h->x_partial = short_last_of(probe);
     }
     bool done = false;
     if (h->use_graph && !h->prof_on && h->pre_seen >= 1) {
@@ -793,6 +906,7 @@ int prefill_common(kraken_handle *h, const int32_t *d_tokens, int batch, int seq
 int prefill_packed(kraken_handle *h, const int32_t *d_tokens, const int32_t *h_seq_lens, int batch, float *d_logits,
                    void *stream) {
     if (!h || !d_tokens || !h_seq_lens || !d_logits || batch < 1) return KRAKEN_EINVAL;
+    h->x_partial = false;
     if (batch > h->cfg.max_batch) return KRAKEN_ECAPACITY;
     long long total = 0;
     int longest = 0;
@@ -831,8 +945,18 @@ int prefill_packed(kraken_handle *h, const int32_t *d_tokens, const int32_t *h_s
         cudaMemcpyAsync(d_pos, h->seq_len.data(), (size_t)batch * 4, cudaMemcpyHostToDevice, st) != cudaSuccess)
         return cuda_check(cudaGetLastError(), "packed prefill: table upload");
     RunCtx rc{h, st, batch, longest, 0, T, nullptr, 0, true, d_row_seq, d_row_pos};
+    // last-position logits only: the last layer runs on one row per sequence past its qkv GEMM (RunCtx::last_only)
+    h->host_len_m1.resize(batch);
+    for (int b = 0; b < batch; ++b) h->host_len_m1[b] = h_seq_lens[b] - 1;
+    int *d_len_m1 = at<int>(h, h->lay.last_len);
+    if (cudaMemcpyAsync(d_len_m1, h->host_len_m1.data(), (size_t)batch * 4, cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return cuda_check(cudaGetLastError(), "packed prefill: table upload");
+    rc.last_only = tuning(KRAKEN_TUNE_LAST_LAYER) != 1;
+    rc.last_rows = rows;
+    rc.last_len_m1 = d_len_m1;
     KR_TRY(run_layers(rc, d_tokens));
     KR_TRY(run_tail(rc, rows, batch, d_logits));
+    h->x_partial = short_last_of(rc);
     h->cur_len = longest;
     h->batch = batch;
     h->last_seqlen = longest;
@@ -931,6 +1055,7 @@ static RunCtx stage_ctx(kraken_handle *h, cudaStream_t st, int stage, int layer,
 
 int kraken_stage_begin(kraken_handle *h, const int32_t *d_tokens, int32_t batch, int32_t seqlen, void *stream) {
     if (!h || !d_tokens || batch < 1 || seqlen < 1) return KRAKEN_EINVAL;
+    h->x_partial = false;   // whatever runs now leaves every row's outputs, or none that kraken_logits_rows may read
     if (batch > h->cfg.max_batch || seqlen > h->cfg.max_pos) return KRAKEN_ECAPACITY;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     h->last_stream = st;
@@ -951,6 +1076,7 @@ int kraken_stage_begin(kraken_handle *h, const int32_t *d_tokens, int32_t batch,
 
 int kraken_stage_begin_decode(kraken_handle *h, const int32_t *d_tokens, int32_t batch, void *stream) {
     if (!h || !d_tokens || batch < 1) return KRAKEN_EINVAL;
+    h->x_partial = false;   // whatever runs now leaves every row's outputs, or none that kraken_logits_rows may read
     if (h->cur_len < 1 || batch != h->batch) return KRAKEN_ESTATE;
     if (h->cur_len + 1 > h->cfg.max_pos) return KRAKEN_ECAPACITY;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -1058,11 +1184,24 @@ int kraken_logits_rows(kraken_handle *h, const int32_t *h_rows, int32_t n_rows, 
     for (int i = 0; i < n_rows; ++i)
         if (h_rows[i] < 0 || h_rows[i] >= h->last_rows) return KRAKEN_EINVAL;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    RunCtx rc{h, st, h->batch, h->last_seqlen, 0, h->last_rows, nullptr, 0};
+    h->last_stream = st;
+    if (h->x_partial) {
+        // the prefill ran its last layer for the last positions only: run that layer on every row now (its inputs,
+        // the previous layer's outputs and their sum, are untouched; K and V are written again with the same values)
+        RunCtx full = rc;
+        if (h->ragged) {
+            full.packed = true;
+            full.row_seq = at<int>(h, h->lay.row_seq);
+            full.row_pos = at<int>(h, h->lay.row_pos);
+        }
+        full.only_layer = h->cfg.n_layer - 1;
+        KR_TRY(run_layers(full, nullptr));
+        h->x_partial = false;
+    }
     int32_t *rows = at<int32_t>(h, h->lay.rows);
     if (cudaMemcpyAsync(rows, h_rows, (size_t)n_rows * 4, cudaMemcpyHostToDevice, st) != cudaSuccess)
         return KRAKEN_ECUDA;
-    RunCtx rc{h, st, h->batch, h->last_seqlen, 0, h->last_rows, nullptr, 0};
-    h->last_stream = st;
     return run_tail(rc, rows, n_rows, d_logits);
 }
 
@@ -1100,6 +1239,7 @@ int decode_body(kraken_handle *h, cudaStream_t st, const int32_t *d_tokens, int 
 
 int kraken_decode_step(kraken_handle *h, const int32_t *d_tokens, int32_t batch, float *d_logits, void *stream) {
     if (!h || !d_tokens || !d_logits || batch < 1) return KRAKEN_EINVAL;
+    h->x_partial = false;   // whatever runs now leaves every row's outputs, or none that kraken_logits_rows may read
     if (h->cur_len < 1 || batch != h->batch) return KRAKEN_ESTATE;
     if (h->cur_len + 1 > h->cfg.max_pos) return KRAKEN_ECAPACITY;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
@@ -1216,6 +1356,7 @@ int kraken_cur_len(kraken_handle *h, int32_t *cur_len) {
 
 int kraken_reset(kraken_handle *h) {
     if (!h) return KRAKEN_EINVAL;
+    h->x_partial = false;   // whatever runs now leaves every row's outputs, or none that kraken_logits_rows may read
     if (cudaStreamSynchronize(h->last_stream) != cudaSuccess) return KRAKEN_ECUDA;
     if (cudaMemset(h->scratch + h->lay.status, 0, 256) != cudaSuccess) return KRAKEN_ECUDA;
     if (cudaMemset(h->scratch + h->lay.ln_cnt, 0, h->lay.ln_cnt_bytes) != cudaSuccess) return KRAKEN_ECUDA;

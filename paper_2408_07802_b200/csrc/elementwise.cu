@@ -396,6 +396,21 @@ gather_concat_kernel(const float *__restrict__ x, long long x_gstride, int group
     }
 }
 
+// dst[g][i][:] = src[g][rows[i]][:] for rows of row_bytes bytes (a multiple of 16), one warp per (group, row)
+__global__ void __launch_bounds__(ROW_WARPS * 32)
+gather_rows_kernel(const uint8_t *__restrict__ src, long long src_gstride, int groups, int row_bytes,
+                   const int32_t *__restrict__ rows, int n_rows, uint8_t *__restrict__ dst) {
+    pdl_wait();
+    pdl_trigger();
+    const long long w = (long long)blockIdx.x * ROW_WARPS + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (w >= (long long)n_rows * groups) return;
+    const int r = static_cast<int>(w % n_rows), g = static_cast<int>(w / n_rows);
+    const uint4 *s = reinterpret_cast<const uint4 *>(src + g * src_gstride + (size_t)rows[r] * row_bytes);
+    uint4 *d = reinterpret_cast<uint4 *>(dst + ((size_t)g * n_rows + r) * row_bytes);
+    for (int v = lane; v < row_bytes / 16; v += 32) d[v] = s[v];
+}
+
 // out = x_0 + x_1 + ... + x_{G-1} element by element, added in ascending group order (the order the
 // down-projection epilogue and LayerNorm-2 use when they form the same cross-branch sum themselves)
 __global__ void __launch_bounds__(256)
@@ -554,6 +569,18 @@ int launch_gather_concat(const float *x, long long x_gstride, int groups, int d,
     return cuda_check(launch_pdl(gather_concat_kernel, dim3(static_cast<unsigned>((warps + ROW_WARPS - 1) / ROW_WARPS)),
                                  dim3(ROW_WARPS * 32), 0, stream, x, x_gstride, groups, d, rows, n_rows, out),
                       "gather: launch");
+}
+
+int launch_gather_rows(const void *src, long long src_gstride_bytes, int groups, int row_bytes, const int32_t *rows,
+                       int n_rows, void *dst, cudaStream_t stream) {
+    if (!src || !dst || !rows || groups < 1 || n_rows < 1 || row_bytes < 16 || (row_bytes & 15) || (src_gstride_bytes & 15) ||
+        (reinterpret_cast<uintptr_t>(src) & 15) || (reinterpret_cast<uintptr_t>(dst) & 15))
+        return KRAKEN_EINVAL;
+    const long long warps = (long long)groups * n_rows;
+    return cuda_check(launch_pdl(gather_rows_kernel, dim3(static_cast<unsigned>((warps + ROW_WARPS - 1) / ROW_WARPS)),
+                                 dim3(ROW_WARPS * 32), 0, stream, static_cast<const uint8_t *>(src), src_gstride_bytes,
+                                 groups, row_bytes, rows, n_rows, static_cast<uint8_t *>(dst)),
+                      "gather rows: launch");
 }
 
 int launch_sum_groups(const float *x, long long gstride, int groups, long long n, float *out, cudaStream_t stream) {

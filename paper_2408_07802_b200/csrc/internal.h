@@ -124,6 +124,9 @@ int launch_sum_groups(const float *x, long long gstride, int groups, long long n
 int launch_gather_concat(const float *x, long long x_gstride, int groups, int d, const int32_t *rows, int n_rows,
                          uint16_t *out, cudaStream_t stream);
 int launch_f32_to_bf16(const float *in, uint16_t *out, long long n, cudaStream_t stream);
+// dst[g][i][:] = src[g][rows[i]][:]; rows of row_bytes bytes (a multiple of 16); rows: device int32 [n_rows]
+int launch_gather_rows(const void *src, long long src_gstride_bytes, int groups, int row_bytes, const int32_t *rows,
+                       int n_rows, void *dst, cudaStream_t stream);
 
 struct AttnParams {
     const uint16_t *q;

@@ -144,7 +144,10 @@ def test_stage_calls_in_lockstep_equal_the_single_gpu_prefill(name, split):
     whole = kr.KrakenModel(kr.make_config(s), w, dev)
     l0 = min(s.seqlen, s.max_pos - 4)               # room for the decode steps below
     tok = ki.uniform_tokens(2, s.vocab, s.batch, l0, dev)
-    ref = whole.prefill(tok)
+    # the pieces run every layer on every row; so does the reference (the single call's shortcut for the last layer's
+    # other rows takes other kernels for the last positions)
+    with kr.tuning(kr.TUNE_LAST_LAYER, 1):
+        ref = whole.prefill(tok)
     engines = []
     for first, count in split:
         mine = bp.slice_weights(w, s.n_branch, first, count, with_concat_bias=first == 0)
@@ -210,7 +213,8 @@ def test_one_nccl_rank_through_the_collective_path_equals_prefill():
         w = ki.make_weights(s, seed=0, device=dev)
         m = kr.KrakenModel(kr.make_config(s), w, dev)
         tok = ki.uniform_tokens(2, s.vocab, s.batch, s.seqlen, dev)
-        ref = m.prefill(tok).clone()
+        with kr.tuning(kr.TUNE_LAST_LAYER, 1):   # every layer on every row, like the pieces
+            ref = m.prefill(tok).clone()
         runner = bp.BranchParallelPrefill(m, bp.TorchDistGroup(), s.n_layer, timing=True)
         got = runner.prefill(tok)
         t = runner.last_timing
