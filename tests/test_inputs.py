@@ -47,3 +47,11 @@ def test_weights_and_tokens_law_and_reproducibility():
 def test_flop_accounting():
     f = ki.algorithmic_flops(ki.CONFIGS["C3"])
     assert abs(f["gemm"] / 1e12 - 105.55) < 0.05 and abs(f["attn"] / 1e12 - 8.80) < 0.02
+    # last-position logits only: the last layer's projections and FFN for the other T - B rows and its attention
+    # for every query but the last are not needed (1/L of that work)
+    s = ki.CONFIGS["C3"]
+    g = ki.algorithmic_flops(s, last_positions_only=True)
+    T, B, N, d, F, H, hd, l = s.batch * s.seqlen, s.batch, s.n_branch, s.d_model, s.d_ff, s.n_head, s.head_dim, s.seqlen
+    assert f["gemm"] - g["gemm"] == 2.0 * (T - B) * N * (d * d + 2 * d * F)
+    assert f["attn"] - g["attn"] == N * B * H * 4.0 * hd * (l * (l + 1) / 2 - l)
+    assert g["tail"] == f["tail"] and 0.975 < g["total"] / f["total"] < 0.985
