@@ -544,13 +544,6 @@ def main():
     tokens = shape.batch * shape.seqlen
     value = replicas.whole_job_throughput(tokens, ms_per_step, world)
 
-    # ---- the same K steps again with every launch bracketed by events: per-kernel device time
-    model.profile_enable(True)
-    for _ in range(args.steps):
-        step()
-    prof_ms, prof_n = model.profile_read()
-    model.profile_enable(False)
-
     # ---- end to end through the host-buffer call: pinned tokens in, logits out, every step
     h_tok = tok.cpu().pin_memory()
     h_log = torch.empty(shape.batch, shape.vocab, dtype=torch.float32).pin_memory()
@@ -568,6 +561,14 @@ def main():
     e2e_ms = s0.elapsed_time(s1) / args.steps
     e2e_ms = replicas.max_over_ranks(e2e_ms, dev)
     e2e_value = replicas.whole_job_throughput(tokens, e2e_ms, world)
+    # ---- the same K steps again with every launch bracketed by events: per-kernel device time
+    model.profile_read()            # (drops the counts of the end-to-end steps)
+    model.profile_enable(True)
+    for _ in range(args.steps):
+        step()
+    prof_ms, prof_n = model.profile_read()
+    model.profile_enable(False)
+
     status = model.device_status()
 
     if rank != 0:
