@@ -812,14 +812,19 @@ def test_layernorm_behind_the_gemm_epilogues_whole_model(name, mode):
         m.close()
 
 
-@pytest.mark.parametrize("name", ["C0", "K0-104", "C0-gqa", "P0", "S0x2"])
+@pytest.mark.parametrize("name", ["C0", "K0-104", "C0-gqa", "P0", "S0x2", "wide-batch"])
 def test_last_layer_on_last_positions_only_equals_the_full_last_layer(name):
     """A prefill that returns last-position logits runs its last layer, past the qkv GEMM, on one row per sequence
     (attention like a decode step over the cache, the projections on batch rows).  Same logits as with the last
     layer on every row (other kernels, other summation order: close, not bit-equal), the same cache bit for bit,
     fewer launches' worth of work; kraken_logits_rows afterwards still gives every row (it completes the layer),
     and a decode step continues from the cache."""
-    s = ki.KrakenShape("S0x2", 2, 3, 256, 4, 1024, 1024, 160, 2, 100, no_combine=1) if name == "S0x2" else ki.CONFIGS[name]
+    if name == "S0x2":
+        s = ki.KrakenShape("S0x2", 2, 3, 256, 4, 1024, 1024, 160, 2, 100, no_combine=1)
+    elif name == "wide-batch":   # 40 sequences: the last layer's batch rows go to the tile GEMM, not the weight-streaming one
+        s = ki.KrakenShape("wide-batch", 3, 2, 128, 2, 256, 640, 24, 40, 20)
+    else:
+        s = ki.CONFIGS[name]
     w = ki.make_weights(s, seed=0, device=DEV)
     l0 = s.seqlen - 1
     tok = ki.uniform_tokens(11, s.vocab, s.batch, l0 + 1, DEV)
