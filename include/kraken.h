@@ -238,7 +238,8 @@ int kraken_storage_dtype(void);
 
 /* Hooks for tests and measurements (not part of the model's arithmetic).  Where the library has two kernels
  * for one step that give the same result and picks by shape, a test can force either one, process-wide:
- * value 0 restores the library's own choice.  Nothing on the launch path reads the environment; the two
+ * value 0 restores the library's own choice.  Set a value before the handle that should see it is created (a handle
+ * may replay a launch sequence it recorded earlier).  Nothing on the launch path reads the environment; the two
  * environment switches of a handle (KRAKEN_NO_GRAPH, KRAKEN_DECODE_ONE_CHAIN) are read once by kraken_create.
  * Errors: EINVAL (unknown key, value outside 0..3). */
 typedef enum kraken_tuning_key {
@@ -343,7 +344,7 @@ int kraken_op_grouped_gemm(const kraken_gemm_args *args, uint32_t *d_status, voi
  * in tensor memory.  out_f32 (and sum) are written as without the LayerNorm.
  * d_scratch: device memory of kraken_gemm_ln_scratch_bytes() bytes, zeroed ONCE by the caller before its first
  * use; every launch leaves its counters at zero again, so launches on one stream can share it (launches that
- * overlap on the device cannot).  gamma, beta: [G][n_out] (beta may be NULL = zeros); y: fp32 [M, n_out] added
+ * overlap on the device cannot; after a launch whose wait gave up, status bit 1, zero the scratch again).  gamma, beta: [G][n_out] (beta may be NULL = zeros); y: fp32 [M, n_out] added
  * to every group's rows before the statistics, or NULL.  Errors: EINVAL (other epilogues, missing pointers),
  * EUNSUPPORTED (m <= 32 rows with n_tile = 8; a row block of more N tiles than CTAs run at once),
  * ECAPACITY (scratch_bytes too small). */
