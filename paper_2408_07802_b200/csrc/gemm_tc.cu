@@ -82,7 +82,8 @@ __device__ __forceinline__ bool next_item(const KernelArgs &ka, int it, int &m_b
     return true;
 }
 
-template <int BN>
+// LN: with a LayerNorm behind the epilogue.  A kernel of its own, so that the plain one carries none of its code.
+template <int BN, bool LN>
 __global__ void __launch_bounds__(NUM_THREADS, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                const KernelArgs ka) {
@@ -189,7 +190,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         const int quarter = warp & 3;          // TMEM lanes this warp may read
         const int half = (warp - 2) >> 2;      // which half of the tile's columns it drains
         constexpr int CHUNKS = BN / 32;        // 32-column chunks of the tile: `half` takes every second one
-        const bool ln = ka.epi.ln_out != nullptr;
+        constexpr bool ln = LN;
         int acc = 0;
         uint32_t acc_phase = 0;
         bool ok = true;
@@ -202,29 +203,46 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const int row = m_blk * BM + quarter * 32 + lane;
             const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
                                    static_cast<uint32_t>(acc * BN);
-            RowStats rs{0.f, 0.f, 0.f};
+            if (!ln) {
 #pragma unroll 1
-            for (int c = half; c < CHUNKS; c += 2) {
-                const int col0 = n_blk * BN + c * 32;
-                if (col0 >= ka.shape.n_out) break;  // uniform across the warp
-                uint32_t r[32];
-                tmem_ld_32x32(t_row + static_cast<uint32_t>(c * 32), r);
-                tmem_ld_wait();
-                const int ncols = min(32, ka.shape.n_out - col0);
-                if (row < ka.shape.m) {
-                    float v[32];
+                for (int c = half; c < CHUNKS; c += 2) {
+                    const int col0 = n_blk * BN + c * 32;
+                    if (col0 >= ka.shape.n_out) break;  // uniform across the warp
+                    uint32_t r[32];
+                    tmem_ld_32x32(t_row + static_cast<uint32_t>(c * 32), r);
+                    tmem_ld_wait();
+                    if (row < ka.shape.m) {
+                        float v[32];
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
-                    if (ln) {
+                        for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+                        const int ncols = min(32, ka.shape.n_out - col0);
+                        epilogue_chunk(ka.epi, g, row, col0, ncols, v);
+                    }
+                }
+            }
+            RowStats rs{0.f, 0.f, 0.f};
+            if (ln) {
+                // first pass with a LayerNorm behind it: the same epilogue, the row statistics, and the row the
+                // LayerNorm sees back into the accumulator's columns
+#pragma unroll 1
+                for (int c = half; c < CHUNKS; c += 2) {
+                    const int col0 = n_blk * BN + c * 32;
+                    if (col0 >= ka.shape.n_out) break;
+                    uint32_t r[32];
+                    tmem_ld_32x32(t_row + static_cast<uint32_t>(c * 32), r);
+                    tmem_ld_wait();
+                    const int ncols = min(32, ka.shape.n_out - col0);
+                    if (row < ka.shape.m) {
+                        float v[32];
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
                         epilogue_chunk_ln(ka.epi, g, row, col0, ncols, v);
                         stats_add_chunk(rs, v, ncols);
 #pragma unroll
                         for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(v[i]);
-                    } else {
-                        epilogue_chunk(ka.epi, g, row, col0, ncols, v);
                     }
+                    tmem_st_32x32(t_row + static_cast<uint32_t>(c * 32), r);
                 }
-                if (ln) tmem_st_32x32(t_row + static_cast<uint32_t>(c * 32), r);   // the row the LayerNorm sees
             }
             if (ln) {
                 // the row's other columns are other CTAs' tiles: leave this part's statistics, wait for the rest
@@ -323,6 +341,7 @@ __device__ __forceinline__ bool next_item_pair(const KernelArgs &ka, int it, int
     return true;
 }
 
+template <bool LN>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(NUM_THREADS, 1)
 gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                     const KernelArgs ka) {
@@ -439,7 +458,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         float *stage = reinterpret_cast<float *>(smem + Cfg::STAGES * Cfg::STAGE_BYTES + 256) +
                        (warp - 2) * EPI_STAGE_FLOATS;
         const bool staged = epilogue_f32_stageable(ka.epi);
-        const bool ln = ka.epi.ln_out != nullptr;
+        constexpr bool ln = LN;
         int acc = 0;
         uint32_t acc_phase = 0;
         bool ok = true;
@@ -453,42 +472,63 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             const int row = row_base + lane;
             const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
                                    static_cast<uint32_t>(acc * BN2);
-            RowStats rs{0.f, 0.f, 0.f};
+            if (!ln) {
 #pragma unroll 1
-            for (int cc = 0; cc < CHUNKS; ++cc) {
-                const int c = half * CHUNKS + cc;
-                const int col0 = n_blk * BN2 + c * 32;
-                if (col0 >= ka.shape.n_out) break;
-                uint32_t r[32];
-                tmem_ld_32x32(t_row + static_cast<uint32_t>(c * 32), r);
-                tmem_ld_wait();
-                const int ncols = min(32, ka.shape.n_out - col0);
-                if (staged && col0 + 32 <= ka.shape.n_out) {
-                    // coalesced path: the whole warp takes part, rows past M are masked inside
-                    float v[32];
+                for (int cc = 0; cc < CHUNKS; ++cc) {
+                    const int c = half * CHUNKS + cc;
+                    const int col0 = n_blk * BN2 + c * 32;
+                    if (col0 >= ka.shape.n_out) break;
+                    uint32_t r[32];
+                    tmem_ld_32x32(t_row + static_cast<uint32_t>(c * 32), r);
+                    tmem_ld_wait();
+                    if (staged && col0 + 32 <= ka.shape.n_out) {
+                        // coalesced path: the whole warp takes part, rows past M are masked inside
+                        float v[32];
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
-                    if (ka.epi.bias) add_bias_chunk(ka.epi.bias + g * ka.epi.bias_gstride + col0, v, 32);
-                    epilogue_f32_staged(ka.epi, g, row_base, ka.shape.m, col0, v, stage, lane, ln);
-                    if (ln) {
+                        for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+                        if (ka.epi.bias) add_bias_chunk(ka.epi.bias + g * ka.epi.bias_gstride + col0, v, 32);
+                        epilogue_f32_staged(ka.epi, g, row_base, ka.shape.m, col0, v, stage, lane);
+                    } else if (row < ka.shape.m) {
+                        float v[32];
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+                        const int ncols = min(32, ka.shape.n_out - col0);
+                        epilogue_chunk(ka.epi, g, row, col0, ncols, v);
+                    }
+                }
+            }
+            RowStats rs{0.f, 0.f, 0.f};
+            if (ln) {
+                // first pass with a LayerNorm behind it (see the single-CTA kernel)
+#pragma unroll 1
+                for (int cc = 0; cc < CHUNKS; ++cc) {
+                    const int c = half * CHUNKS + cc;
+                    const int col0 = n_blk * BN2 + c * 32;
+                    if (col0 >= ka.shape.n_out) break;
+                    uint32_t r[32];
+                    tmem_ld_32x32(t_row + static_cast<uint32_t>(c * 32), r);
+                    tmem_ld_wait();
+                    const int ncols = min(32, ka.shape.n_out - col0);
+                    if (staged && col0 + 32 <= ka.shape.n_out) {
+                        float v[32];
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
+                        if (ka.epi.bias) add_bias_chunk(ka.epi.bias + g * ka.epi.bias_gstride + col0, v, 32);
+                        epilogue_f32_staged(ka.epi, g, row_base, ka.shape.m, col0, v, stage, lane, true);
                         if (row < ka.shape.m) stats_add_chunk(rs, v, 32);
 #pragma unroll
                         for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(v[i]);
-                    }
-                } else if (row < ka.shape.m) {
-                    float v[32];
+                    } else if (row < ka.shape.m) {
+                        float v[32];
 #pragma unroll
-                    for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
-                    if (ln) {
+                        for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
                         epilogue_chunk_ln(ka.epi, g, row, col0, ncols, v);
                         stats_add_chunk(rs, v, ncols);
 #pragma unroll
                         for (int i = 0; i < 32; ++i) r[i] = __float_as_uint(v[i]);
-                    } else {
-                        epilogue_chunk(ka.epi, g, row, col0, ncols, v);
                     }
+                    tmem_st_32x32(t_row + static_cast<uint32_t>(c * 32), r);
                 }
-                if (ln) tmem_st_32x32(t_row + static_cast<uint32_t>(c * 32), r);   // the row the LayerNorm sees
             }
             if (ln) {
                 tmem_st_wait();
@@ -537,6 +577,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     if (warp == 1) tmem_dealloc_pair(tmem_base, Cfg::TMEM_COLS);
 }
 
+template <bool LN>
 int launch_pair(const CUtensorMap &tmA, const CUtensorMap &tmB, const KernelArgs &ka, cudaStream_t stream) {
     using Cfg = PairCfg;
     static DeviceOnce configured;
@@ -544,7 +585,7 @@ int launch_pair(const CUtensorMap &tmA, const CUtensorMap &tmB, const KernelArgs
     const int dev = device_slot();
     if (dev < 0) return KRAKEN_ECUDA;
     if (!configured.done()) {
-        int rc = cuda_check(cudaFuncSetAttribute(gemm_tc_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        int rc = cuda_check(cudaFuncSetAttribute(gemm_tc_pair_kernel<LN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                  Cfg::SMEM_BYTES), "gemm pair: shared memory opt-in");
         if (rc) return rc;
         cudaLaunchConfig_t cfg = {};
@@ -559,7 +600,7 @@ int launch_pair(const CUtensorMap &tmA, const CUtensorMap &tmB, const KernelArgs
         cfg.attrs = &attr;
         cfg.numAttrs = 1;
         int n = 0;
-        if (cudaOccupancyMaxActiveClusters(&n, gemm_tc_pair_kernel, &cfg) != cudaSuccess || n < 1) {
+        if (cudaOccupancyMaxActiveClusters(&n, gemm_tc_pair_kernel<LN>, &cfg) != cudaSuccess || n < 1) {
             cudaGetLastError();
             n = (sm_count() > 0 ? sm_count() : 148) / 2;
         }
@@ -573,22 +614,28 @@ int launch_pair(const CUtensorMap &tmA, const CUtensorMap &tmB, const KernelArgs
     // LayerNorm behind the epilogue: the N tiles of a row block wait for each other, so a round of clusters must
     // hold whole row blocks (a block split over two rounds stalls its first part for a whole tile, every round)
     if (ka.epi.ln_out && clusters > ka.tiles_n) clusters -= clusters % ka.tiles_n;
-    return cuda_check(launch_pdl(gemm_tc_pair_kernel, dim3(2 * clusters), dim3(NUM_THREADS), Cfg::SMEM_BYTES, stream, tmA, tmB, ka),
+    return cuda_check(launch_pdl(gemm_tc_pair_kernel<LN>, dim3(2 * clusters), dim3(NUM_THREADS), Cfg::SMEM_BYTES, stream, tmA, tmB, ka),
                       "gemm pair: launch");
 }
 
-template <int BN>
-int launch_bn(const CUtensorMap &tmA, const CUtensorMap &tmB, const KernelArgs &ka, int grid, cudaStream_t stream) {
+template <int BN, bool LN>
+int launch_bn_as(const CUtensorMap &tmA, const CUtensorMap &tmB, const KernelArgs &ka, int grid, cudaStream_t stream) {
     using Cfg = TileCfg<BN>;
     static DeviceOnce configured;
     if (!configured.done()) {
-        int rc = cuda_check(cudaFuncSetAttribute(gemm_tc_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        int rc = cuda_check(cudaFuncSetAttribute(gemm_tc_kernel<BN, LN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                  Cfg::SMEM_BYTES), "gemm: shared memory opt-in");
         if (rc) return rc;
         configured.set();
     }
-    return cuda_check(launch_pdl(gemm_tc_kernel<BN>, dim3(grid), dim3(NUM_THREADS), Cfg::SMEM_BYTES, stream, tmA, tmB, ka),
+    return cuda_check(launch_pdl(gemm_tc_kernel<BN, LN>, dim3(grid), dim3(NUM_THREADS), Cfg::SMEM_BYTES, stream, tmA, tmB, ka),
                       "gemm: launch");
+}
+
+template <int BN>
+int launch_bn(const CUtensorMap &tmA, const CUtensorMap &tmB, const KernelArgs &ka, int grid, cudaStream_t stream) {
+    return ka.epi.ln_out ? launch_bn_as<BN, true>(tmA, tmB, ka, grid, stream)
+                         : launch_bn_as<BN, false>(tmA, tmB, ka, grid, stream);
 }
 
 }  // namespace
@@ -679,7 +726,8 @@ int launch_gemm_tc(const GemmOperands &op, const GemmShape &s, const EpiParams &
         if (ka.tiles_n > (bn == GEMM_TILE_PAIR ? sms_ / 2 : sms_)) return KRAKEN_EUNSUPPORTED;
     }
     ka.status = d_status;
-    if (bn == GEMM_TILE_PAIR) return launch_pair(*tmA, *tmB, ka, stream);
+    if (bn == GEMM_TILE_PAIR)
+        return epi.ln_out ? launch_pair<true>(*tmA, *tmB, ka, stream) : launch_pair<false>(*tmA, *tmB, ka, stream);
     const long long tiles = (long long)ka.tiles_m * ka.tiles_n;
     const long long units = ka.group_serial ? tiles : tiles * s.groups;
     const int sms = sm_count() > 0 ? sm_count() : 148;
