@@ -327,7 +327,10 @@ typedef struct kraken_gemm_args {
                                                                  weight-streaming kernel for m <= 32 (no RESID_SUM) */
     int32_t n_kv_head;                                        /* QKV only: key/value heads (0 = n_head); the K and V
                                                                  parts of n_out are n_kv_head * head_dim wide each */
-    int32_t reserved[1];
+    int32_t w_constant;                                       /* nonzero: w holds constant data (weights), written by
+                                                                 nothing queued on the stream before this call; the
+                                                                 kernel then fetches its first W tiles while the
+                                                                 stream's previous kernel is still finishing */
 } kraken_gemm_args;
 
 /* Grouped bf16 GEMM on the tensor cores (tcgen05 + TMEM accumulators, TMA operand loads).

@@ -73,7 +73,7 @@ class GemmArgs(C.Structure):
         ("k_cache", C.c_void_p), ("v_cache", C.c_void_p), ("cache_gstride", C.c_int64),
         ("seqlen", C.c_int32), ("pos0", C.c_int32), ("n_head", C.c_int32), ("head_dim", C.c_int32),
         ("max_pos", C.c_int32), ("gelu_tanh", C.c_int32), ("n_tile", C.c_int32), ("n_kv_head", C.c_int32),
-        ("reserved", C.c_int32 * 1),
+        ("w_constant", C.c_int32),
     ]
 
 

@@ -249,6 +249,10 @@ int model_gemm(const RunCtx &rc, GemmKind kind, int layer, int m_rows, const uin
     op.ldw = s.k;
     op.w_gstride = w_gstride;
     op.w = wbase + (layered ? ((long long)layer * N + g0) * w_gstride : 0);
+#ifndef KR_W_EARLY
+#define KR_W_EARLY 1
+#endif
+    op.w_static = KR_W_EARLY != 0;
     if (bias) {
         epi.bias = bias + (layered ? ((long long)layer * N + g0) * s.n_out : 0);
         epi.bias_gstride = s.n_out;
@@ -1491,7 +1495,7 @@ int op_grouped_gemm(const kraken_gemm_args *g, const kraken_gemm_ln_args *ln, ui
             g->out_bf16_gstride % 8 != 0 || g->cache_gstride % 8 != 0)
             return KRAKEN_EUNSUPPORTED;
     }
-    GemmOperands op{g->a, g->a_gstride, g->lda, g->w, g->w_gstride, g->ldw};
+    GemmOperands op{g->a, g->a_gstride, g->lda, g->w, g->w_gstride, g->ldw, g->w_constant != 0};
     GemmShape s{g->groups, g->m, g->n_out, g->k};
     EpiParams e = epi_zero();
     e.kind = k;

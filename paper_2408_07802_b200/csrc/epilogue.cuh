@@ -157,12 +157,48 @@ __device__ __forceinline__ void add_bias_chunk(const uint16_t *bias, float (&v)[
     }
 }
 
+// The same sums with the 32 bias values in shared memory (16-byte aligned; every lane reads the same words).
+__device__ __forceinline__ void add_bias_chunk_parked(const uint16_t *bias, float (&v)[32]) {
+    const uint4 *b4 = reinterpret_cast<const uint4 *>(bias);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const uint4 u = b4[i];
+        v[8 * i + 0] += h16_lo(u.x);
+        v[8 * i + 1] += h16_hi(u.x);
+        v[8 * i + 2] += h16_lo(u.y);
+        v[8 * i + 3] += h16_hi(u.y);
+        v[8 * i + 4] += h16_lo(u.z);
+        v[8 * i + 5] += h16_hi(u.z);
+        v[8 * i + 6] += h16_lo(u.w);
+        v[8 * i + 7] += h16_hi(u.w);
+    }
+}
+
+// A warp parks 128 bias values (those past n_out as zeros) in its shared-memory strip while the MMAs of its tile
+// run; lane l brings values 4 l .. 4 l + 3 of the strip, the bias of columns c .. c + 3.  A load from global memory
+// per 32-column chunk, between the accumulator and the store, cost the chunk about 700 cycles (measured: 16-bit
+// epilogue of a 128 x 256 tile 3.2 -> 2.6 us).
+__device__ __forceinline__ void park_bias(const uint16_t *bias, int c, int n_out, uint16_t *strip, int lane) {
+    uint2 b = make_uint2(0u, 0u);
+    if (c + 4 <= n_out && (reinterpret_cast<uintptr_t>(bias + c) & 7u) == 0) {
+        b = __ldg(reinterpret_cast<const uint2 *>(bias + c));
+    } else {
+        uint32_t e[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) e[i] = c + i < n_out ? bias[c + i] : 0u;
+        b = make_uint2(e[0] | (e[1] << 16), e[2] | (e[3] << 16));
+    }
+    reinterpret_cast<uint2 *>(strip)[lane] = b;
+    __syncwarp();
+}
+
 // One thread finishes 32 consecutive columns (col0 .. col0+31, the first ncols of them valid)
 // of output row `row` of group g.  For KRAKEN_EPI_RESID_SUM the same thread must see the
 // groups of one (row, column) in ascending order (the running sum is read back by its writer).
+// with_bias = false: the caller has added the bias already.
 __device__ __forceinline__ void epilogue_chunk(const EpiParams &p, int g, int row, int col0, int ncols,
-                                               float (&v)[32]) {
-    if (p.bias) add_bias_chunk(p.bias + g * p.bias_gstride + col0, v, ncols);
+                                               float (&v)[32], bool with_bias = true) {
+    if (with_bias && p.bias) add_bias_chunk(p.bias + g * p.bias_gstride + col0, v, ncols);
     switch (p.kind) {
         case KRAKEN_EPI_F32:
             store_f32_chunk(p.out_f32 + g * p.out_f32_gstride + (long long)row * p.ld_out_f32 + col0, v, ncols);

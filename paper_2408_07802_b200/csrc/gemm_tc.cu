@@ -41,7 +41,8 @@ struct TileCfg {
     static constexpr int STAGES = SMEM_BUDGET / STAGE_BYTES > 8 ? 8 : SMEM_BUDGET / STAGE_BYTES;
     // two accumulators; TMEM is allocated in powers of two of at least 32 columns
     static constexpr int TMEM_COLS = 2 * BN <= 64 ? 64 : (2 * BN <= 128 ? 128 : (2 * BN <= 256 ? 256 : 512));
-    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+    static constexpr int EPI_BIAS_BYTES = EPI_WARPS * 256;   // the epilogue warps' strips of bias values
+    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/ + EPI_BIAS_BYTES;
 };
 
 // 32-row slabs of one group as the fused LayerNorm counts them: every tile row, also past M, has its counters
@@ -55,6 +56,7 @@ struct KernelArgs {
     int a_g0, b_g0;      // first group's index along the outermost TMA dimension
     int group_serial;
     int n_fastest;  // tile order inside a group: 1 = n-tiles fastest, 0 = m-tiles fastest
+    int w_early;    // W is not the stream's previous kernel's to write: its first tiles are fetched before that one ends
     uint32_t *status;
 };
 
@@ -124,7 +126,22 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     __syncthreads();
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
-    pdl_wait();   // launched ahead of the end of its predecessor: nothing of the predecessor's is touched before here
+    // Launched ahead of the end of its predecessor: nothing of the predecessor's is touched before pdl_wait().  The
+    // weights are not the predecessor's, so the W tiles of the first stages are on their way while it drains.
+    int pre = 0;
+    if (threadIdx.x == 0 && ka.w_early) {
+        int m_blk, n_blk, g;
+        if (next_item(ka, 0, m_blk, n_blk, g)) {
+            pre = k_blocks < Cfg::STAGES ? k_blocks : Cfg::STAGES;
+            for (int kb = 0; kb < pre; ++kb) {
+                mbar_expect_tx(full_bar + kb, Cfg::STAGE_BYTES);
+                tma_load_3d(tiles + kb * Cfg::STAGE_BYTES + Cfg::A_BYTES, &tmB, full_bar + kb, kb * BK, n_blk * BN,
+                            ka.b_g0 + g * ka.b_gmul);
+            }
+        }
+    }
+    pdl_wait();
+    pdl_trigger();   // the successor's CTAs may take this one's place as soon as it leaves
 
     if (warp == 0) {
         if (lane == 0) {
@@ -134,12 +151,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             int m_blk, n_blk, g;
             for (int it = 0; ok && next_item(ka, it, m_blk, n_blk, g); ++it) {
                 for (int kb = 0; kb < k_blocks; ++kb) {
-                    if (!(ok = mbar_wait(empty_bar + stage, phase ^ 1u, abort_flag))) break;
+                    const bool early = it == 0 && kb < pre;   // stage kb, armed, its W tile under way
+                    if (!early && !(ok = mbar_wait(empty_bar + stage, phase ^ 1u, abort_flag))) break;
                     uint8_t *sa = tiles + stage * Cfg::STAGE_BYTES;
                     uint8_t *sb = sa + Cfg::A_BYTES;
-                    mbar_expect_tx(full_bar + stage, Cfg::STAGE_BYTES);
+                    if (!early) mbar_expect_tx(full_bar + stage, Cfg::STAGE_BYTES);
                     tma_load_3d(sa, &tmA, full_bar + stage, kb * BK, m_blk * BM, ka.a_g0 + g * ka.a_gmul);
-                    tma_load_3d(sb, &tmB, full_bar + stage, kb * BK, n_blk * BN, ka.b_g0 + g * ka.b_gmul);
+                    if (!early) tma_load_3d(sb, &tmB, full_bar + stage, kb * BK, n_blk * BN, ka.b_g0 + g * ka.b_gmul);
                     if (++stage == Cfg::STAGES) {
                         stage = 0;
                         phase ^= 1u;
@@ -191,11 +209,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         const int half = (warp - 2) >> 2;      // which half of the tile's columns it drains
         constexpr int CHUNKS = BN / 32;        // 32-column chunks of the tile: `half` takes every second one
         constexpr bool ln = LN;
+        uint16_t *bias_strip = reinterpret_cast<uint16_t *>(smem + Cfg::STAGES * Cfg::STAGE_BYTES + 256) + (warp - 2) * 128;
         int acc = 0;
         uint32_t acc_phase = 0;
         bool ok = true;
         int m_blk, n_blk, g;
         for (int it = 0; ok && next_item(ka, it, m_blk, n_blk, g); ++it) {
+            // the bias of this warp's chunks (chunk half + 2 i at values 32 i .. 32 i + 31), fetched while the MMAs run
+            if (!ln && ka.epi.bias)
+                park_bias(ka.epi.bias + g * ka.epi.bias_gstride,
+                          n_blk * BN + (half + 2 * (lane >> 3)) * 32 + 4 * (lane & 7), ka.shape.n_out, bias_strip, lane);
             ok = mbar_wait(acc_full + acc, acc_phase, abort_flag);
             ok = __all_sync(0xFFFFFFFFu, ok);
             if (!ok) break;
@@ -216,7 +239,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 #pragma unroll
                         for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
                         const int ncols = min(32, ka.shape.n_out - col0);
-                        epilogue_chunk(ka.epi, g, row, col0, ncols, v);
+                        if (ka.epi.bias) add_bias_chunk_parked(bias_strip + (c >> 1) * 32, v);   // (zeros past n_out)
+                        epilogue_chunk(ka.epi, g, row, col0, ncols, v, false);
                     }
                 }
             }
@@ -312,7 +336,8 @@ struct PairCfg {
     static constexpr int STAGES = 5;
     static constexpr int TMEM_COLS = 2 * BN2;
     static constexpr int EPI_STAGE_BYTES = EPI_WARPS * EPI_STAGE_FLOATS * 4;  // fp32 epilogue staging tiles
-    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 256 + EPI_STAGE_BYTES;
+    static constexpr int EPI_BIAS_BYTES = EPI_WARPS * 256;   // and their strips of bias values (128 columns each)
+    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 256 + EPI_STAGE_BYTES + EPI_BIAS_BYTES;
 };
 
 __device__ __forceinline__ bool next_item_pair(const KernelArgs &ka, int it, int cluster_id, int n_clusters,
@@ -385,7 +410,21 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     cluster_sync_all();  // both CTAs' barriers exist before anything is signalled across the pair
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
+    // (see the single-CTA kernel: the first stages' W tiles are fetched while the predecessor drains)
+    int pre = 0;
+    if (threadIdx.x == 0 && ka.w_early) {
+        int m_blk, n_blk, g;
+        if (next_item_pair(ka, 0, cluster_id, n_clusters, m_blk, n_blk, g)) {
+            pre = k_blocks < Cfg::STAGES ? k_blocks : Cfg::STAGES;
+            for (int kb = 0; kb < pre; ++kb) {
+                if (rank == 0) mbar_expect_tx(full_bar + kb, 2 * Cfg::STAGE_BYTES);
+                tma_load_3d_pair(tiles + kb * Cfg::STAGE_BYTES + Cfg::A_BYTES, &tmB, map_to_cta(smem_u32(full_bar + kb), 0),
+                                 kb * BK, n_blk * BN2 + (int)rank * (BN2 / 2), ka.b_g0 + g * ka.b_gmul);
+            }
+        }
+    }
     pdl_wait();
+    pdl_trigger();
 
     if (warp == 0) {
         if (lane == 0) {
@@ -395,15 +434,17 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             int m_blk, n_blk, g;
             for (int it = 0; ok && next_item_pair(ka, it, cluster_id, n_clusters, m_blk, n_blk, g); ++it) {
                 for (int kb = 0; kb < k_blocks; ++kb) {
-                    if (!(ok = mbar_wait(empty_bar + stage, phase ^ 1u, abort_flag))) break;
+                    const bool early = it == 0 && kb < pre;
+                    if (!early && !(ok = mbar_wait(empty_bar + stage, phase ^ 1u, abort_flag))) break;
                     uint8_t *sa = tiles + stage * Cfg::STAGE_BYTES;
                     uint8_t *sb = sa + Cfg::A_BYTES;
                     const uint32_t leader_full = map_to_cta(smem_u32(full_bar + stage), 0);
-                    if (rank == 0) mbar_expect_tx(full_bar + stage, 2 * Cfg::STAGE_BYTES);
+                    if (rank == 0 && !early) mbar_expect_tx(full_bar + stage, 2 * Cfg::STAGE_BYTES);
                     tma_load_3d_pair(sa, &tmA, leader_full, kb * BK, m_blk * 2 * BM + (int)rank * BM,
                                      ka.a_g0 + g * ka.a_gmul);
-                    tma_load_3d_pair(sb, &tmB, leader_full, kb * BK, n_blk * BN2 + (int)rank * (BN2 / 2),
-                                     ka.b_g0 + g * ka.b_gmul);
+                    if (!early)
+                        tma_load_3d_pair(sb, &tmB, leader_full, kb * BK, n_blk * BN2 + (int)rank * (BN2 / 2),
+                                         ka.b_g0 + g * ka.b_gmul);
                     if (++stage == Cfg::STAGES) {
                         stage = 0;
                         phase ^= 1u;
@@ -457,6 +498,8 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         constexpr int CHUNKS = BN2 / 32 / 2;
         float *stage = reinterpret_cast<float *>(smem + Cfg::STAGES * Cfg::STAGE_BYTES + 256) +
                        (warp - 2) * EPI_STAGE_FLOATS;
+        uint16_t *bias_strip = reinterpret_cast<uint16_t *>(smem + Cfg::STAGES * Cfg::STAGE_BYTES + 256 +
+                                                            Cfg::EPI_STAGE_BYTES) + (warp - 2) * 128;
         const bool staged = epilogue_f32_stageable(ka.epi);
         constexpr bool ln = LN;
         int acc = 0;
@@ -464,12 +507,16 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         bool ok = true;
         int m_blk, n_blk, g;
         for (int it = 0; ok && next_item_pair(ka, it, cluster_id, n_clusters, m_blk, n_blk, g); ++it) {
+            // the bias of this warp's 128 columns, fetched while the MMAs of the tile run
+            if (ka.epi.bias)
+                park_bias(ka.epi.bias + g * ka.epi.bias_gstride, n_blk * BN2 + half * (BN2 / 2) + 4 * lane, ka.shape.n_out,
+                          bias_strip, lane);
+            const int row_base = m_blk * 2 * BM + (int)rank * BM + quarter * 32;
+            const int row = row_base + lane;
             ok = mbar_wait(acc_full + acc, acc_phase, abort_flag);
             ok = __all_sync(0xFFFFFFFFu, ok);
             if (!ok) break;
             tc_fence_after_sync();
-            const int row_base = m_blk * 2 * BM + (int)rank * BM + quarter * 32;
-            const int row = row_base + lane;
             const uint32_t t_row = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) +
                                    static_cast<uint32_t>(acc * BN2);
             if (!ln) {
@@ -486,14 +533,15 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                         float v[32];
 #pragma unroll
                         for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
-                        if (ka.epi.bias) add_bias_chunk(ka.epi.bias + g * ka.epi.bias_gstride + col0, v, 32);
+                        if (ka.epi.bias) add_bias_chunk_parked(bias_strip + cc * 32, v);
                         epilogue_f32_staged(ka.epi, g, row_base, ka.shape.m, col0, v, stage, lane);
                     } else if (row < ka.shape.m) {
                         float v[32];
 #pragma unroll
                         for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]);
                         const int ncols = min(32, ka.shape.n_out - col0);
-                        epilogue_chunk(ka.epi, g, row, col0, ncols, v);
+                        if (ka.epi.bias) add_bias_chunk_parked(bias_strip + cc * 32, v);   // (zeros past n_out)
+                        epilogue_chunk(ka.epi, g, row, col0, ncols, v, false);
                     }
                 }
             }
@@ -725,6 +773,7 @@ int launch_gemm_tc(const GemmOperands &op, const GemmShape &s, const EpiParams &
         const int sms_ = sm_count() > 0 ? sm_count() : 148;
         if (ka.tiles_n > (bn == GEMM_TILE_PAIR ? sms_ / 2 : sms_)) return KRAKEN_EUNSUPPORTED;
     }
+    ka.w_early = op.w_static ? 1 : 0;
     ka.status = d_status;
     if (bn == GEMM_TILE_PAIR)
         return epi.ln_out ? launch_pair<true>(*tmA, *tmB, ka, stream) : launch_pair<false>(*tmA, *tmB, ka, stream);

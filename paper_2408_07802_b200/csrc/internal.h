@@ -94,6 +94,7 @@ struct GemmOperands {
     const void *w;
     long long w_gstride;
     int ldw;
+    bool w_static = false;   // W is not written by the kernel before this one in the stream (model weights)
 };
 int launch_gemm_tc(const GemmOperands &op, const GemmShape &shape, const EpiParams &epi, const CUtensorMap *tmA,
                    const CUtensorMap *tmB, int b_g0, int bn_hint, uint32_t *d_status, cudaStream_t stream);
