@@ -226,6 +226,7 @@ attn_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ 
     tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
     pdl_wait();   // launched ahead of the end of its predecessor: nothing of the predecessor's is touched before here
+    pdl_trigger();   // the successor's CTAs may take this one's place as soon as it leaves
 
     // Every role walks the same item sequence (blockIdx.x, + gridDim.x, ...) and keeps running
     // counters for the barrier phases, so the pipeline never drains between items.
