@@ -125,7 +125,7 @@ def test_layernorm_one_cta_per_row_walks_many_rows(force):
 
 # ------------------------------------------------------------------ grouped GEMM
 
-def gemm_case(G, M, Nout, K, epi, n_tile, seed=0, integer=False, shared_resid=False):
+def gemm_case(G, M, Nout, K, epi, n_tile, seed=0, integer=False, shared_resid=False, w_constant=0):
     if integer:
         a = (ki.hash32(seed, 60, 0, G * M * K, DEV) % 5 - 2).to(torch.bfloat16).reshape(G, M, K)
         w = (ki.hash32(seed, 61, 0, G * Nout * K, DEV) % 5 - 2).to(torch.bfloat16).reshape(G, Nout, K)
@@ -140,6 +140,7 @@ def gemm_case(G, M, Nout, K, epi, n_tile, seed=0, integer=False, shared_resid=Fa
     args.bias, args.bias_gstride = bias.data_ptr(), Nout
     args.groups, args.m, args.n_out, args.k = G, M, Nout, K
     args.epilogue, args.n_tile = epi, n_tile
+    args.w_constant = w_constant
     keep = [a, w, bias]
     out_f32 = out_bf16 = resid = ssum = None
     if epi in (kr.EPI_F32, kr.EPI_RESID_F32, kr.EPI_RESID_SUM):
@@ -180,6 +181,15 @@ def gemm_case(G, M, Nout, K, epi, n_tile, seed=0, integer=False, shared_resid=Fa
 def test_gemm_integer_exact_ragged(n_tile):
     """Small integers make every product and partial sum exact: any mis-placed element shows."""
     r = gemm_case(2, 300, 200, 136, kr.EPI_F32, n_tile, integer=True)
+    assert np.array_equal(r["out_f32"], r["ref"])
+
+
+@pytest.mark.parametrize("n_tile", [64, 256, 512])
+@pytest.mark.parametrize("K", [136, 1000])
+def test_gemm_constant_weights_fetched_before_the_predecessor_ends(n_tile, K):
+    """w_constant: the first stages' W tiles are requested before the kernel waits for the stream's previous kernel
+    (fewer k-blocks than stages, and more); several items per CTA, ragged edges; exact on small integers."""
+    r = gemm_case(3, 700, 1100, K, kr.EPI_F32, n_tile, integer=True, w_constant=1)
     assert np.array_equal(r["out_f32"], r["ref"])
 
 
