@@ -184,6 +184,15 @@ def test_gemm_integer_exact_ragged(n_tile):
     assert np.array_equal(r["out_f32"], r["ref"])
 
 
+@pytest.mark.parametrize("n_tile", [64, 160, 512])
+@pytest.mark.parametrize("Nout", [203, 330])
+def test_gemm_bias_rows_not_aligned(n_tile, Nout):
+    """An odd output width: the second group's bias row starts at an odd element, the last chunk of a tile is ragged
+    (the epilogue warps park their bias values in shared memory piecewise then)."""
+    r = gemm_case(2, 300, Nout, 136, kr.EPI_F32, n_tile, integer=True)
+    assert np.array_equal(r["out_f32"], r["ref"])
+
+
 @pytest.mark.parametrize("n_tile", [64, 256, 512])
 @pytest.mark.parametrize("K", [136, 1000])
 def test_gemm_constant_weights_fetched_before_the_predecessor_ends(n_tile, K):
